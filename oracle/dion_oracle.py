@@ -1,0 +1,165 @@
+"""ctypes front end of the float64 CPU oracle (``dion_oracle.c``).
+
+TEST INFRASTRUCTURE ONLY: imported by the tests, by the smoke check and by the
+benchmark's CPU-baseline leg.  The CUDA library never imports or links this.
+
+Every function takes and returns C-contiguous float64 numpy arrays.  State
+arrays are copied, so callers keep their inputs.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from typing import NamedTuple, Optional
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "dion_oracle.c")
+
+
+def _cpu_tag() -> str:
+    """Short hash of this host's CPU feature flags: the library is compiled with
+    -march=native, so a copy built on another machine must not be reused."""
+    import hashlib
+    flags = ""
+    try:
+        with open("/proc/cpuinfo") as f:
+            for line in f:
+                if line.startswith("flags"):
+                    flags = line
+                    break
+    except OSError:
+        pass
+    return hashlib.sha1(flags.encode()).hexdigest()[:10]
+
+
+_LIB = os.path.join(_HERE, f"libdion_oracle_{_cpu_tag()}.so")
+
+_i64 = ctypes.c_int64
+_dbl = ctypes.c_double
+_ptr = ctypes.c_void_p
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc (-O3 -fopenmp).  Returns the library path."""
+    if (not force and os.path.exists(_LIB)
+            and os.path.getmtime(_LIB) >= os.path.getmtime(_SRC)):
+        return _LIB
+    tmp = _LIB + f".tmp{os.getpid()}"
+    cmd = ["gcc", "-O3", "-march=native", "-fopenmp", "-fPIC", "-shared", "-std=c11",
+           "-fno-fast-math", "-o", tmp, _SRC, "-lm"]
+    subprocess.run(cmd, check=True, capture_output=True)
+    os.replace(tmp, _LIB)
+    return _LIB
+
+
+_lib = None
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        lib = ctypes.CDLL(build())
+        lib.dion_oracle_num_threads.restype = ctypes.c_int
+        lib.dion_oracle_householder_qr.restype = ctypes.c_int
+        lib.dion_oracle_householder_qr.argtypes = [_i64, _i64, _ptr, _ptr, _ptr]
+        lib.dion_oracle_colnorm.restype = None
+        lib.dion_oracle_colnorm.argtypes = [_i64, _i64, _ptr, _dbl, _ptr]
+        lib.dion_oracle_step.restype = ctypes.c_int
+        lib.dion_oracle_step.argtypes = [_i64, _i64, _i64, _ptr, _ptr, _ptr, _ptr,
+                                         _dbl, _dbl, _dbl, _ptr, _ptr, _ptr, _ptr]
+        lib.dion_oracle_sym_power_iter.restype = ctypes.c_int
+        lib.dion_oracle_sym_power_iter.argtypes = [_i64, _i64, _i64, _ptr, _ptr]
+        lib.dion_oracle_lazy_step.restype = ctypes.c_int
+        lib.dion_oracle_lazy_step.argtypes = [_i64, _i64, _i64, _ptr, _ptr, _ptr, _ptr,
+                                              _dbl, _dbl, _dbl, ctypes.c_int, _ptr]
+        _lib = lib
+    return _lib
+
+
+def num_threads() -> int:
+    return int(_load().dion_oracle_num_threads())
+
+
+def _f64(a) -> np.ndarray:
+    return np.ascontiguousarray(np.asarray(a, dtype=np.float64))
+
+
+def _p(a: Optional[np.ndarray]):
+    return None if a is None else a.ctypes.data_as(_ptr)
+
+
+class StepResult(NamedTuple):
+    X: np.ndarray      # m x n, updated parameter
+    M: np.ndarray      # m x n, updated momentum
+    Q: np.ndarray      # n x r, updated right factor (the paper's V_new)
+    d: np.ndarray      # r, column norms of W (singular value estimates)
+    P: np.ndarray      # m x r, B V before orthonormalization
+    U: np.ndarray      # m x r, orthonormal left factor
+    R: np.ndarray      # n x r, the paper's W = B^T U
+    degenerate: int    # number of degenerate Householder columns
+
+
+def householder_qr(P):
+    """Thin QR with diag(R) >= 0.  Returns (U, R_qr)."""
+    P = _f64(P)
+    m, r = P.shape
+    U = np.empty((m, r))
+    Rqr = np.empty((r, r))
+    rc = _load().dion_oracle_householder_qr(m, r, _p(P), _p(U), _p(Rqr))
+    if rc < 0:
+        raise MemoryError("oracle: out of host memory")
+    return U, Rqr
+
+
+def colnorm(W, eps: float):
+    W = _f64(W).copy()
+    n, r = W.shape
+    d = np.empty(r)
+    _load().dion_oracle_colnorm(n, r, _p(W), float(eps), _p(d))
+    return W, d
+
+
+def step(X, M, G, Q, mu: float, eta: float, eps: float = 1e-8) -> StepResult:
+    """One Dion step (Algorithm 1 + 2).  Inputs are not modified."""
+    X = _f64(X).copy(); M = _f64(M).copy(); G = _f64(G); Q = _f64(Q).copy()
+    m, n = X.shape
+    r = Q.shape[1]
+    assert M.shape == (m, n) and G.shape == (m, n) and Q.shape == (n, r)
+    assert 1 <= r <= min(m, n)
+    d = np.empty(r); P = np.empty((m, r)); U = np.empty((m, r)); R = np.empty((n, r))
+    rc = _load().dion_oracle_step(m, n, r, _p(X), _p(M), _p(G), _p(Q), float(mu), float(eta),
+                                  float(eps), _p(d), _p(P), _p(U), _p(R))
+    if rc < 0:
+        raise MemoryError("oracle: out of host memory")
+    return StepResult(X, M, Q, d, P, U, R, rc)
+
+
+def sym_power_iter(M, Q):
+    """SymPowerIter1 (Algorithm 6): Orthonormalize(M^T M V)."""
+    M = _f64(M); Q = _f64(Q).copy()
+    m, n = M.shape
+    r = Q.shape[1]
+    rc = _load().dion_oracle_sym_power_iter(m, n, r, _p(M), _p(Q))
+    if rc < 0:
+        raise MemoryError("oracle: out of host memory")
+    return Q
+
+
+def lazy_step(X, M, G, Q, mu: float, eta: float, eps: float = 1e-8, refresh: bool = False):
+    """One Lazy-Dion step (Algorithm 6).  Returns (X, M, Q, d)."""
+    X = _f64(X).copy(); M = _f64(M).copy(); G = _f64(G); Q = _f64(Q).copy()
+    m, n = X.shape
+    r = Q.shape[1]
+    d = np.empty(r)
+    rc = _load().dion_oracle_lazy_step(m, n, r, _p(X), _p(M), _p(G), _p(Q), float(mu), float(eta),
+                                       float(eps), int(bool(refresh)), _p(d))
+    if rc < 0:
+        raise MemoryError("oracle: out of host memory")
+    return X, M, Q, d
+
+
+if __name__ == "__main__":
+    print(build(force=True))
