@@ -1,0 +1,165 @@
+/*
+ * dion.h -- C-ABI of the B200-native (sm_100a) single-device Dion update step.
+ *
+ * The library implements the unsharded Dion rule of "Dion: Distributed
+ * Orthonormalized Updates" (Algorithm 1 line 3 + Algorithm 2) for one
+ * matrix-valued parameter X (m x n, m = rows = "out" dimension |I|, n = columns
+ * = "in" dimension |J|) with gradient G, momentum M and warm-start right factor
+ * Q (the paper's V, n x r):
+ *
+ *     B  = M + G                               Alg. 2, line 1
+ *     P  = B Q                                 PowerIter1, line 1
+ *     U  = Orthonormalize(P)                   PowerIter1, line 3; Section 3.2
+ *     R  = B^T U                               PowerIter1, line 4  (the paper's W)
+ *     M <- B - (1 - mu) U R^T                  Alg. 2, line 3; Eq. 1 (error feedback)
+ *     Q <- ColNorm(R)                          Alg. 2, line 4
+ *     X <- X - lr * sqrt(m/n) * U Q^T          Alg. 2, lines 5-6; Alg. 1, line 3
+ *
+ * Orthonormalize returns the thin-QR orthonormal factor whose triangular factor
+ * has a positive diagonal.  ColNorm divides column j by (||column j||_2 + eps).
+ *
+ * General conventions
+ *   - Every matrix pointer is a DEVICE pointer owned by the caller; matrices are
+ *     dense row-major with a leading dimension given in ELEMENTS.
+ *   - X, M, Q are updated in place; G is never written.  No two arrays of one
+ *     matrix may overlap.
+ *   - All step calls are asynchronous on the CUDA stream passed in (a
+ *     cudaStream_t cast to void*; NULL = the legacy default stream) and never
+ *     synchronise.  Device-side problems (Cholesky breakdown, non-finite pivot)
+ *     are latched in a status word read by dion_get_status.
+ *   - The context owns only scratch memory (P/U, R, Gram and triangular factors,
+ *     column norms, flags).  It grows on demand with cudaMalloc, which
+ *     synchronises; after the first call with the largest shapes, or when
+ *     dion_config.workspace_bytes was large enough, no call allocates.
+ *   - Every function returns DION_OK (0) or a negative DION_ERR_* code; nothing
+ *     is printed, thrown or aborted.
+ *   - There is no CPU fallback: on a machine without a usable sm_100 device
+ *     dion_init fails with DION_ERR_CUDA.
+ */
+#ifndef DION_H_
+#define DION_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct dion_ctx dion_ctx; /* opaque; owns scratch memory only */
+
+typedef enum { DION_F32 = 0, DION_BF16 = 1 } dion_dtype;
+
+/* Arithmetic of the four large contractions (P, R, U R^T, U Q^T).
+ * DION_PREC_FP32:           products carry fp32 accuracy (fp32 FMA, or a 3-term
+ *                           TF32 split on the tensor cores), fp32 accumulation.
+ * DION_PREC_BF16_OPERANDS:  operands rounded to bf16, fp32 accumulation.       */
+typedef enum { DION_PREC_FP32 = 0, DION_PREC_BF16_OPERANDS = 1 } dion_precision;
+
+/* Orthonormalize (Section 3.2 and the appendix on Cholesky QR).
+ * DION_ORTH_AUTO:        CholeskyQR2 when 4 r <= min(m, n), else shifted CholeskyQR3.
+ * DION_ORTH_CHOLQR2:     two rounds of Cholesky QR.
+ * DION_ORTH_SHIFTED3:    a shifted Cholesky QR round followed by CholeskyQR2
+ *                        (for ill-conditioned panels, e.g. full rank).
+ * DION_ORTH_HOUSEHOLDER: Householder QR (slow, most robust).                   */
+typedef enum {
+  DION_ORTH_AUTO = 0,
+  DION_ORTH_CHOLQR2 = 1,
+  DION_ORTH_SHIFTED3 = 2,
+  DION_ORTH_HOUSEHOLDER = 3
+} dion_orth;
+
+/* Which kernels carry the contractions.
+ * DION_ENGINE_AUTO:   tensor cores (tcgen05) where the shape allows, else SIMT.
+ * DION_ENGINE_SIMT:   fp32 FMA kernels only (any shape).
+ * DION_ENGINE_TENSOR: tensor cores; shapes they cannot take are an error.      */
+typedef enum { DION_ENGINE_AUTO = 0, DION_ENGINE_SIMT = 1, DION_ENGINE_TENSOR = 2 } dion_engine;
+
+enum {
+  DION_OK = 0,
+  DION_ERR_INVALID = -1,    /* NULL pointer, bad enum, count < 0, ...              */
+  DION_ERR_SHAPE = -2,      /* m, n < 1, r outside [1, min(m, n)], ld too small   */
+  DION_ERR_ALIGN = -3,      /* a pointer is not aligned to its element size x 4   */
+  DION_ERR_ALIAS = -4,      /* two arrays of one matrix overlap                   */
+  DION_ERR_NOMEM = -5,      /* scratch allocation failed                          */
+  DION_ERR_CUDA = -6,       /* a CUDA runtime call failed, or no sm_100 device    */
+  DION_ERR_UNSUPPORTED = -7 /* the requested engine cannot take this shape        */
+};
+
+/* Bits of the device status word (dion_get_status). */
+enum {
+  DION_STATUS_BREAKDOWN = 1,  /* a Cholesky pivot was <= 0 or not finite: the step
+                                 that saw it left X, M and Q unchanged            */
+  DION_STATUS_NONFINITE = 2,  /* a column norm of R was not finite                 */
+  DION_STATUS_TIMEOUT = 4     /* a bounded device-side wait ran out                */
+};
+
+typedef struct {
+  float mu;               /* momentum / error-feedback coefficient, beta = 1 - mu (paper: beta = 0.05) */
+  float eps;              /* ColNorm epsilon (1e-8)                                                    */
+  int precision;          /* dion_precision                                                            */
+  int orth;               /* dion_orth                                                                 */
+  int engine;             /* dion_engine                                                               */
+  int device;             /* CUDA device ordinal                                                       */
+  size_t workspace_bytes; /* scratch to reserve at init; 0 = grow on demand                            */
+} dion_config;
+
+/* One matrix parameter and its optimizer state (Algorithm 1: "states M, V"). */
+typedef struct {
+  int64_t m, n, r;      /* 1 <= r <= min(m, n)                                       */
+  void* X;              /* fp32, m x n, in/out                                       */
+  int64_t ldx;
+  void* M;              /* fp32, m x n, in/out (momentum / error-feedback buffer)    */
+  int64_t ldm;
+  const void* G;        /* g_dtype, m x n, read only                                 */
+  int64_t ldg;
+  int g_dtype;          /* dion_dtype                                                */
+  void* Q;              /* fp32, n x r, in/out (right factor; any full-column-rank start) */
+  int64_t ldq;
+  float* colnorm_out;   /* optional: r floats, the column norms of R (estimates of the
+                           leading singular values of B); may be NULL                */
+} dion_matrix;
+
+/* Fill *cfg with the defaults: mu 0.95, eps 1e-8, fp32, AUTO, AUTO, device 0, no reserve. */
+void dion_default_config(dion_config* cfg);
+
+/* Create a context on cfg->device.  Host pointers.  *out is NULL on failure. */
+int dion_init(dion_ctx** out, const dion_config* cfg);
+
+/* One Dion step on one matrix (Algorithm 1 + 2).  `a` is a HOST pointer to a
+ * descriptor holding DEVICE pointers.  lr is the paper's eta; sqrt(m/n) is
+ * applied inside.  If the orthonormalization breaks down, X, M and Q are left
+ * unchanged and DION_STATUS_BREAKDOWN is latched. */
+int dion_step(dion_ctx* ctx, const dion_matrix* a, float lr, void* cuda_stream);
+
+/* The same step on `count` independent matrices (the paper batches matrices of
+ * identical shape; Section 4.1).  Equivalent to `count` dion_step calls in any
+ * order.  `list` is a HOST array.  count == 0 is a no-op. */
+int dion_step_grouped(dion_ctx* ctx, const dion_matrix* list, int count, float lr, void* cuda_stream);
+
+/* One Lazy-Dion step (Algorithm 6): M <- M + G; if refresh != 0, Q <-
+ * Orthonormalize(M^T M Q) (SymPowerIter1); W = M Q; M <- M - (1-mu) W Q^T;
+ * X <- X - lr sqrt(m/n) ColNorm(W) Q^T.  colnorm_out receives the norms of W. */
+int dion_lazy_step(dion_ctx* ctx, const dion_matrix* a, float lr, int refresh, void* cuda_stream);
+
+/* Scratch bytes a step on (m, n, r) needs; 0 if the shape is invalid. */
+size_t dion_workspace_bytes(const dion_ctx* ctx, int64_t m, int64_t n, int64_t r);
+
+/* Synchronises `cuda_stream`, then reports and clears the latched device status
+ * (DION_STATUS_* bits) and the number of steps skipped because of a breakdown
+ * since the last call.  Either output pointer may be NULL. */
+int dion_get_status(dion_ctx* ctx, void* cuda_stream, int* device_status, int* steps_skipped);
+
+/* Number of kernel launches issued by this context so far (host counter). */
+int64_t dion_launch_count(const dion_ctx* ctx);
+
+/* Frees the scratch memory and the context.  NULL is allowed. */
+void dion_destroy(dion_ctx* ctx);
+
+/* Static string for a DION_ERR_* code. */
+const char* dion_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DION_H_ */

@@ -1,0 +1,211 @@
+"""Thin ctypes binding of ``libdion_b200.so`` (the C-ABI declared in ``include/dion.h``).
+
+Argument marshalling only: every arithmetic step runs in the CUDA kernels.
+PyTorch supplies device memory and streams.  There is no CPU or eager-PyTorch
+fallback: if the shared library is missing or no sm_100 device is present the
+calls raise.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Iterable, List, Optional, Sequence, Tuple
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libdion_b200.so")
+
+DION_F32, DION_BF16 = 0, 1
+PREC_FP32, PREC_BF16_OPERANDS = 0, 1
+ORTH_AUTO, ORTH_CHOLQR2, ORTH_SHIFTED3, ORTH_HOUSEHOLDER = 0, 1, 2, 3
+ENGINE_AUTO, ENGINE_SIMT, ENGINE_TENSOR = 0, 1, 2
+STATUS_BREAKDOWN, STATUS_NONFINITE, STATUS_TIMEOUT = 1, 2, 4
+
+EXPORTS = ["dion_default_config", "dion_init", "dion_step", "dion_step_grouped", "dion_lazy_step",
+           "dion_workspace_bytes", "dion_get_status", "dion_launch_count", "dion_destroy",
+           "dion_strerror"]
+
+
+class DionConfig(ctypes.Structure):
+    _fields_ = [("mu", ctypes.c_float), ("eps", ctypes.c_float), ("precision", ctypes.c_int),
+                ("orth", ctypes.c_int), ("engine", ctypes.c_int), ("device", ctypes.c_int),
+                ("workspace_bytes", ctypes.c_size_t)]
+
+
+class DionMatrix(ctypes.Structure):
+    _fields_ = [("m", ctypes.c_int64), ("n", ctypes.c_int64), ("r", ctypes.c_int64),
+                ("X", ctypes.c_void_p), ("ldx", ctypes.c_int64),
+                ("M", ctypes.c_void_p), ("ldm", ctypes.c_int64),
+                ("G", ctypes.c_void_p), ("ldg", ctypes.c_int64), ("g_dtype", ctypes.c_int),
+                ("Q", ctypes.c_void_p), ("ldq", ctypes.c_int64),
+                ("colnorm_out", ctypes.c_void_p)]
+
+
+class DionError(RuntimeError):
+    def __init__(self, code: int, msg: str):
+        super().__init__(f"dion error {code}: {msg}")
+        self.code = code
+
+
+_lib = None
+
+
+def load_library() -> ctypes.CDLL:
+    """Loads the CUDA library; raises if it has not been built."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(f"{LIB_PATH} is missing: run `python -m paper_2504_05295_b200.build` "
+                          "(there is no fallback path)")
+    lib = ctypes.CDLL(LIB_PATH)
+    vp, i64, f32, ci = ctypes.c_void_p, ctypes.c_int64, ctypes.c_float, ctypes.c_int
+    lib.dion_default_config.argtypes = [ctypes.POINTER(DionConfig)]
+    lib.dion_default_config.restype = None
+    lib.dion_init.argtypes = [ctypes.POINTER(vp), ctypes.POINTER(DionConfig)]
+    lib.dion_init.restype = ci
+    lib.dion_step.argtypes = [vp, ctypes.POINTER(DionMatrix), f32, vp]
+    lib.dion_step.restype = ci
+    lib.dion_step_grouped.argtypes = [vp, ctypes.POINTER(DionMatrix), ci, f32, vp]
+    lib.dion_step_grouped.restype = ci
+    lib.dion_lazy_step.argtypes = [vp, ctypes.POINTER(DionMatrix), f32, ci, vp]
+    lib.dion_lazy_step.restype = ci
+    lib.dion_workspace_bytes.argtypes = [vp, i64, i64, i64]
+    lib.dion_workspace_bytes.restype = ctypes.c_size_t
+    lib.dion_get_status.argtypes = [vp, vp, ctypes.POINTER(ci), ctypes.POINTER(ci)]
+    lib.dion_get_status.restype = ci
+    lib.dion_launch_count.argtypes = [vp]
+    lib.dion_launch_count.restype = i64
+    lib.dion_destroy.argtypes = [vp]
+    lib.dion_destroy.restype = None
+    lib.dion_strerror.argtypes = [ci]
+    lib.dion_strerror.restype = ctypes.c_char_p
+    _lib = lib
+    return lib
+
+
+def strerror(code: int) -> str:
+    return load_library().dion_strerror(int(code)).decode()
+
+
+def _check(code: int) -> None:
+    if code != 0:
+        raise DionError(code, strerror(code))
+
+
+def _stream_ptr(stream: Optional[torch.cuda.Stream]) -> int:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return int(stream.cuda_stream)
+
+
+def matrix_desc(X: torch.Tensor, M: torch.Tensor, G: torch.Tensor, Q: torch.Tensor,
+                colnorm_out: Optional[torch.Tensor] = None) -> DionMatrix:
+    """Describes one parameter for the C-ABI.  Tensors must be CUDA, 2-D, row-major
+    (unit stride along the last dimension); a row stride larger than the width is
+    passed on as the leading dimension."""
+    for name, t in (("X", X), ("M", M), ("G", G), ("Q", Q)):
+        if not t.is_cuda or t.dim() != 2 or t.stride(1) != 1:
+            raise ValueError(f"{name} must be a 2-D CUDA tensor with unit column stride")
+    if X.dtype != torch.float32 or M.dtype != torch.float32 or Q.dtype != torch.float32:
+        raise ValueError("X, M and Q must be float32")
+    if G.dtype == torch.float32:
+        gd = DION_F32
+    elif G.dtype == torch.bfloat16:
+        gd = DION_BF16
+    else:
+        raise ValueError("G must be float32 or bfloat16")
+    m, n = X.shape
+    if tuple(M.shape) != (m, n) or tuple(G.shape) != (m, n) or Q.shape[0] != n:
+        raise ValueError("shape mismatch between X, M, G and Q")
+    d = DionMatrix()
+    d.m, d.n, d.r = m, n, Q.shape[1]
+    d.X, d.ldx = X.data_ptr(), X.stride(0)
+    d.M, d.ldm = M.data_ptr(), M.stride(0)
+    d.G, d.ldg, d.g_dtype = G.data_ptr(), G.stride(0), gd
+    d.Q, d.ldq = Q.data_ptr(), Q.stride(0)
+    if colnorm_out is not None:
+        if (not colnorm_out.is_cuda or colnorm_out.dtype != torch.float32
+                or colnorm_out.numel() < Q.shape[1] or not colnorm_out.is_contiguous()):
+            raise ValueError("colnorm_out must be a contiguous float32 CUDA tensor of >= r elements")
+        d.colnorm_out = colnorm_out.data_ptr()
+    else:
+        d.colnorm_out = None
+    return d
+
+
+class Dion:
+    """A library context (``dion_init`` .. ``dion_destroy``)."""
+
+    def __init__(self, mu: float = 0.95, eps: float = 1e-8, precision: int = PREC_FP32,
+                 orth: int = ORTH_AUTO, engine: int = ENGINE_AUTO, device: Optional[int] = None,
+                 workspace_bytes: int = 0):
+        lib = load_library()
+        if device is None:
+            device = torch.cuda.current_device()
+        cfg = DionConfig()
+        lib.dion_default_config(ctypes.byref(cfg))
+        cfg.mu, cfg.eps = mu, eps
+        cfg.precision, cfg.orth, cfg.engine = precision, orth, engine
+        cfg.device, cfg.workspace_bytes = int(device), int(workspace_bytes)
+        self._lib = lib
+        self._ctx = ctypes.c_void_p()
+        _check(lib.dion_init(ctypes.byref(self._ctx), ctypes.byref(cfg)))
+        self.device = int(device)
+
+    def step(self, X, M, G, Q, lr: float, colnorm_out=None, stream=None) -> None:
+        d = matrix_desc(X, M, G, Q, colnorm_out)
+        _check(self._lib.dion_step(self._ctx, ctypes.byref(d), float(lr), _stream_ptr(stream)))
+
+    def step_desc(self, desc: DionMatrix, lr: float, stream_ptr: int) -> None:
+        """dion_step on a prebuilt descriptor (no per-call marshalling)."""
+        _check(self._lib.dion_step(self._ctx, ctypes.byref(desc), float(lr), stream_ptr))
+
+    @staticmethod
+    def pack(descs: Sequence[DionMatrix]):
+        arr = (DionMatrix * len(descs))(*descs)
+        return arr
+
+    def step_grouped(self, mats: Iterable[Tuple], lr: float, stream=None) -> None:
+        """mats: iterable of (X, M, G, Q) or (X, M, G, Q, colnorm_out)."""
+        descs: List[DionMatrix] = [matrix_desc(*t) for t in mats]
+        arr = self.pack(descs)
+        _check(self._lib.dion_step_grouped(self._ctx, arr, len(descs), float(lr), _stream_ptr(stream)))
+
+    def step_grouped_packed(self, arr, count: int, lr: float, stream_ptr: int) -> None:
+        _check(self._lib.dion_step_grouped(self._ctx, arr, int(count), float(lr), stream_ptr))
+
+    def lazy_step(self, X, M, G, Q, lr: float, refresh: bool, colnorm_out=None, stream=None) -> None:
+        d = matrix_desc(X, M, G, Q, colnorm_out)
+        _check(self._lib.dion_lazy_step(self._ctx, ctypes.byref(d), float(lr), int(bool(refresh)),
+                                        _stream_ptr(stream)))
+
+    def workspace_bytes(self, m: int, n: int, r: int) -> int:
+        return int(self._lib.dion_workspace_bytes(self._ctx, m, n, r))
+
+    def get_status(self, stream=None) -> Tuple[int, int]:
+        """Synchronises the stream; returns (status bits, steps skipped) and clears both."""
+        st, sk = ctypes.c_int(0), ctypes.c_int(0)
+        _check(self._lib.dion_get_status(self._ctx, _stream_ptr(stream), ctypes.byref(st), ctypes.byref(sk)))
+        return st.value, sk.value
+
+    def launch_count(self) -> int:
+        return int(self._lib.dion_launch_count(self._ctx))
+
+    def close(self) -> None:
+        if self._ctx:
+            self._lib.dion_destroy(self._ctx)
+            self._ctx = ctypes.c_void_p()
+
+    def __enter__(self):
+        return self
+
+    def __exit__(self, *exc):
+        self.close()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

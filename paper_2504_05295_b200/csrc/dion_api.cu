@@ -1,0 +1,629 @@
+// C-ABI of the Dion step library: context, argument checks, scratch layout and
+// the launch sequence of one step.  All arithmetic runs in the kernels of this
+// directory; the host code only validates and launches.
+#include <math.h>
+#include <new>
+#include <string.h>
+
+#include "dion_common.cuh"
+#include "orth_kernels.cuh"
+#include "simt_gemm.cuh"
+#include "umma_gemm.cuh"
+
+using namespace dion;
+
+namespace {
+
+constexpr int MAX_FLAG_SLOTS = 4096;
+constexpr i64 PART_CAP_FLOATS = (i64)16 << 20;  // split-K partial sums, at most 64 MiB
+
+inline i64 align64(i64 floats) { return (floats + 63) / 64 * 64; }  // 256-byte granules
+
+struct Layout {
+  i64 P0, P1, R, Gram, Linv, Tbuf, Dinv, part, cn_part, d, scal, total;
+  i64 part_floats;
+  int cn_chunks;
+  i64 cn_rows;
+};
+
+}  // namespace
+
+struct dion_ctx {
+  dion_config cfg;
+  int sm_count;
+  float* ws;
+  size_t ws_bytes;
+  int* dev_ints;  // [0] status, [1] skipped, [2..] per-step flags
+  int flag_cursor;
+  int64_t launches;
+};
+
+namespace {
+
+void colnorm_plan(i64 rows, i64 r, int sm, int* chunks, i64* rows_per) {
+  const i64 col_blocks = (r + 127) / 128;
+  i64 want = (4 * (i64)sm + col_blocks - 1) / col_blocks;
+  if (want < 1) want = 1;
+  i64 per = (rows + want - 1) / want;
+  if (per < 32) per = 32;
+  *rows_per = per;
+  *chunks = (int)((rows + per - 1) / per);
+}
+
+Layout make_layout(const dion_ctx* c, i64 m, i64 n, i64 r) {
+  Layout L;
+  const i64 big = (m > n) ? m : n;
+  i64 o = 0;
+  L.P0 = o; o += align64(big * r);
+  L.P1 = o; o += align64(big * r);
+  L.R = o; o += align64(big * r);
+  L.Gram = o; o += align64(r * r);
+  L.Linv = o; o += align64(r * r);
+  L.Tbuf = o; o += align64(r * r);
+  L.Dinv = o; o += align64(((r + NB - 1) / NB) * (i64)NB * NB);
+  // split-K partials: the largest plain-store product of a step is max(m,n) x r
+  i64 pf = 4 * (i64)c->sm_count * 64 * 64;
+  if (pf > PART_CAP_FLOATS) pf = PART_CAP_FLOATS;
+  L.part_floats = pf;
+  L.part = o; o += align64(pf);
+  colnorm_plan(big, r, c->sm_count, &L.cn_chunks, &L.cn_rows);
+  L.cn_part = o; o += align64((i64)(L.cn_chunks + 1) * r);
+  L.d = o; o += align64(r);
+  L.scal = o; o += 64;
+  L.total = o;
+  return L;
+}
+
+int ensure_ws(dion_ctx* c, size_t bytes) {
+  if (bytes <= c->ws_bytes) return DION_OK;
+  if (c->ws != nullptr) {
+    if (cudaDeviceSynchronize() != cudaSuccess) return DION_ERR_CUDA;
+    cudaFree(c->ws);
+    c->ws = nullptr;
+    c->ws_bytes = 0;
+  }
+  void* p = nullptr;
+  if (cudaMalloc(&p, bytes) != cudaSuccess) { cudaGetLastError(); return DION_ERR_NOMEM; }
+  c->ws = (float*)p;
+  c->ws_bytes = bytes;
+  return DION_OK;
+}
+
+#define DION_CHECK_LAUNCH(ctx)                                   \
+  do {                                                           \
+    (ctx)->launches++;                                           \
+    if (cudaGetLastError() != cudaSuccess) return DION_ERR_CUDA; \
+  } while (0)
+#define DION_TRY(expr)              \
+  do {                              \
+    const int rc_ = (expr);         \
+    if (rc_ != DION_OK) return rc_; \
+  } while (0)
+
+GemmArgs gemm_args() {
+  GemmArgs g;
+  memset(&g, 0, sizeof(g));
+  g.alpha = 1.f;
+  g.batch = 1;
+  g.splits = 1;
+  return g;
+}
+
+// Launches one product on the fp32 FMA engine.
+int launch_gemm_simt(dion_ctx* c, GemmArgs g, cudaStream_t st, float* part, i64 part_floats,
+                     bool force64) {
+  if (g.M <= 0 || g.N <= 0) return DION_OK;
+  const i64 t128 = ((g.M + 127) / 128) * ((g.N + 127) / 128) * g.batch;
+  const bool use128 = !force64 && t128 >= c->sm_count;
+  const int BMN = use128 ? 128 : 64;
+  const i64 gm = (g.M + BMN - 1) / BMN, gn = (g.N + BMN - 1) / BMN;
+  int splits = 1;
+  if (!use128 && !force64 && g.epi == EPI_STORE && g.batch == 1 && part != nullptr && g.alpha_dev == nullptr) {
+    const i64 tiles = gm * gn;
+    i64 want = (2 * (i64)c->sm_count + tiles - 1) / tiles;
+    const i64 kmax = g.K / 128;
+    if (want > kmax) want = kmax;
+    if (want > 64) want = 64;
+    while (want > 1 && want * g.M * g.N > part_floats) --want;
+    if (want > 1) splits = (int)want;
+  }
+  g.splits = splits;
+  g.part = part;
+  if (gm > 65535) return DION_ERR_UNSUPPORTED;
+  dim3 grid((unsigned)gn, (unsigned)gm, (unsigned)(splits > 1 ? splits : g.batch));
+  if (use128) k_gemm_simt<128, 128, 8, 8, 8><<<grid, 256, 0, st>>>(g);
+  else k_gemm_simt<64, 64, 16, 4, 4><<<grid, 256, 0, st>>>(g);
+  DION_CHECK_LAUNCH(c);
+  if (splits > 1) {
+    const i64 total = g.M * g.N;
+    int blocks = (int)((total + 255) / 256);
+    if (blocks > 8 * c->sm_count) blocks = 8 * c->sm_count;
+    k_splitk_reduce<<<blocks, 256, 0, st>>>(part, splits, g.M, g.N, g.C, g.ldc, g.alpha, g.tri, BMN, g.skip_flag);
+    DION_CHECK_LAUNCH(c);
+  }
+  return DION_OK;
+}
+
+struct StepCtx {
+  dion_ctx* c;
+  cudaStream_t st;
+  float* ws;
+  Layout L;
+  int* flag;
+  bool tensor;  // tensor-core engine allowed for this matrix
+};
+
+// Engine dispatch: tensor cores when the product qualifies, else fp32 FMA.
+int launch_gemm(StepCtx& s, const GemmArgs& g, bool force64 = false) {
+  if (s.tensor && !force64) {
+    const int rc = umma_try_launch(g, s.c->cfg.precision, s.c->sm_count, s.st);
+    if (rc == 1) { s.c->launches++; return cudaGetLastError() == cudaSuccess ? DION_OK : DION_ERR_CUDA; }
+    if (rc < 0) return rc;
+  }
+  return launch_gemm_simt(s.c, g, s.st, s.ws + s.L.part, s.L.part_floats, force64);
+}
+
+// Blocked right-looking Cholesky of the r x r matrix Gm (lower), diagonal-block
+// inverses into Dinv, then the full inverse of the factor into Linv.
+int potrf_trtri(StepCtx& s, float* Gm, i64 r, const float* shift) {
+  dion_ctx* c = s.c;
+  float* Dinv = s.ws + s.L.Dinv;
+  float* Linv = s.ws + s.L.Linv;
+  float* Tbuf = s.ws + s.L.Tbuf;
+  int* status = c->dev_ints;
+  for (i64 j0 = 0; j0 < r; j0 += NB) {
+    const int jb = (int)((r - j0 < NB) ? (r - j0) : NB);
+    float* Ajj = Gm + j0 * r + j0;
+    float* Dj = Dinv + (j0 / NB) * (NB * NB);
+    k_potrf_diag<<<1, 256, 0, s.st>>>(Ajj, r, jb, Dj, shift, s.flag, status);
+    DION_CHECK_LAUNCH(c);
+    const i64 rem = r - j0 - jb;
+    if (rem > 0) {
+      float* panel = Gm + (j0 + jb) * r + j0;
+      GemmArgs g = gemm_args();  // panel <- panel * Linv_jj^T, in place
+      g.M = rem; g.N = jb; g.K = jb;
+      g.A = panel; g.a_si = r; g.a_sk = 1;
+      g.B = Dj; g.b_sk = 1; g.b_sn = NB;
+      g.C = panel; g.ldc = r; g.epi = EPI_STORE;
+      DION_TRY(launch_gemm_simt(c, g, s.st, nullptr, 0, true));
+      GemmArgs t = gemm_args();  // A22 -= panel * panel^T (lower tiles)
+      t.M = rem; t.N = rem; t.K = jb;
+      t.A = panel; t.a_si = r; t.a_sk = 1;
+      t.B = panel; t.b_sk = 1; t.b_sn = r;
+      t.C = Gm + (j0 + jb) * r + (j0 + jb); t.ldc = r; t.epi = EPI_SUB; t.tri = TRI_LOWER;
+      DION_TRY(launch_gemm_simt(c, t, s.st, nullptr, 0, false));
+    }
+  }
+  {
+    const i64 total = r * r;
+    int blocks = (int)((total + 255) / 256);
+    if (blocks > 8 * c->sm_count) blocks = 8 * c->sm_count;
+    k_linv_init<<<blocks, 256, 0, s.st>>>(Linv, r, r, Dinv);
+    DION_CHECK_LAUNCH(c);
+  }
+  // inverse by doubling: [[L11,0],[L21,L22]]^-1 = [[X11,0],[-X22 L21 X11, X22]]
+  for (i64 b = NB; b < r; b *= 2) {
+    const i64 nfull = r / (2 * b);
+    const i64 tail0 = nfull * 2 * b;
+    const i64 b2_tail = (r - tail0 > b) ? (r - tail0 - b) : 0;
+    for (int pass = 0; pass < 2; ++pass) {
+      const i64 base = (pass == 0) ? 0 : tail0;
+      const i64 rows = (pass == 0) ? b : b2_tail;
+      const int batch = (pass == 0) ? (int)nfull : 1;
+      if (rows <= 0 || batch <= 0) continue;
+      const i64 off21 = (base + b) * r + base, off11 = base * r + base, off22 = (base + b) * r + (base + b);
+      const i64 bs = 2 * b * (r + 1);
+      GemmArgs g1 = gemm_args();  // T = L21 * X11
+      g1.M = rows; g1.N = b; g1.K = b;
+      g1.A = Gm + off21; g1.a_si = r; g1.a_sk = 1;
+      g1.B = Linv + off11; g1.b_sk = r; g1.b_sn = 1;
+      g1.C = Tbuf + off21; g1.ldc = r; g1.epi = EPI_STORE;
+      g1.batch = batch; g1.bsA = bs; g1.bsB = bs; g1.bsC = bs;
+      DION_TRY(launch_gemm_simt(c, g1, s.st, nullptr, 0, false));
+      GemmArgs g2 = gemm_args();  // X21 = -X22 * T
+      g2.M = rows; g2.N = b; g2.K = rows;
+      g2.A = Linv + off22; g2.a_si = r; g2.a_sk = 1;
+      g2.B = Tbuf + off21; g2.b_sk = r; g2.b_sn = 1;
+      g2.C = Linv + off21; g2.ldc = r; g2.epi = EPI_STORE; g2.alpha = -1.f;
+      g2.batch = batch; g2.bsA = bs; g2.bsB = bs; g2.bsC = bs;
+      DION_TRY(launch_gemm_simt(c, g2, s.st, nullptr, 0, false));
+    }
+  }
+  return DION_OK;
+}
+
+// One Cholesky-QR round: Pout = Pin * chol(Pin^T Pin + shift I)^-T.  rows x r panels, ld = r.
+int cholqr_round(StepCtx& s, const float* Pin, float* Pout, i64 rows, i64 r, float shift_scale) {
+  dion_ctx* c = s.c;
+  float* Gm = s.ws + s.L.Gram;
+  GemmArgs g = gemm_args();
+  g.M = r; g.N = r; g.K = rows;
+  g.A = Pin; g.a_si = 1; g.a_sk = r;
+  g.B = Pin; g.b_sk = r; g.b_sn = 1;
+  g.C = Gm; g.ldc = r; g.epi = EPI_STORE; g.tri = TRI_LOWER;
+  DION_TRY(launch_gemm(s, g));
+  const float* shift = nullptr;
+  if (shift_scale > 0.f) {
+    float* sh = s.ws + s.L.scal;
+    k_trace_scaled<<<1, 256, 0, s.st>>>(Gm, r, r, shift_scale, sh);
+    DION_CHECK_LAUNCH(c);
+    shift = sh;
+  }
+  DION_TRY(potrf_trtri(s, Gm, r, shift));
+  GemmArgs u = gemm_args();
+  u.M = rows; u.N = r; u.K = r;
+  u.A = Pin; u.a_si = r; u.a_sk = 1;
+  u.B = s.ws + s.L.Linv; u.b_sk = 1; u.b_sn = r; u.klimit = 1;
+  u.C = Pout; u.ldc = r; u.epi = EPI_STORE;
+  DION_TRY(launch_gemm(s, u));
+  return DION_OK;
+}
+
+int householder(StepCtx& s, float* A, float* V, i64 rows, i64 r) {
+  dion_ctx* c = s.c;
+  float* diag = s.ws + s.L.d;
+  for (i64 j = 0; j < r; ++j) {
+    k_hh_reflector<<<1, 1024, 0, s.st>>>(A, r, rows, j, V, r, diag);
+    DION_CHECK_LAUNCH(c);
+    if (j + 1 < r) {
+      const unsigned gx = (unsigned)((r - j - 1 + 31) / 32);
+      k_hh_apply<<<gx, 256, 0, s.st>>>(A, r, rows, j, V, r, j, j + 1, r);
+      DION_CHECK_LAUNCH(c);
+    }
+  }
+  {
+    const i64 total = rows * r;
+    int blocks = (int)((total + 255) / 256);
+    if (blocks > 8 * c->sm_count) blocks = 8 * c->sm_count;
+    k_set_identity<<<blocks, 256, 0, s.st>>>(A, r, rows, r);
+    DION_CHECK_LAUNCH(c);
+    for (i64 j = r - 1; j >= 0; --j) {
+      // columns < j of the partial product are still unit vectors e_c with c < j: untouched
+      const unsigned gx = (unsigned)((r - j + 31) / 32);
+      k_hh_apply<<<gx, 256, 0, s.st>>>(A, r, rows, j, V, r, j, j, r);
+      DION_CHECK_LAUNCH(c);
+    }
+    k_sign_fix<<<blocks, 256, 0, s.st>>>(A, r, rows, r, diag);
+    DION_CHECK_LAUNCH(c);
+  }
+  return DION_OK;
+}
+
+// Orthonormalize the rows x r panel in ws.P0; returns the buffer that holds U.
+int orthonormalize(StepCtx& s, i64 rows, i64 r, i64 short_dim, float** U_out) {
+  float* P0 = s.ws + s.L.P0;
+  float* P1 = s.ws + s.L.P1;
+  int mode = s.c->cfg.orth;
+  if (mode == DION_ORTH_AUTO) mode = (4 * r <= short_dim) ? DION_ORTH_CHOLQR2 : DION_ORTH_SHIFTED3;
+  if (mode == DION_ORTH_CHOLQR2) {
+    DION_TRY(cholqr_round(s, P0, P1, rows, r, 0.f));
+    DION_TRY(cholqr_round(s, P1, P0, rows, r, 0.f));
+    *U_out = P0;
+  } else if (mode == DION_ORTH_SHIFTED3) {
+    DION_TRY(cholqr_round(s, P0, P1, rows, r, 1e-6f));
+    DION_TRY(cholqr_round(s, P1, P0, rows, r, 0.f));
+    DION_TRY(cholqr_round(s, P0, P1, rows, r, 0.f));
+    *U_out = P1;
+  } else {
+    DION_TRY(householder(s, P0, P1, rows, r));
+    *U_out = P0;
+  }
+  return DION_OK;
+}
+
+int colnorm(StepCtx& s, const float* W, i64 rows, i64 r, float* out, i64 ldo, float* d_out) {
+  dion_ctx* c = s.c;
+  int chunks; i64 per;
+  colnorm_plan(rows, r, c->sm_count, &chunks, &per);
+  float* part = s.ws + s.L.cn_part;
+  dim3 grid((unsigned)((r + 127) / 128), (unsigned)chunks);
+  k_colsumsq_partial<<<grid, 128, 0, s.st>>>(W, r, rows, r, per, part, nullptr);
+  DION_CHECK_LAUNCH(c);
+  k_colnorm_apply<<<grid, 128, 0, s.st>>>(W, r, rows, r, per, chunks, part, c->cfg.eps, out, ldo,
+                                         s.ws + s.L.d, d_out, c->dev_ints, s.flag);
+  DION_CHECK_LAUNCH(c);
+  return DION_OK;
+}
+
+bool overlap(const void* a, size_t na, const void* b, size_t nb) {
+  const uintptr_t a0 = (uintptr_t)a, b0 = (uintptr_t)b;
+  return a0 < b0 + nb && b0 < a0 + na;
+}
+
+int validate(const dion_matrix* a) {
+  if (a == nullptr) return DION_ERR_INVALID;
+  if (a->X == nullptr || a->M == nullptr || a->G == nullptr || a->Q == nullptr) return DION_ERR_INVALID;
+  if (a->g_dtype != DION_F32 && a->g_dtype != DION_BF16) return DION_ERR_INVALID;
+  if (a->m < 1 || a->n < 1) return DION_ERR_SHAPE;
+  if (a->r < 1 || a->r > a->m || a->r > a->n) return DION_ERR_SHAPE;
+  if (a->ldx < a->n || a->ldm < a->n || a->ldg < a->n || a->ldq < a->r) return DION_ERR_SHAPE;
+  const size_t gsz = (a->g_dtype == DION_BF16) ? 2 : 4;
+  if (((uintptr_t)a->X & 3) || ((uintptr_t)a->M & 3) || ((uintptr_t)a->Q & 3) || ((uintptr_t)a->G & (gsz - 1)))
+    return DION_ERR_ALIGN;
+  if (a->colnorm_out != nullptr && ((uintptr_t)a->colnorm_out & 3)) return DION_ERR_ALIGN;
+  const size_t nx = (size_t)((a->m - 1) * a->ldx + a->n) * 4, nm = (size_t)((a->m - 1) * a->ldm + a->n) * 4;
+  const size_t ng = (size_t)((a->m - 1) * a->ldg + a->n) * gsz, nq = (size_t)((a->n - 1) * a->ldq + a->r) * 4;
+  if (overlap(a->X, nx, a->M, nm) || overlap(a->X, nx, a->G, ng) || overlap(a->X, nx, a->Q, nq) ||
+      overlap(a->M, nm, a->G, ng) || overlap(a->M, nm, a->Q, nq) || overlap(a->G, ng, a->Q, nq))
+    return DION_ERR_ALIAS;
+  if (a->colnorm_out != nullptr) {
+    const size_t nc = (size_t)a->r * 4;
+    if (overlap(a->colnorm_out, nc, a->X, nx) || overlap(a->colnorm_out, nc, a->M, nm) ||
+        overlap(a->colnorm_out, nc, a->G, ng) || overlap(a->colnorm_out, nc, a->Q, nq))
+      return DION_ERR_ALIAS;
+  }
+  return DION_OK;
+}
+
+int begin_step(dion_ctx* c, const dion_matrix* a, cudaStream_t st, StepCtx* s) {
+  s->c = c;
+  s->st = st;
+  s->L = make_layout(c, a->m, a->n, a->r);
+  s->ws = c->ws;
+  s->flag = c->dev_ints + 2 + c->flag_cursor;
+  c->flag_cursor = (c->flag_cursor + 1) % MAX_FLAG_SLOTS;
+  s->tensor = (c->cfg.engine != DION_ENGINE_SIMT);
+  if (cudaMemsetAsync(s->flag, 0, sizeof(int), st) != cudaSuccess) return DION_ERR_CUDA;
+  return DION_OK;
+}
+
+// The launch chain of one Dion step (Algorithm 1 + 2).  Scratch must be large enough.
+int step_one(dion_ctx* c, const dion_matrix* a, float lr, cudaStream_t st) {
+  StepCtx s;
+  DION_TRY(begin_step(c, a, st, &s));
+  const i64 m = a->m, n = a->n, r = a->r;
+  const int gmode = (a->g_dtype == DION_BF16) ? ADD_BF16 : ADD_F32;
+  float* P0 = s.ws + s.L.P0;
+  float* R = s.ws + s.L.R;
+  const float* Mp = (const float*)a->M;
+
+  // P = (M + G) Q
+  GemmArgs p = gemm_args();
+  p.M = m; p.N = r; p.K = n;
+  p.A = Mp; p.a_si = a->ldm; p.a_sk = 1;
+  p.A2 = a->G; p.a2_si = a->ldg; p.a2_sk = 1; p.a2_mode = gmode;
+  p.B = (const float*)a->Q; p.b_sk = a->ldq; p.b_sn = 1;
+  p.C = P0; p.ldc = r; p.epi = EPI_STORE;
+  DION_TRY(launch_gemm(s, p));
+
+  // U = Orthonormalize(P)
+  float* U = nullptr;
+  DION_TRY(orthonormalize(s, m, r, (m < n) ? m : n, &U));
+
+  // R = (M + G)^T U
+  GemmArgs w = gemm_args();
+  w.M = n; w.N = r; w.K = m;
+  w.A = Mp; w.a_si = 1; w.a_sk = a->ldm;
+  w.A2 = a->G; w.a2_si = 1; w.a2_sk = a->ldg; w.a2_mode = gmode;
+  w.B = U; w.b_sk = r; w.b_sn = 1;
+  w.C = R; w.ldc = r; w.epi = EPI_STORE;
+  DION_TRY(launch_gemm(s, w));
+
+  // M <- (M + G) - (1 - mu) U R^T
+  GemmArgs e = gemm_args();
+  e.M = m; e.N = n; e.K = r;
+  e.A = U; e.a_si = r; e.a_sk = 1;
+  e.B = R; e.b_sk = 1; e.b_sn = r;
+  e.C = (float*)a->M; e.ldc = a->ldm; e.epi = EPI_ADD2_SUB;
+  e.C2 = a->G; e.ldc2 = a->ldg; e.c2_mode = gmode;
+  e.alpha = 1.f - c->cfg.mu;
+  e.skip_flag = s.flag;
+  DION_TRY(launch_gemm(s, e));
+
+  // Q <- ColNorm(R)
+  DION_TRY(colnorm(s, R, n, r, (float*)a->Q, a->ldq, a->colnorm_out));
+
+  // X <- X - lr sqrt(m/n) U Q^T
+  GemmArgs x = gemm_args();
+  x.M = m; x.N = n; x.K = r;
+  x.A = U; x.a_si = r; x.a_sk = 1;
+  x.B = (const float*)a->Q; x.b_sk = 1; x.b_sn = a->ldq;
+  x.C = (float*)a->X; x.ldc = a->ldx; x.epi = EPI_SUB;
+  x.alpha = lr * sqrtf((float)((double)m / (double)n));
+  x.skip_flag = s.flag;
+  DION_TRY(launch_gemm(s, x));
+
+  k_finish_step<<<1, 1, 0, st>>>(s.flag, c->dev_ints + 1);
+  DION_CHECK_LAUNCH(c);
+  return DION_OK;
+}
+
+// One Lazy-Dion step (Algorithm 6).
+int lazy_one(dion_ctx* c, const dion_matrix* a, float lr, int refresh, cudaStream_t st) {
+  StepCtx s;
+  DION_TRY(begin_step(c, a, st, &s));
+  const i64 m = a->m, n = a->n, r = a->r;
+  const int gmode = (a->g_dtype == DION_BF16) ? ADD_BF16 : ADD_F32;
+  float* P0 = s.ws + s.L.P0;
+  float* R = s.ws + s.L.R;
+  const float* Mp = (const float*)a->M;
+
+  if (refresh) {
+    // T = (M + G) Q  (m x r), Z = (M + G)^T T (n x r), Q <- Orthonormalize(Z)
+    GemmArgs t = gemm_args();
+    t.M = m; t.N = r; t.K = n;
+    t.A = Mp; t.a_si = a->ldm; t.a_sk = 1;
+    t.A2 = a->G; t.a2_si = a->ldg; t.a2_sk = 1; t.a2_mode = gmode;
+    t.B = (const float*)a->Q; t.b_sk = a->ldq; t.b_sn = 1;
+    t.C = R; t.ldc = r; t.epi = EPI_STORE;
+    DION_TRY(launch_gemm(s, t));
+    GemmArgs z = gemm_args();
+    z.M = n; z.N = r; z.K = m;
+    z.A = Mp; z.a_si = 1; z.a_sk = a->ldm;
+    z.A2 = a->G; z.a2_si = 1; z.a2_sk = a->ldg; z.a2_mode = gmode;
+    z.B = R; z.b_sk = r; z.b_sn = 1;
+    z.C = P0; z.ldc = r; z.epi = EPI_STORE;
+    DION_TRY(launch_gemm(s, z));
+    float* V = nullptr;
+    DION_TRY(orthonormalize(s, n, r, (m < n) ? m : n, &V));
+    // copy V into Q unless the round broke down (alpha = 1, identity product is overkill: strided copy kernel)
+    GemmArgs cp = gemm_args();
+    (void)cp;
+    const i64 total = n * r;
+    int blocks = (int)((total + 255) / 256);
+    if (blocks > 8 * c->sm_count) blocks = 8 * c->sm_count;
+    k_copy_panel<<<blocks, 256, 0, st>>>(V, r, (float*)a->Q, a->ldq, n, r, s.flag);
+    DION_CHECK_LAUNCH(c);
+  }
+  // W = (M + G) Q
+  GemmArgs w = gemm_args();
+  w.M = m; w.N = r; w.K = n;
+  w.A = Mp; w.a_si = a->ldm; w.a_sk = 1;
+  w.A2 = a->G; w.a2_si = a->ldg; w.a2_sk = 1; w.a2_mode = gmode;
+  w.B = (const float*)a->Q; w.b_sk = a->ldq; w.b_sn = 1;
+  w.C = R; w.ldc = r; w.epi = EPI_STORE;
+  DION_TRY(launch_gemm(s, w));
+  // M <- (M + G) - (1 - mu) W Q^T
+  GemmArgs e = gemm_args();
+  e.M = m; e.N = n; e.K = r;
+  e.A = R; e.a_si = r; e.a_sk = 1;
+  e.B = (const float*)a->Q; e.b_sk = 1; e.b_sn = a->ldq;
+  e.C = (float*)a->M; e.ldc = a->ldm; e.epi = EPI_ADD2_SUB;
+  e.C2 = a->G; e.ldc2 = a->ldg; e.c2_mode = gmode;
+  e.alpha = 1.f - c->cfg.mu;
+  e.skip_flag = s.flag;
+  DION_TRY(launch_gemm(s, e));
+  // U = ColNorm(W)
+  DION_TRY(colnorm(s, R, m, r, P0, r, a->colnorm_out));
+  // X <- X - lr sqrt(m/n) U Q^T
+  GemmArgs x = gemm_args();
+  x.M = m; x.N = n; x.K = r;
+  x.A = P0; x.a_si = r; x.a_sk = 1;
+  x.B = (const float*)a->Q; x.b_sk = 1; x.b_sn = a->ldq;
+  x.C = (float*)a->X; x.ldc = a->ldx; x.epi = EPI_SUB;
+  x.alpha = lr * sqrtf((float)((double)m / (double)n));
+  x.skip_flag = s.flag;
+  DION_TRY(launch_gemm(s, x));
+  k_finish_step<<<1, 1, 0, st>>>(s.flag, c->dev_ints + 1);
+  DION_CHECK_LAUNCH(c);
+  return DION_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+void dion_default_config(dion_config* cfg) {
+  if (cfg == nullptr) return;
+  cfg->mu = 0.95f;
+  cfg->eps = 1e-8f;
+  cfg->precision = DION_PREC_FP32;
+  cfg->orth = DION_ORTH_AUTO;
+  cfg->engine = DION_ENGINE_AUTO;
+  cfg->device = 0;
+  cfg->workspace_bytes = 0;
+}
+
+int dion_init(dion_ctx** out, const dion_config* cfg) {
+  if (out == nullptr) return DION_ERR_INVALID;
+  *out = nullptr;
+  if (cfg == nullptr) return DION_ERR_INVALID;
+  if (cfg->precision != DION_PREC_FP32 && cfg->precision != DION_PREC_BF16_OPERANDS) return DION_ERR_INVALID;
+  if (cfg->orth < DION_ORTH_AUTO || cfg->orth > DION_ORTH_HOUSEHOLDER) return DION_ERR_INVALID;
+  if (cfg->engine < DION_ENGINE_AUTO || cfg->engine > DION_ENGINE_TENSOR) return DION_ERR_INVALID;
+  if (!(cfg->mu >= 0.f && cfg->mu <= 1.f) || !(cfg->eps >= 0.f)) return DION_ERR_INVALID;
+  int ndev = 0;
+  if (cudaGetDeviceCount(&ndev) != cudaSuccess || cfg->device < 0 || cfg->device >= ndev) {
+    cudaGetLastError();
+    return DION_ERR_CUDA;
+  }
+  cudaDeviceProp prop;
+  if (cudaGetDeviceProperties(&prop, cfg->device) != cudaSuccess) return DION_ERR_CUDA;
+  if (prop.major != 10) return DION_ERR_CUDA;  // built for sm_100a only
+  if (cudaSetDevice(cfg->device) != cudaSuccess) return DION_ERR_CUDA;
+  dion_ctx* c = new (std::nothrow) dion_ctx;
+  if (c == nullptr) return DION_ERR_NOMEM;
+  memset(c, 0, sizeof(*c));
+  c->cfg = *cfg;
+  c->sm_count = prop.multiProcessorCount;
+  void* p = nullptr;
+  if (cudaMalloc(&p, sizeof(int) * (2 + MAX_FLAG_SLOTS)) != cudaSuccess) { delete c; return DION_ERR_NOMEM; }
+  c->dev_ints = (int*)p;
+  if (cudaMemset(p, 0, sizeof(int) * (2 + MAX_FLAG_SLOTS)) != cudaSuccess) { cudaFree(p); delete c; return DION_ERR_CUDA; }
+  if (umma_configure() != DION_OK) { cudaFree(p); delete c; return DION_ERR_CUDA; }
+  if (cfg->workspace_bytes > 0) {
+    const int rc = ensure_ws(c, cfg->workspace_bytes);
+    if (rc != DION_OK) { cudaFree(c->dev_ints); delete c; return rc; }
+  }
+  *out = c;
+  return DION_OK;
+}
+
+size_t dion_workspace_bytes(const dion_ctx* ctx, int64_t m, int64_t n, int64_t r) {
+  if (ctx == nullptr || m < 1 || n < 1 || r < 1 || r > m || r > n) return 0;
+  return (size_t)make_layout(ctx, m, n, r).total * sizeof(float);
+}
+
+int dion_step(dion_ctx* ctx, const dion_matrix* a, float lr, void* cuda_stream) {
+  if (ctx == nullptr) return DION_ERR_INVALID;
+  DION_TRY(validate(a));
+  if (cudaSetDevice(ctx->cfg.device) != cudaSuccess) return DION_ERR_CUDA;
+  DION_TRY(ensure_ws(ctx, dion_workspace_bytes(ctx, a->m, a->n, a->r)));
+  return step_one(ctx, a, lr, (cudaStream_t)cuda_stream);
+}
+
+int dion_step_grouped(dion_ctx* ctx, const dion_matrix* list, int count, float lr, void* cuda_stream) {
+  if (ctx == nullptr || count < 0) return DION_ERR_INVALID;
+  if (count == 0) return DION_OK;
+  if (list == nullptr) return DION_ERR_INVALID;
+  size_t need = 0;
+  for (int i = 0; i < count; ++i) {
+    DION_TRY(validate(&list[i]));
+    const size_t b = dion_workspace_bytes(ctx, list[i].m, list[i].n, list[i].r);
+    if (b > need) need = b;
+  }
+  if (cudaSetDevice(ctx->cfg.device) != cudaSuccess) return DION_ERR_CUDA;
+  DION_TRY(ensure_ws(ctx, need));
+  // The matrices are independent; they share the scratch, so their launch chains
+  // run back to back on the one stream.
+  for (int i = 0; i < count; ++i) DION_TRY(step_one(ctx, &list[i], lr, (cudaStream_t)cuda_stream));
+  return DION_OK;
+}
+
+int dion_lazy_step(dion_ctx* ctx, const dion_matrix* a, float lr, int refresh, void* cuda_stream) {
+  if (ctx == nullptr) return DION_ERR_INVALID;
+  DION_TRY(validate(a));
+  if (cudaSetDevice(ctx->cfg.device) != cudaSuccess) return DION_ERR_CUDA;
+  DION_TRY(ensure_ws(ctx, dion_workspace_bytes(ctx, a->m, a->n, a->r)));
+  return lazy_one(ctx, a, lr, refresh, (cudaStream_t)cuda_stream);
+}
+
+int dion_get_status(dion_ctx* ctx, void* cuda_stream, int* device_status, int* steps_skipped) {
+  if (ctx == nullptr) return DION_ERR_INVALID;
+  if (cudaSetDevice(ctx->cfg.device) != cudaSuccess) return DION_ERR_CUDA;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  int host[2] = {0, 0};
+  if (cudaMemcpyAsync(host, ctx->dev_ints, sizeof(host), cudaMemcpyDeviceToHost, st) != cudaSuccess) return DION_ERR_CUDA;
+  if (cudaMemsetAsync(ctx->dev_ints, 0, sizeof(host), st) != cudaSuccess) return DION_ERR_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return DION_ERR_CUDA;
+  if (device_status != nullptr) *device_status = host[0];
+  if (steps_skipped != nullptr) *steps_skipped = host[1];
+  return DION_OK;
+}
+
+int64_t dion_launch_count(const dion_ctx* ctx) { return ctx == nullptr ? 0 : ctx->launches; }
+
+void dion_destroy(dion_ctx* ctx) {
+  if (ctx == nullptr) return;
+  cudaSetDevice(ctx->cfg.device);
+  cudaDeviceSynchronize();
+  if (ctx->ws != nullptr) cudaFree(ctx->ws);
+  if (ctx->dev_ints != nullptr) cudaFree(ctx->dev_ints);
+  delete ctx;
+}
+
+const char* dion_strerror(int code) {
+  switch (code) {
+    case DION_OK: return "ok";
+    case DION_ERR_INVALID: return "invalid argument";
+    case DION_ERR_SHAPE: return "bad shape, rank or leading dimension";
+    case DION_ERR_ALIGN: return "misaligned pointer";
+    case DION_ERR_ALIAS: return "arrays overlap";
+    case DION_ERR_NOMEM: return "out of device memory";
+    case DION_ERR_CUDA: return "CUDA error or no sm_100 device";
+    case DION_ERR_UNSUPPORTED: return "shape not supported by the requested engine";
+    default: return "unknown error";
+  }
+}
+
+}  // extern "C"

@@ -1,0 +1,52 @@
+// Shared declarations of the Dion CUDA library (device + host helpers).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "dion.h"
+
+namespace dion {
+
+typedef int64_t i64;
+
+// How an operand element is formed from memory.
+enum : int { ADD_NONE = 0, ADD_F32 = 1, ADD_BF16 = 2 };
+// What the epilogue does with an accumulator.
+enum : int {
+  EPI_STORE = 0,      // C = alpha * acc
+  EPI_SUB = 1,        // C = C - alpha * acc
+  EPI_ADD2_SUB = 2    // C = C + C2 - alpha * acc   (error feedback: M <- M + G - beta U R^T)
+};
+// Which output tiles exist.
+enum : int { TRI_FULL = 0, TRI_LOWER = 1 };
+
+// One (optionally batched, optionally split-K) product C = op(A) * op(B).
+// A(i,k) = A[i*a_si + k*a_sk] (+ A2(i,k) of dtype a2_mode with its own strides)
+// B(k,j) = B[k*b_sk + j*b_sn]
+// C(i,j) = C[i*ldc + j]
+struct GemmArgs {
+  i64 M, N, K;
+  const float* A; i64 a_si, a_sk;
+  const void* A2; i64 a2_si, a2_sk; int a2_mode;
+  const float* B; i64 b_sk, b_sn;
+  float* C; i64 ldc;
+  int epi;
+  const void* C2; i64 ldc2; int c2_mode;
+  float alpha;
+  const float* alpha_dev;      // optional: alpha is multiplied by *alpha_dev
+  int batch; i64 bsA, bsB, bsC;  // batch count and element strides
+  int splits; float* part;       // split-K: partial sums, [splits][M][N]
+  int tri;                       // TRI_LOWER: tiles strictly above the diagonal are skipped
+  int klimit;                    // 1: B(k,j) == 0 for k > j  (K loop ends at the tile's last column)
+  const int* skip_flag;          // optional: if *skip_flag != 0 the kernel does nothing
+};
+
+__device__ __forceinline__ float load_add(const void* p, i64 off, int mode) {
+  if (mode == ADD_F32) return reinterpret_cast<const float*>(p)[off];
+  if (mode == ADD_BF16) return __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(p)[off]);
+  return 0.f;
+}
+
+}  // namespace dion

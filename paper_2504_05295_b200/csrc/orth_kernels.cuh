@@ -1,0 +1,230 @@
+// Small kernels of the orthonormalization (r x r factor work) and of ColNorm.
+#pragma once
+
+#include "dion_common.cuh"
+
+namespace dion {
+
+constexpr int NB = 64;  // diagonal block of the blocked Cholesky / triangular inverse
+
+// trace(G) of an r x r matrix -> *out scaled by `scale` (the diagonal shift of the
+// shifted Cholesky QR round).  One block; fixed summation order.
+__global__ void k_trace_scaled(const float* __restrict__ G, i64 ld, i64 r, float scale,
+                               float* __restrict__ out) {
+  __shared__ float red[256];
+  float s = 0.f;
+  for (i64 i = threadIdx.x; i < r; i += blockDim.x) s += G[i * ld + i];
+  red[threadIdx.x] = s;
+  __syncthreads();
+  for (int w = 128; w > 0; w >>= 1) {
+    if ((int)threadIdx.x < w) red[threadIdx.x] += red[threadIdx.x + w];
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) *out = red[0] * scale;
+}
+
+// Cholesky of one jb x jb (jb <= 64) diagonal block, in place (lower factor, the
+// strict upper part of the block is zeroed), plus the inverse of that factor into
+// Dinv (64 x 64, row-major, zero padded).  A pivot that is <= 0 or not finite sets
+// *step_flag and the BREAKDOWN status bit and is replaced by 1 so that everything
+// downstream stays finite.  `shift` (optional) is added to the diagonal first.
+__global__ void __launch_bounds__(256) k_potrf_diag(float* __restrict__ A, i64 ld, int jb,
+                                                    float* __restrict__ Dinv,
+                                                    const float* __restrict__ shift,
+                                                    int* __restrict__ step_flag,
+                                                    int* __restrict__ status) {
+  __shared__ float L[NB][NB + 1];
+  __shared__ float X[NB][NB + 1];
+  const int tid = threadIdx.x;
+  const float sh = (shift != nullptr) ? *shift : 0.f;
+  for (int e = tid; e < NB * NB; e += 256) {
+    const int i = e / NB, c = e % NB;
+    float v = 0.f;
+    if (i < jb && c <= i) v = A[(i64)i * ld + c] + ((i == c) ? sh : 0.f);
+    L[i][c] = v;
+    X[i][c] = 0.f;
+  }
+  __syncthreads();
+  for (int j = 0; j < jb; ++j) {
+    if (tid == 0) {
+      float p = L[j][j];
+      if (!(p > 0.f) || !isfinite(p)) {
+        *step_flag = 1;
+        atomicOr(status, DION_STATUS_BREAKDOWN);
+        p = 1.f;
+      }
+      L[j][j] = sqrtf(p);
+    }
+    __syncthreads();
+    const float d = L[j][j];
+    if (tid > j && tid < jb) L[tid][j] = L[tid][j] / d;
+    __syncthreads();
+    // trailing update of the lower triangle: L[i][c] -= L[i][j] * L[c][j], j < c <= i
+    for (int e = tid; e < NB * NB; e += 256) {
+      const int i = e / NB, c = e % NB;
+      if (c > j && c <= i && i < jb) L[i][c] = fmaf(-L[i][j], L[c][j], L[i][c]);
+    }
+    __syncthreads();
+  }
+  // inverse of the lower factor by forward substitution, one column per thread
+  if (tid < jb) {
+    const int t = tid;
+    for (int i = t; i < jb; ++i) {
+      float s = (i == t) ? 1.f : 0.f;
+      for (int k = t; k < i; ++k) s = fmaf(-L[i][k], X[k][t], s);
+      X[i][t] = s / L[i][i];
+    }
+  }
+  __syncthreads();
+  for (int e = tid; e < NB * NB; e += 256) {
+    const int i = e / NB, c = e % NB;
+    if (i < jb && c < jb) A[(i64)i * ld + c] = (c <= i) ? L[i][c] : 0.f;
+    Dinv[e] = X[i][c];
+  }
+}
+
+// Linv = 0 except the 64 x 64 diagonal blocks, which are copied from Dinv.
+__global__ void k_linv_init(float* __restrict__ Linv, i64 ld, i64 r, const float* __restrict__ Dinv) {
+  const i64 total = r * r;
+  for (i64 e = (i64)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (i64)gridDim.x * blockDim.x) {
+    const i64 i = e / r, c = e % r;
+    float v = 0.f;
+    if (i / NB == c / NB) v = Dinv[(i / NB) * (NB * NB) + (i % NB) * NB + (c % NB)];
+    Linv[i * ld + c] = v;
+  }
+}
+
+// Partial sums of squares per column: part[chunk][j] = sum over the chunk's rows of R[i][j]^2.
+// grid = (ceil(r/128), chunks); 128 threads, one column each (coalesced rows).
+__global__ void __launch_bounds__(128) k_colsumsq_partial(const float* __restrict__ R, i64 ld, i64 n, i64 r,
+                                                          i64 rows_per_chunk, float* __restrict__ part,
+                                                          const int* __restrict__ skip_flag) {
+  if (skip_flag != nullptr && *skip_flag != 0) return;
+  const i64 j = (i64)blockIdx.x * 128 + threadIdx.x;
+  if (j >= r) return;
+  const i64 i0 = (i64)blockIdx.y * rows_per_chunk;
+  const i64 i1 = min(n, i0 + rows_per_chunk);
+  float s = 0.f;
+  for (i64 i = i0; i < i1; ++i) {
+    const float v = R[i * ld + j];
+    s = fmaf(v, v, s);
+  }
+  part[(i64)blockIdx.y * r + j] = s;
+}
+
+// ColNorm: d_j = sqrt(sum of the partials in chunk order); Q[i][j] = R[i][j] / (d_j + eps).
+// Same grid as k_colsumsq_partial.  The chunk-0 blocks also export d.
+__global__ void __launch_bounds__(128) k_colnorm_apply(const float* __restrict__ R, i64 ldr, i64 n, i64 r,
+                                                       i64 rows_per_chunk, int chunks,
+                                                       const float* __restrict__ part, float eps,
+                                                       float* __restrict__ Q, i64 ldq,
+                                                       float* __restrict__ d_ws, float* __restrict__ d_out,
+                                                       int* __restrict__ status,
+                                                       const int* __restrict__ skip_flag) {
+  if (skip_flag != nullptr && *skip_flag != 0) return;
+  const i64 j = (i64)blockIdx.x * 128 + threadIdx.x;
+  if (j >= r) return;
+  float s = 0.f;
+  for (int c = 0; c < chunks; ++c) s += part[(i64)c * r + j];
+  const float d = sqrtf(s);
+  if (blockIdx.y == 0) {
+    d_ws[j] = d;
+    if (d_out != nullptr) d_out[j] = d;
+    if (!isfinite(d)) atomicOr(status, DION_STATUS_NONFINITE);
+  }
+  const float inv = 1.f / (d + eps);
+  const i64 i0 = (i64)blockIdx.y * rows_per_chunk;
+  const i64 i1 = min(n, i0 + rows_per_chunk);
+  for (i64 i = i0; i < i1; ++i) Q[i * ldq + j] = R[i * ldr + j] * inv;
+}
+
+// Copies a rows x r panel (ld = ldv) into Q (ld = ldq) unless the step was flagged.
+__global__ void k_copy_panel(const float* __restrict__ V, i64 ldv, float* __restrict__ Q, i64 ldq,
+                             i64 rows, i64 r, const int* __restrict__ skip_flag) {
+  if (skip_flag != nullptr && *skip_flag != 0) return;
+  const i64 total = rows * r;
+  for (i64 e = (i64)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (i64)gridDim.x * blockDim.x) {
+    const i64 i = e / r, c = e % r;
+    Q[i * ldq + c] = V[i * ldv + c];
+  }
+}
+
+// Counts a skipped step (breakdown) at the end of a step's launch chain.
+__global__ void k_finish_step(const int* __restrict__ step_flag, int* __restrict__ skipped) {
+  if (*step_flag != 0) atomicAdd(skipped, 1);
+}
+
+// ---------------------------------------------------------------------------
+// Householder QR (unblocked), the slow robust mode.
+// ---------------------------------------------------------------------------
+
+// Column j: builds the unit reflector v (stored in V[j:, j]) from A[j:, j] and
+// records R_qr[j][j] = alpha in diag[j].  One block of 1024 threads.
+__global__ void __launch_bounds__(1024) k_hh_reflector(float* __restrict__ A, i64 lda, i64 m, i64 j,
+                                                       float* __restrict__ V, i64 ldv,
+                                                       float* __restrict__ diag) {
+  __shared__ float red[1024];
+  __shared__ float s_alpha, s_vnorm;
+  const int tid = threadIdx.x;
+  float s = 0.f;
+  for (i64 i = j + tid; i < m; i += 1024) { const float v = A[i * lda + j]; s = fmaf(v, v, s); }
+  red[tid] = s;
+  __syncthreads();
+  for (int w = 512; w > 0; w >>= 1) { if (tid < w) red[tid] += red[tid + w]; __syncthreads(); }
+  if (tid == 0) {
+    const float norm = sqrtf(red[0]);
+    const float a0 = A[j * lda + j];
+    const float alpha = (a0 >= 0.f) ? -norm : norm;
+    // ||x - alpha e1||^2 = 2 norm^2 + 2 norm |x0|
+    s_alpha = alpha;
+    s_vnorm = sqrtf(2.f * norm * (norm + fabsf(a0)));
+    diag[j] = alpha;
+  }
+  __syncthreads();
+  const float alpha = s_alpha, vn = s_vnorm;
+  for (i64 i = j + tid; i < m; i += 1024) {
+    float v = A[i * lda + j];
+    if (i == j) v -= alpha;
+    V[i * ldv + j] = (vn > 0.f) ? v / vn : 0.f;
+  }
+}
+
+// T[j0:, c] -= 2 v (v^T T[j0:, c]) for the columns c in [c_begin, c_end); v = V[j0:, vj].
+// grid.x = column chunks of 32; block = 32 x 8 (32 columns, 8 row lanes).
+__global__ void __launch_bounds__(256) k_hh_apply(float* __restrict__ T, i64 ldt, i64 m, i64 j0,
+                                                  const float* __restrict__ V, i64 ldv, i64 vj,
+                                                  i64 c_begin, i64 c_end) {
+  __shared__ float red[8][33];
+  const int cx = threadIdx.x % 32, ry = threadIdx.x / 32;
+  const i64 c = c_begin + (i64)blockIdx.x * 32 + cx;
+  const bool ok = c < c_end;
+  float s = 0.f;
+  if (ok) for (i64 i = j0 + ry; i < m; i += 8) s = fmaf(V[i * ldv + vj], T[i * ldt + c], s);
+  red[ry][cx] = s;
+  __syncthreads();
+  float w = 0.f;
+#pragma unroll
+  for (int k = 0; k < 8; ++k) w += red[k][cx];
+  w *= 2.f;
+  if (ok) for (i64 i = j0 + ry; i < m; i += 8) T[i * ldt + c] = fmaf(-V[i * ldv + vj], w, T[i * ldt + c]);
+}
+
+// U = first r columns of the identity.
+__global__ void k_set_identity(float* __restrict__ U, i64 ld, i64 m, i64 r) {
+  const i64 total = m * r;
+  for (i64 e = (i64)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (i64)gridDim.x * blockDim.x) {
+    const i64 i = e / r, c = e % r;
+    U[i * ld + c] = (i == c) ? 1.f : 0.f;
+  }
+}
+
+// Sign convention: negate column j of U wherever diag[j] (= R_qr[j][j]) < 0.
+__global__ void k_sign_fix(float* __restrict__ U, i64 ld, i64 m, i64 r, const float* __restrict__ diag) {
+  const i64 total = m * r;
+  for (i64 e = (i64)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (i64)gridDim.x * blockDim.x) {
+    const i64 i = e / r, c = e % r;
+    if (diag[c] < 0.f) U[i * ld + c] = -U[i * ld + c];
+  }
+}
+
+}  // namespace dion

@@ -1,0 +1,258 @@
+"""Parity of the CUDA library (through the C-ABI) with the float64 CPU oracle on
+the same seeded inputs.  Needs a B200; run with ``-m gpu``.
+
+Tolerances: relative Frobenius error <= 1e-4 on X, M and Q for the fp32 path and
+<= 3e-2 for the bf16-operand path, after 1 and after 10 steps.
+"""
+import numpy as np
+import pytest
+import torch
+
+from helpers import EPS, ETA, MU, TOL_BF16, TOL_FP32, device_state, oracle_steps, rel, to_np64
+from paper_2504_05295_b200 import binding, build, inputs
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    build.build()
+    assert torch.cuda.is_available(), "GPU tests selected but no CUDA device is visible"
+    binding.load_library()
+
+
+def run_gpu(pb, steps, grads=None, **cfg):
+    X, M, Q = device_state(pb)
+    d = torch.zeros(pb.r, device="cuda")
+    snaps = []
+    with binding.Dion(mu=MU, eps=EPS, **cfg) as opt:
+        for t in range(steps):
+            G = (grads[t] if grads is not None else pb.grad(t)).to("cuda")
+            opt.step(X, M, G, Q, ETA, colnorm_out=d)
+            snaps.append((to_np64(X), to_np64(M), to_np64(Q), to_np64(d)))
+        status, skipped = opt.get_status()
+        launches = opt.launch_count()
+    assert launches > 0
+    return snaps, status, skipped
+
+
+def check(snap, res, tol, tag=""):
+    ex, em, eq = rel(snap[0], res.X), rel(snap[1], res.M), rel(snap[2], res.Q)
+    ed = rel(snap[3], res.d)
+    assert ex <= tol and em <= tol and eq <= tol and ed <= tol, \
+        f"{tag}: X {ex:.2e} M {em:.2e} Q {eq:.2e} d {ed:.2e} (tol {tol:.0e})"
+
+
+ENGINES = [binding.ENGINE_SIMT, binding.ENGINE_AUTO]
+
+
+@pytest.mark.parametrize("engine", ENGINES)
+@pytest.mark.parametrize("orth", [binding.ORTH_AUTO, binding.ORTH_CHOLQR2, binding.ORTH_SHIFTED3,
+                                  binding.ORTH_HOUSEHOLDER])
+def test_config1_after_1_and_10_steps(engine, orth):
+    m, n, r, ks = inputs.config1()
+    pb = inputs.make_problem(m, n, r, seed=0, ks=ks)
+    ref = oracle_steps(pb, 10)
+    snaps, status, skipped = run_gpu(pb, 10, engine=engine, orth=orth)
+    assert status == 0 and skipped == 0
+    check(snaps[0], ref[0], TOL_FP32, "step 1")
+    check(snaps[9], ref[9], TOL_FP32, "step 10")
+
+
+@pytest.mark.parametrize("engine", ENGINES)
+@pytest.mark.parametrize("m,n,r", [(1, 1, 1), (5, 3, 2), (3, 5, 3), (130, 70, 1), (257, 129, 33),
+                                   (200, 333, 65), (129, 1000, 129), (640, 384, 160)])
+def test_ragged_shapes_all_tiles_and_tails(engine, m, n, r):
+    pb = inputs.make_problem(m, n, r, seed=3, ks=min(8, m, n))
+    # at full rank the panel is ill conditioned; use the robust mode there
+    orth = binding.ORTH_HOUSEHOLDER if r == min(m, n) else binding.ORTH_AUTO
+    ref = oracle_steps(pb, 3)
+    snaps, status, skipped = run_gpu(pb, 3, engine=engine, orth=orth)
+    assert status == 0 and skipped == 0
+    tol = TOL_FP32 if r < min(m, n) else 2e-3   # tiny full-rank panels: cond(P) up to 1e4+
+    check(snaps[0], ref[0], tol, "step 1")
+    check(snaps[2], ref[2], tol, "step 3")
+
+
+@pytest.mark.parametrize("engine", ENGINES)
+def test_strided_leading_dimensions(engine):
+    m, n, r = 192, 320, 48
+    pb = inputs.make_problem(m, n, r, seed=4, ks=8)
+    ref = oracle_steps(pb, 2)
+    def padded(t, pad):
+        buf = torch.full((t.shape[0], t.shape[1] + pad), 7.0, device="cuda", dtype=t.dtype)
+        v = buf[:, :t.shape[1]]
+        v.copy_(t)
+        return buf, v
+    Xb, X = padded(pb.X, 4); Mb, M = padded(pb.M, 8); Qb, Q = padded(pb.Q, 12)
+    with binding.Dion(mu=MU, eps=EPS, engine=engine) as opt:
+        for t in range(2):
+            Gb, G = padded(pb.grad(t), 16)
+            opt.step(X, M, G, Q, ETA)
+        assert opt.get_status() == (0, 0)
+    assert rel(to_np64(X), ref[1].X) <= TOL_FP32 and rel(to_np64(M), ref[1].M) <= TOL_FP32
+    assert rel(to_np64(Q), ref[1].Q) <= TOL_FP32
+    # the padding columns were never written
+    assert torch.all(Xb[:, n:] == 7.0) and torch.all(Mb[:, n:] == 7.0) and torch.all(Qb[:, r:] == 7.0)
+
+
+@pytest.mark.parametrize("engine", ENGINES)
+def test_bf16_gradient_storage(engine):
+    m, n, r = 512, 384, 96
+    pb = inputs.make_problem(m, n, r, seed=5, ks=16, g_dtype=torch.bfloat16)
+    ref = oracle_steps(pb, 3)       # the oracle consumes the bf16-rounded values, up-cast exactly
+    snaps, status, skipped = run_gpu(pb, 3, engine=engine)
+    assert status == 0 and skipped == 0
+    check(snaps[2], ref[2], TOL_FP32, "bf16 G, fp32 arithmetic")
+
+
+def test_bf16_operand_mode_within_its_bar():
+    m, n, r = 1024, 768, 192
+    pb = inputs.make_problem(m, n, r, seed=6, ks=32, g_dtype=torch.bfloat16)
+    ref = oracle_steps(pb, 10)
+    snaps, status, skipped = run_gpu(pb, 10, precision=binding.PREC_BF16_OPERANDS)
+    assert status == 0 and skipped == 0
+    check(snaps[0], ref[0], TOL_BF16, "step 1")
+    check(snaps[9], ref[9], TOL_BF16, "step 10")
+
+
+@pytest.mark.parametrize("engine", ENGINES)
+@pytest.mark.parametrize("m,n,r", [(2048, 2048, 512), (2048, 2048, 128), (1024, 4096, 256), (4096, 1024, 256)])
+def test_multi_tile_sizes(engine, m, n, r):
+    pb = inputs.make_problem(m, n, r, seed=7, ks=64)
+    ref = oracle_steps(pb, 2)
+    snaps, status, skipped = run_gpu(pb, 2, engine=engine)
+    assert status == 0 and skipped == 0
+    check(snaps[0], ref[0], TOL_FP32, "step 1")
+    check(snaps[1], ref[1], TOL_FP32, "step 2")
+
+
+@pytest.mark.parametrize("engine", ENGINES)
+def test_full_rank_square_shifted_cholqr3(engine):
+    d = 1024
+    pb = inputs.make_problem(d, d, d, seed=8, ks=64)
+    ref = oracle_steps(pb, 3)
+    snaps, status, skipped = run_gpu(pb, 3, engine=engine)      # AUTO picks the shifted rounds
+    assert status == 0 and skipped == 0
+    check(snaps[0], ref[0], TOL_FP32, "step 1")
+    check(snaps[2], ref[2], TOL_FP32, "step 3")
+    # closed form at full rank: M_new = mu (M + G)
+    B = to_np64(pb.M) + to_np64(pb.grad(0))
+    assert rel(snaps[0][1], MU * B) <= TOL_FP32
+
+
+def test_grouped_equals_single_calls():
+    shapes = [(256, 512, 64), (512, 256, 64), (384, 384, 96), (256, 512, 64), (130, 70, 10)]
+    pbs = [inputs.make_problem(m, n, r, seed=9, k=k, ks=8) for k, (m, n, r) in enumerate(shapes)]
+    single, grouped = [], []
+    with binding.Dion(mu=MU, eps=EPS) as opt:
+        for pb in pbs:
+            X, M, Q = device_state(pb)
+            for t in range(2):
+                opt.step(X, M, pb.grad(t).cuda(), Q, ETA)
+            single.append((X, M, Q))
+        states = [device_state(pb) for pb in pbs]
+        for t in range(2):
+            opt.step_grouped([(X, M, pb.grad(t).cuda(), Q) for pb, (X, M, Q) in zip(pbs, states)], ETA)
+        opt.step_grouped([], ETA)      # empty list is a no-op
+        assert opt.get_status() == (0, 0)
+    for (X1, M1, Q1), (X2, M2, Q2), pb in zip(single, states, pbs):
+        assert torch.equal(X1, X2) and torch.equal(M1, M2) and torch.equal(Q1, Q2)
+        ref = oracle_steps(pb, 2)
+        assert rel(to_np64(X2), ref[1].X) <= TOL_FP32 and rel(to_np64(Q2), ref[1].Q) <= TOL_FP32
+
+
+def test_checkpoint_resume_is_bit_identical():
+    m, n, r, ks = inputs.config1()
+    pb = inputs.make_problem(m, n, r, seed=0, ks=ks)
+    grads = [pb.grad(t).cuda() for t in range(10)]
+    X, M, Q = device_state(pb)
+    with binding.Dion(mu=MU, eps=EPS) as opt:
+        for t in range(10):
+            opt.step(X, M, grads[t], Q, ETA)
+        torch.cuda.synchronize()
+    X2, M2, Q2 = device_state(pb)
+    with binding.Dion(mu=MU, eps=EPS) as opt:
+        for t in range(5):
+            opt.step(X2, M2, grads[t], Q2, ETA)
+        torch.cuda.synchronize()
+    saved = [t.cpu().clone() for t in (X2, M2, Q2)]          # "checkpoint": state is X, M, Q only
+    X3, M3, Q3 = [t.cuda() for t in saved]
+    with binding.Dion(mu=MU, eps=EPS) as opt:                # a fresh context: the library is stateless
+        for t in range(5, 10):
+            opt.step(X3, M3, grads[t], Q3, ETA)
+        torch.cuda.synchronize()
+    assert torch.equal(X, X3) and torch.equal(M, M3) and torch.equal(Q, Q3)
+
+
+def test_breakdown_is_flagged_and_leaves_state_untouched():
+    # a rank-deficient right factor (two equal columns) makes P = B Q rank deficient:
+    # outside the contract for parity, but it must be reported, finite and transactional
+    m, n, r = 256, 320, 32
+    pb = inputs.make_problem(m, n, r, seed=11, ks=8)
+    X, M, Q = device_state(pb)
+    Q[:, 5] = Q[:, 4]
+    Q[:, 9] = 0.0
+    X0, M0, Q0 = X.clone(), M.clone(), Q.clone()
+    G = pb.grad(0).cuda()
+    with binding.Dion(mu=MU, eps=EPS, orth=binding.ORTH_CHOLQR2) as opt:
+        opt.step(X, M, G, Q, ETA)
+        status, skipped = opt.get_status()
+        assert status & binding.STATUS_BREAKDOWN and skipped == 1
+        assert torch.equal(X, X0) and torch.equal(M, M0) and torch.equal(Q, Q0)
+        assert opt.get_status() == (0, 0)                    # reading clears the latch
+        # the context stays usable: a healthy step afterwards matches the oracle
+        Xh, Mh, Qh = device_state(pb)
+        opt.step(Xh, Mh, G, Qh, ETA)
+        assert opt.get_status() == (0, 0)
+    ref = oracle_steps(pb, 1)
+    assert rel(to_np64(Xh), ref[0].X) <= TOL_FP32 and rel(to_np64(Qh), ref[0].Q) <= TOL_FP32
+
+
+def test_zero_gradient_and_momentum_is_finite():
+    m, n, r = 128, 96, 8
+    pb = inputs.make_problem(m, n, r, seed=12, ks=4)
+    X, M, Q = device_state(pb)
+    G = torch.zeros(m, n, device="cuda")
+    for orth in (binding.ORTH_CHOLQR2, binding.ORTH_HOUSEHOLDER):
+        with binding.Dion(mu=MU, eps=EPS, orth=orth) as opt:
+            opt.step(X, M, G, Q, ETA)
+            opt.get_status()
+        assert all(bool(torch.isfinite(t).all()) for t in (X, M, Q))
+
+
+def test_argument_errors():
+    pb = inputs.make_problem(64, 48, 8, seed=13, ks=4)
+    X, M, Q = device_state(pb)
+    G = pb.grad(0).cuda()
+    with binding.Dion() as opt:
+        with pytest.raises(binding.DionError) as e:
+            opt.step(X, M, G, Q[:, :0], ETA)                 # r = 0 (an empty view has a NULL pointer)
+        assert e.value.code in (-1, -2)
+        with pytest.raises(binding.DionError) as e:
+            opt.step(X, X, G, Q, ETA)                        # aliasing
+        assert e.value.code == -4
+        big = torch.zeros(48, 49, device="cuda")
+        with pytest.raises(binding.DionError) as e:
+            opt.step(X, M, G, big, ETA)                      # r > min(m, n)
+        assert e.value.code == -2
+        opt.step(X, M, G, Q, ETA)
+        assert opt.get_status() == (0, 0)
+
+
+def test_lazy_dion_steps_match_oracle():
+    from oracle import dion_oracle as orc
+    m, n, r = 384, 256, 32
+    pb = inputs.make_problem(m, n, r, seed=14, ks=8)
+    X, M, Q = device_state(pb)
+    Xo, Mo, Qo = to_np64(pb.X), to_np64(pb.M), to_np64(pb.Q)
+    d = torch.zeros(r, device="cuda")
+    with binding.Dion(mu=MU, eps=EPS) as opt:
+        for t in range(6):
+            refresh = (t % 3 == 0)
+            G = pb.grad(t)
+            opt.lazy_step(X, M, G.cuda(), Q, ETA, refresh, colnorm_out=d)
+            Xo, Mo, Qo, do = orc.lazy_step(Xo, Mo, to_np64(G), Qo, MU, ETA, EPS, refresh=refresh)
+        assert opt.get_status() == (0, 0)
+    assert rel(to_np64(X), Xo) <= TOL_FP32 and rel(to_np64(M), Mo) <= TOL_FP32
+    assert rel(to_np64(Q), Qo) <= TOL_FP32 and rel(to_np64(d), do) <= TOL_FP32
