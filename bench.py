@@ -1,0 +1,422 @@
+#!/usr/bin/env python
+"""Benchmark of the Dion step (C-ABI CUDA library) on the square-matrix sweep.
+
+One "step" is one pass of the whole hot path (P, Orthonormalize, R, error
+feedback, ColNorm, X update) over one batch of synthetic input: one dion_step
+on each of the nine fp32 cases of the square sweep (2048^2, 4096^2, 8192^2 at
+rank fractions 1, 1/4, 1/16).  The metric is the device time of that pass in
+milliseconds (lower is better); per-case and per-phase times are reported
+beside it.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W]          # this library
+  python bench.py --impl reference ...                          # float64 CPU oracle, bounded sample
+
+For N > 1 launch with torch.distributed.run: every rank runs the same sweep on
+its own GPU (independent replicas, no collective on the data path; weak
+scaling); the time is the max over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "dion_step_time_square_sweep"
+UNIT = "ms"
+MU, ETA, EPS = 0.95, 0.01, 1e-8
+FFMA_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12     # 148 SMs x 128 FMA lanes x 2 flop x max clock
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            d = json.load(f)
+        return {"hbm_gbs": float(d["hbm_gbs"]), "bf16_burst": float(d["bf16_tflops"]),
+                "bf16_sustained": float(d.get("bf16_tflops_sustained", d["bf16_tflops"])), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_burst": 1590.0, "bf16_sustained": 1400.0, "source": "fallback"}
+
+
+def parse_cases(spec, inputs):
+    if not spec:
+        return inputs.config2_cases()
+    out = []
+    for tok in spec.split(","):
+        d, r = tok.split(":")
+        out.append((int(d), int(d), int(r)))
+    return out
+
+
+# ---------------------------------------------------------------------------
+# flop / byte models (algorithmic; stated in the design notes)
+# ---------------------------------------------------------------------------
+
+def orth_mode(m, n, r, orth):
+    if orth == 0:
+        return 1 if 4 * r <= min(m, n) else 2
+    return orth
+
+
+def phase_flops(m, n, r, orth):
+    rounds = {1: 2, 2: 4}.get(orth_mode(m, n, r, orth), 0)
+    if rounds:
+        o = rounds * (2.0 * m * r * r + r ** 3 / 3.0)     # Gram (symmetric half) + Cholesky + solve
+    else:
+        o = 4.0 * m * r * r - 4.0 / 3.0 * r ** 3          # Householder incl. forming the factor
+    g = 2.0 * m * n * r
+    return {"P": g, "ORTH": o, "R": g, "EF": g, "COLNORM": 3.0 * n * r, "X": g}
+
+
+def phase_bytes(m, n, r, orth, gbytes=4):
+    rounds = {1: 2, 2: 4}.get(orth_mode(m, n, r, orth), 2)
+    mn = float(m) * n
+    return {"P": mn * (4 + gbytes) + 4.0 * (n * r + m * r),
+            "ORTH": rounds * 4.0 * (3 * m * r),
+            "R": mn * (4 + gbytes) + 4.0 * (m * r + n * r),
+            "EF": mn * (8 + gbytes) + 4.0 * (m * r + n * r),
+            "COLNORM": 4.0 * 3 * n * r,
+            "X": mn * 8 + 4.0 * (m * r + n * r)}
+
+
+def oracle_flops(m, n, r):
+    return 8.0 * m * n * r + 4.0 * m * r * r - 4.0 / 3.0 * r ** 3
+
+
+# ---------------------------------------------------------------------------
+# clocks sampler
+# ---------------------------------------------------------------------------
+
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, device_index: int):
+        self.proc = None
+        self.path = None
+        self.dev = device_index
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(prefix="dion_clocks_", suffix=".csv")
+            os.close(fd)
+            self.out = open(self.path, "w")
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                                          "-lms", "100", "-i", str(self.dev)], stdout=self.out, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        res = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return res
+        try:
+            self.proc.terminate()
+            self.proc.wait(timeout=5)
+        except Exception:
+            pass
+        try:
+            self.out.close()
+            rows = [l.strip().split(",") for l in open(self.path) if l.strip()]
+            os.unlink(self.path)
+            sm, mx, reasons = [], [], set()
+            names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+            for row in rows:
+                if len(row) < 7:
+                    continue
+                try:
+                    sm.append(float(row[0])); mx.append(float(row[1]))
+                except ValueError:
+                    continue
+                for nm, v in zip(names, row[3:7]):
+                    if v.strip().lower() == "active":
+                        reasons.add(nm)
+            if sm:
+                res = {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(mx), "reasons": sorted(reasons),
+                       "samples": len(sm)}
+        except Exception:
+            pass
+        return res
+
+
+# ---------------------------------------------------------------------------
+# reference arm: the float64 oracle on host cores, bounded sample
+# ---------------------------------------------------------------------------
+
+def oracle_sample_cases(cases):
+    """The smallest matrix size of the sweep at its two low rank fractions."""
+    d0 = min(c[0] for c in cases)
+    pick = [c for c in cases if c[0] == d0 and c[2] < d0]
+    return pick or [min(cases, key=lambda c: oracle_flops(*c))]
+
+
+def time_oracle(cases, steps, warmup):
+    """Times the oracle as it stands on the sample cases.  Returns (ms per sample
+    pass, sample cases, projected ms for the full sweep by flop count, cores)."""
+    import torch
+    from oracle import dion_oracle as orc
+    from paper_2504_05295_b200 import inputs
+    sample = oracle_sample_cases(cases)
+    probs = []
+    for k, (m, n, r) in enumerate(sample):
+        pb = inputs.make_problem(m, n, r, seed=0, k=k, ks=64)
+        probs.append([pb, pb.X.double().numpy(), pb.M.double().numpy(), pb.Q.double().numpy(),
+                      pb.grad(0).double().numpy()])
+    times = []
+    for it in range(warmup + steps):
+        t0 = time.perf_counter()
+        for p in probs:
+            res = orc.step(p[1], p[2], p[4], p[3], MU, ETA, EPS)
+            p[1], p[2], p[3] = res.X, res.M, res.Q
+        dt = (time.perf_counter() - t0) * 1e3
+        if it >= warmup:
+            times.append(dt)
+    ms = sum(times) / len(times)
+    f_sample = sum(oracle_flops(*c) for c in sample)
+    f_full = sum(oracle_flops(*c) for c in cases)
+    return ms, sample, ms * f_full / f_sample, orc.num_threads()
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from paper_2504_05295_b200 import inputs
+    cases = parse_cases(args.cases, inputs)
+    steps, warmup = max(1, min(args.steps, 2)), min(args.warmup, 1)
+    ms, sample, projected, cores = time_oracle(cases, steps, warmup)
+    desc = ("float64 CPU oracle, one step each on " + ", ".join(f"{m}x{n} r={r}" for m, n, r in sample) +
+            f" (measured {ms:.1f} ms); value = that time scaled to the full sweep by the oracle's flop count "
+            "8mnr + 4mr^2 - 4/3 r^3")
+    line = {"impl": "reference", "metric": METRIC, "value": projected, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": steps, "warmup": warmup, "ms_per_step": projected, "higher_is_better": False,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": workload_name(cases), "cases": [list(c) for c in cases]},
+            "cpu_baseline": {"value": projected, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc,
+                             "sample_ms": ms},
+            "e2e": {"value": projected, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+def workload_name(cases):
+    return ("square fp32 sweep: " + ", ".join(f"{m}^2 r={r}" for m, n, r in cases) +
+            "; seeded low-rank (rank 64, s_i=2^-i/2) + 0.1 N(0,1) gradients")
+
+
+# ---------------------------------------------------------------------------
+# this library
+# ---------------------------------------------------------------------------
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2504_05295_b200 import binding, build, inputs
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    build.build()
+    peaks = load_peaks()
+    cases = parse_cases(args.cases, inputs)
+    dev = torch.device("cuda", local)
+    stream = torch.cuda.current_stream()
+    sptr = int(stream.cuda_stream)
+
+    # inputs resident in HBM: per case X, M, Q and a ring of two gradients
+    state = []
+    for k, (m, n, r) in enumerate(cases):
+        pb = inputs.make_problem(m, n, r, seed=rank, k=k, ks=64, device=dev, keep_signal=False)
+        gs = [pb.grad(t) for t in range(2)]
+        d = torch.zeros(r, device=dev)
+        descs = [binding.matrix_desc(pb.X, pb.M, g, pb.Q, d) for g in gs]
+        state.append({"pb": pb, "G": gs, "d": d, "descs": descs})
+    torch.cuda.synchronize()
+
+    opt = binding.Dion(mu=MU, eps=EPS, precision=args.precision, orth=args.orth, engine=args.engine, device=local)
+    need = max(opt.workspace_bytes(m, n, r) for m, n, r in cases)
+
+    def one_step(t, per_case_events=None):
+        for ci, st in enumerate(state):
+            if per_case_events is not None:
+                e0 = torch.cuda.Event(enable_timing=True); e0.record(stream)
+            opt.step_desc(st["descs"][t % 2], ETA, sptr)
+            if per_case_events is not None:
+                e1 = torch.cuda.Event(enable_timing=True); e1.record(stream)
+                per_case_events[ci].append((e0, e1))
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for t in range(args.warmup):
+        one_step(t)
+    torch.cuda.synchronize()
+    status, skipped = opt.get_status()
+
+    # ---- timed region: exactly K steps --------------------------------------------------
+    sampler = ClockSampler(local)
+    case_events = [[] for _ in cases]
+    launches0 = opt.launch_count()
+    opt.profile_enable(True)
+    barrier()
+    sampler.start()
+    e_start = torch.cuda.Event(enable_timing=True); e_end = torch.cuda.Event(enable_timing=True)
+    e_start.record(stream)
+    for t in range(args.steps):
+        one_step(args.warmup + t, case_events)
+    e_end.record(stream)
+    barrier()
+    clocks = sampler.stop()
+    ms_total = e_start.elapsed_time(e_end)
+    phase_ms, phase_launches = opt.profile_read()
+    opt.profile_enable(False)
+    launches = opt.launch_count() - launches0
+    status2, skipped2 = opt.get_status()
+    ms_step = ms_total / args.steps
+    if world > 1:
+        t_ = torch.tensor([ms_step], device=dev)
+        dist.all_reduce(t_, op=dist.ReduceOp.MAX)
+        ms_step = float(t_.item())
+
+    case_ms = [sum(a.elapsed_time(b) for a, b in ev) / len(ev) for ev in case_events]
+
+    # ---- end to end: host gradients in, column norms out, through the same C-ABI call ----
+    host_g = [st["G"][0].cpu().pin_memory() for st in state]
+    host_d = [torch.zeros(st["d"].shape, dtype=torch.float32).pin_memory() for st in state]
+    h2d = sum(g.numel() * g.element_size() for g in host_g)
+    d2h = sum(d.numel() * d.element_size() for d in host_d)
+
+    def e2e_step():
+        for st, hg, hd in zip(state, host_g, host_d):
+            st["G"][0].copy_(hg, non_blocking=True)
+            opt.step_desc(st["descs"][0], ETA, sptr)
+            hd.copy_(st["d"], non_blocking=True)
+
+    e2e_step()
+    barrier()
+    e2e_steps = max(1, min(args.steps, 3))
+    f0 = torch.cuda.Event(enable_timing=True); f1 = torch.cuda.Event(enable_timing=True)
+    f0.record(stream)
+    for _ in range(e2e_steps):
+        e2e_step()
+    f1.record(stream)
+    barrier()
+    e2e_ms = f0.elapsed_time(f1) / e2e_steps
+    if world > 1:
+        t_ = torch.tensor([e2e_ms], device=dev)
+        dist.all_reduce(t_, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t_.item())
+    status3, _ = opt.get_status()
+
+    if rank != 0:
+        opt.close()
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    # ---- roofline of the dominant phase ---------------------------------------------------
+    tot_fl = {p: 0.0 for p in binding.PHASES}
+    tot_by = {p: 0.0 for p in binding.PHASES}
+    for (m, n, r) in cases:
+        fl, by = phase_flops(m, n, r, args.orth), phase_bytes(m, n, r, args.orth)
+        for p in binding.PHASES:
+            tot_fl[p] += fl[p]; tot_by[p] += by[p]
+    dom = max(binding.PHASES, key=lambda p: phase_ms[p])
+    dom_ms = phase_ms[dom] / args.steps
+    tensor_engine = (args.engine != binding.ENGINE_SIMT)
+    if args.precision == binding.PREC_BF16_OPERANDS:
+        flop_peak, flop_bound, peak_note = peaks["bf16_sustained"], "tensor", "bf16 sustained, of " + peaks["source"]
+    elif tensor_engine:
+        flop_peak, flop_bound = peaks["bf16_sustained"] * 0.5, "tensor"
+        peak_note = "tf32 = 1/2 x bf16 sustained, of " + peaks["source"] + "; a 3xTF32 product counts once"
+    else:
+        flop_peak, flop_bound, peak_note = FFMA_PEAK_TFLOPS, "alu", "fp32 FMA: 148 SM x 128 lanes x 2 x 1.965 GHz"
+    t_flop = tot_fl[dom] / (flop_peak * 1e12) * 1e3
+    t_hbm = tot_by[dom] / (peaks["hbm_gbs"] * 1e9) * 1e3
+    if t_hbm >= t_flop:
+        achieved = tot_by[dom] / (dom_ms * 1e-3) / 1e9
+        roof = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                "frac": achieved / peaks["hbm_gbs"], "traffic": None, "peak_note": "copy bandwidth, of " + peaks["source"]}
+    else:
+        achieved = tot_fl[dom] / (dom_ms * 1e-3) / 1e12
+        roof = {"bound": flop_bound, "achieved": achieved, "peak": flop_peak, "unit": "TFLOP/s",
+                "frac": achieved / flop_peak, "traffic": None, "peak_note": peak_note}
+    roof.update({"kernel": "phase " + dom, "ms_per_step": dom_ms,
+                 "launches_per_step": phase_launches[dom] / args.steps,
+                 "algorithmic_flops_per_step": tot_fl[dom], "algorithmic_bytes_per_step": tot_by[dom]})
+
+    phases = {}
+    for p in binding.PHASES:
+        ms_p = phase_ms[p] / args.steps
+        phases[p] = {"ms": ms_p, "share": phase_ms[p] / max(sum(phase_ms.values()), 1e-9),
+                     "tflops": tot_fl[p] / (ms_p * 1e-3) / 1e12 if ms_p > 0 else None,
+                     "gbs": tot_by[p] / (ms_p * 1e-3) / 1e9 if ms_p > 0 else None}
+
+    # ---- CPU baseline: the oracle on a bounded sample (rank 0, N = 1 only) ---------------
+    cpu = None
+    if world == 1 and not args.no_cpu:
+        ms_o, sample, projected, cores = time_oracle(cases, 1, 0)
+        gpu_same = sum(case_ms[cases.index(c)] for c in sample)
+        cpu = {"value": ms_o, "unit": UNIT, "cores": cores, "kind": "oracle",
+               "sample": "one float64 oracle step each on " + ", ".join(f"{m}x{n} r={r}" for m, n, r in sample) +
+                         " (2 of the sweep's cases); value = their summed host time",
+               "gpu_ms_same_cases": gpu_same, "projected_full_sweep_ms": projected}
+
+    line = {"metric": METRIC, "value": ms_step, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": False, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16" if args.precision == binding.PREC_BF16_OPERANDS else "f32",
+            "data": "synthetic",
+            "config": {"workload": workload_name(cases), "cases": [list(c) for c in cases],
+                       "engine": ["auto", "simt", "tensor"][args.engine],
+                       "precision": ["fp32 (3xTF32 on tensor cores / FMA)", "bf16 operands"][args.precision],
+                       "orth": ["auto", "cholqr2", "shifted3", "householder"][args.orth],
+                       "l2": "inputs larger than L2: the sweep's 4 GB of X, M, G cycle through between repeats",
+                       "replicas": world, "workspace_bytes": need},
+            "cases": [{"m": m, "n": n, "r": r, "ms": ms} for (m, n, r), ms in zip(cases, case_ms)],
+            "phases": phases, "roofline": roof, "cpu_baseline": cpu,
+            "e2e": {"value": e2e_ms, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                    "steps": e2e_steps},
+            "gpu_launches": launches, "clocks": clocks,
+            "device_status": {"warmup": status, "timed": status2, "e2e": status3, "steps_skipped": skipped + skipped2}}
+    print(json.dumps(line))
+    opt.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=3)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--cases", default="", help="subset as d:r,d:r (default: the nine cases of the square sweep)")
+    ap.add_argument("--engine", type=int, default=0, help="0 auto, 1 simt, 2 tensor")
+    ap.add_argument("--precision", type=int, default=0, help="0 fp32, 1 bf16 operands")
+    ap.add_argument("--orth", type=int, default=0, help="0 auto, 1 cholqr2, 2 shifted3, 3 householder")
+    ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-baseline leg")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

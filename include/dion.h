@@ -57,10 +57,15 @@ typedef enum { DION_F32 = 0, DION_BF16 = 1 } dion_dtype;
 typedef enum { DION_PREC_FP32 = 0, DION_PREC_BF16_OPERANDS = 1 } dion_precision;
 
 /* Orthonormalize (Section 3.2 and the appendix on Cholesky QR).
- * DION_ORTH_AUTO:        CholeskyQR2 when 4 r <= min(m, n), else shifted CholeskyQR3.
- * DION_ORTH_CHOLQR2:     two rounds of Cholesky QR.
- * DION_ORTH_SHIFTED3:    a shifted Cholesky QR round followed by CholeskyQR2
- *                        (for ill-conditioned panels, e.g. full rank).
+ * DION_ORTH_AUTO:        CholeskyQR2 when 4 r <= min(m, n), else the adaptive rounds.
+ * DION_ORTH_CHOLQR2:     two rounds of Cholesky QR (cond(P) up to about 4e3); a
+ *                        non-positive pivot cancels the step (DION_STATUS_BREAKDOWN).
+ * DION_ORTH_SHIFTED3:    adaptive Cholesky QR rounds for ill-conditioned panels such as
+ *                        full rank: a column whose pivot falls below 1e-4 of its
+ *                        squared norm is deflated, so a round cannot break down and
+ *                        cuts cond(P) by up to ~100; rounds repeat (at most 6) until one sees a
+ *                        well-conditioned panel, one more round then finishes.  The
+ *                        decision is taken on the device; unused rounds are skipped.
  * DION_ORTH_HOUSEHOLDER: Householder QR (slow, most robust).                   */
 typedef enum {
   DION_ORTH_AUTO = 0,
@@ -91,7 +96,9 @@ enum {
   DION_STATUS_BREAKDOWN = 1,  /* a Cholesky pivot was <= 0 or not finite: the step
                                  that saw it left X, M and Q unchanged            */
   DION_STATUS_NONFINITE = 2,  /* a column norm of R was not finite                 */
-  DION_STATUS_TIMEOUT = 4     /* a bounded device-side wait ran out                */
+  DION_STATUS_TIMEOUT = 4,    /* a bounded device-side wait ran out                */
+  DION_STATUS_ILLCOND = 8     /* the adaptive rounds ran out before the panel was seen
+                                 well conditioned; the result may be less accurate  */
 };
 
 typedef struct {
@@ -149,6 +156,32 @@ size_t dion_workspace_bytes(const dion_ctx* ctx, int64_t m, int64_t n, int64_t r
  * (DION_STATUS_* bits) and the number of steps skipped because of a breakdown
  * since the last call.  Either output pointer may be NULL. */
 int dion_get_status(dion_ctx* ctx, void* cuda_stream, int* device_status, int* steps_skipped);
+
+/* Phases of a step, for dion_profile_read. */
+enum {
+  DION_PHASE_P = 0,       /* P = (M + G) Q                      */
+  DION_PHASE_ORTH = 1,    /* U = Orthonormalize(P)              */
+  DION_PHASE_R = 2,       /* R = (M + G)^T U                    */
+  DION_PHASE_EF = 3,      /* M <- (M + G) - (1 - mu) U R^T      */
+  DION_PHASE_COLNORM = 4, /* Q <- ColNorm(R)                    */
+  DION_PHASE_X = 5,       /* X <- X - lr sqrt(m/n) U Q^T        */
+  DION_NUM_PHASES = 6
+};
+
+/* Per-phase device timing with CUDA events recorded on the step's own stream.
+ * dion_profile_enable(ctx, 1) starts recording (and drops earlier records);
+ * dion_profile_enable(ctx, 0) stops.  dion_profile_read synchronises the recorded
+ * events, adds up the elapsed milliseconds and the kernel launches of every
+ * recorded step per phase into ms[DION_NUM_PHASES] / launches[DION_NUM_PHASES]
+ * (host arrays, either may be NULL) and drops the records.  Recording costs two
+ * event records per phase; leave it off when not measuring. */
+int dion_profile_enable(dion_ctx* ctx, int on);
+int dion_profile_read(dion_ctx* ctx, float* ms, int64_t* launches);
+
+/* Synchronises `cuda_stream`, then reports and clears the number of adaptive
+ * Cholesky QR rounds (DION_ORTH_SHIFTED3 / AUTO above rank fraction 1/4) that did
+ * work since the last call; rounds skipped on the device are not counted. */
+int dion_get_orth_rounds(dion_ctx* ctx, void* cuda_stream, int64_t* rounds);
 
 /* Number of kernel launches issued by this context so far (host counter). */
 int64_t dion_launch_count(const dion_ctx* ctx);

@@ -20,11 +20,12 @@ DION_F32, DION_BF16 = 0, 1
 PREC_FP32, PREC_BF16_OPERANDS = 0, 1
 ORTH_AUTO, ORTH_CHOLQR2, ORTH_SHIFTED3, ORTH_HOUSEHOLDER = 0, 1, 2, 3
 ENGINE_AUTO, ENGINE_SIMT, ENGINE_TENSOR = 0, 1, 2
-STATUS_BREAKDOWN, STATUS_NONFINITE, STATUS_TIMEOUT = 1, 2, 4
+STATUS_BREAKDOWN, STATUS_NONFINITE, STATUS_TIMEOUT, STATUS_ILLCOND = 1, 2, 4, 8
 
 EXPORTS = ["dion_default_config", "dion_init", "dion_step", "dion_step_grouped", "dion_lazy_step",
            "dion_workspace_bytes", "dion_get_status", "dion_launch_count", "dion_destroy",
-           "dion_strerror"]
+           "dion_strerror", "dion_profile_enable", "dion_profile_read", "dion_get_orth_rounds"]
+PHASES = ["P", "ORTH", "R", "EF", "COLNORM", "X"]
 
 
 class DionConfig(ctypes.Structure):
@@ -77,6 +78,12 @@ def load_library() -> ctypes.CDLL:
     lib.dion_get_status.restype = ci
     lib.dion_launch_count.argtypes = [vp]
     lib.dion_launch_count.restype = i64
+    lib.dion_profile_enable.argtypes = [vp, ci]
+    lib.dion_profile_enable.restype = ci
+    lib.dion_profile_read.argtypes = [vp, ctypes.POINTER(f32), ctypes.POINTER(i64)]
+    lib.dion_profile_read.restype = ci
+    lib.dion_get_orth_rounds.argtypes = [vp, vp, ctypes.POINTER(i64)]
+    lib.dion_get_orth_rounds.restype = ci
     lib.dion_destroy.argtypes = [vp]
     lib.dion_destroy.restype = None
     lib.dion_strerror.argtypes = [ci]
@@ -189,6 +196,23 @@ class Dion:
         st, sk = ctypes.c_int(0), ctypes.c_int(0)
         _check(self._lib.dion_get_status(self._ctx, _stream_ptr(stream), ctypes.byref(st), ctypes.byref(sk)))
         return st.value, sk.value
+
+    def profile_enable(self, on: bool) -> None:
+        _check(self._lib.dion_profile_enable(self._ctx, int(bool(on))))
+
+    def profile_read(self):
+        """Returns ({phase: ms}, {phase: launches}) summed over the recorded steps."""
+        ms = (ctypes.c_float * len(PHASES))()
+        nl = (ctypes.c_int64 * len(PHASES))()
+        _check(self._lib.dion_profile_read(self._ctx, ms, nl))
+        return ({p: float(ms[i]) for i, p in enumerate(PHASES)},
+                {p: int(nl[i]) for i, p in enumerate(PHASES)})
+
+    def orth_rounds(self, stream=None) -> int:
+        """Adaptive Cholesky QR rounds executed since the last call (synchronises)."""
+        n = ctypes.c_int64(0)
+        _check(self._lib.dion_get_orth_rounds(self._ctx, _stream_ptr(stream), ctypes.byref(n)))
+        return int(n.value)
 
     def launch_count(self) -> int:
         return int(self._lib.dion_launch_count(self._ctx))

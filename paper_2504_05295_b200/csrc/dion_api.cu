@@ -4,6 +4,7 @@
 #include <math.h>
 #include <new>
 #include <string.h>
+#include <vector>
 
 #include "dion_common.cuh"
 #include "orth_kernels.cuh"
@@ -14,13 +15,16 @@ using namespace dion;
 
 namespace {
 
-constexpr int MAX_FLAG_SLOTS = 4096;
+constexpr int MAX_FLAG_SLOTS = 4096;      // step slots of OS_SLOT_INTS ints each
+constexpr int MAX_ROUNDS = 6;             // adaptive Cholesky QR rounds
+constexpr float FLOOR_REL = 1e-4f;        // pivot floor relative to the column's squared norm
+constexpr float GOOD_REL = 1e-3f;         // smallest relative pivot of a well-conditioned round
 constexpr i64 PART_CAP_FLOATS = (i64)16 << 20;  // split-K partial sums, at most 64 MiB
 
 inline i64 align64(i64 floats) { return (floats + 63) / 64 * 64; }  // 256-byte granules
 
 struct Layout {
-  i64 P0, P1, R, Gram, Linv, Tbuf, Dinv, part, cn_part, d, scal, total;
+  i64 P0, P1, R, Gram, Linv, Tbuf, Dinv, DinvP, part, cn_part, d, gdiag, scal, total;
   i64 part_floats;
   int cn_chunks;
   i64 cn_rows;
@@ -36,6 +40,12 @@ struct dion_ctx {
   int* dev_ints;  // [0] status, [1] skipped, [2..] per-step flags
   int flag_cursor;
   int64_t launches;
+  // per-phase profiling (off by default)
+  bool prof_on;
+  std::vector<cudaEvent_t> prof_pool;   // reusable events
+  size_t prof_used;
+  struct ProfRec { int phase; cudaEvent_t e0, e1; int64_t launches; };
+  std::vector<ProfRec> prof_recs;
 };
 
 namespace {
@@ -61,6 +71,7 @@ Layout make_layout(const dion_ctx* c, i64 m, i64 n, i64 r) {
   L.Linv = o; o += align64(r * r);
   L.Tbuf = o; o += align64(r * r);
   L.Dinv = o; o += align64(((r + NB - 1) / NB) * (i64)NB * NB);
+  L.DinvP = o; o += align64(((r + NB - 1) / NB) * (i64)NB * NB);
   // split-K partials: the largest plain-store product of a step is max(m,n) x r
   i64 pf = 4 * (i64)c->sm_count * 64 * 64;
   if (pf > PART_CAP_FLOATS) pf = PART_CAP_FLOATS;
@@ -69,6 +80,7 @@ Layout make_layout(const dion_ctx* c, i64 m, i64 n, i64 r) {
   colnorm_plan(big, r, c->sm_count, &L.cn_chunks, &L.cn_rows);
   L.cn_part = o; o += align64((i64)(L.cn_chunks + 1) * r);
   L.d = o; o += align64(r);
+  L.gdiag = o; o += align64(r);
   L.scal = o; o += 64;
   L.total = o;
   return L;
@@ -149,7 +161,8 @@ struct StepCtx {
   cudaStream_t st;
   float* ws;
   Layout L;
-  int* flag;
+  int* os;    // this step's device state slot (OS_* ints)
+  int* flag;  // = os + OS_FAIL: the step must not write its outputs
   bool tensor;  // tensor-core engine allowed for this matrix
 };
 
@@ -165,17 +178,21 @@ int launch_gemm(StepCtx& s, const GemmArgs& g, bool force64 = false) {
 
 // Blocked right-looking Cholesky of the r x r matrix Gm (lower), diagonal-block
 // inverses into Dinv, then the full inverse of the factor into Linv.
-int potrf_trtri(StepCtx& s, float* Gm, i64 r, const float* shift) {
+int potrf_trtri(StepCtx& s, float* Gm, i64 r, const float* shift, bool adaptive) {
   dion_ctx* c = s.c;
   float* Dinv = s.ws + s.L.Dinv;
   float* Linv = s.ws + s.L.Linv;
   float* Tbuf = s.ws + s.L.Tbuf;
+  const float* gdiag = s.ws + s.L.gdiag;
   int* status = c->dev_ints;
+  const int* skip = adaptive ? (s.os + OS_DONE) : nullptr;
   for (i64 j0 = 0; j0 < r; j0 += NB) {
     const int jb = (int)((r - j0 < NB) ? (r - j0) : NB);
     float* Ajj = Gm + j0 * r + j0;
     float* Dj = Dinv + (j0 / NB) * (NB * NB);
-    k_potrf_diag<<<1, 256, 0, s.st>>>(Ajj, r, jb, Dj, shift, s.flag, status);
+    float* DPj = s.ws + s.L.DinvP + (j0 / NB) * (NB * NB);
+    k_potrf_diag<<<1, 256, 0, s.st>>>(Ajj, r, jb, Dj, DPj, shift, gdiag + j0, adaptive ? FLOOR_REL : 0.f, s.os,
+                                      adaptive ? 1 : 0, status);
     DION_CHECK_LAUNCH(c);
     const i64 rem = r - j0 - jb;
     if (rem > 0) {
@@ -183,14 +200,14 @@ int potrf_trtri(StepCtx& s, float* Gm, i64 r, const float* shift) {
       GemmArgs g = gemm_args();  // panel <- panel * Linv_jj^T, in place
       g.M = rem; g.N = jb; g.K = jb;
       g.A = panel; g.a_si = r; g.a_sk = 1;
-      g.B = Dj; g.b_sk = 1; g.b_sn = NB;
-      g.C = panel; g.ldc = r; g.epi = EPI_STORE;
+      g.B = DPj; g.b_sk = 1; g.b_sn = NB;
+      g.C = panel; g.ldc = r; g.epi = EPI_STORE; g.skip_flag = skip;
       DION_TRY(launch_gemm_simt(c, g, s.st, nullptr, 0, true));
       GemmArgs t = gemm_args();  // A22 -= panel * panel^T (lower tiles)
       t.M = rem; t.N = rem; t.K = jb;
       t.A = panel; t.a_si = r; t.a_sk = 1;
       t.B = panel; t.b_sk = 1; t.b_sn = r;
-      t.C = Gm + (j0 + jb) * r + (j0 + jb); t.ldc = r; t.epi = EPI_SUB; t.tri = TRI_LOWER;
+      t.C = Gm + (j0 + jb) * r + (j0 + jb); t.ldc = r; t.epi = EPI_SUB; t.tri = TRI_LOWER; t.skip_flag = skip;
       DION_TRY(launch_gemm_simt(c, t, s.st, nullptr, 0, false));
     }
   }
@@ -198,7 +215,7 @@ int potrf_trtri(StepCtx& s, float* Gm, i64 r, const float* shift) {
     const i64 total = r * r;
     int blocks = (int)((total + 255) / 256);
     if (blocks > 8 * c->sm_count) blocks = 8 * c->sm_count;
-    k_linv_init<<<blocks, 256, 0, s.st>>>(Linv, r, r, Dinv);
+    k_linv_init<<<blocks, 256, 0, s.st>>>(Linv, r, r, Dinv, skip);
     DION_CHECK_LAUNCH(c);
   }
   // inverse by doubling: [[L11,0],[L21,L22]]^-1 = [[X11,0],[-X22 L21 X11, X22]]
@@ -217,14 +234,14 @@ int potrf_trtri(StepCtx& s, float* Gm, i64 r, const float* shift) {
       g1.M = rows; g1.N = b; g1.K = b;
       g1.A = Gm + off21; g1.a_si = r; g1.a_sk = 1;
       g1.B = Linv + off11; g1.b_sk = r; g1.b_sn = 1;
-      g1.C = Tbuf + off21; g1.ldc = r; g1.epi = EPI_STORE;
+      g1.C = Tbuf + off21; g1.ldc = r; g1.epi = EPI_STORE; g1.skip_flag = skip;
       g1.batch = batch; g1.bsA = bs; g1.bsB = bs; g1.bsC = bs;
       DION_TRY(launch_gemm_simt(c, g1, s.st, nullptr, 0, false));
       GemmArgs g2 = gemm_args();  // X21 = -X22 * T
       g2.M = rows; g2.N = b; g2.K = rows;
       g2.A = Linv + off22; g2.a_si = r; g2.a_sk = 1;
       g2.B = Tbuf + off21; g2.b_sk = r; g2.b_sn = 1;
-      g2.C = Linv + off21; g2.ldc = r; g2.epi = EPI_STORE; g2.alpha = -1.f;
+      g2.C = Linv + off21; g2.ldc = r; g2.epi = EPI_STORE; g2.alpha = -1.f; g2.skip_flag = skip;
       g2.batch = batch; g2.bsA = bs; g2.bsB = bs; g2.bsC = bs;
       DION_TRY(launch_gemm_simt(c, g2, s.st, nullptr, 0, false));
     }
@@ -232,30 +249,40 @@ int potrf_trtri(StepCtx& s, float* Gm, i64 r, const float* shift) {
   return DION_OK;
 }
 
-// One Cholesky-QR round: Pout = Pin * chol(Pin^T Pin + shift I)^-T.  rows x r panels, ld = r.
-int cholqr_round(StepCtx& s, const float* Pin, float* Pout, i64 rows, i64 r, float shift_scale) {
+// One Cholesky-QR round: Pout = Pin * chol(Pin^T Pin)^-T.  rows x r panels, ld = r.
+// adaptive: pivots are floored, the round is skipped (Pout = Pin) once the panel is
+// orthonormal, and the round statistics are evaluated at the end.
+int cholqr_round(StepCtx& s, const float* Pin, float* Pout, i64 rows, i64 r, bool adaptive) {
   dion_ctx* c = s.c;
   float* Gm = s.ws + s.L.Gram;
+  const int* skip = adaptive ? (s.os + OS_DONE) : nullptr;
   GemmArgs g = gemm_args();
   g.M = r; g.N = r; g.K = rows;
   g.A = Pin; g.a_si = 1; g.a_sk = r;
   g.B = Pin; g.b_sk = r; g.b_sn = 1;
-  g.C = Gm; g.ldc = r; g.epi = EPI_STORE; g.tri = TRI_LOWER;
+  g.C = Gm; g.ldc = r; g.epi = EPI_STORE; g.tri = TRI_LOWER; g.skip_flag = skip;
   DION_TRY(launch_gemm(s, g));
-  const float* shift = nullptr;
-  if (shift_scale > 0.f) {
-    float* sh = s.ws + s.L.scal;
-    k_trace_scaled<<<1, 256, 0, s.st>>>(Gm, r, r, shift_scale, sh);
+  float* sh = s.ws + s.L.scal;
+  k_round_begin<<<1, 256, 0, s.st>>>(Gm, r, r, 0.f, s.ws + s.L.gdiag, sh, s.os, adaptive ? 1 : 0);
+  DION_CHECK_LAUNCH(c);
+  DION_TRY(potrf_trtri(s, Gm, r, nullptr, adaptive));
+  if (adaptive) {
+    const i64 total = rows * r;
+    int blocks = (int)((total + 255) / 256);
+    if (blocks > 8 * c->sm_count) blocks = 8 * c->sm_count;
+    k_copy_panel<<<blocks, 256, 0, s.st>>>(Pin, r, Pout, r, rows, r, nullptr, s.os + OS_DONE);
     DION_CHECK_LAUNCH(c);
-    shift = sh;
   }
-  DION_TRY(potrf_trtri(s, Gm, r, shift));
   GemmArgs u = gemm_args();
   u.M = rows; u.N = r; u.K = r;
   u.A = Pin; u.a_si = r; u.a_sk = 1;
   u.B = s.ws + s.L.Linv; u.b_sk = 1; u.b_sn = r; u.klimit = 1;
-  u.C = Pout; u.ldc = r; u.epi = EPI_STORE;
+  u.C = Pout; u.ldc = r; u.epi = EPI_STORE; u.skip_flag = skip;
   DION_TRY(launch_gemm(s, u));
+  if (adaptive) {
+    k_round_end<<<1, 1, 0, s.st>>>(s.os, GOOD_REL, c->dev_ints + 2);
+    DION_CHECK_LAUNCH(c);
+  }
   return DION_OK;
 }
 
@@ -296,14 +323,20 @@ int orthonormalize(StepCtx& s, i64 rows, i64 r, i64 short_dim, float** U_out) {
   int mode = s.c->cfg.orth;
   if (mode == DION_ORTH_AUTO) mode = (4 * r <= short_dim) ? DION_ORTH_CHOLQR2 : DION_ORTH_SHIFTED3;
   if (mode == DION_ORTH_CHOLQR2) {
-    DION_TRY(cholqr_round(s, P0, P1, rows, r, 0.f));
-    DION_TRY(cholqr_round(s, P1, P0, rows, r, 0.f));
+    DION_TRY(cholqr_round(s, P0, P1, rows, r, false));
+    DION_TRY(cholqr_round(s, P1, P0, rows, r, false));
     *U_out = P0;
   } else if (mode == DION_ORTH_SHIFTED3) {
-    DION_TRY(cholqr_round(s, P0, P1, rows, r, 1e-6f));
-    DION_TRY(cholqr_round(s, P1, P0, rows, r, 0.f));
-    DION_TRY(cholqr_round(s, P0, P1, rows, r, 0.f));
-    *U_out = P1;
+    // Adaptive rounds: the device decides after each round whether the panel is done.
+    static_assert(MAX_ROUNDS % 2 == 0, "the result must end in P0");
+    for (int it = 0; it < MAX_ROUNDS; it += 2) {
+      DION_TRY(cholqr_round(s, P0, P1, rows, r, true));
+      DION_TRY(cholqr_round(s, P1, P0, rows, r, true));
+    }
+    k_orth_finish<<<1, 1, 0, s.st>>>(s.os, s.c->dev_ints);
+    s.c->launches++;
+    if (cudaGetLastError() != cudaSuccess) return DION_ERR_CUDA;
+    *U_out = P0;
   } else {
     DION_TRY(householder(s, P0, P1, rows, r));
     *U_out = P0;
@@ -360,12 +393,36 @@ int begin_step(dion_ctx* c, const dion_matrix* a, cudaStream_t st, StepCtx* s) {
   s->st = st;
   s->L = make_layout(c, a->m, a->n, a->r);
   s->ws = c->ws;
-  s->flag = c->dev_ints + 2 + c->flag_cursor;
+  s->os = c->dev_ints + 8 + (i64)c->flag_cursor * OS_SLOT_INTS;
+  s->flag = s->os + OS_FAIL;
   c->flag_cursor = (c->flag_cursor + 1) % MAX_FLAG_SLOTS;
   s->tensor = (c->cfg.engine != DION_ENGINE_SIMT);
-  if (cudaMemsetAsync(s->flag, 0, sizeof(int), st) != cudaSuccess) return DION_ERR_CUDA;
+  if (cudaMemsetAsync(s->os, 0, sizeof(int) * OS_SLOT_INTS, st) != cudaSuccess) return DION_ERR_CUDA;
   return DION_OK;
 }
+
+cudaEvent_t prof_event(dion_ctx* c) {
+  if (c->prof_used == c->prof_pool.size()) {
+    cudaEvent_t e = nullptr;
+    if (cudaEventCreate(&e) != cudaSuccess) return nullptr;
+    c->prof_pool.push_back(e);
+  }
+  return c->prof_pool[c->prof_used++];
+}
+
+// Brackets one phase of a step with events on the step's stream when profiling is on.
+struct PhaseScope {
+  dion_ctx* c; cudaStream_t st; int phase; cudaEvent_t e0; int64_t l0;
+  PhaseScope(dion_ctx* c_, cudaStream_t st_, int phase_) : c(c_), st(st_), phase(phase_), e0(nullptr), l0(c_->launches) {
+    if (c->prof_on) { e0 = prof_event(c); if (e0) cudaEventRecord(e0, st); }
+  }
+  ~PhaseScope() {
+    if (c->prof_on && e0) {
+      cudaEvent_t e1 = prof_event(c);
+      if (e1) { cudaEventRecord(e1, st); c->prof_recs.push_back({phase, e0, e1, c->launches - l0}); }
+    }
+  }
+};
 
 // The launch chain of one Dion step (Algorithm 1 + 2).  Scratch must be large enough.
 int step_one(dion_ctx* c, const dion_matrix* a, float lr, cudaStream_t st) {
@@ -378,6 +435,8 @@ int step_one(dion_ctx* c, const dion_matrix* a, float lr, cudaStream_t st) {
   const float* Mp = (const float*)a->M;
 
   // P = (M + G) Q
+  {
+  PhaseScope ps(c, st, DION_PHASE_P);
   GemmArgs p = gemm_args();
   p.M = m; p.N = r; p.K = n;
   p.A = Mp; p.a_si = a->ldm; p.a_sk = 1;
@@ -385,12 +444,18 @@ int step_one(dion_ctx* c, const dion_matrix* a, float lr, cudaStream_t st) {
   p.B = (const float*)a->Q; p.b_sk = a->ldq; p.b_sn = 1;
   p.C = P0; p.ldc = r; p.epi = EPI_STORE;
   DION_TRY(launch_gemm(s, p));
+  }
 
   // U = Orthonormalize(P)
   float* U = nullptr;
+  {
+  PhaseScope ps(c, st, DION_PHASE_ORTH);
   DION_TRY(orthonormalize(s, m, r, (m < n) ? m : n, &U));
+  }
 
   // R = (M + G)^T U
+  {
+  PhaseScope ps(c, st, DION_PHASE_R);
   GemmArgs w = gemm_args();
   w.M = n; w.N = r; w.K = m;
   w.A = Mp; w.a_si = 1; w.a_sk = a->ldm;
@@ -398,8 +463,11 @@ int step_one(dion_ctx* c, const dion_matrix* a, float lr, cudaStream_t st) {
   w.B = U; w.b_sk = r; w.b_sn = 1;
   w.C = R; w.ldc = r; w.epi = EPI_STORE;
   DION_TRY(launch_gemm(s, w));
+  }
 
   // M <- (M + G) - (1 - mu) U R^T
+  {
+  PhaseScope ps(c, st, DION_PHASE_EF);
   GemmArgs e = gemm_args();
   e.M = m; e.N = n; e.K = r;
   e.A = U; e.a_si = r; e.a_sk = 1;
@@ -409,11 +477,17 @@ int step_one(dion_ctx* c, const dion_matrix* a, float lr, cudaStream_t st) {
   e.alpha = 1.f - c->cfg.mu;
   e.skip_flag = s.flag;
   DION_TRY(launch_gemm(s, e));
+  }
 
   // Q <- ColNorm(R)
+  {
+  PhaseScope ps(c, st, DION_PHASE_COLNORM);
   DION_TRY(colnorm(s, R, n, r, (float*)a->Q, a->ldq, a->colnorm_out));
+  }
 
   // X <- X - lr sqrt(m/n) U Q^T
+  {
+  PhaseScope ps(c, st, DION_PHASE_X);
   GemmArgs x = gemm_args();
   x.M = m; x.N = n; x.K = r;
   x.A = U; x.a_si = r; x.a_sk = 1;
@@ -422,9 +496,9 @@ int step_one(dion_ctx* c, const dion_matrix* a, float lr, cudaStream_t st) {
   x.alpha = lr * sqrtf((float)((double)m / (double)n));
   x.skip_flag = s.flag;
   DION_TRY(launch_gemm(s, x));
-
   k_finish_step<<<1, 1, 0, st>>>(s.flag, c->dev_ints + 1);
   DION_CHECK_LAUNCH(c);
+  }
   return DION_OK;
 }
 
@@ -462,7 +536,7 @@ int lazy_one(dion_ctx* c, const dion_matrix* a, float lr, int refresh, cudaStrea
     const i64 total = n * r;
     int blocks = (int)((total + 255) / 256);
     if (blocks > 8 * c->sm_count) blocks = 8 * c->sm_count;
-    k_copy_panel<<<blocks, 256, 0, st>>>(V, r, (float*)a->Q, a->ldq, n, r, s.flag);
+    k_copy_panel<<<blocks, 256, 0, st>>>(V, r, (float*)a->Q, a->ldq, n, r, s.flag, nullptr);
     DION_CHECK_LAUNCH(c);
   }
   // W = (M + G) Q
@@ -531,15 +605,16 @@ int dion_init(dion_ctx** out, const dion_config* cfg) {
   if (cudaGetDeviceProperties(&prop, cfg->device) != cudaSuccess) return DION_ERR_CUDA;
   if (prop.major != 10) return DION_ERR_CUDA;  // built for sm_100a only
   if (cudaSetDevice(cfg->device) != cudaSuccess) return DION_ERR_CUDA;
-  dion_ctx* c = new (std::nothrow) dion_ctx;
+  dion_ctx* c = new (std::nothrow) dion_ctx();
   if (c == nullptr) return DION_ERR_NOMEM;
-  memset(c, 0, sizeof(*c));
+  c->ws = nullptr; c->ws_bytes = 0; c->dev_ints = nullptr; c->flag_cursor = 0; c->launches = 0;
+  c->prof_on = false; c->prof_used = 0;
   c->cfg = *cfg;
   c->sm_count = prop.multiProcessorCount;
   void* p = nullptr;
-  if (cudaMalloc(&p, sizeof(int) * (2 + MAX_FLAG_SLOTS)) != cudaSuccess) { delete c; return DION_ERR_NOMEM; }
+  if (cudaMalloc(&p, sizeof(int) * (8 + MAX_FLAG_SLOTS * OS_SLOT_INTS)) != cudaSuccess) { delete c; return DION_ERR_NOMEM; }
   c->dev_ints = (int*)p;
-  if (cudaMemset(p, 0, sizeof(int) * (2 + MAX_FLAG_SLOTS)) != cudaSuccess) { cudaFree(p); delete c; return DION_ERR_CUDA; }
+  if (cudaMemset(p, 0, sizeof(int) * (8 + MAX_FLAG_SLOTS * OS_SLOT_INTS)) != cudaSuccess) { cudaFree(p); delete c; return DION_ERR_CUDA; }
   if (umma_configure() != DION_OK) { cudaFree(p); delete c; return DION_ERR_CUDA; }
   if (cfg->workspace_bytes > 0) {
     const int rc = ensure_ws(c, cfg->workspace_bytes);
@@ -601,6 +676,49 @@ int dion_get_status(dion_ctx* ctx, void* cuda_stream, int* device_status, int* s
   return DION_OK;
 }
 
+int dion_profile_enable(dion_ctx* ctx, int on) {
+  if (ctx == nullptr) return DION_ERR_INVALID;
+  ctx->prof_on = (on != 0);
+  if (on) { ctx->prof_recs.clear(); ctx->prof_used = 0; }
+  return DION_OK;
+}
+
+int dion_profile_read(dion_ctx* ctx, float* ms, int64_t* launches) {
+  if (ctx == nullptr) return DION_ERR_INVALID;
+  if (cudaSetDevice(ctx->cfg.device) != cudaSuccess) return DION_ERR_CUDA;
+  float acc[DION_NUM_PHASES] = {0};
+  int64_t nl[DION_NUM_PHASES] = {0};
+  int rc = DION_OK;
+  for (const auto& rec : ctx->prof_recs) {
+    float t = 0.f;
+    if (cudaEventSynchronize(rec.e1) != cudaSuccess || cudaEventElapsedTime(&t, rec.e0, rec.e1) != cudaSuccess) {
+      rc = DION_ERR_CUDA;
+      break;
+    }
+    acc[rec.phase] += t;
+    nl[rec.phase] += rec.launches;
+  }
+  ctx->prof_recs.clear();
+  ctx->prof_used = 0;
+  for (int i = 0; i < DION_NUM_PHASES; ++i) {
+    if (ms != nullptr) ms[i] = acc[i];
+    if (launches != nullptr) launches[i] = nl[i];
+  }
+  return rc;
+}
+
+int dion_get_orth_rounds(dion_ctx* ctx, void* cuda_stream, int64_t* rounds) {
+  if (ctx == nullptr || rounds == nullptr) return DION_ERR_INVALID;
+  if (cudaSetDevice(ctx->cfg.device) != cudaSuccess) return DION_ERR_CUDA;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  int host = 0;
+  if (cudaMemcpyAsync(&host, ctx->dev_ints + 2, sizeof(int), cudaMemcpyDeviceToHost, st) != cudaSuccess) return DION_ERR_CUDA;
+  if (cudaMemsetAsync(ctx->dev_ints + 2, 0, sizeof(int), st) != cudaSuccess) return DION_ERR_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return DION_ERR_CUDA;
+  *rounds = host;
+  return DION_OK;
+}
+
 int64_t dion_launch_count(const dion_ctx* ctx) { return ctx == nullptr ? 0 : ctx->launches; }
 
 void dion_destroy(dion_ctx* ctx) {
@@ -609,6 +727,7 @@ void dion_destroy(dion_ctx* ctx) {
   cudaDeviceSynchronize();
   if (ctx->ws != nullptr) cudaFree(ctx->ws);
   if (ctx->dev_ints != nullptr) cudaFree(ctx->dev_ints);
+  for (cudaEvent_t e : ctx->prof_pool) cudaEventDestroy(e);
   delete ctx;
 }
 

@@ -7,36 +7,70 @@ namespace dion {
 
 constexpr int NB = 64;  // diagonal block of the blocked Cholesky / triangular inverse
 
-// trace(G) of an r x r matrix -> *out scaled by `scale` (the diagonal shift of the
-// shifted Cholesky QR round).  One block; fixed summation order.
-__global__ void k_trace_scaled(const float* __restrict__ G, i64 ld, i64 r, float scale,
-                               float* __restrict__ out) {
+// Per-step device state of the orthonormalization (ints, one slot per step).
+enum : int {
+  OS_FAIL = 0,      // the step must not write X, M, Q (breakdown)
+  OS_DONE = 1,      // adaptive rounds: the panel is orthonormal, later rounds are skipped
+  OS_GOOD = 2,      // adaptive rounds: the last round saw a well-conditioned panel
+  OS_FLOORED = 3,   // pivots raised to the floor in the current round
+  OS_MINREL = 4,    // float bits: min over columns of pivot / original diagonal, current round
+  OS_ROUNDS = 5,    // rounds that did work
+  OS_SLOT_INTS = 8
+};
+
+// Round set-up on the r x r Gram matrix G (one block): saves diag(G) to gdiag, writes
+// shift = scale * trace(G) (fixed summation order) and resets the round statistics.
+__global__ void k_round_begin(const float* __restrict__ G, i64 ld, i64 r, float scale,
+                              float* __restrict__ gdiag, float* __restrict__ shift,
+                              int* __restrict__ os, int adaptive) {
+  if (adaptive && os[OS_DONE] != 0) return;
   __shared__ float red[256];
   float s = 0.f;
-  for (i64 i = threadIdx.x; i < r; i += blockDim.x) s += G[i * ld + i];
+  for (i64 i = threadIdx.x; i < r; i += blockDim.x) {
+    const float v = G[i * ld + i];
+    gdiag[i] = v;
+    s += v;
+  }
   red[threadIdx.x] = s;
   __syncthreads();
   for (int w = 128; w > 0; w >>= 1) {
     if ((int)threadIdx.x < w) red[threadIdx.x] += red[threadIdx.x + w];
     __syncthreads();
   }
-  if (threadIdx.x == 0) *out = red[0] * scale;
+  if (threadIdx.x == 0) {
+    *shift = red[0] * scale;
+    os[OS_FLOORED] = 0;
+    os[OS_MINREL] = 0x7f800000;  // +inf
+  }
 }
 
 // Cholesky of one jb x jb (jb <= 64) diagonal block, in place (lower factor, the
 // strict upper part of the block is zeroed), plus the inverse of that factor into
-// Dinv (64 x 64, row-major, zero padded).  A pivot that is <= 0 or not finite sets
-// *step_flag and the BREAKDOWN status bit and is replaced by 1 so that everything
-// downstream stays finite.  `shift` (optional) is added to the diagonal first.
+// Dinv (64 x 64, row-major, zero padded).  `shift` is added to the diagonal first.
+// floor_rel == 0 (plain Cholesky QR): a pivot that is <= 0 or not finite sets
+//   os[OS_FAIL] and the BREAKDOWN status bit and is replaced by 1 so that everything
+//   downstream stays finite.
+// floor_rel > 0 (adaptive rounds): a pivot below floor_rel * gdiag[j] (gdiag = the
+//   diagonal of the Gram matrix before elimination) is below the rounding noise of
+//   the Gram matrix.  Column j is then deflated: its diagonal entry becomes
+//   sqrt(floor), the entries below it zero, so the noisy column never reaches the
+//   trailing matrix.  The factor stays triangular and nonsingular for any panel;
+//   the round only improves the conditioning and a later round finishes the job.
+//   DinvP is Dinv with the rows of deflated columns zeroed: the panel below this
+//   block is multiplied by DinvP^T, which yields the zero columns of the factor.
 __global__ void __launch_bounds__(256) k_potrf_diag(float* __restrict__ A, i64 ld, int jb,
-                                                    float* __restrict__ Dinv,
+                                                    float* __restrict__ Dinv, float* __restrict__ DinvP,
                                                     const float* __restrict__ shift,
-                                                    int* __restrict__ step_flag,
+                                                    const float* __restrict__ gdiag, float floor_rel,
+                                                    int* __restrict__ os, int adaptive,
                                                     int* __restrict__ status) {
+  if (adaptive && os[OS_DONE] != 0) return;
   __shared__ float L[NB][NB + 1];
   __shared__ float X[NB][NB + 1];
+  __shared__ int deflated[NB];
   const int tid = threadIdx.x;
   const float sh = (shift != nullptr) ? *shift : 0.f;
+  if (tid < NB) deflated[tid] = 0;
   for (int e = tid; e < NB * NB; e += 256) {
     const int i = e / NB, c = e % NB;
     float v = 0.f;
@@ -45,11 +79,23 @@ __global__ void __launch_bounds__(256) k_potrf_diag(float* __restrict__ A, i64 l
     X[i][c] = 0.f;
   }
   __syncthreads();
+  int floored = 0;
+  float minrel = __int_as_float(0x7f800000);
   for (int j = 0; j < jb; ++j) {
     if (tid == 0) {
       float p = L[j][j];
-      if (!(p > 0.f) || !isfinite(p)) {
-        *step_flag = 1;
+      if (floor_rel > 0.f) {
+        const float g = gdiag[j] + sh;
+        const float fl = floor_rel * g;
+        if (!(p > fl) || !isfinite(p)) {
+          p = (fl > 0.f && isfinite(fl)) ? fl : 1.f;   // zero or non-finite column: unit pivot
+          ++floored;
+          deflated[j] = 1;
+        } else {
+          minrel = fminf(minrel, p / g);
+        }
+      } else if (!(p > 0.f) || !isfinite(p)) {
+        os[OS_FAIL] = 1;
         atomicOr(status, DION_STATUS_BREAKDOWN);
         p = 1.f;
       }
@@ -57,7 +103,7 @@ __global__ void __launch_bounds__(256) k_potrf_diag(float* __restrict__ A, i64 l
     }
     __syncthreads();
     const float d = L[j][j];
-    if (tid > j && tid < jb) L[tid][j] = L[tid][j] / d;
+    if (tid > j && tid < jb) L[tid][j] = deflated[j] ? 0.f : L[tid][j] / d;
     __syncthreads();
     // trailing update of the lower triangle: L[i][c] -= L[i][j] * L[c][j], j < c <= i
     for (int e = tid; e < NB * NB; e += 256) {
@@ -65,6 +111,10 @@ __global__ void __launch_bounds__(256) k_potrf_diag(float* __restrict__ A, i64 l
       if (c > j && c <= i && i < jb) L[i][c] = fmaf(-L[i][j], L[c][j], L[i][c]);
     }
     __syncthreads();
+  }
+  if (tid == 0 && floor_rel > 0.f) {
+    if (floored) atomicAdd(&os[OS_FLOORED], floored);
+    atomicMin(&os[OS_MINREL], __float_as_int(minrel));
   }
   // inverse of the lower factor by forward substitution, one column per thread
   if (tid < jb) {
@@ -80,11 +130,39 @@ __global__ void __launch_bounds__(256) k_potrf_diag(float* __restrict__ A, i64 l
     const int i = e / NB, c = e % NB;
     if (i < jb && c < jb) A[(i64)i * ld + c] = (c <= i) ? L[i][c] : 0.f;
     Dinv[e] = X[i][c];
+    if (DinvP != nullptr) DinvP[e] = deflated[i] ? 0.f : X[i][c];
+  }
+}
+
+// End of an adaptive round (one thread).  A round that raised no pivot and whose
+// smallest relative pivot is >= good_rel saw a panel with cond <~ 1/sqrt(good_rel):
+// one more round after it brings orthonormality to rounding level, then the
+// remaining rounds are skipped.
+__global__ void k_round_end(int* __restrict__ os, float good_rel, int* __restrict__ rounds_total) {
+  if (os[OS_DONE] != 0) return;
+  os[OS_ROUNDS] += 1;
+  atomicAdd(rounds_total, 1);
+  if (os[OS_GOOD] != 0) { os[OS_DONE] = 1; return; }
+  const float minrel = __int_as_float(os[OS_MINREL]);
+  if (os[OS_FLOORED] == 0 && minrel >= good_rel) os[OS_GOOD] = 1;
+}
+
+// After the last adaptive round: a panel that never became well conditioned is
+// reported; if pivots were still being raised the step is cancelled (rank-deficient P).
+__global__ void k_orth_finish(int* __restrict__ os, int* __restrict__ status) {
+  if (os[OS_DONE] != 0) return;
+  if (os[OS_GOOD] == 0 && os[OS_FLOORED] != 0) {
+    os[OS_FAIL] = 1;
+    atomicOr(status, DION_STATUS_BREAKDOWN);
+  } else {
+    atomicOr(status, DION_STATUS_ILLCOND);
   }
 }
 
 // Linv = 0 except the 64 x 64 diagonal blocks, which are copied from Dinv.
-__global__ void k_linv_init(float* __restrict__ Linv, i64 ld, i64 r, const float* __restrict__ Dinv) {
+__global__ void k_linv_init(float* __restrict__ Linv, i64 ld, i64 r, const float* __restrict__ Dinv,
+                            const int* __restrict__ skip_flag) {
+  if (skip_flag != nullptr && *skip_flag != 0) return;
   const i64 total = r * r;
   for (i64 e = (i64)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (i64)gridDim.x * blockDim.x) {
     const i64 i = e / r, c = e % r;
@@ -139,9 +217,12 @@ __global__ void __launch_bounds__(128) k_colnorm_apply(const float* __restrict__
 }
 
 // Copies a rows x r panel (ld = ldv) into Q (ld = ldq) unless the step was flagged.
+// `only_if` (optional): the copy happens only when *only_if != 0.
 __global__ void k_copy_panel(const float* __restrict__ V, i64 ldv, float* __restrict__ Q, i64 ldq,
-                             i64 rows, i64 r, const int* __restrict__ skip_flag) {
+                             i64 rows, i64 r, const int* __restrict__ skip_flag,
+                             const int* __restrict__ only_if) {
   if (skip_flag != nullptr && *skip_flag != 0) return;
+  if (only_if != nullptr && *only_if == 0) return;
   const i64 total = rows * r;
   for (i64 e = (i64)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (i64)gridDim.x * blockDim.x) {
     const i64 i = e / r, c = e % r;
