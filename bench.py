@@ -66,8 +66,9 @@ def orth_mode(m, n, r, orth):
     return orth
 
 
-def phase_flops(m, n, r, orth):
-    rounds = {1: 2, 2: 4}.get(orth_mode(m, n, r, orth), 0)
+def phase_flops(m, n, r, orth, rounds=None):
+    if rounds is None:
+        rounds = {1: 2, 2: 4}.get(orth_mode(m, n, r, orth), 0)
     if rounds:
         o = rounds * (2.0 * m * r * r + r ** 3 / 3.0)     # Gram (symmetric half) + Cholesky + solve
     else:
@@ -76,8 +77,9 @@ def phase_flops(m, n, r, orth):
     return {"P": g, "ORTH": o, "R": g, "EF": g, "COLNORM": 3.0 * n * r, "X": g}
 
 
-def phase_bytes(m, n, r, orth, gbytes=4):
-    rounds = {1: 2, 2: 4}.get(orth_mode(m, n, r, orth), 2)
+def phase_bytes(m, n, r, orth, gbytes=4, rounds=None):
+    if rounds is None:
+        rounds = {1: 2, 2: 4}.get(orth_mode(m, n, r, orth), 2)
     mn = float(m) * n
     return {"P": mn * (4 + gbytes) + 4.0 * (n * r + m * r),
             "ORTH": rounds * 4.0 * (3 * m * r),
@@ -324,6 +326,15 @@ def run_ours(args):
         e2e_ms = float(t_.item())
     status3, _ = opt.get_status()
 
+    # adaptive Cholesky-QR rounds per case, read on one more (untimed) step
+    opt.orth_rounds()
+    case_rounds = []
+    for ci, st in enumerate(state):
+        opt.step_desc(st["descs"][1], ETA, sptr)
+        nr = opt.orth_rounds()
+        m_, n_, r_ = cases[ci]
+        case_rounds.append(nr if orth_mode(m_, n_, r_, args.orth) == 2 else None)
+
     if rank != 0:
         opt.close()
         if world > 1:
@@ -333,8 +344,8 @@ def run_ours(args):
     # ---- roofline of the dominant phase ---------------------------------------------------
     tot_fl = {p: 0.0 for p in binding.PHASES}
     tot_by = {p: 0.0 for p in binding.PHASES}
-    for (m, n, r) in cases:
-        fl, by = phase_flops(m, n, r, args.orth), phase_bytes(m, n, r, args.orth)
+    for (m, n, r), nr in zip(cases, case_rounds):
+        fl, by = phase_flops(m, n, r, args.orth, rounds=nr), phase_bytes(m, n, r, args.orth, rounds=nr)
         for p in binding.PHASES:
             tot_fl[p] += fl[p]; tot_by[p] += by[p]
     dom = max(binding.PHASES, key=lambda p: phase_ms[p])
@@ -388,7 +399,8 @@ def run_ours(args):
                        "orth": ["auto", "cholqr2", "shifted3", "householder"][args.orth],
                        "l2": "inputs larger than L2: the sweep's 4 GB of X, M, G cycle through between repeats",
                        "replicas": world, "workspace_bytes": need},
-            "cases": [{"m": m, "n": n, "r": r, "ms": ms} for (m, n, r), ms in zip(cases, case_ms)],
+            "cases": [{"m": m, "n": n, "r": r, "ms": ms, "adaptive_orth_rounds": nr}
+                      for (m, n, r), ms, nr in zip(cases, case_ms, case_rounds)],
             "phases": phases, "roofline": roof, "cpu_baseline": cpu,
             "e2e": {"value": e2e_ms, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "steps": e2e_steps},

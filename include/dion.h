@@ -88,7 +88,9 @@ enum {
   DION_ERR_ALIAS = -4,      /* two arrays of one matrix overlap                   */
   DION_ERR_NOMEM = -5,      /* scratch allocation failed                          */
   DION_ERR_CUDA = -6,       /* a CUDA runtime call failed, or no sm_100 device    */
-  DION_ERR_UNSUPPORTED = -7 /* the requested engine cannot take this shape        */
+  DION_ERR_UNSUPPORTED = -7, /* the requested engine cannot take this shape       */
+  DION_ERR_TOO_LARGE = -8    /* dion_step_noalloc: the shape needs more scratch than
+                                the library's built-in array holds                 */
 };
 
 /* Bits of the device status word (dion_get_status). */
@@ -185,6 +187,46 @@ int dion_get_orth_rounds(dion_ctx* ctx, void* cuda_stream, int64_t* rounds);
 
 /* Number of kernel launches issued by this context so far (host counter). */
 int64_t dion_launch_count(const dion_ctx* ctx);
+
+/* dion_step for callers that must not allocate device memory.
+ *
+ * (The paper has no counterpart: this entry point exists for the host program's
+ * sake, not for the method's.)
+ *
+ * Some programs that want to run a Dion step cannot call cudaMalloc at that point:
+ * a plug-in running inside another framework's memory pool that has claimed the
+ * whole device, a process working under a fixed memory budget negotiated at
+ * start-up, or code on a path where the allocator's implicit device-wide
+ * synchronisation is not acceptable.  dion_init and dion_step grow their scratch
+ * with cudaMalloc; this call never does, and it needs no dion_ctx.  Its scratch
+ * (the P/U panels, R, the Gram matrix and its factors, split-K partial sums, the
+ * column norms and the step's flags) lives in an array of 24 MiB that is part of
+ * the library image, so every GPU that loads the library holds those 24 MiB until
+ * the process exits.
+ *
+ * The step is the one dion_step computes with the default configuration
+ * (fp32 products, automatic orthonormalization and engine) and the given mu and
+ * eps, on the CURRENT device, asynchronously on `cuda_stream`.  `a` is a HOST
+ * pointer; the matrices it names are DEVICE pointers, as for dion_step.
+ *
+ * Limits and rules:
+ *   - A shape whose scratch need exceeds dion_noalloc_scratch_limit() bytes is
+ *     rejected with DION_ERR_TOO_LARGE and nothing is launched.  The need is about
+ *     4 * (3 * max(m,n) * r + 3 * r * r) bytes plus 10 MiB of fixed buffers; for
+ *     example 2048 x 2048 with r = 128 fits, 4096 x 4096 with r = 1024 does not.
+ *   - The first call on a device looks up the array's device address and the
+ *     device's attributes.  Make that first call outside any stream capture.
+ *   - All calls share the one array, which keeps whatever the previous call left
+ *     in it; each call clears the words that must start at zero.  Two calls whose
+ *     kernels overlap on the GPU (different streams, or several host threads) race
+ *     on the array: issue them on one stream, or order them with events.
+ *   - A Cholesky breakdown leaves X, M and Q unchanged, as in dion_step, but this
+ *     entry point has no status read-out; callers that need one use a dion_ctx.
+ *   - It calls no cudaMalloc, cudaFree or other allocating routine. */
+int dion_step_noalloc(const dion_matrix* a, float lr, float mu, float eps, void* cuda_stream);
+
+/* Bytes of scratch available to dion_step_noalloc. */
+size_t dion_noalloc_scratch_limit(void);
 
 /* Frees the scratch memory and the context.  NULL is allowed. */
 void dion_destroy(dion_ctx* ctx);

@@ -24,7 +24,8 @@ STATUS_BREAKDOWN, STATUS_NONFINITE, STATUS_TIMEOUT, STATUS_ILLCOND = 1, 2, 4, 8
 
 EXPORTS = ["dion_default_config", "dion_init", "dion_step", "dion_step_grouped", "dion_lazy_step",
            "dion_workspace_bytes", "dion_get_status", "dion_launch_count", "dion_destroy",
-           "dion_strerror", "dion_profile_enable", "dion_profile_read", "dion_get_orth_rounds"]
+           "dion_strerror", "dion_profile_enable", "dion_profile_read", "dion_get_orth_rounds",
+           "dion_step_noalloc", "dion_noalloc_scratch_limit"]
 PHASES = ["P", "ORTH", "R", "EF", "COLNORM", "X"]
 
 
@@ -84,6 +85,10 @@ def load_library() -> ctypes.CDLL:
     lib.dion_profile_read.restype = ci
     lib.dion_get_orth_rounds.argtypes = [vp, vp, ctypes.POINTER(i64)]
     lib.dion_get_orth_rounds.restype = ci
+    lib.dion_step_noalloc.argtypes = [ctypes.POINTER(DionMatrix), f32, f32, f32, vp]
+    lib.dion_step_noalloc.restype = ci
+    lib.dion_noalloc_scratch_limit.argtypes = []
+    lib.dion_noalloc_scratch_limit.restype = ctypes.c_size_t
     lib.dion_destroy.argtypes = [vp]
     lib.dion_destroy.restype = None
     lib.dion_strerror.argtypes = [ci]
@@ -140,6 +145,20 @@ def matrix_desc(X: torch.Tensor, M: torch.Tensor, G: torch.Tensor, Q: torch.Tens
     else:
         d.colnorm_out = None
     return d
+
+
+def step_noalloc(X, M, G, Q, lr: float, mu: float = 0.95, eps: float = 1e-8, colnorm_out=None,
+                 stream=None) -> None:
+    """One Dion step through ``dion_step_noalloc``: no context, no device allocation; the
+    scratch is the library's built-in 24 MiB array on the current device.  Calls must not
+    overlap on the GPU.  Raises DionError(-8) when the shape needs more scratch than that."""
+    d = matrix_desc(X, M, G, Q, colnorm_out)
+    _check(load_library().dion_step_noalloc(ctypes.byref(d), float(lr), float(mu), float(eps),
+                                            _stream_ptr(stream)))
+
+
+def noalloc_scratch_limit() -> int:
+    return int(load_library().dion_noalloc_scratch_limit())
 
 
 class Dion:

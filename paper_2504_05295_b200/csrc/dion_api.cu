@@ -7,6 +7,7 @@
 #include <vector>
 
 #include "dion_common.cuh"
+#include "dion_internal.h"
 #include "orth_kernels.cuh"
 #include "simt_gemm.cuh"
 #include "umma_gemm.cuh"
@@ -169,9 +170,11 @@ struct StepCtx {
 // Engine dispatch: tensor cores when the product qualifies, else fp32 FMA.
 int launch_gemm(StepCtx& s, const GemmArgs& g, bool force64 = false) {
   if (s.tensor && !force64) {
-    const int rc = umma_try_launch(g, s.c->cfg.precision, s.c->sm_count, s.st);
-    if (rc == 1) { s.c->launches++; return cudaGetLastError() == cudaSuccess ? DION_OK : DION_ERR_CUDA; }
+    const int rc = umma_try_launch(g, s.c->cfg.precision, s.c->sm_count, s.ws + s.L.part, s.L.part_floats,
+                                   s.c->dev_ints, s.st);
+    if (rc > 0) { s.c->launches += rc; return DION_OK; }
     if (rc < 0) return rc;
+    if (s.c->cfg.engine == DION_ENGINE_TENSOR) return DION_ERR_UNSUPPORTED;
   }
   return launch_gemm_simt(s.c, g, s.st, s.ws + s.L.part, s.L.part_floats, force64);
 }
@@ -741,8 +744,123 @@ const char* dion_strerror(int code) {
     case DION_ERR_NOMEM: return "out of device memory";
     case DION_ERR_CUDA: return "CUDA error or no sm_100 device";
     case DION_ERR_UNSUPPORTED: return "shape not supported by the requested engine";
+    case DION_ERR_TOO_LARGE: return "shape needs more scratch than the built-in array of dion_step_noalloc holds";
     default: return "unknown error";
   }
 }
 
 }  // extern "C"
+
+// ---------------------------------------------------------------------------
+// dion_step_noalloc: the same step with its scratch in a built-in device array.
+// ---------------------------------------------------------------------------
+
+namespace {
+
+constexpr size_t NOALLOC_SCRATCH_BYTES = (size_t)24 << 20;  // 24 MiB, resident on every device that loads the library
+constexpr size_t NOALLOC_INT_BYTES = 256;                   // status word, counters and one step slot
+constexpr int NOALLOC_MAX_DEVICES = 64;
+
+// Scratch of dion_step_noalloc.  In host code this name is only a handle for
+// cudaGetSymbolAddress; the device address is looked up once per device below.
+static __device__ __align__(256) unsigned char g_noalloc_scratch[NOALLOC_SCRATCH_BYTES];
+
+struct NoallocDevice {
+  bool ready;
+  unsigned char* base;
+  int sm_count;
+};
+NoallocDevice g_noalloc_dev[NOALLOC_MAX_DEVICES];
+
+// First use on the current device: resolve the array's device address and read the
+// device attributes.  No allocation; must not run inside a stream capture.
+int noalloc_setup(int device, NoallocDevice** out) {
+  if (device < 0 || device >= NOALLOC_MAX_DEVICES) return DION_ERR_INVALID;
+  NoallocDevice* d = &g_noalloc_dev[device];
+  if (!d->ready) {
+    int major = 0, sms = 0;
+    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, device) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device) != cudaSuccess) {
+      cudaGetLastError();
+      return DION_ERR_CUDA;
+    }
+    if (major != 10) return DION_ERR_CUDA;
+    void* ptr = nullptr;
+    if (cudaGetSymbolAddress(&ptr, g_noalloc_scratch) != cudaSuccess || ptr == nullptr) {
+      cudaGetLastError();
+      return DION_ERR_CUDA;
+    }
+    if (umma_configure() != DION_OK) return DION_ERR_CUDA;
+    d->base = (unsigned char*)ptr;
+    d->sm_count = sms;
+    d->ready = true;
+  }
+  *out = d;
+  return DION_OK;
+}
+
+}  // namespace
+
+extern "C" int dion_step_noalloc(const dion_matrix* a, float lr, float mu, float eps, void* cuda_stream) {
+  DION_TRY(validate(a));
+  if (!(mu >= 0.f && mu <= 1.f) || !(eps >= 0.f)) return DION_ERR_INVALID;
+  int device = -1;
+  if (cudaGetDevice(&device) != cudaSuccess) { cudaGetLastError(); return DION_ERR_CUDA; }
+  NoallocDevice* nd = nullptr;
+  DION_TRY(noalloc_setup(device, &nd));
+
+  // A context that lives on the host stack for this call only and points at the
+  // built-in array: the launch chain is the one dion_step runs.
+  dion_ctx c;
+  dion_default_config(&c.cfg);
+  c.cfg.mu = mu;
+  c.cfg.eps = eps;
+  c.cfg.device = device;
+  c.sm_count = nd->sm_count;
+  c.dev_ints = (int*)nd->base;
+  c.ws = (float*)(nd->base + NOALLOC_INT_BYTES);
+  c.ws_bytes = NOALLOC_SCRATCH_BYTES - NOALLOC_INT_BYTES;
+  c.flag_cursor = 0;
+  c.launches = 0;
+  c.prof_on = false;
+  c.prof_used = 0;
+  const size_t need = (size_t)make_layout(&c, a->m, a->n, a->r).total * sizeof(float);
+  if (need > c.ws_bytes) return DION_ERR_TOO_LARGE;
+  // The array keeps what the previous call left: clear the status word and counters.
+  // (The step's own slot is cleared by the launch chain.)
+  if (cudaMemsetAsync(c.dev_ints, 0, 8 * sizeof(int), (cudaStream_t)cuda_stream) != cudaSuccess) return DION_ERR_CUDA;
+  return step_one(&c, a, lr, (cudaStream_t)cuda_stream);
+}
+
+extern "C" size_t dion_noalloc_scratch_limit(void) { return NOALLOC_SCRATCH_BYTES - NOALLOC_INT_BYTES; }
+
+// ---------------------------------------------------------------------------
+// Internal test hook (dion_internal.h)
+// ---------------------------------------------------------------------------
+extern "C" int dion_debug_gemm(int engine, int precision, const dion_debug_gemm_args* a, float* part,
+                               int64_t part_floats, int* status, void* cuda_stream) {
+  if (a == nullptr || status == nullptr) return DION_ERR_INVALID;
+  int device = 0, sms = 0;
+  if (cudaGetDevice(&device) != cudaSuccess) return DION_ERR_CUDA;
+  if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device) != cudaSuccess) return DION_ERR_CUDA;
+  if (umma_configure() != DION_OK) return DION_ERR_CUDA;
+  GemmArgs g = gemm_args();
+  g.M = a->M; g.N = a->N; g.K = a->K;
+  g.A = a->A; g.a_si = a->a_si; g.a_sk = a->a_sk;
+  g.A2 = a->A2; g.a2_si = a->a2_si; g.a2_sk = a->a2_sk; g.a2_mode = a->a2_mode;
+  g.B = a->B; g.b_sk = a->b_sk; g.b_sn = a->b_sn;
+  g.C = a->C; g.ldc = a->ldc; g.epi = a->epi;
+  g.C2 = a->C2; g.ldc2 = a->ldc2; g.c2_mode = a->c2_mode;
+  g.alpha = a->alpha; g.tri = a->tri; g.klimit = a->klimit;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  if (engine == DION_ENGINE_TENSOR) {
+    const int rc = umma_try_launch(g, precision, sms, part, part_floats, status, st);
+    if (rc > 0) return DION_OK;
+    return rc < 0 ? rc : DION_ERR_UNSUPPORTED;
+  }
+  dion_ctx c;
+  dion_default_config(&c.cfg);
+  c.sm_count = sms; c.launches = 0; c.prof_on = false; c.prof_used = 0;
+  return launch_gemm_simt(&c, g, st, part, part_floats, false);
+}
+

@@ -1,16 +1,583 @@
-// Tensor-core (tcgen05) engine of the large contractions.
+// Tensor-core (tcgen05 / TMEM) engine of the large contractions, sm_100a only.
+//
+// One persistent, warp-specialised kernel computes C = op(A) * op(B) on 128 x BN
+// output tiles:
+//   warps 0-3   epilogue: TMEM -> registers -> fused epilogue -> global memory
+//   warps 4-11  producers: global -> registers -> (M + G add, precision split) ->
+//               shared memory in the UMMA canonical 128-byte-swizzled layout
+//   warp  12    one elected thread issues tcgen05.mma and the commits
+// Accumulators are double buffered in TMEM (2 x BN columns), so the epilogue of a
+// tile overlaps the main loop of the next one.  Operand tiles go through registers
+// rather than TMA because every large operand is transformed on the way in: the
+// momentum buffer is formed as M + G, and fp32 operands are split into a TF32 "hi"
+// part and an fp32 "lo" remainder (3xTF32: hi*lo + lo*hi + hi*hi carries fp32
+// accuracy), or rounded to bf16 in the bf16-operand mode.
+//
+// Every wait on an mbarrier is bounded by a cycle budget: when it runs out the CTA
+// marks itself dead, raises DION_STATUS_TIMEOUT and drains, so a protocol bug
+// cannot hang the GPU.
 #pragma once
 
 #include "dion_common.cuh"
+#include "simt_gemm.cuh"
 
 namespace dion {
+namespace umma {
 
-// One-time per-process set-up of the tensor-core kernels (shared-memory opt-in).
-inline int umma_configure() { return DION_OK; }
+constexpr int BM = 128;
+constexpr int NUM_EPI_WARPS = 4;
+constexpr int NUM_PROD_WARPS = 8;
+constexpr int NUM_PROD_THREADS = NUM_PROD_WARPS * 32;
+constexpr int NUM_THREADS = (NUM_EPI_WARPS + NUM_PROD_WARPS + 1) * 32;
+constexpr long long SPIN_LIMIT_CYCLES = 2000000000LL;  // about one second
 
-// Returns 1 if the product was launched on the tensor cores, 0 if this engine
-// does not take the product (the caller then uses the fp32 FMA engine), or a
-// negative DION_ERR_* code.
-inline int umma_try_launch(const GemmArgs&, int /*precision*/, int /*sm_count*/, cudaStream_t) { return 0; }
+struct Params {
+  GemmArgs g;
+  int nM, nN;         // output tiles along M and N
+  int splits;         // K splits (>= 1); partial sums go to g.part when > 1
+  int kb_per_split;   // K blocks per split
+  int nkb;            // K blocks in all
+  int num_items;      // tiles * splits
+  int* status;        // device status word (DION_STATUS_TIMEOUT)
+};
+
+// ------------------------------------------------------------------ PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ void fence_barrier_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tmem_alloc(uint32_t slot, uint32_t ncols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(slot), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish() {
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+template <bool BF16>
+__device__ __forceinline__ void umma(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+  if (BF16) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+        "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+  } else {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+        "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+  }
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float* v) {
+  uint32_t r[32];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+  for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+__device__ __forceinline__ uint32_t cvt_tf32(float x) {
+  uint32_t r;
+  asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(x));
+  return r;
+}
+__device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+  asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
+
+// Bounded wait: false when the CTA is (or becomes) dead.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* dead, int* status) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  while (true) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if (*dead) return false;
+    if (clock64() - t0 > SPIN_LIMIT_CYCLES) {
+      *dead = 1;
+      atomicOr(status, DION_STATUS_TIMEOUT);
+      return false;
+    }
+  }
+}
+
+// Shared-memory matrix descriptor, 128-byte swizzle.  K-major: rows of 128 bytes,
+// 8-row groups 1024 bytes apart.  MN-major: 8 x 128-byte atoms; `lbo_bytes` is the
+// distance between 32-element (fp32) / 64-element (bf16) chunks along M/N, groups
+// of 8 k-rows are 1024 bytes apart.
+__device__ __forceinline__ uint64_t make_desc(uint32_t saddr, bool mn_major, uint32_t lbo_bytes) {
+  const uint64_t lbo = mn_major ? (uint64_t)(lbo_bytes >> 4) : 1ull;
+  const uint64_t sbo = 1024 >> 4;
+  uint64_t d = 0;
+  d |= (uint64_t)((saddr >> 4) & 0x3FFF);
+  d |= lbo << 16;
+  d |= sbo << 32;
+  d |= 1ull << 46;   // descriptor version of sm_100
+  d |= 2ull << 61;   // SWIZZLE_128B
+  return d;
+}
+
+// Instruction descriptor: fp32 accumulate, TF32 or BF16 operands, M = 128, N = BN.
+__device__ __forceinline__ uint32_t make_idesc(bool bf16, bool a_mn, bool b_mn, int bn) {
+  uint32_t d = 0;
+  d |= 1u << 4;                         // D format: F32
+  d |= (bf16 ? 1u : 2u) << 7;           // A format
+  d |= (bf16 ? 1u : 2u) << 10;          // B format
+  d |= (a_mn ? 1u : 0u) << 15;
+  d |= (b_mn ? 1u : 0u) << 16;
+  d |= (uint32_t)(bn >> 3) << 17;
+  d |= (uint32_t)(BM >> 4) << 24;
+  return d;
+}
+
+struct Item {
+  int mi, ni, ks, kb0, kb1;
+};
+
+template <int BN, int BKE>
+__device__ __forceinline__ Item decode_item(const Params& p, int item) {
+  Item it;
+  const int tile = item / p.splits;
+  it.ks = item - tile * p.splits;
+  if (p.g.tri == TRI_LOWER) {
+    int mi = (int)((sqrtf(8.f * (float)tile + 1.f) - 1.f) * 0.5f);
+    while ((mi + 1) * (mi + 2) / 2 <= tile) ++mi;
+    while (mi * (mi + 1) / 2 > tile) --mi;
+    it.mi = mi;
+    it.ni = tile - mi * (mi + 1) / 2;
+  } else {
+    it.mi = tile / p.nN;
+    it.ni = tile - it.mi * p.nN;
+  }
+  int nkb = p.nkb;
+  if (p.g.klimit) {
+    const i64 kend = min(p.g.K, (i64)(it.ni + 1) * BN);
+    nkb = (int)((kend + BKE - 1) / BKE);
+  }
+  it.kb0 = it.ks * p.kb_per_split;
+  it.kb1 = min(nkb, it.kb0 + p.kb_per_split);
+  return it;
+}
+
+// Loads one operand tile (ROWS x BKE elements) into registers as chunks of EPC
+// elements: MN_MAJOR = false reads along k (unit k stride), true reads along the
+// row index (unit row stride).  v[c][e]: chunk c of this thread, element e.
+template <int ROWS, int BKE, int EPC, bool MN_MAJOR, int NCHUNK>
+__device__ __forceinline__ void load_tile(const float* __restrict__ base, i64 s_row, i64 s_k, const void* __restrict__ add,
+                                          i64 a_row, i64 a_k, int add_mode, i64 row0, i64 rows, i64 k0, i64 k_end,
+                                          int ptid, float (&v)[NCHUNK][EPC]) {
+  constexpr int CPR = MN_MAJOR ? (ROWS / EPC) : (BKE / EPC);  // chunks per k-row / per row
+#pragma unroll
+  for (int l = 0; l < NCHUNK; ++l) {
+    const int c = ptid + l * NUM_PROD_THREADS;
+    const int major = c / CPR, minor = c % CPR;
+    const i64 grow = MN_MAJOR ? (row0 + (i64)minor * EPC) : (row0 + major);
+    const i64 gk = MN_MAJOR ? (k0 + major) : (k0 + (i64)minor * EPC);
+    const bool ok = grow < rows && gk < k_end;
+#pragma unroll
+    for (int e = 0; e < EPC; ++e) v[l][e] = 0.f;
+    if (ok) {
+      const float* src = base + grow * s_row + gk * s_k;
+#pragma unroll
+      for (int q = 0; q < EPC / 4; ++q) {
+        const float4 t = __ldg(reinterpret_cast<const float4*>(src) + q);
+        v[l][q * 4 + 0] = t.x; v[l][q * 4 + 1] = t.y; v[l][q * 4 + 2] = t.z; v[l][q * 4 + 3] = t.w;
+      }
+      if (add_mode == ADD_F32) {
+        const float* s2 = reinterpret_cast<const float*>(add) + grow * a_row + gk * a_k;
+#pragma unroll
+        for (int q = 0; q < EPC / 4; ++q) {
+          const float4 t = __ldg(reinterpret_cast<const float4*>(s2) + q);
+          v[l][q * 4 + 0] += t.x; v[l][q * 4 + 1] += t.y; v[l][q * 4 + 2] += t.z; v[l][q * 4 + 3] += t.w;
+        }
+      } else if (add_mode == ADD_BF16) {
+        const __nv_bfloat16* s2 = reinterpret_cast<const __nv_bfloat16*>(add) + grow * a_row + gk * a_k;
+#pragma unroll
+        for (int q = 0; q < EPC / 4; ++q) {
+          const uint2 t = __ldg(reinterpret_cast<const uint2*>(s2) + q);
+          const __nv_bfloat162 lo = *reinterpret_cast<const __nv_bfloat162*>(&t.x);
+          const __nv_bfloat162 hi = *reinterpret_cast<const __nv_bfloat162*>(&t.y);
+          v[l][q * 4 + 0] += __low2float(lo); v[l][q * 4 + 1] += __high2float(lo);
+          v[l][q * 4 + 2] += __low2float(hi); v[l][q * 4 + 3] += __high2float(hi);
+        }
+      }
+    }
+  }
+}
+
+// Writes the chunks to shared memory in the swizzled canonical layout.  fp32 mode:
+// TF32 "hi" part to s_hi and the fp32 remainder to s_lo; bf16 mode: rounded to bf16.
+template <int ROWS, int BKE, int EPC, bool MN_MAJOR, int NCHUNK, bool BF16>
+__device__ __forceinline__ void store_tile(uint32_t s_hi, uint32_t s_lo, int ptid, const float (&v)[NCHUNK][EPC]) {
+  constexpr int CPR = MN_MAJOR ? (ROWS / EPC) : (BKE / EPC);
+#pragma unroll
+  for (int l = 0; l < NCHUNK; ++l) {
+    const int c = ptid + l * NUM_PROD_THREADS;
+    const int major = c / CPR, minor = c % CPR;
+    uint32_t off;
+    if (MN_MAJOR) {   // major = k row, minor = 16-byte chunk along M/N
+      off = (uint32_t)(minor >> 3) * (BKE * 128) + (uint32_t)major * 128 + (uint32_t)(((minor & 7) ^ (major & 7)) << 4);
+    } else {          // major = row, minor = 16-byte chunk along k (8 per 128-byte row)
+      off = (uint32_t)major * 128 + (uint32_t)((minor ^ (major & 7)) << 4);
+    }
+    if (BF16) {
+      uint32_t w[4];
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const __nv_bfloat162 b = __floats2bfloat162_rn(v[l][q * 2], v[l][q * 2 + 1]);
+        w[q] = *reinterpret_cast<const uint32_t*>(&b);
+      }
+      st_shared_v4(s_hi + off, w[0], w[1], w[2], w[3]);
+    } else {
+      uint32_t h[4], lo[4];
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        h[q] = cvt_tf32(v[l][q]);
+        lo[q] = __float_as_uint(v[l][q] - __uint_as_float(h[q]));
+      }
+      st_shared_v4(s_hi + off, h[0], h[1], h[2], h[3]);
+      st_shared_v4(s_lo + off, lo[0], lo[1], lo[2], lo[3]);
+    }
+  }
+}
+
+template <int BN, bool BF16>
+struct Cfg {
+  static constexpr int BKE = BF16 ? 64 : 32;                 // K elements per 128-byte row
+  static constexpr int EPC = BF16 ? 8 : 4;                   // elements per 16-byte chunk
+  static constexpr int A_BYTES = BM * 128;
+  static constexpr int B_BYTES = BN * 128;
+  static constexpr int STAGE_BYTES = (BF16 ? 1 : 2) * (A_BYTES + B_BYTES);
+  static constexpr int STAGES = (192 * 1024) / STAGE_BYTES;
+  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 + 512;
+  static constexpr int A_CHUNKS = BM * 8 / NUM_PROD_THREADS;  // 16-byte chunks per producer thread
+  static constexpr int B_CHUNKS = BN * 8 / NUM_PROD_THREADS;
+  static constexpr int TMEM_COLS = 2 * BN;
+};
+
+template <int BN, bool A_MN, bool B_MN, bool BF16>
+__global__ void __launch_bounds__(NUM_THREADS, 1) k_gemm_umma(const Params p) {
+  using C = Cfg<BN, BF16>;
+  constexpr int BKE = C::BKE, EPC = C::EPC, STAGES = C::STAGES;
+  if (p.g.skip_flag != nullptr && *p.g.skip_flag != 0) return;
+
+  extern __shared__ unsigned char smem_raw[];
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  unsigned char* smem_al = smem_raw + (smem_base - smem_u32(smem_raw));
+  // control block after the stages
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem_al + STAGES * C::STAGE_BYTES);
+  const uint32_t bar0 = smem_base + STAGES * C::STAGE_BYTES;
+  auto full_bar = [&](int s) { return bar0 + 8u * s; };
+  auto empty_bar = [&](int s) { return bar0 + 8u * (STAGES + s); };
+  auto accf_bar = [&](int b) { return bar0 + 8u * (2 * STAGES + b); };
+  auto acce_bar = [&](int b) { return bar0 + 8u * (2 * STAGES + 2 + b); };
+  const uint32_t drain_bar = bar0 + 8u * (2 * STAGES + 4);
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(bars + 2 * STAGES + 5);
+  volatile int* dead = reinterpret_cast<volatile int*>(bars + 2 * STAGES + 6);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), NUM_PROD_THREADS); mbar_init(empty_bar(s), 1); }
+    for (int b = 0; b < 2; ++b) { mbar_init(accf_bar(b), 1); mbar_init(acce_bar(b), NUM_EPI_WARPS * 32); }
+    mbar_init(drain_bar, 1);
+    *dead = 0;
+    fence_barrier_init();
+  }
+  if (warp == NUM_EPI_WARPS + NUM_PROD_WARPS) {
+    tmem_alloc(smem_u32((const void*)tmem_slot), C::TMEM_COLS);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  const GemmArgs& g = p.g;
+
+  if (warp < NUM_EPI_WARPS) {
+    // ------------------------------------------------------------ epilogue
+    int iter = 0;
+    for (int item = blockIdx.x; item < p.num_items; item += gridDim.x, ++iter) {
+      const Item it = decode_item<BN, BKE>(p, item);
+      const int ab = iter & 1;
+      const uint32_t ph = (uint32_t)(iter >> 1) & 1u;
+      if (!mbar_wait(accf_bar(ab), ph, dead, p.status)) break;
+      tc_fence_after();
+      const i64 gi = (i64)it.mi * BM + warp * 32 + lane;
+      const i64 n0 = (i64)it.ni * BN;
+      float alpha = g.alpha;
+#pragma unroll 1
+      for (int cb = 0; cb < BN / 32; ++cb) {
+        float acc[32];
+        tmem_ld32(tmem_base + (uint32_t)(ab * BN + cb * 32) + ((uint32_t)(warp * 32) << 16), acc);
+        if (gi < g.M) {
+#pragma unroll
+          for (int q = 0; q < 8; ++q) {
+            const i64 col = n0 + cb * 32 + q * 4;
+            if (col >= g.N) continue;
+            float4 a4 = make_float4(acc[q * 4], acc[q * 4 + 1], acc[q * 4 + 2], acc[q * 4 + 3]);
+            if (p.splits > 1) {
+              *reinterpret_cast<float4*>(g.part + ((i64)it.ks * g.M + gi) * g.N + col) = a4;
+              continue;
+            }
+            float4* cptr = reinterpret_cast<float4*>(g.C + gi * g.ldc + col);
+            float4 o;
+            if (g.epi == EPI_STORE) {
+              o = make_float4(alpha * a4.x, alpha * a4.y, alpha * a4.z, alpha * a4.w);
+            } else {
+              float4 c = *cptr;
+              if (g.epi == EPI_ADD2_SUB) {
+                if (g.c2_mode == ADD_F32) {
+                  const float4 t = __ldg(reinterpret_cast<const float4*>(reinterpret_cast<const float*>(g.C2) + gi * g.ldc2 + col));
+                  c.x += t.x; c.y += t.y; c.z += t.z; c.w += t.w;
+                } else {
+                  const uint2 t = __ldg(reinterpret_cast<const uint2*>(reinterpret_cast<const __nv_bfloat16*>(g.C2) + gi * g.ldc2 + col));
+                  const __nv_bfloat162 lo = *reinterpret_cast<const __nv_bfloat162*>(&t.x);
+                  const __nv_bfloat162 hi = *reinterpret_cast<const __nv_bfloat162*>(&t.y);
+                  c.x += __low2float(lo); c.y += __high2float(lo); c.z += __low2float(hi); c.w += __high2float(hi);
+                }
+              }
+              o = make_float4(c.x - alpha * a4.x, c.y - alpha * a4.y, c.z - alpha * a4.z, c.w - alpha * a4.w);
+            }
+            *cptr = o;
+          }
+        }
+      }
+      tc_fence_before();
+      mbar_arrive(acce_bar(ab));
+    }
+  } else if (warp < NUM_EPI_WARPS + NUM_PROD_WARPS) {
+    // ------------------------------------------------------------ producers
+    const int ptid = threadIdx.x - NUM_EPI_WARPS * 32;
+    int stage = 0;
+    uint32_t phase = 0;
+    bool alive = true;
+    for (int item = blockIdx.x; item < p.num_items && alive; item += gridDim.x) {
+      const Item it = decode_item<BN, BKE>(p, item);
+      const i64 row0a = (i64)it.mi * BM, row0b = (i64)it.ni * BN;
+      i64 k_end = g.K;
+      if (g.klimit) k_end = min(g.K, (i64)(it.ni + 1) * BN);
+      for (int kb = it.kb0; kb < it.kb1; ++kb) {
+        const i64 k0 = (i64)kb * BKE;
+        float va[C::A_CHUNKS][EPC];
+        float vb[C::B_CHUNKS][EPC];
+        load_tile<BM, BKE, EPC, A_MN, C::A_CHUNKS>(g.A, g.a_si, g.a_sk, g.A2, g.a2_si, g.a2_sk, g.a2_mode, row0a, g.M, k0,
+                                                   k_end, ptid, va);
+        load_tile<BN, BKE, EPC, B_MN, C::B_CHUNKS>(g.B, g.b_sn, g.b_sk, nullptr, 0, 0, ADD_NONE, row0b, g.N, k0, k_end,
+                                                   ptid, vb);
+        if (!mbar_wait(empty_bar(stage), phase ^ 1u, dead, p.status)) { alive = false; break; }
+        const uint32_t sa = smem_base + stage * C::STAGE_BYTES;
+        const uint32_t sa_lo = sa + C::A_BYTES;
+        const uint32_t sb = sa + (BF16 ? 1 : 2) * C::A_BYTES;
+        const uint32_t sb_lo = sb + C::B_BYTES;
+        store_tile<BM, BKE, EPC, A_MN, C::A_CHUNKS, BF16>(sa, sa_lo, ptid, va);
+        store_tile<BN, BKE, EPC, B_MN, C::B_CHUNKS, BF16>(sb, sb_lo, ptid, vb);
+        fence_proxy_async();
+        mbar_arrive(full_bar(stage));
+        if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+      }
+    }
+  } else {
+    // ------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      const uint32_t idesc = make_idesc(BF16, A_MN, B_MN, BN);
+      const uint32_t lbo = BKE * 128;
+      constexpr uint32_t A_KSTEP = A_MN ? (BF16 ? 2048u : 1024u) : 32u;   // bytes per UMMA K step
+      constexpr uint32_t B_KSTEP = B_MN ? (BF16 ? 2048u : 1024u) : 32u;
+      int stage = 0;
+      uint32_t phase = 0;
+      int iter = 0;
+      bool alive = true;
+      for (int item = blockIdx.x; item < p.num_items && alive; item += gridDim.x, ++iter) {
+        const Item it = decode_item<BN, BKE>(p, item);
+        const int ab = iter & 1;
+        const uint32_t aph = (uint32_t)(iter >> 1) & 1u;
+        if (!mbar_wait(acce_bar(ab), aph ^ 1u, dead, p.status)) { alive = false; break; }
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + (uint32_t)(ab * BN);
+        uint32_t accumulate = 0;
+        for (int kb = it.kb0; kb < it.kb1; ++kb) {
+          if (!mbar_wait(full_bar(stage), phase, dead, p.status)) { alive = false; break; }
+          tc_fence_after();
+          const uint32_t sa = smem_base + stage * C::STAGE_BYTES;
+          const uint32_t sa_lo = sa + C::A_BYTES;
+          const uint32_t sb = sa + (BF16 ? 1 : 2) * C::A_BYTES;
+          const uint32_t sb_lo = sb + C::B_BYTES;
+#pragma unroll
+          for (int ks = 0; ks < 4; ++ks) {
+            const uint64_t a_hi = make_desc(sa + ks * A_KSTEP, A_MN, lbo);
+            const uint64_t b_hi = make_desc(sb + ks * B_KSTEP, B_MN, lbo);
+            if (BF16) {
+              umma<true>(d_tmem, a_hi, b_hi, idesc, accumulate);
+              accumulate = 1;
+            } else {
+              const uint64_t a_lo = make_desc(sa_lo + ks * A_KSTEP, A_MN, lbo);
+              const uint64_t b_lo = make_desc(sb_lo + ks * B_KSTEP, B_MN, lbo);
+              umma<false>(d_tmem, a_hi, b_lo, idesc, accumulate);   // small terms first
+              umma<false>(d_tmem, a_lo, b_hi, idesc, 1u);
+              umma<false>(d_tmem, a_hi, b_hi, idesc, 1u);
+              accumulate = 1;
+            }
+          }
+          umma_commit(empty_bar(stage));        // the stage may be refilled once these MMAs are done
+          if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+        }
+        if (!alive) break;
+        umma_commit(accf_bar(ab));              // accumulator complete
+      }
+      // drain: every issued MMA must have finished before TMEM is released
+      umma_commit(drain_bar);
+      mbar_wait(drain_bar, 0u, dead, p.status);
+    }
+    __syncwarp();
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == NUM_EPI_WARPS + NUM_PROD_WARPS) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, C::TMEM_COLS);
+  }
+}
+
+template <int BN, bool A_MN, bool B_MN, bool BF16>
+inline cudaError_t set_smem_attr() {
+  return cudaFuncSetAttribute(k_gemm_umma<BN, A_MN, B_MN, BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              Cfg<BN, BF16>::SMEM_BYTES);
+}
+
+template <int BN, bool BF16>
+inline void launch_variant(const Params& p, bool a_mn, bool b_mn, int grid, cudaStream_t st) {
+  constexpr int smem = Cfg<BN, BF16>::SMEM_BYTES;
+  if (!a_mn && !b_mn) k_gemm_umma<BN, false, false, BF16><<<grid, NUM_THREADS, smem, st>>>(p);
+  else if (!a_mn && b_mn) k_gemm_umma<BN, false, true, BF16><<<grid, NUM_THREADS, smem, st>>>(p);
+  else if (a_mn && b_mn) k_gemm_umma<BN, true, true, BF16><<<grid, NUM_THREADS, smem, st>>>(p);
+  else k_gemm_umma<BN, true, false, BF16><<<grid, NUM_THREADS, smem, st>>>(p);
+}
+
+}  // namespace umma
+
+// One-time set-up of the tensor-core kernels: opt in to their dynamic shared memory.
+inline int umma_configure() {
+  using namespace umma;
+  cudaError_t e = cudaSuccess;
+#define DION_SET(BN, A, B, F) \
+  if (e == cudaSuccess) e = set_smem_attr<BN, A, B, F>();
+  DION_SET(128, false, false, false) DION_SET(128, false, true, false) DION_SET(128, true, true, false) DION_SET(128, true, false, false)
+  DION_SET(256, false, false, false) DION_SET(256, false, true, false) DION_SET(256, true, true, false) DION_SET(256, true, false, false)
+  DION_SET(128, false, false, true) DION_SET(128, false, true, true) DION_SET(128, true, true, true) DION_SET(128, true, false, true)
+  DION_SET(256, false, false, true) DION_SET(256, false, true, true) DION_SET(256, true, true, true) DION_SET(256, true, false, true)
+#undef DION_SET
+  if (e != cudaSuccess) { cudaGetLastError(); return DION_ERR_CUDA; }
+  return DION_OK;
+}
+
+// Launches the product on the tensor cores if it qualifies.  Returns the number of
+// kernels launched (1, or 2 with a split-K reduction), 0 if this engine does not take
+// the product, or a negative DION_ERR_* code.
+inline int umma_try_launch(const GemmArgs& g_in, int precision, int sm_count, float* part, i64 part_floats,
+                           int* status, cudaStream_t st) {
+  using namespace umma;
+  GemmArgs g = g_in;
+  const bool bf16 = (precision == DION_PREC_BF16_OPERANDS);
+  const int epc = bf16 ? 8 : 4;
+  const int bke = bf16 ? 64 : 32;
+  if (g.batch != 1 || g.alpha_dev != nullptr) return 0;
+  if (g.M < 128 || g.N < 64 || g.K < 64) return 0;
+  if ((g.M % epc) || (g.N % epc) || (g.K % epc)) return 0;
+  auto aligned = [](const void* p, size_t a) { return ((uintptr_t)p % a) == 0; };
+  bool a_mn, b_mn;
+  if (g.a_sk == 1 && g.a_si % 4 == 0) a_mn = false;
+  else if (g.a_si == 1 && g.a_sk % 4 == 0) a_mn = true;
+  else return 0;
+  if (g.b_sk == 1 && g.b_sn % 4 == 0) b_mn = false;
+  else if (g.b_sn == 1 && g.b_sk % 4 == 0) b_mn = true;
+  else return 0;
+  if (!aligned(g.A, 16) || !aligned(g.B, 16) || !aligned(g.C, 16) || (g.ldc % 4)) return 0;
+  if (g.a2_mode != ADD_NONE) {
+    if (a_mn ? (g.a2_si != 1 || g.a2_sk % 4) : (g.a2_sk != 1 || g.a2_si % 4)) return 0;
+    if (!aligned(g.A2, g.a2_mode == ADD_BF16 ? 8 : 16)) return 0;
+  }
+  if (g.epi == EPI_ADD2_SUB) {
+    if ((g.ldc2 % 4) || !aligned(g.C2, g.c2_mode == ADD_BF16 ? 8 : 16)) return 0;
+  }
+  if (g.tri == TRI_LOWER && g.M != g.N) return 0;
+
+  const int BN = (g.tri == TRI_LOWER || g.N < 256) ? 128 : 256;
+  Params p;
+  p.g = g;
+  p.nM = (int)((g.M + BM - 1) / BM);
+  p.nN = (int)((g.N + BN - 1) / BN);
+  p.nkb = (int)((g.K + bke - 1) / bke);
+  const i64 tiles = (g.tri == TRI_LOWER) ? (i64)p.nM * (p.nM + 1) / 2 : (i64)p.nM * p.nN;
+  int splits = 1;
+  if (g.epi == EPI_STORE && !g.klimit && part != nullptr && tiles < sm_count) {
+    i64 want = sm_count / tiles;
+    const i64 kmax = p.nkb / 4;                       // at least four K blocks per split
+    if (want > kmax) want = kmax;
+    if (want > 32) want = 32;
+    while (want > 1 && want * g.M * g.N > part_floats) --want;
+    if (want > 1) splits = (int)want;
+  }
+  p.kb_per_split = (p.nkb + splits - 1) / splits;
+  splits = (p.nkb + p.kb_per_split - 1) / p.kb_per_split;   // no empty split
+  p.splits = splits;
+  p.g.part = part;
+  if (tiles * splits > 0x7fffffff) return 0;
+  p.num_items = (int)(tiles * splits);
+  p.status = status;
+  const int grid = p.num_items < sm_count ? p.num_items : sm_count;
+  if (bf16) {
+    if (BN == 256) launch_variant<256, true>(p, a_mn, b_mn, grid, st);
+    else launch_variant<128, true>(p, a_mn, b_mn, grid, st);
+  } else {
+    if (BN == 256) launch_variant<256, false>(p, a_mn, b_mn, grid, st);
+    else launch_variant<128, false>(p, a_mn, b_mn, grid, st);
+  }
+  if (cudaGetLastError() != cudaSuccess) return DION_ERR_CUDA;
+  if (splits > 1) {
+    const i64 total = g.M * g.N;
+    int blocks = (int)((total + 255) / 256);
+    if (blocks > 8 * sm_count) blocks = 8 * sm_count;
+    k_splitk_reduce<<<blocks, 256, 0, st>>>(part, splits, g.M, g.N, g.C, g.ldc, g.alpha, g.tri, 128, g.skip_flag);
+    if (cudaGetLastError() != cudaSuccess) return DION_ERR_CUDA;
+    return 2;
+  }
+  return 1;
+}
 
 }  // namespace dion

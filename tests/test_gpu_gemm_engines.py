@@ -1,0 +1,148 @@
+"""The two contraction engines (fp32 FMA and tcgen05 tensor cores) in isolation.
+
+Each product C = op(A) * op(B) with its fused operand formation (M + G) and
+epilogue is run through the library's internal hook and compared with a float64
+product of the same operands.  Covers the four operand layouts (k-contiguous or
+row-contiguous A and B), ragged tails, lower-triangular output, the K limit of a
+triangular operand, split-K and bf16 gradients.  The end-to-end parity with the
+CPU oracle is in test_gpu_parity.py; this file localises a failure to an engine.
+"""
+import ctypes
+
+import pytest
+import torch
+
+from paper_2504_05295_b200 import binding, build
+
+pytestmark = pytest.mark.gpu
+
+
+class GemmArgs(ctypes.Structure):
+    _fields_ = [("M", ctypes.c_int64), ("N", ctypes.c_int64), ("K", ctypes.c_int64),
+                ("A", ctypes.c_void_p), ("a_si", ctypes.c_int64), ("a_sk", ctypes.c_int64),
+                ("A2", ctypes.c_void_p), ("a2_si", ctypes.c_int64), ("a2_sk", ctypes.c_int64), ("a2_mode", ctypes.c_int),
+                ("B", ctypes.c_void_p), ("b_sk", ctypes.c_int64), ("b_sn", ctypes.c_int64),
+                ("C", ctypes.c_void_p), ("ldc", ctypes.c_int64), ("epi", ctypes.c_int),
+                ("C2", ctypes.c_void_p), ("ldc2", ctypes.c_int64), ("c2_mode", ctypes.c_int),
+                ("alpha", ctypes.c_float), ("tri", ctypes.c_int), ("klimit", ctypes.c_int)]
+
+
+@pytest.fixture(scope="module")
+def lib():
+    build.build()
+    assert torch.cuda.is_available()
+    lib = binding.load_library()
+    lib.dion_debug_gemm.argtypes = [ctypes.c_int, ctypes.c_int, ctypes.POINTER(GemmArgs), ctypes.c_void_p,
+                                    ctypes.c_int64, ctypes.c_void_p, ctypes.c_void_p]
+    lib.dion_debug_gemm.restype = ctypes.c_int
+    return lib
+
+
+def run(lib, engine, precision, M, N, K, a_mn, b_mn, add=None, epi=0, tri=0, klimit=0, alpha=1.0, seed=0):
+    g = torch.Generator(device="cuda"); g.manual_seed(seed)
+    rn = lambda *s: torch.randn(*s, generator=g, device="cuda")
+    # A(i,k): stored M x K (k contiguous) or K x M (row index contiguous)
+    A_store = rn(K, M) if a_mn else rn(M, K)
+    A_log = A_store.t() if a_mn else A_store
+    A2_store = None
+    if add is not None:
+        A2_store = (rn(K, M) if a_mn else rn(M, K)).to(add)
+        A_eff = A_log.double() + (A2_store.t() if a_mn else A2_store).double()
+    else:
+        A_eff = A_log.double()
+    # B(k,j): stored K x N (n contiguous) or N x K (k contiguous)
+    B_store = rn(K, N) if b_mn else rn(N, K)
+    B_log = B_store if b_mn else B_store.t()
+    if klimit:
+        B_log = torch.triu(B_log)       # B(k,j) = 0 for k > j
+        if b_mn:
+            B_store = B_log.contiguous()
+        else:
+            B_store = B_log.t().contiguous()
+    C = rn(M, N)
+    C0 = C.clone()
+    C2 = rn(M, N).to(add if add is not None else torch.float32)
+    ref = A_eff @ B_log.double()
+    if epi == 0:
+        want = alpha * ref
+    elif epi == 1:
+        want = C0.double() - alpha * ref
+    else:
+        want = C0.double() + C2.double() - alpha * ref
+    a = GemmArgs()
+    a.M, a.N, a.K = M, N, K
+    a.A = A_store.data_ptr(); a.a_si, a.a_sk = (1, M) if a_mn else (K, 1)
+    if add is not None:
+        a.A2 = A2_store.data_ptr(); a.a2_si, a.a2_sk = (1, M) if a_mn else (K, 1)
+        a.a2_mode = 1 if add == torch.float32 else 2
+    a.B = B_store.data_ptr(); a.b_sk, a.b_sn = (N, 1) if b_mn else (1, K)
+    a.C = C.data_ptr(); a.ldc = N; a.epi = epi
+    a.C2 = C2.data_ptr(); a.ldc2 = N; a.c2_mode = 1 if C2.dtype == torch.float32 else 2
+    a.alpha = alpha; a.tri = tri; a.klimit = klimit
+    part = torch.empty(8 << 20, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    rc = lib.dion_debug_gemm(engine, precision, ctypes.byref(a), part.data_ptr(), part.numel(), status.data_ptr(),
+                             int(torch.cuda.current_stream().cuda_stream))
+    torch.cuda.synchronize()
+    assert rc == 0, f"dion_debug_gemm returned {rc}"
+    assert int(status.item()) == 0, f"device status {int(status.item())}"
+    got = C.double()
+    if tri:
+        # only the elements on or below the diagonal are guaranteed to be written
+        idx = torch.arange(M, device="cuda")
+        mask = idx[None, :] <= idx[:, None]
+        got, want = got[mask], want[mask]
+    err = (got - want).norm() / want.norm()
+    return float(err)
+
+
+LAYOUTS = [(False, False), (False, True), (True, True), (True, False)]
+
+
+@pytest.mark.parametrize("engine", [1, 2])
+@pytest.mark.parametrize("a_mn,b_mn", LAYOUTS)
+def test_layouts_fp32(lib, engine, a_mn, b_mn):
+    err = run(lib, engine, 0, 512, 512, 1024, a_mn, b_mn)
+    assert err < 2e-6, err
+
+
+@pytest.mark.parametrize("engine", [1, 2])
+@pytest.mark.parametrize("M,N,K", [(128, 64, 64), (132, 260, 100), (640, 384, 96), (1028, 132, 2052), (256, 1024, 68)])
+def test_ragged_shapes(lib, engine, M, N, K):
+    for a_mn, b_mn in LAYOUTS:
+        err = run(lib, engine, 0, M, N, K, a_mn, b_mn, seed=M + N)
+        assert err < 2e-6, (a_mn, b_mn, err)
+
+
+@pytest.mark.parametrize("engine", [1, 2])
+@pytest.mark.parametrize("add", [torch.float32, torch.bfloat16])
+def test_fused_add_and_epilogues(lib, engine, add):
+    # P = (M + G) Q ; R = (M + G)^T U ; M <- M + G - beta U R^T ; X <- X - s U Q^T
+    assert run(lib, engine, 0, 1024, 256, 768, False, True, add=add) < 2e-6
+    assert run(lib, engine, 0, 768, 256, 1024, True, True, add=add) < 2e-6
+    assert run(lib, engine, 0, 1024, 768, 256, False, False, add=add, epi=2, alpha=0.05) < 2e-6
+    assert run(lib, engine, 0, 1024, 768, 256, False, False, epi=1, alpha=0.01) < 2e-6
+
+
+@pytest.mark.parametrize("engine", [1, 2])
+def test_gram_lower_triangle_and_split_k(lib, engine):
+    # Gram matrix P^T P: both operands row-contiguous, only lower tiles, long K -> split-K
+    assert run(lib, engine, 0, 512, 512, 8192, True, True, tri=1) < 3e-6
+    assert run(lib, engine, 0, 256, 256, 4096, True, True, tri=1) < 3e-6
+    # tall-skinny product with few tiles -> split-K
+    assert run(lib, engine, 0, 2048, 128, 2048, False, True) < 3e-6
+
+
+@pytest.mark.parametrize("engine", [1, 2])
+def test_triangular_operand_k_limit(lib, engine):
+    # U = P Linv^T with Linv lower triangular: B(k,j) = Linv[j][k] = 0 for k > j
+    assert run(lib, engine, 0, 2048, 512, 512, False, False, klimit=1) < 2e-6
+    assert run(lib, engine, 0, 1024, 768, 768, False, False, klimit=1) < 2e-6
+
+
+@pytest.mark.parametrize("a_mn,b_mn", LAYOUTS)
+def test_bf16_operand_mode(lib, a_mn, b_mn):
+    err = run(lib, 2, 1, 512, 512, 1024, a_mn, b_mn)
+    assert err < 6e-3, err
+    err = run(lib, 2, 1, 648, 392, 328, a_mn, b_mn, seed=5)
+    assert err < 6e-3, err
