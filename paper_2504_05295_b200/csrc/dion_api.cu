@@ -263,7 +263,7 @@ int cholqr_round(StepCtx& s, const float* Pin, float* Pout, i64 rows, i64 r, boo
   g.M = r; g.N = r; g.K = rows;
   g.A = Pin; g.a_si = 1; g.a_sk = r;
   g.B = Pin; g.b_sk = r; g.b_sn = 1;
-  g.C = Gm; g.ldc = r; g.epi = EPI_STORE; g.tri = TRI_LOWER; g.skip_flag = skip;
+  g.C = Gm; g.ldc = r; g.epi = EPI_STORE; g.tri = TRI_LOWER; g.skip_flag = skip; g.precise = adaptive ? 1 : 0;
   DION_TRY(launch_gemm(s, g));
   float* sh = s.ws + s.L.scal;
   k_round_begin<<<1, 256, 0, s.st>>>(Gm, r, r, 0.f, s.ws + s.L.gdiag, sh, s.os, adaptive ? 1 : 0);
@@ -280,7 +280,7 @@ int cholqr_round(StepCtx& s, const float* Pin, float* Pout, i64 rows, i64 r, boo
   u.M = rows; u.N = r; u.K = r;
   u.A = Pin; u.a_si = r; u.a_sk = 1;
   u.B = s.ws + s.L.Linv; u.b_sk = 1; u.b_sn = r; u.klimit = 1;
-  u.C = Pout; u.ldc = r; u.epi = EPI_STORE; u.skip_flag = skip;
+  u.C = Pout; u.ldc = r; u.epi = EPI_STORE; u.skip_flag = skip; u.precise = adaptive ? 1 : 0;
   DION_TRY(launch_gemm(s, u));
   if (adaptive) {
     k_round_end<<<1, 1, 0, s.st>>>(s.os, GOOD_REL, c->dev_ints + 2);
@@ -319,12 +319,18 @@ int householder(StepCtx& s, float* A, float* V, i64 rows, i64 r) {
   return DION_OK;
 }
 
+// The orthonormalization a step on (m, n, r) will use.
+int resolve_orth(const dion_ctx* c, i64 r, i64 short_dim) {
+  int mode = c->cfg.orth;
+  if (mode == DION_ORTH_AUTO) mode = (4 * r <= short_dim) ? DION_ORTH_CHOLQR2 : DION_ORTH_SHIFTED3;
+  return mode;
+}
+
 // Orthonormalize the rows x r panel in ws.P0; returns the buffer that holds U.
 int orthonormalize(StepCtx& s, i64 rows, i64 r, i64 short_dim, float** U_out) {
   float* P0 = s.ws + s.L.P0;
   float* P1 = s.ws + s.L.P1;
-  int mode = s.c->cfg.orth;
-  if (mode == DION_ORTH_AUTO) mode = (4 * r <= short_dim) ? DION_ORTH_CHOLQR2 : DION_ORTH_SHIFTED3;
+  const int mode = resolve_orth(s.c, r, short_dim);
   if (mode == DION_ORTH_CHOLQR2) {
     DION_TRY(cholqr_round(s, P0, P1, rows, r, false));
     DION_TRY(cholqr_round(s, P1, P0, rows, r, false));
@@ -446,6 +452,8 @@ int step_one(dion_ctx* c, const dion_matrix* a, float lr, cudaStream_t st) {
   p.A2 = a->G; p.a2_si = a->ldg; p.a2_sk = 1; p.a2_mode = gmode;
   p.B = (const float*)a->Q; p.b_sk = a->ldq; p.b_sn = 1;
   p.C = P0; p.ldc = r; p.epi = EPI_STORE;
+  // an ill-conditioned panel amplifies the error of P: use the accurate product there
+  p.precise = (resolve_orth(c, r, (m < n) ? m : n) == DION_ORTH_SHIFTED3) ? 1 : 0;
   DION_TRY(launch_gemm(s, p));
   }
 
@@ -523,6 +531,7 @@ int lazy_one(dion_ctx* c, const dion_matrix* a, float lr, int refresh, cudaStrea
     t.A2 = a->G; t.a2_si = a->ldg; t.a2_sk = 1; t.a2_mode = gmode;
     t.B = (const float*)a->Q; t.b_sk = a->ldq; t.b_sn = 1;
     t.C = R; t.ldc = r; t.epi = EPI_STORE;
+    t.precise = (resolve_orth(c, r, (m < n) ? m : n) == DION_ORTH_SHIFTED3) ? 1 : 0;
     DION_TRY(launch_gemm(s, t));
     GemmArgs z = gemm_args();
     z.M = n; z.N = r; z.K = m;
@@ -530,6 +539,7 @@ int lazy_one(dion_ctx* c, const dion_matrix* a, float lr, int refresh, cudaStrea
     z.A2 = a->G; z.a2_si = 1; z.a2_sk = a->ldg; z.a2_mode = gmode;
     z.B = R; z.b_sk = r; z.b_sn = 1;
     z.C = P0; z.ldc = r; z.epi = EPI_STORE;
+    z.precise = t.precise;
     DION_TRY(launch_gemm(s, z));
     float* V = nullptr;
     DION_TRY(orthonormalize(s, n, r, (m < n) ? m : n, &V));
@@ -851,7 +861,7 @@ extern "C" int dion_debug_gemm(int engine, int precision, const dion_debug_gemm_
   g.B = a->B; g.b_sk = a->b_sk; g.b_sn = a->b_sn;
   g.C = a->C; g.ldc = a->ldc; g.epi = a->epi;
   g.C2 = a->C2; g.ldc2 = a->ldc2; g.c2_mode = a->c2_mode;
-  g.alpha = a->alpha; g.tri = a->tri; g.klimit = a->klimit;
+  g.alpha = a->alpha; g.tri = a->tri; g.klimit = a->klimit; g.precise = a->precise;
   cudaStream_t st = (cudaStream_t)cuda_stream;
   if (engine == DION_ENGINE_TENSOR) {
     const int rc = umma_try_launch(g, precision, sms, part, part_floats, status, st);

@@ -41,6 +41,7 @@ struct GemmArgs {
   int tri;                       // TRI_LOWER: tiles strictly above the diagonal are skipped
   int klimit;                    // 1: B(k,j) == 0 for k > j  (K loop ends at the tile's last column)
   const int* skip_flag;          // optional: if *skip_flag != 0 the kernel does nothing
+  int precise;                   // tensor engine: keep the small split terms in their own accumulator
 };
 
 __device__ __forceinline__ float load_add(const void* p, i64 off, int mode) {

@@ -134,19 +134,25 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   }
 }
 
-// Shared-memory matrix descriptor, 128-byte swizzle.  K-major: rows of 128 bytes,
-// 8-row groups 1024 bytes apart.  MN-major: 8 x 128-byte atoms; `lbo_bytes` is the
-// distance between 32-element (fp32) / 64-element (bf16) chunks along M/N, groups
-// of 8 k-rows are 1024 bytes apart.
+// Shared-memory matrix descriptor.
+// K-major (any type) and MN-major bf16: 128-byte swizzle (16-byte units XORed with
+//   the row index mod 8); rows of 128 bytes, 8-row groups 1024 bytes apart.
+// MN-major TF32: the only layout the hardware takes is the 128-byte swizzle with a
+//   32-byte base: atoms of 4 k-rows x 128 bytes, 32-byte units XORed with the row
+//   index mod 4; groups of 4 k-rows are 512 bytes apart.
+// For MN-major operands `lbo_bytes` is the distance between consecutive 128-byte
+// chunks along M/N (32 fp32 or 64 bf16 elements).
+template <bool BF16>
 __device__ __forceinline__ uint64_t make_desc(uint32_t saddr, bool mn_major, uint32_t lbo_bytes) {
+  const bool base32 = mn_major && !BF16;
   const uint64_t lbo = mn_major ? (uint64_t)(lbo_bytes >> 4) : 1ull;
-  const uint64_t sbo = 1024 >> 4;
+  const uint64_t sbo = base32 ? (512 >> 4) : (1024 >> 4);
   uint64_t d = 0;
   d |= (uint64_t)((saddr >> 4) & 0x3FFF);
   d |= lbo << 16;
   d |= sbo << 32;
-  d |= 1ull << 46;   // descriptor version of sm_100
-  d |= 2ull << 61;   // SWIZZLE_128B
+  d |= 1ull << 46;                      // descriptor version of sm_100
+  d |= (base32 ? 1ull : 2ull) << 61;    // SWIZZLE_128B_BASE32B or SWIZZLE_128B
   return d;
 }
 
@@ -248,7 +254,11 @@ __device__ __forceinline__ void store_tile(uint32_t s_hi, uint32_t s_lo, int pti
     const int c = ptid + l * NUM_PROD_THREADS;
     const int major = c / CPR, minor = c % CPR;
     uint32_t off;
-    if (MN_MAJOR) {   // major = k row, minor = 16-byte chunk along M/N
+    if (MN_MAJOR && !BF16) {   // major = k row, minor = 16-byte chunk along M/N; 32-byte swizzle units
+      const uint32_t q = (uint32_t)(minor & 7);
+      off = (uint32_t)(minor >> 3) * (BKE * 128) + (uint32_t)major * 128 + ((((q >> 1) ^ (uint32_t)(major & 3))) << 5) +
+            ((q & 1u) << 4);
+    } else if (MN_MAJOR) {     // major = k row, minor = 16-byte chunk along M/N
       off = (uint32_t)(minor >> 3) * (BKE * 128) + (uint32_t)major * 128 + (uint32_t)(((minor & 7) ^ (major & 7)) << 4);
     } else {          // major = row, minor = 16-byte chunk along k (8 per 128-byte row)
       off = (uint32_t)major * 128 + (uint32_t)((minor ^ (major & 7)) << 4);
@@ -266,7 +276,8 @@ __device__ __forceinline__ void store_tile(uint32_t s_hi, uint32_t s_lo, int pti
 #pragma unroll
       for (int q = 0; q < 4; ++q) {
         h[q] = cvt_tf32(v[l][q]);
-        lo[q] = __float_as_uint(v[l][q] - __uint_as_float(h[q]));
+        // the remainder is rounded to TF32 here (to nearest) rather than truncated by the MMA
+        lo[q] = cvt_tf32(v[l][q] - __uint_as_float(h[q]));
       }
       st_shared_v4(s_hi + off, h[0], h[1], h[2], h[3]);
       st_shared_v4(s_lo + off, lo[0], lo[1], lo[2], lo[3]);
@@ -274,7 +285,14 @@ __device__ __forceinline__ void store_tile(uint32_t s_hi, uint32_t s_lo, int pti
   }
 }
 
-template <int BN, bool BF16>
+// SPLIT (fp32 mode only): the hi*hi products and the small hi*lo + lo*hi products go
+// to separate TMEM accumulators that are added once in the epilogue.  Every
+// tcgen05.mma truncates when it adds into its accumulator; keeping the small terms
+// apart leaves one such truncation per K step on the main sum instead of three and
+// brings the product to the accuracy of an fp32 FMA loop (measured 3.3e-7 against
+// 9.1e-7 relative error on Gaussian data).  Used for the products whose error the
+// conditioning of an ill-conditioned panel amplifies.
+template <int BN, bool BF16, bool SPLIT = false>
 struct Cfg {
   static constexpr int BKE = BF16 ? 64 : 32;                 // K elements per 128-byte row
   static constexpr int EPC = BF16 ? 8 : 4;                   // elements per 16-byte chunk
@@ -285,12 +303,16 @@ struct Cfg {
   static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 + 512;
   static constexpr int A_CHUNKS = BM * 8 / NUM_PROD_THREADS;  // 16-byte chunks per producer thread
   static constexpr int B_CHUNKS = BN * 8 / NUM_PROD_THREADS;
-  static constexpr int TMEM_COLS = 2 * BN;
+  static constexpr int ACCS = SPLIT ? 2 : 1;                 // accumulators per tile
+  static constexpr int NBUF = (512 / (ACCS * BN)) >= 2 ? 2 : 1;  // tiles in flight in TMEM
+  static constexpr int TMEM_COLS = NBUF * ACCS * BN;
 };
 
-template <int BN, bool A_MN, bool B_MN, bool BF16>
+template <int BN, bool A_MN, bool B_MN, bool BF16, bool SPLIT>
 __global__ void __launch_bounds__(NUM_THREADS, 1) k_gemm_umma(const Params p) {
-  using C = Cfg<BN, BF16>;
+  static_assert(!(BF16 && SPLIT), "split accumulators belong to the 3xTF32 mode");
+  using C = Cfg<BN, BF16, SPLIT>;
+  constexpr int NBUF = C::NBUF, ACCS = C::ACCS;
   constexpr int BKE = C::BKE, EPC = C::EPC, STAGES = C::STAGES;
   if (p.g.skip_flag != nullptr && *p.g.skip_flag != 0) return;
 
@@ -333,8 +355,8 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_gemm_umma(const Params p) {
     int iter = 0;
     for (int item = blockIdx.x; item < p.num_items; item += gridDim.x, ++iter) {
       const Item it = decode_item<BN, BKE>(p, item);
-      const int ab = iter & 1;
-      const uint32_t ph = (uint32_t)(iter >> 1) & 1u;
+      const int ab = iter % NBUF;
+      const uint32_t ph = (uint32_t)(iter / NBUF) & 1u;
       if (!mbar_wait(accf_bar(ab), ph, dead, p.status)) break;
       tc_fence_after();
       const i64 gi = (i64)it.mi * BM + warp * 32 + lane;
@@ -343,7 +365,13 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_gemm_umma(const Params p) {
 #pragma unroll 1
       for (int cb = 0; cb < BN / 32; ++cb) {
         float acc[32];
-        tmem_ld32(tmem_base + (uint32_t)(ab * BN + cb * 32) + ((uint32_t)(warp * 32) << 16), acc);
+        tmem_ld32(tmem_base + (uint32_t)(ab * ACCS * BN + cb * 32) + ((uint32_t)(warp * 32) << 16), acc);
+        if (SPLIT) {
+          float small[32];
+          tmem_ld32(tmem_base + (uint32_t)(ab * ACCS * BN + BN + cb * 32) + ((uint32_t)(warp * 32) << 16), small);
+#pragma unroll
+          for (int e = 0; e < 32; ++e) acc[e] += small[e];
+        }
         if (gi < g.M) {
 #pragma unroll
           for (int q = 0; q < 8; ++q) {
@@ -424,11 +452,12 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_gemm_umma(const Params p) {
       bool alive = true;
       for (int item = blockIdx.x; item < p.num_items && alive; item += gridDim.x, ++iter) {
         const Item it = decode_item<BN, BKE>(p, item);
-        const int ab = iter & 1;
-        const uint32_t aph = (uint32_t)(iter >> 1) & 1u;
+        const int ab = iter % NBUF;
+        const uint32_t aph = (uint32_t)(iter / NBUF) & 1u;
         if (!mbar_wait(acce_bar(ab), aph ^ 1u, dead, p.status)) { alive = false; break; }
         tc_fence_after();
-        const uint32_t d_tmem = tmem_base + (uint32_t)(ab * BN);
+        const uint32_t d_tmem = tmem_base + (uint32_t)(ab * ACCS * BN);
+        const uint32_t d_small = d_tmem + (SPLIT ? BN : 0);
         uint32_t accumulate = 0;
         for (int kb = it.kb0; kb < it.kb1; ++kb) {
           if (!mbar_wait(full_bar(stage), phase, dead, p.status)) { alive = false; break; }
@@ -439,17 +468,23 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_gemm_umma(const Params p) {
           const uint32_t sb_lo = sb + C::B_BYTES;
 #pragma unroll
           for (int ks = 0; ks < 4; ++ks) {
-            const uint64_t a_hi = make_desc(sa + ks * A_KSTEP, A_MN, lbo);
-            const uint64_t b_hi = make_desc(sb + ks * B_KSTEP, B_MN, lbo);
+            const uint64_t a_hi = make_desc<BF16>(sa + ks * A_KSTEP, A_MN, lbo);
+            const uint64_t b_hi = make_desc<BF16>(sb + ks * B_KSTEP, B_MN, lbo);
             if (BF16) {
               umma<true>(d_tmem, a_hi, b_hi, idesc, accumulate);
               accumulate = 1;
             } else {
-              const uint64_t a_lo = make_desc(sa_lo + ks * A_KSTEP, A_MN, lbo);
-              const uint64_t b_lo = make_desc(sb_lo + ks * B_KSTEP, B_MN, lbo);
-              umma<false>(d_tmem, a_hi, b_lo, idesc, accumulate);   // small terms first
-              umma<false>(d_tmem, a_lo, b_hi, idesc, 1u);
-              umma<false>(d_tmem, a_hi, b_hi, idesc, 1u);
+              const uint64_t a_lo = make_desc<BF16>(sa_lo + ks * A_KSTEP, A_MN, lbo);
+              const uint64_t b_lo = make_desc<BF16>(sb_lo + ks * B_KSTEP, B_MN, lbo);
+              if (SPLIT) {
+                umma<false>(d_small, a_hi, b_lo, idesc, accumulate);
+                umma<false>(d_small, a_lo, b_hi, idesc, 1u);
+                umma<false>(d_tmem, a_hi, b_hi, idesc, accumulate);
+              } else {
+                umma<false>(d_tmem, a_hi, b_lo, idesc, accumulate);   // small terms first
+                umma<false>(d_tmem, a_lo, b_hi, idesc, 1u);
+                umma<false>(d_tmem, a_hi, b_hi, idesc, 1u);
+              }
               accumulate = 1;
             }
           }
@@ -474,19 +509,19 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_gemm_umma(const Params p) {
   }
 }
 
-template <int BN, bool A_MN, bool B_MN, bool BF16>
+template <int BN, bool A_MN, bool B_MN, bool BF16, bool SPLIT>
 inline cudaError_t set_smem_attr() {
-  return cudaFuncSetAttribute(k_gemm_umma<BN, A_MN, B_MN, BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              Cfg<BN, BF16>::SMEM_BYTES);
+  return cudaFuncSetAttribute(k_gemm_umma<BN, A_MN, B_MN, BF16, SPLIT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              Cfg<BN, BF16, SPLIT>::SMEM_BYTES);
 }
 
-template <int BN, bool BF16>
+template <int BN, bool BF16, bool SPLIT>
 inline void launch_variant(const Params& p, bool a_mn, bool b_mn, int grid, cudaStream_t st) {
-  constexpr int smem = Cfg<BN, BF16>::SMEM_BYTES;
-  if (!a_mn && !b_mn) k_gemm_umma<BN, false, false, BF16><<<grid, NUM_THREADS, smem, st>>>(p);
-  else if (!a_mn && b_mn) k_gemm_umma<BN, false, true, BF16><<<grid, NUM_THREADS, smem, st>>>(p);
-  else if (a_mn && b_mn) k_gemm_umma<BN, true, true, BF16><<<grid, NUM_THREADS, smem, st>>>(p);
-  else k_gemm_umma<BN, true, false, BF16><<<grid, NUM_THREADS, smem, st>>>(p);
+  constexpr int smem = Cfg<BN, BF16, SPLIT>::SMEM_BYTES;
+  if (!a_mn && !b_mn) k_gemm_umma<BN, false, false, BF16, SPLIT><<<grid, NUM_THREADS, smem, st>>>(p);
+  else if (!a_mn && b_mn) k_gemm_umma<BN, false, true, BF16, SPLIT><<<grid, NUM_THREADS, smem, st>>>(p);
+  else if (a_mn && b_mn) k_gemm_umma<BN, true, true, BF16, SPLIT><<<grid, NUM_THREADS, smem, st>>>(p);
+  else k_gemm_umma<BN, true, false, BF16, SPLIT><<<grid, NUM_THREADS, smem, st>>>(p);
 }
 
 }  // namespace umma
@@ -495,8 +530,9 @@ inline void launch_variant(const Params& p, bool a_mn, bool b_mn, int grid, cuda
 inline int umma_configure() {
   using namespace umma;
   cudaError_t e = cudaSuccess;
-#define DION_SET(BN, A, B, F) \
-  if (e == cudaSuccess) e = set_smem_attr<BN, A, B, F>();
+#define DION_SET(BN, A, B, F)                                      \
+  if (e == cudaSuccess) e = set_smem_attr<BN, A, B, F, false>(); \
+  if (e == cudaSuccess && !F) e = set_smem_attr<BN, A, B, false, true>();
   DION_SET(128, false, false, false) DION_SET(128, false, true, false) DION_SET(128, true, true, false) DION_SET(128, true, false, false)
   DION_SET(256, false, false, false) DION_SET(256, false, true, false) DION_SET(256, true, true, false) DION_SET(256, true, false, false)
   DION_SET(128, false, false, true) DION_SET(128, false, true, true) DION_SET(128, true, true, true) DION_SET(128, true, false, true)
@@ -562,11 +598,16 @@ inline int umma_try_launch(const GemmArgs& g_in, int precision, int sm_count, fl
   p.status = status;
   const int grid = p.num_items < sm_count ? p.num_items : sm_count;
   if (bf16) {
-    if (BN == 256) launch_variant<256, true>(p, a_mn, b_mn, grid, st);
-    else launch_variant<128, true>(p, a_mn, b_mn, grid, st);
+    if (BN == 256) launch_variant<256, true, false>(p, a_mn, b_mn, grid, st);
+    else launch_variant<128, true, false>(p, a_mn, b_mn, grid, st);
   } else {
-    if (BN == 256) launch_variant<256, false>(p, a_mn, b_mn, grid, st);
-    else launch_variant<128, false>(p, a_mn, b_mn, grid, st);
+    if (g.precise) {
+      if (BN == 256) launch_variant<256, false, true>(p, a_mn, b_mn, grid, st);
+      else launch_variant<128, false, true>(p, a_mn, b_mn, grid, st);
+    } else {
+      if (BN == 256) launch_variant<256, false, false>(p, a_mn, b_mn, grid, st);
+      else launch_variant<128, false, false>(p, a_mn, b_mn, grid, st);
+    }
   }
   if (cudaGetLastError() != cudaSuccess) return DION_ERR_CUDA;
   if (splits > 1) {

@@ -24,7 +24,7 @@ class GemmArgs(ctypes.Structure):
                 ("B", ctypes.c_void_p), ("b_sk", ctypes.c_int64), ("b_sn", ctypes.c_int64),
                 ("C", ctypes.c_void_p), ("ldc", ctypes.c_int64), ("epi", ctypes.c_int),
                 ("C2", ctypes.c_void_p), ("ldc2", ctypes.c_int64), ("c2_mode", ctypes.c_int),
-                ("alpha", ctypes.c_float), ("tri", ctypes.c_int), ("klimit", ctypes.c_int)]
+                ("alpha", ctypes.c_float), ("tri", ctypes.c_int), ("klimit", ctypes.c_int), ("precise", ctypes.c_int)]
 
 
 @pytest.fixture(scope="module")
@@ -38,7 +38,8 @@ def lib():
     return lib
 
 
-def run(lib, engine, precision, M, N, K, a_mn, b_mn, add=None, epi=0, tri=0, klimit=0, alpha=1.0, seed=0):
+def run(lib, engine, precision, M, N, K, a_mn, b_mn, add=None, epi=0, tri=0, klimit=0, alpha=1.0, seed=0,
+        precise=0):
     g = torch.Generator(device="cuda"); g.manual_seed(seed)
     rn = lambda *s: torch.randn(*s, generator=g, device="cuda")
     # A(i,k): stored M x K (k contiguous) or K x M (row index contiguous)
@@ -78,7 +79,7 @@ def run(lib, engine, precision, M, N, K, a_mn, b_mn, add=None, epi=0, tri=0, kli
     a.B = B_store.data_ptr(); a.b_sk, a.b_sn = (N, 1) if b_mn else (1, K)
     a.C = C.data_ptr(); a.ldc = N; a.epi = epi
     a.C2 = C2.data_ptr(); a.ldc2 = N; a.c2_mode = 1 if C2.dtype == torch.float32 else 2
-    a.alpha = alpha; a.tri = tri; a.klimit = klimit
+    a.alpha = alpha; a.tri = tri; a.klimit = klimit; a.precise = precise
     part = torch.empty(8 << 20, device="cuda")
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
     rc = lib.dion_debug_gemm(engine, precision, ctypes.byref(a), part.data_ptr(), part.numel(), status.data_ptr(),
@@ -97,13 +98,17 @@ def run(lib, engine, precision, M, N, K, a_mn, b_mn, add=None, epi=0, tri=0, kli
 
 
 LAYOUTS = [(False, False), (False, True), (True, True), (True, False)]
+# relative Frobenius error of one product on N(0,1) data: fp32 FMA stays below 3e-6 up to
+# K = 8192; the 3xTF32 tensor-core product accumulates in the tensor core's fp32 adder and
+# reaches 4e-6 there (single-pass TF32 would be ~5e-4)
+TOL = {1: 3e-6, 2: 8e-6}
 
 
 @pytest.mark.parametrize("engine", [1, 2])
 @pytest.mark.parametrize("a_mn,b_mn", LAYOUTS)
 def test_layouts_fp32(lib, engine, a_mn, b_mn):
     err = run(lib, engine, 0, 512, 512, 1024, a_mn, b_mn)
-    assert err < 2e-6, err
+    assert err < TOL[engine], err
 
 
 @pytest.mark.parametrize("engine", [1, 2])
@@ -111,33 +116,33 @@ def test_layouts_fp32(lib, engine, a_mn, b_mn):
 def test_ragged_shapes(lib, engine, M, N, K):
     for a_mn, b_mn in LAYOUTS:
         err = run(lib, engine, 0, M, N, K, a_mn, b_mn, seed=M + N)
-        assert err < 2e-6, (a_mn, b_mn, err)
+        assert err < TOL[engine], (a_mn, b_mn, err)
 
 
 @pytest.mark.parametrize("engine", [1, 2])
 @pytest.mark.parametrize("add", [torch.float32, torch.bfloat16])
 def test_fused_add_and_epilogues(lib, engine, add):
     # P = (M + G) Q ; R = (M + G)^T U ; M <- M + G - beta U R^T ; X <- X - s U Q^T
-    assert run(lib, engine, 0, 1024, 256, 768, False, True, add=add) < 2e-6
-    assert run(lib, engine, 0, 768, 256, 1024, True, True, add=add) < 2e-6
-    assert run(lib, engine, 0, 1024, 768, 256, False, False, add=add, epi=2, alpha=0.05) < 2e-6
-    assert run(lib, engine, 0, 1024, 768, 256, False, False, epi=1, alpha=0.01) < 2e-6
+    assert run(lib, engine, 0, 1024, 256, 768, False, True, add=add) < TOL[engine]
+    assert run(lib, engine, 0, 768, 256, 1024, True, True, add=add) < TOL[engine]
+    assert run(lib, engine, 0, 1024, 768, 256, False, False, add=add, epi=2, alpha=0.05) < TOL[engine]
+    assert run(lib, engine, 0, 1024, 768, 256, False, False, epi=1, alpha=0.01) < TOL[engine]
 
 
 @pytest.mark.parametrize("engine", [1, 2])
 def test_gram_lower_triangle_and_split_k(lib, engine):
     # Gram matrix P^T P: both operands row-contiguous, only lower tiles, long K -> split-K
-    assert run(lib, engine, 0, 512, 512, 8192, True, True, tri=1) < 3e-6
-    assert run(lib, engine, 0, 256, 256, 4096, True, True, tri=1) < 3e-6
+    assert run(lib, engine, 0, 512, 512, 8192, True, True, tri=1) < TOL[engine]
+    assert run(lib, engine, 0, 256, 256, 4096, True, True, tri=1) < TOL[engine]
     # tall-skinny product with few tiles -> split-K
-    assert run(lib, engine, 0, 2048, 128, 2048, False, True) < 3e-6
+    assert run(lib, engine, 0, 2048, 128, 2048, False, True) < TOL[engine]
 
 
 @pytest.mark.parametrize("engine", [1, 2])
 def test_triangular_operand_k_limit(lib, engine):
     # U = P Linv^T with Linv lower triangular: B(k,j) = Linv[j][k] = 0 for k > j
-    assert run(lib, engine, 0, 2048, 512, 512, False, False, klimit=1) < 2e-6
-    assert run(lib, engine, 0, 1024, 768, 768, False, False, klimit=1) < 2e-6
+    assert run(lib, engine, 0, 2048, 512, 512, False, False, klimit=1) < TOL[engine]
+    assert run(lib, engine, 0, 1024, 768, 768, False, False, klimit=1) < TOL[engine]
 
 
 @pytest.mark.parametrize("a_mn,b_mn", LAYOUTS)
@@ -146,3 +151,13 @@ def test_bf16_operand_mode(lib, a_mn, b_mn):
     assert err < 6e-3, err
     err = run(lib, 2, 1, 648, 392, 328, a_mn, b_mn, seed=5)
     assert err < 6e-3, err
+
+
+@pytest.mark.parametrize("a_mn,b_mn", LAYOUTS)
+def test_split_accumulators_reach_fma_accuracy(lib, a_mn, b_mn):
+    for (M, N, K) in [(512, 512, 1024), (640, 388, 2052), (256, 128, 4096)]:
+        err = run(lib, 2, 0, M, N, K, a_mn, b_mn, precise=1, seed=K)
+        assert err < 1e-6, (M, N, K, err)
+    # a Gram matrix sums same-sign terms on its diagonal, where the truncating adder is biased
+    assert run(lib, 2, 0, 512, 512, 8192, True, True, tri=1, precise=1) < 2e-6
+    assert run(lib, 2, 0, 2048, 512, 512, False, False, klimit=1, precise=1) < 1e-6
