@@ -179,9 +179,63 @@ int launch_gemm(StepCtx& s, const GemmArgs& g, bool force64 = false) {
   return launch_gemm_simt(s.c, g, s.st, s.ws + s.L.part, s.L.part_floats, force64);
 }
 
-// Blocked right-looking Cholesky of the r x r matrix Gm (lower), diagonal-block
-// inverses into Dinv, then the full inverse of the factor into Linv.
-int potrf_trtri(StepCtx& s, float* Gm, i64 r, const float* shift, bool adaptive) {
+constexpr i64 NBO = 512;  // outer block of the two-level Cholesky
+
+int grid_for(const dion_ctx* c, i64 total) {
+  i64 blocks = (total + 255) / 256;
+  if (blocks > 8 * (i64)c->sm_count) blocks = 8 * (i64)c->sm_count;
+  if (blocks < 1) blocks = 1;
+  return (int)blocks;
+}
+
+// Inverse of a lower-triangular matrix by doubling, on the diagonal square [o, o+sz):
+// [[L11,0],[L21,L22]]^-1 = [[X11,0],[-X22 L21 X11, X22]], for block sizes b_from, 2 b_from, ...
+// while b < sz.  The diagonal blocks of size b_from of Linv must already hold their inverses.
+int trtri_levels(StepCtx& s, const float* Gm, float* Linv, float* Tbuf, i64 r, i64 o, i64 sz, i64 b_from,
+                 const int* skip, int precise) {
+  for (i64 b = b_from; b < sz; b *= 2) {
+    const i64 nfull = sz / (2 * b);
+    const i64 tail0 = nfull * 2 * b;
+    const i64 b2_tail = (sz - tail0 > b) ? (sz - tail0 - b) : 0;
+    for (int pass = 0; pass < 2; ++pass) {
+      const i64 base = o + ((pass == 0) ? 0 : tail0);
+      const i64 rows = (pass == 0) ? b : b2_tail;
+      const int batch = (pass == 0) ? (int)nfull : 1;
+      if (rows <= 0 || batch <= 0) continue;
+      const i64 off21 = (base + b) * r + base, off11 = base * r + base, off22 = (base + b) * r + (base + b);
+      const i64 bs = 2 * b * (r + 1);
+      const bool big = b >= NBO;   // large blocks: one launch per pair, tensor cores where they qualify
+      const int launches = big ? batch : 1;
+      for (int q = 0; q < launches; ++q) {
+        const i64 sh = big ? (i64)q * bs : 0;
+        GemmArgs g1 = gemm_args();  // T = L21 * X11
+        g1.M = rows; g1.N = b; g1.K = b;
+        g1.A = Gm + off21 + sh; g1.a_si = r; g1.a_sk = 1;
+        g1.B = Linv + off11 + sh; g1.b_sk = r; g1.b_sn = 1;
+        g1.C = Tbuf + off21 + sh; g1.ldc = r; g1.epi = EPI_STORE; g1.skip_flag = skip; g1.precise = precise;
+        GemmArgs g2 = gemm_args();  // X21 = -X22 * T
+        g2.M = rows; g2.N = b; g2.K = rows;
+        g2.A = Linv + off22 + sh; g2.a_si = r; g2.a_sk = 1;
+        g2.B = Tbuf + off21 + sh; g2.b_sk = r; g2.b_sn = 1;
+        g2.C = Linv + off21 + sh; g2.ldc = r; g2.epi = EPI_STORE; g2.alpha = -1.f; g2.skip_flag = skip; g2.precise = precise;
+        if (big) {
+          DION_TRY(launch_gemm(s, g1));
+          DION_TRY(launch_gemm(s, g2));
+        } else {
+          g1.batch = batch; g1.bsA = bs; g1.bsB = bs; g1.bsC = bs;
+          g2.batch = batch; g2.bsA = bs; g2.bsB = bs; g2.bsC = bs;
+          DION_TRY(launch_gemm_simt(s.c, g1, s.st, nullptr, 0, false));
+          DION_TRY(launch_gemm_simt(s.c, g2, s.st, nullptr, 0, false));
+        }
+      }
+    }
+  }
+  return DION_OK;
+}
+
+// Cholesky of the diagonal square [o, o+sz) of Gm (sz <= NBO), right-looking with 64-wide
+// blocks on the FMA engine, followed by the inverse of that square's factor into Linv.
+int potrf_inner(StepCtx& s, float* Gm, i64 r, i64 o, i64 sz, const float* shift, bool adaptive) {
   dion_ctx* c = s.c;
   float* Dinv = s.ws + s.L.Dinv;
   float* Linv = s.ws + s.L.Linv;
@@ -189,18 +243,18 @@ int potrf_trtri(StepCtx& s, float* Gm, i64 r, const float* shift, bool adaptive)
   const float* gdiag = s.ws + s.L.gdiag;
   int* status = c->dev_ints;
   const int* skip = adaptive ? (s.os + OS_DONE) : nullptr;
-  for (i64 j0 = 0; j0 < r; j0 += NB) {
-    const int jb = (int)((r - j0 < NB) ? (r - j0) : NB);
+  for (i64 j0 = o; j0 < o + sz; j0 += NB) {
+    const int jb = (int)((o + sz - j0 < NB) ? (o + sz - j0) : NB);
     float* Ajj = Gm + j0 * r + j0;
     float* Dj = Dinv + (j0 / NB) * (NB * NB);
     float* DPj = s.ws + s.L.DinvP + (j0 / NB) * (NB * NB);
     k_potrf_diag<<<1, 256, 0, s.st>>>(Ajj, r, jb, Dj, DPj, shift, gdiag + j0, adaptive ? FLOOR_REL : 0.f, s.os,
                                       adaptive ? 1 : 0, status);
     DION_CHECK_LAUNCH(c);
-    const i64 rem = r - j0 - jb;
+    const i64 rem = o + sz - j0 - jb;
     if (rem > 0) {
       float* panel = Gm + (j0 + jb) * r + j0;
-      GemmArgs g = gemm_args();  // panel <- panel * Linv_jj^T, in place
+      GemmArgs g = gemm_args();  // panel <- panel * Linv_jj^T, in place (one column tile)
       g.M = rem; g.N = jb; g.K = jb;
       g.A = panel; g.a_si = r; g.a_sk = 1;
       g.B = DPj; g.b_sk = 1; g.b_sn = NB;
@@ -214,41 +268,50 @@ int potrf_trtri(StepCtx& s, float* Gm, i64 r, const float* shift, bool adaptive)
       DION_TRY(launch_gemm_simt(c, t, s.st, nullptr, 0, false));
     }
   }
-  {
-    const i64 total = r * r;
-    int blocks = (int)((total + 255) / 256);
-    if (blocks > 8 * c->sm_count) blocks = 8 * c->sm_count;
-    k_linv_init<<<blocks, 256, 0, s.st>>>(Linv, r, r, Dinv, skip);
-    DION_CHECK_LAUNCH(c);
+  k_linv_init<<<grid_for(c, sz * sz), 256, 0, s.st>>>(Linv, r, o, sz, Dinv, skip);
+  DION_CHECK_LAUNCH(c);
+  return trtri_levels(s, Gm, Linv, Tbuf, r, o, sz, NB, skip, 0);
+}
+
+// Two-level blocked Cholesky of the r x r matrix Gm (lower) and the full inverse of its
+// factor into Linv.  Outer blocks of 512 columns: the diagonal square is factored and
+// inverted by potrf_inner, the panel below it is multiplied by that inverse and the
+// trailing matrix is updated with one rank-512 product (tensor cores where it qualifies).
+int potrf_trtri(StepCtx& s, float* Gm, i64 r, const float* shift, bool adaptive) {
+  dion_ctx* c = s.c;
+  float* Linv = s.ws + s.L.Linv;
+  float* Tbuf = s.ws + s.L.Tbuf;
+  const int* skip = adaptive ? (s.os + OS_DONE) : nullptr;
+  const int precise = adaptive ? 1 : 0;
+  if (r > NBO) {
+    // everything outside the diagonal squares starts at zero (the product U = P Linv^T reads whole tiles)
+    if (cudaMemsetAsync(Linv, 0, sizeof(float) * (size_t)r * (size_t)r, s.st) != cudaSuccess) return DION_ERR_CUDA;
   }
-  // inverse by doubling: [[L11,0],[L21,L22]]^-1 = [[X11,0],[-X22 L21 X11, X22]]
-  for (i64 b = NB; b < r; b *= 2) {
-    const i64 nfull = r / (2 * b);
-    const i64 tail0 = nfull * 2 * b;
-    const i64 b2_tail = (r - tail0 > b) ? (r - tail0 - b) : 0;
-    for (int pass = 0; pass < 2; ++pass) {
-      const i64 base = (pass == 0) ? 0 : tail0;
-      const i64 rows = (pass == 0) ? b : b2_tail;
-      const int batch = (pass == 0) ? (int)nfull : 1;
-      if (rows <= 0 || batch <= 0) continue;
-      const i64 off21 = (base + b) * r + base, off11 = base * r + base, off22 = (base + b) * r + (base + b);
-      const i64 bs = 2 * b * (r + 1);
-      GemmArgs g1 = gemm_args();  // T = L21 * X11
-      g1.M = rows; g1.N = b; g1.K = b;
-      g1.A = Gm + off21; g1.a_si = r; g1.a_sk = 1;
-      g1.B = Linv + off11; g1.b_sk = r; g1.b_sn = 1;
-      g1.C = Tbuf + off21; g1.ldc = r; g1.epi = EPI_STORE; g1.skip_flag = skip;
-      g1.batch = batch; g1.bsA = bs; g1.bsB = bs; g1.bsC = bs;
-      DION_TRY(launch_gemm_simt(c, g1, s.st, nullptr, 0, false));
-      GemmArgs g2 = gemm_args();  // X21 = -X22 * T
-      g2.M = rows; g2.N = b; g2.K = rows;
-      g2.A = Linv + off22; g2.a_si = r; g2.a_sk = 1;
-      g2.B = Tbuf + off21; g2.b_sk = r; g2.b_sn = 1;
-      g2.C = Linv + off21; g2.ldc = r; g2.epi = EPI_STORE; g2.alpha = -1.f; g2.skip_flag = skip;
-      g2.batch = batch; g2.bsA = bs; g2.bsB = bs; g2.bsC = bs;
-      DION_TRY(launch_gemm_simt(c, g2, s.st, nullptr, 0, false));
+  for (i64 J0 = 0; J0 < r; J0 += NBO) {
+    const i64 sz = (r - J0 < NBO) ? (r - J0) : NBO;
+    DION_TRY(potrf_inner(s, Gm, r, J0, sz, shift, adaptive));
+    const i64 rem = r - J0 - sz;
+    if (rem > 0) {
+      float* panel = Gm + (J0 + sz) * r + J0;
+      float* ptmp = Tbuf + (J0 + sz) * r + J0;
+      GemmArgs g = gemm_args();  // Lpanel = panel * Linv_JJ^T (out of place, then copied back)
+      g.M = rem; g.N = sz; g.K = sz;
+      g.A = panel; g.a_si = r; g.a_sk = 1;
+      g.B = Linv + J0 * r + J0; g.b_sk = 1; g.b_sn = r; g.klimit = 1;
+      g.C = ptmp; g.ldc = r; g.epi = EPI_STORE; g.skip_flag = skip; g.precise = precise;
+      DION_TRY(launch_gemm(s, g));
+      k_copy_block<<<grid_for(c, rem * sz), 256, 0, s.st>>>(ptmp, r, panel, r, rem, sz, skip);
+      DION_CHECK_LAUNCH(c);
+      GemmArgs t = gemm_args();  // A22 -= Lpanel * Lpanel^T (lower tiles)
+      t.M = rem; t.N = rem; t.K = sz;
+      t.A = panel; t.a_si = r; t.a_sk = 1;
+      t.B = panel; t.b_sk = 1; t.b_sn = r;
+      t.C = Gm + (J0 + sz) * r + (J0 + sz); t.ldc = r; t.epi = EPI_SUB; t.tri = TRI_LOWER; t.skip_flag = skip;
+      t.precise = precise;
+      DION_TRY(launch_gemm(s, t));
     }
   }
+  if (r > NBO) DION_TRY(trtri_levels(s, Gm, Linv, Tbuf, r, 0, r, NBO, skip, precise));
   return DION_OK;
 }
 

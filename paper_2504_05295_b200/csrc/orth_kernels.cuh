@@ -65,67 +65,153 @@ __global__ void __launch_bounds__(256) k_potrf_diag(float* __restrict__ A, i64 l
                                                     int* __restrict__ os, int adaptive,
                                                     int* __restrict__ status) {
   if (adaptive && os[OS_DONE] != 0) return;
+  // The block is factored in four 16-column sub-panels: the 16 x 16 diagonal piece in
+  // one warp with shuffles, the rows below it by one thread per row, the trailing
+  // update by all threads -- three block-wide barriers per sub-panel instead of three
+  // per column.  The inverse is built from 16 x 16 inverses by doubling.
+  constexpr int W = 16;
   __shared__ float L[NB][NB + 1];
   __shared__ float X[NB][NB + 1];
+  __shared__ float T[NB / 2][NB / 2 + 1];
+  __shared__ float gd[NB];
   __shared__ int deflated[NB];
-  const int tid = threadIdx.x;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const float sh = (shift != nullptr) ? *shift : 0.f;
-  if (tid < NB) deflated[tid] = 0;
+  if (tid < NB) {
+    deflated[tid] = 0;
+    gd[tid] = (floor_rel > 0.f && tid < jb) ? gdiag[tid] + sh : 0.f;
+  }
   for (int e = tid; e < NB * NB; e += 256) {
     const int i = e / NB, c = e % NB;
     float v = 0.f;
     if (i < jb && c <= i) v = A[(i64)i * ld + c] + ((i == c) ? sh : 0.f);
+    if (i >= jb && c == i) v = 1.f;   // identity padding of a ragged last block
     L[i][c] = v;
     X[i][c] = 0.f;
   }
   __syncthreads();
-  int floored = 0;
+
+  int floored = 0, failed = 0;
   float minrel = __int_as_float(0x7f800000);
-  for (int j = 0; j < jb; ++j) {
-    if (tid == 0) {
-      float p = L[j][j];
-      if (floor_rel > 0.f) {
-        const float g = gdiag[j] + sh;
-        const float fl = floor_rel * g;
-        if (!(p > fl) || !isfinite(p)) {
-          p = (fl > 0.f && isfinite(fl)) ? fl : 1.f;   // zero or non-finite column: unit pivot
-          ++floored;
-          deflated[j] = 1;
-        } else {
-          minrel = fminf(minrel, p / g);
+#pragma unroll 1
+  for (int c0 = 0; c0 < NB; c0 += W) {
+    if (warp == 0) {
+      // 16 x 16 diagonal piece: lane i (< 16) holds row c0 + i
+      const int i = lane & (W - 1);
+      float d[W];
+#pragma unroll
+      for (int k = 0; k < W; ++k) d[k] = L[c0 + i][c0 + k];
+#pragma unroll
+      for (int j = 0; j < W; ++j) {
+        float p = __shfl_sync(0xffffffffu, d[j], j);
+        bool defl = false;
+        if (c0 + j < jb) {
+          if (floor_rel > 0.f) {
+            const float g = gd[c0 + j];
+            const float fl = floor_rel * g;
+            if (!(p > fl) || !isfinite(p)) {
+              p = (fl > 0.f && isfinite(fl)) ? fl : 1.f;   // zero or non-finite column: unit pivot
+              defl = true;
+              ++floored;
+            } else {
+              minrel = fminf(minrel, p / g);
+            }
+          } else if (!(p > 0.f) || !isfinite(p)) {
+            failed = 1;
+            p = 1.f;
+          }
         }
-      } else if (!(p > 0.f) || !isfinite(p)) {
-        os[OS_FAIL] = 1;
-        atomicOr(status, DION_STATUS_BREAKDOWN);
-        p = 1.f;
+        const float dj = sqrtf(p);
+        float v = d[j];
+        if (i == j) v = dj;
+        else if (i > j) v = defl ? 0.f : v / dj;
+        d[j] = v;
+        if (lane == 0 && defl) deflated[c0 + j] = 1;
+#pragma unroll
+        for (int c = j + 1; c < W; ++c) {
+          const float vc = __shfl_sync(0xffffffffu, v, c);
+          if (i >= c) d[c] = fmaf(-v, vc, d[c]);
+        }
       }
-      L[j][j] = sqrtf(p);
+      if (lane < W) {
+#pragma unroll
+        for (int k = 0; k < W; ++k)
+          if (k <= i) L[c0 + i][c0 + k] = d[k];
+      }
     }
     __syncthreads();
-    const float d = L[j][j];
-    if (tid > j && tid < jb) L[tid][j] = deflated[j] ? 0.f : L[tid][j] / d;
+    const int below = NB - c0 - W;   // rows under the diagonal piece
+    if (tid < below) {
+      const int i = c0 + W + tid;
+      float x[W];
+#pragma unroll
+      for (int j = 0; j < W; ++j) {
+        float sacc = L[i][c0 + j];
+#pragma unroll
+        for (int k = 0; k < j; ++k) sacc = fmaf(-x[k], L[c0 + j][c0 + k], sacc);
+        x[j] = deflated[c0 + j] ? 0.f : sacc / L[c0 + j][c0 + j];
+      }
+#pragma unroll
+      for (int j = 0; j < W; ++j) L[i][c0 + j] = x[j];
+    }
     __syncthreads();
-    // trailing update of the lower triangle: L[i][c] -= L[i][j] * L[c][j], j < c <= i
-    for (int e = tid; e < NB * NB; e += 256) {
-      const int i = e / NB, c = e % NB;
-      if (c > j && c <= i && i < jb) L[i][c] = fmaf(-L[i][j], L[c][j], L[i][c]);
+    for (int e = tid; e < below * below; e += 256) {
+      const int ii = e / below, cc = e % below;
+      if (cc <= ii) {
+        const int i = c0 + W + ii, c = c0 + W + cc;
+        float sacc = 0.f;
+#pragma unroll
+        for (int k = 0; k < W; ++k) sacc = fmaf(L[i][c0 + k], L[c][c0 + k], sacc);
+        L[i][c] -= sacc;
+      }
     }
     __syncthreads();
   }
-  if (tid == 0 && floor_rel > 0.f) {
-    if (floored) atomicAdd(&os[OS_FLOORED], floored);
-    atomicMin(&os[OS_MINREL], __float_as_int(minrel));
-  }
-  // inverse of the lower factor by forward substitution, one column per thread
-  if (tid < jb) {
-    const int t = tid;
-    for (int i = t; i < jb; ++i) {
-      float s = (i == t) ? 1.f : 0.f;
-      for (int k = t; k < i; ++k) s = fmaf(-L[i][k], X[k][t], s);
-      X[i][t] = s / L[i][i];
+  if (tid == 0) {
+    if (floor_rel > 0.f) {
+      if (floored) atomicAdd(&os[OS_FLOORED], floored);
+      atomicMin(&os[OS_MINREL], __float_as_int(minrel));
+    } else if (failed) {
+      os[OS_FAIL] = 1;
+      atomicOr(status, DION_STATUS_BREAKDOWN);
     }
+  }
+
+  // inverse of the factor: 16 x 16 diagonal inverses by forward substitution ...
+  if (tid < NB) {
+    const int b0 = (tid / W) * W, q = tid % W;
+    float x[W];
+#pragma unroll
+    for (int i = 0; i < W; ++i) {
+      float sacc = (i == q) ? 1.f : 0.f;
+#pragma unroll
+      for (int k = 0; k < i; ++k)
+        if (k >= q) sacc = fmaf(-L[b0 + i][b0 + k], x[k], sacc);
+      x[i] = (i >= q) ? sacc / L[b0 + i][b0 + i] : 0.f;
+    }
+#pragma unroll
+    for (int i = 0; i < W; ++i) X[b0 + i][b0 + q] = x[i];
   }
   __syncthreads();
+  // ... then [[X11, 0], [-X22 L21 X11, X22]] for block sizes 16 and 32
+#pragma unroll 1
+  for (int b = W; b < NB; b *= 2) {
+    const int npairs = NB / (2 * b);
+    for (int e = tid; e < npairs * b * b; e += 256) {
+      const int pr = e / (b * b), rr = (e / b) % b, cc = e % b, base = pr * 2 * b;
+      float sacc = 0.f;
+      for (int k = cc; k < b; ++k) sacc = fmaf(L[base + b + rr][base + k], X[base + k][base + cc], sacc);
+      T[pr * b + rr][cc] = sacc;
+    }
+    __syncthreads();
+    for (int e = tid; e < npairs * b * b; e += 256) {
+      const int pr = e / (b * b), rr = (e / b) % b, cc = e % b, base = pr * 2 * b;
+      float sacc = 0.f;
+      for (int k = 0; k <= rr; ++k) sacc = fmaf(X[base + b + rr][base + b + k], T[pr * b + k][cc], sacc);
+      X[base + b + rr][base + cc] = -sacc;
+    }
+    __syncthreads();
+  }
   for (int e = tid; e < NB * NB; e += 256) {
     const int i = e / NB, c = e % NB;
     if (i < jb && c < jb) A[(i64)i * ld + c] = (c <= i) ? L[i][c] : 0.f;
@@ -159,16 +245,28 @@ __global__ void k_orth_finish(int* __restrict__ os, int* __restrict__ status) {
   }
 }
 
-// Linv = 0 except the 64 x 64 diagonal blocks, which are copied from Dinv.
-__global__ void k_linv_init(float* __restrict__ Linv, i64 ld, i64 r, const float* __restrict__ Dinv,
+// The sz x sz diagonal square of Linv that starts at row/column o (a multiple of 64):
+// zero, except its 64 x 64 diagonal blocks, which are copied from Dinv.
+__global__ void k_linv_init(float* __restrict__ Linv, i64 ld, i64 o, i64 sz, const float* __restrict__ Dinv,
                             const int* __restrict__ skip_flag) {
   if (skip_flag != nullptr && *skip_flag != 0) return;
-  const i64 total = r * r;
+  const i64 total = sz * sz;
   for (i64 e = (i64)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (i64)gridDim.x * blockDim.x) {
-    const i64 i = e / r, c = e % r;
+    const i64 i = o + e / sz, c = o + e % sz;
     float v = 0.f;
     if (i / NB == c / NB) v = Dinv[(i / NB) * (NB * NB) + (i % NB) * NB + (c % NB)];
     Linv[i * ld + c] = v;
+  }
+}
+
+// Copies a rows x cols block between two matrices (leading dimensions lds, ldd).
+__global__ void k_copy_block(const float* __restrict__ src, i64 lds, float* __restrict__ dst, i64 ldd,
+                             i64 rows, i64 cols, const int* __restrict__ skip_flag) {
+  if (skip_flag != nullptr && *skip_flag != 0) return;
+  const i64 total = rows * cols;
+  for (i64 e = (i64)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (i64)gridDim.x * blockDim.x) {
+    const i64 i = e / cols, c = e % cols;
+    dst[i * ldd + c] = src[i * lds + c];
   }
 }
 
