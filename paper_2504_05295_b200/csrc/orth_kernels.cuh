@@ -65,15 +65,16 @@ __global__ void __launch_bounds__(256) k_potrf_diag(float* __restrict__ A, i64 l
                                                     int* __restrict__ os, int adaptive,
                                                     int* __restrict__ status) {
   if (adaptive && os[OS_DONE] != 0) return;
-  // The block is factored in four 16-column sub-panels: the 16 x 16 diagonal piece in
-  // one warp with shuffles, the rows below it by one thread per row, the trailing
-  // update by all threads -- three block-wide barriers per sub-panel instead of three
-  // per column.  The inverse is built from 16 x 16 inverses by doubling.
+  // The block is factored in four 16-column sub-panels: the 16 x 16 diagonal piece by
+  // one warp (two warp barriers per column), the rows below it by one thread per row,
+  // the trailing update by all threads -- three block-wide barriers per sub-panel
+  // instead of three per column.  The inverse is built from 16 x 16 inverses by doubling.
   constexpr int W = 16;
   __shared__ float L[NB][NB + 1];
   __shared__ float X[NB][NB + 1];
   __shared__ float T[NB / 2][NB / 2 + 1];
   __shared__ float gd[NB];
+  __shared__ float rdiag[NB];     // 1 / L[j][j]
   __shared__ int deflated[NB];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const float sh = (shift != nullptr) ? *shift : 0.f;
@@ -81,13 +82,21 @@ __global__ void __launch_bounds__(256) k_potrf_diag(float* __restrict__ A, i64 l
     deflated[tid] = 0;
     gd[tid] = (floor_rel > 0.f && tid < jb) ? gdiag[tid] + sh : 0.f;
   }
-  for (int e = tid; e < NB * NB; e += 256) {
-    const int i = e / NB, c = e % NB;
-    float v = 0.f;
-    if (i < jb && c <= i) v = A[(i64)i * ld + c] + ((i == c) ? sh : 0.f);
-    if (i >= jb && c == i) v = 1.f;   // identity padding of a ragged last block
-    L[i][c] = v;
-    X[i][c] = 0.f;
+  {
+    float v[NB * NB / 256];
+#pragma unroll
+    for (int l = 0; l < NB * NB / 256; ++l) {
+      const int e = tid + l * 256, i = e / NB, c = e % NB;
+      v[l] = (i < jb && c <= i) ? A[(i64)i * ld + c] : 0.f;
+    }
+#pragma unroll
+    for (int l = 0; l < NB * NB / 256; ++l) {
+      const int e = tid + l * 256, i = e / NB, c = e % NB;
+      float x = v[l];
+      if (i == c) x = (i < jb) ? x + sh : 1.f;   // identity padding of a ragged last block
+      L[i][c] = x;
+      X[i][c] = 0.f;
+    }
   }
   __syncthreads();
 
@@ -96,14 +105,11 @@ __global__ void __launch_bounds__(256) k_potrf_diag(float* __restrict__ A, i64 l
 #pragma unroll 1
   for (int c0 = 0; c0 < NB; c0 += W) {
     if (warp == 0) {
-      // 16 x 16 diagonal piece: lane i (< 16) holds row c0 + i
-      const int i = lane & (W - 1);
-      float d[W];
-#pragma unroll
-      for (int k = 0; k < W; ++k) d[k] = L[c0 + i][c0 + k];
-#pragma unroll
+      // 16 x 16 diagonal piece: lane -> row c0 + (lane % 16), column half lane / 16
+      const int i = lane & (W - 1), half = lane >> 4;
+#pragma unroll 1
       for (int j = 0; j < W; ++j) {
-        float p = __shfl_sync(0xffffffffu, d[j], j);
+        float p = L[c0 + j][c0 + j];
         bool defl = false;
         if (c0 + j < jb) {
           if (floor_rel > 0.f) {
@@ -121,22 +127,24 @@ __global__ void __launch_bounds__(256) k_potrf_diag(float* __restrict__ A, i64 l
             p = 1.f;
           }
         }
-        const float dj = sqrtf(p);
-        float v = d[j];
-        if (i == j) v = dj;
-        else if (i > j) v = defl ? 0.f : v / dj;
-        d[j] = v;
-        if (lane == 0 && defl) deflated[c0 + j] = 1;
-#pragma unroll
-        for (int c = j + 1; c < W; ++c) {
-          const float vc = __shfl_sync(0xffffffffu, v, c);
-          if (i >= c) d[c] = fmaf(-v, vc, d[c]);
+        const float inv = rsqrtf(p);
+        float v = 0.f;
+        if (i > j && !defl) v = L[c0 + i][c0 + j] * inv;
+        __syncwarp();
+        if (half == 0) {
+          if (i == j) { L[c0 + j][c0 + j] = p * inv; rdiag[c0 + j] = inv; if (defl) deflated[c0 + j] = 1; }
+          else if (i > j) L[c0 + i][c0 + j] = v;
         }
-      }
-      if (lane < W) {
+        __syncwarp();
+        // rank-1 update of the remaining columns of this piece (each lane: 8 columns of its row)
+        if (i > j) {
 #pragma unroll
-        for (int k = 0; k < W; ++k)
-          if (k <= i) L[c0 + i][c0 + k] = d[k];
+          for (int q = 0; q < W / 2; ++q) {
+            const int c = half * (W / 2) + q;
+            if (c > j && c <= i) L[c0 + i][c0 + c] = fmaf(-v, L[c0 + c][c0 + j], L[c0 + i][c0 + c]);
+          }
+        }
+        __syncwarp();
       }
     }
     __syncthreads();
@@ -149,7 +157,7 @@ __global__ void __launch_bounds__(256) k_potrf_diag(float* __restrict__ A, i64 l
         float sacc = L[i][c0 + j];
 #pragma unroll
         for (int k = 0; k < j; ++k) sacc = fmaf(-x[k], L[c0 + j][c0 + k], sacc);
-        x[j] = deflated[c0 + j] ? 0.f : sacc / L[c0 + j][c0 + j];
+        x[j] = deflated[c0 + j] ? 0.f : sacc * rdiag[c0 + j];
       }
 #pragma unroll
       for (int j = 0; j < W; ++j) L[i][c0 + j] = x[j];
@@ -187,7 +195,7 @@ __global__ void __launch_bounds__(256) k_potrf_diag(float* __restrict__ A, i64 l
 #pragma unroll
       for (int k = 0; k < i; ++k)
         if (k >= q) sacc = fmaf(-L[b0 + i][b0 + k], x[k], sacc);
-      x[i] = (i >= q) ? sacc / L[b0 + i][b0 + i] : 0.f;
+      x[i] = (i >= q) ? sacc * rdiag[b0 + i] : 0.f;
     }
 #pragma unroll
     for (int i = 0; i < W; ++i) X[b0 + i][b0 + q] = x[i];
