@@ -120,16 +120,23 @@ __device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t
 }
 
 // Bounded wait: false when the CTA is (or becomes) dead.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* dead, int* status) {
+// `sleep_ns` > 0 backs off between polls so that a waiting warp does not take issue
+// slots from the producer warps.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* dead, int* status,
+                                          unsigned sleep_ns = 0) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
+  unsigned polls = 0;
   while (true) {
     if (mbar_try_wait(bar, parity)) return true;
-    if (*dead) return false;
-    if (clock64() - t0 > SPIN_LIMIT_CYCLES) {
-      *dead = 1;
-      atomicOr(status, DION_STATUS_TIMEOUT);
-      return false;
+    if (sleep_ns) __nanosleep(sleep_ns);
+    if ((++polls & 63u) == 0) {
+      if (*dead) return false;
+      if (clock64() - t0 > SPIN_LIMIT_CYCLES) {
+        *dead = 1;
+        atomicOr(status, DION_STATUS_TIMEOUT);
+        return false;
+      }
     }
   }
 }
@@ -198,92 +205,112 @@ __device__ __forceinline__ Item decode_item(const Params& p, int item) {
   return it;
 }
 
-// Loads one operand tile (ROWS x BKE elements) into registers as chunks of EPC
-// elements: MN_MAJOR = false reads along k (unit k stride), true reads along the
-// row index (unit row stride).  v[c][e]: chunk c of this thread, element e.
-template <int ROWS, int BKE, int EPC, bool MN_MAJOR, int NCHUNK>
-__device__ __forceinline__ void load_tile(const float* __restrict__ base, i64 s_row, i64 s_k, const void* __restrict__ add,
-                                          i64 a_row, i64 a_k, int add_mode, i64 row0, i64 rows, i64 k0, i64 k_end,
-                                          int ptid, float (&v)[NCHUNK][EPC]) {
-  constexpr int CPR = MN_MAJOR ? (ROWS / EPC) : (BKE / EPC);  // chunks per k-row / per row
-#pragma unroll
-  for (int l = 0; l < NCHUNK; ++l) {
-    const int c = ptid + l * NUM_PROD_THREADS;
-    const int major = c / CPR, minor = c % CPR;
-    const i64 grow = MN_MAJOR ? (row0 + (i64)minor * EPC) : (row0 + major);
-    const i64 gk = MN_MAJOR ? (k0 + major) : (k0 + (i64)minor * EPC);
-    const bool ok = grow < rows && gk < k_end;
-#pragma unroll
-    for (int e = 0; e < EPC; ++e) v[l][e] = 0.f;
-    if (ok) {
-      const float* src = base + grow * s_row + gk * s_k;
-#pragma unroll
-      for (int q = 0; q < EPC / 4; ++q) {
-        const float4 t = __ldg(reinterpret_cast<const float4*>(src) + q);
-        v[l][q * 4 + 0] = t.x; v[l][q * 4 + 1] = t.y; v[l][q * 4 + 2] = t.z; v[l][q * 4 + 3] = t.w;
-      }
-      if (add_mode == ADD_F32) {
-        const float* s2 = reinterpret_cast<const float*>(add) + grow * a_row + gk * a_k;
-#pragma unroll
-        for (int q = 0; q < EPC / 4; ++q) {
-          const float4 t = __ldg(reinterpret_cast<const float4*>(s2) + q);
-          v[l][q * 4 + 0] += t.x; v[l][q * 4 + 1] += t.y; v[l][q * 4 + 2] += t.z; v[l][q * 4 + 3] += t.w;
-        }
-      } else if (add_mode == ADD_BF16) {
-        const __nv_bfloat16* s2 = reinterpret_cast<const __nv_bfloat16*>(add) + grow * a_row + gk * a_k;
-#pragma unroll
-        for (int q = 0; q < EPC / 4; ++q) {
-          const uint2 t = __ldg(reinterpret_cast<const uint2*>(s2) + q);
-          const __nv_bfloat162 lo = *reinterpret_cast<const __nv_bfloat162*>(&t.x);
-          const __nv_bfloat162 hi = *reinterpret_cast<const __nv_bfloat162*>(&t.y);
-          v[l][q * 4 + 0] += __low2float(lo); v[l][q * 4 + 1] += __high2float(lo);
-          v[l][q * 4 + 2] += __low2float(hi); v[l][q * 4 + 3] += __high2float(hi);
-        }
-      }
-    }
-  }
-}
-
-// Writes the chunks to shared memory in the swizzled canonical layout.  fp32 mode:
-// TF32 "hi" part to s_hi and the fp32 remainder to s_lo; bf16 mode: rounded to bf16.
+// Where the 16-byte chunks of one producer thread sit, computed once per kernel:
+// an operand tile is ROWS x BKE elements and is cut into chunks of EPC elements.
+// MN_MAJOR = false: memory is contiguous along k (chunk = EPC consecutive k of one
+// row); true: contiguous along the row index (chunk = EPC consecutive rows at one k).
+//   goff  element offset of the chunk from the tile's (row0, k0) corner in memory
+//   soff  byte offset of the chunk in the stage buffer (swizzled canonical layout)
+//   rpos / kpos  first row / k of the chunk inside the tile (for the edge predicates)
 template <int ROWS, int BKE, int EPC, bool MN_MAJOR, int NCHUNK, bool BF16>
-__device__ __forceinline__ void store_tile(uint32_t s_hi, uint32_t s_lo, int ptid, const float (&v)[NCHUNK][EPC]) {
-  constexpr int CPR = MN_MAJOR ? (ROWS / EPC) : (BKE / EPC);
+struct TileMap {
+  uint32_t goff[NCHUNK];
+  uint32_t goff2[NCHUNK];
+  uint32_t soff[NCHUNK];   // bits 0-19 offset, 20-25 kpos, 26-31 unused
+  uint16_t rpos[NCHUNK];
+
+  __device__ __forceinline__ void init(int ptid, i64 s_row, i64 s_k, i64 s2_row, i64 s2_k) {
+    constexpr int CPR = MN_MAJOR ? (ROWS / EPC) : (BKE / EPC);   // chunks per k-row / per row
 #pragma unroll
-  for (int l = 0; l < NCHUNK; ++l) {
-    const int c = ptid + l * NUM_PROD_THREADS;
-    const int major = c / CPR, minor = c % CPR;
-    uint32_t off;
-    if (MN_MAJOR && !BF16) {   // major = k row, minor = 16-byte chunk along M/N; 32-byte swizzle units
-      const uint32_t q = (uint32_t)(minor & 7);
-      off = (uint32_t)(minor >> 3) * (BKE * 128) + (uint32_t)major * 128 + ((((q >> 1) ^ (uint32_t)(major & 3))) << 5) +
-            ((q & 1u) << 4);
-    } else if (MN_MAJOR) {     // major = k row, minor = 16-byte chunk along M/N
-      off = (uint32_t)(minor >> 3) * (BKE * 128) + (uint32_t)major * 128 + (uint32_t)(((minor & 7) ^ (major & 7)) << 4);
-    } else {          // major = row, minor = 16-byte chunk along k (8 per 128-byte row)
-      off = (uint32_t)major * 128 + (uint32_t)((minor ^ (major & 7)) << 4);
-    }
-    if (BF16) {
-      uint32_t w[4];
-#pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        const __nv_bfloat162 b = __floats2bfloat162_rn(v[l][q * 2], v[l][q * 2 + 1]);
-        w[q] = *reinterpret_cast<const uint32_t*>(&b);
+    for (int l = 0; l < NCHUNK; ++l) {
+      const int c = ptid + l * NUM_PROD_THREADS;
+      const int major = c / CPR, minor = c % CPR;
+      const int row = MN_MAJOR ? minor * EPC : major;
+      const int kk = MN_MAJOR ? major : minor * EPC;
+      goff[l] = (uint32_t)(row * s_row + kk * s_k);
+      goff2[l] = (uint32_t)(row * s2_row + kk * s2_k);
+      rpos[l] = (uint16_t)row;
+      uint32_t off;
+      if (MN_MAJOR && !BF16) {   // TF32, row-contiguous: 32-byte swizzle units, atoms of 4 k-rows
+        const uint32_t q = (uint32_t)(minor & 7);
+        off = (uint32_t)(minor >> 3) * (BKE * 128) + (uint32_t)major * 128 + ((((q >> 1) ^ (uint32_t)(major & 3))) << 5) +
+              ((q & 1u) << 4);
+      } else if (MN_MAJOR) {     // bf16, row-contiguous
+        off = (uint32_t)(minor >> 3) * (BKE * 128) + (uint32_t)major * 128 + (uint32_t)(((minor & 7) ^ (major & 7)) << 4);
+      } else {                   // k-contiguous: rows of 128 bytes, 16-byte units XOR (row mod 8)
+        off = (uint32_t)major * 128 + (uint32_t)((minor ^ (major & 7)) << 4);
       }
-      st_shared_v4(s_hi + off, w[0], w[1], w[2], w[3]);
-    } else {
-      uint32_t h[4], lo[4];
-#pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        h[q] = cvt_tf32(v[l][q]);
-        // the remainder is rounded to TF32 here (to nearest) rather than truncated by the MMA
-        lo[q] = cvt_tf32(v[l][q] - __uint_as_float(h[q]));
-      }
-      st_shared_v4(s_hi + off, h[0], h[1], h[2], h[3]);
-      st_shared_v4(s_lo + off, lo[0], lo[1], lo[2], lo[3]);
+      soff[l] = off | ((uint32_t)kk << 20);
     }
   }
-}
+
+  // Loads the tile whose corner is at `src` (and `src2` for the fused addend).  `rows_left`
+  // / `k_left`: how many rows / k remain from the corner (edge tiles are zero filled).
+  __device__ __forceinline__ void load(const float* __restrict__ src, const void* __restrict__ src2, int add_mode,
+                                       i64 rows_left, i64 k_left, float (&v)[NCHUNK][EPC]) const {
+    const bool interior = rows_left >= ROWS && k_left >= BKE;
+#pragma unroll
+    for (int l = 0; l < NCHUNK; ++l) {
+      const bool ok = interior || ((i64)rpos[l] < rows_left && (i64)(soff[l] >> 20) < k_left);
+      if (ok) {
+        const float* s1 = src + goff[l];
+#pragma unroll
+        for (int q = 0; q < EPC / 4; ++q) {
+          const float4 t = __ldg(reinterpret_cast<const float4*>(s1) + q);
+          v[l][q * 4 + 0] = t.x; v[l][q * 4 + 1] = t.y; v[l][q * 4 + 2] = t.z; v[l][q * 4 + 3] = t.w;
+        }
+        if (add_mode == ADD_F32) {
+          const float* s2 = reinterpret_cast<const float*>(src2) + goff2[l];
+#pragma unroll
+          for (int q = 0; q < EPC / 4; ++q) {
+            const float4 t = __ldg(reinterpret_cast<const float4*>(s2) + q);
+            v[l][q * 4 + 0] += t.x; v[l][q * 4 + 1] += t.y; v[l][q * 4 + 2] += t.z; v[l][q * 4 + 3] += t.w;
+          }
+        } else if (add_mode == ADD_BF16) {
+          const __nv_bfloat16* s2 = reinterpret_cast<const __nv_bfloat16*>(src2) + goff2[l];
+#pragma unroll
+          for (int q = 0; q < EPC / 4; ++q) {
+            const uint2 t = __ldg(reinterpret_cast<const uint2*>(s2) + q);
+            const __nv_bfloat162 lo = *reinterpret_cast<const __nv_bfloat162*>(&t.x);
+            const __nv_bfloat162 hi = *reinterpret_cast<const __nv_bfloat162*>(&t.y);
+            v[l][q * 4 + 0] += __low2float(lo); v[l][q * 4 + 1] += __high2float(lo);
+            v[l][q * 4 + 2] += __low2float(hi); v[l][q * 4 + 3] += __high2float(hi);
+          }
+        }
+      } else {
+#pragma unroll
+        for (int e = 0; e < EPC; ++e) v[l][e] = 0.f;
+      }
+    }
+  }
+
+  // Writes the chunks to shared memory.  fp32 mode: TF32 "hi" part to s_hi and the TF32-
+  // rounded remainder to s_lo; bf16 mode: rounded to bf16 into s_hi.
+  __device__ __forceinline__ void store(uint32_t s_hi, uint32_t s_lo, const float (&v)[NCHUNK][EPC]) const {
+#pragma unroll
+    for (int l = 0; l < NCHUNK; ++l) {
+      const uint32_t off = soff[l] & 0xFFFFFu;
+      if (BF16) {
+        uint32_t w[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          const __nv_bfloat162 b = __floats2bfloat162_rn(v[l][q * 2], v[l][q * 2 + 1]);
+          w[q] = *reinterpret_cast<const uint32_t*>(&b);
+        }
+        st_shared_v4(s_hi + off, w[0], w[1], w[2], w[3]);
+      } else {
+        uint32_t h[4], lo[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          h[q] = cvt_tf32(v[l][q]);
+          lo[q] = __float_as_uint(v[l][q] - __uint_as_float(h[q]));
+        }
+        st_shared_v4(s_hi + off, h[0], h[1], h[2], h[3]);
+        st_shared_v4(s_lo + off, lo[0], lo[1], lo[2], lo[3]);
+      }
+    }
+  }
+};
 
 // SPLIT (fp32 mode only): the hi*hi products and the small hi*lo + lo*hi products go
 // to separate TMEM accumulators that are added once in the epilogue.  Every
@@ -357,7 +384,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_gemm_umma(const Params p) {
       const Item it = decode_item<BN, BKE>(p, item);
       const int ab = iter % NBUF;
       const uint32_t ph = (uint32_t)(iter / NBUF) & 1u;
-      if (!mbar_wait(accf_bar(ab), ph, dead, p.status)) break;
+      if (!mbar_wait(accf_bar(ab), ph, dead, p.status, 256)) break;
       tc_fence_after();
       const i64 gi = (i64)it.mi * BM + warp * 32 + lane;
       const i64 n0 = (i64)it.ni * BN;
@@ -411,6 +438,11 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_gemm_umma(const Params p) {
   } else if (warp < NUM_EPI_WARPS + NUM_PROD_WARPS) {
     // ------------------------------------------------------------ producers
     const int ptid = threadIdx.x - NUM_EPI_WARPS * 32;
+    TileMap<BM, BKE, EPC, A_MN, C::A_CHUNKS, BF16> ma;
+    TileMap<BN, BKE, EPC, B_MN, C::B_CHUNKS, BF16> mb;
+    ma.init(ptid, g.a_si, g.a_sk, g.a2_si, g.a2_sk);
+    mb.init(ptid, g.b_sn, g.b_sk, 0, 0);
+    const int a2_elem = (g.a2_mode == ADD_BF16) ? 2 : 4;
     int stage = 0;
     uint32_t phase = 0;
     bool alive = true;
@@ -419,21 +451,22 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_gemm_umma(const Params p) {
       const i64 row0a = (i64)it.mi * BM, row0b = (i64)it.ni * BN;
       i64 k_end = g.K;
       if (g.klimit) k_end = min(g.K, (i64)(it.ni + 1) * BN);
+      const float* a_row = g.A + row0a * g.a_si;
+      const char* a2_row = reinterpret_cast<const char*>(g.A2) + row0a * g.a2_si * a2_elem;
+      const float* b_row = g.B + row0b * g.b_sn;
       for (int kb = it.kb0; kb < it.kb1; ++kb) {
         const i64 k0 = (i64)kb * BKE;
         float va[C::A_CHUNKS][EPC];
         float vb[C::B_CHUNKS][EPC];
-        load_tile<BM, BKE, EPC, A_MN, C::A_CHUNKS>(g.A, g.a_si, g.a_sk, g.A2, g.a2_si, g.a2_sk, g.a2_mode, row0a, g.M, k0,
-                                                   k_end, ptid, va);
-        load_tile<BN, BKE, EPC, B_MN, C::B_CHUNKS>(g.B, g.b_sn, g.b_sk, nullptr, 0, 0, ADD_NONE, row0b, g.N, k0, k_end,
-                                                   ptid, vb);
+        ma.load(a_row + k0 * g.a_sk, a2_row + k0 * g.a2_sk * a2_elem, g.a2_mode, g.M - row0a, k_end - k0, va);
+        mb.load(b_row + k0 * g.b_sk, nullptr, ADD_NONE, g.N - row0b, k_end - k0, vb);
         if (!mbar_wait(empty_bar(stage), phase ^ 1u, dead, p.status)) { alive = false; break; }
         const uint32_t sa = smem_base + stage * C::STAGE_BYTES;
         const uint32_t sa_lo = sa + C::A_BYTES;
         const uint32_t sb = sa + (BF16 ? 1 : 2) * C::A_BYTES;
         const uint32_t sb_lo = sb + C::B_BYTES;
-        store_tile<BM, BKE, EPC, A_MN, C::A_CHUNKS, BF16>(sa, sa_lo, ptid, va);
-        store_tile<BN, BKE, EPC, B_MN, C::B_CHUNKS, BF16>(sb, sb_lo, ptid, vb);
+        ma.store(sa, sa_lo, va);
+        mb.store(sb, sb_lo, vb);
         fence_proxy_async();
         mbar_arrive(full_bar(stage));
         if (++stage == STAGES) { stage = 0; phase ^= 1u; }
@@ -454,13 +487,13 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_gemm_umma(const Params p) {
         const Item it = decode_item<BN, BKE>(p, item);
         const int ab = iter % NBUF;
         const uint32_t aph = (uint32_t)(iter / NBUF) & 1u;
-        if (!mbar_wait(acce_bar(ab), aph ^ 1u, dead, p.status)) { alive = false; break; }
+        if (!mbar_wait(acce_bar(ab), aph ^ 1u, dead, p.status, 64)) { alive = false; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(ab * ACCS * BN);
         const uint32_t d_small = d_tmem + (SPLIT ? BN : 0);
         uint32_t accumulate = 0;
         for (int kb = it.kb0; kb < it.kb1; ++kb) {
-          if (!mbar_wait(full_bar(stage), phase, dead, p.status)) { alive = false; break; }
+          if (!mbar_wait(full_bar(stage), phase, dead, p.status, 32)) { alive = false; break; }
           tc_fence_after();
           const uint32_t sa = smem_base + stage * C::STAGE_BYTES;
           const uint32_t sa_lo = sa + C::A_BYTES;
@@ -496,7 +529,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_gemm_umma(const Params p) {
       }
       // drain: every issued MMA must have finished before TMEM is released
       umma_commit(drain_bar);
-      mbar_wait(drain_bar, 0u, dead, p.status);
+      mbar_wait(drain_bar, 0u, dead, p.status, 64);
     }
     __syncwarp();
   }
