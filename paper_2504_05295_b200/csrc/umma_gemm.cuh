@@ -246,41 +246,56 @@ struct TileMap {
 
   // Loads the tile whose corner is at `src` (and `src2` for the fused addend).  `rows_left`
   // / `k_left`: how many rows / k remain from the corner (edge tiles are zero filled).
+  // All loads are issued before any value is used, so their latencies overlap; the
+  // addend is kept raw in `w` (fp32 values, or packed bf16 pairs) until add() runs.
   __device__ __forceinline__ void load(const float* __restrict__ src, const void* __restrict__ src2, int add_mode,
-                                       i64 rows_left, i64 k_left, float (&v)[NCHUNK][EPC]) const {
+                                       i64 rows_left, i64 k_left, float (&v)[NCHUNK][EPC], float (&w)[NCHUNK][EPC]) const {
     const bool interior = rows_left >= ROWS && k_left >= BKE;
 #pragma unroll
     for (int l = 0; l < NCHUNK; ++l) {
       const bool ok = interior || ((i64)rpos[l] < rows_left && (i64)(soff[l] >> 20) < k_left);
-      if (ok) {
-        const float* s1 = src + goff[l];
+#pragma unroll
+      for (int q = 0; q < EPC / 4; ++q) {
+        float4 t = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (ok) t = __ldg(reinterpret_cast<const float4*>(src + goff[l]) + q);
+        v[l][q * 4 + 0] = t.x; v[l][q * 4 + 1] = t.y; v[l][q * 4 + 2] = t.z; v[l][q * 4 + 3] = t.w;
+      }
+      if (add_mode == ADD_F32) {
 #pragma unroll
         for (int q = 0; q < EPC / 4; ++q) {
-          const float4 t = __ldg(reinterpret_cast<const float4*>(s1) + q);
-          v[l][q * 4 + 0] = t.x; v[l][q * 4 + 1] = t.y; v[l][q * 4 + 2] = t.z; v[l][q * 4 + 3] = t.w;
+          float4 t = make_float4(0.f, 0.f, 0.f, 0.f);
+          if (ok) t = __ldg(reinterpret_cast<const float4*>(reinterpret_cast<const float*>(src2) + goff2[l]) + q);
+          w[l][q * 4 + 0] = t.x; w[l][q * 4 + 1] = t.y; w[l][q * 4 + 2] = t.z; w[l][q * 4 + 3] = t.w;
         }
-        if (add_mode == ADD_F32) {
-          const float* s2 = reinterpret_cast<const float*>(src2) + goff2[l];
+      } else if (add_mode == ADD_BF16) {
 #pragma unroll
-          for (int q = 0; q < EPC / 4; ++q) {
-            const float4 t = __ldg(reinterpret_cast<const float4*>(s2) + q);
-            v[l][q * 4 + 0] += t.x; v[l][q * 4 + 1] += t.y; v[l][q * 4 + 2] += t.z; v[l][q * 4 + 3] += t.w;
-          }
-        } else if (add_mode == ADD_BF16) {
-          const __nv_bfloat16* s2 = reinterpret_cast<const __nv_bfloat16*>(src2) + goff2[l];
-#pragma unroll
-          for (int q = 0; q < EPC / 4; ++q) {
-            const uint2 t = __ldg(reinterpret_cast<const uint2*>(s2) + q);
-            const __nv_bfloat162 lo = *reinterpret_cast<const __nv_bfloat162*>(&t.x);
-            const __nv_bfloat162 hi = *reinterpret_cast<const __nv_bfloat162*>(&t.y);
-            v[l][q * 4 + 0] += __low2float(lo); v[l][q * 4 + 1] += __high2float(lo);
-            v[l][q * 4 + 2] += __low2float(hi); v[l][q * 4 + 3] += __high2float(hi);
-          }
+        for (int q = 0; q < EPC / 4; ++q) {
+          uint2 t = make_uint2(0u, 0u);
+          if (ok) t = __ldg(reinterpret_cast<const uint2*>(reinterpret_cast<const __nv_bfloat16*>(src2) + goff2[l]) + q);
+          w[l][q * 4 + 0] = __uint_as_float(t.x); w[l][q * 4 + 1] = __uint_as_float(t.y);
         }
-      } else {
-#pragma unroll
-        for (int e = 0; e < EPC; ++e) v[l][e] = 0.f;
       }
+    }
+  }
+
+  // v += addend (after load()).
+  __device__ __forceinline__ void add(int add_mode, float (&v)[NCHUNK][EPC], const float (&w)[NCHUNK][EPC]) const {
+    if (add_mode == ADD_F32) {
+#pragma unroll
+      for (int l = 0; l < NCHUNK; ++l)
+#pragma unroll
+        for (int e = 0; e < EPC; ++e) v[l][e] += w[l][e];
+    } else if (add_mode == ADD_BF16) {
+#pragma unroll
+      for (int l = 0; l < NCHUNK; ++l)
+#pragma unroll
+        for (int q = 0; q < EPC / 4; ++q) {
+          const uint32_t x = __float_as_uint(w[l][q * 4 + 0]), y = __float_as_uint(w[l][q * 4 + 1]);
+          const __nv_bfloat162 lo = *reinterpret_cast<const __nv_bfloat162*>(&x);
+          const __nv_bfloat162 hi = *reinterpret_cast<const __nv_bfloat162*>(&y);
+          v[l][q * 4 + 0] += __low2float(lo); v[l][q * 4 + 1] += __high2float(lo);
+          v[l][q * 4 + 2] += __low2float(hi); v[l][q * 4 + 3] += __high2float(hi);
+        }
     }
   }
 
@@ -456,11 +471,12 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_gemm_umma(const Params p) {
       const float* b_row = g.B + row0b * g.b_sn;
       for (int kb = it.kb0; kb < it.kb1; ++kb) {
         const i64 k0 = (i64)kb * BKE;
-        float va[C::A_CHUNKS][EPC];
+        float va[C::A_CHUNKS][EPC], wa[C::A_CHUNKS][EPC];
         float vb[C::B_CHUNKS][EPC];
-        ma.load(a_row + k0 * g.a_sk, a2_row + k0 * g.a2_sk * a2_elem, g.a2_mode, g.M - row0a, k_end - k0, va);
-        mb.load(b_row + k0 * g.b_sk, nullptr, ADD_NONE, g.N - row0b, k_end - k0, vb);
+        ma.load(a_row + k0 * g.a_sk, a2_row + k0 * g.a2_sk * a2_elem, g.a2_mode, g.M - row0a, k_end - k0, va, wa);
+        mb.load(b_row + k0 * g.b_sk, nullptr, ADD_NONE, g.N - row0b, k_end - k0, vb, vb);
         if (!mbar_wait(empty_bar(stage), phase ^ 1u, dead, p.status)) { alive = false; break; }
+        ma.add(g.a2_mode, va, wa);
         const uint32_t sa = smem_base + stage * C::STAGE_BYTES;
         const uint32_t sa_lo = sa + C::A_BYTES;
         const uint32_t sb = sa + (BF16 ? 1 : 2) * C::A_BYTES;
