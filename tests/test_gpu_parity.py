@@ -256,3 +256,100 @@ def test_lazy_dion_steps_match_oracle():
         assert opt.get_status() == (0, 0)
     assert rel(to_np64(X), Xo) <= TOL_FP32 and rel(to_np64(M), Mo) <= TOL_FP32
     assert rel(to_np64(Q), Qo) <= TOL_FP32 and rel(to_np64(d), do) <= TOL_FP32
+
+
+# ---------------------------------------------------------------------------
+# Benchmark-size cases.  One full-size element-wise comparison that the oracle
+# finishes in tens of seconds, then properties that hold at any size, evaluated in
+# float64 on the device (test-side arithmetic; the step itself is the library's).
+# ---------------------------------------------------------------------------
+
+def test_4096_square_quarter_rank_against_oracle():
+    m = n = 4096
+    r = 1024
+    pb = inputs.make_problem(m, n, r, seed=15, ks=64)
+    ref = oracle_steps(pb, 1)
+    snaps, status, skipped = run_gpu(pb, 1)
+    assert status == 0 and skipped == 0
+    check(snaps[0], ref[0], TOL_FP32, "4096^2 r=1024, step 1")
+
+
+def step_properties(m, n, r, g_dtype, tol=TOL_FP32, precision=binding.PREC_FP32, steps=2):
+    """Runs `steps` library steps on device-generated inputs and checks, in float64, what the
+    rule fixes for the last one: the factors can be read back from the outputs because
+    (X - X')/s = U Q'^T and R = Q' diag(d + eps)."""
+    pb = inputs.make_problem(m, n, r, seed=16, ks=64, g_dtype=g_dtype, device="cuda", keep_signal=False)
+    X, M, Q = pb.X, pb.M, pb.Q
+    d = torch.zeros(r, device="cuda")
+    with binding.Dion(mu=MU, eps=EPS, precision=precision) as opt:
+        for t in range(steps):
+            G = pb.grad(t)
+            X0, M0 = X.clone(), M.clone()
+            opt.step(X, M, G, Q, ETA, colnorm_out=d)
+        assert opt.get_status() == (0, 0)
+    s = ETA * (m / n) ** 0.5
+    B = M0.double() + G.double()
+    Qn = Q.double()
+    delta = (X0.double() - X.double()) / s                      # U Q'^T
+    U = torch.linalg.solve(Qn.t() @ Qn, (delta @ Qn).t()).t()   # U = delta Q' (Q'^T Q')^-1
+    del delta
+    R = Qn * (d.double() + EPS)
+    eye = torch.eye(r, device="cuda", dtype=torch.float64)
+    # fp32 X carries eta-scaled updates: U is read back with ~1e-7 / (eta * |U_ij|) relative noise
+    tol_u = max(tol, 3e-4)
+    assert float((U.t() @ U - eye).abs().max()) <= tol_u
+    assert float(torch.linalg.norm(B.t() @ U - R) / torch.linalg.norm(R)) <= tol_u
+    assert float(torch.linalg.norm(B - (1 - MU) * (U @ R.t()) - M.double()) / torch.linalg.norm(M.double())) <= tol
+    nq = torch.linalg.norm(Qn, dim=0)
+    assert float((nq - 1).abs().max()) <= 1e-5
+    upd = float(torch.linalg.norm(X0.double() - X.double()))
+    assert abs(upd - s * r ** 0.5) <= 1e-3 * s * r ** 0.5
+    assert float(torch.linalg.norm(d.double() - torch.linalg.norm(B.t() @ U, dim=0)) / torch.linalg.norm(d.double())) <= tol_u
+
+
+@pytest.mark.parametrize("m,n,r", [(8192, 8192, 512), (8192, 8192, 2048), (2048, 2048, 2048), (4096, 4096, 4096)])
+def test_properties_on_the_square_sweep_sizes(m, n, r):
+    step_properties(m, n, r, torch.float32)
+
+
+@pytest.mark.parametrize("m,n,r", [(4096, 4096, 1024), (1024, 4096, 256), (14336, 4096, 1024), (4096, 14336, 1024)])
+def test_properties_on_llama8b_shapes_bf16_gradients(m, n, r):
+    step_properties(m, n, r, torch.bfloat16)
+
+
+@pytest.mark.parametrize("m,n,r", [(16384, 16384, 1024), (32768, 32768, 512)])
+def test_properties_on_the_large_square_sizes(m, n, r):
+    step_properties(m, n, r, torch.float32, steps=1)
+    torch.cuda.empty_cache()
+
+
+@pytest.mark.parametrize("m,n,r", [(1024, 16384, 256), (53248, 16384, 1024), (16384, 53248, 1024)])
+def test_properties_on_llama405b_shapes_bf16_gradients(m, n, r):
+    step_properties(m, n, r, torch.bfloat16, steps=1)
+    torch.cuda.empty_cache()
+
+
+@pytest.mark.parametrize("m,n,r", [(1792, 512, 128), (512, 1792, 128), (128, 512, 32)])
+def test_llama_aspect_ratios_bf16_gradients_against_oracle(m, n, r):
+    pb = inputs.make_problem(m, n, r, seed=17, ks=32, g_dtype=torch.bfloat16)
+    ref = oracle_steps(pb, 3)
+    snaps, status, skipped = run_gpu(pb, 3)
+    assert status == 0 and skipped == 0
+    check(snaps[0], ref[0], TOL_FP32, "step 1")
+    check(snaps[2], ref[2], TOL_FP32, "step 3")
+
+
+def test_grouped_llama_like_block_list_against_oracle():
+    # two "layers" of the seven block shapes, scaled down by 8, rank fraction 1/4, bf16 gradients
+    shapes = [(nm, m // 8, n // 8) for nm, m, n in inputs.llama_block_shapes(4096, 1024, 14336)] * 2
+    pbs = [inputs.make_problem(m, n, min(m, n) // 4, seed=18, k=k, ks=16, g_dtype=torch.bfloat16)
+           for k, (nm, m, n) in enumerate(shapes)]
+    states = [device_state(pb) for pb in pbs]
+    with binding.Dion(mu=MU, eps=EPS) as opt:
+        for t in range(2):
+            opt.step_grouped([(X, M, pb.grad(t).cuda(), Q) for pb, (X, M, Q) in zip(pbs, states)], ETA)
+        assert opt.get_status() == (0, 0)
+    for pb, (X, M, Q) in zip(pbs, states):
+        ref = oracle_steps(pb, 2)
+        assert rel(to_np64(X), ref[1].X) <= TOL_FP32 and rel(to_np64(M), ref[1].M) <= TOL_FP32
+        assert rel(to_np64(Q), ref[1].Q) <= TOL_FP32
