@@ -19,7 +19,8 @@ namespace {
 constexpr int MAX_FLAG_SLOTS = 4096;      // step slots of OS_SLOT_INTS ints each
 constexpr int MAX_ROUNDS = 6;             // adaptive Cholesky QR rounds
 constexpr float FLOOR_REL = 1e-4f;        // pivot floor relative to the column's squared norm
-constexpr float GOOD_REL = 1e-3f;         // smallest relative pivot of a well-conditioned round
+constexpr float GOOD_REL = 1e-4f;         // smallest relative pivot of a round that one more round can finish
+constexpr float DONE_REL = 0.9f;          // smallest relative pivot of a round whose input was already orthonormal
 constexpr i64 PART_CAP_FLOATS = (i64)16 << 20;  // split-K partial sums, at most 64 MiB
 
 inline i64 align64(i64 floats) { return (floats + 63) / 64 * 64; }  // 256-byte granules
@@ -346,7 +347,7 @@ int cholqr_round(StepCtx& s, const float* Pin, float* Pout, i64 rows, i64 r, boo
   u.C = Pout; u.ldc = r; u.epi = EPI_STORE; u.skip_flag = skip; u.precise = adaptive ? 1 : 0;
   DION_TRY(launch_gemm(s, u));
   if (adaptive) {
-    k_round_end<<<1, 1, 0, s.st>>>(s.os, GOOD_REL, c->dev_ints + 2);
+    k_round_end<<<1, 1, 0, s.st>>>(s.os, GOOD_REL, DONE_REL, c->dev_ints + 2);
     DION_CHECK_LAUNCH(c);
   }
   return DION_OK;

@@ -228,17 +228,23 @@ __global__ void __launch_bounds__(256) k_potrf_diag(float* __restrict__ A, i64 l
   }
 }
 
-// End of an adaptive round (one thread).  A round that raised no pivot and whose
-// smallest relative pivot is >= good_rel saw a panel with cond <~ 1/sqrt(good_rel):
-// one more round after it brings orthonormality to rounding level, then the
-// remaining rounds are skipped.
-__global__ void k_round_end(int* __restrict__ os, float good_rel, int* __restrict__ rounds_total) {
+// End of an adaptive round (one thread).  `minrel`, the smallest pivot relative to its
+// column's squared norm, estimates 1 / cond^2 of the round's input panel.
+//   - no pivot raised and minrel >= done_rel: the input was already orthonormal to
+//     ~(1 - done_rel), so this round's output is orthonormal to rounding level: done;
+//   - no pivot raised and minrel >= good_rel: cond <~ 1 / sqrt(good_rel); one more
+//     round brings orthonormality to rounding level (the CholeskyQR2 argument), after
+//     which the remaining rounds are skipped.
+__global__ void k_round_end(int* __restrict__ os, float good_rel, float done_rel, int* __restrict__ rounds_total) {
   if (os[OS_DONE] != 0) return;
   os[OS_ROUNDS] += 1;
   atomicAdd(rounds_total, 1);
   if (os[OS_GOOD] != 0) { os[OS_DONE] = 1; return; }
   const float minrel = __int_as_float(os[OS_MINREL]);
-  if (os[OS_FLOORED] == 0 && minrel >= good_rel) os[OS_GOOD] = 1;
+  if (os[OS_FLOORED] == 0) {
+    if (minrel >= done_rel) os[OS_DONE] = 1;
+    else if (minrel >= good_rel) os[OS_GOOD] = 1;
+  }
 }
 
 // After the last adaptive round: a panel that never became well conditioned is
