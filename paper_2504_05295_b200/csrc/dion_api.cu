@@ -2,6 +2,7 @@
 // the launch sequence of one step.  All arithmetic runs in the kernels of this
 // directory; the host code only validates and launches.
 #include <math.h>
+#include <stdlib.h>
 #include <new>
 #include <string.h>
 #include <vector>
@@ -928,7 +929,8 @@ extern "C" int dion_debug_gemm(int engine, int precision, const dion_debug_gemm_
   g.alpha = a->alpha; g.tri = a->tri; g.klimit = a->klimit; g.precise = a->precise;
   cudaStream_t st = (cudaStream_t)cuda_stream;
   if (engine == DION_ENGINE_TENSOR) {
-    const int rc = umma_try_launch(g, precision, sms, part, part_floats, status, st);
+    const char* dbg = getenv("DION_DEBUG_GEMM");   // timing experiments of this hook only
+    const int rc = umma_try_launch(g, precision, sms, part, part_floats, status, st, dbg ? atoi(dbg) : 0);
     if (rc > 0) return DION_OK;
     return rc < 0 ? rc : DION_ERR_UNSUPPORTED;
   }

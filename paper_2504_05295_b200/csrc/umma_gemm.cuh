@@ -39,6 +39,7 @@ struct Params {
   int nkb;            // K blocks in all
   int num_items;      // tiles * splits
   int* status;        // device status word (DION_STATUS_TIMEOUT)
+  int debug;          // internal timing experiments: 1 no global loads, 2 no loads/stores, 4 no MMAs
 };
 
 // ------------------------------------------------------------------ PTX wrappers
@@ -375,7 +376,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_gemm_umma(const Params p) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), NUM_PROD_THREADS); mbar_init(empty_bar(s), 1); }
+    for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), NUM_PROD_WARPS); mbar_init(empty_bar(s), 1); }
     for (int b = 0; b < 2; ++b) { mbar_init(accf_bar(b), 1); mbar_init(acce_bar(b), NUM_EPI_WARPS * 32); }
     mbar_init(drain_bar, 1);
     *dead = 0;
@@ -473,8 +474,19 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_gemm_umma(const Params p) {
         const i64 k0 = (i64)kb * BKE;
         float va[C::A_CHUNKS][EPC], wa[C::A_CHUNKS][EPC];
         float vb[C::B_CHUNKS][EPC];
+        if (p.debug & 3) {
+#pragma unroll
+          for (int l = 0; l < C::A_CHUNKS; ++l)
+#pragma unroll
+            for (int e = 0; e < EPC; ++e) { va[l][e] = 1.f; wa[l][e] = 0.f; }
+#pragma unroll
+          for (int l = 0; l < C::B_CHUNKS; ++l)
+#pragma unroll
+            for (int e = 0; e < EPC; ++e) vb[l][e] = 1.f;
+        } else {
         ma.load(a_row + k0 * g.a_sk, a2_row + k0 * g.a2_sk * a2_elem, g.a2_mode, g.M - row0a, k_end - k0, va, wa);
         mb.load(b_row + k0 * g.b_sk, nullptr, ADD_NONE, g.N - row0b, k_end - k0, vb, vb);
+        }
         if (!mbar_wait(empty_bar(stage), phase ^ 1u, dead, p.status)) { alive = false; break; }
         ma.add(g.a2_mode, va, wa);
         const uint32_t sa = smem_base + stage * C::STAGE_BYTES;
@@ -483,8 +495,11 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_gemm_umma(const Params p) {
         const uint32_t sb_lo = sb + C::B_BYTES;
         ma.store(sa, sa_lo, va);
         mb.store(sb, sb_lo, vb);
+        // every thread makes its own writes visible to the tensor core's (async) proxy, then
+        // one lane per warp arrives: 8 arrivals per stage instead of 256 serialised ones
         fence_proxy_async();
-        mbar_arrive(full_bar(stage));
+        __syncwarp();
+        if (lane == 0) mbar_arrive(full_bar(stage));
         if (++stage == STAGES) { stage = 0; phase ^= 1u; }
       }
     }
@@ -509,14 +524,14 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_gemm_umma(const Params p) {
         const uint32_t d_small = d_tmem + (SPLIT ? BN : 0);
         uint32_t accumulate = 0;
         for (int kb = it.kb0; kb < it.kb1; ++kb) {
-          if (!mbar_wait(full_bar(stage), phase, dead, p.status, 32)) { alive = false; break; }
+          if (!mbar_wait(full_bar(stage), phase, dead, p.status)) { alive = false; break; }
           tc_fence_after();
           const uint32_t sa = smem_base + stage * C::STAGE_BYTES;
           const uint32_t sa_lo = sa + C::A_BYTES;
           const uint32_t sb = sa + (BF16 ? 1 : 2) * C::A_BYTES;
           const uint32_t sb_lo = sb + C::B_BYTES;
 #pragma unroll
-          for (int ks = 0; ks < 4; ++ks) {
+          for (int ks = 0; ks < ((p.debug & 4) ? 0 : 4); ++ks) {
             const uint64_t a_hi = make_desc<BF16>(sa + ks * A_KSTEP, A_MN, lbo);
             const uint64_t b_hi = make_desc<BF16>(sb + ks * B_KSTEP, B_MN, lbo);
             if (BF16) {
@@ -595,7 +610,7 @@ inline int umma_configure() {
 // kernels launched (1, or 2 with a split-K reduction), 0 if this engine does not take
 // the product, or a negative DION_ERR_* code.
 inline int umma_try_launch(const GemmArgs& g_in, int precision, int sm_count, float* part, i64 part_floats,
-                           int* status, cudaStream_t st) {
+                           int* status, cudaStream_t st, int debug = 0) {
   using namespace umma;
   GemmArgs g = g_in;
   const bool bf16 = (precision == DION_PREC_BF16_OPERANDS);
@@ -645,6 +660,7 @@ inline int umma_try_launch(const GemmArgs& g_in, int precision, int sm_count, fl
   if (tiles * splits > 0x7fffffff) return 0;
   p.num_items = (int)(tiles * splits);
   p.status = status;
+  p.debug = debug;
   const int grid = p.num_items < sm_count ? p.num_items : sm_count;
   if (bf16) {
     if (BN == 256) launch_variant<256, true, false>(p, a_mn, b_mn, grid, st);
