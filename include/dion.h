@@ -167,7 +167,8 @@ enum {
   DION_PHASE_EF = 3,      /* M <- (M + G) - (1 - mu) U R^T      */
   DION_PHASE_COLNORM = 4, /* Q <- ColNorm(R)                    */
   DION_PHASE_X = 5,       /* X <- X - lr sqrt(m/n) U Q^T        */
-  DION_NUM_PHASES = 6
+  DION_PHASE_ORTH_GEMM = 6, /* the part of DION_PHASE_ORTH spent in tensor-core products */
+  DION_NUM_PHASES = 7
 };
 
 /* Per-phase device timing with CUDA events recorded on the step's own stream.

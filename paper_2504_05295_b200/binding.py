@@ -26,7 +26,7 @@ EXPORTS = ["dion_default_config", "dion_init", "dion_step", "dion_step_grouped",
            "dion_workspace_bytes", "dion_get_status", "dion_launch_count", "dion_destroy",
            "dion_strerror", "dion_profile_enable", "dion_profile_read", "dion_get_orth_rounds",
            "dion_step_noalloc", "dion_noalloc_scratch_limit"]
-PHASES = ["P", "ORTH", "R", "EF", "COLNORM", "X"]
+PHASES = ["P", "ORTH", "R", "EF", "COLNORM", "X", "ORTH_GEMM"]
 
 
 class DionConfig(ctypes.Structure):

@@ -159,6 +159,29 @@ int launch_gemm_simt(dion_ctx* c, GemmArgs g, cudaStream_t st, float* part, i64 
   return DION_OK;
 }
 
+cudaEvent_t prof_event(dion_ctx* c) {
+  if (c->prof_used == c->prof_pool.size()) {
+    cudaEvent_t e = nullptr;
+    if (cudaEventCreate(&e) != cudaSuccess) return nullptr;
+    c->prof_pool.push_back(e);
+  }
+  return c->prof_pool[c->prof_used++];
+}
+
+// Brackets one phase of a step with events on the step's stream when profiling is on.
+struct PhaseScope {
+  dion_ctx* c; cudaStream_t st; int phase; cudaEvent_t e0; int64_t l0;
+  PhaseScope(dion_ctx* c_, cudaStream_t st_, int phase_) : c(c_), st(st_), phase(phase_), e0(nullptr), l0(c_->launches) {
+    if (c->prof_on && phase >= 0) { e0 = prof_event(c); if (e0) cudaEventRecord(e0, st); }
+  }
+  ~PhaseScope() {
+    if (c->prof_on && e0) {
+      cudaEvent_t e1 = prof_event(c);
+      if (e1) { cudaEventRecord(e1, st); c->prof_recs.push_back({phase, e0, e1, c->launches - l0}); }
+    }
+  }
+};
+
 struct StepCtx {
   dion_ctx* c;
   cudaStream_t st;
@@ -167,11 +190,13 @@ struct StepCtx {
   int* os;    // this step's device state slot (OS_* ints)
   int* flag;  // = os + OS_FAIL: the step must not write its outputs
   bool tensor;  // tensor-core engine allowed for this matrix
+  bool in_orth; // inside the orthonormalization (for the profiling phases)
 };
 
 // Engine dispatch: tensor cores when the product qualifies, else fp32 FMA.
 int launch_gemm(StepCtx& s, const GemmArgs& g, bool force64 = false) {
   if (s.tensor && !force64) {
+    PhaseScope ps(s.c, s.st, s.in_orth ? DION_PHASE_ORTH_GEMM : -1);
     const int rc = umma_try_launch(g, s.c->cfg.precision, s.c->sm_count, s.ws + s.L.part, s.L.part_floats,
                                    s.c->dev_ints, s.st);
     if (rc > 0) { s.c->launches += rc; return DION_OK; }
@@ -471,32 +496,10 @@ int begin_step(dion_ctx* c, const dion_matrix* a, cudaStream_t st, StepCtx* s) {
   s->flag = s->os + OS_FAIL;
   c->flag_cursor = (c->flag_cursor + 1) % MAX_FLAG_SLOTS;
   s->tensor = (c->cfg.engine != DION_ENGINE_SIMT);
+  s->in_orth = false;
   if (cudaMemsetAsync(s->os, 0, sizeof(int) * OS_SLOT_INTS, st) != cudaSuccess) return DION_ERR_CUDA;
   return DION_OK;
 }
-
-cudaEvent_t prof_event(dion_ctx* c) {
-  if (c->prof_used == c->prof_pool.size()) {
-    cudaEvent_t e = nullptr;
-    if (cudaEventCreate(&e) != cudaSuccess) return nullptr;
-    c->prof_pool.push_back(e);
-  }
-  return c->prof_pool[c->prof_used++];
-}
-
-// Brackets one phase of a step with events on the step's stream when profiling is on.
-struct PhaseScope {
-  dion_ctx* c; cudaStream_t st; int phase; cudaEvent_t e0; int64_t l0;
-  PhaseScope(dion_ctx* c_, cudaStream_t st_, int phase_) : c(c_), st(st_), phase(phase_), e0(nullptr), l0(c_->launches) {
-    if (c->prof_on) { e0 = prof_event(c); if (e0) cudaEventRecord(e0, st); }
-  }
-  ~PhaseScope() {
-    if (c->prof_on && e0) {
-      cudaEvent_t e1 = prof_event(c);
-      if (e1) { cudaEventRecord(e1, st); c->prof_recs.push_back({phase, e0, e1, c->launches - l0}); }
-    }
-  }
-};
 
 // The launch chain of one Dion step (Algorithm 1 + 2).  Scratch must be large enough.
 int step_one(dion_ctx* c, const dion_matrix* a, float lr, cudaStream_t st) {
@@ -526,7 +529,10 @@ int step_one(dion_ctx* c, const dion_matrix* a, float lr, cudaStream_t st) {
   float* U = nullptr;
   {
   PhaseScope ps(c, st, DION_PHASE_ORTH);
-  DION_TRY(orthonormalize(s, m, r, (m < n) ? m : n, &U));
+  s.in_orth = true;
+  const int rc_orth = orthonormalize(s, m, r, (m < n) ? m : n, &U);
+  s.in_orth = false;
+  DION_TRY(rc_orth);
   }
 
   // R = (M + G)^T U
