@@ -46,14 +46,33 @@ def load_peaks():
     return {"hbm_gbs": 6650.0, "bf16_burst": 1590.0, "bf16_sustained": 1400.0, "source": "fallback"}
 
 
-def parse_cases(spec, inputs):
-    if not spec:
-        return inputs.config2_cases()
-    out = []
-    for tok in spec.split(","):
-        d, r = tok.split(":")
-        out.append((int(d), int(d), int(r)))
-    return out
+def parse_cases(spec, inputs, workload="sweep"):
+    """Cases are (m, n, r) for fp32 gradients or (m, n, r, "bf16").  --cases takes d:r or mxn:r[:bf16]."""
+    if spec:
+        out = []
+        for tok in spec.split(","):
+            f = tok.split(":")
+            if "x" in f[0]:
+                m, n = (int(v) for v in f[0].split("x"))
+            else:
+                m = n = int(f[0])
+            case = (m, n, int(f[1]))
+            if len(f) > 2 and f[2] == "bf16":
+                case = case + ("bf16",)
+            out.append(case)
+        return out
+    if workload == "large":
+        return inputs.config3_cases()
+    if workload == "llama8b":
+        return [(m, n, min(m, n) // 4, "bf16") for _, m, n in inputs.config4_shapes()]
+    if workload == "llama405b":
+        return ([(m, n, min(m, n) // 4, "bf16") for _, m, n in inputs.config5_shapes()] +
+                [(m, n, min(m, n) // 16, "bf16") for _, m, n in inputs.config5_shapes()])
+    return inputs.config2_cases()
+
+
+def case_gbytes(c):
+    return 2 if len(c) > 3 and c[3] == "bf16" else 4
 
 
 # ---------------------------------------------------------------------------
@@ -159,10 +178,11 @@ class ClockSampler:
 # ---------------------------------------------------------------------------
 
 def oracle_sample_cases(cases):
-    """The smallest matrix size of the sweep at its two low rank fractions."""
-    d0 = min(c[0] for c in cases)
-    pick = [c for c in cases if c[0] == d0 and c[2] < d0]
-    return pick or [min(cases, key=lambda c: oracle_flops(*c))]
+    """The smallest matrix size of the workload at its low rank fractions (at most two cases)."""
+    uniq = sorted(set(tuple(c[:3]) for c in cases), key=lambda c: oracle_flops(*c))
+    d0 = min(c[0] * c[1] for c in uniq)
+    pick = [c for c in uniq if c[0] * c[1] == d0 and c[2] < min(c[0], c[1])][:2]
+    return pick or [uniq[0]]
 
 
 def time_oracle(cases, steps, warmup):
@@ -188,7 +208,7 @@ def time_oracle(cases, steps, warmup):
             times.append(dt)
     ms = sum(times) / len(times)
     f_sample = sum(oracle_flops(*c) for c in sample)
-    f_full = sum(oracle_flops(*c) for c in cases)
+    f_full = sum(oracle_flops(*c[:3]) for c in cases)
     return ms, sample, ms * f_full / f_sample, orc.num_threads()
 
 
@@ -197,7 +217,7 @@ def run_reference(args):
     if rank != 0:
         return
     from paper_2504_05295_b200 import inputs
-    cases = parse_cases(args.cases, inputs)
+    cases = parse_cases(args.cases, inputs, args.workload)
     steps, warmup = max(1, min(args.steps, 2)), min(args.warmup, 1)
     ms, sample, projected, cores = time_oracle(cases, steps, warmup)
     desc = ("float64 CPU oracle, one step each on " + ", ".join(f"{m}x{n} r={r}" for m, n, r in sample) +
@@ -215,8 +235,10 @@ def run_reference(args):
 
 
 def workload_name(cases):
-    return ("square fp32 sweep: " + ", ".join(f"{m}^2 r={r}" for m, n, r in cases) +
-            "; seeded low-rank (rank 64, s_i=2^-i/2) + 0.1 N(0,1) gradients")
+    import collections
+    cnt = collections.Counter((c[0], c[1], c[2], "bf16 G" if case_gbytes(c) == 2 else "fp32 G") for c in cases)
+    return ("; ".join(f"{k}x {m}x{n} r={r} {g}" if k > 1 else f"{m}x{n} r={r} {g}" for (m, n, r, g), k in cnt.items()) +
+            "; fp32 X, M, Q; seeded low-rank (rank 64, s_i=2^-i/2) + 0.1 N(0,1) gradients")
 
 
 # ---------------------------------------------------------------------------
@@ -238,15 +260,18 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     build.build()
     peaks = load_peaks()
-    cases = parse_cases(args.cases, inputs)
+    cases = parse_cases(args.cases, inputs, args.workload)
     dev = torch.device("cuda", local)
     stream = torch.cuda.current_stream()
     sptr = int(stream.cuda_stream)
 
     # inputs resident in HBM: per case X, M, Q and a ring of two gradients
     state = []
-    for k, (m, n, r) in enumerate(cases):
-        pb = inputs.make_problem(m, n, r, seed=rank, k=k, ks=64, device=dev, keep_signal=False)
+    grouped = args.workload in ("llama8b", "llama405b") and not args.cases
+    for k, c in enumerate(cases):
+        m, n, r = c[:3]
+        pb = inputs.make_problem(m, n, r, seed=rank, k=k, ks=64, device=dev, keep_signal=False,
+                                 g_dtype=torch.bfloat16 if case_gbytes(c) == 2 else torch.float32)
         gs = [pb.grad(t) for t in range(2)]
         d = torch.zeros(r, device=dev)
         descs = [binding.matrix_desc(pb.X, pb.M, g, pb.Q, d) for g in gs]
@@ -254,9 +279,13 @@ def run_ours(args):
     torch.cuda.synchronize()
 
     opt = binding.Dion(mu=MU, eps=EPS, precision=args.precision, orth=args.orth, engine=args.engine, device=local)
-    need = max(opt.workspace_bytes(m, n, r) for m, n, r in cases)
+    need = max(opt.workspace_bytes(*c[:3]) for c in cases)
+    packed = [binding.Dion.pack([st["descs"][i] for st in state]) for i in range(2)]
 
     def one_step(t, per_case_events=None):
+        if grouped:     # one dion_step_grouped call over the whole list
+            opt.step_grouped_packed(packed[t % 2], len(state), ETA, sptr)
+            return
         for ci, st in enumerate(state):
             if per_case_events is not None:
                 e0 = torch.cuda.Event(enable_timing=True); e0.record(stream)
@@ -300,7 +329,7 @@ def run_ours(args):
         dist.all_reduce(t_, op=dist.ReduceOp.MAX)
         ms_step = float(t_.item())
 
-    case_ms = [sum(a.elapsed_time(b) for a, b in ev) / len(ev) for ev in case_events]
+    case_ms = [sum(a.elapsed_time(b) for a, b in ev) / len(ev) if ev else None for ev in case_events]
 
     # ---- end to end: host gradients in, column norms out, through the same C-ABI call ----
     host_g = [st["G"][0].cpu().pin_memory() for st in state]
@@ -334,10 +363,12 @@ def run_ours(args):
     opt.orth_rounds()
     case_rounds = []
     for ci, st in enumerate(state):
+        m_, n_, r_ = cases[ci][:3]
+        if orth_mode(m_, n_, r_, args.orth) != 2:
+            case_rounds.append(None)
+            continue
         opt.step_desc(st["descs"][1], ETA, sptr)
-        nr = opt.orth_rounds()
-        m_, n_, r_ = cases[ci]
-        case_rounds.append(nr if orth_mode(m_, n_, r_, args.orth) == 2 else None)
+        case_rounds.append(opt.orth_rounds())
 
     if rank != 0:
         opt.close()
@@ -348,8 +379,10 @@ def run_ours(args):
     # ---- roofline of the dominant phase ---------------------------------------------------
     tot_fl = {p: 0.0 for p in binding.PHASES}
     tot_by = {p: 0.0 for p in binding.PHASES}
-    for (m, n, r), nr in zip(cases, case_rounds):
-        fl, by = phase_flops(m, n, r, args.orth, rounds=nr), phase_bytes(m, n, r, args.orth, rounds=nr)
+    for c, nr in zip(cases, case_rounds):
+        m, n, r = c[:3]
+        fl = phase_flops(m, n, r, args.orth, rounds=nr)
+        by = phase_bytes(m, n, r, args.orth, gbytes=case_gbytes(c), rounds=nr)
         for p in binding.PHASES:
             tot_fl[p] += fl[p]; tot_by[p] += by[p]
     # The dominant kernel is the tcgen05 contraction kernel: the four large products plus the
@@ -401,24 +434,27 @@ def run_ours(args):
     cpu = None
     if world == 1 and not args.no_cpu:
         ms_o, sample, projected, cores = time_oracle(cases, 1, 0)
-        gpu_same = sum(case_ms[cases.index(c)] for c in sample)
+        idx = [[tuple(x[:3]) for x in cases].index(c) for c in sample]
+        gpu_same = None if grouped else sum(case_ms[i] for i in idx)
         cpu = {"value": ms_o, "unit": UNIT, "cores": cores, "kind": "oracle",
                "sample": "one float64 oracle step each on " + ", ".join(f"{m}x{n} r={r}" for m, n, r in sample) +
-                         " (2 of the sweep's cases); value = their summed host time",
+                         "; value = their summed host time",
                "gpu_ms_same_cases": gpu_same, "projected_full_sweep_ms": projected}
 
     line = {"metric": METRIC, "value": ms_step, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": False, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16" if args.precision == binding.PREC_BF16_OPERANDS else "f32",
             "data": "synthetic",
-            "config": {"workload": workload_name(cases), "cases": [list(c) for c in cases],
+            "config": {"workload": workload_name(cases), "workload_id": args.workload, "n_matrices": len(cases),
+                       "call": "one dion_step_grouped call per step" if grouped else "one dion_step call per matrix per step",
                        "engine": ["auto", "simt", "tensor"][args.engine],
                        "precision": ["fp32 (3xTF32 on tensor cores / FMA)", "bf16 operands"][args.precision],
                        "orth": ["auto", "cholqr2", "shifted3", "householder"][args.orth],
-                       "l2": "inputs larger than L2: the sweep's 4 GB of X, M, G cycle through between repeats",
+                       "l2": "inputs larger than L2: the workload's X, M, G (GBs) cycle through between repeats",
                        "replicas": world, "workspace_bytes": need},
-            "cases": [{"m": m, "n": n, "r": r, "ms": ms, "adaptive_orth_rounds": nr}
-                      for (m, n, r), ms, nr in zip(cases, case_ms, case_rounds)],
+            "cases": ([] if len(cases) > 32 else
+                      [{"m": c[0], "n": c[1], "r": c[2], "ms": ms, "adaptive_orth_rounds": nr}
+                       for c, ms, nr in zip(cases, case_ms, case_rounds)]),
             "phases": phases, "roofline": roof, "cpu_baseline": cpu,
             "e2e": {"value": e2e_ms, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "steps": e2e_steps},
@@ -436,6 +472,8 @@ def main():
     ap.add_argument("--steps", type=int, default=3)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="sweep", choices=["sweep", "large", "llama8b", "llama405b"],
+                    help="sweep: nine square fp32 cases (default); large: 16384^2 / 32768^2; llama8b / llama405b: grouped lists")
     ap.add_argument("--cases", default="", help="subset as d:r,d:r (default: the nine cases of the square sweep)")
     ap.add_argument("--engine", type=int, default=0, help="0 auto, 1 simt, 2 tensor")
     ap.add_argument("--precision", type=int, default=0, help="0 fp32, 1 bf16 operands")
