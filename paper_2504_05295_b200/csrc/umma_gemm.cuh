@@ -373,7 +373,8 @@ struct Cfg {
   static constexpr int B_BYTES = BN * 128;
   static constexpr int STAGE_BYTES = (BF16 ? 1 : 2) * (A_BYTES + B_BYTES);
   static constexpr int STAGES = (192 * 1024) / STAGE_BYTES;
-  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 + 512;
+  static constexpr int G16_BYTES = BF16 ? 0 : BM * 32 * 2;   // bf16 addend tile of the TMA variant (per stage)
+  static constexpr int SMEM_BYTES = STAGES * (STAGE_BYTES + G16_BYTES) + 1024 + 512;
   static constexpr int A_CHUNKS = BM * 8 / NUM_PROD_THREADS;  // 16-byte chunks per producer thread
   static constexpr int B_CHUNKS = BN * 8 / NUM_PROD_THREADS;
   static constexpr int ACCS = SPLIT ? 2 : 1;                 // accumulators per tile
@@ -401,8 +402,10 @@ __global__ void __launch_bounds__(TMA ? NUM_THREADS_TMA : NUM_THREADS, 1) k_gemm
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   unsigned char* smem_al = smem_raw + (smem_base - smem_u32(smem_raw));
   // control block after the stages
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem_al + STAGES * C::STAGE_BYTES);
-  const uint32_t bar0 = smem_base + STAGES * C::STAGE_BYTES;
+  // after the stages: the bf16 addend staging of the TMA variant, then the control block
+  const uint32_t g16_base = smem_base + STAGES * C::STAGE_BYTES;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem_al + STAGES * (C::STAGE_BYTES + C::G16_BYTES));
+  const uint32_t bar0 = smem_base + STAGES * (C::STAGE_BYTES + C::G16_BYTES);
   auto full_bar = [&](int s) { return bar0 + 8u * s; };
   auto empty_bar = [&](int s) { return bar0 + 8u * (STAGES + s); };
   auto accf_bar = [&](int b) { return bar0 + 8u * (2 * STAGES + b); };
@@ -517,6 +520,22 @@ __global__ void __launch_bounds__(TMA ? NUM_THREADS_TMA : NUM_THREADS, 1) k_gemm
       // in-place conversion of the tiles the TMA warp loaded; the split is elementwise, so
       // each thread simply takes the 16-byte units ptid, ptid + 256, ... of the buffers
       const bool add = (g.a2_mode == ADD_F32);
+      const bool add16 = (g.a2_mode == ADD_BF16);
+      // bf16 addend: where the four bf16 values of each of this thread's A units sit in the
+      // (unswizzled) staging tile; the unit index is un-swizzled back to (row, k)
+      uint32_t g16off[C::A_CHUNKS];
+#pragma unroll
+      for (int l = 0; l < C::A_CHUNKS; ++l) {
+        const uint32_t u = (uint32_t)ptid + l * NUM_PROD_THREADS;
+        if (!A_MN) {
+          const uint32_t row = u >> 3, minor = (u & 7u) ^ (row & 7u);
+          g16off[l] = row * 64u + minor * 8u;
+        } else {
+          const uint32_t c = u >> 8, kk = (u >> 3) & 31u, qs = u & 7u;
+          const uint32_t q = ((((qs >> 1) ^ (kk & 3u))) << 1) | (qs & 1u);
+          g16off[l] = kk * 256u + (c * 32u + q * 4u) * 2u;
+        }
+      }
       int stage = 0;
       uint32_t phase = 0;
       bool alive = true;
@@ -524,6 +543,7 @@ __global__ void __launch_bounds__(TMA ? NUM_THREADS_TMA : NUM_THREADS, 1) k_gemm
         const Item it = decode_item<BN, BKE>(p, item);
         for (int kb = it.kb0; kb < it.kb1; ++kb) {
           if (!mbar_wait(raw_bar(stage), phase, dead, p.status)) { alive = false; break; }
+          const uint32_t sg16 = g16_base + stage * C::G16_BYTES;
           const uint32_t sa = smem_base + stage * C::STAGE_BYTES + (uint32_t)ptid * 16u;
           const uint32_t sa_lo = sa + C::A_BYTES;
           const uint32_t sb = sa + 2 * C::A_BYTES;
@@ -533,13 +553,20 @@ __global__ void __launch_bounds__(TMA ? NUM_THREADS_TMA : NUM_THREADS, 1) k_gemm
           for (int l = 0; l < C::A_CHUNKS; ++l) {
             xa[l] = lds128(sa + l * (NUM_PROD_THREADS * 16));
             if (add) ga[l] = lds128(sa_lo + l * (NUM_PROD_THREADS * 16));
+            if (add16) {
+              uint32_t w0, w1;
+              asm volatile("ld.shared.v2.b32 {%0, %1}, [%2];" : "=r"(w0), "=r"(w1) : "r"(sg16 + g16off[l]) : "memory");
+              const __nv_bfloat162 lo2 = *reinterpret_cast<const __nv_bfloat162*>(&w0);
+              const __nv_bfloat162 hi2 = *reinterpret_cast<const __nv_bfloat162*>(&w1);
+              ga[l] = make_float4(__low2float(lo2), __high2float(lo2), __low2float(hi2), __high2float(hi2));
+            }
           }
 #pragma unroll
           for (int l = 0; l < C::B_CHUNKS; ++l) xb[l] = lds128(sb + l * (NUM_PROD_THREADS * 16));
 #pragma unroll
           for (int l = 0; l < C::A_CHUNKS; ++l) {
             float4 x = xa[l];
-            if (add) {
+            if (add || add16) {
               x.x += ga[l].x; x.y += ga[l].y; x.z += ga[l].z; x.w += ga[l].w;
               sts128(sa + l * (NUM_PROD_THREADS * 16), x);
             }
@@ -613,7 +640,8 @@ __global__ void __launch_bounds__(TMA ? NUM_THREADS_TMA : NUM_THREADS, 1) k_gemm
     // ------------------------------------------------------------ TMA issuer
     if (lane == 0) {
       const bool add = (g.a2_mode == ADD_F32);
-      const uint32_t bytes = (uint32_t)(C::A_BYTES * (add ? 2 : 1) + C::B_BYTES);
+      const bool add16 = (g.a2_mode == ADD_BF16);
+      const uint32_t bytes = (uint32_t)(C::A_BYTES * (add ? 2 : 1) + C::B_BYTES + (add16 ? C::G16_BYTES : 0));
       int stage = 0;
       uint32_t phase = 0;
       bool alive = true;
@@ -628,6 +656,10 @@ __global__ void __launch_bounds__(TMA ? NUM_THREADS_TMA : NUM_THREADS, 1) k_gemm
           const uint32_t sb = sa + 2 * C::A_BYTES;
           const uint32_t bar = raw_bar(stage);
           mbar_expect_tx(bar, bytes);
+          if (add16) {   // bf16 addend tile, unswizzled: [row][32 k] or [k][128 rows]
+            if (!A_MN) tma_load_2d(g16_base + stage * C::G16_BYTES, &p.tmA2, k0, row0a, bar);
+            else tma_load_2d(g16_base + stage * C::G16_BYTES, &p.tmA2, row0a, k0, bar);
+          }
           if (!A_MN) {
             tma_load_2d(sa, &p.tmA, k0, row0a, bar);
             if (add) tma_load_2d(sa_lo, &p.tmA2, k0, row0a, bar);
@@ -766,6 +798,22 @@ inline EncodeTiledFn encode_tiled_fn() {
 //   128-byte swizzle.  mn_major = true: memory is [K][rows] with k stride `ld`; box = 32
 //   rows x 32 k, 128-byte swizzle with 32-byte atoms (the layout the TF32 MMA reads for a
 //   row-contiguous operand).
+// Tensor map of the bf16 addend of A: unswizzled tiles, [128 rows][32 k] (k contiguous) or
+// [32 k][128 rows] (row index contiguous).
+inline bool make_addend16_map(CUtensorMap* map, const void* ptr, i64 rows, i64 K, i64 ld, bool mn_major) {
+  EncodeTiledFn fn = encode_tiled_fn();
+  if (fn == nullptr) return false;
+  cuuint64_t gdim[2], gstride[1];
+  cuuint32_t box[2], estr[2] = {1, 1};
+  if (!mn_major) { gdim[0] = (cuuint64_t)K; gdim[1] = (cuuint64_t)rows; box[0] = 32; box[1] = BM; }
+  else { gdim[0] = (cuuint64_t)rows; gdim[1] = (cuuint64_t)K; box[0] = BM; box[1] = 32; }
+  gstride[0] = (cuuint64_t)ld * 2;
+  const CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), gdim, gstride, box, estr,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
 inline bool make_operand_map(CUtensorMap* map, const void* ptr, i64 rows, i64 K, i64 ld, bool mn_major, int box_rows) {
   EncodeTiledFn fn = encode_tiled_fn();
   if (fn == nullptr) return false;
@@ -867,7 +915,12 @@ inline int umma_try_launch(const GemmArgs& g_in, int precision, int sm_count, fl
   p.kc = 32;   // 1024 (fp32) or 2048 (bf16) k elements per accumulation chain
   const int grid = p.num_items < sm_count ? p.num_items : sm_count;
   // TMA variant: fp32 mode, fp32 (or no) addend, dimensions the tensor maps can describe
-  bool tma = !bf16 && g.a2_mode != ADD_BF16 && !(debug & 16) && g.M < (1ll << 31) && g.N < (1ll << 31) && g.K < (1ll << 31);
+  bool tma = !bf16 && !(debug & 16) && g.M < (1ll << 31) && g.N < (1ll << 31) && g.K < (1ll << 31);
+  if (tma && g.a2_mode == ADD_BF16) {   // the bf16 addend needs 16-byte aligned rows for its tensor map
+    const i64 ld2 = a_mn ? g.a2_sk : g.a2_si;
+    tma = (ld2 % 8 == 0) && (((uintptr_t)g.A2 % 16) == 0) &&
+          make_addend16_map(&p.tmA2, g.A2, g.M, g.K, ld2, a_mn);
+  }
   if (tma) {
     const i64 lda = a_mn ? g.a_sk : g.a_si, ldb = b_mn ? g.b_sk : g.b_sn;
     tma = make_operand_map(&p.tmA, g.A, g.M, g.K, lda, a_mn, BM) && make_operand_map(&p.tmB, g.B, g.N, g.K, ldb, b_mn, BN);
