@@ -143,7 +143,12 @@ int dion_step(dion_ctx* ctx, const dion_matrix* a, float lr, void* cuda_stream);
 
 /* The same step on `count` independent matrices (the paper batches matrices of
  * identical shape; Section 4.1).  Equivalent to `count` dion_step calls in any
- * order.  `list` is a HOST array.  count == 0 is a no-op. */
+ * order, bit for bit.  `list` is a HOST array.  count == 0 is a no-op.
+ * Matrices of identical (m, n, r) are stepped together, up to 64 at a time: their
+ * large products are launched one after another, the small kernels of the
+ * factorization once for all of them.  Each matrix of such a chain needs its own
+ * scratch slice, so the context's scratch grows to at most max(16 GiB,
+ * dion_config.workspace_bytes), or to one matrix's need if that is larger. */
 int dion_step_grouped(dion_ctx* ctx, const dion_matrix* list, int count, float lr, void* cuda_stream);
 
 /* One Lazy-Dion step (Algorithm 6): M <- M + G; if refresh != 0, Q <-

@@ -18,6 +18,8 @@ using namespace dion;
 namespace {
 
 constexpr int MAX_FLAG_SLOTS = 4096;      // step slots of OS_SLOT_INTS ints each
+constexpr int MAX_CHAIN = 64;              // matrices of one shape stepped together by dion_step_grouped
+constexpr size_t GROUP_SCRATCH_BYTES = (size_t)16 << 30;  // scratch dion_step_grouped may use for that (or cfg.workspace_bytes)
 constexpr int MAX_ROUNDS = 6;             // adaptive Cholesky QR rounds
 constexpr float FLOOR_REL = 1e-4f;        // pivot floor relative to the column's squared norm
 constexpr float GOOD_REL = 1e-4f;         // smallest relative pivot of a round that one more round can finish
@@ -120,6 +122,7 @@ GemmArgs gemm_args() {
   memset(&g, 0, sizeof(g));
   g.alpha = 1.f;
   g.batch = 1;
+  g.batch2 = 1;
   g.splits = 1;
   return g;
 }
@@ -128,12 +131,12 @@ GemmArgs gemm_args() {
 int launch_gemm_simt(dion_ctx* c, GemmArgs g, cudaStream_t st, float* part, i64 part_floats,
                      bool force64) {
   if (g.M <= 0 || g.N <= 0) return DION_OK;
-  const i64 t128 = ((g.M + 127) / 128) * ((g.N + 127) / 128) * g.batch;
+  const i64 t128 = ((g.M + 127) / 128) * ((g.N + 127) / 128) * g.batch * (g.batch2 > 1 ? g.batch2 : 1);
   const bool use128 = !force64 && t128 >= c->sm_count;
   const int BMN = use128 ? 128 : 64;
   const i64 gm = (g.M + BMN - 1) / BMN, gn = (g.N + BMN - 1) / BMN;
   int splits = 1;
-  if (!use128 && !force64 && g.epi == EPI_STORE && g.batch == 1 && part != nullptr && g.alpha_dev == nullptr) {
+  if (!use128 && !force64 && g.epi == EPI_STORE && g.batch == 1 && g.batch2 <= 1 && part != nullptr && g.alpha_dev == nullptr) {
     const i64 tiles = gm * gn;
     i64 want = (2 * (i64)c->sm_count + tiles - 1) / tiles;
     const i64 kmax = g.K / 128;
@@ -145,7 +148,9 @@ int launch_gemm_simt(dion_ctx* c, GemmArgs g, cudaStream_t st, float* part, i64 
   g.splits = splits;
   g.part = part;
   if (gm > 65535) return DION_ERR_UNSUPPORTED;
-  dim3 grid((unsigned)gn, (unsigned)gm, (unsigned)(splits > 1 ? splits : g.batch));
+  if (g.batch2 < 1) g.batch2 = 1;
+  if (splits > 1 && g.batch2 > 1) return DION_ERR_INVALID;
+  dim3 grid((unsigned)gn, (unsigned)gm, (unsigned)(splits > 1 ? splits : g.batch * g.batch2));
   if (use128) k_gemm_simt<128, 128, 8, 8, 8><<<grid, 256, 0, st>>>(g);
   else k_gemm_simt<64, 64, 16, 4, 4><<<grid, 256, 0, st>>>(g);
   DION_CHECK_LAUNCH(c);
@@ -182,28 +187,48 @@ struct PhaseScope {
   }
 };
 
+// One launch chain works on `nb` matrices of identical (m, n, r) at a time (nb = 1 for
+// dion_step): the large products are launched per matrix, the small kernels of the
+// factorization once for all of them (one block or batch entry per matrix).  Matrix b
+// uses the scratch slice that starts b * wstride floats after `ws` and the state slot
+// b * OS_SLOT_INTS ints after `os`.
 struct StepCtx {
   dion_ctx* c;
   cudaStream_t st;
   float* ws;
   Layout L;
-  int* os;    // this step's device state slot (OS_* ints)
+  int nb;
+  i64 wstride;
+  int* os;    // first device state slot (OS_* ints)
   int* flag;  // = os + OS_FAIL: the step must not write its outputs
   bool tensor;  // tensor-core engine allowed for this matrix
   bool in_orth; // inside the orthonormalization (for the profiling phases)
+  float* W(int b, i64 off) const { return ws + (i64)b * wstride + off; }
+  int* OS(int b) const { return os + (i64)b * OS_SLOT_INTS; }
 };
 
 // Engine dispatch: tensor cores when the product qualifies, else fp32 FMA.
-int launch_gemm(StepCtx& s, const GemmArgs& g, bool force64 = false) {
+// `b`: the matrix of the batch the product belongs to (selects its split-K scratch).
+int launch_gemm(StepCtx& s, const GemmArgs& g, int b = 0, bool force64 = false) {
   if (s.tensor && !force64) {
     PhaseScope ps(s.c, s.st, s.in_orth ? DION_PHASE_ORTH_GEMM : -1);
-    const int rc = umma_try_launch(g, s.c->cfg.precision, s.c->sm_count, s.ws + s.L.part, s.L.part_floats,
+    const int rc = umma_try_launch(g, s.c->cfg.precision, s.c->sm_count, s.W(b, s.L.part), s.L.part_floats,
                                    s.c->dev_ints, s.st);
     if (rc > 0) { s.c->launches += rc; return DION_OK; }
     if (rc < 0) return rc;
     if (s.c->cfg.engine == DION_ENGINE_TENSOR) return DION_ERR_UNSUPPORTED;
   }
-  return launch_gemm_simt(s.c, g, s.st, s.ws + s.L.part, s.L.part_floats, force64);
+  return launch_gemm_simt(s.c, g, s.st, s.W(b, s.L.part), s.L.part_floats, force64);
+}
+
+// Shifts the workspace-resident operands of a product to matrix b of the batch.
+GemmArgs for_matrix(const StepCtx& s, GemmArgs g, int b, bool a_ws, bool b_ws, bool c_ws) {
+  const i64 o = (i64)b * s.wstride;
+  if (a_ws) g.A += o;
+  if (b_ws) g.B += o;
+  if (c_ws) g.C += o;
+  if (g.skip_flag != nullptr) g.skip_flag += (i64)b * OS_SLOT_INTS;
+  return g;
 }
 
 constexpr i64 NBO = 512;  // outer block of the two-level Cholesky
@@ -215,11 +240,21 @@ int grid_for(const dion_ctx* c, i64 total) {
   return (int)blocks;
 }
 
+// Marks a small (FMA-engine) product as batched over the nb matrices of the chain.
+void over_batch(const StepCtx& s, GemmArgs& g) {
+  g.batch2 = s.nb;
+  g.bs2 = s.wstride;
+  g.skip_stride = OS_SLOT_INTS;
+}
+
 // Inverse of a lower-triangular matrix by doubling, on the diagonal square [o, o+sz):
 // [[L11,0],[L21,L22]]^-1 = [[X11,0],[-X22 L21 X11, X22]], for block sizes b_from, 2 b_from, ...
 // while b < sz.  The diagonal blocks of size b_from of Linv must already hold their inverses.
-int trtri_levels(StepCtx& s, const float* Gm, float* Linv, float* Tbuf, i64 r, i64 o, i64 sz, i64 b_from,
-                 const int* skip, int precise) {
+// Offsets are relative to each matrix's scratch slice.
+int trtri_levels(StepCtx& s, i64 r, i64 o, i64 sz, i64 b_from, const int* skip, int precise) {
+  const float* Gm = s.ws + s.L.Gram;
+  float* Linv = s.ws + s.L.Linv;
+  float* Tbuf = s.ws + s.L.Tbuf;
   for (i64 b = b_from; b < sz; b *= 2) {
     const i64 nfull = sz / (2 * b);
     const i64 tail0 = nfull * 2 * b;
@@ -231,7 +266,7 @@ int trtri_levels(StepCtx& s, const float* Gm, float* Linv, float* Tbuf, i64 r, i
       if (rows <= 0 || batch <= 0) continue;
       const i64 off21 = (base + b) * r + base, off11 = base * r + base, off22 = (base + b) * r + (base + b);
       const i64 bs = 2 * b * (r + 1);
-      const bool big = b >= NBO;   // large blocks: one launch per pair, tensor cores where they qualify
+      const bool big = b >= NBO;   // large blocks: one launch per pair and matrix, tensor cores where they qualify
       const int launches = big ? batch : 1;
       for (int q = 0; q < launches; ++q) {
         const i64 sh = big ? (i64)q * bs : 0;
@@ -246,11 +281,11 @@ int trtri_levels(StepCtx& s, const float* Gm, float* Linv, float* Tbuf, i64 r, i
         g2.B = Tbuf + off21 + sh; g2.b_sk = r; g2.b_sn = 1;
         g2.C = Linv + off21 + sh; g2.ldc = r; g2.epi = EPI_STORE; g2.alpha = -1.f; g2.skip_flag = skip; g2.precise = precise;
         if (big) {
-          DION_TRY(launch_gemm(s, g1));
-          DION_TRY(launch_gemm(s, g2));
+          for (int m = 0; m < s.nb; ++m) DION_TRY(launch_gemm(s, for_matrix(s, g1, m, true, true, true), m));
+          for (int m = 0; m < s.nb; ++m) DION_TRY(launch_gemm(s, for_matrix(s, g2, m, true, true, true), m));
         } else {
-          g1.batch = batch; g1.bsA = bs; g1.bsB = bs; g1.bsC = bs;
-          g2.batch = batch; g2.bsA = bs; g2.bsB = bs; g2.bsC = bs;
+          g1.batch = batch; g1.bsA = bs; g1.bsB = bs; g1.bsC = bs; over_batch(s, g1);
+          g2.batch = batch; g2.bsA = bs; g2.bsB = bs; g2.bsC = bs; over_batch(s, g2);
           DION_TRY(launch_gemm_simt(s.c, g1, s.st, nullptr, 0, false));
           DION_TRY(launch_gemm_simt(s.c, g2, s.st, nullptr, 0, false));
         }
@@ -260,13 +295,13 @@ int trtri_levels(StepCtx& s, const float* Gm, float* Linv, float* Tbuf, i64 r, i
   return DION_OK;
 }
 
-// Cholesky of the diagonal square [o, o+sz) of Gm (sz <= NBO), right-looking with 64-wide
-// blocks on the FMA engine, followed by the inverse of that square's factor into Linv.
-int potrf_inner(StepCtx& s, float* Gm, i64 r, i64 o, i64 sz, const float* shift, bool adaptive) {
+// Cholesky of the diagonal square [o, o+sz) of each Gram matrix (sz <= NBO), right-looking with
+// 64-wide blocks on the FMA engine, followed by the inverse of that square's factor into Linv.
+int potrf_inner(StepCtx& s, i64 r, i64 o, i64 sz, const float* shift, bool adaptive) {
   dion_ctx* c = s.c;
+  float* Gm = s.ws + s.L.Gram;
   float* Dinv = s.ws + s.L.Dinv;
   float* Linv = s.ws + s.L.Linv;
-  float* Tbuf = s.ws + s.L.Tbuf;
   const float* gdiag = s.ws + s.L.gdiag;
   int* status = c->dev_ints;
   const int* skip = adaptive ? (s.os + OS_DONE) : nullptr;
@@ -275,8 +310,8 @@ int potrf_inner(StepCtx& s, float* Gm, i64 r, i64 o, i64 sz, const float* shift,
     float* Ajj = Gm + j0 * r + j0;
     float* Dj = Dinv + (j0 / NB) * (NB * NB);
     float* DPj = s.ws + s.L.DinvP + (j0 / NB) * (NB * NB);
-    k_potrf_diag<<<1, 256, 0, s.st>>>(Ajj, r, jb, Dj, DPj, shift, gdiag + j0, adaptive ? FLOOR_REL : 0.f, s.os,
-                                      adaptive ? 1 : 0, status);
+    k_potrf_diag<<<s.nb, 256, 0, s.st>>>(Ajj, r, jb, Dj, DPj, shift, gdiag + j0, adaptive ? FLOOR_REL : 0.f, s.os,
+                                         adaptive ? 1 : 0, status, s.wstride);
     DION_CHECK_LAUNCH(c);
     const i64 rem = o + sz - j0 - jb;
     if (rem > 0) {
@@ -286,37 +321,44 @@ int potrf_inner(StepCtx& s, float* Gm, i64 r, i64 o, i64 sz, const float* shift,
       g.A = panel; g.a_si = r; g.a_sk = 1;
       g.B = DPj; g.b_sk = 1; g.b_sn = NB;
       g.C = panel; g.ldc = r; g.epi = EPI_STORE; g.skip_flag = skip;
+      over_batch(s, g);
       DION_TRY(launch_gemm_simt(c, g, s.st, nullptr, 0, true));
       GemmArgs t = gemm_args();  // A22 -= panel * panel^T (lower tiles)
       t.M = rem; t.N = rem; t.K = jb;
       t.A = panel; t.a_si = r; t.a_sk = 1;
       t.B = panel; t.b_sk = 1; t.b_sn = r;
       t.C = Gm + (j0 + jb) * r + (j0 + jb); t.ldc = r; t.epi = EPI_SUB; t.tri = TRI_LOWER; t.skip_flag = skip;
-      DION_TRY(launch_gemm_simt(c, t, s.st, nullptr, 0, false));
+      over_batch(s, t);
+      DION_TRY(launch_gemm_simt(c, t, s.st, nullptr, 0, true));
     }
   }
-  k_linv_init<<<grid_for(c, sz * sz), 256, 0, s.st>>>(Linv, r, o, sz, Dinv, skip);
-  DION_CHECK_LAUNCH(c);
-  return trtri_levels(s, Gm, Linv, Tbuf, r, o, sz, NB, skip, 0);
+  {
+    dim3 grid((unsigned)grid_for(c, sz * sz), (unsigned)s.nb);
+    k_linv_init<<<grid, 256, 0, s.st>>>(Linv, r, o, sz, Dinv, skip, s.wstride);
+    DION_CHECK_LAUNCH(c);
+  }
+  return trtri_levels(s, r, o, sz, NB, skip, 0);
 }
 
-// Two-level blocked Cholesky of the r x r matrix Gm (lower) and the full inverse of its
+// Two-level blocked Cholesky of each r x r Gram matrix (lower) and the full inverse of its
 // factor into Linv.  Outer blocks of 512 columns: the diagonal square is factored and
 // inverted by potrf_inner, the panel below it is multiplied by that inverse and the
 // trailing matrix is updated with one rank-512 product (tensor cores where it qualifies).
-int potrf_trtri(StepCtx& s, float* Gm, i64 r, const float* shift, bool adaptive) {
+int potrf_trtri(StepCtx& s, i64 r, const float* shift, bool adaptive) {
   dion_ctx* c = s.c;
+  float* Gm = s.ws + s.L.Gram;
   float* Linv = s.ws + s.L.Linv;
   float* Tbuf = s.ws + s.L.Tbuf;
   const int* skip = adaptive ? (s.os + OS_DONE) : nullptr;
   const int precise = adaptive ? 1 : 0;
   if (r > NBO) {
     // everything outside the diagonal squares starts at zero (the product U = P Linv^T reads whole tiles)
-    if (cudaMemsetAsync(Linv, 0, sizeof(float) * (size_t)r * (size_t)r, s.st) != cudaSuccess) return DION_ERR_CUDA;
+    for (int m = 0; m < s.nb; ++m)
+      if (cudaMemsetAsync(s.W(m, s.L.Linv), 0, sizeof(float) * (size_t)r * (size_t)r, s.st) != cudaSuccess) return DION_ERR_CUDA;
   }
   for (i64 J0 = 0; J0 < r; J0 += NBO) {
     const i64 sz = (r - J0 < NBO) ? (r - J0) : NBO;
-    DION_TRY(potrf_inner(s, Gm, r, J0, sz, shift, adaptive));
+    DION_TRY(potrf_inner(s, r, J0, sz, shift, adaptive));
     const i64 rem = r - J0 - sz;
     if (rem > 0) {
       float* panel = Gm + (J0 + sz) * r + J0;
@@ -326,62 +368,63 @@ int potrf_trtri(StepCtx& s, float* Gm, i64 r, const float* shift, bool adaptive)
       g.A = panel; g.a_si = r; g.a_sk = 1;
       g.B = Linv + J0 * r + J0; g.b_sk = 1; g.b_sn = r; g.klimit = 1;
       g.C = ptmp; g.ldc = r; g.epi = EPI_STORE; g.skip_flag = skip; g.precise = precise;
-      DION_TRY(launch_gemm(s, g));
-      k_copy_block<<<grid_for(c, rem * sz), 256, 0, s.st>>>(ptmp, r, panel, r, rem, sz, skip);
-      DION_CHECK_LAUNCH(c);
+      for (int m = 0; m < s.nb; ++m) DION_TRY(launch_gemm(s, for_matrix(s, g, m, true, true, true), m));
+      {
+        dim3 grid((unsigned)grid_for(c, rem * sz), (unsigned)s.nb);
+        k_copy_block<<<grid, 256, 0, s.st>>>(ptmp, r, panel, r, rem, sz, skip, s.wstride);
+        DION_CHECK_LAUNCH(c);
+      }
       GemmArgs t = gemm_args();  // A22 -= Lpanel * Lpanel^T (lower tiles)
       t.M = rem; t.N = rem; t.K = sz;
       t.A = panel; t.a_si = r; t.a_sk = 1;
       t.B = panel; t.b_sk = 1; t.b_sn = r;
       t.C = Gm + (J0 + sz) * r + (J0 + sz); t.ldc = r; t.epi = EPI_SUB; t.tri = TRI_LOWER; t.skip_flag = skip;
       t.precise = precise;
-      DION_TRY(launch_gemm(s, t));
+      for (int m = 0; m < s.nb; ++m) DION_TRY(launch_gemm(s, for_matrix(s, t, m, true, true, true), m));
     }
   }
-  if (r > NBO) DION_TRY(trtri_levels(s, Gm, Linv, Tbuf, r, 0, r, NBO, skip, precise));
+  if (r > NBO) DION_TRY(trtri_levels(s, r, 0, r, NBO, skip, precise));
   return DION_OK;
 }
 
-// One Cholesky-QR round: Pout = Pin * chol(Pin^T Pin)^-T.  rows x r panels, ld = r.
-// adaptive: pivots are floored, the round is skipped (Pout = Pin) once the panel is
-// orthonormal, and the round statistics are evaluated at the end.
-int cholqr_round(StepCtx& s, const float* Pin, float* Pout, i64 rows, i64 r, bool adaptive) {
+// One Cholesky-QR round on every matrix of the chain: Pout = Pin * chol(Pin^T Pin)^-T.
+// rows x r panels, ld = r; pin_off / pout_off are offsets in the scratch slice.
+// adaptive: columns with negligible pivots are deflated, the round is skipped (Pout = Pin)
+// once the panel is orthonormal, and the round statistics are evaluated at the end.
+int cholqr_round(StepCtx& s, i64 pin_off, i64 pout_off, i64 rows, i64 r, bool adaptive) {
   dion_ctx* c = s.c;
-  float* Gm = s.ws + s.L.Gram;
   const int* skip = adaptive ? (s.os + OS_DONE) : nullptr;
   GemmArgs g = gemm_args();
   g.M = r; g.N = r; g.K = rows;
-  g.A = Pin; g.a_si = 1; g.a_sk = r;
-  g.B = Pin; g.b_sk = r; g.b_sn = 1;
-  g.C = Gm; g.ldc = r; g.epi = EPI_STORE; g.tri = TRI_LOWER; g.skip_flag = skip; g.precise = adaptive ? 1 : 0;
-  DION_TRY(launch_gemm(s, g));
-  float* sh = s.ws + s.L.scal;
-  k_round_begin<<<1, 256, 0, s.st>>>(Gm, r, r, 0.f, s.ws + s.L.gdiag, sh, s.os, adaptive ? 1 : 0);
+  g.A = s.ws + pin_off; g.a_si = 1; g.a_sk = r;
+  g.B = s.ws + pin_off; g.b_sk = r; g.b_sn = 1;
+  g.C = s.ws + s.L.Gram; g.ldc = r; g.epi = EPI_STORE; g.tri = TRI_LOWER; g.skip_flag = skip; g.precise = adaptive ? 1 : 0;
+  for (int m = 0; m < s.nb; ++m) DION_TRY(launch_gemm(s, for_matrix(s, g, m, true, true, true), m));
+  k_round_begin<<<s.nb, 256, 0, s.st>>>(s.ws + s.L.Gram, r, r, 0.f, s.ws + s.L.gdiag, s.ws + s.L.scal, s.os,
+                                        adaptive ? 1 : 0, s.wstride);
   DION_CHECK_LAUNCH(c);
-  DION_TRY(potrf_trtri(s, Gm, r, nullptr, adaptive));
+  DION_TRY(potrf_trtri(s, r, nullptr, adaptive));
   if (adaptive) {
-    const i64 total = rows * r;
-    int blocks = (int)((total + 255) / 256);
-    if (blocks > 8 * c->sm_count) blocks = 8 * c->sm_count;
-    k_copy_panel<<<blocks, 256, 0, s.st>>>(Pin, r, Pout, r, rows, r, nullptr, s.os + OS_DONE);
+    dim3 grid((unsigned)grid_for(c, rows * r), (unsigned)s.nb);
+    k_copy_panel<<<grid, 256, 0, s.st>>>(s.ws + pin_off, r, s.ws + pout_off, r, rows, r, nullptr, s.os + OS_DONE, s.wstride);
     DION_CHECK_LAUNCH(c);
   }
   GemmArgs u = gemm_args();
   u.M = rows; u.N = r; u.K = r;
-  u.A = Pin; u.a_si = r; u.a_sk = 1;
+  u.A = s.ws + pin_off; u.a_si = r; u.a_sk = 1;
   u.B = s.ws + s.L.Linv; u.b_sk = 1; u.b_sn = r; u.klimit = 1;
-  u.C = Pout; u.ldc = r; u.epi = EPI_STORE; u.skip_flag = skip; u.precise = adaptive ? 1 : 0;
-  DION_TRY(launch_gemm(s, u));
+  u.C = s.ws + pout_off; u.ldc = r; u.epi = EPI_STORE; u.skip_flag = skip; u.precise = adaptive ? 1 : 0;
+  for (int m = 0; m < s.nb; ++m) DION_TRY(launch_gemm(s, for_matrix(s, u, m, true, true, true), m));
   if (adaptive) {
-    k_round_end<<<1, 1, 0, s.st>>>(s.os, GOOD_REL, DONE_REL, c->dev_ints + 2);
+    k_round_end<<<s.nb, 1, 0, s.st>>>(s.os, GOOD_REL, DONE_REL, c->dev_ints + 2);
     DION_CHECK_LAUNCH(c);
   }
   return DION_OK;
 }
 
-int householder(StepCtx& s, float* A, float* V, i64 rows, i64 r) {
+int householder(StepCtx& s, float* A, float* V, i64 rows, i64 r, int b) {
   dion_ctx* c = s.c;
-  float* diag = s.ws + s.L.d;
+  float* diag = s.W(b, s.L.d);
   for (i64 j = 0; j < r; ++j) {
     k_hh_reflector<<<1, 1024, 0, s.st>>>(A, r, rows, j, V, r, diag);
     DION_CHECK_LAUNCH(c);
@@ -416,43 +459,43 @@ int resolve_orth(const dion_ctx* c, i64 r, i64 short_dim) {
   return mode;
 }
 
-// Orthonormalize the rows x r panel in ws.P0; returns the buffer that holds U.
-int orthonormalize(StepCtx& s, i64 rows, i64 r, i64 short_dim, float** U_out) {
-  float* P0 = s.ws + s.L.P0;
-  float* P1 = s.ws + s.L.P1;
+// Orthonormalize the rows x r panel in P0 of every matrix of the chain; *U_off is the
+// scratch offset of the buffer that holds U afterwards.
+int orthonormalize(StepCtx& s, i64 rows, i64 r, i64 short_dim, i64* U_off) {
   const int mode = resolve_orth(s.c, r, short_dim);
   if (mode == DION_ORTH_CHOLQR2) {
-    DION_TRY(cholqr_round(s, P0, P1, rows, r, false));
-    DION_TRY(cholqr_round(s, P1, P0, rows, r, false));
-    *U_out = P0;
+    DION_TRY(cholqr_round(s, s.L.P0, s.L.P1, rows, r, false));
+    DION_TRY(cholqr_round(s, s.L.P1, s.L.P0, rows, r, false));
+    *U_off = s.L.P0;
   } else if (mode == DION_ORTH_SHIFTED3) {
     // Adaptive rounds: the device decides after each round whether the panel is done.
     static_assert(MAX_ROUNDS % 2 == 0, "the result must end in P0");
     for (int it = 0; it < MAX_ROUNDS; it += 2) {
-      DION_TRY(cholqr_round(s, P0, P1, rows, r, true));
-      DION_TRY(cholqr_round(s, P1, P0, rows, r, true));
+      DION_TRY(cholqr_round(s, s.L.P0, s.L.P1, rows, r, true));
+      DION_TRY(cholqr_round(s, s.L.P1, s.L.P0, rows, r, true));
     }
-    k_orth_finish<<<1, 1, 0, s.st>>>(s.os, s.c->dev_ints);
+    k_orth_finish<<<s.nb, 1, 0, s.st>>>(s.os, s.c->dev_ints);
     s.c->launches++;
     if (cudaGetLastError() != cudaSuccess) return DION_ERR_CUDA;
-    *U_out = P0;
+    *U_off = s.L.P0;
   } else {
-    DION_TRY(householder(s, P0, P1, rows, r));
-    *U_out = P0;
+    for (int m = 0; m < s.nb; ++m) DION_TRY(householder(s, s.W(m, s.L.P0), s.W(m, s.L.P1), rows, r, m));
+    *U_off = s.L.P0;
   }
   return DION_OK;
 }
 
-int colnorm(StepCtx& s, const float* W, i64 rows, i64 r, float* out, i64 ldo, float* d_out) {
+// ColNorm of matrix b's W (rows x r, ld = r) into `out`.
+int colnorm(StepCtx& s, int b, const float* W, i64 rows, i64 r, float* out, i64 ldo, float* d_out) {
   dion_ctx* c = s.c;
   int chunks; i64 per;
   colnorm_plan(rows, r, c->sm_count, &chunks, &per);
-  float* part = s.ws + s.L.cn_part;
+  float* part = s.W(b, s.L.cn_part);
   dim3 grid((unsigned)((r + 127) / 128), (unsigned)chunks);
   k_colsumsq_partial<<<grid, 128, 0, s.st>>>(W, r, rows, r, per, part, nullptr);
   DION_CHECK_LAUNCH(c);
   k_colnorm_apply<<<grid, 128, 0, s.st>>>(W, r, rows, r, per, chunks, part, c->cfg.eps, out, ldo,
-                                         s.ws + s.L.d, d_out, c->dev_ints, s.flag);
+                                         s.W(b, s.L.d), d_out, c->dev_ints, s.OS(b) + OS_FAIL);
   DION_CHECK_LAUNCH(c);
   return DION_OK;
 }
@@ -487,50 +530,54 @@ int validate(const dion_matrix* a) {
   return DION_OK;
 }
 
-int begin_step(dion_ctx* c, const dion_matrix* a, cudaStream_t st, StepCtx* s) {
+int begin_step(dion_ctx* c, const dion_matrix* a, int nb, cudaStream_t st, StepCtx* s) {
   s->c = c;
   s->st = st;
   s->L = make_layout(c, a->m, a->n, a->r);
   s->ws = c->ws;
+  s->nb = nb;
+  s->wstride = s->L.total;
+  if (c->flag_cursor + nb > MAX_FLAG_SLOTS) c->flag_cursor = 0;   // the slots of a chain are contiguous
   s->os = c->dev_ints + 8 + (i64)c->flag_cursor * OS_SLOT_INTS;
   s->flag = s->os + OS_FAIL;
-  c->flag_cursor = (c->flag_cursor + 1) % MAX_FLAG_SLOTS;
+  c->flag_cursor = (c->flag_cursor + nb) % MAX_FLAG_SLOTS;
   s->tensor = (c->cfg.engine != DION_ENGINE_SIMT);
   s->in_orth = false;
-  if (cudaMemsetAsync(s->os, 0, sizeof(int) * OS_SLOT_INTS, st) != cudaSuccess) return DION_ERR_CUDA;
+  if (cudaMemsetAsync(s->os, 0, sizeof(int) * OS_SLOT_INTS * nb, st) != cudaSuccess) return DION_ERR_CUDA;
   return DION_OK;
 }
 
-// The launch chain of one Dion step (Algorithm 1 + 2).  Scratch must be large enough.
-int step_one(dion_ctx* c, const dion_matrix* a, float lr, cudaStream_t st) {
+// The launch chain of one Dion step (Algorithm 1 + 2) on `nb` matrices of identical
+// (m, n, r), phase by phase.  Scratch must hold nb slices.
+int step_batch(dion_ctx* c, const dion_matrix* const* list, int nb, float lr, cudaStream_t st) {
   StepCtx s;
-  DION_TRY(begin_step(c, a, st, &s));
-  const i64 m = a->m, n = a->n, r = a->r;
-  const int gmode = (a->g_dtype == DION_BF16) ? ADD_BF16 : ADD_F32;
-  float* P0 = s.ws + s.L.P0;
-  float* R = s.ws + s.L.R;
-  const float* Mp = (const float*)a->M;
+  const dion_matrix* a0 = list[0];
+  DION_TRY(begin_step(c, a0, nb, st, &s));
+  const i64 m = a0->m, n = a0->n, r = a0->r;
 
   // P = (M + G) Q
   {
   PhaseScope ps(c, st, DION_PHASE_P);
-  GemmArgs p = gemm_args();
-  p.M = m; p.N = r; p.K = n;
-  p.A = Mp; p.a_si = a->ldm; p.a_sk = 1;
-  p.A2 = a->G; p.a2_si = a->ldg; p.a2_sk = 1; p.a2_mode = gmode;
-  p.B = (const float*)a->Q; p.b_sk = a->ldq; p.b_sn = 1;
-  p.C = P0; p.ldc = r; p.epi = EPI_STORE;
-  // an ill-conditioned panel amplifies the error of P: use the accurate product there
-  p.precise = (resolve_orth(c, r, (m < n) ? m : n) == DION_ORTH_SHIFTED3) ? 1 : 0;
-  DION_TRY(launch_gemm(s, p));
+  for (int b = 0; b < nb; ++b) {
+    const dion_matrix* a = list[b];
+    GemmArgs p = gemm_args();
+    p.M = m; p.N = r; p.K = n;
+    p.A = (const float*)a->M; p.a_si = a->ldm; p.a_sk = 1;
+    p.A2 = a->G; p.a2_si = a->ldg; p.a2_sk = 1; p.a2_mode = (a->g_dtype == DION_BF16) ? ADD_BF16 : ADD_F32;
+    p.B = (const float*)a->Q; p.b_sk = a->ldq; p.b_sn = 1;
+    p.C = s.W(b, s.L.P0); p.ldc = r; p.epi = EPI_STORE;
+    // an ill-conditioned panel amplifies the error of P: use the accurate product there
+    p.precise = (resolve_orth(c, r, (m < n) ? m : n) == DION_ORTH_SHIFTED3) ? 1 : 0;
+    DION_TRY(launch_gemm(s, p, b));
+  }
   }
 
   // U = Orthonormalize(P)
-  float* U = nullptr;
+  i64 U_off = 0;
   {
   PhaseScope ps(c, st, DION_PHASE_ORTH);
   s.in_orth = true;
-  const int rc_orth = orthonormalize(s, m, r, (m < n) ? m : n, &U);
+  const int rc_orth = orthonormalize(s, m, r, (m < n) ? m : n, &U_off);
   s.in_orth = false;
   DION_TRY(rc_orth);
   }
@@ -538,56 +585,72 @@ int step_one(dion_ctx* c, const dion_matrix* a, float lr, cudaStream_t st) {
   // R = (M + G)^T U
   {
   PhaseScope ps(c, st, DION_PHASE_R);
-  GemmArgs w = gemm_args();
-  w.M = n; w.N = r; w.K = m;
-  w.A = Mp; w.a_si = 1; w.a_sk = a->ldm;
-  w.A2 = a->G; w.a2_si = 1; w.a2_sk = a->ldg; w.a2_mode = gmode;
-  w.B = U; w.b_sk = r; w.b_sn = 1;
-  w.C = R; w.ldc = r; w.epi = EPI_STORE;
-  DION_TRY(launch_gemm(s, w));
+  for (int b = 0; b < nb; ++b) {
+    const dion_matrix* a = list[b];
+    GemmArgs w = gemm_args();
+    w.M = n; w.N = r; w.K = m;
+    w.A = (const float*)a->M; w.a_si = 1; w.a_sk = a->ldm;
+    w.A2 = a->G; w.a2_si = 1; w.a2_sk = a->ldg; w.a2_mode = (a->g_dtype == DION_BF16) ? ADD_BF16 : ADD_F32;
+    w.B = s.W(b, U_off); w.b_sk = r; w.b_sn = 1;
+    w.C = s.W(b, s.L.R); w.ldc = r; w.epi = EPI_STORE;
+    DION_TRY(launch_gemm(s, w, b));
+  }
   }
 
   // M <- (M + G) - (1 - mu) U R^T
   {
   PhaseScope ps(c, st, DION_PHASE_EF);
-  GemmArgs e = gemm_args();
-  e.M = m; e.N = n; e.K = r;
-  e.A = U; e.a_si = r; e.a_sk = 1;
-  e.B = R; e.b_sk = 1; e.b_sn = r;
-  e.C = (float*)a->M; e.ldc = a->ldm; e.epi = EPI_ADD2_SUB;
-  e.C2 = a->G; e.ldc2 = a->ldg; e.c2_mode = gmode;
-  e.alpha = 1.f - c->cfg.mu;
-  e.skip_flag = s.flag;
-  DION_TRY(launch_gemm(s, e));
+  for (int b = 0; b < nb; ++b) {
+    const dion_matrix* a = list[b];
+    GemmArgs e = gemm_args();
+    e.M = m; e.N = n; e.K = r;
+    e.A = s.W(b, U_off); e.a_si = r; e.a_sk = 1;
+    e.B = s.W(b, s.L.R); e.b_sk = 1; e.b_sn = r;
+    e.C = (float*)a->M; e.ldc = a->ldm; e.epi = EPI_ADD2_SUB;
+    e.C2 = a->G; e.ldc2 = a->ldg; e.c2_mode = (a->g_dtype == DION_BF16) ? ADD_BF16 : ADD_F32;
+    e.alpha = 1.f - c->cfg.mu;
+    e.skip_flag = s.OS(b) + OS_FAIL;
+    DION_TRY(launch_gemm(s, e, b));
+  }
   }
 
   // Q <- ColNorm(R)
   {
   PhaseScope ps(c, st, DION_PHASE_COLNORM);
-  DION_TRY(colnorm(s, R, n, r, (float*)a->Q, a->ldq, a->colnorm_out));
+  for (int b = 0; b < nb; ++b) {
+    const dion_matrix* a = list[b];
+    DION_TRY(colnorm(s, b, s.W(b, s.L.R), n, r, (float*)a->Q, a->ldq, a->colnorm_out));
+  }
   }
 
   // X <- X - lr sqrt(m/n) U Q^T
   {
   PhaseScope ps(c, st, DION_PHASE_X);
-  GemmArgs x = gemm_args();
-  x.M = m; x.N = n; x.K = r;
-  x.A = U; x.a_si = r; x.a_sk = 1;
-  x.B = (const float*)a->Q; x.b_sk = 1; x.b_sn = a->ldq;
-  x.C = (float*)a->X; x.ldc = a->ldx; x.epi = EPI_SUB;
-  x.alpha = lr * sqrtf((float)((double)m / (double)n));
-  x.skip_flag = s.flag;
-  DION_TRY(launch_gemm(s, x));
-  k_finish_step<<<1, 1, 0, st>>>(s.flag, c->dev_ints + 1);
+  for (int b = 0; b < nb; ++b) {
+    const dion_matrix* a = list[b];
+    GemmArgs x = gemm_args();
+    x.M = m; x.N = n; x.K = r;
+    x.A = s.W(b, U_off); x.a_si = r; x.a_sk = 1;
+    x.B = (const float*)a->Q; x.b_sk = 1; x.b_sn = a->ldq;
+    x.C = (float*)a->X; x.ldc = a->ldx; x.epi = EPI_SUB;
+    x.alpha = lr * sqrtf((float)((double)m / (double)n));
+    x.skip_flag = s.OS(b) + OS_FAIL;
+    DION_TRY(launch_gemm(s, x, b));
+  }
+  k_finish_step<<<nb, 1, 0, st>>>(s.flag, c->dev_ints + 1);
   DION_CHECK_LAUNCH(c);
   }
   return DION_OK;
 }
 
+int step_one(dion_ctx* c, const dion_matrix* a, float lr, cudaStream_t st) {
+  return step_batch(c, &a, 1, lr, st);
+}
+
 // One Lazy-Dion step (Algorithm 6).
 int lazy_one(dion_ctx* c, const dion_matrix* a, float lr, int refresh, cudaStream_t st) {
   StepCtx s;
-  DION_TRY(begin_step(c, a, st, &s));
+  DION_TRY(begin_step(c, a, 1, st, &s));
   const i64 m = a->m, n = a->n, r = a->r;
   const int gmode = (a->g_dtype == DION_BF16) ? ADD_BF16 : ADD_F32;
   float* P0 = s.ws + s.L.P0;
@@ -612,15 +675,16 @@ int lazy_one(dion_ctx* c, const dion_matrix* a, float lr, int refresh, cudaStrea
     z.C = P0; z.ldc = r; z.epi = EPI_STORE;
     z.precise = t.precise;
     DION_TRY(launch_gemm(s, z));
-    float* V = nullptr;
-    DION_TRY(orthonormalize(s, n, r, (m < n) ? m : n, &V));
+    i64 V_off = 0;
+    DION_TRY(orthonormalize(s, n, r, (m < n) ? m : n, &V_off));
+    const float* V = s.ws + V_off;
     // copy V into Q unless the round broke down (alpha = 1, identity product is overkill: strided copy kernel)
     GemmArgs cp = gemm_args();
     (void)cp;
     const i64 total = n * r;
     int blocks = (int)((total + 255) / 256);
     if (blocks > 8 * c->sm_count) blocks = 8 * c->sm_count;
-    k_copy_panel<<<blocks, 256, 0, st>>>(V, r, (float*)a->Q, a->ldq, n, r, s.flag, nullptr);
+    k_copy_panel<<<blocks, 256, 0, st>>>(V, r, (float*)a->Q, a->ldq, n, r, s.flag, nullptr, 0);
     DION_CHECK_LAUNCH(c);
   }
   // W = (M + G) Q
@@ -642,7 +706,7 @@ int lazy_one(dion_ctx* c, const dion_matrix* a, float lr, int refresh, cudaStrea
   e.skip_flag = s.flag;
   DION_TRY(launch_gemm(s, e));
   // U = ColNorm(W)
-  DION_TRY(colnorm(s, R, m, r, P0, r, a->colnorm_out));
+  DION_TRY(colnorm(s, 0, R, m, r, P0, r, a->colnorm_out));
   // X <- X - lr sqrt(m/n) U Q^T
   GemmArgs x = gemm_args();
   x.M = m; x.N = n; x.K = r;
@@ -725,17 +789,37 @@ int dion_step_grouped(dion_ctx* ctx, const dion_matrix* list, int count, float l
   if (ctx == nullptr || count < 0) return DION_ERR_INVALID;
   if (count == 0) return DION_OK;
   if (list == nullptr) return DION_ERR_INVALID;
+  for (int i = 0; i < count; ++i) DION_TRY(validate(&list[i]));
+  if (cudaSetDevice(ctx->cfg.device) != cudaSuccess) return DION_ERR_CUDA;
+  // Matrices of identical (m, n, r) form a class (the paper's batch axis).  A class is
+  // stepped in chains of up to `cap` matrices that share each small kernel launch of the
+  // factorization; every matrix of a chain has its own scratch slice.
+  const size_t budget = ctx->cfg.workspace_bytes > GROUP_SCRATCH_BYTES ? ctx->cfg.workspace_bytes : GROUP_SCRATCH_BYTES;
+  std::vector<char> done((size_t)count, 0);
+  std::vector<const dion_matrix*> chain;
   size_t need = 0;
+  std::vector<std::vector<const dion_matrix*>> chains;
   for (int i = 0; i < count; ++i) {
-    DION_TRY(validate(&list[i]));
-    const size_t b = dion_workspace_bytes(ctx, list[i].m, list[i].n, list[i].r);
+    if (done[i]) continue;
+    const size_t one = dion_workspace_bytes(ctx, list[i].m, list[i].n, list[i].r);
+    size_t cap = one > 0 ? budget / one : 1;
+    if (cap < 1) cap = 1;
+    if (cap > MAX_CHAIN) cap = MAX_CHAIN;
+    chain.clear();
+    for (int j = i; j < count; ++j) {
+      if (done[j] || list[j].m != list[i].m || list[j].n != list[i].n || list[j].r != list[i].r) continue;
+      done[j] = 1;
+      chain.push_back(&list[j]);
+      if (chain.size() == cap) { chains.push_back(chain); chain.clear(); }
+    }
+    if (!chain.empty()) chains.push_back(chain);
+  }
+  for (const auto& ch : chains) {
+    const size_t b = dion_workspace_bytes(ctx, ch[0]->m, ch[0]->n, ch[0]->r) * ch.size();
     if (b > need) need = b;
   }
-  if (cudaSetDevice(ctx->cfg.device) != cudaSuccess) return DION_ERR_CUDA;
   DION_TRY(ensure_ws(ctx, need));
-  // The matrices are independent; they share the scratch, so their launch chains
-  // run back to back on the one stream.
-  for (int i = 0; i < count; ++i) DION_TRY(step_one(ctx, &list[i], lr, (cudaStream_t)cuda_stream));
+  for (const auto& ch : chains) DION_TRY(step_batch(ctx, ch.data(), (int)ch.size(), lr, (cudaStream_t)cuda_stream));
   return DION_OK;
 }
 

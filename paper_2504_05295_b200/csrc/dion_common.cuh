@@ -37,6 +37,8 @@ struct GemmArgs {
   float alpha;
   const float* alpha_dev;      // optional: alpha is multiplied by *alpha_dev
   int batch; i64 bsA, bsB, bsC;  // batch count and element strides
+  int batch2; i64 bs2;           // outer batch (one per matrix of a grouped call): stride of A, B, C alike
+  i64 skip_stride;               // ints between the skip flags of consecutive outer batch entries
   int splits; float* part;       // split-K: partial sums, [splits][M][N]
   int tri;                       // TRI_LOWER: tiles strictly above the diagonal are skipped
   int klimit;                    // 1: B(k,j) == 0 for k > j  (K loop ends at the tile's last column)

@@ -20,9 +20,13 @@ enum : int {
 
 // Round set-up on the r x r Gram matrix G (one block): saves diag(G) to gdiag, writes
 // shift = scale * trace(G) (fixed summation order) and resets the round statistics.
+// Batched: block b works on the matrix whose scratch starts b * wstride floats further and
+// whose state slot is b slots further.
 __global__ void k_round_begin(const float* __restrict__ G, i64 ld, i64 r, float scale,
                               float* __restrict__ gdiag, float* __restrict__ shift,
-                              int* __restrict__ os, int adaptive) {
+                              int* __restrict__ os, int adaptive, i64 wstride) {
+  G += (i64)blockIdx.x * wstride; gdiag += (i64)blockIdx.x * wstride; shift += (i64)blockIdx.x * wstride;
+  os += (i64)blockIdx.x * OS_SLOT_INTS;
   if (adaptive && os[OS_DONE] != 0) return;
   __shared__ float red[256];
   float s = 0.f;
@@ -63,7 +67,13 @@ __global__ void __launch_bounds__(256) k_potrf_diag(float* __restrict__ A, i64 l
                                                     const float* __restrict__ shift,
                                                     const float* __restrict__ gdiag, float floor_rel,
                                                     int* __restrict__ os, int adaptive,
-                                                    int* __restrict__ status) {
+                                                    int* __restrict__ status, i64 wstride) {
+  {  // batched: block b -> matrix b
+    const i64 wo = (i64)blockIdx.x * wstride;
+    A += wo; Dinv += wo; DinvP += wo; gdiag += wo;
+    if (shift != nullptr) shift += wo;
+    os += (i64)blockIdx.x * OS_SLOT_INTS;
+  }
   if (adaptive && os[OS_DONE] != 0) return;
   // The block is factored in four 16-column sub-panels: the 16 x 16 diagonal piece by
   // one warp (two warp barriers per column), the rows below it by one thread per row,
@@ -236,6 +246,7 @@ __global__ void __launch_bounds__(256) k_potrf_diag(float* __restrict__ A, i64 l
 //     round brings orthonormality to rounding level (the CholeskyQR2 argument), after
 //     which the remaining rounds are skipped.
 __global__ void k_round_end(int* __restrict__ os, float good_rel, float done_rel, int* __restrict__ rounds_total) {
+  os += (i64)blockIdx.x * OS_SLOT_INTS;
   if (os[OS_DONE] != 0) return;
   os[OS_ROUNDS] += 1;
   atomicAdd(rounds_total, 1);
@@ -250,6 +261,7 @@ __global__ void k_round_end(int* __restrict__ os, float good_rel, float done_rel
 // After the last adaptive round: a panel that never became well conditioned is
 // reported; if pivots were still being raised the step is cancelled (rank-deficient P).
 __global__ void k_orth_finish(int* __restrict__ os, int* __restrict__ status) {
+  os += (i64)blockIdx.x * OS_SLOT_INTS;
   if (os[OS_DONE] != 0) return;
   if (os[OS_GOOD] == 0 && os[OS_FLOORED] != 0) {
     os[OS_FAIL] = 1;
@@ -262,8 +274,9 @@ __global__ void k_orth_finish(int* __restrict__ os, int* __restrict__ status) {
 // The sz x sz diagonal square of Linv that starts at row/column o (a multiple of 64):
 // zero, except its 64 x 64 diagonal blocks, which are copied from Dinv.
 __global__ void k_linv_init(float* __restrict__ Linv, i64 ld, i64 o, i64 sz, const float* __restrict__ Dinv,
-                            const int* __restrict__ skip_flag) {
-  if (skip_flag != nullptr && *skip_flag != 0) return;
+                            const int* __restrict__ skip_flag, i64 wstride) {
+  Linv += (i64)blockIdx.y * wstride; Dinv += (i64)blockIdx.y * wstride;   // batched over blockIdx.y
+  if (skip_flag != nullptr && skip_flag[(i64)blockIdx.y * OS_SLOT_INTS] != 0) return;
   const i64 total = sz * sz;
   for (i64 e = (i64)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (i64)gridDim.x * blockDim.x) {
     const i64 i = o + e / sz, c = o + e % sz;
@@ -275,8 +288,9 @@ __global__ void k_linv_init(float* __restrict__ Linv, i64 ld, i64 o, i64 sz, con
 
 // Copies a rows x cols block between two matrices (leading dimensions lds, ldd).
 __global__ void k_copy_block(const float* __restrict__ src, i64 lds, float* __restrict__ dst, i64 ldd,
-                             i64 rows, i64 cols, const int* __restrict__ skip_flag) {
-  if (skip_flag != nullptr && *skip_flag != 0) return;
+                             i64 rows, i64 cols, const int* __restrict__ skip_flag, i64 wstride) {
+  src += (i64)blockIdx.y * wstride; dst += (i64)blockIdx.y * wstride;     // batched over blockIdx.y
+  if (skip_flag != nullptr && skip_flag[(i64)blockIdx.y * OS_SLOT_INTS] != 0) return;
   const i64 total = rows * cols;
   for (i64 e = (i64)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (i64)gridDim.x * blockDim.x) {
     const i64 i = e / cols, c = e % cols;
@@ -332,9 +346,11 @@ __global__ void __launch_bounds__(128) k_colnorm_apply(const float* __restrict__
 // `only_if` (optional): the copy happens only when *only_if != 0.
 __global__ void k_copy_panel(const float* __restrict__ V, i64 ldv, float* __restrict__ Q, i64 ldq,
                              i64 rows, i64 r, const int* __restrict__ skip_flag,
-                             const int* __restrict__ only_if) {
-  if (skip_flag != nullptr && *skip_flag != 0) return;
-  if (only_if != nullptr && *only_if == 0) return;
+                             const int* __restrict__ only_if, i64 wstride) {
+  V += (i64)blockIdx.y * wstride;                                         // batched over blockIdx.y
+  if (wstride != 0) Q += (i64)blockIdx.y * wstride;
+  if (skip_flag != nullptr && skip_flag[(i64)blockIdx.y * OS_SLOT_INTS] != 0) return;
+  if (only_if != nullptr && only_if[(i64)blockIdx.y * OS_SLOT_INTS] == 0) return;
   const i64 total = rows * r;
   for (i64 e = (i64)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (i64)gridDim.x * blockDim.x) {
     const i64 i = e / r, c = e % r;
@@ -344,7 +360,7 @@ __global__ void k_copy_panel(const float* __restrict__ V, i64 ldv, float* __rest
 
 // Counts a skipped step (breakdown) at the end of a step's launch chain.
 __global__ void k_finish_step(const int* __restrict__ step_flag, int* __restrict__ skipped) {
-  if (*step_flag != 0) atomicAdd(skipped, 1);
+  if (step_flag[(i64)blockIdx.x * OS_SLOT_INTS] != 0) atomicAdd(skipped, 1);
 }
 
 // ---------------------------------------------------------------------------

@@ -12,7 +12,12 @@ template <int BM, int BN, int BK, int TM, int TN>
 __global__ void __launch_bounds__(256) k_gemm_simt(const GemmArgs g) {
   static_assert((BM / TM) * (BN / TN) == 256, "256 threads per tile");
   static_assert(TM % 4 == 0 && TN % 4 == 0, "micro tile in groups of 4");
-  if (g.skip_flag != nullptr && *g.skip_flag != 0) return;
+  // blockIdx.z = inner batch index + batch * outer batch index (or the K split)
+  i64 batch = 0, outer = 0;
+  int split = 0;
+  if (g.splits > 1) split = blockIdx.z;
+  else { batch = blockIdx.z % g.batch; outer = blockIdx.z / g.batch; }
+  if (g.skip_flag != nullptr && g.skip_flag[outer * g.skip_stride] != 0) return;
 
   constexpr int LDA_S = BM + 4, LDB_S = BN + 4;
   constexpr int A_PER = BM * BK / 256, B_PER = BN * BK / 256;
@@ -26,10 +31,6 @@ __global__ void __launch_bounds__(256) k_gemm_simt(const GemmArgs g) {
   const i64 i0 = (i64)blockIdx.y * BM, j0 = (i64)blockIdx.x * BN;
   if (g.tri == TRI_LOWER && j0 > i0 + BM - 1) return;
 
-  int split = 0;
-  i64 batch = 0;
-  if (g.splits > 1) split = blockIdx.z; else batch = blockIdx.z;
-
   i64 k_begin = 0, k_end = g.K;
   if (g.klimit) k_end = min(g.K, j0 + BN);
   if (g.splits > 1) {
@@ -39,8 +40,8 @@ __global__ void __launch_bounds__(256) k_gemm_simt(const GemmArgs g) {
     k_end = min(k_end, k_begin + per);
   }
 
-  const float* A = g.A + batch * g.bsA;
-  const float* B = g.B + batch * g.bsB;
+  const float* A = g.A + batch * g.bsA + outer * g.bs2;
+  const float* B = g.B + batch * g.bsB + outer * g.bs2;
   const bool a_kcontig = (g.a_sk == 1);
   const bool b_ncontig = (g.b_sn == 1);
 
@@ -138,7 +139,7 @@ __global__ void __launch_bounds__(256) k_gemm_simt(const GemmArgs g) {
     return;
   }
 
-  float* C = g.C + batch * g.bsC;
+  float* C = g.C + batch * g.bsC + outer * g.bs2;
 #pragma unroll
   for (int x = 0; x < TM; ++x) {
     const i64 gi = i0 + (x / 4) * SM_STRIDE + ty * 4 + (x % 4);
