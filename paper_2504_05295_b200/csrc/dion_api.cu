@@ -344,14 +344,14 @@ int potrf_inner(StepCtx& s, i64 r, i64 o, i64 sz, const float* shift, bool adapt
 // factor into Linv.  Outer blocks of 512 columns: the diagonal square is factored and
 // inverted by potrf_inner, the panel below it is multiplied by that inverse and the
 // trailing matrix is updated with one rank-512 product (tensor cores where it qualifies).
-int potrf_trtri(StepCtx& s, i64 r, const float* shift, bool adaptive) {
+int potrf_trtri(StepCtx& s, i64 r, const float* shift, bool adaptive, bool full_inverse) {
   dion_ctx* c = s.c;
   float* Gm = s.ws + s.L.Gram;
   float* Linv = s.ws + s.L.Linv;
   float* Tbuf = s.ws + s.L.Tbuf;
   const int* skip = adaptive ? (s.os + OS_DONE) : nullptr;
   const int precise = adaptive ? 1 : 0;
-  if (r > NBO) {
+  if (r > NBO && full_inverse) {
     // everything outside the diagonal squares starts at zero (the product U = P Linv^T reads whole tiles)
     for (int m = 0; m < s.nb; ++m)
       if (cudaMemsetAsync(s.W(m, s.L.Linv), 0, sizeof(float) * (size_t)r * (size_t)r, s.st) != cudaSuccess) return DION_ERR_CUDA;
@@ -383,7 +383,7 @@ int potrf_trtri(StepCtx& s, i64 r, const float* shift, bool adaptive) {
       for (int m = 0; m < s.nb; ++m) DION_TRY(launch_gemm(s, for_matrix(s, t, m, true, true, true), m));
     }
   }
-  if (r > NBO) DION_TRY(trtri_levels(s, r, 0, r, NBO, skip, precise));
+  if (r > NBO && full_inverse) DION_TRY(trtri_levels(s, r, 0, r, NBO, skip, precise));
   return DION_OK;
 }
 
@@ -403,11 +403,49 @@ int cholqr_round(StepCtx& s, i64 pin_off, i64 pout_off, i64 rows, i64 r, bool ad
   k_round_begin<<<s.nb, 256, 0, s.st>>>(s.ws + s.L.Gram, r, r, 0.f, s.ws + s.L.gdiag, s.ws + s.L.scal, s.os,
                                         adaptive ? 1 : 0, s.wstride);
   DION_CHECK_LAUNCH(c);
-  DION_TRY(potrf_trtri(s, r, nullptr, adaptive));
+  // Tall panels with r > 512: blocked triangular solve with the 512-column diagonal inverses
+  // only (the levels of the triangular inverse above 512 are never formed).
+  const bool trsm = (r > NBO) && (rows >= 8192);   // 512-column products need >= 128 row tiles to fill the GPU
+  DION_TRY(potrf_trtri(s, r, nullptr, adaptive, !trsm));
   if (adaptive) {
     dim3 grid((unsigned)grid_for(c, rows * r), (unsigned)s.nb);
     k_copy_panel<<<grid, 256, 0, s.st>>>(s.ws + pin_off, r, s.ws + pout_off, r, rows, r, nullptr, s.os + OS_DONE, s.wstride);
     DION_CHECK_LAUNCH(c);
+  }
+  if (trsm) {
+    // Pout_J = (Pin_J - sum_{K<J} Pout_K L_{J,K}^T) Linv_JJ^T, block columns J of 512
+    const float* Lm = s.ws + s.L.Gram;     // the factor, lower
+    float* Wt = s.ws + s.L.R;              // rows x 512 temporary (R is free during the orthonormalization)
+    for (i64 J0 = 0; J0 < r; J0 += NBO) {
+      const i64 sz = (r - J0 < NBO) ? (r - J0) : NBO;
+      const float* rhs = s.ws + pin_off + J0;
+      i64 rhs_ld = r;
+      if (J0 > 0) {
+        GemmArgs w = gemm_args();
+        w.M = rows; w.N = sz; w.K = J0;
+        w.A = s.ws + pout_off; w.a_si = r; w.a_sk = 1;
+        w.B = Lm + J0 * r; w.b_sk = 1; w.b_sn = r;
+        w.C = Wt; w.ldc = NBO; w.epi = EPI_C2_SUB; w.C2 = rhs; w.ldc2 = r; w.c2_mode = ADD_F32;
+        w.skip_flag = skip; w.precise = adaptive ? 1 : 0;
+        for (int m = 0; m < s.nb; ++m) {
+          GemmArgs wm = for_matrix(s, w, m, true, true, true);
+          wm.C2 = (const float*)wm.C2 + (i64)m * s.wstride;
+          DION_TRY(launch_gemm(s, wm, m));
+        }
+        rhs = Wt; rhs_ld = NBO;
+      }
+      GemmArgs v = gemm_args();
+      v.M = rows; v.N = sz; v.K = sz;
+      v.A = rhs; v.a_si = rhs_ld; v.a_sk = 1;
+      v.B = s.ws + s.L.Linv + J0 * r + J0; v.b_sk = 1; v.b_sn = r; v.klimit = 1;
+      v.C = s.ws + pout_off + J0; v.ldc = r; v.epi = EPI_STORE; v.skip_flag = skip; v.precise = adaptive ? 1 : 0;
+      for (int m = 0; m < s.nb; ++m) DION_TRY(launch_gemm(s, for_matrix(s, v, m, true, true, true), m));
+    }
+    if (adaptive) {
+      k_round_end<<<s.nb, 1, 0, s.st>>>(s.os, GOOD_REL, DONE_REL, c->dev_ints + 2);
+      DION_CHECK_LAUNCH(c);
+    }
+    return DION_OK;
   }
   GemmArgs u = gemm_args();
   u.M = rows; u.N = r; u.K = r;

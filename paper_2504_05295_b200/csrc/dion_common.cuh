@@ -17,7 +17,8 @@ enum : int { ADD_NONE = 0, ADD_F32 = 1, ADD_BF16 = 2 };
 enum : int {
   EPI_STORE = 0,      // C = alpha * acc
   EPI_SUB = 1,        // C = C - alpha * acc
-  EPI_ADD2_SUB = 2    // C = C + C2 - alpha * acc   (error feedback: M <- M + G - beta U R^T)
+  EPI_ADD2_SUB = 2,   // C = C + C2 - alpha * acc   (error feedback: M <- M + G - beta U R^T)
+  EPI_C2_SUB = 3      // C = C2 - alpha * acc       (blocked triangular solve; C2 is fp32)
 };
 // Which output tiles exist.
 enum : int { TRI_FULL = 0, TRI_LOWER = 1 };

@@ -154,6 +154,8 @@ __global__ void __launch_bounds__(256) k_gemm_simt(const GemmArgs g) {
         *c = v;
       } else if (g.epi == EPI_SUB) {
         *c = *c - v;
+      } else if (g.epi == EPI_C2_SUB) {
+        *c = load_add(g.C2, gi * g.ldc2 + gj, ADD_F32) - v;
       } else {
         *c = (*c + load_add(g.C2, gi * g.ldc2 + gj, g.c2_mode)) - v;
       }
