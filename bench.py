@@ -120,6 +120,17 @@ def oracle_flops(m, n, r):
     return 8.0 * m * n * r + 4.0 * m * r * r - 4.0 / 3.0 * r ** 3
 
 
+def max_over_ranks(value: float, device=None) -> float:
+    """Max of a per-rank scalar over the default process group (identity without one)."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(value)
+    t = torch.tensor([float(value)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
 # ---------------------------------------------------------------------------
 # clocks sampler
 # ---------------------------------------------------------------------------
@@ -155,8 +166,19 @@ class ClockSampler:
             pass
         try:
             self.out.close()
-            rows = [l.strip().split(",") for l in open(self.path) if l.strip()]
+            lines = open(self.path).read().splitlines()
             os.unlink(self.path)
+            res = self.parse(lines)
+        except Exception:
+            pass
+        return res
+
+    @staticmethod
+    def parse(lines):
+        """Median SM clock, max clock and the throttle reasons seen in nvidia-smi CSV lines."""
+        res = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if True:
+            rows = [l.strip().split(",") for l in lines if l.strip()]
             sm, mx, reasons = [], [], set()
             names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
             for row in rows:
@@ -172,8 +194,6 @@ class ClockSampler:
             if sm:
                 res = {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(mx), "reasons": sorted(reasons),
                        "samples": len(sm)}
-        except Exception:
-            pass
         return res
 
 
@@ -328,10 +348,7 @@ def run_ours(args):
     launches = opt.launch_count() - launches0
     status2, skipped2 = opt.get_status()
     ms_step = ms_total / args.steps
-    if world > 1:
-        t_ = torch.tensor([ms_step], device=dev)
-        dist.all_reduce(t_, op=dist.ReduceOp.MAX)
-        ms_step = float(t_.item())
+    ms_step = max_over_ranks(ms_step, dev)
 
     case_ms = [sum(a.elapsed_time(b) for a, b in ev) / len(ev) if ev else None for ev in case_events]
 
@@ -357,10 +374,7 @@ def run_ours(args):
     f1.record(stream)
     barrier()
     e2e_ms = f0.elapsed_time(f1) / e2e_steps
-    if world > 1:
-        t_ = torch.tensor([e2e_ms], device=dev)
-        dist.all_reduce(t_, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t_.item())
+    e2e_ms = max_over_ranks(e2e_ms, dev)
     status3, _ = opt.get_status()
 
     # adaptive Cholesky-QR rounds per case, read on one more (untimed) step

@@ -240,9 +240,9 @@ def test_argument_errors():
         assert opt.get_status() == (0, 0)
 
 
-def test_lazy_dion_steps_match_oracle():
+@pytest.mark.parametrize("m,n,r", [(384, 256, 32), (1536, 1024, 128)])
+def test_lazy_dion_steps_match_oracle(m, n, r):
     from oracle import dion_oracle as orc
-    m, n, r = 384, 256, 32
     pb = inputs.make_problem(m, n, r, seed=14, ks=8)
     X, M, Q = device_state(pb)
     Xo, Mo, Qo = to_np64(pb.X), to_np64(pb.M), to_np64(pb.Q)
