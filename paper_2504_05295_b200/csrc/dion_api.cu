@@ -1067,4 +1067,3 @@ extern "C" int dion_debug_gemm(int engine, int precision, const dion_debug_gemm_
   c.sm_count = sms; c.launches = 0; c.prof_on = false; c.prof_used = 0;
   return launch_gemm_simt(&c, g, st, part, part_floats, false);
 }
-

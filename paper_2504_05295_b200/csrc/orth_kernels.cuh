@@ -130,7 +130,7 @@ __global__ void __launch_bounds__(256) k_potrf_diag(float* __restrict__ A, i64 l
               defl = true;
               ++floored;
             } else {
-              minrel = fminf(minrel, p / g);
+              minrel = fminf(minrel, __fdividef(p, g));
             }
           } else if (!(p > 0.f) || !isfinite(p)) {
             failed = 1;
@@ -217,16 +217,26 @@ __global__ void __launch_bounds__(256) k_potrf_diag(float* __restrict__ A, i64 l
     const int npairs = NB / (2 * b);
     for (int e = tid; e < npairs * b * b; e += 256) {
       const int pr = e / (b * b), rr = (e / b) % b, cc = e % b, base = pr * 2 * b;
-      float sacc = 0.f;
-      for (int k = cc; k < b; ++k) sacc = fmaf(L[base + b + rr][base + k], X[base + k][base + cc], sacc);
-      T[pr * b + rr][cc] = sacc;
+      float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;   // X11 is lower triangular: k >= cc; zeros above are stored
+      for (int k = cc & ~3; k < b; k += 4) {
+        s0 = fmaf(L[base + b + rr][base + k], X[base + k][base + cc], s0);
+        s1 = fmaf(L[base + b + rr][base + k + 1], X[base + k + 1][base + cc], s1);
+        s2 = fmaf(L[base + b + rr][base + k + 2], X[base + k + 2][base + cc], s2);
+        s3 = fmaf(L[base + b + rr][base + k + 3], X[base + k + 3][base + cc], s3);
+      }
+      T[pr * b + rr][cc] = (s0 + s1) + (s2 + s3);
     }
     __syncthreads();
     for (int e = tid; e < npairs * b * b; e += 256) {
       const int pr = e / (b * b), rr = (e / b) % b, cc = e % b, base = pr * 2 * b;
-      float sacc = 0.f;
-      for (int k = 0; k <= rr; ++k) sacc = fmaf(X[base + b + rr][base + b + k], T[pr * b + k][cc], sacc);
-      X[base + b + rr][base + cc] = -sacc;
+      float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;   // X22 is lower triangular: k <= rr; zeros above are stored
+      for (int k = 0; k <= rr; k += 4) {
+        s0 = fmaf(X[base + b + rr][base + b + k], T[pr * b + k][cc], s0);
+        s1 = fmaf(X[base + b + rr][base + b + k + 1], T[pr * b + k + 1][cc], s1);
+        s2 = fmaf(X[base + b + rr][base + b + k + 2], T[pr * b + k + 2][cc], s2);
+        s3 = fmaf(X[base + b + rr][base + b + k + 3], T[pr * b + k + 3][cc], s3);
+      }
+      X[base + b + rr][base + cc] = -((s0 + s1) + (s2 + s3));
     }
     __syncthreads();
   }
