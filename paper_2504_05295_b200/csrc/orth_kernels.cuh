@@ -140,20 +140,20 @@ __global__ void __launch_bounds__(256) k_potrf_diag(float* __restrict__ A, i64 l
         const float inv = rsqrtf(p);
         float v = 0.f;
         if (i > j && !defl) v = L[c0 + i][c0 + j] * inv;
-        __syncwarp();
         if (half == 0) {
-          if (i == j) { L[c0 + j][c0 + j] = p * inv; rdiag[c0 + j] = inv; if (defl) deflated[c0 + j] = 1; }
+          if (i == j) { rdiag[c0 + j] = inv; if (defl) deflated[c0 + j] = 1; }
           else if (i > j) L[c0 + i][c0 + j] = v;
         }
-        __syncwarp();
-        // rank-1 update of the remaining columns of this piece (each lane: 8 columns of its row)
-        if (i > j) {
+        // rank-1 update of the remaining columns of this piece: each lane owns 8 columns of its
+        // row; the column-j entry of row c comes by shuffle from the lane that just computed it
+        // (both halves hold the same v), so one warp barrier per column is enough
 #pragma unroll
-          for (int q = 0; q < W / 2; ++q) {
-            const int c = half * (W / 2) + q;
-            if (c > j && c <= i) L[c0 + i][c0 + c] = fmaf(-v, L[c0 + c][c0 + j], L[c0 + i][c0 + c]);
-          }
+        for (int q = 0; q < W / 2; ++q) {
+          const int c = half * (W / 2) + q;
+          const float vc = __shfl_sync(0xffffffffu, v, c);
+          if (c > j && c <= i) L[c0 + i][c0 + c] = fmaf(-v, vc, L[c0 + i][c0 + c]);
         }
+        if (half == 0 && i == j) L[c0 + j][c0 + j] = p * inv;   // after every lane has read the pivot
         __syncwarp();
       }
     }
