@@ -231,6 +231,16 @@ GemmArgs for_matrix(const StepCtx& s, GemmArgs g, int b, bool a_ws, bool b_ws, b
   return g;
 }
 
+// One-time opt-in to the dynamic shared memory of the kernels that need more than 48 KB.
+int configure_kernels() {
+  if (umma_configure() != DION_OK) return DION_ERR_CUDA;
+  if (cudaFuncSetAttribute(k_chol_step, cudaFuncAttributeMaxDynamicSharedMemorySize, CHOL_STEP_SMEM) != cudaSuccess) {
+    cudaGetLastError();
+    return DION_ERR_CUDA;
+  }
+  return DION_OK;
+}
+
 constexpr i64 NBO = 512;  // outer block of the two-level Cholesky
 
 int grid_for(const dion_ctx* c, i64 total) {
@@ -297,40 +307,36 @@ int trtri_levels(StepCtx& s, i64 r, i64 o, i64 sz, i64 b_from, const int* skip, 
 
 // Cholesky of the diagonal square [o, o+sz) of each Gram matrix (sz <= NBO), right-looking with
 // 64-wide blocks on the FMA engine, followed by the inverse of that square's factor into Linv.
-int potrf_inner(StepCtx& s, i64 r, i64 o, i64 sz, const float* shift, bool adaptive) {
+int potrf_inner(StepCtx& s, i64 r, i64 o, i64 sz, bool adaptive) {
   dion_ctx* c = s.c;
   float* Gm = s.ws + s.L.Gram;
   float* Dinv = s.ws + s.L.Dinv;
+  float* DinvP = s.ws + s.L.DinvP;
   float* Linv = s.ws + s.L.Linv;
+  float* Tbuf = s.ws + s.L.Tbuf;
   const float* gdiag = s.ws + s.L.gdiag;
   int* status = c->dev_ints;
   const int* skip = adaptive ? (s.os + OS_DONE) : nullptr;
-  for (i64 j0 = o; j0 < o + sz; j0 += NB) {
-    const int jb = (int)((o + sz - j0 < NB) ? (o + sz - j0) : NB);
-    float* Ajj = Gm + j0 * r + j0;
-    float* Dj = Dinv + (j0 / NB) * (NB * NB);
-    float* DPj = s.ws + s.L.DinvP + (j0 / NB) * (NB * NB);
-    k_potrf_diag<<<s.nb, 256, 0, s.st>>>(Ajj, r, jb, Dj, DPj, shift, gdiag + j0, adaptive ? FLOOR_REL : 0.f, s.os,
-                                         adaptive ? 1 : 0, status, s.wstride);
+  const float floor_rel = adaptive ? FLOOR_REL : 0.f;
+  const int nblk = (int)((sz + NB - 1) / NB);
+  {
+    const int jb = (int)((sz < NB) ? sz : NB);
+    k_potrf_diag<<<s.nb, 256, 0, s.st>>>(Gm + o * r + o, r, jb, Dinv + (o / NB) * (NB * NB), DinvP + (o / NB) * (NB * NB),
+                                         gdiag + o, floor_rel, s.os, adaptive ? 1 : 0, status, s.wstride);
     DION_CHECK_LAUNCH(c);
-    const i64 rem = o + sz - j0 - jb;
-    if (rem > 0) {
-      float* panel = Gm + (j0 + jb) * r + j0;
-      GemmArgs g = gemm_args();  // panel <- panel * Linv_jj^T, in place (one column tile)
-      g.M = rem; g.N = jb; g.K = jb;
-      g.A = panel; g.a_si = r; g.a_sk = 1;
-      g.B = DPj; g.b_sk = 1; g.b_sn = NB;
-      g.C = panel; g.ldc = r; g.epi = EPI_STORE; g.skip_flag = skip;
-      over_batch(s, g);
-      DION_TRY(launch_gemm_simt(c, g, s.st, nullptr, 0, true));
-      GemmArgs t = gemm_args();  // A22 -= panel * panel^T (lower tiles)
-      t.M = rem; t.N = rem; t.K = jb;
-      t.A = panel; t.a_si = r; t.a_sk = 1;
-      t.B = panel; t.b_sk = 1; t.b_sn = r;
-      t.C = Gm + (j0 + jb) * r + (j0 + jb); t.ldc = r; t.epi = EPI_SUB; t.tri = TRI_LOWER; t.skip_flag = skip;
-      over_batch(s, t);
-      DION_TRY(launch_gemm_simt(c, t, s.st, nullptr, 0, true));
-    }
+  }
+  // one launch per block column: panel, trailing update and the next diagonal block
+  for (int j = 0; j + 1 < nblk; ++j) {
+    const int nt = nblk - 1 - j;
+    dim3 grid((unsigned)(nt * (nt + 1) / 2), (unsigned)s.nb);
+    k_chol_step<<<grid, 256, CHOL_STEP_SMEM, s.st>>>(Gm, r, o, sz, j, Dinv, DinvP, Tbuf, gdiag, floor_rel, s.os,
+                                                     adaptive ? 1 : 0, status, s.wstride);
+    DION_CHECK_LAUNCH(c);
+  }
+  if (nblk > 1) {
+    dim3 grid((unsigned)grid_for(c, sz * sz), (unsigned)s.nb);
+    k_copy_lower_blocks<<<grid, 256, 0, s.st>>>(Tbuf, Gm, r, o, sz, skip, s.wstride);
+    DION_CHECK_LAUNCH(c);
   }
   {
     dim3 grid((unsigned)grid_for(c, sz * sz), (unsigned)s.nb);
@@ -344,7 +350,7 @@ int potrf_inner(StepCtx& s, i64 r, i64 o, i64 sz, const float* shift, bool adapt
 // factor into Linv.  Outer blocks of 512 columns: the diagonal square is factored and
 // inverted by potrf_inner, the panel below it is multiplied by that inverse and the
 // trailing matrix is updated with one rank-512 product (tensor cores where it qualifies).
-int potrf_trtri(StepCtx& s, i64 r, const float* shift, bool adaptive, bool full_inverse) {
+int potrf_trtri(StepCtx& s, i64 r, bool adaptive, bool full_inverse) {
   dion_ctx* c = s.c;
   float* Gm = s.ws + s.L.Gram;
   float* Linv = s.ws + s.L.Linv;
@@ -358,7 +364,7 @@ int potrf_trtri(StepCtx& s, i64 r, const float* shift, bool adaptive, bool full_
   }
   for (i64 J0 = 0; J0 < r; J0 += NBO) {
     const i64 sz = (r - J0 < NBO) ? (r - J0) : NBO;
-    DION_TRY(potrf_inner(s, r, J0, sz, shift, adaptive));
+    DION_TRY(potrf_inner(s, r, J0, sz, adaptive));
     const i64 rem = r - J0 - sz;
     if (rem > 0) {
       float* panel = Gm + (J0 + sz) * r + J0;
@@ -406,7 +412,7 @@ int cholqr_round(StepCtx& s, i64 pin_off, i64 pout_off, i64 rows, i64 r, bool ad
   // Tall panels with r > 512: blocked triangular solve with the 512-column diagonal inverses
   // only (the levels of the triangular inverse above 512 are never formed).
   const bool trsm = (r > NBO) && (rows >= 8192);   // 512-column products need >= 128 row tiles to fill the GPU
-  DION_TRY(potrf_trtri(s, r, nullptr, adaptive, !trsm));
+  DION_TRY(potrf_trtri(s, r, adaptive, !trsm));
   if (adaptive) {
     dim3 grid((unsigned)grid_for(c, rows * r), (unsigned)s.nb);
     k_copy_panel<<<grid, 256, 0, s.st>>>(s.ws + pin_off, r, s.ws + pout_off, r, rows, r, nullptr, s.os + OS_DONE, s.wstride);
@@ -801,7 +807,7 @@ int dion_init(dion_ctx** out, const dion_config* cfg) {
   if (cudaMalloc(&p, sizeof(int) * (8 + MAX_FLAG_SLOTS * OS_SLOT_INTS)) != cudaSuccess) { delete c; return DION_ERR_NOMEM; }
   c->dev_ints = (int*)p;
   if (cudaMemset(p, 0, sizeof(int) * (8 + MAX_FLAG_SLOTS * OS_SLOT_INTS)) != cudaSuccess) { cudaFree(p); delete c; return DION_ERR_CUDA; }
-  if (umma_configure() != DION_OK) { cudaFree(p); delete c; return DION_ERR_CUDA; }
+  if (configure_kernels() != DION_OK) { cudaFree(p); delete c; return DION_ERR_CUDA; }
   if (cfg->workspace_bytes > 0) {
     const int rc = ensure_ws(c, cfg->workspace_bytes);
     if (rc != DION_OK) { cudaFree(c->dev_ints); delete c; return rc; }
@@ -993,7 +999,7 @@ int noalloc_setup(int device, NoallocDevice** out) {
       cudaGetLastError();
       return DION_ERR_CUDA;
     }
-    if (umma_configure() != DION_OK) return DION_ERR_CUDA;
+    if (configure_kernels() != DION_OK) return DION_ERR_CUDA;
     d->base = (unsigned char*)ptr;
     d->sm_count = sms;
     d->ready = true;
@@ -1046,7 +1052,7 @@ extern "C" int dion_debug_gemm(int engine, int precision, const dion_debug_gemm_
   int device = 0, sms = 0;
   if (cudaGetDevice(&device) != cudaSuccess) return DION_ERR_CUDA;
   if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device) != cudaSuccess) return DION_ERR_CUDA;
-  if (umma_configure() != DION_OK) return DION_ERR_CUDA;
+  if (configure_kernels() != DION_OK) return DION_ERR_CUDA;
   GemmArgs g = gemm_args();
   g.M = a->M; g.N = a->N; g.K = a->K;
   g.A = a->A; g.a_si = a->a_si; g.a_sk = a->a_sk;

@@ -48,68 +48,23 @@ __global__ void k_round_begin(const float* __restrict__ G, i64 ld, i64 r, float 
   }
 }
 
-// Cholesky of one jb x jb (jb <= 64) diagonal block, in place (lower factor, the
-// strict upper part of the block is zeroed), plus the inverse of that factor into
-// Dinv (64 x 64, row-major, zero padded).  `shift` is added to the diagonal first.
-// floor_rel == 0 (plain Cholesky QR): a pivot that is <= 0 or not finite sets
-//   os[OS_FAIL] and the BREAKDOWN status bit and is replaced by 1 so that everything
-//   downstream stays finite.
-// floor_rel > 0 (adaptive rounds): a pivot below floor_rel * gdiag[j] (gdiag = the
-//   diagonal of the Gram matrix before elimination) is below the rounding noise of
-//   the Gram matrix.  Column j is then deflated: its diagonal entry becomes
-//   sqrt(floor), the entries below it zero, so the noisy column never reaches the
-//   trailing matrix.  The factor stays triangular and nonsingular for any panel;
-//   the round only improves the conditioning and a later round finishes the job.
-//   DinvP is Dinv with the rows of deflated columns zeroed: the panel below this
-//   block is multiplied by DinvP^T, which yields the zero columns of the factor.
-__global__ void __launch_bounds__(256) k_potrf_diag(float* __restrict__ A, i64 ld, int jb,
-                                                    float* __restrict__ Dinv, float* __restrict__ DinvP,
-                                                    const float* __restrict__ shift,
-                                                    const float* __restrict__ gdiag, float floor_rel,
-                                                    int* __restrict__ os, int adaptive,
-                                                    int* __restrict__ status, i64 wstride) {
-  {  // batched: block b -> matrix b
-    const i64 wo = (i64)blockIdx.x * wstride;
-    A += wo; Dinv += wo; DinvP += wo; gdiag += wo;
-    if (shift != nullptr) shift += wo;
-    os += (i64)blockIdx.x * OS_SLOT_INTS;
-  }
-  if (adaptive && os[OS_DONE] != 0) return;
-  // The block is factored in four 16-column sub-panels: the 16 x 16 diagonal piece by
-  // one warp (two warp barriers per column), the rows below it by one thread per row,
-  // the trailing update by all threads -- three block-wide barriers per sub-panel
-  // instead of three per column.  The inverse is built from 16 x 16 inverses by doubling.
-  constexpr int W = 16;
-  __shared__ float L[NB][NB + 1];
-  __shared__ float X[NB][NB + 1];
-  __shared__ float T[NB / 2][NB / 2 + 1];
-  __shared__ float gd[NB];
-  __shared__ float rdiag[NB];     // 1 / L[j][j]
-  __shared__ int deflated[NB];
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const float sh = (shift != nullptr) ? *shift : 0.f;
-  if (tid < NB) {
-    deflated[tid] = 0;
-    gd[tid] = (floor_rel > 0.f && tid < jb) ? gdiag[tid] + sh : 0.f;
-  }
-  {
-    float v[NB * NB / 256];
-#pragma unroll
-    for (int l = 0; l < NB * NB / 256; ++l) {
-      const int e = tid + l * 256, i = e / NB, c = e % NB;
-      v[l] = (i < jb && c <= i) ? A[(i64)i * ld + c] : 0.f;
-    }
-#pragma unroll
-    for (int l = 0; l < NB * NB / 256; ++l) {
-      const int e = tid + l * 256, i = e / NB, c = e % NB;
-      float x = v[l];
-      if (i == c) x = (i < jb) ? x + sh : 1.f;   // identity padding of a ragged last block
-      L[i][c] = x;
-      X[i][c] = 0.f;
-    }
-  }
-  __syncthreads();
+typedef float (*blk_t)[NB + 1];
+typedef float (*half_blk_t)[NB / 2 + 1];
 
+// Cholesky factor and its inverse of the 64 x 64 block held in L (shared memory; lower
+// triangle, identity padding beyond a ragged block of jb columns), by the 256 threads of
+// a CTA.  On return L holds the factor, X its inverse, deflated[] the deflated columns.
+// X must be zero on entry, gd[] hold the floors' reference values, deflated[] zeros,
+// and a block-wide barrier must separate those writes from the call.
+// The block is factored in four 16-column sub-panels: the 16 x 16 diagonal piece by
+// one warp (one warp barrier per column), the rows below it by one thread per row,
+// the trailing update by all threads -- three block-wide barriers per sub-panel
+// instead of three per column.  The inverse is built from 16 x 16 inverses by doubling.
+__device__ __forceinline__ void potrf_block(blk_t L, blk_t X, half_blk_t T, const float* gd, float* rdiag,
+                                            int* deflated, int jb, float floor_rel, int* __restrict__ os,
+                                            int* __restrict__ status) {
+  constexpr int W = 16;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   int floored = 0, failed = 0;
   float minrel = __int_as_float(0x7f800000);
 #pragma unroll 1
@@ -240,11 +195,203 @@ __global__ void __launch_bounds__(256) k_potrf_diag(float* __restrict__ A, i64 l
     }
     __syncthreads();
   }
+}
+
+// Cholesky of one jb x jb (jb <= 64) diagonal block, in place (lower factor, the
+// strict upper part of the block is zeroed), plus the inverse of that factor into
+// Dinv (64 x 64, row-major, zero padded).
+// floor_rel == 0 (plain Cholesky QR): a pivot that is <= 0 or not finite sets
+//   os[OS_FAIL] and the BREAKDOWN status bit and is replaced by 1 so that everything
+//   downstream stays finite.
+// floor_rel > 0 (adaptive rounds): a pivot below floor_rel * gdiag[j] (gdiag = the
+//   diagonal of the Gram matrix before elimination) is below the rounding noise of
+//   the Gram matrix.  Column j is then deflated: its diagonal entry becomes
+//   sqrt(floor), the entries below it zero, so the noisy column never reaches the
+//   trailing matrix.  The factor stays triangular and nonsingular for any panel;
+//   the round only improves the conditioning and a later round finishes the job.
+//   DinvP is Dinv with the rows of deflated columns zeroed: the panel below this
+//   block is multiplied by DinvP^T, which yields the zero columns of the factor.
+__global__ void __launch_bounds__(256) k_potrf_diag(float* __restrict__ A, i64 ld, int jb,
+                                                    float* __restrict__ Dinv, float* __restrict__ DinvP,
+                                                    const float* __restrict__ gdiag, float floor_rel,
+                                                    int* __restrict__ os, int adaptive,
+                                                    int* __restrict__ status, i64 wstride) {
+  {  // batched: block b -> matrix b
+    const i64 wo = (i64)blockIdx.x * wstride;
+    A += wo; Dinv += wo; DinvP += wo; gdiag += wo;
+    os += (i64)blockIdx.x * OS_SLOT_INTS;
+  }
+  if (adaptive && os[OS_DONE] != 0) return;
+  __shared__ float L[NB][NB + 1];
+  __shared__ float X[NB][NB + 1];
+  __shared__ float T[NB / 2][NB / 2 + 1];
+  __shared__ float gd[NB];
+  __shared__ float rdiag[NB];     // 1 / L[j][j]
+  __shared__ int deflated[NB];
+  const int tid = threadIdx.x;
+  if (tid < NB) {
+    deflated[tid] = 0;
+    gd[tid] = (floor_rel > 0.f && tid < jb) ? gdiag[tid] : 0.f;
+  }
+  {
+    float v[NB * NB / 256];
+#pragma unroll
+    for (int l = 0; l < NB * NB / 256; ++l) {
+      const int e = tid + l * 256, i = e / NB, c = e % NB;
+      v[l] = (i < jb && c <= i) ? A[(i64)i * ld + c] : 0.f;
+    }
+#pragma unroll
+    for (int l = 0; l < NB * NB / 256; ++l) {
+      const int e = tid + l * 256, i = e / NB, c = e % NB;
+      float x = v[l];
+      if (i == c && i >= jb) x = 1.f;   // identity padding of a ragged last block
+      L[i][c] = x;
+      X[i][c] = 0.f;
+    }
+  }
+  __syncthreads();
+
+  potrf_block(L, X, T, gd, rdiag, deflated, jb, floor_rel, os, status);
   for (int e = tid; e < NB * NB; e += 256) {
     const int i = e / NB, c = e % NB;
     if (i < jb && c < jb) A[(i64)i * ld + c] = (c <= i) ? L[i][c] : 0.f;
     Dinv[e] = X[i][c];
-    if (DinvP != nullptr) DinvP[e] = deflated[i] ? 0.f : X[i][c];
+    DinvP[e] = deflated[i] ? 0.f : X[i][c];
+  }
+}
+
+// acc[a][b] += sum_k A[4 ty + a][k] * B[tx + 16 b][k]  (64 x 64 x 64, operands in shared memory)
+__device__ __forceinline__ void mm_nt_64(blk_t A, blk_t B, int ty, int tx, float (&acc)[4][4]) {
+#pragma unroll 8
+  for (int k = 0; k < NB; ++k) {
+    float av[4], bv[4];
+#pragma unroll
+    for (int a = 0; a < 4; ++a) av[a] = A[ty * 4 + a][k];
+#pragma unroll
+    for (int b = 0; b < 4; ++b) bv[b] = B[tx + 16 * b][k];
+#pragma unroll
+    for (int a = 0; a < 4; ++a)
+#pragma unroll
+      for (int b = 0; b < 4; ++b) acc[a][b] = fmaf(av[a], bv[b], acc[a][b]);
+  }
+}
+
+constexpr int CHOL_STEP_SMEM = 3 * NB * (NB + 1) * (int)sizeof(float);
+
+// One step of the right-looking 64-column Cholesky inside the diagonal square [o, o+sz)
+// of the Gram matrix, in ONE launch: with the diagonal block of block column j already
+// factored (its inverse in DinvP), CTA (bi, bk), bk <= bi, forms the two 64-row pieces
+// L_i = A[i][j] DinvP^T and L_k of block column j of the factor, and subtracts
+// L_i L_k^T from the trailing block (i, k).  The CTA of the next diagonal block
+// (bi = bk = 0) then factors and inverts that block right away, so that the next step
+// can start at the next launch; the other CTAs run beside it.  The L pieces go to Lout
+// (same offsets as in A): block column j of A is still read by the other CTAs of this
+// launch, so it cannot be overwritten here; the caller copies Lout back after the last step.
+__global__ void __launch_bounds__(256) k_chol_step(float* __restrict__ A, i64 ld, i64 o, i64 sz, int j,
+                                                   float* __restrict__ Dinv, float* __restrict__ DinvP,
+                                                   float* __restrict__ Lout,
+                                                   const float* __restrict__ gdiag, float floor_rel,
+                                                   int* __restrict__ os, int adaptive,
+                                                   int* __restrict__ status, i64 wstride) {
+  {
+    const i64 wo = (i64)blockIdx.y * wstride;
+    A += wo; Dinv += wo; DinvP += wo; Lout += wo; gdiag += wo;
+    os += (i64)blockIdx.y * OS_SLOT_INTS;
+  }
+  if (adaptive && os[OS_DONE] != 0) return;
+  extern __shared__ __align__(16) float chol_smem[];
+  blk_t S0 = reinterpret_cast<blk_t>(chol_smem);
+  blk_t S1 = reinterpret_cast<blk_t>(chol_smem + NB * (NB + 1));
+  blk_t S2 = reinterpret_cast<blk_t>(chol_smem + 2 * NB * (NB + 1));
+  __shared__ float gd[NB];
+  __shared__ float rdiag[NB];
+  __shared__ int deflated[NB];
+  const int tid = threadIdx.x, ty = tid >> 4, tx = tid & 15;
+  int bi = 0;
+  while ((bi + 1) * (bi + 2) / 2 <= (int)blockIdx.x) ++bi;
+  const int bk = (int)blockIdx.x - bi * (bi + 1) / 2;
+  const i64 cj = o + (i64)j * NB;                    // first column of block column j
+  const i64 ri = cj + (i64)NB * (1 + bi), rk = cj + (i64)NB * (1 + bk);
+  const int rows_i = (int)((o + sz - ri < NB) ? (o + sz - ri) : NB);
+  const int rows_k = (int)((o + sz - rk < NB) ? (o + sz - rk) : NB);
+  const bool diag = (bi == bk);
+  const float* DPj = DinvP + (cj / NB) * (NB * NB);
+  {
+    float vi[NB * NB / 256], vk[NB * NB / 256], vd[NB * NB / 256];
+#pragma unroll
+    for (int l = 0; l < NB * NB / 256; ++l) {
+      const int e = tid + l * 256, i = e / NB, c = e % NB;
+      vi[l] = (i < rows_i) ? A[(ri + i) * ld + cj + c] : 0.f;
+      vk[l] = (!diag && i < rows_k) ? A[(rk + i) * ld + cj + c] : 0.f;
+      vd[l] = DPj[e];
+    }
+#pragma unroll
+    for (int l = 0; l < NB * NB / 256; ++l) {
+      const int e = tid + l * 256, i = e / NB, c = e % NB;
+      S0[i][c] = vi[l];
+      S1[i][c] = vk[l];
+      S2[i][c] = vd[l];
+    }
+  }
+  __syncthreads();
+  float li[4][4] = {}, lk[4][4] = {};
+  mm_nt_64(S0, S2, ty, tx, li);
+  if (!diag) mm_nt_64(S1, S2, ty, tx, lk);
+  __syncthreads();
+#pragma unroll
+  for (int a = 0; a < 4; ++a)
+#pragma unroll
+    for (int b = 0; b < 4; ++b) {
+      S0[ty * 4 + a][tx + 16 * b] = li[a][b];
+      if (!diag) S1[ty * 4 + a][tx + 16 * b] = lk[a][b];
+      if (bk == 0 && ty * 4 + a < rows_i) Lout[(ri + ty * 4 + a) * ld + cj + tx + 16 * b] = li[a][b];
+    }
+  __syncthreads();
+  float acc[4][4] = {};
+  mm_nt_64(S0, diag ? S0 : S1, ty, tx, acc);
+  const bool next_diag = (bi == 0 && bk == 0);
+#pragma unroll
+  for (int a = 0; a < 4; ++a)
+#pragma unroll
+    for (int b = 0; b < 4; ++b) {
+      const int i = ty * 4 + a, c = tx + 16 * b;
+      float v = 0.f;
+      if (i < rows_i && c < rows_k) {
+        v = A[(ri + i) * ld + rk + c] - acc[a][b];
+        if (!next_diag) A[(ri + i) * ld + rk + c] = v;
+      }
+      if (next_diag) S2[i][c] = (c < i) ? v : ((c == i) ? ((i < rows_i) ? v : 1.f) : 0.f);
+    }
+  if (!next_diag) return;
+  // the next diagonal block: factor and invert it here
+  if (tid < NB) {
+    deflated[tid] = 0;
+    gd[tid] = (floor_rel > 0.f && tid < rows_i) ? gdiag[ri + tid] : 0.f;
+  }
+  __syncthreads();                // every thread is done reading S0 / S1
+  for (int e = tid; e < NB * NB; e += 256) S1[e / NB][e % NB] = 0.f;
+  __syncthreads();
+  potrf_block(S2, S1, reinterpret_cast<half_blk_t>(chol_smem), gd, rdiag, deflated, rows_i, floor_rel, os, status);
+  float* Dn = Dinv + (ri / NB) * (NB * NB);
+  float* DPn = DinvP + (ri / NB) * (NB * NB);
+  for (int e = tid; e < NB * NB; e += 256) {
+    const int i = e / NB, c = e % NB;
+    if (i < rows_i && c < rows_i) A[(ri + i) * ld + ri + c] = (c <= i) ? S2[i][c] : 0.f;
+    Dn[e] = S1[i][c];
+    DPn[e] = deflated[i] ? 0.f : S1[i][c];
+  }
+}
+
+// After the last k_chol_step of a square: the blocks of the factor strictly below the
+// block diagonal move from Lout into A.
+__global__ void k_copy_lower_blocks(const float* __restrict__ Lout, float* __restrict__ A, i64 ld, i64 o, i64 sz,
+                                    const int* __restrict__ skip_flag, i64 wstride) {
+  Lout += (i64)blockIdx.y * wstride; A += (i64)blockIdx.y * wstride;
+  if (skip_flag != nullptr && skip_flag[(i64)blockIdx.y * OS_SLOT_INTS] != 0) return;
+  const i64 total = sz * sz;
+  for (i64 e = (i64)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (i64)gridDim.x * blockDim.x) {
+    const i64 i = e / sz, c = e % sz;
+    if (i / NB > c / NB) A[(o + i) * ld + o + c] = Lout[(o + i) * ld + o + c];
   }
 }
 
