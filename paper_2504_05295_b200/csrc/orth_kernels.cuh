@@ -64,17 +64,24 @@ __device__ __forceinline__ void potrf_block(blk_t L, blk_t X, half_blk_t T, cons
                                             int* deflated, int jb, float floor_rel, int* __restrict__ os,
                                             int* __restrict__ status) {
   constexpr int W = 16;
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int tid = threadIdx.x;
   int floored = 0, failed = 0;
   float minrel = __int_as_float(0x7f800000);
 #pragma unroll 1
   for (int c0 = 0; c0 < NB; c0 += W) {
-    if (warp == 0) {
-      // 16 x 16 diagonal piece: lane -> row c0 + (lane % 16), column half lane / 16
-      const int i = lane & (W - 1), half = lane >> 4;
-#pragma unroll 1
+    if (tid == 0) {
+      // 16 x 16 diagonal piece: one thread, the whole lower triangle in registers.  The chain
+      // pivot -> rsqrt -> scale -> update of the next pivot is serial whatever the thread count;
+      // one thread runs it without any barrier or shuffle and fills the gaps with the rest of
+      // the rank-1 update.
+      float a[W][W];
+#pragma unroll
+      for (int i = 0; i < W; ++i)
+#pragma unroll
+        for (int c = 0; c <= i; ++c) a[i][c] = L[c0 + i][c0 + c];
+#pragma unroll
       for (int j = 0; j < W; ++j) {
-        float p = L[c0 + j][c0 + j];
+        float p = a[j][j];
         bool defl = false;
         if (c0 + j < jb) {
           if (floor_rel > 0.f) {
@@ -93,24 +100,21 @@ __device__ __forceinline__ void potrf_block(blk_t L, blk_t X, half_blk_t T, cons
           }
         }
         const float inv = rsqrtf(p);
-        float v = 0.f;
-        if (i > j && !defl) v = L[c0 + i][c0 + j] * inv;
-        if (half == 0) {
-          if (i == j) { rdiag[c0 + j] = inv; if (defl) deflated[c0 + j] = 1; }
-          else if (i > j) L[c0 + i][c0 + j] = v;
-        }
-        // rank-1 update of the remaining columns of this piece: each lane owns 8 columns of its
-        // row; the column-j entry of row c comes by shuffle from the lane that just computed it
-        // (both halves hold the same v), so one warp barrier per column is enough
+        const float sc = defl ? 0.f : inv;
+        a[j][j] = p * inv;
+        rdiag[c0 + j] = inv;
+        if (defl) deflated[c0 + j] = 1;
 #pragma unroll
-        for (int q = 0; q < W / 2; ++q) {
-          const int c = half * (W / 2) + q;
-          const float vc = __shfl_sync(0xffffffffu, v, c);
-          if (c > j && c <= i) L[c0 + i][c0 + c] = fmaf(-v, vc, L[c0 + i][c0 + c]);
-        }
-        if (half == 0 && i == j) L[c0 + j][c0 + j] = p * inv;   // after every lane has read the pivot
-        __syncwarp();
+        for (int i = j + 1; i < W; ++i) a[i][j] *= sc;
+#pragma unroll
+        for (int c = j + 1; c < W; ++c)
+#pragma unroll
+          for (int i = c; i < W; ++i) a[i][c] = fmaf(-a[i][j], a[c][j], a[i][c]);
       }
+#pragma unroll
+      for (int i = 0; i < W; ++i)
+#pragma unroll
+        for (int c = 0; c <= i; ++c) L[c0 + i][c0 + c] = a[i][c];
     }
     __syncthreads();
     const int below = NB - c0 - W;   // rows under the diagonal piece
