@@ -127,6 +127,16 @@ typedef struct {
   int64_t ldq;
   float* colnorm_out;   /* optional: r floats, the column norms of R (estimates of the
                            leading singular values of B); may be NULL                */
+  int transposed;       /* 0: standard form.  1: transposed form (Section 4.3, "other
+                           variants": the power iteration runs on M^T): Q is m x r,
+                             P = B^T Q (n x r),  U = Orthonormalize(P),  R = B U (m x r),
+                             M <- B - (1 - mu) R U^T,  Q <- ColNorm(R),
+                             X <- X - lr * sqrt(m/n) * Q U^T.
+                           This is the standard step applied to X^T, M^T, G^T with the
+                           arrays left in place; the factor sqrt(m/n) stays that of the
+                           stored m x n parameter (rows = "out"), so both forms scale
+                           the update alike.  It puts the orthonormalized panel on the
+                           n side: cheaper when m > n.  dion_lazy_step rejects it.   */
 } dion_matrix;
 
 /* Fill *cfg with the defaults: mu 0.95, eps 1e-8, fp32, AUTO, AUTO, device 0, no reserve. */

@@ -137,6 +137,21 @@ def step(X, M, G, Q, mu: float, eta: float, eps: float = 1e-8) -> StepResult:
     return StepResult(X, M, Q, d, P, U, R, rc)
 
 
+def step_transposed(X, M, G, Q, mu: float, eta: float, eps: float = 1e-8) -> StepResult:
+    """One Dion step in the transposed form (Section 4.3, "other variants": the power
+    iteration runs on M^T).  By definition this is the standard step on the transposed
+    arrays, X^T, M^T, G^T (n x m) with Q of shape m x r.  The update keeps the factor
+    sqrt(m/n) of the stored m x n parameter (rows = "out"): the standard step on the
+    n x m arrays applies sqrt(n/m), so it is given eta * m / n.
+    Returns X, M (m x n again), Q (m x r), d, and P, U (n x r), R (m x r)."""
+    X = _f64(X); M = _f64(M); G = _f64(G)
+    m, n = X.shape
+    res = step(np.ascontiguousarray(X.T), np.ascontiguousarray(M.T), np.ascontiguousarray(G.T), Q,
+               mu, float(eta) * m / n, eps)
+    return StepResult(np.ascontiguousarray(res.X.T), np.ascontiguousarray(res.M.T), res.Q, res.d,
+                      res.P, res.U, res.R, res.degenerate)
+
+
 def sym_power_iter(M, Q):
     """SymPowerIter1 (Algorithm 6): Orthonormalize(M^T M V)."""
     M = _f64(M); Q = _f64(Q).copy()

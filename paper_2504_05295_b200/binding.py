@@ -41,7 +41,7 @@ class DionMatrix(ctypes.Structure):
                 ("M", ctypes.c_void_p), ("ldm", ctypes.c_int64),
                 ("G", ctypes.c_void_p), ("ldg", ctypes.c_int64), ("g_dtype", ctypes.c_int),
                 ("Q", ctypes.c_void_p), ("ldq", ctypes.c_int64),
-                ("colnorm_out", ctypes.c_void_p)]
+                ("colnorm_out", ctypes.c_void_p), ("transposed", ctypes.c_int)]
 
 
 class DionError(RuntimeError):
@@ -113,10 +113,10 @@ def _stream_ptr(stream: Optional[torch.cuda.Stream]) -> int:
 
 
 def matrix_desc(X: torch.Tensor, M: torch.Tensor, G: torch.Tensor, Q: torch.Tensor,
-                colnorm_out: Optional[torch.Tensor] = None) -> DionMatrix:
+                colnorm_out: Optional[torch.Tensor] = None, transposed: bool = False) -> DionMatrix:
     """Describes one parameter for the C-ABI.  Tensors must be CUDA, 2-D, row-major
     (unit stride along the last dimension); a row stride larger than the width is
-    passed on as the leading dimension."""
+    passed on as the leading dimension.  Q is n x r, or m x r in the transposed form."""
     for name, t in (("X", X), ("M", M), ("G", G), ("Q", Q)):
         if not t.is_cuda or t.dim() != 2 or t.stride(1) != 1:
             raise ValueError(f"{name} must be a 2-D CUDA tensor with unit column stride")
@@ -129,7 +129,7 @@ def matrix_desc(X: torch.Tensor, M: torch.Tensor, G: torch.Tensor, Q: torch.Tens
     else:
         raise ValueError("G must be float32 or bfloat16")
     m, n = X.shape
-    if tuple(M.shape) != (m, n) or tuple(G.shape) != (m, n) or Q.shape[0] != n:
+    if tuple(M.shape) != (m, n) or tuple(G.shape) != (m, n) or Q.shape[0] != (m if transposed else n):
         raise ValueError("shape mismatch between X, M, G and Q")
     d = DionMatrix()
     d.m, d.n, d.r = m, n, Q.shape[1]
@@ -144,15 +144,16 @@ def matrix_desc(X: torch.Tensor, M: torch.Tensor, G: torch.Tensor, Q: torch.Tens
         d.colnorm_out = colnorm_out.data_ptr()
     else:
         d.colnorm_out = None
+    d.transposed = int(bool(transposed))
     return d
 
 
 def step_noalloc(X, M, G, Q, lr: float, mu: float = 0.95, eps: float = 1e-8, colnorm_out=None,
-                 stream=None) -> None:
+                 stream=None, transposed: bool = False) -> None:
     """One Dion step through ``dion_step_noalloc``: no context, no device allocation; the
     scratch is the library's built-in 24 MiB array on the current device.  Calls must not
     overlap on the GPU.  Raises DionError(-8) when the shape needs more scratch than that."""
-    d = matrix_desc(X, M, G, Q, colnorm_out)
+    d = matrix_desc(X, M, G, Q, colnorm_out, transposed)
     _check(load_library().dion_step_noalloc(ctypes.byref(d), float(lr), float(mu), float(eps),
                                             _stream_ptr(stream)))
 
@@ -180,8 +181,8 @@ class Dion:
         _check(lib.dion_init(ctypes.byref(self._ctx), ctypes.byref(cfg)))
         self.device = int(device)
 
-    def step(self, X, M, G, Q, lr: float, colnorm_out=None, stream=None) -> None:
-        d = matrix_desc(X, M, G, Q, colnorm_out)
+    def step(self, X, M, G, Q, lr: float, colnorm_out=None, stream=None, transposed: bool = False) -> None:
+        d = matrix_desc(X, M, G, Q, colnorm_out, transposed)
         _check(self._lib.dion_step(self._ctx, ctypes.byref(d), float(lr), _stream_ptr(stream)))
 
     def step_desc(self, desc: DionMatrix, lr: float, stream_ptr: int) -> None:
@@ -194,7 +195,8 @@ class Dion:
         return arr
 
     def step_grouped(self, mats: Iterable[Tuple], lr: float, stream=None) -> None:
-        """mats: iterable of (X, M, G, Q) or (X, M, G, Q, colnorm_out)."""
+        """mats: iterable of (X, M, G, Q), (X, M, G, Q, colnorm_out) or
+        (X, M, G, Q, colnorm_out, transposed)."""
         descs: List[DionMatrix] = [matrix_desc(*t) for t in mats]
         arr = self.pack(descs)
         _check(self._lib.dion_step_grouped(self._ctx, arr, len(descs), float(lr), _stream_ptr(stream)))

@@ -419,7 +419,9 @@ int cholqr_round(StepCtx& s, i64 pin_off, i64 pout_off, i64 rows, i64 r, bool ad
     DION_CHECK_LAUNCH(c);
   }
   if (trsm) {
-    // Pout_J = (Pin_J - sum_{K<J} Pout_K L_{J,K}^T) Linv_JJ^T, block columns J of 512
+    // Pout_J = (Pin_J - sum_{K<J} Pout_K L_{J,K}^T) Linv_JJ^T, block columns J of 512.
+    // The solves run with the plain 3xTF32 product: their rounding error enters U once (~1e-6),
+    // whereas an error in the Gram matrix or its factor is amplified by the panel's conditioning.
     const float* Lm = s.ws + s.L.Gram;     // the factor, lower
     float* Wt = s.ws + s.L.R;              // rows x 512 temporary (R is free during the orthonormalization)
     for (i64 J0 = 0; J0 < r; J0 += NBO) {
@@ -432,7 +434,7 @@ int cholqr_round(StepCtx& s, i64 pin_off, i64 pout_off, i64 rows, i64 r, bool ad
         w.A = s.ws + pout_off; w.a_si = r; w.a_sk = 1;
         w.B = Lm + J0 * r; w.b_sk = 1; w.b_sn = r;
         w.C = Wt; w.ldc = NBO; w.epi = EPI_C2_SUB; w.C2 = rhs; w.ldc2 = r; w.c2_mode = ADD_F32;
-        w.skip_flag = skip; w.precise = adaptive ? 1 : 0;
+        w.skip_flag = skip;
         for (int m = 0; m < s.nb; ++m) {
           GemmArgs wm = for_matrix(s, w, m, true, true, true);
           wm.C2 = (const float*)wm.C2 + (i64)m * s.wstride;
@@ -444,7 +446,7 @@ int cholqr_round(StepCtx& s, i64 pin_off, i64 pout_off, i64 rows, i64 r, bool ad
       v.M = rows; v.N = sz; v.K = sz;
       v.A = rhs; v.a_si = rhs_ld; v.a_sk = 1;
       v.B = s.ws + s.L.Linv + J0 * r + J0; v.b_sk = 1; v.b_sn = r; v.klimit = 1;
-      v.C = s.ws + pout_off + J0; v.ldc = r; v.epi = EPI_STORE; v.skip_flag = skip; v.precise = adaptive ? 1 : 0;
+      v.C = s.ws + pout_off + J0; v.ldc = r; v.epi = EPI_STORE; v.skip_flag = skip;
       for (int m = 0; m < s.nb; ++m) DION_TRY(launch_gemm(s, for_matrix(s, v, m, true, true, true), m));
     }
     if (adaptive) {
@@ -457,7 +459,7 @@ int cholqr_round(StepCtx& s, i64 pin_off, i64 pout_off, i64 rows, i64 r, bool ad
   u.M = rows; u.N = r; u.K = r;
   u.A = s.ws + pin_off; u.a_si = r; u.a_sk = 1;
   u.B = s.ws + s.L.Linv; u.b_sk = 1; u.b_sn = r; u.klimit = 1;
-  u.C = s.ws + pout_off; u.ldc = r; u.epi = EPI_STORE; u.skip_flag = skip; u.precise = adaptive ? 1 : 0;
+  u.C = s.ws + pout_off; u.ldc = r; u.epi = EPI_STORE; u.skip_flag = skip;
   for (int m = 0; m < s.nb; ++m) DION_TRY(launch_gemm(s, for_matrix(s, u, m, true, true, true), m));
   if (adaptive) {
     k_round_end<<<s.nb, 1, 0, s.st>>>(s.os, GOOD_REL, DONE_REL, c->dev_ints + 2);
@@ -556,12 +558,14 @@ int validate(const dion_matrix* a) {
   if (a->m < 1 || a->n < 1) return DION_ERR_SHAPE;
   if (a->r < 1 || a->r > a->m || a->r > a->n) return DION_ERR_SHAPE;
   if (a->ldx < a->n || a->ldm < a->n || a->ldg < a->n || a->ldq < a->r) return DION_ERR_SHAPE;
+  if (a->transposed != 0 && a->transposed != 1) return DION_ERR_INVALID;
+  const i64 qrows = a->transposed ? a->m : a->n;
   const size_t gsz = (a->g_dtype == DION_BF16) ? 2 : 4;
   if (((uintptr_t)a->X & 3) || ((uintptr_t)a->M & 3) || ((uintptr_t)a->Q & 3) || ((uintptr_t)a->G & (gsz - 1)))
     return DION_ERR_ALIGN;
   if (a->colnorm_out != nullptr && ((uintptr_t)a->colnorm_out & 3)) return DION_ERR_ALIGN;
   const size_t nx = (size_t)((a->m - 1) * a->ldx + a->n) * 4, nm = (size_t)((a->m - 1) * a->ldm + a->n) * 4;
-  const size_t ng = (size_t)((a->m - 1) * a->ldg + a->n) * gsz, nq = (size_t)((a->n - 1) * a->ldq + a->r) * 4;
+  const size_t ng = (size_t)((a->m - 1) * a->ldg + a->n) * gsz, nq = (size_t)((qrows - 1) * a->ldq + a->r) * 4;
   if (overlap(a->X, nx, a->M, nm) || overlap(a->X, nx, a->G, ng) || overlap(a->X, nx, a->Q, nq) ||
       overlap(a->M, nm, a->G, ng) || overlap(a->M, nm, a->Q, nq) || overlap(a->G, ng, a->Q, nq))
     return DION_ERR_ALIAS;
@@ -599,15 +603,23 @@ int step_batch(dion_ctx* c, const dion_matrix* const* list, int nb, float lr, cu
   DION_TRY(begin_step(c, a0, nb, st, &s));
   const i64 m = a0->m, n = a0->n, r = a0->r;
 
-  // P = (M + G) Q
+  // Standard form: the power iteration runs on B = M + G (panel P = B Q, m x r; Q is n x r).
+  // Transposed form: it runs on B^T (panel P = B^T Q, n x r; Q is m x r), and the rank-r
+  // products come out transposed: M <- B - (1 - mu) R U^T, X <- X - lr sqrt(m/n) Q U^T.
+  const bool tr = a0->transposed != 0;
+  const i64 prow = tr ? n : m;     // rows of the panel that is orthonormalized
+  const i64 qrow = tr ? m : n;     // rows of R and Q
+  const auto g_mode = [](const dion_matrix* a) { return (a->g_dtype == DION_BF16) ? ADD_BF16 : ADD_F32; };
+
+  // P = (M + G) Q   (transposed form: (M + G)^T Q)
   {
   PhaseScope ps(c, st, DION_PHASE_P);
   for (int b = 0; b < nb; ++b) {
     const dion_matrix* a = list[b];
     GemmArgs p = gemm_args();
-    p.M = m; p.N = r; p.K = n;
-    p.A = (const float*)a->M; p.a_si = a->ldm; p.a_sk = 1;
-    p.A2 = a->G; p.a2_si = a->ldg; p.a2_sk = 1; p.a2_mode = (a->g_dtype == DION_BF16) ? ADD_BF16 : ADD_F32;
+    p.M = prow; p.N = r; p.K = qrow;
+    p.A = (const float*)a->M; p.a_si = tr ? 1 : a->ldm; p.a_sk = tr ? a->ldm : 1;
+    p.A2 = a->G; p.a2_si = tr ? 1 : a->ldg; p.a2_sk = tr ? a->ldg : 1; p.a2_mode = g_mode(a);
     p.B = (const float*)a->Q; p.b_sk = a->ldq; p.b_sn = 1;
     p.C = s.W(b, s.L.P0); p.ldc = r; p.epi = EPI_STORE;
     // an ill-conditioned panel amplifies the error of P: use the accurate product there
@@ -621,37 +633,37 @@ int step_batch(dion_ctx* c, const dion_matrix* const* list, int nb, float lr, cu
   {
   PhaseScope ps(c, st, DION_PHASE_ORTH);
   s.in_orth = true;
-  const int rc_orth = orthonormalize(s, m, r, (m < n) ? m : n, &U_off);
+  const int rc_orth = orthonormalize(s, prow, r, (m < n) ? m : n, &U_off);
   s.in_orth = false;
   DION_TRY(rc_orth);
   }
 
-  // R = (M + G)^T U
+  // R = (M + G)^T U   (transposed form: (M + G) U)
   {
   PhaseScope ps(c, st, DION_PHASE_R);
   for (int b = 0; b < nb; ++b) {
     const dion_matrix* a = list[b];
     GemmArgs w = gemm_args();
-    w.M = n; w.N = r; w.K = m;
-    w.A = (const float*)a->M; w.a_si = 1; w.a_sk = a->ldm;
-    w.A2 = a->G; w.a2_si = 1; w.a2_sk = a->ldg; w.a2_mode = (a->g_dtype == DION_BF16) ? ADD_BF16 : ADD_F32;
+    w.M = qrow; w.N = r; w.K = prow;
+    w.A = (const float*)a->M; w.a_si = tr ? a->ldm : 1; w.a_sk = tr ? 1 : a->ldm;
+    w.A2 = a->G; w.a2_si = tr ? a->ldg : 1; w.a2_sk = tr ? 1 : a->ldg; w.a2_mode = g_mode(a);
     w.B = s.W(b, U_off); w.b_sk = r; w.b_sn = 1;
     w.C = s.W(b, s.L.R); w.ldc = r; w.epi = EPI_STORE;
     DION_TRY(launch_gemm(s, w, b));
   }
   }
 
-  // M <- (M + G) - (1 - mu) U R^T
+  // M <- (M + G) - (1 - mu) U R^T   (transposed form: R U^T)
   {
   PhaseScope ps(c, st, DION_PHASE_EF);
   for (int b = 0; b < nb; ++b) {
     const dion_matrix* a = list[b];
     GemmArgs e = gemm_args();
     e.M = m; e.N = n; e.K = r;
-    e.A = s.W(b, U_off); e.a_si = r; e.a_sk = 1;
-    e.B = s.W(b, s.L.R); e.b_sk = 1; e.b_sn = r;
+    e.A = s.W(b, tr ? s.L.R : U_off); e.a_si = r; e.a_sk = 1;
+    e.B = s.W(b, tr ? U_off : s.L.R); e.b_sk = 1; e.b_sn = r;
     e.C = (float*)a->M; e.ldc = a->ldm; e.epi = EPI_ADD2_SUB;
-    e.C2 = a->G; e.ldc2 = a->ldg; e.c2_mode = (a->g_dtype == DION_BF16) ? ADD_BF16 : ADD_F32;
+    e.C2 = a->G; e.ldc2 = a->ldg; e.c2_mode = g_mode(a);
     e.alpha = 1.f - c->cfg.mu;
     e.skip_flag = s.OS(b) + OS_FAIL;
     DION_TRY(launch_gemm(s, e, b));
@@ -663,19 +675,24 @@ int step_batch(dion_ctx* c, const dion_matrix* const* list, int nb, float lr, cu
   PhaseScope ps(c, st, DION_PHASE_COLNORM);
   for (int b = 0; b < nb; ++b) {
     const dion_matrix* a = list[b];
-    DION_TRY(colnorm(s, b, s.W(b, s.L.R), n, r, (float*)a->Q, a->ldq, a->colnorm_out));
+    DION_TRY(colnorm(s, b, s.W(b, s.L.R), qrow, r, (float*)a->Q, a->ldq, a->colnorm_out));
   }
   }
 
-  // X <- X - lr sqrt(m/n) U Q^T
+  // X <- X - lr sqrt(m/n) U Q^T   (transposed form: Q U^T)
   {
   PhaseScope ps(c, st, DION_PHASE_X);
   for (int b = 0; b < nb; ++b) {
     const dion_matrix* a = list[b];
     GemmArgs x = gemm_args();
     x.M = m; x.N = n; x.K = r;
-    x.A = s.W(b, U_off); x.a_si = r; x.a_sk = 1;
-    x.B = (const float*)a->Q; x.b_sk = 1; x.b_sn = a->ldq;
+    if (tr) {
+      x.A = (const float*)a->Q; x.a_si = a->ldq; x.a_sk = 1;
+      x.B = s.W(b, U_off); x.b_sk = 1; x.b_sn = r;
+    } else {
+      x.A = s.W(b, U_off); x.a_si = r; x.a_sk = 1;
+      x.B = (const float*)a->Q; x.b_sk = 1; x.b_sn = a->ldq;
+    }
     x.C = (float*)a->X; x.ldc = a->ldx; x.epi = EPI_SUB;
     x.alpha = lr * sqrtf((float)((double)m / (double)n));
     x.skip_flag = s.OS(b) + OS_FAIL;
@@ -851,7 +868,8 @@ int dion_step_grouped(dion_ctx* ctx, const dion_matrix* list, int count, float l
     if (cap > MAX_CHAIN) cap = MAX_CHAIN;
     chain.clear();
     for (int j = i; j < count; ++j) {
-      if (done[j] || list[j].m != list[i].m || list[j].n != list[i].n || list[j].r != list[i].r) continue;
+      if (done[j] || list[j].m != list[i].m || list[j].n != list[i].n || list[j].r != list[i].r ||
+          list[j].transposed != list[i].transposed) continue;
       done[j] = 1;
       chain.push_back(&list[j]);
       if (chain.size() == cap) { chains.push_back(chain); chain.clear(); }
@@ -870,6 +888,7 @@ int dion_step_grouped(dion_ctx* ctx, const dion_matrix* list, int count, float l
 int dion_lazy_step(dion_ctx* ctx, const dion_matrix* a, float lr, int refresh, void* cuda_stream) {
   if (ctx == nullptr) return DION_ERR_INVALID;
   DION_TRY(validate(a));
+  if (a->transposed) return DION_ERR_INVALID;   // Algorithm 6 is built in the standard form only
   if (cudaSetDevice(ctx->cfg.device) != cudaSuccess) return DION_ERR_CUDA;
   DION_TRY(ensure_ws(ctx, dion_workspace_bytes(ctx, a->m, a->n, a->r)));
   return lazy_one(ctx, a, lr, refresh, (cudaStream_t)cuda_stream);

@@ -3,6 +3,7 @@ declares; argument errors are reported as codes (no compute is attempted)."""
 import ctypes
 import os
 import re
+import subprocess
 
 import pytest
 
@@ -38,10 +39,27 @@ def test_header_symbols_are_exported(lib):
         assert hasattr(raw, nm), f"{nm} declared in include/ but not exported"
 
 
-def test_struct_layout_matches_header():
-    # 3 x int64, then (pointer, int64) pairs; g_dtype is padded to 8 bytes
-    assert ctypes.sizeof(binding.DionMatrix) == 8 * 3 + 16 + 16 + 24 + 16 + 8
-    assert ctypes.sizeof(binding.DionConfig) == 32
+def test_struct_layout_matches_header(tmp_path):
+    # the C compiler's view of include/dion.h against the ctypes structures, field by field
+    fields_m = [f for f, _ in binding.DionMatrix._fields_]
+    fields_c = [f for f, _ in binding.DionConfig._fields_]
+    src = tmp_path / "layout.c"
+    lines = ['#include <stdio.h>', '#include <stddef.h>', '#include "dion.h"', 'int main(void) {',
+             '  printf("%zu %zu\\n", sizeof(dion_matrix), sizeof(dion_config));']
+    lines += [f'  printf("%zu\\n", offsetof(dion_matrix, {f}));' for f in fields_m]
+    lines += [f'  printf("%zu\\n", offsetof(dion_config, {f}));' for f in fields_c]
+    lines += ['  return 0;', '}']
+    src.write_text("\n".join(lines))
+    exe = tmp_path / "layout"
+    inc = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "include")
+    subprocess.run(["gcc", "-I", inc, str(src), "-o", str(exe)], check=True)
+    out = subprocess.run([str(exe)], check=True, capture_output=True, text=True).stdout.split()
+    vals = [int(v) for v in out]
+    assert vals[0] == ctypes.sizeof(binding.DionMatrix) and vals[1] == ctypes.sizeof(binding.DionConfig)
+    got = vals[2:]
+    want = [getattr(binding.DionMatrix, f).offset for f in fields_m] + \
+           [getattr(binding.DionConfig, f).offset for f in fields_c]
+    assert got == want
 
 
 def test_error_codes_and_strings(lib):

@@ -154,6 +154,45 @@ def test_update_norm(m, n, r):
     assert abs(expect - ETA * np.sqrt(m / n) * np.sqrt(r)) < 1e-6 * expect
 
 
+# -- transposed form (Section 4.3, "other variants"): invariants written out on the stored arrays --
+
+@pytest.mark.parametrize("m,n,r", [(40, 24, 6), (24, 40, 6), (20, 20, 20), (48, 16, 16)])
+def test_transposed_form_invariants(m, n, r):
+    rng = np.random.default_rng(300 + m + n + r)
+    X = 0.02 * rng.standard_normal((m, n)); M = rng.standard_normal((m, n)); G = rng.standard_normal((m, n))
+    Q = rng.standard_normal((m, r)); Q /= np.linalg.norm(Q, axis=0)        # the warm start lives on the m side
+    res = orc.step_transposed(X, M, G, Q, MU, ETA, EPS)
+    B = M + G
+    # the panel is B^T Q (n x r); its orthonormal factor from the library QR, sign-fixed
+    q, rr = np.linalg.qr(B.T @ Q)
+    U = q * np.sign(np.diag(rr))
+    assert res.U.shape == (n, r) and rel(res.U, U) < 1e-10
+    R = B @ U                                                              # m x r
+    assert rel(res.R, R) < 1e-10
+    assert rel(res.M, B - (1 - MU) * R @ U.T) < 1e-10                      # error feedback, transposed product
+    d = np.linalg.norm(R, axis=0)
+    assert np.allclose(res.d, d, rtol=1e-10)
+    assert res.Q.shape == (m, r) and rel(res.Q, R / (d + EPS)) < 1e-10
+    # the update keeps sqrt(m/n) of the stored parameter and has the transposed outer product
+    assert rel(X - res.X, ETA * np.sqrt(m / n) * res.Q @ U.T) < 1e-10
+    # rows of the update lie in span(U): (X - X') (I - U U^T) = 0
+    D = X - res.X
+    assert np.linalg.norm(D - (D @ U) @ U.T) < 1e-12 * np.linalg.norm(D)
+    if r == min(m, n):
+        assert rel(res.M, MU * B) < 1e-10                                  # full rank: R U^T = B
+
+
+def test_transposed_form_differs_from_standard_form():
+    # the two forms orthonormalize different panels: same subspace iteration target, different update
+    rng = np.random.default_rng(31)
+    m = n = 12; r = 3
+    X, M, G, Q = draw(rng, m, n, r)
+    a = orc.step(X, M, G, Q, MU, ETA, EPS)
+    b = orc.step_transposed(X, M, G, Q, MU, ETA, EPS)
+    assert rel(a.X, b.X) > 1e-3
+    assert abs(np.linalg.norm(a.X - X) - np.linalg.norm(b.X - X)) < 1e-6 * np.linalg.norm(a.X - X)   # same scale
+
+
 # -- pin 6: two-sided orthogonal equivariance (catches layout / transposition) --
 
 def test_orthogonal_equivariance():
