@@ -298,8 +298,12 @@ def run_ours(args):
                                  g_dtype=torch.bfloat16 if case_gbytes(c) == 2 else torch.float32)
         gs = [pb.grad(t) for t in range(2)]
         d = torch.zeros(r, device=dev)
-        descs = [binding.matrix_desc(pb.X, pb.M, g, pb.Q, d) for g in gs]
-        state.append({"pb": pb, "G": gs, "d": d, "descs": descs})
+        # --form short-side: the transposed form wherever it shortens the orthonormalized panel
+        tr = args.form == "short-side" and m > n
+        if tr:
+            pb.Q = inputs.row_side_factor(pb)
+        descs = [binding.matrix_desc(pb.X, pb.M, g, pb.Q, d, tr) for g in gs]
+        state.append({"pb": pb, "G": gs, "d": d, "descs": descs, "transposed": tr})
     torch.cuda.synchronize()
 
     opt = binding.Dion(mu=MU, eps=EPS, precision=args.precision, orth=args.orth, engine=args.engine, device=local)
@@ -472,6 +476,7 @@ def run_ours(args):
                        "engine": ["auto", "simt", "tensor"][args.engine],
                        "precision": ["fp32 (3xTF32 on tensor cores / FMA)", "bf16 operands"][args.precision],
                        "orth": ["auto", "cholqr2", "shifted3", "householder"][args.orth],
+                       "form": args.form, "n_transposed": sum(1 for st in state if st["transposed"]),
                        "l2": "inputs larger than L2: the workload's X, M, G (GBs) cycle through between repeats",
                        "replicas": world, "workspace_bytes": need},
             "cases": ([] if len(cases) > 32 else
@@ -500,6 +505,8 @@ def main():
     ap.add_argument("--engine", type=int, default=0, help="0 auto, 1 simt, 2 tensor")
     ap.add_argument("--precision", type=int, default=0, help="0 fp32, 1 bf16 operands")
     ap.add_argument("--orth", type=int, default=0, help="0 auto, 1 cholqr2, 2 shifted3, 3 householder")
+    ap.add_argument("--form", default="standard", choices=["standard", "short-side"],
+                    help="short-side: matrices with m > n take the transposed form (panel n x r instead of m x r)")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-baseline leg")
     args = ap.parse_args()
     if args.impl == "reference":

@@ -114,6 +114,15 @@ def make_problem(m: int, n: int, r: int, seed: int = 0, k: int = 0, ks: int = 64
     return DionProblem(m, n, r, X, M, Q, S, Us, Vs, s, sk, g_dtype)
 
 
+def row_side_factor(pb: DionProblem, device=None) -> torch.Tensor:
+    """Warm-start factor of the transposed form: m x r, unit-norm Gaussian columns,
+    drawn from the matrix's own seed (independent of its n x r factor)."""
+    dev = pb.X.device if device is None else device
+    gen = _gen(matrix_seed(pb.seed, 104729), dev)
+    Q = _randn((pb.m, pb.r), gen, dev)
+    return (Q / torch.linalg.vector_norm(Q.double(), dim=0).float()).contiguous()
+
+
 # ---------------------------------------------------------------------------
 # The benchmark configurations (shapes only; tensors are drawn by make_problem)
 # ---------------------------------------------------------------------------
