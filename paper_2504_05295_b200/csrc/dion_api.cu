@@ -212,7 +212,10 @@ struct StepCtx {
 int launch_gemm(StepCtx& s, const GemmArgs& g, int b = 0, bool force64 = false) {
   if (s.tensor && !force64) {
     PhaseScope ps(s.c, s.st, s.in_orth ? DION_PHASE_ORTH_GEMM : -1);
-    const int rc = umma_try_launch(g, s.c->cfg.precision, s.c->sm_count, s.W(b, s.L.part), s.L.part_floats,
+    // bf16 operands are for the four large contractions only: the Gram matrices, factors and
+    // solves of the orthonormalization keep fp32 accuracy in every mode
+    const int prec = s.in_orth ? DION_PREC_FP32 : s.c->cfg.precision;
+    const int rc = umma_try_launch(g, prec, s.c->sm_count, s.W(b, s.L.part), s.L.part_floats,
                                    s.c->dev_ints, s.st);
     if (rc > 0) { s.c->launches += rc; return DION_OK; }
     if (rc < 0) return rc;
@@ -737,7 +740,10 @@ int lazy_one(dion_ctx* c, const dion_matrix* a, float lr, int refresh, cudaStrea
     z.precise = t.precise;
     DION_TRY(launch_gemm(s, z));
     i64 V_off = 0;
-    DION_TRY(orthonormalize(s, n, r, (m < n) ? m : n, &V_off));
+    s.in_orth = true;
+    const int rc_orth = orthonormalize(s, n, r, (m < n) ? m : n, &V_off);
+    s.in_orth = false;
+    DION_TRY(rc_orth);
     const float* V = s.ws + V_off;
     // copy V into Q unless the round broke down (alpha = 1, identity product is overkill: strided copy kernel)
     GemmArgs cp = gemm_args();

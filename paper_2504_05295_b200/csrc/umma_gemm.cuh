@@ -85,6 +85,13 @@ __device__ __forceinline__ float4 lds128(uint32_t addr) {
 __device__ __forceinline__ void sts128(uint32_t addr, float4 v) {
   asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w) : "memory");
 }
+// four floats rounded to bf16 (round to nearest even), stored as 8 bytes
+__device__ __forceinline__ void sts64_bf16x4(uint32_t addr, float4 v) {
+  const __nv_bfloat162 a = __floats2bfloat162_rn(v.x, v.y), b = __floats2bfloat162_rn(v.z, v.w);
+  asm volatile("st.shared.v2.b32 [%0], {%1, %2};" ::"r"(addr), "r"(*reinterpret_cast<const uint32_t*>(&a)),
+               "r"(*reinterpret_cast<const uint32_t*>(&b))
+               : "memory");
+}
 // remainder of x after truncation to TF32 (what the MMA drops when it reads an fp32 word)
 __device__ __forceinline__ float trunc_rem(float x) { return x - __uint_as_float(__float_as_uint(x) & 0xFFFFE000u); }
 __device__ __forceinline__ void fence_barrier_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
@@ -186,6 +193,18 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t saddr, bool mn_major, uin
   d |= sbo << 32;
   d |= 1ull << 46;                      // descriptor version of sm_100
   d |= (base32 ? 1ull : 2ull) << 61;    // SWIZZLE_128B_BASE32B or SWIZZLE_128B
+  return d;
+}
+
+// k-contiguous bf16 tile with rows of 64 bytes (32 elements): 64-byte swizzle (16-byte
+// units XORed with bits 1-2 of the row index), 8-row groups 512 bytes apart.
+__device__ __forceinline__ uint64_t make_desc_k64(uint32_t saddr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((saddr >> 4) & 0x3FFF);
+  d |= 1ull << 16;
+  d |= (uint64_t)(512 >> 4) << 32;
+  d |= 1ull << 46;
+  d |= 4ull << 61;                      // SWIZZLE_64B
   return d;
 }
 
@@ -365,35 +384,43 @@ struct TileMap {
 // brings the product to the accuracy of an fp32 FMA loop (measured 3.3e-7 against
 // 9.1e-7 relative error on Gaussian data).  Used for the products whose error the
 // conditioning of an ill-conditioned panel amplifies.
-template <int BN, bool BF16, bool SPLIT = false>
+template <int BN, bool BF16, bool SPLIT = false, bool TMA = false>
 struct Cfg {
-  static constexpr int BKE = BF16 ? 64 : 32;                 // K elements per 128-byte row
-  static constexpr int EPC = BF16 ? 8 : 4;                   // elements per 16-byte chunk
+  // BT: bf16 operands formed in shared memory from TMA-loaded fp32 tiles (K block of 32, as in
+  // the fp32 TMA variant).  A stage then holds the raw fp32 tiles of A, of its fp32 addend and
+  // of B, followed by the bf16 operand tiles of A and B (half the bytes each).
+  static constexpr bool BT = BF16 && TMA;
+  static constexpr int BKE = (BF16 && !TMA) ? 64 : 32;       // K elements per stage
+  static constexpr int EPC = (BF16 && !TMA) ? 8 : 4;         // elements per 16-byte chunk of the register path
   static constexpr int A_BYTES = BM * 128;
   static constexpr int B_BYTES = BN * 128;
-  static constexpr int STAGE_BYTES = (BF16 ? 1 : 2) * (A_BYTES + B_BYTES);
+  static constexpr int STAGE_BYTES = BT ? (2 * A_BYTES + B_BYTES + A_BYTES / 2 + B_BYTES / 2)
+                                        : (BF16 ? 1 : 2) * (A_BYTES + B_BYTES);
   static constexpr int STAGES = (192 * 1024) / STAGE_BYTES;
-  static constexpr int G16_BYTES = BF16 ? 0 : BM * 32 * 2;   // bf16 addend tile of the TMA variant (per stage)
+  static constexpr int G16_BYTES = (BF16 && !TMA) ? 0 : BM * 32 * 2;   // bf16 addend tile of the TMA variants (per stage)
   static constexpr int SMEM_BYTES = STAGES * (STAGE_BYTES + G16_BYTES) + 1024 + 512;
   static constexpr int A_CHUNKS = BM * 8 / NUM_PROD_THREADS;  // 16-byte chunks per producer thread
   static constexpr int B_CHUNKS = BN * 8 / NUM_PROD_THREADS;
   static constexpr int ACCS = SPLIT ? 2 : 1;                 // accumulators per tile
   static constexpr int NBUF = (512 / (ACCS * BN)) >= 2 ? 2 : 1;  // tiles in flight in TMEM
   static constexpr int TMEM_COLS = NBUF * ACCS * BN;
+  static constexpr int KSTEPS = BT ? 2 : 4;                  // UMMA K steps per stage
 };
 
-// TMA = true (fp32 mode): a dedicated warp loads the raw fp32 tiles of A, of its addend and
+// TMA = true: a dedicated warp loads the raw fp32 tiles of A, of its addend and
 // of B with TMA straight into the stage buffers (A and B into their "hi" halves, the
 // addend into A's "lo" half).  The 8 producer warps then only convert in place: the MMA
 // truncates an fp32 word to TF32 by itself, so the raw word serves as the "hi" operand
 // and only the truncation remainder is written to the "lo" half (after the M + G add
 // for a fused A).  Loads of one stage overlap conversion and MMAs of the other, and
 // out-of-range rows / k are zero filled by the TMA unit.
+// TMA with bf16 operands: the same loads; the producer warps add, round to bf16 and write
+// the operand tiles the MMA reads (k-contiguous: rows of 64 bytes, 64-byte swizzle;
+// row-contiguous: 128-byte rows of 64 row indices, 128-byte swizzle); one MMA per K step.
 template <int BN, bool A_MN, bool B_MN, bool BF16, bool SPLIT, bool TMA>
 __global__ void __launch_bounds__(TMA ? NUM_THREADS_TMA : NUM_THREADS, 1) k_gemm_umma(const __grid_constant__ Params p) {
   static_assert(!(BF16 && SPLIT), "split accumulators belong to the 3xTF32 mode");
-  static_assert(!(BF16 && TMA), "the TMA variant converts fp32 tiles in place");
-  using C = Cfg<BN, BF16, SPLIT>;
+  using C = Cfg<BN, BF16, SPLIT, TMA>;
   constexpr int NBUF = C::NBUF, ACCS = C::ACCS;
   constexpr int BKE = C::BKE, EPC = C::EPC, STAGES = C::STAGES;
   if (p.g.skip_flag != nullptr && *p.g.skip_flag != 0) return;
@@ -536,6 +563,24 @@ __global__ void __launch_bounds__(TMA ? NUM_THREADS_TMA : NUM_THREADS, 1) k_gemm
           g16off[l] = kk * 256u + (c * 32u + q * 4u) * 2u;
         }
       }
+      // bf16 operands: byte offset of each unit's four bf16 values in the operand tile
+      uint32_t aout[C::A_CHUNKS], bout[C::B_CHUNKS];
+      if (C::BT) {
+        auto out_off = [](uint32_t u, bool mn) -> uint32_t {
+          if (!mn) {   // unit u = (row, swizzled 16-byte chunk) of a 128-byte fp32 row
+            const uint32_t row = u >> 3, kc = (u & 7u) ^ (row & 7u);
+            return row * 64u + ((((kc >> 1) ^ ((row >> 1) & 3u))) << 4) + (kc & 1u) * 8u;
+          }
+          // unit u = (32-row column chunk c, k row kk, swizzled unit qs): rows c*32 + q*4 .. +3 at k = kk
+          const uint32_t c = u >> 8, kk = (u >> 3) & 31u, qs = u & 7u;
+          const uint32_t q = ((((qs >> 1) ^ (kk & 3u))) << 1) | (qs & 1u);
+          return (c >> 1) * (uint32_t)(BKE * 128) + kk * 128u + (((((c & 1u) << 2) | (q >> 1)) ^ (kk & 7u)) << 4) + (q & 1u) * 8u;
+        };
+#pragma unroll
+        for (int l = 0; l < C::A_CHUNKS; ++l) aout[l] = out_off((uint32_t)ptid + l * NUM_PROD_THREADS, A_MN);
+#pragma unroll
+        for (int l = 0; l < C::B_CHUNKS; ++l) bout[l] = out_off((uint32_t)ptid + l * NUM_PROD_THREADS, B_MN);
+      }
       int stage = 0;
       uint32_t phase = 0;
       bool alive = true;
@@ -563,6 +608,18 @@ __global__ void __launch_bounds__(TMA ? NUM_THREADS_TMA : NUM_THREADS, 1) k_gemm
           }
 #pragma unroll
           for (int l = 0; l < C::B_CHUNKS; ++l) xb[l] = lds128(sb + l * (NUM_PROD_THREADS * 16));
+          if (C::BT) {
+            const uint32_t a_out = smem_base + stage * C::STAGE_BYTES + 2 * C::A_BYTES + C::B_BYTES;
+            const uint32_t b_out = a_out + C::A_BYTES / 2;
+#pragma unroll
+            for (int l = 0; l < C::A_CHUNKS; ++l) {
+              float4 x = xa[l];
+              if (add || add16) { x.x += ga[l].x; x.y += ga[l].y; x.z += ga[l].z; x.w += ga[l].w; }
+              sts64_bf16x4(a_out + aout[l], x);
+            }
+#pragma unroll
+            for (int l = 0; l < C::B_CHUNKS; ++l) sts64_bf16x4(b_out + bout[l], xb[l]);
+          } else {
 #pragma unroll
           for (int l = 0; l < C::A_CHUNKS; ++l) {
             float4 x = xa[l];
@@ -576,6 +633,7 @@ __global__ void __launch_bounds__(TMA ? NUM_THREADS_TMA : NUM_THREADS, 1) k_gemm
           for (int l = 0; l < C::B_CHUNKS; ++l) {
             const float4 x = xb[l];
             sts128(sb_lo + l * (NUM_PROD_THREADS * 16), make_float4(trunc_rem(x.x), trunc_rem(x.y), trunc_rem(x.z), trunc_rem(x.w)));
+          }
           }
           fence_proxy_async();
           __syncwarp();
@@ -706,14 +764,16 @@ __global__ void __launch_bounds__(TMA ? NUM_THREADS_TMA : NUM_THREADS, 1) k_gemm
         for (int kb = kbc; kb < kbc1; ++kb) {
           if (!mbar_wait(full_bar(stage), phase, dead, p.status)) { alive = false; break; }
           tc_fence_after();
-          const uint32_t sa = smem_base + stage * C::STAGE_BYTES;
+          const uint32_t st0 = smem_base + stage * C::STAGE_BYTES;
+          // bf16 operands formed from TMA tiles sit behind the raw tiles of the stage
+          const uint32_t sa = C::BT ? st0 + 2 * C::A_BYTES + C::B_BYTES : st0;
           const uint32_t sa_lo = sa + C::A_BYTES;
-          const uint32_t sb = sa + (BF16 ? 1 : 2) * C::A_BYTES;
+          const uint32_t sb = C::BT ? sa + C::A_BYTES / 2 : sa + (BF16 ? 1 : 2) * C::A_BYTES;
           const uint32_t sb_lo = sb + C::B_BYTES;
 #pragma unroll
-          for (int ks = 0; ks < ((p.debug & 4) ? 0 : 4); ++ks) {
-            const uint64_t a_hi = make_desc<BF16>(sa + ks * A_KSTEP, A_MN, lbo);
-            const uint64_t b_hi = make_desc<BF16>(sb + ks * B_KSTEP, B_MN, lbo);
+          for (int ks = 0; ks < ((p.debug & 4) ? 0 : C::KSTEPS); ++ks) {
+            const uint64_t a_hi = (C::BT && !A_MN) ? make_desc_k64(sa + ks * A_KSTEP) : make_desc<BF16>(sa + ks * A_KSTEP, A_MN, lbo);
+            const uint64_t b_hi = (C::BT && !B_MN) ? make_desc_k64(sb + ks * B_KSTEP) : make_desc<BF16>(sb + ks * B_KSTEP, B_MN, lbo);
             if (BF16) {
               umma<true>(d_tmem, a_hi, b_hi, idesc, accumulate);
               accumulate = 1;
@@ -759,12 +819,12 @@ __global__ void __launch_bounds__(TMA ? NUM_THREADS_TMA : NUM_THREADS, 1) k_gemm
 template <int BN, bool A_MN, bool B_MN, bool BF16, bool SPLIT, bool TMA>
 inline cudaError_t set_smem_attr() {
   return cudaFuncSetAttribute(k_gemm_umma<BN, A_MN, B_MN, BF16, SPLIT, TMA>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              Cfg<BN, BF16, SPLIT>::SMEM_BYTES);
+                              Cfg<BN, BF16, SPLIT, TMA>::SMEM_BYTES);
 }
 
 template <int BN, bool BF16, bool SPLIT, bool TMA>
 inline void launch_variant(const Params& p, bool a_mn, bool b_mn, int grid, cudaStream_t st) {
-  constexpr int smem = Cfg<BN, BF16, SPLIT>::SMEM_BYTES;
+  constexpr int smem = Cfg<BN, BF16, SPLIT, TMA>::SMEM_BYTES;
   constexpr int threads = TMA ? NUM_THREADS_TMA : NUM_THREADS;
   if (!a_mn && !b_mn) k_gemm_umma<BN, false, false, BF16, SPLIT, TMA><<<grid, threads, smem, st>>>(p);
   else if (!a_mn && b_mn) k_gemm_umma<BN, false, true, BF16, SPLIT, TMA><<<grid, threads, smem, st>>>(p);
@@ -846,7 +906,8 @@ inline int umma_configure() {
   if (e == cudaSuccess) e = set_smem_attr<BN, A, B, F, false, false>();    \
   if (e == cudaSuccess && !F) e = set_smem_attr<BN, A, B, false, true, false>();  \
   if (e == cudaSuccess && !F) e = set_smem_attr<BN, A, B, false, false, true>();  \
-  if (e == cudaSuccess && !F) e = set_smem_attr<BN, A, B, false, true, true>();
+  if (e == cudaSuccess && !F) e = set_smem_attr<BN, A, B, false, true, true>();  \
+  if (e == cudaSuccess && F) e = set_smem_attr<BN, A, B, true, false, true>();
   DION_SET(128, false, false, false) DION_SET(128, false, true, false) DION_SET(128, true, true, false) DION_SET(128, true, false, false)
   DION_SET(256, false, false, false) DION_SET(256, false, true, false) DION_SET(256, true, true, false) DION_SET(256, true, false, false)
   DION_SET(128, false, false, true) DION_SET(128, false, true, true) DION_SET(128, true, true, true) DION_SET(128, true, false, true)
@@ -866,7 +927,6 @@ inline int umma_try_launch(const GemmArgs& g_in, int precision, int sm_count, fl
   GemmArgs g = g_in;
   const bool bf16 = (precision == DION_PREC_BF16_OPERANDS);
   const int epc = bf16 ? 8 : 4;
-  const int bke = bf16 ? 64 : 32;
   if (g.batch != 1 || g.alpha_dev != nullptr) return 0;
   if (g.M < 128 || g.N < 64 || g.K < 64) return 0;
   if ((g.M % epc) || (g.N % epc) || (g.K % epc)) return 0;
@@ -891,6 +951,20 @@ inline int umma_try_launch(const GemmArgs& g_in, int precision, int sm_count, fl
   const int BN = (g.tri == TRI_LOWER || g.N < 256) ? 128 : 256;
   Params p;
   p.g = g;
+  // TMA variant: fp32 operands in memory (both precision modes), dimensions the tensor maps can describe
+  bool tma = !(debug & 16) && g.M < (1ll << 31) && g.N < (1ll << 31) && g.K < (1ll << 31);
+  if (tma && g.a2_mode == ADD_BF16) {   // the bf16 addend needs 16-byte aligned rows for its tensor map
+    const i64 ld2 = a_mn ? g.a2_sk : g.a2_si;
+    tma = (ld2 % 8 == 0) && (((uintptr_t)g.A2 % 16) == 0) &&
+          make_addend16_map(&p.tmA2, g.A2, g.M, g.K, ld2, a_mn);
+  }
+  if (tma) {
+    const i64 lda = a_mn ? g.a_sk : g.a_si, ldb = b_mn ? g.b_sk : g.b_sn;
+    tma = make_operand_map(&p.tmA, g.A, g.M, g.K, lda, a_mn, BM) && make_operand_map(&p.tmB, g.B, g.N, g.K, ldb, b_mn, BN);
+    if (tma && g.a2_mode == ADD_F32)
+      tma = make_operand_map(&p.tmA2, g.A2, g.M, g.K, a_mn ? g.a2_sk : g.a2_si, a_mn, BM);
+  }
+  const int bke = (bf16 && !tma) ? 64 : 32;
   p.nM = (int)((g.M + BM - 1) / BM);
   p.nN = (int)((g.N + BN - 1) / BN);
   p.nkb = (int)((g.K + bke - 1) / bke);
@@ -912,24 +986,14 @@ inline int umma_try_launch(const GemmArgs& g_in, int precision, int sm_count, fl
   p.num_items = (int)(tiles * splits);
   p.status = status;
   p.debug = debug;
-  // 32 K blocks per accumulation chain: 1024 k in fp32 mode (8e-6 relative error, 1.4e-6 with
-  // split accumulators), 2048 k in bf16 mode
+  // 32 K blocks per accumulation chain: 1024 k (8e-6 relative error in fp32 mode, 1.4e-6 with
+  // split accumulators); 2048 k for bf16 operands loaded through registers
   p.kc = 32;
   const int grid = p.num_items < sm_count ? p.num_items : sm_count;
-  // TMA variant: fp32 mode, fp32 (or no) addend, dimensions the tensor maps can describe
-  bool tma = !bf16 && !(debug & 16) && g.M < (1ll << 31) && g.N < (1ll << 31) && g.K < (1ll << 31);
-  if (tma && g.a2_mode == ADD_BF16) {   // the bf16 addend needs 16-byte aligned rows for its tensor map
-    const i64 ld2 = a_mn ? g.a2_sk : g.a2_si;
-    tma = (ld2 % 8 == 0) && (((uintptr_t)g.A2 % 16) == 0) &&
-          make_addend16_map(&p.tmA2, g.A2, g.M, g.K, ld2, a_mn);
-  }
-  if (tma) {
-    const i64 lda = a_mn ? g.a_sk : g.a_si, ldb = b_mn ? g.b_sk : g.b_sn;
-    tma = make_operand_map(&p.tmA, g.A, g.M, g.K, lda, a_mn, BM) && make_operand_map(&p.tmB, g.B, g.N, g.K, ldb, b_mn, BN);
-    if (tma && g.a2_mode == ADD_F32)
-      tma = make_operand_map(&p.tmA2, g.A2, g.M, g.K, a_mn ? g.a2_sk : g.a2_si, a_mn, BM);
-  }
-  if (bf16) {
+  if (bf16 && tma) {
+    if (BN == 256) launch_variant<256, true, false, true>(p, a_mn, b_mn, grid, st);
+    else launch_variant<128, true, false, true>(p, a_mn, b_mn, grid, st);
+  } else if (bf16) {
     if (BN == 256) launch_variant<256, true, false, false>(p, a_mn, b_mn, grid, st);
     else launch_variant<128, true, false, false>(p, a_mn, b_mn, grid, st);
   } else if (tma) {

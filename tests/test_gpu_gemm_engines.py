@@ -145,12 +145,36 @@ def test_triangular_operand_k_limit(lib, engine):
     assert run(lib, engine, 0, 1024, 768, 768, False, False, klimit=1) < TOL[engine]
 
 
+@pytest.fixture(params=["tma", "registers"])
+def bf16_path(request, monkeypatch):
+    # bf16 operands are formed from TMA-loaded fp32 tiles by default; bit 16 of the hook's
+    # debug word selects the variant whose producer warps load through registers
+    if request.param == "registers":
+        monkeypatch.setenv("DION_DEBUG_GEMM", "16")
+    else:
+        monkeypatch.delenv("DION_DEBUG_GEMM", raising=False)
+    return request.param
+
+
 @pytest.mark.parametrize("a_mn,b_mn", LAYOUTS)
-def test_bf16_operand_mode(lib, a_mn, b_mn):
+def test_bf16_operand_mode(lib, bf16_path, a_mn, b_mn):
     err = run(lib, 2, 1, 512, 512, 1024, a_mn, b_mn)
     assert err < 6e-3, err
     err = run(lib, 2, 1, 648, 392, 328, a_mn, b_mn, seed=5)
     assert err < 6e-3, err
+    err = run(lib, 2, 1, 256, 1024, 2080, a_mn, b_mn, seed=6)      # two accumulation chunks on the TMA path
+    assert err < 6e-3, err
+
+
+@pytest.mark.parametrize("add", [torch.float32, torch.bfloat16])
+def test_bf16_operand_mode_fused_add_and_epilogues(lib, bf16_path, add):
+    assert run(lib, 2, 1, 1024, 256, 768, False, True, add=add) < 6e-3
+    assert run(lib, 2, 1, 768, 256, 1024, True, True, add=add) < 6e-3
+    # the rank-r updates: the product (entries ~16 here) is scaled by alpha before it meets C (entries ~1)
+    assert run(lib, 2, 1, 1024, 768, 256, False, False, add=add, epi=2, alpha=0.05) < 3e-3
+    assert run(lib, 2, 1, 1024, 768, 256, False, False, epi=1, alpha=0.01) < 1e-3
+    assert run(lib, 2, 1, 512, 512, 4096, True, True, tri=1) < 6e-3
+    assert run(lib, 2, 1, 1024, 768, 768, False, False, klimit=1) < 6e-3
 
 
 @pytest.mark.parametrize("a_mn,b_mn", LAYOUTS)
