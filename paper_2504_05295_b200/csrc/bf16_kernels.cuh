@@ -1,0 +1,82 @@
+// bf16-operand mode: the operands of the four large contractions as bf16 arrays in scratch.
+#pragma once
+
+#include "dion_common.cuh"
+
+namespace dion {
+
+__device__ __forceinline__ uint32_t pack_bf16x2(float a, float b) {
+  const __nv_bfloat162 v = __floats2bfloat162_rn(a, b);
+  return *reinterpret_cast<const uint32_t*>(&v);
+}
+
+// B16 = bf16(M + G), rows x cols, B16 dense with leading dimension cols (a multiple of 8).
+// One thread per 8 consecutive elements of a row.  VEC: M (and G) rows start 16-byte
+// aligned (pointer and leading dimension), so the loads are 128-bit.
+template <bool VEC>
+__global__ void __launch_bounds__(256) k_form_b16(const float* __restrict__ M, i64 ldm, const void* __restrict__ G,
+                                                  i64 ldg, int g_mode, i64 rows, i64 cols,
+                                                  __nv_bfloat16* __restrict__ out) {
+  const i64 per_row = cols / 8;
+  const i64 total = rows * per_row;
+  for (i64 e = (i64)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (i64)gridDim.x * blockDim.x) {
+    const i64 i = e / per_row, c = (e - i * per_row) * 8;
+    float v[8];
+    const float* mp = M + i * ldm + c;
+    if (VEC) {
+      const float4 a = __ldg(reinterpret_cast<const float4*>(mp)), b = __ldg(reinterpret_cast<const float4*>(mp) + 1);
+      v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w; v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
+    } else {
+#pragma unroll
+      for (int q = 0; q < 8; ++q) v[q] = mp[q];
+    }
+    if (g_mode == ADD_F32) {
+      const float* gp = reinterpret_cast<const float*>(G) + i * ldg + c;
+      if (VEC) {
+        const float4 a = __ldg(reinterpret_cast<const float4*>(gp)), b = __ldg(reinterpret_cast<const float4*>(gp) + 1);
+        v[0] += a.x; v[1] += a.y; v[2] += a.z; v[3] += a.w; v[4] += b.x; v[5] += b.y; v[6] += b.z; v[7] += b.w;
+      } else {
+#pragma unroll
+        for (int q = 0; q < 8; ++q) v[q] += gp[q];
+      }
+    } else if (g_mode == ADD_BF16) {
+      const __nv_bfloat16* gp = reinterpret_cast<const __nv_bfloat16*>(G) + i * ldg + c;
+      if (VEC) {
+        const uint4 w = __ldg(reinterpret_cast<const uint4*>(gp));
+        const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          const __nv_bfloat162 h = *reinterpret_cast<const __nv_bfloat162*>(&ww[q]);
+          v[2 * q] += __low2float(h); v[2 * q + 1] += __high2float(h);
+        }
+      } else {
+#pragma unroll
+        for (int q = 0; q < 8; ++q) v[q] += __bfloat162float(gp[q]);
+      }
+    }
+    uint4 o;
+    o.x = pack_bf16x2(v[0], v[1]); o.y = pack_bf16x2(v[2], v[3]);
+    o.z = pack_bf16x2(v[4], v[5]); o.w = pack_bf16x2(v[6], v[7]);
+    *reinterpret_cast<uint4*>(out + i * cols + c) = o;
+  }
+}
+
+// out = bf16(src), rows x cols (cols a multiple of 8, src rows 16-byte aligned), out dense.
+// skip_flag (optional): nothing is written when *skip_flag != 0.
+__global__ void __launch_bounds__(256) k_to_bf16(const float* __restrict__ src, i64 lds, i64 rows, i64 cols,
+                                                 __nv_bfloat16* __restrict__ out, const int* __restrict__ skip_flag) {
+  if (skip_flag != nullptr && *skip_flag != 0) return;
+  const i64 per_row = cols / 8;
+  const i64 total = rows * per_row;
+  for (i64 e = (i64)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (i64)gridDim.x * blockDim.x) {
+    const i64 i = e / per_row, c = (e - i * per_row) * 8;
+    const float4 a = *reinterpret_cast<const float4*>(src + i * lds + c);
+    const float4 b = *(reinterpret_cast<const float4*>(src + i * lds + c) + 1);
+    uint4 o;
+    o.x = pack_bf16x2(a.x, a.y); o.y = pack_bf16x2(a.z, a.w);
+    o.z = pack_bf16x2(b.x, b.y); o.w = pack_bf16x2(b.z, b.w);
+    *reinterpret_cast<uint4*>(out + i * cols + c) = o;
+  }
+}
+
+}  // namespace dion

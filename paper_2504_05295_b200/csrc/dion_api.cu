@@ -7,6 +7,7 @@
 #include <string.h>
 #include <vector>
 
+#include "bf16_kernels.cuh"
 #include "dion_common.cuh"
 #include "dion_internal.h"
 #include "orth_kernels.cuh"
@@ -30,6 +31,7 @@ inline i64 align64(i64 floats) { return (floats + 63) / 64 * 64; }  // 256-byte 
 
 struct Layout {
   i64 P0, P1, R, Gram, Linv, Tbuf, Dinv, DinvP, part, cn_part, d, gdiag, scal, total;
+  i64 B16, Q16, U16, R16;   // bf16-operand mode: bf16(M + G) and the bf16 copies of Q, U, R (offsets in floats)
   i64 part_floats;
   int cn_chunks;
   i64 cn_rows;
@@ -87,6 +89,13 @@ Layout make_layout(const dion_ctx* c, i64 m, i64 n, i64 r) {
   L.d = o; o += align64(r);
   L.gdiag = o; o += align64(r);
   L.scal = o; o += 64;
+  L.B16 = L.Q16 = L.U16 = L.R16 = 0;
+  if (c->cfg.precision == DION_PREC_BF16_OPERANDS) {
+    L.B16 = o; o += align64((m * n + 1) / 2);
+    L.Q16 = o; o += align64((big * r + 1) / 2);
+    L.U16 = o; o += align64((big * r + 1) / 2);
+    L.R16 = o; o += align64((big * r + 1) / 2);
+  }
   L.total = o;
   return L;
 }
@@ -221,6 +230,7 @@ int launch_gemm(StepCtx& s, const GemmArgs& g, int b = 0, bool force64 = false) 
     if (rc < 0) return rc;
     if (s.c->cfg.engine == DION_ENGINE_TENSOR) return DION_ERR_UNSUPPORTED;
   }
+  if (g.ab16) return DION_ERR_UNSUPPORTED;   // bf16 arrays are read by the tensor engine only
   return launch_gemm_simt(s.c, g, s.st, s.W(b, s.L.part), s.L.part_floats, force64);
 }
 
@@ -614,6 +624,19 @@ int step_batch(dion_ctx* c, const dion_matrix* const* list, int nb, float lr, cu
   const i64 qrow = tr ? m : n;     // rows of R and Q
   const auto g_mode = [](const dion_matrix* a) { return (a->g_dtype == DION_BF16) ? ADD_BF16 : ADD_F32; };
 
+  // bf16-operand mode on the tensor engine: bf16(M + G) is formed once per step and the four
+  // products read bf16 arrays (B16, and the bf16 copies of Q, U, R) straight through TMA.
+  bool d16 = s.tensor && c->cfg.precision == DION_PREC_BF16_OPERANDS && m % 8 == 0 && n % 8 == 0 && r % 8 == 0 &&
+             m >= 128 && n >= 128 && r >= 64;
+  for (int b = 0; b < nb && d16; ++b)
+    if (((uintptr_t)list[b]->Q & 15) || (list[b]->ldq % 4)) d16 = false;
+  auto bf = [&](int b, i64 off) { return reinterpret_cast<__nv_bfloat16*>(s.W(b, off)); };
+  auto to_bf16 = [&](const float* src, i64 lds, i64 rows, i64 cols, __nv_bfloat16* out) -> int {
+    k_to_bf16<<<grid_for(c, rows * cols / 8), 256, 0, st>>>(src, lds, rows, cols, out, nullptr);
+    DION_CHECK_LAUNCH(c);
+    return DION_OK;
+  };
+
   // P = (M + G) Q   (transposed form: (M + G)^T Q)
   {
   PhaseScope ps(c, st, DION_PHASE_P);
@@ -621,12 +644,26 @@ int step_batch(dion_ctx* c, const dion_matrix* const* list, int nb, float lr, cu
     const dion_matrix* a = list[b];
     GemmArgs p = gemm_args();
     p.M = prow; p.N = r; p.K = qrow;
-    p.A = (const float*)a->M; p.a_si = tr ? 1 : a->ldm; p.a_sk = tr ? a->ldm : 1;
-    p.A2 = a->G; p.a2_si = tr ? 1 : a->ldg; p.a2_sk = tr ? a->ldg : 1; p.a2_mode = g_mode(a);
-    p.B = (const float*)a->Q; p.b_sk = a->ldq; p.b_sn = 1;
+    if (d16) {
+      const bool vec = !((uintptr_t)a->M & 15) && a->ldm % 4 == 0 &&
+                       (a->g_dtype == DION_BF16 ? (!((uintptr_t)a->G & 15) && a->ldg % 8 == 0)
+                                                : (!((uintptr_t)a->G & 15) && a->ldg % 4 == 0));
+      const int grid = grid_for(c, m * n / 8);
+      if (vec) k_form_b16<true><<<grid, 256, 0, st>>>((const float*)a->M, a->ldm, a->G, a->ldg, g_mode(a), m, n, bf(b, s.L.B16));
+      else k_form_b16<false><<<grid, 256, 0, st>>>((const float*)a->M, a->ldm, a->G, a->ldg, g_mode(a), m, n, bf(b, s.L.B16));
+      DION_CHECK_LAUNCH(c);
+      DION_TRY(to_bf16((const float*)a->Q, a->ldq, qrow, r, bf(b, s.L.Q16)));
+      p.ab16 = 1;
+      p.A = (const float*)bf(b, s.L.B16); p.a_si = tr ? 1 : n; p.a_sk = tr ? n : 1;
+      p.B = (const float*)bf(b, s.L.Q16); p.b_sk = r; p.b_sn = 1;
+    } else {
+      p.A = (const float*)a->M; p.a_si = tr ? 1 : a->ldm; p.a_sk = tr ? a->ldm : 1;
+      p.A2 = a->G; p.a2_si = tr ? 1 : a->ldg; p.a2_sk = tr ? a->ldg : 1; p.a2_mode = g_mode(a);
+      p.B = (const float*)a->Q; p.b_sk = a->ldq; p.b_sn = 1;
+    }
     p.C = s.W(b, s.L.P0); p.ldc = r; p.epi = EPI_STORE;
     // an ill-conditioned panel amplifies the error of P: use the accurate product there
-    p.precise = (resolve_orth(c, r, (m < n) ? m : n) == DION_ORTH_SHIFTED3) ? 1 : 0;
+    p.precise = (!d16 && resolve_orth(c, r, (m < n) ? m : n) == DION_ORTH_SHIFTED3) ? 1 : 0;
     DION_TRY(launch_gemm(s, p, b));
   }
   }
@@ -648,9 +685,16 @@ int step_batch(dion_ctx* c, const dion_matrix* const* list, int nb, float lr, cu
     const dion_matrix* a = list[b];
     GemmArgs w = gemm_args();
     w.M = qrow; w.N = r; w.K = prow;
-    w.A = (const float*)a->M; w.a_si = tr ? a->ldm : 1; w.a_sk = tr ? 1 : a->ldm;
-    w.A2 = a->G; w.a2_si = tr ? a->ldg : 1; w.a2_sk = tr ? 1 : a->ldg; w.a2_mode = g_mode(a);
-    w.B = s.W(b, U_off); w.b_sk = r; w.b_sn = 1;
+    if (d16) {
+      DION_TRY(to_bf16(s.W(b, U_off), r, prow, r, bf(b, s.L.U16)));
+      w.ab16 = 1;
+      w.A = (const float*)bf(b, s.L.B16); w.a_si = tr ? n : 1; w.a_sk = tr ? 1 : n;
+      w.B = (const float*)bf(b, s.L.U16); w.b_sk = r; w.b_sn = 1;
+    } else {
+      w.A = (const float*)a->M; w.a_si = tr ? a->ldm : 1; w.a_sk = tr ? 1 : a->ldm;
+      w.A2 = a->G; w.a2_si = tr ? a->ldg : 1; w.a2_sk = tr ? 1 : a->ldg; w.a2_mode = g_mode(a);
+      w.B = s.W(b, U_off); w.b_sk = r; w.b_sn = 1;
+    }
     w.C = s.W(b, s.L.R); w.ldc = r; w.epi = EPI_STORE;
     DION_TRY(launch_gemm(s, w, b));
   }
@@ -663,8 +707,15 @@ int step_batch(dion_ctx* c, const dion_matrix* const* list, int nb, float lr, cu
     const dion_matrix* a = list[b];
     GemmArgs e = gemm_args();
     e.M = m; e.N = n; e.K = r;
-    e.A = s.W(b, tr ? s.L.R : U_off); e.a_si = r; e.a_sk = 1;
-    e.B = s.W(b, tr ? U_off : s.L.R); e.b_sk = 1; e.b_sn = r;
+    if (d16) {
+      DION_TRY(to_bf16(s.W(b, s.L.R), r, qrow, r, bf(b, s.L.R16)));
+      e.ab16 = 1;
+      e.A = (const float*)bf(b, tr ? s.L.R16 : s.L.U16); e.a_si = r; e.a_sk = 1;
+      e.B = (const float*)bf(b, tr ? s.L.U16 : s.L.R16); e.b_sk = 1; e.b_sn = r;
+    } else {
+      e.A = s.W(b, tr ? s.L.R : U_off); e.a_si = r; e.a_sk = 1;
+      e.B = s.W(b, tr ? U_off : s.L.R); e.b_sk = 1; e.b_sn = r;
+    }
     e.C = (float*)a->M; e.ldc = a->ldm; e.epi = EPI_ADD2_SUB;
     e.C2 = a->G; e.ldc2 = a->ldg; e.c2_mode = g_mode(a);
     e.alpha = 1.f - c->cfg.mu;
@@ -689,7 +740,12 @@ int step_batch(dion_ctx* c, const dion_matrix* const* list, int nb, float lr, cu
     const dion_matrix* a = list[b];
     GemmArgs x = gemm_args();
     x.M = m; x.N = n; x.K = r;
-    if (tr) {
+    if (d16) {
+      DION_TRY(to_bf16((const float*)a->Q, a->ldq, qrow, r, bf(b, s.L.Q16)));
+      x.ab16 = 1;
+      x.A = (const float*)bf(b, tr ? s.L.Q16 : s.L.U16); x.a_si = r; x.a_sk = 1;
+      x.B = (const float*)bf(b, tr ? s.L.U16 : s.L.Q16); x.b_sk = 1; x.b_sn = r;
+    } else if (tr) {
       x.A = (const float*)a->Q; x.a_si = a->ldq; x.a_sk = 1;
       x.B = s.W(b, U_off); x.b_sk = 1; x.b_sn = r;
     } else {
@@ -1085,7 +1141,7 @@ extern "C" int dion_debug_gemm(int engine, int precision, const dion_debug_gemm_
   g.B = a->B; g.b_sk = a->b_sk; g.b_sn = a->b_sn;
   g.C = a->C; g.ldc = a->ldc; g.epi = a->epi;
   g.C2 = a->C2; g.ldc2 = a->ldc2; g.c2_mode = a->c2_mode;
-  g.alpha = a->alpha; g.tri = a->tri; g.klimit = a->klimit; g.precise = a->precise;
+  g.alpha = a->alpha; g.tri = a->tri; g.klimit = a->klimit; g.precise = a->precise; g.ab16 = a->ab16;
   cudaStream_t st = (cudaStream_t)cuda_stream;
   if (engine == DION_ENGINE_TENSOR) {
     const char* dbg = getenv("DION_DEBUG_GEMM");   // timing experiments of this hook only

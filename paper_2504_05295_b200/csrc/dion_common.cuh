@@ -45,6 +45,7 @@ struct GemmArgs {
   int klimit;                    // 1: B(k,j) == 0 for k > j  (K loop ends at the tile's last column)
   const int* skip_flag;          // optional: if *skip_flag != 0 the kernel does nothing
   int precise;                   // tensor engine: keep the small split terms in their own accumulator
+  int ab16;                      // tensor engine only: A and B point to bf16 arrays (strides in elements), no addend
 };
 
 __device__ __forceinline__ float load_add(const void* p, i64 off, int mode) {

@@ -21,6 +21,7 @@ typedef struct {
   int tri;                                       /* 1: only tiles on or below the diagonal */
   int klimit;                                    /* 1: B(k,j) = 0 for k > j                */
   int precise;                                   /* 1: split accumulators (tensor engine)  */
+  int ab16;                                      /* 1: A and B are bf16 arrays (tensor engine) */
 } dion_debug_gemm_args;
 
 /* engine: 1 = fp32 FMA, 2 = tensor cores (returns DION_ERR_UNSUPPORTED if the

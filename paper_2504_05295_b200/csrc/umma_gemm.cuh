@@ -384,20 +384,22 @@ struct TileMap {
 // brings the product to the accuracy of an fp32 FMA loop (measured 3.3e-7 against
 // 9.1e-7 relative error on Gaussian data).  Used for the products whose error the
 // conditioning of an ill-conditioned panel amplifies.
-template <int BN, bool BF16, bool SPLIT = false, bool TMA = false>
+template <int BN, bool BF16, bool SPLIT = false, bool TMA = false, bool D16 = false>
 struct Cfg {
   // BT: bf16 operands formed in shared memory from TMA-loaded fp32 tiles (K block of 32, as in
   // the fp32 TMA variant).  A stage then holds the raw fp32 tiles of A, of its fp32 addend and
   // of B, followed by the bf16 operand tiles of A and B (half the bytes each).
-  static constexpr bool BT = BF16 && TMA;
-  static constexpr int BKE = (BF16 && !TMA) ? 64 : 32;       // K elements per stage
+  // D16: both operands are bf16 arrays in memory; TMA writes the operand tiles themselves
+  // (K block of 64, 128-byte swizzle) and the producer warps have nothing to do.
+  static constexpr bool BT = BF16 && TMA && !D16;
+  static constexpr int BKE = (BF16 && (!TMA || D16)) ? 64 : 32;   // K elements per stage
   static constexpr int EPC = (BF16 && !TMA) ? 8 : 4;         // elements per 16-byte chunk of the register path
   static constexpr int A_BYTES = BM * 128;
   static constexpr int B_BYTES = BN * 128;
   static constexpr int STAGE_BYTES = BT ? (2 * A_BYTES + B_BYTES + A_BYTES / 2 + B_BYTES / 2)
                                         : (BF16 ? 1 : 2) * (A_BYTES + B_BYTES);
   static constexpr int STAGES = (192 * 1024) / STAGE_BYTES;
-  static constexpr int G16_BYTES = (BF16 && !TMA) ? 0 : BM * 32 * 2;   // bf16 addend tile of the TMA variants (per stage)
+  static constexpr int G16_BYTES = ((BF16 && !TMA) || D16) ? 0 : BM * 32 * 2;   // bf16 addend tile of the TMA variants (per stage)
   static constexpr int SMEM_BYTES = STAGES * (STAGE_BYTES + G16_BYTES) + 1024 + 512;
   static constexpr int A_CHUNKS = BM * 8 / NUM_PROD_THREADS;  // 16-byte chunks per producer thread
   static constexpr int B_CHUNKS = BN * 8 / NUM_PROD_THREADS;
@@ -417,10 +419,11 @@ struct Cfg {
 // TMA with bf16 operands: the same loads; the producer warps add, round to bf16 and write
 // the operand tiles the MMA reads (k-contiguous: rows of 64 bytes, 64-byte swizzle;
 // row-contiguous: 128-byte rows of 64 row indices, 128-byte swizzle); one MMA per K step.
-template <int BN, bool A_MN, bool B_MN, bool BF16, bool SPLIT, bool TMA>
+template <int BN, bool A_MN, bool B_MN, bool BF16, bool SPLIT, bool TMA, bool D16 = false>
 __global__ void __launch_bounds__(TMA ? NUM_THREADS_TMA : NUM_THREADS, 1) k_gemm_umma(const __grid_constant__ Params p) {
   static_assert(!(BF16 && SPLIT), "split accumulators belong to the 3xTF32 mode");
-  using C = Cfg<BN, BF16, SPLIT, TMA>;
+  static_assert(!D16 || (BF16 && TMA), "bf16 operands in memory are loaded by TMA");
+  using C = Cfg<BN, BF16, SPLIT, TMA, D16>;
   constexpr int NBUF = C::NBUF, ACCS = C::ACCS;
   constexpr int BKE = C::BKE, EPC = C::EPC, STAGES = C::STAGES;
   if (p.g.skip_flag != nullptr && *p.g.skip_flag != 0) return;
@@ -543,7 +546,9 @@ __global__ void __launch_bounds__(TMA ? NUM_THREADS_TMA : NUM_THREADS, 1) k_gemm
   } else if (warp < NUM_EPI_WARPS + NUM_PROD_WARPS) {
     // ------------------------------------------------------------ producers
     const int ptid = threadIdx.x - NUM_EPI_WARPS * 32;
-    if (TMA) {
+    if (D16) {
+      // nothing to convert: the TMA warp fills the operand tiles
+    } else if (TMA) {
       // in-place conversion of the tiles the TMA warp loaded; the split is elementwise, so
       // each thread simply takes the 16-byte units ptid, ptid + 256, ... of the buffers
       const bool add = (g.a2_mode == ADD_F32);
@@ -711,8 +716,23 @@ __global__ void __launch_bounds__(TMA ? NUM_THREADS_TMA : NUM_THREADS, 1) k_gemm
           const int k0 = kb * BKE;
           const uint32_t sa = smem_base + stage * C::STAGE_BYTES;
           const uint32_t sa_lo = sa + C::A_BYTES;
-          const uint32_t sb = sa + 2 * C::A_BYTES;
+          const uint32_t sb = sa + (D16 ? 1 : 2) * C::A_BYTES;
           const uint32_t bar = raw_bar(stage);
+          if (D16) {   // bf16 tiles: [rows][64 k] boxes, or [64 k][64 rows] boxes per 64-row chunk
+            mbar_expect_tx(bar, (uint32_t)(C::A_BYTES + C::B_BYTES));
+            if (!A_MN) tma_load_2d(sa, &p.tmA, k0, row0a, bar);
+            else {
+#pragma unroll
+              for (int c = 0; c < BM / 64; ++c) tma_load_2d(sa + c * (BKE * 128), &p.tmA, row0a + 64 * c, k0, bar);
+            }
+            if (!B_MN) tma_load_2d(sb, &p.tmB, k0, row0b, bar);
+            else {
+#pragma unroll
+              for (int c = 0; c < BN / 64; ++c) tma_load_2d(sb + c * (BKE * 128), &p.tmB, row0b + 64 * c, k0, bar);
+            }
+            if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+            continue;
+          }
           mbar_expect_tx(bar, bytes);
           if (add16) {   // bf16 addend tile, unswizzled: [row][32 k] or [k][128 rows]
             if (!A_MN) tma_load_2d(g16_base + stage * C::G16_BYTES, &p.tmA2, k0, row0a, bar);
@@ -762,7 +782,7 @@ __global__ void __launch_bounds__(TMA ? NUM_THREADS_TMA : NUM_THREADS, 1) k_gemm
         const uint32_t d_small = d_tmem + (SPLIT ? BN : 0);
         uint32_t accumulate = 0;
         for (int kb = kbc; kb < kbc1; ++kb) {
-          if (!mbar_wait(full_bar(stage), phase, dead, p.status)) { alive = false; break; }
+          if (!mbar_wait(D16 ? raw_bar(stage) : full_bar(stage), phase, dead, p.status)) { alive = false; break; }
           tc_fence_after();
           const uint32_t st0 = smem_base + stage * C::STAGE_BYTES;
           // bf16 operands formed from TMA tiles sit behind the raw tiles of the stage
@@ -816,20 +836,20 @@ __global__ void __launch_bounds__(TMA ? NUM_THREADS_TMA : NUM_THREADS, 1) k_gemm
   }
 }
 
-template <int BN, bool A_MN, bool B_MN, bool BF16, bool SPLIT, bool TMA>
+template <int BN, bool A_MN, bool B_MN, bool BF16, bool SPLIT, bool TMA, bool D16 = false>
 inline cudaError_t set_smem_attr() {
-  return cudaFuncSetAttribute(k_gemm_umma<BN, A_MN, B_MN, BF16, SPLIT, TMA>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              Cfg<BN, BF16, SPLIT, TMA>::SMEM_BYTES);
+  return cudaFuncSetAttribute(k_gemm_umma<BN, A_MN, B_MN, BF16, SPLIT, TMA, D16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              Cfg<BN, BF16, SPLIT, TMA, D16>::SMEM_BYTES);
 }
 
-template <int BN, bool BF16, bool SPLIT, bool TMA>
+template <int BN, bool BF16, bool SPLIT, bool TMA, bool D16 = false>
 inline void launch_variant(const Params& p, bool a_mn, bool b_mn, int grid, cudaStream_t st) {
-  constexpr int smem = Cfg<BN, BF16, SPLIT, TMA>::SMEM_BYTES;
+  constexpr int smem = Cfg<BN, BF16, SPLIT, TMA, D16>::SMEM_BYTES;
   constexpr int threads = TMA ? NUM_THREADS_TMA : NUM_THREADS;
-  if (!a_mn && !b_mn) k_gemm_umma<BN, false, false, BF16, SPLIT, TMA><<<grid, threads, smem, st>>>(p);
-  else if (!a_mn && b_mn) k_gemm_umma<BN, false, true, BF16, SPLIT, TMA><<<grid, threads, smem, st>>>(p);
-  else if (a_mn && b_mn) k_gemm_umma<BN, true, true, BF16, SPLIT, TMA><<<grid, threads, smem, st>>>(p);
-  else k_gemm_umma<BN, true, false, BF16, SPLIT, TMA><<<grid, threads, smem, st>>>(p);
+  if (!a_mn && !b_mn) k_gemm_umma<BN, false, false, BF16, SPLIT, TMA, D16><<<grid, threads, smem, st>>>(p);
+  else if (!a_mn && b_mn) k_gemm_umma<BN, false, true, BF16, SPLIT, TMA, D16><<<grid, threads, smem, st>>>(p);
+  else if (a_mn && b_mn) k_gemm_umma<BN, true, true, BF16, SPLIT, TMA, D16><<<grid, threads, smem, st>>>(p);
+  else k_gemm_umma<BN, true, false, BF16, SPLIT, TMA, D16><<<grid, threads, smem, st>>>(p);
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
@@ -874,6 +894,22 @@ inline bool make_addend16_map(CUtensorMap* map, const void* ptr, i64 rows, i64 K
   return r == CUDA_SUCCESS;
 }
 
+// Tensor map of a bf16 operand: box = 64 k x box_rows rows (k contiguous) or 64 rows x 64 k
+// (row index contiguous), 128-byte swizzle: exactly the tile the bf16 MMA reads.
+inline bool make_operand16_map(CUtensorMap* map, const void* ptr, i64 rows, i64 K, i64 ld, bool mn_major, int box_rows) {
+  EncodeTiledFn fn = encode_tiled_fn();
+  if (fn == nullptr) return false;
+  cuuint64_t gdim[2], gstride[1];
+  cuuint32_t box[2], estr[2] = {1, 1};
+  if (!mn_major) { gdim[0] = (cuuint64_t)K; gdim[1] = (cuuint64_t)rows; box[0] = 64; box[1] = (cuuint32_t)box_rows; }
+  else { gdim[0] = (cuuint64_t)rows; gdim[1] = (cuuint64_t)K; box[0] = 64; box[1] = 64; }
+  gstride[0] = (cuuint64_t)ld * 2;
+  const CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), gdim, gstride, box, estr,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
 inline bool make_operand_map(CUtensorMap* map, const void* ptr, i64 rows, i64 K, i64 ld, bool mn_major, int box_rows) {
   EncodeTiledFn fn = encode_tiled_fn();
   if (fn == nullptr) return false;
@@ -907,7 +943,8 @@ inline int umma_configure() {
   if (e == cudaSuccess && !F) e = set_smem_attr<BN, A, B, false, true, false>();  \
   if (e == cudaSuccess && !F) e = set_smem_attr<BN, A, B, false, false, true>();  \
   if (e == cudaSuccess && !F) e = set_smem_attr<BN, A, B, false, true, true>();  \
-  if (e == cudaSuccess && F) e = set_smem_attr<BN, A, B, true, false, true>();
+  if (e == cudaSuccess && F) e = set_smem_attr<BN, A, B, true, false, true>();    \
+  if (e == cudaSuccess && F) e = set_smem_attr<BN, A, B, true, false, true, true>();
   DION_SET(128, false, false, false) DION_SET(128, false, true, false) DION_SET(128, true, true, false) DION_SET(128, true, false, false)
   DION_SET(256, false, false, false) DION_SET(256, false, true, false) DION_SET(256, true, true, false) DION_SET(256, true, false, false)
   DION_SET(128, false, false, true) DION_SET(128, false, true, true) DION_SET(128, true, true, true) DION_SET(128, true, false, true)
@@ -925,18 +962,21 @@ inline int umma_try_launch(const GemmArgs& g_in, int precision, int sm_count, fl
                            int* status, cudaStream_t st, int debug = 0) {
   using namespace umma;
   GemmArgs g = g_in;
-  const bool bf16 = (precision == DION_PREC_BF16_OPERANDS);
+  const bool d16 = g.ab16 != 0;      // bf16 operands in memory
+  const bool bf16 = d16 || (precision == DION_PREC_BF16_OPERANDS);
   const int epc = bf16 ? 8 : 4;
+  const int sm = d16 ? 8 : 4;        // stride granularity: 16 bytes
   if (g.batch != 1 || g.alpha_dev != nullptr) return 0;
   if (g.M < 128 || g.N < 64 || g.K < 64) return 0;
   if ((g.M % epc) || (g.N % epc) || (g.K % epc)) return 0;
+  if (d16 && g.a2_mode != ADD_NONE) return 0;
   auto aligned = [](const void* p, size_t a) { return ((uintptr_t)p % a) == 0; };
   bool a_mn, b_mn;
-  if (g.a_sk == 1 && g.a_si % 4 == 0) a_mn = false;
-  else if (g.a_si == 1 && g.a_sk % 4 == 0) a_mn = true;
+  if (g.a_sk == 1 && g.a_si % sm == 0) a_mn = false;
+  else if (g.a_si == 1 && g.a_sk % sm == 0) a_mn = true;
   else return 0;
-  if (g.b_sk == 1 && g.b_sn % 4 == 0) b_mn = false;
-  else if (g.b_sn == 1 && g.b_sk % 4 == 0) b_mn = true;
+  if (g.b_sk == 1 && g.b_sn % sm == 0) b_mn = false;
+  else if (g.b_sn == 1 && g.b_sk % sm == 0) b_mn = true;
   else return 0;
   if (!aligned(g.A, 16) || !aligned(g.B, 16) || !aligned(g.C, 16) || (g.ldc % 4)) return 0;
   if (g.a2_mode != ADD_NONE) {
@@ -952,19 +992,25 @@ inline int umma_try_launch(const GemmArgs& g_in, int precision, int sm_count, fl
   Params p;
   p.g = g;
   // TMA variant: fp32 operands in memory (both precision modes), dimensions the tensor maps can describe
-  bool tma = !(debug & 16) && g.M < (1ll << 31) && g.N < (1ll << 31) && g.K < (1ll << 31);
+  bool tma = (d16 || !(debug & 16)) && g.M < (1ll << 31) && g.N < (1ll << 31) && g.K < (1ll << 31);
+  if (d16) {
+    const i64 lda = a_mn ? g.a_sk : g.a_si, ldb = b_mn ? g.b_sk : g.b_sn;
+    if (!tma || !make_operand16_map(&p.tmA, g.A, g.M, g.K, lda, a_mn, BM) ||
+        !make_operand16_map(&p.tmB, g.B, g.N, g.K, ldb, b_mn, BN))
+      return 0;
+  } else
   if (tma && g.a2_mode == ADD_BF16) {   // the bf16 addend needs 16-byte aligned rows for its tensor map
     const i64 ld2 = a_mn ? g.a2_sk : g.a2_si;
     tma = (ld2 % 8 == 0) && (((uintptr_t)g.A2 % 16) == 0) &&
           make_addend16_map(&p.tmA2, g.A2, g.M, g.K, ld2, a_mn);
   }
-  if (tma) {
+  if (tma && !d16) {
     const i64 lda = a_mn ? g.a_sk : g.a_si, ldb = b_mn ? g.b_sk : g.b_sn;
     tma = make_operand_map(&p.tmA, g.A, g.M, g.K, lda, a_mn, BM) && make_operand_map(&p.tmB, g.B, g.N, g.K, ldb, b_mn, BN);
     if (tma && g.a2_mode == ADD_F32)
       tma = make_operand_map(&p.tmA2, g.A2, g.M, g.K, a_mn ? g.a2_sk : g.a2_si, a_mn, BM);
   }
-  const int bke = (bf16 && !tma) ? 64 : 32;
+  const int bke = (bf16 && (!tma || d16)) ? 64 : 32;
   p.nM = (int)((g.M + BM - 1) / BM);
   p.nN = (int)((g.N + BN - 1) / BN);
   p.nkb = (int)((g.K + bke - 1) / bke);
@@ -990,7 +1036,10 @@ inline int umma_try_launch(const GemmArgs& g_in, int precision, int sm_count, fl
   // split accumulators); 2048 k for bf16 operands loaded through registers
   p.kc = 32;
   const int grid = p.num_items < sm_count ? p.num_items : sm_count;
-  if (bf16 && tma) {
+  if (d16) {
+    if (BN == 256) launch_variant<256, true, false, true, true>(p, a_mn, b_mn, grid, st);
+    else launch_variant<128, true, false, true, true>(p, a_mn, b_mn, grid, st);
+  } else if (bf16 && tma) {
     if (BN == 256) launch_variant<256, true, false, true>(p, a_mn, b_mn, grid, st);
     else launch_variant<128, true, false, true>(p, a_mn, b_mn, grid, st);
   } else if (bf16) {

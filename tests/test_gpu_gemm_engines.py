@@ -24,7 +24,8 @@ class GemmArgs(ctypes.Structure):
                 ("B", ctypes.c_void_p), ("b_sk", ctypes.c_int64), ("b_sn", ctypes.c_int64),
                 ("C", ctypes.c_void_p), ("ldc", ctypes.c_int64), ("epi", ctypes.c_int),
                 ("C2", ctypes.c_void_p), ("ldc2", ctypes.c_int64), ("c2_mode", ctypes.c_int),
-                ("alpha", ctypes.c_float), ("tri", ctypes.c_int), ("klimit", ctypes.c_int), ("precise", ctypes.c_int)]
+                ("alpha", ctypes.c_float), ("tri", ctypes.c_int), ("klimit", ctypes.c_int), ("precise", ctypes.c_int),
+                ("ab16", ctypes.c_int)]
 
 
 @pytest.fixture(scope="module")
@@ -39,11 +40,13 @@ def lib():
 
 
 def run(lib, engine, precision, M, N, K, a_mn, b_mn, add=None, epi=0, tri=0, klimit=0, alpha=1.0, seed=0,
-        precise=0):
+        precise=0, ab16=False):
     g = torch.Generator(device="cuda"); g.manual_seed(seed)
     rn = lambda *s: torch.randn(*s, generator=g, device="cuda")
     # A(i,k): stored M x K (k contiguous) or K x M (row index contiguous)
     A_store = rn(K, M) if a_mn else rn(M, K)
+    if ab16:                             # operands stored as bf16: the reference sees the rounded values
+        A_store = A_store.to(torch.bfloat16)
     A_log = A_store.t() if a_mn else A_store
     A2_store = None
     if add is not None:
@@ -53,6 +56,8 @@ def run(lib, engine, precision, M, N, K, a_mn, b_mn, add=None, epi=0, tri=0, kli
         A_eff = A_log.double()
     # B(k,j): stored K x N (n contiguous) or N x K (k contiguous)
     B_store = rn(K, N) if b_mn else rn(N, K)
+    if ab16:
+        B_store = B_store.to(torch.bfloat16)
     B_log = B_store if b_mn else B_store.t()
     if klimit:
         B_log = torch.triu(B_log)       # B(k,j) = 0 for k > j
@@ -79,7 +84,7 @@ def run(lib, engine, precision, M, N, K, a_mn, b_mn, add=None, epi=0, tri=0, kli
     a.B = B_store.data_ptr(); a.b_sk, a.b_sn = (N, 1) if b_mn else (1, K)
     a.C = C.data_ptr(); a.ldc = N; a.epi = epi
     a.C2 = C2.data_ptr(); a.ldc2 = N; a.c2_mode = 1 if C2.dtype == torch.float32 else 2
-    a.alpha = alpha; a.tri = tri; a.klimit = klimit; a.precise = precise
+    a.alpha = alpha; a.tri = tri; a.klimit = klimit; a.precise = precise; a.ab16 = int(ab16)
     part = torch.empty(8 << 20, device="cuda")
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
     rc = lib.dion_debug_gemm(engine, precision, ctypes.byref(a), part.data_ptr(), part.numel(), status.data_ptr(),
@@ -175,6 +180,21 @@ def test_bf16_operand_mode_fused_add_and_epilogues(lib, bf16_path, add):
     assert run(lib, 2, 1, 1024, 768, 256, False, False, epi=1, alpha=0.01) < 1e-3
     assert run(lib, 2, 1, 512, 512, 4096, True, True, tri=1) < 6e-3
     assert run(lib, 2, 1, 1024, 768, 768, False, False, klimit=1) < 6e-3
+
+
+@pytest.mark.parametrize("a_mn,b_mn", LAYOUTS)
+def test_bf16_arrays_as_operands(lib, a_mn, b_mn):
+    # the operands are exact in bf16, so only the (truncating) fp32 accumulation separates the result from float64
+    for (M, N, K) in [(512, 512, 1024), (648, 392, 328), (256, 1024, 4160), (128, 64, 64)]:
+        err = run(lib, 2, 1, M, N, K, a_mn, b_mn, ab16=True, seed=M + K)
+        assert err < 1e-5, (M, N, K, err)
+
+
+def test_bf16_arrays_epilogues_and_lower_triangle(lib):
+    assert run(lib, 2, 1, 1024, 768, 256, False, False, ab16=True, epi=2, alpha=0.05) < 1e-5
+    assert run(lib, 2, 1, 1024, 768, 256, False, False, ab16=True, epi=1, alpha=0.01) < 1e-5
+    assert run(lib, 2, 1, 512, 512, 4096, True, True, ab16=True, tri=1) < 1e-5
+    assert run(lib, 2, 1, 2048, 128, 2048, False, True, ab16=True) < 1e-5      # split-K
 
 
 @pytest.mark.parametrize("a_mn,b_mn", LAYOUTS)
