@@ -51,53 +51,85 @@ __global__ void k_round_begin(const float* __restrict__ G, i64 ld, i64 r, float 
 typedef float (*blk_t)[NB + 1];
 typedef float (*half_blk_t)[NB / 2 + 1];
 
+// One doubling level of the triangular inverse inside a 64 x 64 block: for every pair of
+// adjacent B x B diagonal blocks, X21 = -X22 (L21 X11).  256 threads, two block-wide barriers.
+template <int B>
+__device__ __forceinline__ void trtri_level(blk_t L, blk_t X, half_blk_t T, int tid) {
+  constexpr int NPAIRS = NB / (2 * B);
+  for (int e = tid; e < NPAIRS * B * B; e += 256) {
+    const int pr = e / (B * B), rr = (e / B) % B, cc = e % B, base = pr * 2 * B;
+    float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;   // X11 is lower triangular: k >= cc; zeros above are stored
+    for (int k = cc & ~3; k < B; k += 4) {
+      s0 = fmaf(L[base + B + rr][base + k], X[base + k][base + cc], s0);
+      s1 = fmaf(L[base + B + rr][base + k + 1], X[base + k + 1][base + cc], s1);
+      s2 = fmaf(L[base + B + rr][base + k + 2], X[base + k + 2][base + cc], s2);
+      s3 = fmaf(L[base + B + rr][base + k + 3], X[base + k + 3][base + cc], s3);
+    }
+    T[pr * B + rr][cc] = (s0 + s1) + (s2 + s3);
+  }
+  __syncthreads();
+  for (int e = tid; e < NPAIRS * B * B; e += 256) {
+    const int pr = e / (B * B), rr = (e / B) % B, cc = e % B, base = pr * 2 * B;
+    float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;   // X22 is lower triangular: k <= rr; zeros above are stored
+    for (int k = 0; k <= rr; k += 4) {
+      s0 = fmaf(X[base + B + rr][base + B + k], T[pr * B + k][cc], s0);
+      s1 = fmaf(X[base + B + rr][base + B + k + 1], T[pr * B + k + 1][cc], s1);
+      s2 = fmaf(X[base + B + rr][base + B + k + 2], T[pr * B + k + 2][cc], s2);
+      s3 = fmaf(X[base + B + rr][base + B + k + 3], T[pr * B + k + 3][cc], s3);
+    }
+    X[base + B + rr][base + cc] = -((s0 + s1) + (s2 + s3));
+  }
+  __syncthreads();
+}
+
 // Cholesky factor and its inverse of the 64 x 64 block held in L (shared memory; lower
 // triangle, identity padding beyond a ragged block of jb columns), by the 256 threads of
 // a CTA.  On return L holds the factor, X its inverse, deflated[] the deflated columns.
 // X must be zero on entry, gd[] hold the floors' reference values, deflated[] zeros,
 // and a block-wide barrier must separate those writes from the call.
 // The block is factored in four 16-column sub-panels: the 16 x 16 diagonal piece by
-// one warp (one warp barrier per column), the rows below it by one thread per row,
-// the trailing update by all threads -- three block-wide barriers per sub-panel
+// one warp (rows in registers, shuffles, no barrier), the rows below it by one thread per
+// row, the trailing update by all threads -- three block-wide barriers per sub-panel
 // instead of three per column.  The inverse is built from 16 x 16 inverses by doubling.
 __device__ __forceinline__ void potrf_block(blk_t L, blk_t X, half_blk_t T, const float* gd, float* rdiag,
                                             int* deflated, int jb, float floor_rel, int* __restrict__ os,
                                             int* __restrict__ status) {
-  constexpr int W = 16;
+  constexpr int W = 16;    // base blocks of the inverse
+  constexpr int WF = 8;    // sub-panel width of the factorization
   const int tid = threadIdx.x;
   int floored = 0, failed = 0;
   float minrel = __int_as_float(0x7f800000);
+  const float inf = __int_as_float(0x7f800000);
 #pragma unroll 1
-  for (int c0 = 0; c0 < NB; c0 += W) {
+  for (int c0 = 0; c0 < NB; c0 += WF) {
     if (tid == 0) {
-      // 16 x 16 diagonal piece: one thread, the whole lower triangle in registers.  The chain
-      // pivot -> rsqrt -> scale -> update of the next pivot is serial whatever the thread count;
-      // one thread runs it without any barrier or shuffle and fills the gaps with the rest of
-      // the rank-1 update.
-      float a[W][W];
+      // WF x WF diagonal piece: one thread, the lower triangle in registers.  The chain
+      // pivot -> rsqrt -> scale -> update of the next pivot is serial whatever the thread
+      // count; one thread runs it without any barrier or shuffle.  Padding columns of a
+      // ragged block (unit diagonal, gd = 0) pass every test.
+      float a[WF][WF], g[WF];
 #pragma unroll
-      for (int i = 0; i < W; ++i)
+      for (int i = 0; i < WF; ++i) {
+        g[i] = gd[c0 + i];
 #pragma unroll
         for (int c = 0; c <= i; ++c) a[i][c] = L[c0 + i][c0 + c];
+      }
 #pragma unroll
-      for (int j = 0; j < W; ++j) {
+      for (int j = 0; j < WF; ++j) {
         float p = a[j][j];
+        const float fl = floor_rel * g[j];           // 0 in the plain mode
         bool defl = false;
-        if (c0 + j < jb) {
+        if (!(p > fl) || !(p < inf)) {
           if (floor_rel > 0.f) {
-            const float g = gd[c0 + j];
-            const float fl = floor_rel * g;
-            if (!(p > fl) || !isfinite(p)) {
-              p = (fl > 0.f && isfinite(fl)) ? fl : 1.f;   // zero or non-finite column: unit pivot
-              defl = true;
-              ++floored;
-            } else {
-              minrel = fminf(minrel, __fdividef(p, g));
-            }
-          } else if (!(p > 0.f) || !isfinite(p)) {
+            p = (fl > 0.f && fl < inf) ? fl : 1.f;   // zero or non-finite column: unit pivot
+            defl = true;
+            ++floored;
+          } else {
             failed = 1;
             p = 1.f;
           }
+        } else {
+          minrel = fminf(minrel, __fdividef(p, g[j]));
         }
         const float inv = rsqrtf(p);
         const float sc = defl ? 0.f : inv;
@@ -105,43 +137,41 @@ __device__ __forceinline__ void potrf_block(blk_t L, blk_t X, half_blk_t T, cons
         rdiag[c0 + j] = inv;
         if (defl) deflated[c0 + j] = 1;
 #pragma unroll
-        for (int i = j + 1; i < W; ++i) a[i][j] *= sc;
+        for (int i = j + 1; i < WF; ++i) a[i][j] *= sc;
 #pragma unroll
-        for (int c = j + 1; c < W; ++c)
+        for (int c = j + 1; c < WF; ++c)
 #pragma unroll
-          for (int i = c; i < W; ++i) a[i][c] = fmaf(-a[i][j], a[c][j], a[i][c]);
+          for (int i = c; i < WF; ++i) a[i][c] = fmaf(-a[i][j], a[c][j], a[i][c]);
       }
 #pragma unroll
-      for (int i = 0; i < W; ++i)
+      for (int i = 0; i < WF; ++i)
 #pragma unroll
         for (int c = 0; c <= i; ++c) L[c0 + i][c0 + c] = a[i][c];
     }
     __syncthreads();
-    const int below = NB - c0 - W;   // rows under the diagonal piece
+    const int below = NB - c0 - WF;   // rows under the diagonal piece
     if (tid < below) {
-      const int i = c0 + W + tid;
-      float x[W];
+      const int i = c0 + WF + tid;
+      float x[WF];
 #pragma unroll
-      for (int j = 0; j < W; ++j) {
+      for (int j = 0; j < WF; ++j) {
         float sacc = L[i][c0 + j];
 #pragma unroll
         for (int k = 0; k < j; ++k) sacc = fmaf(-x[k], L[c0 + j][c0 + k], sacc);
         x[j] = deflated[c0 + j] ? 0.f : sacc * rdiag[c0 + j];
       }
 #pragma unroll
-      for (int j = 0; j < W; ++j) L[i][c0 + j] = x[j];
+      for (int j = 0; j < WF; ++j) L[i][c0 + j] = x[j];
     }
     __syncthreads();
-    for (int e = tid; e < below * below; e += 256) {
-      const int ii = e / below, cc = e % below;
-      if (cc <= ii) {
-        const int i = c0 + W + ii, c = c0 + W + cc;
+    for (int ii = tid >> 4; ii < below; ii += 16)
+      for (int cc = tid & 15; cc <= ii; cc += 16) {
+        const int i = c0 + WF + ii, c = c0 + WF + cc;
         float sacc = 0.f;
 #pragma unroll
-        for (int k = 0; k < W; ++k) sacc = fmaf(L[i][c0 + k], L[c][c0 + k], sacc);
+        for (int k = 0; k < WF; ++k) sacc = fmaf(L[i][c0 + k], L[c][c0 + k], sacc);
         L[i][c] -= sacc;
       }
-    }
     __syncthreads();
   }
   if (tid == 0) {
@@ -171,34 +201,8 @@ __device__ __forceinline__ void potrf_block(blk_t L, blk_t X, half_blk_t T, cons
   }
   __syncthreads();
   // ... then [[X11, 0], [-X22 L21 X11, X22]] for block sizes 16 and 32
-#pragma unroll 1
-  for (int b = W; b < NB; b *= 2) {
-    const int npairs = NB / (2 * b);
-    for (int e = tid; e < npairs * b * b; e += 256) {
-      const int pr = e / (b * b), rr = (e / b) % b, cc = e % b, base = pr * 2 * b;
-      float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;   // X11 is lower triangular: k >= cc; zeros above are stored
-      for (int k = cc & ~3; k < b; k += 4) {
-        s0 = fmaf(L[base + b + rr][base + k], X[base + k][base + cc], s0);
-        s1 = fmaf(L[base + b + rr][base + k + 1], X[base + k + 1][base + cc], s1);
-        s2 = fmaf(L[base + b + rr][base + k + 2], X[base + k + 2][base + cc], s2);
-        s3 = fmaf(L[base + b + rr][base + k + 3], X[base + k + 3][base + cc], s3);
-      }
-      T[pr * b + rr][cc] = (s0 + s1) + (s2 + s3);
-    }
-    __syncthreads();
-    for (int e = tid; e < npairs * b * b; e += 256) {
-      const int pr = e / (b * b), rr = (e / b) % b, cc = e % b, base = pr * 2 * b;
-      float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;   // X22 is lower triangular: k <= rr; zeros above are stored
-      for (int k = 0; k <= rr; k += 4) {
-        s0 = fmaf(X[base + b + rr][base + b + k], T[pr * b + k][cc], s0);
-        s1 = fmaf(X[base + b + rr][base + b + k + 1], T[pr * b + k + 1][cc], s1);
-        s2 = fmaf(X[base + b + rr][base + b + k + 2], T[pr * b + k + 2][cc], s2);
-        s3 = fmaf(X[base + b + rr][base + b + k + 3], T[pr * b + k + 3][cc], s3);
-      }
-      X[base + b + rr][base + cc] = -((s0 + s1) + (s2 + s3));
-    }
-    __syncthreads();
-  }
+  trtri_level<16>(L, X, T, tid);
+  trtri_level<32>(L, X, T, tid);
 }
 
 // Cholesky of one jb x jb (jb <= 64) diagonal block, in place (lower factor, the
@@ -264,23 +268,35 @@ __global__ void __launch_bounds__(256) k_potrf_diag(float* __restrict__ A, i64 l
   }
 }
 
+// Operand tiles of the 64 x 64 x 64 products: rows of 68 floats (16-byte aligned rows for
+// 128-bit loads along k; the row patterns below stay free of bank conflicts).
+constexpr int MMS = NB + 4;
+typedef float (*mm_t)[MMS];
+
 // acc[a][b] += sum_k A[4 ty + a][k] * B[tx + 16 b][k]  (64 x 64 x 64, operands in shared memory)
-__device__ __forceinline__ void mm_nt_64(blk_t A, blk_t B, int ty, int tx, float (&acc)[4][4]) {
-#pragma unroll 8
-  for (int k = 0; k < NB; ++k) {
-    float av[4], bv[4];
+__device__ __forceinline__ void mm_nt_64(mm_t A, mm_t B, int ty, int tx, float (&acc)[4][4]) {
+#pragma unroll 4
+  for (int k = 0; k < NB; k += 4) {
+    float4 av[4], bv[4];
 #pragma unroll
-    for (int a = 0; a < 4; ++a) av[a] = A[ty * 4 + a][k];
+    for (int a = 0; a < 4; ++a) av[a] = *reinterpret_cast<const float4*>(&A[ty * 4 + a][k]);
 #pragma unroll
-    for (int b = 0; b < 4; ++b) bv[b] = B[tx + 16 * b][k];
+    for (int b = 0; b < 4; ++b) bv[b] = *reinterpret_cast<const float4*>(&B[tx + 16 * b][k]);
 #pragma unroll
     for (int a = 0; a < 4; ++a)
 #pragma unroll
-      for (int b = 0; b < 4; ++b) acc[a][b] = fmaf(av[a], bv[b], acc[a][b]);
+      for (int b = 0; b < 4; ++b) {
+        float t = acc[a][b];
+        t = fmaf(av[a].x, bv[b].x, t);
+        t = fmaf(av[a].y, bv[b].y, t);
+        t = fmaf(av[a].z, bv[b].z, t);
+        t = fmaf(av[a].w, bv[b].w, t);
+        acc[a][b] = t;
+      }
   }
 }
 
-constexpr int CHOL_STEP_SMEM = 3 * NB * (NB + 1) * (int)sizeof(float);
+constexpr int CHOL_STEP_SMEM = 3 * NB * MMS * (int)sizeof(float);
 
 // One step of the right-looking 64-column Cholesky inside the diagonal square [o, o+sz)
 // of the Gram matrix, in ONE launch: with the diagonal block of block column j already
@@ -304,9 +320,9 @@ __global__ void __launch_bounds__(256) k_chol_step(float* __restrict__ A, i64 ld
   }
   if (adaptive && os[OS_DONE] != 0) return;
   extern __shared__ __align__(16) float chol_smem[];
-  blk_t S0 = reinterpret_cast<blk_t>(chol_smem);
-  blk_t S1 = reinterpret_cast<blk_t>(chol_smem + NB * (NB + 1));
-  blk_t S2 = reinterpret_cast<blk_t>(chol_smem + 2 * NB * (NB + 1));
+  mm_t S0 = reinterpret_cast<mm_t>(chol_smem);
+  mm_t S1 = reinterpret_cast<mm_t>(chol_smem + NB * MMS);
+  mm_t S2 = reinterpret_cast<mm_t>(chol_smem + 2 * NB * MMS);
   __shared__ float gd[NB];
   __shared__ float rdiag[NB];
   __shared__ int deflated[NB];
@@ -319,7 +335,9 @@ __global__ void __launch_bounds__(256) k_chol_step(float* __restrict__ A, i64 ld
   const int rows_i = (int)((o + sz - ri < NB) ? (o + sz - ri) : NB);
   const int rows_k = (int)((o + sz - rk < NB) ? (o + sz - rk) : NB);
   const bool diag = (bi == bk);
+  const bool next_diag = (bi == 0 && bk == 0);
   const float* DPj = DinvP + (cj / NB) * (NB * NB);
+  float cblk[4][4];      // this thread's entries of trailing block (i, k), fetched ahead of the products
   {
     float vi[NB * NB / 256], vk[NB * NB / 256], vd[NB * NB / 256];
 #pragma unroll
@@ -329,6 +347,13 @@ __global__ void __launch_bounds__(256) k_chol_step(float* __restrict__ A, i64 ld
       vk[l] = (!diag && i < rows_k) ? A[(rk + i) * ld + cj + c] : 0.f;
       vd[l] = DPj[e];
     }
+#pragma unroll
+    for (int a = 0; a < 4; ++a)
+#pragma unroll
+      for (int b = 0; b < 4; ++b) {
+        const int i = ty * 4 + a, c = tx + 16 * b;
+        cblk[a][b] = (i < rows_i && c < rows_k) ? A[(ri + i) * ld + rk + c] : 0.f;
+      }
 #pragma unroll
     for (int l = 0; l < NB * NB / 256; ++l) {
       const int e = tid + l * 256, i = e / NB, c = e % NB;
@@ -353,36 +378,44 @@ __global__ void __launch_bounds__(256) k_chol_step(float* __restrict__ A, i64 ld
   __syncthreads();
   float acc[4][4] = {};
   mm_nt_64(S0, diag ? S0 : S1, ty, tx, acc);
-  const bool next_diag = (bi == 0 && bk == 0);
+  if (!next_diag) {
+#pragma unroll
+    for (int a = 0; a < 4; ++a)
+#pragma unroll
+      for (int b = 0; b < 4; ++b) {
+        const int i = ty * 4 + a, c = tx + 16 * b;
+        if (i < rows_i && c < rows_k) A[(ri + i) * ld + rk + c] = cblk[a][b] - acc[a][b];
+      }
+    return;
+  }
+  // the next diagonal block: factor and invert it here.  The three buffers are reused as the
+  // factor L (65-float rows, S2: the inverse of the previous block is no longer needed), its
+  // inverse X (S1) and the scratch T of the inverse levels (S0).
+  blk_t Lb = reinterpret_cast<blk_t>(chol_smem + 2 * NB * MMS);
+  blk_t Xb = reinterpret_cast<blk_t>(chol_smem + NB * MMS);
+  if (tid < NB) {
+    deflated[tid] = 0;
+    gd[tid] = (floor_rel > 0.f && tid < rows_i) ? gdiag[ri + tid] : 0.f;
+  }
+  __syncthreads();                // every thread is done reading S0 / S1 / S2
 #pragma unroll
   for (int a = 0; a < 4; ++a)
 #pragma unroll
     for (int b = 0; b < 4; ++b) {
       const int i = ty * 4 + a, c = tx + 16 * b;
-      float v = 0.f;
-      if (i < rows_i && c < rows_k) {
-        v = A[(ri + i) * ld + rk + c] - acc[a][b];
-        if (!next_diag) A[(ri + i) * ld + rk + c] = v;
-      }
-      if (next_diag) S2[i][c] = (c < i) ? v : ((c == i) ? ((i < rows_i) ? v : 1.f) : 0.f);
+      const float v = cblk[a][b] - acc[a][b];
+      Lb[i][c] = (c < i) ? v : ((c == i) ? ((i < rows_i) ? v : 1.f) : 0.f);
     }
-  if (!next_diag) return;
-  // the next diagonal block: factor and invert it here
-  if (tid < NB) {
-    deflated[tid] = 0;
-    gd[tid] = (floor_rel > 0.f && tid < rows_i) ? gdiag[ri + tid] : 0.f;
-  }
-  __syncthreads();                // every thread is done reading S0 / S1
-  for (int e = tid; e < NB * NB; e += 256) S1[e / NB][e % NB] = 0.f;
+  for (int e = tid; e < NB * NB; e += 256) Xb[e / NB][e % NB] = 0.f;
   __syncthreads();
-  potrf_block(S2, S1, reinterpret_cast<half_blk_t>(chol_smem), gd, rdiag, deflated, rows_i, floor_rel, os, status);
+  potrf_block(Lb, Xb, reinterpret_cast<half_blk_t>(chol_smem), gd, rdiag, deflated, rows_i, floor_rel, os, status);
   float* Dn = Dinv + (ri / NB) * (NB * NB);
   float* DPn = DinvP + (ri / NB) * (NB * NB);
   for (int e = tid; e < NB * NB; e += 256) {
     const int i = e / NB, c = e % NB;
-    if (i < rows_i && c < rows_i) A[(ri + i) * ld + ri + c] = (c <= i) ? S2[i][c] : 0.f;
-    Dn[e] = S1[i][c];
-    DPn[e] = deflated[i] ? 0.f : S1[i][c];
+    if (i < rows_i && c < rows_i) A[(ri + i) * ld + ri + c] = (c <= i) ? Lb[i][c] : 0.f;
+    Dn[e] = Xb[i][c];
+    DPn[e] = deflated[i] ? 0.f : Xb[i][c];
   }
 }
 
