@@ -384,7 +384,7 @@ struct TileMap {
 // brings the product to the accuracy of an fp32 FMA loop (measured 3.3e-7 against
 // 9.1e-7 relative error on Gaussian data).  Used for the products whose error the
 // conditioning of an ill-conditioned panel amplifies.
-template <int BN, bool BF16, bool SPLIT = false, bool TMA = false, bool D16 = false>
+template <int BN, bool BF16, bool SPLIT = false, bool TMA = false, bool D16 = false, bool CE = false>
 struct Cfg {
   // BT: bf16 operands formed in shared memory from TMA-loaded fp32 tiles (K block of 32, as in
   // the fp32 TMA variant).  A stage then holds the raw fp32 tiles of A, of its fp32 addend and
@@ -398,9 +398,16 @@ struct Cfg {
   static constexpr int B_BYTES = BN * 128;
   static constexpr int STAGE_BYTES = BT ? (2 * A_BYTES + B_BYTES + A_BYTES / 2 + B_BYTES / 2)
                                         : (BF16 ? 1 : 2) * (A_BYTES + B_BYTES);
-  static constexpr int STAGES = (192 * 1024) / STAGE_BYTES;
+  // CE (coalesced epilogue): each epilogue warp transposes its 32 x 32 accumulator slabs through a
+  // private shared-memory tile (32 rows of 36 floats), so that one global access of the warp
+  // covers four 128-byte row segments instead of 32 rows; paid for with one stage.
+  static constexpr int EPI_TILE_FLOATS = 32 * 36;
+  // D16: the producer warps have no conversion work and serve as epilogue warps too
+  static constexpr int EPI_WARPS = D16 ? NUM_EPI_WARPS + NUM_PROD_WARPS : NUM_EPI_WARPS;
+  static constexpr int EPI_BYTES = CE ? EPI_WARPS * EPI_TILE_FLOATS * 4 : 0;
+  static constexpr int STAGES = CE ? (232448 - 1536 - EPI_BYTES) / STAGE_BYTES : (192 * 1024) / STAGE_BYTES;
   static constexpr int G16_BYTES = ((BF16 && !TMA) || D16) ? 0 : BM * 32 * 2;   // bf16 addend tile of the TMA variants (per stage)
-  static constexpr int SMEM_BYTES = STAGES * (STAGE_BYTES + G16_BYTES) + 1024 + 512;
+  static constexpr int SMEM_BYTES = STAGES * (STAGE_BYTES + G16_BYTES) + EPI_BYTES + 1024 + 512;
   static constexpr int A_CHUNKS = BM * 8 / NUM_PROD_THREADS;  // 16-byte chunks per producer thread
   static constexpr int B_CHUNKS = BN * 8 / NUM_PROD_THREADS;
   static constexpr int ACCS = SPLIT ? 2 : 1;                 // accumulators per tile
@@ -419,11 +426,12 @@ struct Cfg {
 // TMA with bf16 operands: the same loads; the producer warps add, round to bf16 and write
 // the operand tiles the MMA reads (k-contiguous: rows of 64 bytes, 64-byte swizzle;
 // row-contiguous: 128-byte rows of 64 row indices, 128-byte swizzle); one MMA per K step.
-template <int BN, bool A_MN, bool B_MN, bool BF16, bool SPLIT, bool TMA, bool D16 = false>
+template <int BN, bool A_MN, bool B_MN, bool BF16, bool SPLIT, bool TMA, bool D16 = false, bool CE = false>
 __global__ void __launch_bounds__(TMA ? NUM_THREADS_TMA : NUM_THREADS, 1) k_gemm_umma(const __grid_constant__ Params p) {
   static_assert(!(BF16 && SPLIT), "split accumulators belong to the 3xTF32 mode");
   static_assert(!D16 || (BF16 && TMA), "bf16 operands in memory are loaded by TMA");
-  using C = Cfg<BN, BF16, SPLIT, TMA, D16>;
+  static_assert(!CE || D16, "the coalesced epilogue is built for the bf16-array variant");
+  using C = Cfg<BN, BF16, SPLIT, TMA, D16, CE>;
   constexpr int NBUF = C::NBUF, ACCS = C::ACCS;
   constexpr int BKE = C::BKE, EPC = C::EPC, STAGES = C::STAGES;
   if (p.g.skip_flag != nullptr && *p.g.skip_flag != 0) return;
@@ -434,8 +442,9 @@ __global__ void __launch_bounds__(TMA ? NUM_THREADS_TMA : NUM_THREADS, 1) k_gemm
   // control block after the stages
   // after the stages: the bf16 addend staging of the TMA variant, then the control block
   const uint32_t g16_base = smem_base + STAGES * C::STAGE_BYTES;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem_al + STAGES * (C::STAGE_BYTES + C::G16_BYTES));
-  const uint32_t bar0 = smem_base + STAGES * (C::STAGE_BYTES + C::G16_BYTES);
+  float* epi_tiles = reinterpret_cast<float*>(smem_al + STAGES * (C::STAGE_BYTES + C::G16_BYTES));
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem_al + STAGES * (C::STAGE_BYTES + C::G16_BYTES) + C::EPI_BYTES);
+  const uint32_t bar0 = smem_base + STAGES * (C::STAGE_BYTES + C::G16_BYTES) + C::EPI_BYTES;
   auto full_bar = [&](int s) { return bar0 + 8u * s; };
   auto empty_bar = [&](int s) { return bar0 + 8u * (STAGES + s); };
   auto accf_bar = [&](int b) { return bar0 + 8u * (2 * STAGES + b); };
@@ -449,7 +458,7 @@ __global__ void __launch_bounds__(TMA ? NUM_THREADS_TMA : NUM_THREADS, 1) k_gemm
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), NUM_PROD_WARPS); mbar_init(empty_bar(s), 1); }
-    for (int b = 0; b < 2; ++b) { mbar_init(accf_bar(b), 1); mbar_init(acce_bar(b), NUM_EPI_WARPS * 32); }
+    for (int b = 0; b < 2; ++b) { mbar_init(accf_bar(b), 1); mbar_init(acce_bar(b), C::EPI_WARPS * 32); }
     mbar_init(drain_bar, 1);
     if (TMA) for (int s = 0; s < STAGES; ++s) mbar_init(raw_bar(s), 1);
     *dead = 0;
@@ -466,7 +475,7 @@ __global__ void __launch_bounds__(TMA ? NUM_THREADS_TMA : NUM_THREADS, 1) k_gemm
 
   const GemmArgs& g = p.g;
 
-  if (warp < NUM_EPI_WARPS) {
+  if (warp < C::EPI_WARPS) {
     // ------------------------------------------------------------ epilogue
     // The tensor core adds into its accumulator with truncation, so the error of a long
     // accumulation chain grows linearly with its length (measured 7e-9 per k element).
@@ -477,7 +486,8 @@ __global__ void __launch_bounds__(TMA ? NUM_THREADS_TMA : NUM_THREADS, 1) k_gemm
     bool alive = true;
     for (int item = blockIdx.x; item < p.num_items && alive; item += gridDim.x) {
       const Item it = decode_item<BN, BKE>(p, item);
-      const int quad = warp & 3, half = warp >> 2;   // TMEM lane quadrant, column half
+      const int quad = warp & 3, half = warp >> 2;   // TMEM lane quadrant, column part
+      constexpr int SLABS = (BN / 32) / (C::EPI_WARPS / 4);   // 32-column slabs per warp
       const i64 gi = (i64)it.mi * BM + quad * 32 + lane;
       const i64 n0 = (i64)it.ni * BN;
       const float alpha = g.alpha;
@@ -488,7 +498,7 @@ __global__ void __launch_bounds__(TMA ? NUM_THREADS_TMA : NUM_THREADS, 1) k_gemm
         if (!mbar_wait(accf_bar(ab), ph, dead, p.status, 256)) { alive = false; break; }
         tc_fence_after();
 #pragma unroll 1
-        for (int cb = half * (BN / 64); cb < (half + 1) * (BN / 64); ++cb) {
+        for (int cb = half * SLABS; cb < (half + 1) * SLABS; ++cb) {
           float acc[32];
           tmem_ld32(tmem_base + (uint32_t)(ab * ACCS * BN + cb * 32) + ((uint32_t)(quad * 32) << 16), acc);
           if (SPLIT) {
@@ -497,6 +507,54 @@ __global__ void __launch_bounds__(TMA ? NUM_THREADS_TMA : NUM_THREADS, 1) k_gemm
 #pragma unroll
             for (int e = 0; e < 32; ++e) acc[e] += small[e];
           }
+          if (CE) {
+            // transpose the 32 x 32 slab: lane = row on the TMEM side, lane = (row mod 4, 4 columns) on the
+            // memory side, so that every global access of the warp is four full 128-byte row segments
+            float* tb = epi_tiles + warp * C::EPI_TILE_FLOATS;
+#pragma unroll
+            for (int q = 0; q < 8; ++q)
+              *reinterpret_cast<float4*>(tb + lane * 36 + 4 * q) = make_float4(acc[4 * q], acc[4 * q + 1], acc[4 * q + 2], acc[4 * q + 3]);
+            __syncwarp();
+            const bool to_part = p.splits > 1;
+            const bool need_c = !first || (!to_part && g.epi != EPI_STORE && g.epi != EPI_C2_SUB);
+            const bool add_c2 = !to_part && first && (g.epi == EPI_ADD2_SUB || g.epi == EPI_C2_SUB);
+            const bool c2_f32 = (g.c2_mode == ADD_F32 || g.epi == EPI_C2_SUB);
+            const i64 col = n0 + cb * 32 + 4 * (lane & 7);
+            float4* cptr[8];
+            float4 cur[8], c2v[8];
+            bool ok[8];
+#pragma unroll
+            for (int q = 0; q < 8; ++q) {
+              const i64 row = (i64)it.mi * BM + quad * 32 + 4 * q + (lane >> 3);
+              ok[q] = row < g.M && col < g.N;
+              cptr[q] = to_part ? reinterpret_cast<float4*>(g.part + ((i64)it.ks * g.M + row) * g.N + col)
+                                : reinterpret_cast<float4*>(g.C + row * g.ldc + col);
+              cur[q] = make_float4(0.f, 0.f, 0.f, 0.f);
+              c2v[q] = make_float4(0.f, 0.f, 0.f, 0.f);
+              if (ok[q] && need_c) cur[q] = *cptr[q];
+              if (ok[q] && add_c2) {
+                if (c2_f32) {
+                  c2v[q] = __ldg(reinterpret_cast<const float4*>(reinterpret_cast<const float*>(g.C2) + row * g.ldc2 + col));
+                } else {
+                  const uint2 t = __ldg(reinterpret_cast<const uint2*>(reinterpret_cast<const __nv_bfloat16*>(g.C2) + row * g.ldc2 + col));
+                  const __nv_bfloat162 lo = *reinterpret_cast<const __nv_bfloat162*>(&t.x);
+                  const __nv_bfloat162 hi = *reinterpret_cast<const __nv_bfloat162*>(&t.y);
+                  c2v[q] = make_float4(__low2float(lo), __high2float(lo), __low2float(hi), __high2float(hi));
+                }
+              }
+            }
+            float f = 1.f;
+            if (!to_part) f = (g.epi != EPI_STORE) ? -alpha : alpha;
+#pragma unroll
+            for (int q = 0; q < 8; ++q) {
+              if (!ok[q]) continue;
+              const float4 a4 = *reinterpret_cast<const float4*>(tb + (4 * q + (lane >> 3)) * 36 + 4 * (lane & 7));
+              float4 c = cur[q];
+              c.x += c2v[q].x; c.y += c2v[q].y; c.z += c2v[q].z; c.w += c2v[q].w;
+              *cptr[q] = make_float4(fmaf(f, a4.x, c.x), fmaf(f, a4.y, c.y), fmaf(f, a4.z, c.z), fmaf(f, a4.w, c.w));
+            }
+            __syncwarp();      // the tile is rewritten by the next slab
+          } else
           if (gi < g.M) {
             float4* cptr[8];
             float4 cur[8];
@@ -836,20 +894,20 @@ __global__ void __launch_bounds__(TMA ? NUM_THREADS_TMA : NUM_THREADS, 1) k_gemm
   }
 }
 
-template <int BN, bool A_MN, bool B_MN, bool BF16, bool SPLIT, bool TMA, bool D16 = false>
+template <int BN, bool A_MN, bool B_MN, bool BF16, bool SPLIT, bool TMA, bool D16 = false, bool CE = false>
 inline cudaError_t set_smem_attr() {
-  return cudaFuncSetAttribute(k_gemm_umma<BN, A_MN, B_MN, BF16, SPLIT, TMA, D16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              Cfg<BN, BF16, SPLIT, TMA, D16>::SMEM_BYTES);
+  return cudaFuncSetAttribute(k_gemm_umma<BN, A_MN, B_MN, BF16, SPLIT, TMA, D16, CE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              Cfg<BN, BF16, SPLIT, TMA, D16, CE>::SMEM_BYTES);
 }
 
-template <int BN, bool BF16, bool SPLIT, bool TMA, bool D16 = false>
+template <int BN, bool BF16, bool SPLIT, bool TMA, bool D16 = false, bool CE = false>
 inline void launch_variant(const Params& p, bool a_mn, bool b_mn, int grid, cudaStream_t st) {
-  constexpr int smem = Cfg<BN, BF16, SPLIT, TMA, D16>::SMEM_BYTES;
+  constexpr int smem = Cfg<BN, BF16, SPLIT, TMA, D16, CE>::SMEM_BYTES;
   constexpr int threads = TMA ? NUM_THREADS_TMA : NUM_THREADS;
-  if (!a_mn && !b_mn) k_gemm_umma<BN, false, false, BF16, SPLIT, TMA, D16><<<grid, threads, smem, st>>>(p);
-  else if (!a_mn && b_mn) k_gemm_umma<BN, false, true, BF16, SPLIT, TMA, D16><<<grid, threads, smem, st>>>(p);
-  else if (a_mn && b_mn) k_gemm_umma<BN, true, true, BF16, SPLIT, TMA, D16><<<grid, threads, smem, st>>>(p);
-  else k_gemm_umma<BN, true, false, BF16, SPLIT, TMA, D16><<<grid, threads, smem, st>>>(p);
+  if (!a_mn && !b_mn) k_gemm_umma<BN, false, false, BF16, SPLIT, TMA, D16, CE><<<grid, threads, smem, st>>>(p);
+  else if (!a_mn && b_mn) k_gemm_umma<BN, false, true, BF16, SPLIT, TMA, D16, CE><<<grid, threads, smem, st>>>(p);
+  else if (a_mn && b_mn) k_gemm_umma<BN, true, true, BF16, SPLIT, TMA, D16, CE><<<grid, threads, smem, st>>>(p);
+  else k_gemm_umma<BN, true, false, BF16, SPLIT, TMA, D16, CE><<<grid, threads, smem, st>>>(p);
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
@@ -944,7 +1002,8 @@ inline int umma_configure() {
   if (e == cudaSuccess && !F) e = set_smem_attr<BN, A, B, false, false, true>();  \
   if (e == cudaSuccess && !F) e = set_smem_attr<BN, A, B, false, true, true>();  \
   if (e == cudaSuccess && F) e = set_smem_attr<BN, A, B, true, false, true>();    \
-  if (e == cudaSuccess && F) e = set_smem_attr<BN, A, B, true, false, true, true>();
+  if (e == cudaSuccess && F) e = set_smem_attr<BN, A, B, true, false, true, true>();    \
+  if (e == cudaSuccess && F) e = set_smem_attr<BN, A, B, true, false, true, true, true>();
   DION_SET(128, false, false, false) DION_SET(128, false, true, false) DION_SET(128, true, true, false) DION_SET(128, true, false, false)
   DION_SET(256, false, false, false) DION_SET(256, false, true, false) DION_SET(256, true, true, false) DION_SET(256, true, false, false)
   DION_SET(128, false, false, true) DION_SET(128, false, true, true) DION_SET(128, true, true, true) DION_SET(128, true, false, true)
@@ -1036,7 +1095,10 @@ inline int umma_try_launch(const GemmArgs& g_in, int precision, int sm_count, fl
   // split accumulators); 2048 k for bf16 operands loaded through registers
   p.kc = 32;
   const int grid = p.num_items < sm_count ? p.num_items : sm_count;
-  if (d16) {
+  if (d16 && g.epi != EPI_STORE) {   // output-bound products: coalesced epilogue
+    if (BN == 256) launch_variant<256, true, false, true, true, true>(p, a_mn, b_mn, grid, st);
+    else launch_variant<128, true, false, true, true, true>(p, a_mn, b_mn, grid, st);
+  } else if (d16) {
     if (BN == 256) launch_variant<256, true, false, true, true>(p, a_mn, b_mn, grid, st);
     else launch_variant<128, true, false, true, true>(p, a_mn, b_mn, grid, st);
   } else if (bf16 && tma) {
