@@ -106,14 +106,35 @@ def test_bf16_gradient_storage(engine):
     check(snaps[2], ref[2], TOL_FP32, "bf16 G, fp32 arithmetic")
 
 
-def test_bf16_operand_mode_within_its_bar():
-    m, n, r = 1024, 768, 192
-    pb = inputs.make_problem(m, n, r, seed=6, ks=32, g_dtype=torch.bfloat16)
+@pytest.mark.parametrize("m,n,r,gdt", [(1024, 768, 192, torch.bfloat16), (768, 1024, 192, torch.float32),
+                                       (2048, 2048, 512, torch.bfloat16), (1000, 776, 100, torch.bfloat16),
+                                       (644, 388, 68, torch.float32)])
+def test_bf16_operand_mode_within_its_bar(m, n, r, gdt):
+    # shapes whose dimensions are multiples of 8 run the four products on bf16 arrays formed once per
+    # step; the others round fp32 tiles to bf16 inside the kernel
+    pb = inputs.make_problem(m, n, r, seed=6, ks=32, g_dtype=gdt)
     ref = oracle_steps(pb, 10)
     snaps, status, skipped = run_gpu(pb, 10, precision=binding.PREC_BF16_OPERANDS)
     assert status == 0 and skipped == 0
     check(snaps[0], ref[0], TOL_BF16, "step 1")
     check(snaps[9], ref[9], TOL_BF16, "step 10")
+
+
+def test_bf16_operand_mode_grouped_equals_single_calls():
+    shapes = [(512, 256, 64), (256, 512, 64), (512, 256, 64), (384, 384, 96)]
+    pbs = [inputs.make_problem(m, n, r, seed=8, k=k, ks=16, g_dtype=torch.bfloat16) for k, (m, n, r) in enumerate(shapes)]
+    with binding.Dion(mu=MU, eps=EPS, precision=binding.PREC_BF16_OPERANDS) as opt:
+        single = []
+        for pb in pbs:
+            X, M, Q = device_state(pb)
+            opt.step(X, M, pb.grad(0).cuda(), Q, ETA)
+            single.append((X, M, Q))
+        grouped = [device_state(pb) for pb in pbs]
+        opt.step_grouped([(X, M, pb.grad(0).cuda(), Q) for pb, (X, M, Q) in zip(pbs, grouped)], ETA)
+        assert opt.get_status() == (0, 0)
+    for k, (a, b) in enumerate(zip(single, grouped)):
+        for name, u, v in zip("XMQ", a, b):
+            assert torch.equal(u, v), f"matrix {k}: {name} differs"
 
 
 @pytest.mark.parametrize("engine", ENGINES)
@@ -315,6 +336,13 @@ def test_properties_on_the_square_sweep_sizes(m, n, r):
 @pytest.mark.parametrize("m,n,r", [(4096, 4096, 1024), (1024, 4096, 256), (14336, 4096, 1024), (4096, 14336, 1024)])
 def test_properties_on_llama8b_shapes_bf16_gradients(m, n, r):
     step_properties(m, n, r, torch.bfloat16)
+
+
+@pytest.mark.parametrize("m,n,r,gdt", [(8192, 8192, 512, torch.float32), (4096, 4096, 4096, torch.float32),
+                                       (14336, 4096, 1024, torch.bfloat16), (16384, 16384, 1024, torch.float32)])
+def test_properties_in_bf16_operand_mode_at_bench_sizes(m, n, r, gdt):
+    step_properties(m, n, r, gdt, tol=TOL_BF16, precision=binding.PREC_BF16_OPERANDS, steps=2 if m < 16384 else 1)
+    torch.cuda.empty_cache()
 
 
 @pytest.mark.parametrize("m,n,r", [(16384, 16384, 1024), (32768, 32768, 512)])

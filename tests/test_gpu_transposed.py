@@ -9,7 +9,7 @@ import numpy as np
 import pytest
 import torch
 
-from helpers import EPS, ETA, MU, TOL_FP32, rel, to_np64
+from helpers import EPS, ETA, MU, TOL_BF16, TOL_FP32, rel, to_np64
 from oracle import dion_oracle as orc
 from paper_2504_05295_b200 import binding, build, inputs
 
@@ -116,3 +116,20 @@ def test_transposed_argument_checks():
             d = binding.matrix_desc(X, M, G, Qm, None, True)
             binding._check(opt._lib.dion_lazy_step(opt._ctx, d, ETA, 1, int(torch.cuda.current_stream().cuda_stream)))
         assert opt.get_status() == (0, 0)
+
+
+@pytest.mark.parametrize("m,n,r", [(1024, 512, 128), (520, 1032, 72), (1000, 776, 100)])
+def test_transposed_form_in_bf16_operand_mode(m, n, r):
+    # the first two shapes take the bf16-array products (every dimension a multiple of 8), the last one
+    # the variant that rounds fp32 tiles inside the kernel
+    pb = inputs.make_problem(m, n, r, seed=26, ks=16, g_dtype=torch.bfloat16)
+    Q0 = row_side_factor(m, r, 7)
+    ref = oracle_chain(pb, Q0, 5)
+    X, M, Q = pb.X.cuda().clone(), pb.M.cuda().clone(), Q0.cuda().clone()
+    with binding.Dion(mu=MU, eps=EPS, precision=binding.PREC_BF16_OPERANDS) as opt:
+        for t in range(5):
+            opt.step(X, M, pb.grad(t).cuda(), Q, ETA, transposed=True)
+        assert opt.get_status() == (0, 0)
+    for name, got, want in (("X", X, ref[4].X), ("M", M, ref[4].M), ("Q", Q, ref[4].Q)):
+        e = rel(to_np64(got), want)
+        assert e <= TOL_BF16, f"{name} off by {e:.2e}"
