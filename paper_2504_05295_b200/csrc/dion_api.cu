@@ -3,6 +3,7 @@
 // directory; the host code only validates and launches.
 #include <math.h>
 #include <stdlib.h>
+#include <functional>
 #include <new>
 #include <string.h>
 #include <vector>
@@ -53,6 +54,10 @@ struct dion_ctx {
   size_t prof_used;
   struct ProfRec { int phase; cudaEvent_t e0, e1; int64_t launches; };
   std::vector<ProfRec> prof_recs;
+  // second stream for work that can run beside the serial Cholesky chain, and its fork/join events
+  cudaStream_t side = nullptr;
+  cudaEvent_t side_ev[32] = {};
+  int side_cursor = 0;
 };
 
 namespace {
@@ -212,6 +217,7 @@ struct StepCtx {
   int* flag;  // = os + OS_FAIL: the step must not write its outputs
   bool tensor;  // tensor-core engine allowed for this matrix
   bool in_orth; // inside the orthonormalization (for the profiling phases)
+  bool no_split = false;  // launches on the side stream: the split-K scratch belongs to the main stream
   float* W(int b, i64 off) const { return ws + (i64)b * wstride + off; }
   int* OS(int b) const { return os + (i64)b * OS_SLOT_INTS; }
 };
@@ -224,14 +230,14 @@ int launch_gemm(StepCtx& s, const GemmArgs& g, int b = 0, bool force64 = false) 
     // bf16 operands are for the four large contractions only: the Gram matrices, factors and
     // solves of the orthonormalization keep fp32 accuracy in every mode
     const int prec = s.in_orth ? DION_PREC_FP32 : s.c->cfg.precision;
-    const int rc = umma_try_launch(g, prec, s.c->sm_count, s.W(b, s.L.part), s.L.part_floats,
+    const int rc = umma_try_launch(g, prec, s.c->sm_count, s.no_split ? nullptr : s.W(b, s.L.part), s.L.part_floats,
                                    s.c->dev_ints, s.st);
     if (rc > 0) { s.c->launches += rc; return DION_OK; }
     if (rc < 0) return rc;
     if (s.c->cfg.engine == DION_ENGINE_TENSOR) return DION_ERR_UNSUPPORTED;
   }
   if (g.ab16) return DION_ERR_UNSUPPORTED;   // bf16 arrays are read by the tensor engine only
-  return launch_gemm_simt(s.c, g, s.st, s.W(b, s.L.part), s.L.part_floats, force64);
+  return launch_gemm_simt(s.c, g, s.st, s.no_split ? nullptr : s.W(b, s.L.part), s.L.part_floats, force64);
 }
 
 // Shifts the workspace-resident operands of a product to matrix b of the batch.
@@ -363,7 +369,8 @@ int potrf_inner(StepCtx& s, i64 r, i64 o, i64 sz, bool adaptive) {
 // factor into Linv.  Outer blocks of 512 columns: the diagonal square is factored and
 // inverted by potrf_inner, the panel below it is multiplied by that inverse and the
 // trailing matrix is updated with one rank-512 product (tensor cores where it qualifies).
-int potrf_trtri(StepCtx& s, i64 r, bool adaptive, bool full_inverse) {
+int potrf_trtri(StepCtx& s, i64 r, bool adaptive, bool full_inverse,
+                const std::function<int(i64, i64)>* after_block = nullptr) {
   dion_ctx* c = s.c;
   float* Gm = s.ws + s.L.Gram;
   float* Linv = s.ws + s.L.Linv;
@@ -378,6 +385,7 @@ int potrf_trtri(StepCtx& s, i64 r, bool adaptive, bool full_inverse) {
   for (i64 J0 = 0; J0 < r; J0 += NBO) {
     const i64 sz = (r - J0 < NBO) ? (r - J0) : NBO;
     DION_TRY(potrf_inner(s, r, J0, sz, adaptive));
+    if (after_block != nullptr) DION_TRY((*after_block)(J0, sz));   // block column J of the factor and its inverse are final
     const i64 rem = r - J0 - sz;
     if (rem > 0) {
       float* panel = Gm + (J0 + sz) * r + J0;
@@ -425,8 +433,7 @@ int cholqr_round(StepCtx& s, i64 pin_off, i64 pout_off, i64 rows, i64 r, bool ad
   // Tall panels with r > 512: blocked triangular solve with the 512-column diagonal inverses
   // only (the levels of the triangular inverse above 512 are never formed).
   const bool trsm = (r > NBO) && (rows >= 8192);   // 512-column products need >= 128 row tiles to fill the GPU
-  DION_TRY(potrf_trtri(s, r, adaptive, !trsm));
-  if (adaptive) {
+  if (adaptive) {   // a finished panel is passed through (before anything writes Pout)
     dim3 grid((unsigned)grid_for(c, rows * r), (unsigned)s.nb);
     k_copy_panel<<<grid, 256, 0, s.st>>>(s.ws + pin_off, r, s.ws + pout_off, r, rows, r, nullptr, s.os + OS_DONE, s.wstride);
     DION_CHECK_LAUNCH(c);
@@ -435,10 +442,12 @@ int cholqr_round(StepCtx& s, i64 pin_off, i64 pout_off, i64 rows, i64 r, bool ad
     // Pout_J = (Pin_J - sum_{K<J} Pout_K L_{J,K}^T) Linv_JJ^T, block columns J of 512.
     // The solves run with the plain 3xTF32 product: their rounding error enters U once (~1e-6),
     // whereas an error in the Gram matrix or its factor is amplified by the panel's conditioning.
+    // Block column J needs row block J of the factor and the inverse of its diagonal square, both
+    // final once the factorization has passed J: the solves run on a second stream beside the rest
+    // of the factorization, whose serial 64-column chain leaves most SMs idle.
     const float* Lm = s.ws + s.L.Gram;     // the factor, lower
     float* Wt = s.ws + s.L.R;              // rows x 512 temporary (R is free during the orthonormalization)
-    for (i64 J0 = 0; J0 < r; J0 += NBO) {
-      const i64 sz = (r - J0 < NBO) ? (r - J0) : NBO;
+    auto solve_block = [&](i64 J0, i64 sz) -> int {
       const float* rhs = s.ws + pin_off + J0;
       i64 rhs_ld = r;
       if (J0 > 0) {
@@ -461,6 +470,25 @@ int cholqr_round(StepCtx& s, i64 pin_off, i64 pout_off, i64 rows, i64 r, bool ad
       v.B = s.ws + s.L.Linv + J0 * r + J0; v.b_sk = 1; v.b_sn = r; v.klimit = 1;
       v.C = s.ws + pout_off + J0; v.ldc = r; v.epi = EPI_STORE; v.skip_flag = skip;
       for (int m = 0; m < s.nb; ++m) DION_TRY(launch_gemm(s, for_matrix(s, v, m, true, true, true), m));
+      return DION_OK;
+    };
+    if (c->side != nullptr) {
+      cudaStream_t main_st = s.st;
+      auto next_event = [&]() { cudaEvent_t e = c->side_ev[c->side_cursor]; c->side_cursor = (c->side_cursor + 1) % 32; return e; };
+      const std::function<int(i64, i64)> after_block = [&](i64 J0, i64 sz) -> int {
+        cudaEvent_t e = next_event();
+        if (cudaEventRecord(e, main_st) != cudaSuccess || cudaStreamWaitEvent(c->side, e, 0) != cudaSuccess) return DION_ERR_CUDA;
+        s.st = c->side; s.no_split = true;
+        const int rc = solve_block(J0, sz);
+        s.st = main_st; s.no_split = false;
+        return rc;
+      };
+      DION_TRY(potrf_trtri(s, r, adaptive, false, &after_block));
+      cudaEvent_t e = next_event();   // join: the round ends when the last solve has finished
+      if (cudaEventRecord(e, c->side) != cudaSuccess || cudaStreamWaitEvent(main_st, e, 0) != cudaSuccess) return DION_ERR_CUDA;
+    } else {
+      DION_TRY(potrf_trtri(s, r, adaptive, false));
+      for (i64 J0 = 0; J0 < r; J0 += NBO) DION_TRY(solve_block(J0, (r - J0 < NBO) ? (r - J0) : NBO));
     }
     if (adaptive) {
       k_round_end<<<s.nb, 1, 0, s.st>>>(s.os, GOOD_REL, DONE_REL, c->dev_ints + 2);
@@ -468,6 +496,7 @@ int cholqr_round(StepCtx& s, i64 pin_off, i64 pout_off, i64 rows, i64 r, bool ad
     }
     return DION_OK;
   }
+  DION_TRY(potrf_trtri(s, r, adaptive, true));
   GemmArgs u = gemm_args();
   u.M = rows; u.N = r; u.K = r;
   u.A = s.ws + pin_off; u.a_si = r; u.a_sk = 1;
@@ -887,6 +916,13 @@ int dion_init(dion_ctx** out, const dion_config* cfg) {
   c->dev_ints = (int*)p;
   if (cudaMemset(p, 0, sizeof(int) * (8 + MAX_FLAG_SLOTS * OS_SLOT_INTS)) != cudaSuccess) { cudaFree(p); delete c; return DION_ERR_CUDA; }
   if (configure_kernels() != DION_OK) { cudaFree(p); delete c; return DION_ERR_CUDA; }
+  if (cudaStreamCreateWithFlags(&c->side, cudaStreamNonBlocking) != cudaSuccess) { cudaGetLastError(); c->side = nullptr; }
+  for (int i = 0; i < 32 && c->side != nullptr; ++i)
+    if (cudaEventCreateWithFlags(&c->side_ev[i], cudaEventDisableTiming) != cudaSuccess) {
+      cudaGetLastError();
+      cudaStreamDestroy(c->side);
+      c->side = nullptr;      // no look-ahead: everything runs on the caller's stream
+    }
   if (cfg->workspace_bytes > 0) {
     const int rc = ensure_ws(c, cfg->workspace_bytes);
     if (rc != DION_OK) { cudaFree(c->dev_ints); delete c; return rc; }
@@ -1021,6 +1057,9 @@ void dion_destroy(dion_ctx* ctx) {
   if (ctx->ws != nullptr) cudaFree(ctx->ws);
   if (ctx->dev_ints != nullptr) cudaFree(ctx->dev_ints);
   for (cudaEvent_t e : ctx->prof_pool) cudaEventDestroy(e);
+  for (int i = 0; i < 32; ++i)
+    if (ctx->side_ev[i] != nullptr) cudaEventDestroy(ctx->side_ev[i]);
+  if (ctx->side != nullptr) cudaStreamDestroy(ctx->side);
   delete ctx;
 }
 
