@@ -432,7 +432,9 @@ int cholqr_round(StepCtx& s, i64 pin_off, i64 pout_off, i64 rows, i64 r, bool ad
   DION_CHECK_LAUNCH(c);
   // Tall panels with r > 512: blocked triangular solve with the 512-column diagonal inverses
   // only (the levels of the triangular inverse above 512 are never formed).
-  const bool trsm = (r > NBO) && (rows >= 8192);   // 512-column products need >= 128 row tiles to fill the GPU
+  // alone, 512-column products need >= 128 row tiles to fill the GPU; beside the factorization
+  // (second stream) they are background work at any height
+  const bool trsm = (r > NBO) && (rows >= 8192 || c->side != nullptr);
   if (adaptive) {   // a finished panel is passed through (before anything writes Pout)
     dim3 grid((unsigned)grid_for(c, rows * r), (unsigned)s.nb);
     k_copy_panel<<<grid, 256, 0, s.st>>>(s.ws + pin_off, r, s.ws + pout_off, r, rows, r, nullptr, s.os + OS_DONE, s.wstride);
