@@ -26,7 +26,14 @@
  *   - All step calls are asynchronous on the CUDA stream passed in (a
  *     cudaStream_t cast to void*; NULL = the legacy default stream) and never
  *     synchronise.  Device-side problems (Cholesky breakdown, non-finite pivot)
- *     are latched in a status word read by dion_get_status.
+ *     are latched in a status word read by dion_get_status.  Work issued after
+ *     a call on the same stream sees its results.  Inside a call the library
+ *     may run part of the orthonormalization on a second stream of its own,
+ *     forked from and joined back to the caller's stream with events; nothing
+ *     of a call is left running outside that order.
+ *   - A context's scratch is shared by its calls: two calls on one context must
+ *     not overlap on the GPU (issue them on one stream or order them with
+ *     events); use one context per concurrent stream.
  *   - The context owns only scratch memory (P/U, R, Gram and triangular factors,
  *     column norms, flags).  It grows on demand with cudaMalloc, which
  *     synchronises; after the first call with the largest shapes, or when
