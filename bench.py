@@ -92,6 +92,13 @@ def orth_mode(m, n, r, orth):
 def phase_flops(m, n, r, orth, rounds=None):
     if rounds is None:
         rounds = {1: 2, 2: 4}.get(orth_mode(m, n, r, orth), 0)
+    if orth == 4:
+        # randomized Cholesky QR (the paper's cost table): sketch 2.5 m r^2, QR of the sketch 11/6 r^3,
+        # triangular solve m r^2, then one Cholesky-QR round
+        o = 2.5 * m * r * r + 11.0 / 6.0 * r ** 3 + m * r * r + (2.0 * m * r * r + r ** 3 / 3.0)
+        g = 2.0 * m * n * r
+        og = 3.5 * m * r * r + r ** 3 / 3.0 + (2.0 * m * r * r + 2.0 / 3.0 * r ** 3)
+        return {"P": g, "ORTH": o, "R": g, "EF": g, "COLNORM": 3.0 * n * r, "X": g, "ORTH_GEMM": og}
     if rounds:
         o = rounds * (2.0 * m * r * r + r ** 3 / 3.0)     # Gram (symmetric half) + Cholesky + solve
     else:
@@ -302,8 +309,9 @@ def run_ours(args):
         tr = args.form == "short-side" and m > n
         if tr:
             pb.Q = inputs.row_side_factor(pb)
-        descs = [binding.matrix_desc(pb.X, pb.M, g, pb.Q, d, tr) for g in gs]
-        state.append({"pb": pb, "G": gs, "d": d, "descs": descs, "transposed": tr})
+        sk = inputs.sketch_matrix(pb, transposed=tr) if args.orth == 4 else None   # Algorithm 4's S, 1.25 r rows
+        descs = [binding.matrix_desc(pb.X, pb.M, g, pb.Q, d, tr, sk) for g in gs]
+        state.append({"pb": pb, "G": gs, "d": d, "descs": descs, "transposed": tr, "sketch": sk})
     torch.cuda.synchronize()
 
     opt = binding.Dion(mu=MU, eps=EPS, precision=args.precision, orth=args.orth, engine=args.engine, device=local)
@@ -502,7 +510,7 @@ def run_ours(args):
                        "call": "one dion_step_grouped call per step" if grouped else "one dion_step call per matrix per step",
                        "engine": ["auto", "simt", "tensor"][args.engine],
                        "precision": ["fp32 (3xTF32 on tensor cores / FMA)", "bf16 operands"][args.precision],
-                       "orth": ["auto", "cholqr2", "shifted3", "householder"][args.orth],
+                       "orth": ["auto", "cholqr2", "shifted3", "householder", "rcqr"][args.orth],
                        "form": args.form, "n_transposed": sum(1 for st in state if st["transposed"]),
                        "l2": "inputs larger than L2: the workload's X, M, G (GBs) cycle through between repeats",
                        "replicas": world, "workspace_bytes": need},
@@ -531,7 +539,7 @@ def main():
     ap.add_argument("--cases", default="", help="subset as d:r,d:r (default: the nine cases of the square sweep)")
     ap.add_argument("--engine", type=int, default=0, help="0 auto, 1 simt, 2 tensor")
     ap.add_argument("--precision", type=int, default=0, help="0 fp32, 1 bf16 operands")
-    ap.add_argument("--orth", type=int, default=0, help="0 auto, 1 cholqr2, 2 shifted3, 3 householder")
+    ap.add_argument("--orth", type=int, default=0, help="0 auto, 1 cholqr2, 2 shifted3, 3 householder, 4 randomized Cholesky QR")
     ap.add_argument("--form", default="standard", choices=["standard", "short-side"],
                     help="short-side: matrices with m > n take the transposed form (panel n x r instead of m x r)")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-baseline leg")

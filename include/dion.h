@@ -73,12 +73,20 @@ typedef enum { DION_PREC_FP32 = 0, DION_PREC_BF16_OPERANDS = 1 } dion_precision;
  *                        cuts cond(P) by up to ~100; rounds repeat (at most 6) until one sees a
  *                        well-conditioned panel, one more round then finishes.  The
  *                        decision is taken on the device; unused rounds are skipped.
- * DION_ORTH_HOUSEHOLDER: Householder QR (slow, most robust).                   */
+ * DION_ORTH_HOUSEHOLDER: Householder QR (slow, most robust).
+ * DION_ORTH_RCQR:        randomized Cholesky QR, the paper's Distributed-Orthonormalize
+ *                        (Algorithm 4) on one device: with the caller's sketching matrix S
+ *                        (dion_matrix.sketch), R1 = triangular factor of QR(S P) (Householder,
+ *                        on the small sketch), B = P R1^-1, R2 = Cholesky(B^T B),
+ *                        U = B R2^-1.  Handles ill-conditioned panels with one Gram matrix;
+ *                        the unblocked Householder factorization of the sketch makes it slow
+ *                        for large r.  dion_lazy_step treats it as DION_ORTH_AUTO.           */
 typedef enum {
   DION_ORTH_AUTO = 0,
   DION_ORTH_CHOLQR2 = 1,
   DION_ORTH_SHIFTED3 = 2,
-  DION_ORTH_HOUSEHOLDER = 3
+  DION_ORTH_HOUSEHOLDER = 3,
+  DION_ORTH_RCQR = 4
 } dion_orth;
 
 /* Which kernels carry the contractions.
@@ -144,6 +152,13 @@ typedef struct {
                            stored m x n parameter (rows = "out"), so both forms scale
                            the update alike.  It puts the orthonormalized panel on the
                            n side: cheaper when m > n.  dion_lazy_step rejects it.   */
+  const void* sketch;   /* DION_ORTH_RCQR only (else ignored, may be NULL): the sketching
+                           matrix S of Algorithm 4, fp32, sketch_rows x p row-major, where
+                           p = m (n in the transposed form) is the number of rows of the
+                           panel; read only.  The paper draws 1.25 r Gaussian rows; U does
+                           not depend on S in exact arithmetic.                      */
+  int64_t sketch_rows;  /* r <= sketch_rows <= 2 r                                   */
+  int64_t ld_sketch;    /* >= p                                                      */
 } dion_matrix;
 
 /* Fill *cfg with the defaults: mu 0.95, eps 1e-8, fp32, AUTO, AUTO, device 0, no reserve. */

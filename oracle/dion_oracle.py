@@ -152,6 +152,40 @@ def step_transposed(X, M, G, Q, mu: float, eta: float, eps: float = 1e-8) -> Ste
                       res.P, res.U, res.R, res.degenerate)
 
 
+def rcqr_orthonormalize(P, S):
+    """Distributed-Orthonormalize (Algorithm 4) on one device, step by step in float64:
+    sketch Pt = S P; R1 = triangular factor of QR(Pt); B = P R1^-1; R2 = Cholesky(B^T B)
+    (upper factor); U = B R2^-1.  S is the caller's sketching matrix (k x m, k >= r).
+    The signs of R1 are normalised to a positive diagonal, so U is the thin-QR factor of P
+    with positive diagonal whatever S is."""
+    P = _f64(P); S = _f64(S)
+    m, r = P.shape
+    assert S.shape[1] == m and S.shape[0] >= r
+    Pt = S @ P
+    R1 = np.linalg.qr(Pt, mode="r")
+    R1 = R1 * np.sign(np.diag(R1))[:, None]
+    B = np.linalg.solve(R1.T, P.T).T            # B R1 = P
+    G = B.T @ B
+    R2 = np.linalg.cholesky(G).T                # G = R2^T R2
+    U = np.linalg.solve(R2.T, B.T).T            # U R2 = B
+    return U
+
+
+def step_rcqr(X, M, G, Q, S, mu: float, eta: float, eps: float = 1e-8) -> StepResult:
+    """One Dion step (Algorithm 1 + 2) whose Orthonormalize is Algorithm 4 with sketch S."""
+    X = _f64(X); M = _f64(M); G = _f64(G); Q = _f64(Q)
+    m, n = X.shape
+    B = M + G
+    P = B @ Q
+    U = rcqr_orthonormalize(P, S)
+    R = B.T @ U
+    Mn = B - (1.0 - mu) * (U @ R.T)
+    d = np.sqrt((R * R).sum(axis=0))
+    Qn = R / (d + eps)
+    Xn = X - eta * np.sqrt(m / n) * (U @ Qn.T)
+    return StepResult(Xn, Mn, Qn, d, P, U, R, 0)
+
+
 def sym_power_iter(M, Q):
     """SymPowerIter1 (Algorithm 6): Orthonormalize(M^T M V)."""
     M = _f64(M); Q = _f64(Q).copy()

@@ -18,7 +18,7 @@ LIB_PATH = os.path.join(_HERE, "libdion_b200.so")
 
 DION_F32, DION_BF16 = 0, 1
 PREC_FP32, PREC_BF16_OPERANDS = 0, 1
-ORTH_AUTO, ORTH_CHOLQR2, ORTH_SHIFTED3, ORTH_HOUSEHOLDER = 0, 1, 2, 3
+ORTH_AUTO, ORTH_CHOLQR2, ORTH_SHIFTED3, ORTH_HOUSEHOLDER, ORTH_RCQR = 0, 1, 2, 3, 4
 ENGINE_AUTO, ENGINE_SIMT, ENGINE_TENSOR = 0, 1, 2
 STATUS_BREAKDOWN, STATUS_NONFINITE, STATUS_TIMEOUT, STATUS_ILLCOND = 1, 2, 4, 8
 
@@ -41,7 +41,8 @@ class DionMatrix(ctypes.Structure):
                 ("M", ctypes.c_void_p), ("ldm", ctypes.c_int64),
                 ("G", ctypes.c_void_p), ("ldg", ctypes.c_int64), ("g_dtype", ctypes.c_int),
                 ("Q", ctypes.c_void_p), ("ldq", ctypes.c_int64),
-                ("colnorm_out", ctypes.c_void_p), ("transposed", ctypes.c_int)]
+                ("colnorm_out", ctypes.c_void_p), ("transposed", ctypes.c_int),
+                ("sketch", ctypes.c_void_p), ("sketch_rows", ctypes.c_int64), ("ld_sketch", ctypes.c_int64)]
 
 
 class DionError(RuntimeError):
@@ -113,7 +114,8 @@ def _stream_ptr(stream: Optional[torch.cuda.Stream]) -> int:
 
 
 def matrix_desc(X: torch.Tensor, M: torch.Tensor, G: torch.Tensor, Q: torch.Tensor,
-                colnorm_out: Optional[torch.Tensor] = None, transposed: bool = False) -> DionMatrix:
+                colnorm_out: Optional[torch.Tensor] = None, transposed: bool = False,
+                sketch: Optional[torch.Tensor] = None) -> DionMatrix:
     """Describes one parameter for the C-ABI.  Tensors must be CUDA, 2-D, row-major
     (unit stride along the last dimension); a row stride larger than the width is
     passed on as the leading dimension.  Q is n x r, or m x r in the transposed form."""
@@ -145,6 +147,13 @@ def matrix_desc(X: torch.Tensor, M: torch.Tensor, G: torch.Tensor, Q: torch.Tens
     else:
         d.colnorm_out = None
     d.transposed = int(bool(transposed))
+    if sketch is not None:
+        if (not sketch.is_cuda or sketch.dtype != torch.float32 or sketch.dim() != 2 or sketch.stride(1) != 1
+                or sketch.shape[1] != (n if transposed else m)):
+            raise ValueError("sketch must be a float32 CUDA matrix with one column per panel row")
+        d.sketch, d.sketch_rows, d.ld_sketch = sketch.data_ptr(), sketch.shape[0], sketch.stride(0)
+    else:
+        d.sketch, d.sketch_rows, d.ld_sketch = None, 0, 0
     return d
 
 
@@ -181,8 +190,9 @@ class Dion:
         _check(lib.dion_init(ctypes.byref(self._ctx), ctypes.byref(cfg)))
         self.device = int(device)
 
-    def step(self, X, M, G, Q, lr: float, colnorm_out=None, stream=None, transposed: bool = False) -> None:
-        d = matrix_desc(X, M, G, Q, colnorm_out, transposed)
+    def step(self, X, M, G, Q, lr: float, colnorm_out=None, stream=None, transposed: bool = False,
+             sketch=None) -> None:
+        d = matrix_desc(X, M, G, Q, colnorm_out, transposed, sketch)
         _check(self._lib.dion_step(self._ctx, ctypes.byref(d), float(lr), _stream_ptr(stream)))
 
     def step_desc(self, desc: DionMatrix, lr: float, stream_ptr: int) -> None:
@@ -196,7 +206,7 @@ class Dion:
 
     def step_grouped(self, mats: Iterable[Tuple], lr: float, stream=None) -> None:
         """mats: iterable of (X, M, G, Q), (X, M, G, Q, colnorm_out) or
-        (X, M, G, Q, colnorm_out, transposed)."""
+        (X, M, G, Q, colnorm_out, transposed[, sketch])."""
         descs: List[DionMatrix] = [matrix_desc(*t) for t in mats]
         arr = self.pack(descs)
         _check(self._lib.dion_step_grouped(self._ctx, arr, len(descs), float(lr), _stream_ptr(stream)))

@@ -32,6 +32,7 @@ inline i64 align64(i64 floats) { return (floats + 63) / 64 * 64; }  // 256-byte 
 
 struct Layout {
   i64 P0, P1, R, Gram, Linv, Tbuf, Dinv, DinvP, part, cn_part, d, gdiag, scal, total;
+  i64 Sk, SkV;              // randomized Cholesky QR: the sketch S P and its Householder vectors (2r x r each)
   i64 B16, Q16, U16, R16;   // bf16-operand mode: bf16(M + G) and the bf16 copies of Q, U, R (offsets in floats)
   i64 part_floats;
   int cn_chunks;
@@ -94,6 +95,11 @@ Layout make_layout(const dion_ctx* c, i64 m, i64 n, i64 r) {
   L.d = o; o += align64(r);
   L.gdiag = o; o += align64(r);
   L.scal = o; o += 64;
+  L.Sk = L.SkV = 0;
+  if (c->cfg.orth == DION_ORTH_RCQR) {
+    L.Sk = o; o += align64(2 * r * r);
+    L.SkV = o; o += align64(2 * r * r);
+  }
   L.B16 = L.Q16 = L.U16 = L.R16 = 0;
   if (c->cfg.precision == DION_PREC_BF16_OPERANDS) {
     L.B16 = o; o += align64((m * n + 1) / 2);
@@ -217,6 +223,7 @@ struct StepCtx {
   int* flag;  // = os + OS_FAIL: the step must not write its outputs
   bool tensor;  // tensor-core engine allowed for this matrix
   bool in_orth; // inside the orthonormalization (for the profiling phases)
+  const dion_matrix* const* list = nullptr;   // the matrices of the chain (sketch pointers of the RCQR mode)
   bool no_split = false;  // launches on the side stream: the split-K scratch belongs to the main stream
   float* W(int b, i64 off) const { return ws + (i64)b * wstride + off; }
   int* OS(int b) const { return os + (i64)b * OS_SLOT_INTS; }
@@ -512,7 +519,9 @@ int cholqr_round(StepCtx& s, i64 pin_off, i64 pout_off, i64 rows, i64 r, bool ad
   return DION_OK;
 }
 
-int householder(StepCtx& s, float* A, float* V, i64 rows, i64 r, int b) {
+// Householder factorization of the rows x r matrix A (ld = r): reflectors into V, the triangular
+// factor into the rows of A above the diagonal and its diagonal into the matrix's d scratch.
+int householder_factor(StepCtx& s, float* A, float* V, i64 rows, i64 r, int b) {
   dion_ctx* c = s.c;
   float* diag = s.W(b, s.L.d);
   for (i64 j = 0; j < r; ++j) {
@@ -524,6 +533,13 @@ int householder(StepCtx& s, float* A, float* V, i64 rows, i64 r, int b) {
       DION_CHECK_LAUNCH(c);
     }
   }
+  return DION_OK;
+}
+
+int householder(StepCtx& s, float* A, float* V, i64 rows, i64 r, int b) {
+  dion_ctx* c = s.c;
+  float* diag = s.W(b, s.L.d);
+  DION_TRY(householder_factor(s, A, V, rows, r, b));
   {
     const i64 total = rows * r;
     int blocks = (int)((total + 255) / 256);
@@ -542,6 +558,55 @@ int householder(StepCtx& s, float* A, float* V, i64 rows, i64 r, int b) {
   return DION_OK;
 }
 
+// Randomized Cholesky QR (Algorithm 4 on one device) of the rows x r panel in P0 of every
+// matrix of the chain; U ends in P0.
+//   Pt = S P (sketch_rows x r);  R1 = triangular factor of QR(Pt), diag > 0 (Householder);
+//   B = P R1^-1 (as P Linv^T with Linv = (R1^T)^-1, the triangular-inverse path of the
+//   Cholesky-QR rounds);  then one plain Cholesky-QR round on B: R2 = Cholesky(B^T B), U = B R2^-1.
+int rcqr(StepCtx& s, i64 rows, i64 r) {
+  dion_ctx* c = s.c;
+  if (s.list == nullptr) return DION_ERR_INVALID;
+  for (int b = 0; b < s.nb; ++b) {
+    const dion_matrix* a = s.list[b];
+    const i64 k = a->sketch_rows;
+    float* Pt = s.W(b, s.L.Sk);
+    GemmArgs g = gemm_args();
+    g.M = k; g.N = r; g.K = rows;
+    g.A = (const float*)a->sketch; g.a_si = a->ld_sketch; g.a_sk = 1;
+    g.B = s.W(b, s.L.P0); g.b_sk = r; g.b_sn = 1;
+    g.C = Pt; g.ldc = r; g.epi = EPI_STORE; g.precise = 1;
+    DION_TRY(launch_gemm(s, g, b));
+    DION_TRY(householder_factor(s, Pt, s.W(b, s.L.SkV), k, r, b));
+    k_rt_to_lower<<<grid_for(c, r * r), 256, 0, s.st>>>(Pt, r, s.W(b, s.L.d), s.W(b, s.L.Gram), r, r,
+                                                         s.OS(b) + OS_FAIL, c->dev_ints);
+    DION_CHECK_LAUNCH(c);
+  }
+  // Linv = (R1^T)^-1: 64 x 64 diagonal inverses, then the doubling levels
+  {
+    dim3 grid((unsigned)((r + NB - 1) / NB), (unsigned)s.nb);
+    k_trtri_diag<<<grid, 256, 0, s.st>>>(s.ws + s.L.Gram, r, r, s.ws + s.L.Dinv, s.wstride);
+    DION_CHECK_LAUNCH(c);
+  }
+  if (r > NBO)
+    for (int m = 0; m < s.nb; ++m)
+      if (cudaMemsetAsync(s.W(m, s.L.Linv), 0, sizeof(float) * (size_t)r * (size_t)r, s.st) != cudaSuccess) return DION_ERR_CUDA;
+  for (i64 J0 = 0; J0 < r; J0 += NBO) {
+    const i64 sz = (r - J0 < NBO) ? (r - J0) : NBO;
+    dim3 grid((unsigned)grid_for(c, sz * sz), (unsigned)s.nb);
+    k_linv_init<<<grid, 256, 0, s.st>>>(s.ws + s.L.Linv, r, J0, sz, s.ws + s.L.Dinv, nullptr, s.wstride);
+    DION_CHECK_LAUNCH(c);
+    DION_TRY(trtri_levels(s, r, J0, sz, NB, nullptr, 0));
+  }
+  if (r > NBO) DION_TRY(trtri_levels(s, r, 0, r, NBO, nullptr, 1));
+  GemmArgs u = gemm_args();   // B = P Linv^T
+  u.M = rows; u.N = r; u.K = r;
+  u.A = s.ws + s.L.P0; u.a_si = r; u.a_sk = 1;
+  u.B = s.ws + s.L.Linv; u.b_sk = 1; u.b_sn = r; u.klimit = 1;
+  u.C = s.ws + s.L.P1; u.ldc = r; u.epi = EPI_STORE; u.precise = 1;
+  for (int m = 0; m < s.nb; ++m) DION_TRY(launch_gemm(s, for_matrix(s, u, m, true, true, true), m));
+  return cholqr_round(s, s.L.P1, s.L.P0, rows, r, false);
+}
+
 // The orthonormalization a step on (m, n, r) will use.
 int resolve_orth(const dion_ctx* c, i64 r, i64 short_dim) {
   int mode = c->cfg.orth;
@@ -552,7 +617,9 @@ int resolve_orth(const dion_ctx* c, i64 r, i64 short_dim) {
 // Orthonormalize the rows x r panel in P0 of every matrix of the chain; *U_off is the
 // scratch offset of the buffer that holds U afterwards.
 int orthonormalize(StepCtx& s, i64 rows, i64 r, i64 short_dim, i64* U_off) {
-  const int mode = resolve_orth(s.c, r, short_dim);
+  int mode = resolve_orth(s.c, r, short_dim);
+  if (mode == DION_ORTH_RCQR && s.list == nullptr)   // no sketches on this path (Lazy-Dion): as AUTO
+    mode = (4 * r <= short_dim) ? DION_ORTH_CHOLQR2 : DION_ORTH_SHIFTED3;
   if (mode == DION_ORTH_CHOLQR2) {
     DION_TRY(cholqr_round(s, s.L.P0, s.L.P1, rows, r, false));
     DION_TRY(cholqr_round(s, s.L.P1, s.L.P0, rows, r, false));
@@ -567,6 +634,9 @@ int orthonormalize(StepCtx& s, i64 rows, i64 r, i64 short_dim, i64* U_off) {
     k_orth_finish<<<s.nb, 1, 0, s.st>>>(s.os, s.c->dev_ints);
     s.c->launches++;
     if (cudaGetLastError() != cudaSuccess) return DION_ERR_CUDA;
+    *U_off = s.L.P0;
+  } else if (mode == DION_ORTH_RCQR) {
+    DION_TRY(rcqr(s, rows, r));
     *U_off = s.L.P0;
   } else {
     for (int m = 0; m < s.nb; ++m) DION_TRY(householder(s, s.W(m, s.L.P0), s.W(m, s.L.P1), rows, r, m));
@@ -646,6 +716,15 @@ int step_batch(dion_ctx* c, const dion_matrix* const* list, int nb, float lr, cu
   const dion_matrix* a0 = list[0];
   DION_TRY(begin_step(c, a0, nb, st, &s));
   const i64 m = a0->m, n = a0->n, r = a0->r;
+  s.list = list;
+  if (c->cfg.orth == DION_ORTH_RCQR) {
+    const i64 panel_rows = a0->transposed ? n : m;
+    for (int b = 0; b < nb; ++b) {
+      const dion_matrix* a = list[b];
+      if (a->sketch == nullptr || ((uintptr_t)a->sketch & 3)) return DION_ERR_INVALID;
+      if (a->sketch_rows < r || a->sketch_rows > 2 * r || a->ld_sketch < panel_rows) return DION_ERR_SHAPE;
+    }
+  }
 
   // Standard form: the power iteration runs on B = M + G (panel P = B Q, m x r; Q is n x r).
   // Transposed form: it runs on B^T (panel P = B^T Q, n x r; Q is m x r), and the rank-r
@@ -895,7 +974,7 @@ int dion_init(dion_ctx** out, const dion_config* cfg) {
   *out = nullptr;
   if (cfg == nullptr) return DION_ERR_INVALID;
   if (cfg->precision != DION_PREC_FP32 && cfg->precision != DION_PREC_BF16_OPERANDS) return DION_ERR_INVALID;
-  if (cfg->orth < DION_ORTH_AUTO || cfg->orth > DION_ORTH_HOUSEHOLDER) return DION_ERR_INVALID;
+  if (cfg->orth < DION_ORTH_AUTO || cfg->orth > DION_ORTH_RCQR) return DION_ERR_INVALID;
   if (cfg->engine < DION_ENGINE_AUTO || cfg->engine > DION_ENGINE_TENSOR) return DION_ERR_INVALID;
   if (!(cfg->mu >= 0.f && cfg->mu <= 1.f) || !(cfg->eps >= 0.f)) return DION_ERR_INVALID;
   int ndev = 0;

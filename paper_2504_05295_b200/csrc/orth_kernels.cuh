@@ -82,6 +82,31 @@ __device__ __forceinline__ void trtri_level(blk_t L, blk_t X, half_blk_t T, int 
   __syncthreads();
 }
 
+// Inverse X of the lower-triangular 64 x 64 block L (shared memory; rdiag[i] = 1 / L[i][i];
+// X zero on entry): 16 x 16 diagonal inverses by forward substitution, then doubling.
+// Called by all 256 threads after a block-wide barrier; ends with one.
+__device__ __forceinline__ void invert_block(blk_t L, blk_t X, half_blk_t T, const float* rdiag, int tid) {
+  constexpr int W = 16;
+  if (tid < NB) {
+    const int b0 = (tid / W) * W, q = tid % W;
+    float x[W];
+#pragma unroll
+    for (int i = 0; i < W; ++i) {
+      float sacc = (i == q) ? 1.f : 0.f;
+#pragma unroll
+      for (int k = 0; k < i; ++k)
+        if (k >= q) sacc = fmaf(-L[b0 + i][b0 + k], x[k], sacc);
+      x[i] = (i >= q) ? sacc * rdiag[b0 + i] : 0.f;
+    }
+#pragma unroll
+    for (int i = 0; i < W; ++i) X[b0 + i][b0 + q] = x[i];
+  }
+  __syncthreads();
+  // ... then [[X11, 0], [-X22 L21 X11, X22]] for block sizes 16 and 32
+  trtri_level<16>(L, X, T, tid);
+  trtri_level<32>(L, X, T, tid);
+}
+
 // Cholesky factor and its inverse of the 64 x 64 block held in L (shared memory; lower
 // triangle, identity padding beyond a ragged block of jb columns), by the 256 threads of
 // a CTA.  On return L holds the factor, X its inverse, deflated[] the deflated columns.
@@ -184,25 +209,7 @@ __device__ __forceinline__ void potrf_block(blk_t L, blk_t X, half_blk_t T, cons
     }
   }
 
-  // inverse of the factor: 16 x 16 diagonal inverses by forward substitution ...
-  if (tid < NB) {
-    const int b0 = (tid / W) * W, q = tid % W;
-    float x[W];
-#pragma unroll
-    for (int i = 0; i < W; ++i) {
-      float sacc = (i == q) ? 1.f : 0.f;
-#pragma unroll
-      for (int k = 0; k < i; ++k)
-        if (k >= q) sacc = fmaf(-L[b0 + i][b0 + k], x[k], sacc);
-      x[i] = (i >= q) ? sacc * rdiag[b0 + i] : 0.f;
-    }
-#pragma unroll
-    for (int i = 0; i < W; ++i) X[b0 + i][b0 + q] = x[i];
-  }
-  __syncthreads();
-  // ... then [[X11, 0], [-X22 L21 X11, X22]] for block sizes 16 and 32
-  trtri_level<16>(L, X, T, tid);
-  trtri_level<32>(L, X, T, tid);
+  invert_block(L, X, T, rdiag, tid);
 }
 
 // Cholesky of one jb x jb (jb <= 64) diagonal block, in place (lower factor, the
@@ -555,6 +562,58 @@ __global__ void k_copy_panel(const float* __restrict__ V, i64 ldv, float* __rest
 // Counts a skipped step (breakdown) at the end of a step's launch chain.
 __global__ void k_finish_step(const int* __restrict__ step_flag, int* __restrict__ skipped) {
   if (step_flag[(i64)blockIdx.x * OS_SLOT_INTS] != 0) atomicAdd(skipped, 1);
+}
+
+// Inverse of every 64 x 64 diagonal block of the lower-triangular r x r matrix A into Dinv
+// (block j -> Dinv + j * 64 * 64, zero padded).  grid = (blocks, matrices).
+__global__ void __launch_bounds__(256) k_trtri_diag(const float* __restrict__ A, i64 ld, i64 r,
+                                                    float* __restrict__ Dinv, i64 wstride) {
+  A += (i64)blockIdx.y * wstride; Dinv += (i64)blockIdx.y * wstride;
+  __shared__ float L[NB][NB + 1];
+  __shared__ float X[NB][NB + 1];
+  __shared__ float T[NB / 2][NB / 2 + 1];
+  __shared__ float rdiag[NB];
+  const int tid = threadIdx.x;
+  const i64 j0 = (i64)blockIdx.x * NB;
+  const int jb = (int)((r - j0 < NB) ? (r - j0) : NB);
+  for (int e = tid; e < NB * NB; e += 256) {
+    const int i = e / NB, c = e % NB;
+    float v = (i < jb && c <= i) ? A[(j0 + i) * ld + j0 + c] : 0.f;
+    if (i == c && i >= jb) v = 1.f;
+    L[i][c] = v;
+    X[i][c] = 0.f;
+  }
+  __syncthreads();
+  if (tid < NB) rdiag[tid] = 1.f / L[tid][tid];
+  __syncthreads();
+  invert_block(L, X, T, rdiag, tid);
+  float* D = Dinv + (i64)blockIdx.x * (NB * NB);
+  for (int e = tid; e < NB * NB; e += 256) D[e] = X[e / NB][e % NB];
+}
+
+// After the Householder factorization of a k x r sketch held in A (rows 0..r-1 carry the
+// triangular factor above the diagonal, diag[] its diagonal): writes L = R^T with the sign
+// convention diag(R) > 0 (row j of R is negated when diag[j] < 0) into the lower triangle of G,
+// zeros above.  A diagonal entry that is zero or not finite (rank-deficient sketch) sets
+// *fail and the BREAKDOWN status bit and is replaced by 1.
+__global__ void k_rt_to_lower(const float* __restrict__ A, i64 lda, const float* __restrict__ diag,
+                              float* __restrict__ G, i64 ldg, i64 r, int* __restrict__ fail, int* __restrict__ status) {
+  const i64 total = r * r;
+  for (i64 e = (i64)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (i64)gridDim.x * blockDim.x) {
+    const i64 i = e / r, j = e % r;     // L[i][j] = R[j][i]
+    float v = 0.f;
+    if (j < i) {
+      v = (diag[j] < 0.f) ? -A[j * lda + i] : A[j * lda + i];
+    } else if (j == i) {
+      v = fabsf(diag[i]);
+      if (!(v > 0.f) || !isfinite(v)) {
+        v = 1.f;
+        *fail = 1;
+        atomicOr(status, DION_STATUS_BREAKDOWN);
+      }
+    }
+    G[i * ldg + j] = v;
+  }
 }
 
 // ---------------------------------------------------------------------------

@@ -23,6 +23,7 @@ rank fractions <= 1/4 and ill conditioned (1e4 .. 1e6) at full rank.
 """
 from __future__ import annotations
 
+import math
 from dataclasses import dataclass
 from typing import List, Optional, Tuple
 
@@ -121,6 +122,17 @@ def row_side_factor(pb: DionProblem, device=None) -> torch.Tensor:
     gen = _gen(matrix_seed(pb.seed, 104729), dev)
     Q = _randn((pb.m, pb.r), gen, dev)
     return (Q / torch.linalg.vector_norm(Q.double(), dim=0).float()).contiguous()
+
+
+def sketch_matrix(pb: DionProblem, rows: Optional[int] = None, transposed: bool = False, device=None) -> torch.Tensor:
+    """Sketching matrix of the randomized Cholesky QR (Algorithm 4): `rows` x p Gaussian entries of
+    standard deviation 1/sqrt(rows), p = the number of panel rows (m, or n in the transposed form);
+    rows defaults to ceil(1.25 r).  Drawn from the matrix's own seed."""
+    dev = pb.X.device if device is None else device
+    k = int(math.ceil(1.25 * pb.r)) if rows is None else int(rows)
+    p = pb.n if transposed else pb.m
+    gen = _gen(matrix_seed(pb.seed, 15485863), dev)
+    return (_randn((k, p), gen, dev) / math.sqrt(k)).contiguous()
 
 
 # ---------------------------------------------------------------------------

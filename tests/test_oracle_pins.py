@@ -193,6 +193,37 @@ def test_transposed_form_differs_from_standard_form():
     assert abs(np.linalg.norm(a.X - X) - np.linalg.norm(b.X - X)) < 1e-6 * np.linalg.norm(a.X - X)   # same scale
 
 
+# -- randomized Cholesky QR (Algorithm 4) as Orthonormalize -------------------------
+
+@pytest.mark.parametrize("m,r,decades", [(120, 24, 0), (200, 40, 6), (64, 64, 3)])
+def test_rcqr_returns_the_qr_factor_whatever_the_sketch(m, r, decades):
+    rng = np.random.default_rng(40 + m + r)
+    P = rng.standard_normal((m, r)) @ np.diag(10.0 ** -np.linspace(0, decades, r)) @ rng.standard_normal((r, r))
+    q, rr = np.linalg.qr(P)
+    q = q * np.sign(np.diag(rr))                                   # library QR, positive diagonal
+    k = int(np.ceil(1.25 * r))
+    U1 = orc.rcqr_orthonormalize(P, rng.standard_normal((k, m)) / np.sqrt(k))
+    U2 = orc.rcqr_orthonormalize(P, 7.0 * rng.standard_normal((2 * r, m)))   # other rows, other scale
+    cond = np.linalg.cond(P)
+    assert np.abs(U1.T @ U1 - np.eye(r)).max() < 1e-12
+    assert rel(U1, q) < 1e-13 * cond and rel(U2, q) < 1e-13 * cond
+    assert rel(U1 @ (U1.T @ P), P) < 1e-12                         # range(U) = range(P)
+    Rq = U1.T @ P                                                  # triangular with positive diagonal
+    assert np.abs(np.tril(Rq, -1)).max() < 1e-9 * np.abs(Rq).max() * max(1.0, cond * 1e-6)
+    assert np.all(np.diag(Rq) > 0)
+
+
+def test_step_rcqr_equals_the_plain_step():
+    rng = np.random.default_rng(41)
+    m, n, r = 48, 36, 9
+    X, M, G, Q = draw(rng, m, n, r)
+    S = rng.standard_normal((12, m)) / np.sqrt(12)
+    a = orc.step(X, M, G, Q, MU, ETA, EPS)
+    b = orc.step_rcqr(X, M, G, Q, S, MU, ETA, EPS)
+    for name in ("X", "M", "Q", "d", "U", "R"):
+        assert rel(getattr(b, name), getattr(a, name)) < 1e-11, name
+
+
 # -- pin 6: two-sided orthogonal equivariance (catches layout / transposition) --
 
 def test_orthogonal_equivariance():
