@@ -299,11 +299,15 @@ def run_ours(args):
     # inputs resident in HBM: per case X, M, Q and a ring of two gradients
     state = []
     grouped = args.workload in ("llama8b", "llama405b") and not args.cases
+    dp_sync = args.sync == "dp"
+    if dp_sync and (grouped or args.form != "standard" or args.orth == 4):
+        raise SystemExit("--sync dp steps single matrices in the standard form")
     for k, c in enumerate(cases):
         m, n, r = c[:3]
-        pb = inputs.make_problem(m, n, r, seed=rank, k=k, ks=64, device=dev, keep_signal=False,
+        # data-parallel ranks share X and Q (one seed) and see their own gradients (noise seeded per rank below)
+        pb = inputs.make_problem(m, n, r, seed=0 if dp_sync else rank, k=k, ks=64, device=dev, keep_signal=False,
                                  g_dtype=torch.bfloat16 if case_gbytes(c) == 2 else torch.float32)
-        gs = [pb.grad(t) for t in range(2)]
+        gs = [pb.grad(t + (2 * rank if dp_sync else 0)) for t in range(2)]
         d = torch.zeros(r, device=dev)
         # --form short-side: the transposed form wherever it shortens the orthonormalized panel
         tr = args.form == "short-side" and m > n
@@ -318,7 +322,15 @@ def run_ours(args):
     need = max(opt.workspace_bytes(*c[:3]) for c in cases)
     packed = [binding.Dion.pack([st["descs"][i] for st in state]) for i in range(2)]
 
+    steppers = None
+    if dp_sync:
+        from paper_2504_05295_b200 import dp
+        steppers = [dp.DpStepper(opt, [st["descs"][i] for st in state], dev) for i in range(2)]
+
     def one_step(t, per_case_events=None):
+        if dp_sync:     # project all, all-reduce P, factor all, all-reduce W, finish all
+            steppers[t % 2].step(ETA, stream)
+            return
         if grouped:     # one dion_step_grouped call over the whole list
             opt.step_grouped_packed(packed[t % 2], len(state), ETA, sptr)
             return
@@ -388,9 +400,12 @@ def run_ours(args):
                 st["G"][0].copy_(hg, non_blocking=True)
                 ev = torch.cuda.Event(); ev.record(copy_stream)
                 landed.append(ev)
-        if grouped:
+        if grouped or dp_sync:
             stream.wait_event(landed[-1])
-            opt.step_grouped_packed(packed[0], len(state), ETA, sptr)
+            if grouped:
+                opt.step_grouped_packed(packed[0], len(state), ETA, sptr)
+            else:
+                steppers[0].step(ETA, stream)
             ev = torch.cuda.Event(); ev.record(stream)
             for k, (st, hd) in enumerate(zip(state, host_d)):
                 hd.copy_(st["d"], non_blocking=True)
@@ -511,6 +526,8 @@ def run_ours(args):
                        "engine": ["auto", "simt", "tensor"][args.engine],
                        "precision": ["fp32 (3xTF32 on tensor cores / FMA)", "bf16 operands"][args.precision],
                        "orth": ["auto", "cholqr2", "shifted3", "householder", "rcqr"][args.orth],
+                       "sync": ("compressed data-parallel sync: P and W all-reduced (mean) over the ranks"
+                                if dp_sync else "none (independent replicas)"),
                        "form": args.form, "n_transposed": sum(1 for st in state if st["transposed"]),
                        "l2": "inputs larger than L2: the workload's X, M, G (GBs) cycle through between repeats",
                        "replicas": world, "workspace_bytes": need},
@@ -542,6 +559,9 @@ def main():
     ap.add_argument("--orth", type=int, default=0, help="0 auto, 1 cholqr2, 2 shifted3, 3 householder, 4 randomized Cholesky QR")
     ap.add_argument("--form", default="standard", choices=["standard", "short-side"],
                     help="short-side: matrices with m > n take the transposed form (panel n x r instead of m x r)")
+    ap.add_argument("--sync", default="replicas", choices=["replicas", "dp"],
+                    help="dp: compressed data-parallel sync (P and W all-reduced over the ranks, same X and Q on "
+                         "every rank) instead of independent replicas; standard form, not for the grouped workloads")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-baseline leg")
     args = ap.parse_args()
     if args.impl == "reference":

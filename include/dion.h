@@ -191,6 +191,28 @@ int dion_lazy_step(dion_ctx* ctx, const dion_matrix* a, float lr, int refresh, v
 /* Scratch bytes a step on (m, n, r) needs; 0 if the shape is invalid. */
 size_t dion_workspace_bytes(const dion_ctx* ctx, int64_t m, int64_t n, int64_t r);
 
+/* Compressed data-parallel gradient sync (Section 3.3; the two AllReduce lines of PowerIter1 in
+ * Algorithm 2): the step of dion_step in three calls, between which the caller averages the two
+ * low-rank factors over the data-parallel ranks (any all-reduce; the library makes no collective
+ * call).  Every rank holds the same X and Q, its own gradient G and its own momentum M
+ * ("decoupled momentum"); the weight update is the one dion_step makes on the rank-averaged M and
+ * G, and the rank average of the M buffers is that step's M.  With one rank and no all-reduce the
+ * three calls give dion_step's result.
+ *   dion_dp_project: P (m x r, dense, ld = r, DEVICE, 16-byte aligned) <- (M + G) Q; clears *dp_flag.
+ *   -- caller: P <- mean over ranks --
+ *   dion_dp_factor:  PU holds the averaged P on entry and U = Orthonormalize(P) on return;
+ *                    W (n x r, dense, ld = r) <- (M + G)^T U; sets *dp_flag on a breakdown.
+ *   -- caller: W <- mean over ranks --
+ *   dion_dp_finish:  M <- (M + G) - (1 - mu) U W^T, Q <- ColNorm(W), X <- X - lr sqrt(m/n) U Q^T;
+ *                    does nothing (and counts a skipped step) when *dp_flag != 0.
+ * `a` must describe the same arrays in the three calls and G must stay unchanged between them;
+ * dp_flag is one DEVICE int owned by the caller, one per matrix in flight.  Standard form only;
+ * DION_ORTH_RCQR is not available here (DION_ERR_UNSUPPORTED).  Asynchronous on `cuda_stream`. */
+int dion_dp_project(dion_ctx* ctx, const dion_matrix* a, float* P, int* dp_flag, void* cuda_stream);
+int dion_dp_factor(dion_ctx* ctx, const dion_matrix* a, float* PU, float* W, int* dp_flag, void* cuda_stream);
+int dion_dp_finish(dion_ctx* ctx, const dion_matrix* a, const float* U, const float* W, const int* dp_flag,
+                   float lr, void* cuda_stream);
+
 /* Synchronises `cuda_stream`, then reports and clears the latched device status
  * (DION_STATUS_* bits) and the number of steps skipped because of a breakdown
  * since the last call.  Either output pointer may be NULL. */

@@ -186,6 +186,24 @@ def step_rcqr(X, M, G, Q, S, mu: float, eta: float, eps: float = 1e-8) -> StepRe
     return StepResult(Xn, Mn, Qn, d, P, U, R, 0)
 
 
+def dp_step(X, Ms, Gs, Q, mu: float, eta: float, eps: float = 1e-8):
+    """One Dion step with compressed data-parallel sync (Section 3.3; the AllReduce lines of
+    PowerIter1): rank i holds its own momentum Ms[i] and gradient Gs[i], all ranks hold X and Q.
+    P and W are averaged over the ranks; each momentum takes the same low-rank correction.
+    Returns (X, [M_i], Q, d)."""
+    X = _f64(X); Q = _f64(Q)
+    Bs = [_f64(M) + _f64(G) for M, G in zip(Ms, Gs)]
+    m, n = X.shape
+    P = sum(B @ Q for B in Bs) / len(Bs)                     # AllReduce (mean) of the local B_i V
+    U, _ = householder_qr(P)                                 # Orthonormalize: thin QR, positive diagonal
+    W = sum(B.T @ U for B in Bs) / len(Bs)                   # AllReduce (mean) of the local B_i^T U
+    d = np.sqrt((W * W).sum(axis=0))
+    Qn = W / (d + eps)
+    Mn = [B - (1.0 - mu) * (U @ W.T) for B in Bs]
+    Xn = X - eta * np.sqrt(m / n) * (U @ Qn.T)
+    return Xn, Mn, Qn, d
+
+
 def sym_power_iter(M, Q):
     """SymPowerIter1 (Algorithm 6): Orthonormalize(M^T M V)."""
     M = _f64(M); Q = _f64(Q).copy()

@@ -25,7 +25,8 @@ STATUS_BREAKDOWN, STATUS_NONFINITE, STATUS_TIMEOUT, STATUS_ILLCOND = 1, 2, 4, 8
 EXPORTS = ["dion_default_config", "dion_init", "dion_step", "dion_step_grouped", "dion_lazy_step",
            "dion_workspace_bytes", "dion_get_status", "dion_launch_count", "dion_destroy",
            "dion_strerror", "dion_profile_enable", "dion_profile_read", "dion_get_orth_rounds",
-           "dion_step_noalloc", "dion_noalloc_scratch_limit"]
+           "dion_step_noalloc", "dion_noalloc_scratch_limit", "dion_dp_project", "dion_dp_factor",
+           "dion_dp_finish"]
 PHASES = ["P", "ORTH", "R", "EF", "COLNORM", "X", "ORTH_GEMM"]
 
 
@@ -90,6 +91,12 @@ def load_library() -> ctypes.CDLL:
     lib.dion_step_noalloc.restype = ci
     lib.dion_noalloc_scratch_limit.argtypes = []
     lib.dion_noalloc_scratch_limit.restype = ctypes.c_size_t
+    lib.dion_dp_project.argtypes = [vp, ctypes.POINTER(DionMatrix), vp, vp, vp]
+    lib.dion_dp_project.restype = ci
+    lib.dion_dp_factor.argtypes = [vp, ctypes.POINTER(DionMatrix), vp, vp, vp, vp]
+    lib.dion_dp_factor.restype = ci
+    lib.dion_dp_finish.argtypes = [vp, ctypes.POINTER(DionMatrix), vp, vp, vp, f32, vp]
+    lib.dion_dp_finish.restype = ci
     lib.dion_destroy.argtypes = [vp]
     lib.dion_destroy.restype = None
     lib.dion_strerror.argtypes = [ci]
@@ -218,6 +225,20 @@ class Dion:
         d = matrix_desc(X, M, G, Q, colnorm_out)
         _check(self._lib.dion_lazy_step(self._ctx, ctypes.byref(d), float(lr), int(bool(refresh)),
                                         _stream_ptr(stream)))
+
+    def dp_project(self, desc: DionMatrix, P: torch.Tensor, flag: torch.Tensor, stream=None) -> None:
+        """P <- (M + G) Q for the compressed data-parallel sync; the caller then averages P over the ranks."""
+        _check(self._lib.dion_dp_project(self._ctx, ctypes.byref(desc), P.data_ptr(), flag.data_ptr(), _stream_ptr(stream)))
+
+    def dp_factor(self, desc: DionMatrix, PU: torch.Tensor, W: torch.Tensor, flag: torch.Tensor, stream=None) -> None:
+        """PU: averaged P in, U out; W <- (M + G)^T U; the caller then averages W over the ranks."""
+        _check(self._lib.dion_dp_factor(self._ctx, ctypes.byref(desc), PU.data_ptr(), W.data_ptr(), flag.data_ptr(),
+                                        _stream_ptr(stream)))
+
+    def dp_finish(self, desc: DionMatrix, U: torch.Tensor, W: torch.Tensor, flag: torch.Tensor, lr: float,
+                  stream=None) -> None:
+        _check(self._lib.dion_dp_finish(self._ctx, ctypes.byref(desc), U.data_ptr(), W.data_ptr(), flag.data_ptr(),
+                                        float(lr), _stream_ptr(stream)))
 
     def workspace_bytes(self, m: int, n: int, r: int) -> int:
         return int(self._lib.dion_workspace_bytes(self._ctx, m, n, r))

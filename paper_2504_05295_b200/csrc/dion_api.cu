@@ -646,16 +646,18 @@ int orthonormalize(StepCtx& s, i64 rows, i64 r, i64 short_dim, i64* U_off) {
 }
 
 // ColNorm of matrix b's W (rows x r, ld = r) into `out`.
-int colnorm(StepCtx& s, int b, const float* W, i64 rows, i64 r, float* out, i64 ldo, float* d_out) {
+int colnorm(StepCtx& s, int b, const float* W, i64 rows, i64 r, float* out, i64 ldo, float* d_out,
+            const int* skip = nullptr, i64 ldw = 0) {
+  if (ldw == 0) ldw = r;
   dion_ctx* c = s.c;
   int chunks; i64 per;
   colnorm_plan(rows, r, c->sm_count, &chunks, &per);
   float* part = s.W(b, s.L.cn_part);
   dim3 grid((unsigned)((r + 127) / 128), (unsigned)chunks);
-  k_colsumsq_partial<<<grid, 128, 0, s.st>>>(W, r, rows, r, per, part, nullptr);
+  k_colsumsq_partial<<<grid, 128, 0, s.st>>>(W, ldw, rows, r, per, part, nullptr);
   DION_CHECK_LAUNCH(c);
-  k_colnorm_apply<<<grid, 128, 0, s.st>>>(W, r, rows, r, per, chunks, part, c->cfg.eps, out, ldo,
-                                         s.W(b, s.L.d), d_out, c->dev_ints, s.OS(b) + OS_FAIL);
+  k_colnorm_apply<<<grid, 128, 0, s.st>>>(W, ldw, rows, r, per, chunks, part, c->cfg.eps, out, ldo,
+                                         s.W(b, s.L.d), d_out, c->dev_ints, skip != nullptr ? skip : s.OS(b) + OS_FAIL);
   DION_CHECK_LAUNCH(c);
   return DION_OK;
 }
@@ -1071,6 +1073,97 @@ int dion_lazy_step(dion_ctx* ctx, const dion_matrix* a, float lr, int refresh, v
   if (cudaSetDevice(ctx->cfg.device) != cudaSuccess) return DION_ERR_CUDA;
   DION_TRY(ensure_ws(ctx, dion_workspace_bytes(ctx, a->m, a->n, a->r)));
   return lazy_one(ctx, a, lr, refresh, (cudaStream_t)cuda_stream);
+}
+
+// ---- compressed data-parallel sync: the step in three calls --------------------------------
+
+namespace {
+
+int dp_check(dion_ctx* ctx, const dion_matrix* a, const void* p0, const void* p1, const int* flag) {
+  if (ctx == nullptr || p0 == nullptr || p1 == nullptr || flag == nullptr) return DION_ERR_INVALID;
+  DION_TRY(validate(a));
+  if (a->transposed) return DION_ERR_INVALID;
+  if (((uintptr_t)p0 & 15) || ((uintptr_t)p1 & 15) || ((uintptr_t)flag & 3)) return DION_ERR_ALIGN;
+  if (cudaSetDevice(ctx->cfg.device) != cudaSuccess) return DION_ERR_CUDA;
+  return ensure_ws(ctx, dion_workspace_bytes(ctx, a->m, a->n, a->r));
+}
+
+GemmArgs dp_b_product(const dion_matrix* a, bool transposed_b, const float* rhs, float* out) {
+  const i64 m = a->m, n = a->n, r = a->r;
+  GemmArgs g = gemm_args();
+  g.M = transposed_b ? n : m; g.N = r; g.K = transposed_b ? m : n;
+  g.A = (const float*)a->M; g.a_si = transposed_b ? 1 : a->ldm; g.a_sk = transposed_b ? a->ldm : 1;
+  g.A2 = a->G; g.a2_si = transposed_b ? 1 : a->ldg; g.a2_sk = transposed_b ? a->ldg : 1;
+  g.a2_mode = (a->g_dtype == DION_BF16) ? ADD_BF16 : ADD_F32;
+  g.B = rhs; g.b_sk = r; g.b_sn = 1;
+  g.C = out; g.ldc = r; g.epi = EPI_STORE;
+  return g;
+}
+
+}  // namespace
+
+int dion_dp_project(dion_ctx* ctx, const dion_matrix* a, float* P, int* dp_flag, void* cuda_stream) {
+  DION_TRY(dp_check(ctx, a, P, P, dp_flag));
+  StepCtx s;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  DION_TRY(begin_step(ctx, a, 1, st, &s));
+  if (cudaMemsetAsync(dp_flag, 0, sizeof(int), st) != cudaSuccess) return DION_ERR_CUDA;
+  GemmArgs p = dp_b_product(a, false, (const float*)a->Q, P);
+  p.b_sk = a->ldq;
+  p.precise = (resolve_orth(ctx, a->r, (a->m < a->n) ? a->m : a->n) == DION_ORTH_SHIFTED3) ? 1 : 0;
+  return launch_gemm(s, p, 0);
+}
+
+int dion_dp_factor(dion_ctx* ctx, const dion_matrix* a, float* PU, float* W, int* dp_flag, void* cuda_stream) {
+  DION_TRY(dp_check(ctx, a, PU, W, dp_flag));
+  if (ctx->cfg.orth == DION_ORTH_RCQR) return DION_ERR_UNSUPPORTED;
+  StepCtx s;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  DION_TRY(begin_step(ctx, a, 1, st, &s));
+  const i64 m = a->m, n = a->n, r = a->r;
+  dim3 grid((unsigned)grid_for(ctx, m * r), 1);
+  k_copy_block<<<grid, 256, 0, st>>>(PU, r, s.ws + s.L.P0, r, m, r, nullptr, 0);
+  DION_CHECK_LAUNCH(ctx);
+  i64 U_off = 0;
+  s.in_orth = true;
+  const int rc = orthonormalize(s, m, r, (m < n) ? m : n, &U_off);
+  s.in_orth = false;
+  DION_TRY(rc);
+  k_copy_block<<<grid, 256, 0, st>>>(s.ws + U_off, r, PU, r, m, r, nullptr, 0);
+  DION_CHECK_LAUNCH(ctx);
+  k_latch_flag<<<1, 1, 0, st>>>(s.flag, dp_flag);      // a breakdown cancels dion_dp_finish
+  DION_CHECK_LAUNCH(ctx);
+  return launch_gemm(s, dp_b_product(a, true, PU, W), 0);
+}
+
+int dion_dp_finish(dion_ctx* ctx, const dion_matrix* a, const float* U, const float* W, const int* dp_flag,
+                   float lr, void* cuda_stream) {
+  DION_TRY(dp_check(ctx, a, U, W, dp_flag));
+  StepCtx s;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  DION_TRY(begin_step(ctx, a, 1, st, &s));
+  const i64 m = a->m, n = a->n, r = a->r;
+  GemmArgs e = gemm_args();      // M <- (M + G) - (1 - mu) U W^T, with this rank's M and G
+  e.M = m; e.N = n; e.K = r;
+  e.A = U; e.a_si = r; e.a_sk = 1;
+  e.B = W; e.b_sk = 1; e.b_sn = r;
+  e.C = (float*)a->M; e.ldc = a->ldm; e.epi = EPI_ADD2_SUB;
+  e.C2 = a->G; e.ldc2 = a->ldg; e.c2_mode = (a->g_dtype == DION_BF16) ? ADD_BF16 : ADD_F32;
+  e.alpha = 1.f - ctx->cfg.mu;
+  e.skip_flag = dp_flag;
+  DION_TRY(launch_gemm(s, e, 0));
+  DION_TRY(colnorm(s, 0, W, n, r, (float*)a->Q, a->ldq, a->colnorm_out, dp_flag));
+  GemmArgs x = gemm_args();      // X <- X - lr sqrt(m/n) U Q^T
+  x.M = m; x.N = n; x.K = r;
+  x.A = U; x.a_si = r; x.a_sk = 1;
+  x.B = (const float*)a->Q; x.b_sk = 1; x.b_sn = a->ldq;
+  x.C = (float*)a->X; x.ldc = a->ldx; x.epi = EPI_SUB;
+  x.alpha = lr * sqrtf((float)((double)m / (double)n));
+  x.skip_flag = dp_flag;
+  DION_TRY(launch_gemm(s, x, 0));
+  k_finish_step<<<1, 1, 0, st>>>(dp_flag, ctx->dev_ints + 1);
+  DION_CHECK_LAUNCH(ctx);
+  return DION_OK;
 }
 
 int dion_get_status(dion_ctx* ctx, void* cuda_stream, int* device_status, int* steps_skipped) {

@@ -559,6 +559,11 @@ __global__ void k_copy_panel(const float* __restrict__ V, i64 ldv, float* __rest
   }
 }
 
+// *dst = 1 if *src != 0 (carries a breakdown from one call of a multi-call step to the next).
+__global__ void k_latch_flag(const int* __restrict__ src, int* __restrict__ dst) {
+  if (*src != 0) *dst = 1;
+}
+
 // Counts a skipped step (breakdown) at the end of a step's launch chain.
 __global__ void k_finish_step(const int* __restrict__ step_flag, int* __restrict__ skipped) {
   if (step_flag[(i64)blockIdx.x * OS_SLOT_INTS] != 0) atomicAdd(skipped, 1);

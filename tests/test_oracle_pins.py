@@ -224,6 +224,23 @@ def test_step_rcqr_equals_the_plain_step():
         assert rel(getattr(b, name), getattr(a, name)) < 1e-11, name
 
 
+# -- compressed data-parallel sync (Section 3.3): same weight update as the synchronized step ------
+
+@pytest.mark.parametrize("ranks", [1, 2, 3])
+def test_dp_sync_gives_the_update_of_the_averaged_step(ranks):
+    rng = np.random.default_rng(50 + ranks)
+    m, n, r = 40, 28, 7
+    X, _, _, Q = draw(rng, m, n, r)
+    Ms = [rng.standard_normal((m, n)) for _ in range(ranks)]
+    Gs = [rng.standard_normal((m, n)) for _ in range(ranks)]
+    Xn, Mn, Qn, d = orc.dp_step(X, Ms, Gs, Q, MU, ETA, EPS)
+    ref = orc.step(X, sum(Ms) / ranks, sum(Gs) / ranks, Q, MU, ETA, EPS)
+    assert rel(Xn, ref.X) < 1e-12 and rel(Qn, ref.Q) < 1e-12 and rel(d, ref.d) < 1e-12
+    assert rel(sum(Mn) / ranks, ref.M) < 1e-12              # the mean momentum is the synchronized one
+    if ranks > 1:                                           # the local momenta stay decoupled
+        assert rel(Mn[0] - Mn[1], (Ms[0] + Gs[0]) - (Ms[1] + Gs[1])) < 1e-12
+
+
 # -- pin 6: two-sided orthogonal equivariance (catches layout / transposition) --
 
 def test_orthogonal_equivariance():
