@@ -498,6 +498,16 @@ def run_ours(args):
                                  "per step, all launches"})
     if tensor_engine:
         roof["traffic"] = NCU_TRAFFIC_RATIO * dom_by
+    # The four large products alone (never overlapped with other work; the products inside the
+    # orthonormalization run partly beside its serial chain on a second stream, so their event
+    # durations include waiting for SMs).
+    big = ["P", "R", "EF", "X"]
+    big_ms = sum(phase_ms[p] for p in big) / args.steps
+    if big_ms > 0 and "pipe_frac" in roof:
+        big_tf = sum(tot_fl[p] for p in big) / (big_ms * 1e-3) / 1e12
+        roof["large_products"] = {"phases": big, "ms_per_step": big_ms, "achieved": big_tf,
+                                  "frac": big_tf / flop_peak, "pipe_frac": big_tf * mma_per_product / flop_peak,
+                                  "gbs": sum(tot_by[p] for p in big) / (big_ms * 1e-3) / 1e9}
 
     phases = {}
     for p in binding.PHASES:
