@@ -3,15 +3,22 @@
 // One persistent, warp-specialised kernel computes C = op(A) * op(B) on 128 x BN
 // output tiles:
 //   warps 0-7   epilogue: TMEM -> registers -> fused epilogue -> global memory
-//   warps 8-15  producers: global -> registers -> (M + G add, precision split) ->
-//               shared memory in the UMMA canonical 128-byte-swizzled layout
+//   warps 8-15  producers / converters (see the variants below)
 //   warp  16    one elected thread issues tcgen05.mma and the commits
+//   warp  17    (TMA variants) one elected thread issues the cp.async.bulk.tensor loads
 // Accumulators are double buffered in TMEM (2 x BN columns), so the epilogue of a
-// tile overlaps the main loop of the next one.  Operand tiles go through registers
-// rather than TMA because every large operand is transformed on the way in: the
-// momentum buffer is formed as M + G, and fp32 operands are split into a TF32 "hi"
-// part and an fp32 "lo" remainder (3xTF32: hi*lo + lo*hi + hi*hi carries fp32
-// accuracy), or rounded to bf16 in the bf16-operand mode.
+// tile overlaps the main loop of the next one.  Every large operand is transformed on
+// the way in: the momentum buffer is formed as M + G, and fp32 operands are split into
+// a TF32 "hi" part and an fp32 "lo" remainder (3xTF32: hi*lo + lo*hi + hi*hi carries
+// fp32 accuracy), or rounded to bf16 in the bf16-operand mode.  Variants:
+//   TMA, fp32 mode (default): raw fp32 tiles land in the stage buffers by TMA; the
+//     producer warps add and split in place.
+//   TMA, bf16 operands from fp32 arrays: same loads; the producer warps add, round and
+//     write bf16 operand tiles.
+//   bf16 arrays (D16): TMA writes the operand tiles themselves; the producer warps join
+//     the epilogue; optionally with the coalesced epilogue (CE).
+//   register path: the producer warps load global memory through registers (operands a
+//     tensor map cannot describe).
 //
 // Every wait on an mbarrier is bounded by a cycle budget: when it runs out the CTA
 // marks itself dead, raises DION_STATUS_TIMEOUT and drains, so a protocol bug
