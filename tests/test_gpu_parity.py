@@ -183,6 +183,27 @@ def test_grouped_equals_single_calls():
         assert rel(to_np64(X2), ref[1].X) <= TOL_FP32 and rel(to_np64(Q2), ref[1].Q) <= TOL_FP32
 
 
+@pytest.mark.parametrize("shape,orth", [((2560, 1536, 640), binding.ORTH_AUTO), ((1280, 1280, 1280), binding.ORTH_AUTO)])
+def test_grouped_chain_above_512_columns_equals_single_calls(shape, orth):
+    # r > 512: two-level Cholesky, blocked solves on the second stream, three matrices sharing every small launch
+    m, n, r = shape
+    pbs = [inputs.make_problem(m, n, r, seed=12, k=k, ks=32) for k in range(3)]
+    with binding.Dion(mu=MU, eps=EPS, orth=orth) as opt:
+        single = []
+        for pb in pbs:
+            X, M, Q = device_state(pb)
+            opt.step(X, M, pb.grad(0).cuda(), Q, ETA)
+            single.append((X, M, Q))
+        states = [device_state(pb) for pb in pbs]
+        opt.step_grouped([(X, M, pb.grad(0).cuda(), Q) for pb, (X, M, Q) in zip(pbs, states)], ETA)
+        assert opt.get_status() == (0, 0)
+    for k, ((X1, M1, Q1), (X2, M2, Q2)) in enumerate(zip(single, states)):
+        assert torch.equal(X1, X2) and torch.equal(M1, M2) and torch.equal(Q1, Q2), k
+    ref = oracle_steps(pbs[0], 1)[0]
+    tol = TOL_FP32 if r < min(m, n) else 2e-3
+    assert rel(to_np64(states[0][1]), ref.M) <= TOL_FP32 and rel(to_np64(states[0][0]), ref.X) <= tol
+
+
 def test_checkpoint_resume_is_bit_identical():
     m, n, r, ks = inputs.config1()
     pb = inputs.make_problem(m, n, r, seed=0, ks=ks)
