@@ -123,6 +123,28 @@ def phase_bytes(m, n, r, orth, gbytes=4, rounds=None):
             "ORTH_GEMM": rounds * 4.0 * (3 * m * r + 4 * r * r)}
 
 
+def case_report(c, ms, rounds, args, peaks, binding):
+    """Per-case line: time and the roofline that binds it.  t_hbm: the 7-pass model (read M and G twice,
+    read-modify-write M, read-modify-write X) at the measured copy bandwidth; t_tensor: the four products
+    (and the orthonormalization, always 3xTF32) at the tensor peak of their arithmetic, TF32 taken as half
+    the measured bf16 peak and a 3xTF32 product as three TF32 passes."""
+    m, n, r = c[:3]
+    out = {"m": m, "n": n, "r": r, "ms": ms, "adaptive_orth_rounds": rounds}
+    if ms is None or args.engine == binding.ENGINE_SIMT:
+        return out
+    gb = case_gbytes(c)
+    fl = phase_flops(m, n, r, args.orth, rounds=rounds)
+    model_bytes = float(m) * n * (20 + 2 * gb) + 4.0 * (3 * n * r + 3 * m * r)
+    tf32x3 = peaks["bf16_sustained"] * 0.5 / 3.0
+    prod_peak = peaks["bf16_sustained"] if args.precision == binding.PREC_BF16_OPERANDS else tf32x3
+    t_hbm = model_bytes / (peaks["hbm_gbs"] * 1e9) * 1e3
+    t_tensor = (sum(fl[p] for p in ("P", "R", "EF", "X")) / (prod_peak * 1e12) + fl["ORTH"] / (tf32x3 * 1e12)) * 1e3
+    bound = "hbm" if t_hbm >= t_tensor else "tensor"
+    out.update({"t_hbm_ms": t_hbm, "t_tensor_ms": t_tensor, "bound": bound,
+                "roofline_frac": max(t_hbm, t_tensor) / ms, "model_gbs": model_bytes / (ms * 1e-3) / 1e9})
+    return out
+
+
 def oracle_flops(m, n, r):
     return 8.0 * m * n * r + 4.0 * m * r * r - 4.0 / 3.0 * r ** 3
 
@@ -542,8 +564,7 @@ def run_ours(args):
                        "l2": "inputs larger than L2: the workload's X, M, G (GBs) cycle through between repeats",
                        "replicas": world, "workspace_bytes": need},
             "cases": ([] if len(cases) > 32 else
-                      [{"m": c[0], "n": c[1], "r": c[2], "ms": ms, "adaptive_orth_rounds": nr}
-                       for c, ms, nr in zip(cases, case_ms, case_rounds)]),
+                      [case_report(c, ms, nr, args, peaks, binding) for c, ms, nr in zip(cases, case_ms, case_rounds)]),
             "phases": phases, "roofline": roof, "cpu_baseline": cpu,
             "e2e": {"value": e2e_ms, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "steps": e2e_steps},
