@@ -1000,8 +1000,12 @@ inline bool make_operand_map(CUtensorMap* map, const void* ptr, i64 rows, i64 K,
 // One-time set-up of the tensor-core kernels: opt in to their dynamic shared memory.
 inline int umma_configure() {
   using namespace umma;
-  static bool done = false;
-  if (done) return DION_OK;
+  // function attributes belong to a device's context: once per device of this process
+  static bool done_on[64] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return DION_ERR_CUDA; }
+  const bool tracked = dev >= 0 && dev < 64;
+  if (tracked && done_on[dev]) return DION_OK;
   cudaError_t e = cudaSuccess;
 #define DION_SET(BN, A, B, F)                                              \
   if (e == cudaSuccess) e = set_smem_attr<BN, A, B, F, false, false>();    \
@@ -1017,7 +1021,7 @@ inline int umma_configure() {
   DION_SET(256, false, false, true) DION_SET(256, false, true, true) DION_SET(256, true, true, true) DION_SET(256, true, false, true)
 #undef DION_SET
   if (e != cudaSuccess) { cudaGetLastError(); return DION_ERR_CUDA; }
-  done = true;
+  if (tracked) done_on[dev] = true;
   return DION_OK;
 }
 
