@@ -173,6 +173,19 @@ __device__ __forceinline__ void potrf_block(blk_t L, blk_t X, half_blk_t T, cons
 #pragma unroll
         for (int c = 0; c <= i; ++c) L[c0 + i][c0 + c] = a[i][c];
     }
+    else if (tid >= 32 && c0 > 0) {
+      // meanwhile warps 1-7 finish the trailing update of the previous sub-panel: its columns from
+      // c0 + WF on (the WF columns the piece and the next panel need were updated right away)
+      const int p0 = c0 - WF;                       // the previous sub-panel's first column
+      const int t2 = tid - 32, ty = t2 >> 4, tx = t2 & 15;
+      for (int i = c0 + WF + ty; i < NB; i += 14)
+        for (int c = c0 + WF + tx; c <= i; c += 16) {
+          float sacc = 0.f;
+#pragma unroll
+          for (int k = 0; k < WF; ++k) sacc = fmaf(L[i][p0 + k], L[c][p0 + k], sacc);
+          L[i][c] -= sacc;
+        }
+    }
     __syncthreads();
     const int below = NB - c0 - WF;   // rows under the diagonal piece
     if (tid < below) {
@@ -189,14 +202,17 @@ __device__ __forceinline__ void potrf_block(blk_t L, blk_t X, half_blk_t T, cons
       for (int j = 0; j < WF; ++j) L[i][c0 + j] = x[j];
     }
     __syncthreads();
-    for (int ii = tid >> 4; ii < below; ii += 16)
-      for (int cc = tid & 15; cc <= ii; cc += 16) {
-        const int i = c0 + WF + ii, c = c0 + WF + cc;
+    // trailing update, first part: the WF columns that the next diagonal piece and the panel below
+    // it need (thread -> (row, column)); the rest is deferred to run beside the next diagonal piece
+    for (int e = tid; e < below * WF; e += 256) {
+      const int i = c0 + WF + e / WF, c = c0 + WF + e % WF;
+      if (c <= i) {
         float sacc = 0.f;
 #pragma unroll
         for (int k = 0; k < WF; ++k) sacc = fmaf(L[i][c0 + k], L[c][c0 + k], sacc);
         L[i][c] -= sacc;
       }
+    }
     __syncthreads();
   }
   if (tid == 0) {
