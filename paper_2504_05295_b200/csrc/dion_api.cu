@@ -147,6 +147,18 @@ GemmArgs gemm_args() {
   return g;
 }
 
+// Launch with programmatic stream serialization (see pdl_enter in the kernels).
+template <typename... KArgs, typename... Args>
+cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr; cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, args...);
+}
+
 // Launches one product on the fp32 FMA engine.
 int launch_gemm_simt(dion_ctx* c, GemmArgs g, cudaStream_t st, float* part, i64 part_floats,
                      bool force64) {
@@ -171,8 +183,8 @@ int launch_gemm_simt(dion_ctx* c, GemmArgs g, cudaStream_t st, float* part, i64 
   if (g.batch2 < 1) g.batch2 = 1;
   if (splits > 1 && g.batch2 > 1) return DION_ERR_INVALID;
   dim3 grid((unsigned)gn, (unsigned)gm, (unsigned)(splits > 1 ? splits : g.batch * g.batch2));
-  if (use128) k_gemm_simt<128, 128, 8, 8, 8><<<grid, 256, 0, st>>>(g);
-  else k_gemm_simt<64, 64, 16, 4, 4><<<grid, 256, 0, st>>>(g);
+  if (use128) launch_pdl(k_gemm_simt<128, 128, 8, 8, 8>, grid, dim3(256), 0, st, g);
+  else launch_pdl(k_gemm_simt<64, 64, 16, 4, 4>, grid, dim3(256), 0, st, g);
   DION_CHECK_LAUNCH(c);
   if (splits > 1) {
     const i64 total = g.M * g.N;
@@ -347,26 +359,26 @@ int potrf_inner(StepCtx& s, i64 r, i64 o, i64 sz, bool adaptive) {
   const int nblk = (int)((sz + NB - 1) / NB);
   {
     const int jb = (int)((sz < NB) ? sz : NB);
-    k_potrf_diag<<<s.nb, 256, 0, s.st>>>(Gm + o * r + o, r, jb, Dinv + (o / NB) * (NB * NB), DinvP + (o / NB) * (NB * NB),
-                                         gdiag + o, floor_rel, s.os, adaptive ? 1 : 0, status, s.wstride);
+    launch_pdl(k_potrf_diag, dim3((unsigned)s.nb), dim3(256), 0, s.st, Gm + o * r + o, r, jb, Dinv + (o / NB) * (NB * NB),
+               DinvP + (o / NB) * (NB * NB), gdiag + o, floor_rel, s.os, adaptive ? 1 : 0, status, s.wstride);
     DION_CHECK_LAUNCH(c);
   }
   // one launch per block column: panel, trailing update and the next diagonal block
   for (int j = 0; j + 1 < nblk; ++j) {
     const int nt = nblk - 1 - j;
     dim3 grid((unsigned)(nt * (nt + 1) / 2), (unsigned)s.nb);
-    k_chol_step<<<grid, 256, CHOL_STEP_SMEM, s.st>>>(Gm, r, o, sz, j, Dinv, DinvP, Tbuf, gdiag, floor_rel, s.os,
-                                                     adaptive ? 1 : 0, status, s.wstride);
+    launch_pdl(k_chol_step, grid, dim3(256), CHOL_STEP_SMEM, s.st, Gm, r, o, sz, j, Dinv, DinvP, Tbuf, gdiag, floor_rel,
+               s.os, adaptive ? 1 : 0, status, s.wstride);
     DION_CHECK_LAUNCH(c);
   }
   if (nblk > 1) {
     dim3 grid((unsigned)grid_for(c, sz * sz), (unsigned)s.nb);
-    k_copy_lower_blocks<<<grid, 256, 0, s.st>>>(Tbuf, Gm, r, o, sz, skip, s.wstride);
+    launch_pdl(k_copy_lower_blocks, grid, dim3(256), 0, s.st, (const float*)Tbuf, Gm, r, o, sz, skip, s.wstride);
     DION_CHECK_LAUNCH(c);
   }
   {
     dim3 grid((unsigned)grid_for(c, sz * sz), (unsigned)s.nb);
-    k_linv_init<<<grid, 256, 0, s.st>>>(Linv, r, o, sz, Dinv, skip, s.wstride);
+    launch_pdl(k_linv_init, grid, dim3(256), 0, s.st, Linv, r, o, sz, (const float*)Dinv, skip, s.wstride);
     DION_CHECK_LAUNCH(c);
   }
   return trtri_levels(s, r, o, sz, NB, skip, 0);

@@ -48,6 +48,15 @@ struct GemmArgs {
   int ab16;                      // tensor engine only: A and B point to bf16 arrays (strides in elements), no addend
 };
 
+// Programmatic dependent launch (the small kernels of the serial Cholesky chain): lets the next
+// launch of the stream be scheduled while this grid runs, then waits until the grids this one
+// depends on have completed and their writes are visible.  A kernel launched without the
+// attribute passes through both at once.
+__device__ __forceinline__ void pdl_enter() {
+  asm volatile("griddepcontrol.launch_dependents;");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
 __device__ __forceinline__ float load_add(const void* p, i64 off, int mode) {
   if (mode == ADD_F32) return reinterpret_cast<const float*>(p)[off];
   if (mode == ADD_BF16) return __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(p)[off]);

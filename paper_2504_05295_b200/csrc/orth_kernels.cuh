@@ -252,6 +252,7 @@ __global__ void __launch_bounds__(256) k_potrf_diag(float* __restrict__ A, i64 l
     A += wo; Dinv += wo; DinvP += wo; gdiag += wo;
     os += (i64)blockIdx.x * OS_SLOT_INTS;
   }
+  pdl_enter();
   if (adaptive && os[OS_DONE] != 0) return;
   __shared__ float L[NB][NB + 1];
   __shared__ float X[NB][NB + 1];
@@ -341,6 +342,9 @@ __global__ void __launch_bounds__(256) k_chol_step(float* __restrict__ A, i64 ld
     A += wo; Dinv += wo; DinvP += wo; Lout += wo; gdiag += wo;
     os += (i64)blockIdx.y * OS_SLOT_INTS;
   }
+  // Launched with programmatic stream serialization: the next step's CTAs may be scheduled while
+  // this grid still runs (they wait here), which takes the launch latency off the serial chain.
+  pdl_enter();
   if (adaptive && os[OS_DONE] != 0) return;
   extern __shared__ __align__(16) float chol_smem[];
   mm_t S0 = reinterpret_cast<mm_t>(chol_smem);
@@ -447,6 +451,7 @@ __global__ void __launch_bounds__(256) k_chol_step(float* __restrict__ A, i64 ld
 __global__ void k_copy_lower_blocks(const float* __restrict__ Lout, float* __restrict__ A, i64 ld, i64 o, i64 sz,
                                     const int* __restrict__ skip_flag, i64 wstride) {
   Lout += (i64)blockIdx.y * wstride; A += (i64)blockIdx.y * wstride;
+  pdl_enter();
   if (skip_flag != nullptr && skip_flag[(i64)blockIdx.y * OS_SLOT_INTS] != 0) return;
   const i64 total = sz * sz;
   for (i64 e = (i64)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (i64)gridDim.x * blockDim.x) {
@@ -493,6 +498,7 @@ __global__ void k_orth_finish(int* __restrict__ os, int* __restrict__ status) {
 __global__ void k_linv_init(float* __restrict__ Linv, i64 ld, i64 o, i64 sz, const float* __restrict__ Dinv,
                             const int* __restrict__ skip_flag, i64 wstride) {
   Linv += (i64)blockIdx.y * wstride; Dinv += (i64)blockIdx.y * wstride;   // batched over blockIdx.y
+  pdl_enter();
   if (skip_flag != nullptr && skip_flag[(i64)blockIdx.y * OS_SLOT_INTS] != 0) return;
   const i64 total = sz * sz;
   for (i64 e = (i64)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (i64)gridDim.x * blockDim.x) {

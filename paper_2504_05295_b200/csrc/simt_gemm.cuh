@@ -10,6 +10,7 @@ namespace dion {
 
 template <int BM, int BN, int BK, int TM, int TN>
 __global__ void __launch_bounds__(256) k_gemm_simt(const GemmArgs g) {
+  pdl_enter();
   static_assert((BM / TM) * (BN / TN) == 256, "256 threads per tile");
   static_assert(TM % 4 == 0 && TN % 4 == 0, "micro tile in groups of 4");
   // blockIdx.z = inner batch index + batch * outer batch index (or the K split)
