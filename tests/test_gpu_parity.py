@@ -204,6 +204,27 @@ def test_grouped_chain_above_512_columns_equals_single_calls(shape, orth):
     assert rel(to_np64(states[0][1]), ref.M) <= TOL_FP32 and rel(to_np64(states[0][0]), ref.X) <= tol
 
 
+@pytest.mark.parametrize("m,n,r,precision", [(2048, 2048, 2048, binding.PREC_FP32), (3072, 2048, 1024, binding.PREC_FP32),
+                                             (2048, 2048, 768, binding.PREC_BF16_OPERANDS)])
+def test_repeated_runs_are_bit_identical(m, n, r, precision):
+    # the look-ahead on the library's second stream and the dependent launches must not make a step
+    # depend on timing: the same two steps from the same state give the same bits every time
+    pb = inputs.make_problem(m, n, r, seed=13, ks=64, device="cuda", keep_signal=False)
+    gs = [pb.grad(t) for t in range(2)]
+    ref = None
+    with binding.Dion(mu=MU, eps=EPS, precision=precision) as opt:
+        for rep in range(3):
+            X, M, Q = pb.X.clone(), pb.M.clone(), pb.Q.clone()
+            for t in range(2):
+                opt.step(X, M, gs[t], Q, ETA)
+            torch.cuda.synchronize()
+            if ref is None:
+                ref = (X, M, Q)
+            else:
+                assert all(torch.equal(a, b) for a, b in zip(ref, (X, M, Q))), rep
+        assert opt.get_status() == (0, 0)
+
+
 def test_checkpoint_resume_is_bit_identical():
     m, n, r, ks = inputs.config1()
     pb = inputs.make_problem(m, n, r, seed=0, ks=ks)
