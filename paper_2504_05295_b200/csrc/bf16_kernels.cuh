@@ -17,6 +17,7 @@ template <bool VEC>
 __global__ void __launch_bounds__(256) k_form_b16(const float* __restrict__ M, i64 ldm, const void* __restrict__ G,
                                                   i64 ldg, int g_mode, i64 rows, i64 cols,
                                                   __nv_bfloat16* __restrict__ out) {
+  pdl_enter();
   const i64 per_row = cols / 8;
   const i64 total = rows * per_row;
   for (i64 e = (i64)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (i64)gridDim.x * blockDim.x) {
@@ -65,6 +66,7 @@ __global__ void __launch_bounds__(256) k_form_b16(const float* __restrict__ M, i
 // skip_flag (optional): nothing is written when *skip_flag != 0.
 __global__ void __launch_bounds__(256) k_to_bf16(const float* __restrict__ src, i64 lds, i64 rows, i64 cols,
                                                  __nv_bfloat16* __restrict__ out, const int* __restrict__ skip_flag) {
+  pdl_enter();
   if (skip_flag != nullptr && *skip_flag != 0) return;
   const i64 per_row = cols / 8;
   const i64 total = rows * per_row;

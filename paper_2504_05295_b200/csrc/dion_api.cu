@@ -190,7 +190,7 @@ int launch_gemm_simt(dion_ctx* c, GemmArgs g, cudaStream_t st, float* part, i64 
     const i64 total = g.M * g.N;
     int blocks = (int)((total + 255) / 256);
     if (blocks > 8 * c->sm_count) blocks = 8 * c->sm_count;
-    k_splitk_reduce<<<blocks, 256, 0, st>>>(part, splits, g.M, g.N, g.C, g.ldc, g.alpha, g.tri, BMN, g.skip_flag);
+    launch_pdl(k_splitk_reduce, dim3((unsigned)(blocks)), dim3(256), 0, st, part, splits, g.M, g.N, g.C, g.ldc, g.alpha, g.tri, BMN, g.skip_flag);
     DION_CHECK_LAUNCH(c);
   }
   return DION_OK;
@@ -417,7 +417,7 @@ int potrf_trtri(StepCtx& s, i64 r, bool adaptive, bool full_inverse,
       for (int m = 0; m < s.nb; ++m) DION_TRY(launch_gemm(s, for_matrix(s, g, m, true, true, true), m));
       {
         dim3 grid((unsigned)grid_for(c, rem * sz), (unsigned)s.nb);
-        k_copy_block<<<grid, 256, 0, s.st>>>(ptmp, r, panel, r, rem, sz, skip, s.wstride);
+        launch_pdl(k_copy_block, grid, dim3(256), 0, s.st, ptmp, r, panel, r, rem, sz, skip, s.wstride);
         DION_CHECK_LAUNCH(c);
       }
       GemmArgs t = gemm_args();  // A22 -= Lpanel * Lpanel^T (lower tiles)
@@ -446,7 +446,7 @@ int cholqr_round(StepCtx& s, i64 pin_off, i64 pout_off, i64 rows, i64 r, bool ad
   g.B = s.ws + pin_off; g.b_sk = r; g.b_sn = 1;
   g.C = s.ws + s.L.Gram; g.ldc = r; g.epi = EPI_STORE; g.tri = TRI_LOWER; g.skip_flag = skip; g.precise = adaptive ? 1 : 0;
   for (int m = 0; m < s.nb; ++m) DION_TRY(launch_gemm(s, for_matrix(s, g, m, true, true, true), m));
-  k_round_begin<<<s.nb, 256, 0, s.st>>>(s.ws + s.L.Gram, r, r, 0.f, s.ws + s.L.gdiag, s.ws + s.L.scal, s.os,
+  launch_pdl(k_round_begin, dim3((unsigned)(s.nb)), dim3(256), 0, s.st, s.ws + s.L.Gram, r, r, 0.f, s.ws + s.L.gdiag, s.ws + s.L.scal, s.os,
                                         adaptive ? 1 : 0, s.wstride);
   DION_CHECK_LAUNCH(c);
   // Tall panels with r > 512: blocked triangular solve with the 512-column diagonal inverses
@@ -456,7 +456,7 @@ int cholqr_round(StepCtx& s, i64 pin_off, i64 pout_off, i64 rows, i64 r, bool ad
   const bool trsm = (r > NBO) && (rows >= 8192 || c->side != nullptr);
   if (adaptive) {   // a finished panel is passed through (before anything writes Pout)
     dim3 grid((unsigned)grid_for(c, rows * r), (unsigned)s.nb);
-    k_copy_panel<<<grid, 256, 0, s.st>>>(s.ws + pin_off, r, s.ws + pout_off, r, rows, r, nullptr, s.os + OS_DONE, s.wstride);
+    launch_pdl(k_copy_panel, grid, dim3(256), 0, s.st, s.ws + pin_off, r, s.ws + pout_off, r, rows, r, nullptr, s.os + OS_DONE, s.wstride);
     DION_CHECK_LAUNCH(c);
   }
   if (trsm) {
@@ -512,7 +512,7 @@ int cholqr_round(StepCtx& s, i64 pin_off, i64 pout_off, i64 rows, i64 r, bool ad
       for (i64 J0 = 0; J0 < r; J0 += NBO) DION_TRY(solve_block(J0, (r - J0 < NBO) ? (r - J0) : NBO));
     }
     if (adaptive) {
-      k_round_end<<<s.nb, 1, 0, s.st>>>(s.os, GOOD_REL, DONE_REL, c->dev_ints + 2);
+      launch_pdl(k_round_end, dim3((unsigned)(s.nb)), dim3(1), 0, s.st, s.os, GOOD_REL, DONE_REL, c->dev_ints + 2);
       DION_CHECK_LAUNCH(c);
     }
     return DION_OK;
@@ -525,7 +525,7 @@ int cholqr_round(StepCtx& s, i64 pin_off, i64 pout_off, i64 rows, i64 r, bool ad
   u.C = s.ws + pout_off; u.ldc = r; u.epi = EPI_STORE; u.skip_flag = skip;
   for (int m = 0; m < s.nb; ++m) DION_TRY(launch_gemm(s, for_matrix(s, u, m, true, true, true), m));
   if (adaptive) {
-    k_round_end<<<s.nb, 1, 0, s.st>>>(s.os, GOOD_REL, DONE_REL, c->dev_ints + 2);
+    launch_pdl(k_round_end, dim3((unsigned)(s.nb)), dim3(1), 0, s.st, s.os, GOOD_REL, DONE_REL, c->dev_ints + 2);
     DION_CHECK_LAUNCH(c);
   }
   return DION_OK;
@@ -589,14 +589,14 @@ int rcqr(StepCtx& s, i64 rows, i64 r) {
     g.C = Pt; g.ldc = r; g.epi = EPI_STORE; g.precise = 1;
     DION_TRY(launch_gemm(s, g, b));
     DION_TRY(householder_factor(s, Pt, s.W(b, s.L.SkV), k, r, b));
-    k_rt_to_lower<<<grid_for(c, r * r), 256, 0, s.st>>>(Pt, r, s.W(b, s.L.d), s.W(b, s.L.Gram), r, r,
+    launch_pdl(k_rt_to_lower, dim3((unsigned)(grid_for(c, r * r))), dim3(256), 0, s.st, Pt, r, s.W(b, s.L.d), s.W(b, s.L.Gram), r, r,
                                                          s.OS(b) + OS_FAIL, c->dev_ints);
     DION_CHECK_LAUNCH(c);
   }
   // Linv = (R1^T)^-1: 64 x 64 diagonal inverses, then the doubling levels
   {
     dim3 grid((unsigned)((r + NB - 1) / NB), (unsigned)s.nb);
-    k_trtri_diag<<<grid, 256, 0, s.st>>>(s.ws + s.L.Gram, r, r, s.ws + s.L.Dinv, s.wstride);
+    launch_pdl(k_trtri_diag, grid, dim3(256), 0, s.st, s.ws + s.L.Gram, r, r, s.ws + s.L.Dinv, s.wstride);
     DION_CHECK_LAUNCH(c);
   }
   if (r > NBO)
@@ -605,7 +605,7 @@ int rcqr(StepCtx& s, i64 rows, i64 r) {
   for (i64 J0 = 0; J0 < r; J0 += NBO) {
     const i64 sz = (r - J0 < NBO) ? (r - J0) : NBO;
     dim3 grid((unsigned)grid_for(c, sz * sz), (unsigned)s.nb);
-    k_linv_init<<<grid, 256, 0, s.st>>>(s.ws + s.L.Linv, r, J0, sz, s.ws + s.L.Dinv, nullptr, s.wstride);
+    launch_pdl(k_linv_init, grid, dim3(256), 0, s.st, s.ws + s.L.Linv, r, J0, sz, s.ws + s.L.Dinv, nullptr, s.wstride);
     DION_CHECK_LAUNCH(c);
     DION_TRY(trtri_levels(s, r, J0, sz, NB, nullptr, 0));
   }
@@ -643,7 +643,7 @@ int orthonormalize(StepCtx& s, i64 rows, i64 r, i64 short_dim, i64* U_off) {
       DION_TRY(cholqr_round(s, s.L.P0, s.L.P1, rows, r, true));
       DION_TRY(cholqr_round(s, s.L.P1, s.L.P0, rows, r, true));
     }
-    k_orth_finish<<<s.nb, 1, 0, s.st>>>(s.os, s.c->dev_ints);
+    launch_pdl(k_orth_finish, dim3((unsigned)(s.nb)), dim3(1), 0, s.st, s.os, s.c->dev_ints);
     s.c->launches++;
     if (cudaGetLastError() != cudaSuccess) return DION_ERR_CUDA;
     *U_off = s.L.P0;
@@ -666,9 +666,9 @@ int colnorm(StepCtx& s, int b, const float* W, i64 rows, i64 r, float* out, i64 
   colnorm_plan(rows, r, c->sm_count, &chunks, &per);
   float* part = s.W(b, s.L.cn_part);
   dim3 grid((unsigned)((r + 127) / 128), (unsigned)chunks);
-  k_colsumsq_partial<<<grid, 128, 0, s.st>>>(W, ldw, rows, r, per, part, nullptr);
+  launch_pdl(k_colsumsq_partial, grid, dim3(128), 0, s.st, W, ldw, rows, r, per, part, nullptr);
   DION_CHECK_LAUNCH(c);
-  k_colnorm_apply<<<grid, 128, 0, s.st>>>(W, ldw, rows, r, per, chunks, part, c->cfg.eps, out, ldo,
+  launch_pdl(k_colnorm_apply, grid, dim3(128), 0, s.st, W, ldw, rows, r, per, chunks, part, c->cfg.eps, out, ldo,
                                          s.W(b, s.L.d), d_out, c->dev_ints, skip != nullptr ? skip : s.OS(b) + OS_FAIL);
   DION_CHECK_LAUNCH(c);
   return DION_OK;
@@ -756,7 +756,7 @@ int step_batch(dion_ctx* c, const dion_matrix* const* list, int nb, float lr, cu
     if (((uintptr_t)list[b]->Q & 15) || (list[b]->ldq % 4)) d16 = false;
   auto bf = [&](int b, i64 off) { return reinterpret_cast<__nv_bfloat16*>(s.W(b, off)); };
   auto to_bf16 = [&](const float* src, i64 lds, i64 rows, i64 cols, __nv_bfloat16* out) -> int {
-    k_to_bf16<<<grid_for(c, rows * cols / 8), 256, 0, st>>>(src, lds, rows, cols, out, nullptr);
+    launch_pdl(k_to_bf16, dim3((unsigned)(grid_for(c, rows * cols / 8))), dim3(256), 0, st, src, lds, rows, cols, out, nullptr);
     DION_CHECK_LAUNCH(c);
     return DION_OK;
   };
@@ -773,8 +773,8 @@ int step_batch(dion_ctx* c, const dion_matrix* const* list, int nb, float lr, cu
                        (a->g_dtype == DION_BF16 ? (!((uintptr_t)a->G & 15) && a->ldg % 8 == 0)
                                                 : (!((uintptr_t)a->G & 15) && a->ldg % 4 == 0));
       const int grid = grid_for(c, m * n / 8);
-      if (vec) k_form_b16<true><<<grid, 256, 0, st>>>((const float*)a->M, a->ldm, a->G, a->ldg, g_mode(a), m, n, bf(b, s.L.B16));
-      else k_form_b16<false><<<grid, 256, 0, st>>>((const float*)a->M, a->ldm, a->G, a->ldg, g_mode(a), m, n, bf(b, s.L.B16));
+      if (vec) launch_pdl(k_form_b16<true>, grid, dim3(256), 0, st, (const float*)a->M, a->ldm, a->G, a->ldg, g_mode(a), m, n, bf(b, s.L.B16));
+      else launch_pdl(k_form_b16<false>, grid, dim3(256), 0, st, (const float*)a->M, a->ldm, a->G, a->ldg, g_mode(a), m, n, bf(b, s.L.B16));
       DION_CHECK_LAUNCH(c);
       DION_TRY(to_bf16((const float*)a->Q, a->ldq, qrow, r, bf(b, s.L.Q16)));
       p.ab16 = 1;
@@ -881,7 +881,7 @@ int step_batch(dion_ctx* c, const dion_matrix* const* list, int nb, float lr, cu
     x.skip_flag = s.OS(b) + OS_FAIL;
     DION_TRY(launch_gemm(s, x, b));
   }
-  k_finish_step<<<nb, 1, 0, st>>>(s.flag, c->dev_ints + 1);
+  launch_pdl(k_finish_step, dim3((unsigned)(nb)), dim3(1), 0, st, s.flag, c->dev_ints + 1);
   DION_CHECK_LAUNCH(c);
   }
   return DION_OK;
@@ -931,7 +931,7 @@ int lazy_one(dion_ctx* c, const dion_matrix* a, float lr, int refresh, cudaStrea
     const i64 total = n * r;
     int blocks = (int)((total + 255) / 256);
     if (blocks > 8 * c->sm_count) blocks = 8 * c->sm_count;
-    k_copy_panel<<<blocks, 256, 0, st>>>(V, r, (float*)a->Q, a->ldq, n, r, s.flag, nullptr, 0);
+    launch_pdl(k_copy_panel, dim3((unsigned)(blocks)), dim3(256), 0, st, V, r, (float*)a->Q, a->ldq, n, r, s.flag, nullptr, 0);
     DION_CHECK_LAUNCH(c);
   }
   // W = (M + G) Q
@@ -963,7 +963,7 @@ int lazy_one(dion_ctx* c, const dion_matrix* a, float lr, int refresh, cudaStrea
   x.alpha = lr * sqrtf((float)((double)m / (double)n));
   x.skip_flag = s.flag;
   DION_TRY(launch_gemm(s, x));
-  k_finish_step<<<1, 1, 0, st>>>(s.flag, c->dev_ints + 1);
+  launch_pdl(k_finish_step, dim3((unsigned)(1)), dim3(1), 0, st, s.flag, c->dev_ints + 1);
   DION_CHECK_LAUNCH(c);
   return DION_OK;
 }
@@ -1134,16 +1134,16 @@ int dion_dp_factor(dion_ctx* ctx, const dion_matrix* a, float* PU, float* W, int
   DION_TRY(begin_step(ctx, a, 1, st, &s));
   const i64 m = a->m, n = a->n, r = a->r;
   dim3 grid((unsigned)grid_for(ctx, m * r), 1);
-  k_copy_block<<<grid, 256, 0, st>>>(PU, r, s.ws + s.L.P0, r, m, r, nullptr, 0);
+  launch_pdl(k_copy_block, grid, dim3(256), 0, st, PU, r, s.ws + s.L.P0, r, m, r, nullptr, 0);
   DION_CHECK_LAUNCH(ctx);
   i64 U_off = 0;
   s.in_orth = true;
   const int rc = orthonormalize(s, m, r, (m < n) ? m : n, &U_off);
   s.in_orth = false;
   DION_TRY(rc);
-  k_copy_block<<<grid, 256, 0, st>>>(s.ws + U_off, r, PU, r, m, r, nullptr, 0);
+  launch_pdl(k_copy_block, grid, dim3(256), 0, st, s.ws + U_off, r, PU, r, m, r, nullptr, 0);
   DION_CHECK_LAUNCH(ctx);
-  k_latch_flag<<<1, 1, 0, st>>>(s.flag, dp_flag);      // a breakdown cancels dion_dp_finish
+  launch_pdl(k_latch_flag, dim3((unsigned)(1)), dim3(1), 0, st, s.flag, dp_flag);      // a breakdown cancels dion_dp_finish
   DION_CHECK_LAUNCH(ctx);
   return launch_gemm(s, dp_b_product(a, true, PU, W), 0);
 }
@@ -1173,7 +1173,7 @@ int dion_dp_finish(dion_ctx* ctx, const dion_matrix* a, const float* U, const fl
   x.alpha = lr * sqrtf((float)((double)m / (double)n));
   x.skip_flag = dp_flag;
   DION_TRY(launch_gemm(s, x, 0));
-  k_finish_step<<<1, 1, 0, st>>>(dp_flag, ctx->dev_ints + 1);
+  launch_pdl(k_finish_step, dim3((unsigned)(1)), dim3(1), 0, st, dp_flag, ctx->dev_ints + 1);
   DION_CHECK_LAUNCH(ctx);
   return DION_OK;
 }

@@ -25,6 +25,7 @@ enum : int {
 __global__ void k_round_begin(const float* __restrict__ G, i64 ld, i64 r, float scale,
                               float* __restrict__ gdiag, float* __restrict__ shift,
                               int* __restrict__ os, int adaptive, i64 wstride) {
+  pdl_enter();
   G += (i64)blockIdx.x * wstride; gdiag += (i64)blockIdx.x * wstride; shift += (i64)blockIdx.x * wstride;
   os += (i64)blockIdx.x * OS_SLOT_INTS;
   if (adaptive && os[OS_DONE] != 0) return;
@@ -468,6 +469,7 @@ __global__ void k_copy_lower_blocks(const float* __restrict__ Lout, float* __res
 //     round brings orthonormality to rounding level (the CholeskyQR2 argument), after
 //     which the remaining rounds are skipped.
 __global__ void k_round_end(int* __restrict__ os, float good_rel, float done_rel, int* __restrict__ rounds_total) {
+  pdl_enter();
   os += (i64)blockIdx.x * OS_SLOT_INTS;
   if (os[OS_DONE] != 0) return;
   os[OS_ROUNDS] += 1;
@@ -483,6 +485,7 @@ __global__ void k_round_end(int* __restrict__ os, float good_rel, float done_rel
 // After the last adaptive round: a panel that never became well conditioned is
 // reported; if pivots were still being raised the step is cancelled (rank-deficient P).
 __global__ void k_orth_finish(int* __restrict__ os, int* __restrict__ status) {
+  pdl_enter();
   os += (i64)blockIdx.x * OS_SLOT_INTS;
   if (os[OS_DONE] != 0) return;
   if (os[OS_GOOD] == 0 && os[OS_FLOORED] != 0) {
@@ -512,6 +515,7 @@ __global__ void k_linv_init(float* __restrict__ Linv, i64 ld, i64 o, i64 sz, con
 // Copies a rows x cols block between two matrices (leading dimensions lds, ldd).
 __global__ void k_copy_block(const float* __restrict__ src, i64 lds, float* __restrict__ dst, i64 ldd,
                              i64 rows, i64 cols, const int* __restrict__ skip_flag, i64 wstride) {
+  pdl_enter();
   src += (i64)blockIdx.y * wstride; dst += (i64)blockIdx.y * wstride;     // batched over blockIdx.y
   if (skip_flag != nullptr && skip_flag[(i64)blockIdx.y * OS_SLOT_INTS] != 0) return;
   const i64 total = rows * cols;
@@ -526,6 +530,7 @@ __global__ void k_copy_block(const float* __restrict__ src, i64 lds, float* __re
 __global__ void __launch_bounds__(128) k_colsumsq_partial(const float* __restrict__ R, i64 ld, i64 n, i64 r,
                                                           i64 rows_per_chunk, float* __restrict__ part,
                                                           const int* __restrict__ skip_flag) {
+  pdl_enter();
   if (skip_flag != nullptr && *skip_flag != 0) return;
   const i64 j = (i64)blockIdx.x * 128 + threadIdx.x;
   if (j >= r) return;
@@ -548,6 +553,7 @@ __global__ void __launch_bounds__(128) k_colnorm_apply(const float* __restrict__
                                                        float* __restrict__ d_ws, float* __restrict__ d_out,
                                                        int* __restrict__ status,
                                                        const int* __restrict__ skip_flag) {
+  pdl_enter();
   if (skip_flag != nullptr && *skip_flag != 0) return;
   const i64 j = (i64)blockIdx.x * 128 + threadIdx.x;
   if (j >= r) return;
@@ -570,6 +576,7 @@ __global__ void __launch_bounds__(128) k_colnorm_apply(const float* __restrict__
 __global__ void k_copy_panel(const float* __restrict__ V, i64 ldv, float* __restrict__ Q, i64 ldq,
                              i64 rows, i64 r, const int* __restrict__ skip_flag,
                              const int* __restrict__ only_if, i64 wstride) {
+  pdl_enter();
   V += (i64)blockIdx.y * wstride;                                         // batched over blockIdx.y
   if (wstride != 0) Q += (i64)blockIdx.y * wstride;
   if (skip_flag != nullptr && skip_flag[(i64)blockIdx.y * OS_SLOT_INTS] != 0) return;
@@ -583,11 +590,13 @@ __global__ void k_copy_panel(const float* __restrict__ V, i64 ldv, float* __rest
 
 // *dst = 1 if *src != 0 (carries a breakdown from one call of a multi-call step to the next).
 __global__ void k_latch_flag(const int* __restrict__ src, int* __restrict__ dst) {
+  pdl_enter();
   if (*src != 0) *dst = 1;
 }
 
 // Counts a skipped step (breakdown) at the end of a step's launch chain.
 __global__ void k_finish_step(const int* __restrict__ step_flag, int* __restrict__ skipped) {
+  pdl_enter();
   if (step_flag[(i64)blockIdx.x * OS_SLOT_INTS] != 0) atomicAdd(skipped, 1);
 }
 
@@ -595,6 +604,7 @@ __global__ void k_finish_step(const int* __restrict__ step_flag, int* __restrict
 // (block j -> Dinv + j * 64 * 64, zero padded).  grid = (blocks, matrices).
 __global__ void __launch_bounds__(256) k_trtri_diag(const float* __restrict__ A, i64 ld, i64 r,
                                                     float* __restrict__ Dinv, i64 wstride) {
+  pdl_enter();
   A += (i64)blockIdx.y * wstride; Dinv += (i64)blockIdx.y * wstride;
   __shared__ float L[NB][NB + 1];
   __shared__ float X[NB][NB + 1];
@@ -625,6 +635,7 @@ __global__ void __launch_bounds__(256) k_trtri_diag(const float* __restrict__ A,
 // *fail and the BREAKDOWN status bit and is replaced by 1.
 __global__ void k_rt_to_lower(const float* __restrict__ A, i64 lda, const float* __restrict__ diag,
                               float* __restrict__ G, i64 ldg, i64 r, int* __restrict__ fail, int* __restrict__ status) {
+  pdl_enter();
   const i64 total = r * r;
   for (i64 e = (i64)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (i64)gridDim.x * blockDim.x) {
     const i64 i = e / r, j = e % r;     // L[i][j] = R[j][i]

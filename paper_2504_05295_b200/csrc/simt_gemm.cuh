@@ -168,6 +168,7 @@ __global__ void __launch_bounds__(256) k_gemm_simt(const GemmArgs g) {
 __global__ void k_splitk_reduce(const float* __restrict__ part, int splits, i64 M, i64 N,
                                 float* __restrict__ C, i64 ldc, float alpha, int tri, int tile,
                                 const int* skip_flag) {
+  pdl_enter();
   if (skip_flag != nullptr && *skip_flag != 0) return;
   const i64 total = M * N;
   for (i64 e = (i64)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (i64)gridDim.x * blockDim.x) {
