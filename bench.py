@@ -130,7 +130,7 @@ def case_report(c, ms, rounds, args, peaks, binding):
     the measured bf16 peak and a 3xTF32 product as three TF32 passes."""
     m, n, r = c[:3]
     out = {"m": m, "n": n, "r": r, "ms": ms, "adaptive_orth_rounds": rounds}
-    if ms is None or args.engine == binding.ENGINE_SIMT:
+    if ms is None or args.engine == binding.ENGINE_SIMT or args.lazy:
         return out
     gb = case_gbytes(c)
     fl = phase_flops(m, n, r, args.orth, rounds=rounds)
@@ -324,6 +324,8 @@ def run_ours(args):
     dp_sync = args.sync == "dp"
     if dp_sync and (grouped or args.form != "standard" or args.orth == 4):
         raise SystemExit("--sync dp steps single matrices in the standard form")
+    if args.lazy and (grouped or dp_sync or args.form != "standard" or args.orth == 4):
+        raise SystemExit("--lazy steps single matrices in the standard form")
     for k, c in enumerate(cases):
         m, n, r = c[:3]
         # data-parallel ranks share X and Q (one seed) and see their own gradients (noise seeded per rank below)
@@ -352,6 +354,15 @@ def run_ours(args):
     def one_step(t, per_case_events=None):
         if dp_sync:     # project all, all-reduce P, factor all, all-reduce W, finish all
             steppers[t % 2].step(ETA, stream)
+            return
+        if args.lazy:   # Lazy-Dion: the right factor is refreshed every K-th step only
+            for ci, st in enumerate(state):
+                if per_case_events is not None:
+                    e0 = torch.cuda.Event(enable_timing=True); e0.record(stream)
+                opt.lazy_step_desc(st["descs"][t % 2], ETA, t % args.lazy == 0, sptr)
+                if per_case_events is not None:
+                    e1 = torch.cuda.Event(enable_timing=True); e1.record(stream)
+                    per_case_events[ci].append((e0, e1))
             return
         if grouped:     # one dion_step_grouped call over the whole list
             opt.step_grouped_packed(packed[t % 2], len(state), ETA, sptr)
@@ -435,7 +446,10 @@ def run_ours(args):
         else:
             for k, (st, hd) in enumerate(zip(state, host_d)):
                 stream.wait_event(landed[k])
-                opt.step_desc(st["descs"][0], ETA, sptr)
+                if args.lazy:
+                    opt.lazy_step_desc(st["descs"][0], ETA, False, sptr)
+                else:
+                    opt.step_desc(st["descs"][0], ETA, sptr)
                 ev = torch.cuda.Event(); ev.record(stream)
                 done_ev[k] = ev
                 hd.copy_(st["d"], non_blocking=True)
@@ -477,6 +491,15 @@ def run_ours(args):
         m, n, r = c[:3]
         fl = phase_flops(m, n, r, args.orth, rounds=nr)
         by = phase_bytes(m, n, r, args.orth, gbytes=case_gbytes(c), rounds=nr)
+        if args.lazy:
+            # per step: W = B Q, the M update and the X update (2 m n r each); per refresh two more passes
+            # over B (T = B Q, Z = B^T T) and the orthonormalization of an n x r panel
+            refresh = sum(1 for t in range(args.warmup, args.warmup + args.steps) if t % args.lazy == 0) / args.steps
+            flo = phase_flops(n, m, r, args.orth)
+            fl["R"] = 0.0; by["R"] = 0.0
+            fl["ORTH"] = refresh * (4.0 * m * n * r + flo["ORTH"]); fl["ORTH_GEMM"] = refresh * flo["ORTH_GEMM"]
+            by["ORTH"] = refresh * (2.0 * by["P"] + by["ORTH"]); by["ORTH_GEMM"] = refresh * by["ORTH_GEMM"]
+            fl["COLNORM"] = 3.0 * m * r
         for p in binding.PHASES:
             tot_fl[p] += fl[p]; tot_by[p] += by[p]
     # The dominant kernel is the tcgen05 contraction kernel: the four large products plus the
@@ -560,6 +583,7 @@ def run_ours(args):
                        "orth": ["auto", "cholqr2", "shifted3", "householder", "rcqr"][args.orth],
                        "sync": ("compressed data-parallel sync: P and W all-reduced (mean) over the ranks"
                                 if dp_sync else "none (independent replicas)"),
+                       "rule": ("Lazy-Dion (Algorithm 6), refresh every %d steps" % args.lazy) if args.lazy else "Dion (Algorithm 1 + 2)",
                        "form": args.form, "n_transposed": sum(1 for st in state if st["transposed"]),
                        "l2": "inputs larger than L2: the workload's X, M, G (GBs) cycle through between repeats",
                        "replicas": world, "workspace_bytes": need},
@@ -590,6 +614,9 @@ def main():
     ap.add_argument("--orth", type=int, default=0, help="0 auto, 1 cholqr2, 2 shifted3, 3 householder, 4 randomized Cholesky QR")
     ap.add_argument("--form", default="standard", choices=["standard", "short-side"],
                     help="short-side: matrices with m > n take the transposed form (panel n x r instead of m x r)")
+    ap.add_argument("--lazy", type=int, default=0,
+                    help="K > 0: Lazy-Dion (Algorithm 6): dion_lazy_step with a SymPowerIter1 refresh every K-th step "
+                         "instead of dion_step; single matrices, standard form")
     ap.add_argument("--sync", default="replicas", choices=["replicas", "dp"],
                     help="dp: compressed data-parallel sync (P and W all-reduced over the ranks, same X and Q on "
                          "every rank) instead of independent replicas; standard form, not for the grouped workloads")

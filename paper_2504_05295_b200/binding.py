@@ -240,6 +240,9 @@ class Dion:
         _check(self._lib.dion_dp_finish(self._ctx, ctypes.byref(desc), U.data_ptr(), W.data_ptr(), flag.data_ptr(),
                                         float(lr), _stream_ptr(stream)))
 
+    def lazy_step_desc(self, desc: DionMatrix, lr: float, refresh: bool, stream_ptr: int) -> None:
+        _check(self._lib.dion_lazy_step(self._ctx, ctypes.byref(desc), float(lr), int(bool(refresh)), stream_ptr))
+
     def workspace_bytes(self, m: int, n: int, r: int) -> int:
         return int(self._lib.dion_workspace_bytes(self._ctx, m, n, r))
 

@@ -900,24 +900,63 @@ int lazy_one(dion_ctx* c, const dion_matrix* a, float lr, int refresh, cudaStrea
   float* P0 = s.ws + s.L.P0;
   float* R = s.ws + s.L.R;
   const float* Mp = (const float*)a->M;
-
-  if (refresh) {
-    // T = (M + G) Q  (m x r), Z = (M + G)^T T (n x r), Q <- Orthonormalize(Z)
+  // bf16-operand mode on the tensor engine: as in the Dion step, bf16(M + G) is formed once and the
+  // products read bf16 arrays (B16, and bf16 copies of Q, T / W, ColNorm(W))
+  const bool d16 = s.tensor && c->cfg.precision == DION_PREC_BF16_OPERANDS && m % 8 == 0 && n % 8 == 0 && r % 8 == 0 &&
+                   m >= 128 && n >= 128 && r >= 64 && !((uintptr_t)a->Q & 15) && a->ldq % 4 == 0;
+  auto bf = [&](i64 off) { return reinterpret_cast<__nv_bfloat16*>(s.ws + off); };
+  auto to_bf16 = [&](const float* src, i64 lds, i64 rows, i64 cols, __nv_bfloat16* out) -> int {
+    launch_pdl(k_to_bf16, dim3((unsigned)grid_for(c, rows * cols / 8)), dim3(256), 0, st, src, lds, rows, cols, out, nullptr);
+    DION_CHECK_LAUNCH(c);
+    return DION_OK;
+  };
+  // B Q -> out (m x r): the fused fp32 path, or B16 Q16
+  auto b_times_q = [&](float* out, int precise) -> int {
     GemmArgs t = gemm_args();
     t.M = m; t.N = r; t.K = n;
-    t.A = Mp; t.a_si = a->ldm; t.a_sk = 1;
-    t.A2 = a->G; t.a2_si = a->ldg; t.a2_sk = 1; t.a2_mode = gmode;
-    t.B = (const float*)a->Q; t.b_sk = a->ldq; t.b_sn = 1;
-    t.C = R; t.ldc = r; t.epi = EPI_STORE;
-    t.precise = (resolve_orth(c, r, (m < n) ? m : n) == DION_ORTH_SHIFTED3) ? 1 : 0;
-    DION_TRY(launch_gemm(s, t));
+    if (d16) {
+      DION_TRY(to_bf16((const float*)a->Q, a->ldq, n, r, bf(s.L.Q16)));
+      t.ab16 = 1;
+      t.A = (const float*)bf(s.L.B16); t.a_si = n; t.a_sk = 1;
+      t.B = (const float*)bf(s.L.Q16); t.b_sk = r; t.b_sn = 1;
+    } else {
+      t.A = Mp; t.a_si = a->ldm; t.a_sk = 1;
+      t.A2 = a->G; t.a2_si = a->ldg; t.a2_sk = 1; t.a2_mode = gmode;
+      t.B = (const float*)a->Q; t.b_sk = a->ldq; t.b_sn = 1;
+      t.precise = precise;
+    }
+    t.C = out; t.ldc = r; t.epi = EPI_STORE;
+    return launch_gemm(s, t);
+  };
+  if (d16) {
+    const bool vec = !((uintptr_t)a->M & 15) && a->ldm % 4 == 0 && !((uintptr_t)a->G & 15) &&
+                     a->ldg % ((a->g_dtype == DION_BF16) ? 8 : 4) == 0;
+    const dim3 grid((unsigned)grid_for(c, m * n / 8));
+    if (vec) launch_pdl(k_form_b16<true>, grid, dim3(256), 0, st, Mp, a->ldm, a->G, a->ldg, gmode, m, n, bf(s.L.B16));
+    else launch_pdl(k_form_b16<false>, grid, dim3(256), 0, st, Mp, a->ldm, a->G, a->ldg, gmode, m, n, bf(s.L.B16));
+    DION_CHECK_LAUNCH(c);
+  }
+
+  if (refresh) {
+    // profiling: the whole refresh (SymPowerIter1) is booked as the ORTH phase
+    PhaseScope ps_orth(c, st, DION_PHASE_ORTH);
+    // T = (M + G) Q  (m x r), Z = (M + G)^T T (n x r), Q <- Orthonormalize(Z)
+    const int precise = (resolve_orth(c, r, (m < n) ? m : n) == DION_ORTH_SHIFTED3) ? 1 : 0;
+    DION_TRY(b_times_q(R, precise));
     GemmArgs z = gemm_args();
     z.M = n; z.N = r; z.K = m;
-    z.A = Mp; z.a_si = 1; z.a_sk = a->ldm;
-    z.A2 = a->G; z.a2_si = 1; z.a2_sk = a->ldg; z.a2_mode = gmode;
-    z.B = R; z.b_sk = r; z.b_sn = 1;
+    if (d16) {
+      DION_TRY(to_bf16(R, r, m, r, bf(s.L.U16)));
+      z.ab16 = 1;
+      z.A = (const float*)bf(s.L.B16); z.a_si = 1; z.a_sk = n;
+      z.B = (const float*)bf(s.L.U16); z.b_sk = r; z.b_sn = 1;
+    } else {
+      z.A = Mp; z.a_si = 1; z.a_sk = a->ldm;
+      z.A2 = a->G; z.a2_si = 1; z.a2_sk = a->ldg; z.a2_mode = gmode;
+      z.B = R; z.b_sk = r; z.b_sn = 1;
+      z.precise = precise;
+    }
     z.C = P0; z.ldc = r; z.epi = EPI_STORE;
-    z.precise = t.precise;
     DION_TRY(launch_gemm(s, z));
     i64 V_off = 0;
     s.in_orth = true;
@@ -925,9 +964,7 @@ int lazy_one(dion_ctx* c, const dion_matrix* a, float lr, int refresh, cudaStrea
     s.in_orth = false;
     DION_TRY(rc_orth);
     const float* V = s.ws + V_off;
-    // copy V into Q unless the round broke down (alpha = 1, identity product is overkill: strided copy kernel)
-    GemmArgs cp = gemm_args();
-    (void)cp;
+    // copy V into Q unless the round broke down
     const i64 total = n * r;
     int blocks = (int)((total + 255) / 256);
     if (blocks > 8 * c->sm_count) blocks = 8 * c->sm_count;
@@ -935,30 +972,48 @@ int lazy_one(dion_ctx* c, const dion_matrix* a, float lr, int refresh, cudaStrea
     DION_CHECK_LAUNCH(c);
   }
   // W = (M + G) Q
-  GemmArgs w = gemm_args();
-  w.M = m; w.N = r; w.K = n;
-  w.A = Mp; w.a_si = a->ldm; w.a_sk = 1;
-  w.A2 = a->G; w.a2_si = a->ldg; w.a2_sk = 1; w.a2_mode = gmode;
-  w.B = (const float*)a->Q; w.b_sk = a->ldq; w.b_sn = 1;
-  w.C = R; w.ldc = r; w.epi = EPI_STORE;
-  DION_TRY(launch_gemm(s, w));
+  {
+  PhaseScope ps(c, st, DION_PHASE_P);
+  DION_TRY(b_times_q(R, 0));
+  }
   // M <- (M + G) - (1 - mu) W Q^T
+  {
+  PhaseScope ps(c, st, DION_PHASE_EF);
   GemmArgs e = gemm_args();
   e.M = m; e.N = n; e.K = r;
-  e.A = R; e.a_si = r; e.a_sk = 1;
-  e.B = (const float*)a->Q; e.b_sk = 1; e.b_sn = a->ldq;
+  if (d16) {   // Q16 was written by b_times_q just above
+    DION_TRY(to_bf16(R, r, m, r, bf(s.L.U16)));
+    e.ab16 = 1;
+    e.A = (const float*)bf(s.L.U16); e.a_si = r; e.a_sk = 1;
+    e.B = (const float*)bf(s.L.Q16); e.b_sk = 1; e.b_sn = r;
+  } else {
+    e.A = R; e.a_si = r; e.a_sk = 1;
+    e.B = (const float*)a->Q; e.b_sk = 1; e.b_sn = a->ldq;
+  }
   e.C = (float*)a->M; e.ldc = a->ldm; e.epi = EPI_ADD2_SUB;
   e.C2 = a->G; e.ldc2 = a->ldg; e.c2_mode = gmode;
   e.alpha = 1.f - c->cfg.mu;
   e.skip_flag = s.flag;
   DION_TRY(launch_gemm(s, e));
+  }
   // U = ColNorm(W)
+  {
+  PhaseScope ps(c, st, DION_PHASE_COLNORM);
   DION_TRY(colnorm(s, 0, R, m, r, P0, r, a->colnorm_out));
+  }
   // X <- X - lr sqrt(m/n) U Q^T
+  PhaseScope ps_x(c, st, DION_PHASE_X);
   GemmArgs x = gemm_args();
   x.M = m; x.N = n; x.K = r;
-  x.A = P0; x.a_si = r; x.a_sk = 1;
-  x.B = (const float*)a->Q; x.b_sk = 1; x.b_sn = a->ldq;
+  if (d16) {
+    DION_TRY(to_bf16(P0, r, m, r, bf(s.L.R16)));
+    x.ab16 = 1;
+    x.A = (const float*)bf(s.L.R16); x.a_si = r; x.a_sk = 1;
+    x.B = (const float*)bf(s.L.Q16); x.b_sk = 1; x.b_sn = r;
+  } else {
+    x.A = P0; x.a_si = r; x.a_sk = 1;
+    x.B = (const float*)a->Q; x.b_sk = 1; x.b_sn = a->ldq;
+  }
   x.C = (float*)a->X; x.ldc = a->ldx; x.epi = EPI_SUB;
   x.alpha = lr * sqrtf((float)((double)m / (double)n));
   x.skip_flag = s.flag;

@@ -303,22 +303,25 @@ def test_argument_errors():
         assert opt.get_status() == (0, 0)
 
 
-@pytest.mark.parametrize("m,n,r", [(384, 256, 32), (1536, 1024, 128)])
-def test_lazy_dion_steps_match_oracle(m, n, r):
+@pytest.mark.parametrize("m,n,r,precision", [(384, 256, 32, binding.PREC_FP32), (1536, 1024, 128, binding.PREC_FP32),
+                                             (1536, 1024, 128, binding.PREC_BF16_OPERANDS),
+                                             (1000, 776, 100, binding.PREC_BF16_OPERANDS)])
+def test_lazy_dion_steps_match_oracle(m, n, r, precision):
     from oracle import dion_oracle as orc
     pb = inputs.make_problem(m, n, r, seed=14, ks=8)
     X, M, Q = device_state(pb)
     Xo, Mo, Qo = to_np64(pb.X), to_np64(pb.M), to_np64(pb.Q)
     d = torch.zeros(r, device="cuda")
-    with binding.Dion(mu=MU, eps=EPS) as opt:
+    tol = TOL_FP32 if precision == binding.PREC_FP32 else TOL_BF16
+    with binding.Dion(mu=MU, eps=EPS, precision=precision) as opt:
         for t in range(6):
             refresh = (t % 3 == 0)
             G = pb.grad(t)
             opt.lazy_step(X, M, G.cuda(), Q, ETA, refresh, colnorm_out=d)
             Xo, Mo, Qo, do = orc.lazy_step(Xo, Mo, to_np64(G), Qo, MU, ETA, EPS, refresh=refresh)
         assert opt.get_status() == (0, 0)
-    assert rel(to_np64(X), Xo) <= TOL_FP32 and rel(to_np64(M), Mo) <= TOL_FP32
-    assert rel(to_np64(Q), Qo) <= TOL_FP32 and rel(to_np64(d), do) <= TOL_FP32
+    assert rel(to_np64(X), Xo) <= tol and rel(to_np64(M), Mo) <= tol
+    assert rel(to_np64(Q), Qo) <= tol and rel(to_np64(d), do) <= tol
 
 
 # ---------------------------------------------------------------------------
