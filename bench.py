@@ -99,6 +99,12 @@ def phase_flops(m, n, r, orth, rounds=None):
         g = 2.0 * m * n * r
         og = 3.5 * m * r * r + r ** 3 / 3.0 + (2.0 * m * r * r + 2.0 / 3.0 * r ** 3)
         return {"P": g, "ORTH": o, "R": g, "EF": g, "COLNORM": 3.0 * n * r, "X": g, "ORTH_GEMM": og}
+    if rounds == 1 and orth_mode(m, n, r, orth) == 1:
+        # CholeskyQR2 whose second round was skipped on the device: one round plus the Gram matrix of the check
+        o = 3.0 * m * r * r + r ** 3 / 3.0
+        g = 2.0 * m * n * r
+        og = 3.0 * m * r * r + 2.0 / 3.0 * r ** 3
+        return {"P": g, "ORTH": o, "R": g, "EF": g, "COLNORM": 3.0 * n * r, "X": g, "ORTH_GEMM": og}
     if rounds:
         o = rounds * (2.0 * m * r * r + r ** 3 / 3.0)     # Gram (symmetric half) + Cholesky + solve
     else:
@@ -472,7 +478,7 @@ def run_ours(args):
     case_rounds = []
     for ci, st in enumerate(state):
         m_, n_, r_ = cases[ci][:3]
-        if orth_mode(m_, n_, r_, args.orth) != 2:
+        if orth_mode(m_, n_, r_, args.orth) not in (1, 2):
             case_rounds.append(None)
             continue
         opt.step_desc(st["descs"][1], ETA, sptr)

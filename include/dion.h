@@ -67,6 +67,9 @@ typedef enum { DION_PREC_FP32 = 0, DION_PREC_BF16_OPERANDS = 1 } dion_precision;
  * DION_ORTH_AUTO:        CholeskyQR2 when 4 r <= min(m, n), else the adaptive rounds.
  * DION_ORTH_CHOLQR2:     two rounds of Cholesky QR (cond(P) up to about 4e3); a
  *                        non-positive pivot cancels the step (DION_STATUS_BREAKDOWN).
+ *                        The Gram matrix of the second round doubles as a measurement of
+ *                        the first: if max |U1^T U1 - I| <= 1e-5 the rest of the second
+ *                        round is skipped on the device (well-conditioned panels).
  * DION_ORTH_SHIFTED3:    adaptive Cholesky QR rounds for ill-conditioned panels such as
  *                        full rank: a column whose pivot falls below 1e-4 of its
  *                        squared norm is deflated, so a round cannot break down and
@@ -240,9 +243,10 @@ enum {
 int dion_profile_enable(dion_ctx* ctx, int on);
 int dion_profile_read(dion_ctx* ctx, float* ms, int64_t* launches);
 
-/* Synchronises `cuda_stream`, then reports and clears the number of adaptive
- * Cholesky QR rounds (DION_ORTH_SHIFTED3 / AUTO above rank fraction 1/4) that did
- * work since the last call; rounds skipped on the device are not counted. */
+/* Synchronises `cuda_stream`, then reports and clears the number of Cholesky QR
+ * rounds (the adaptive rounds of DION_ORTH_SHIFTED3, the one or two rounds of
+ * DION_ORTH_CHOLQR2) that did work since the last call; rounds skipped on the
+ * device are not counted. */
 int dion_get_orth_rounds(dion_ctx* ctx, void* cuda_stream, int64_t* rounds);
 
 /* Number of kernel launches issued by this context so far (host counter). */

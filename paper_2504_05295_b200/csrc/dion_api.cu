@@ -25,6 +25,7 @@ constexpr size_t GROUP_SCRATCH_BYTES = (size_t)16 << 30;  // scratch dion_step_g
 constexpr int MAX_ROUNDS = 6;             // adaptive Cholesky QR rounds
 constexpr float FLOOR_REL = 1e-4f;        // pivot floor relative to the column's squared norm
 constexpr float GOOD_REL = 1e-4f;         // smallest relative pivot of a round that one more round can finish
+constexpr float ORTH_TAU = 1e-5f;         // CholeskyQR2: max |U1^T U1 - I| below which the second round is skipped
 constexpr float DONE_REL = 0.9f;          // smallest relative pivot of a round whose input was already orthonormal
 constexpr i64 PART_CAP_FLOATS = (i64)16 << 20;  // split-K partial sums, at most 64 MiB
 
@@ -345,7 +346,19 @@ int trtri_levels(StepCtx& s, i64 r, i64 o, i64 sz, i64 b_from, const int* skip, 
 
 // Cholesky of the diagonal square [o, o+sz) of each Gram matrix (sz <= NBO), right-looking with
 // 64-wide blocks on the FMA engine, followed by the inverse of that square's factor into Linv.
-int potrf_inner(StepCtx& s, i64 r, i64 o, i64 sz, bool adaptive) {
+// How a Cholesky-QR round runs.
+enum : int {
+  RM_PLAIN = 0,     // no device-side control
+  RM_ADAPTIVE = 1,  // deflating pivots, skipped once the panel is done, split-accumulator products, round statistics
+  RM_FIRST = 2,     // first round of CholeskyQR2: plain control, split-accumulator products
+  RM_CHECKED = 3    // second round of CholeskyQR2: the Gram matrix is always formed; if it is the identity to
+                    // ORTH_TAU the rest of the round is skipped (Pout = Pin)
+};
+inline bool rm_skips(int mode) { return mode == RM_ADAPTIVE || mode == RM_CHECKED; }
+inline bool rm_precise(int mode) { return mode == RM_ADAPTIVE || mode == RM_FIRST; }
+
+int potrf_inner(StepCtx& s, i64 r, i64 o, i64 sz, int mode) {
+  const bool adaptive = rm_skips(mode);
   dion_ctx* c = s.c;
   float* Gm = s.ws + s.L.Gram;
   float* Dinv = s.ws + s.L.Dinv;
@@ -355,7 +368,7 @@ int potrf_inner(StepCtx& s, i64 r, i64 o, i64 sz, bool adaptive) {
   const float* gdiag = s.ws + s.L.gdiag;
   int* status = c->dev_ints;
   const int* skip = adaptive ? (s.os + OS_DONE) : nullptr;
-  const float floor_rel = adaptive ? FLOOR_REL : 0.f;
+  const float floor_rel = (mode == RM_ADAPTIVE) ? FLOOR_REL : 0.f;
   const int nblk = (int)((sz + NB - 1) / NB);
   {
     const int jb = (int)((sz < NB) ? sz : NB);
@@ -388,14 +401,15 @@ int potrf_inner(StepCtx& s, i64 r, i64 o, i64 sz, bool adaptive) {
 // factor into Linv.  Outer blocks of 512 columns: the diagonal square is factored and
 // inverted by potrf_inner, the panel below it is multiplied by that inverse and the
 // trailing matrix is updated with one rank-512 product (tensor cores where it qualifies).
-int potrf_trtri(StepCtx& s, i64 r, bool adaptive, bool full_inverse,
+int potrf_trtri(StepCtx& s, i64 r, int mode, bool full_inverse,
                 const std::function<int(i64, i64)>* after_block = nullptr) {
+  const bool adaptive = rm_skips(mode);
   dion_ctx* c = s.c;
   float* Gm = s.ws + s.L.Gram;
   float* Linv = s.ws + s.L.Linv;
   float* Tbuf = s.ws + s.L.Tbuf;
   const int* skip = adaptive ? (s.os + OS_DONE) : nullptr;
-  const int precise = adaptive ? 1 : 0;
+  const int precise = rm_precise(mode) ? 1 : 0;
   if (r > NBO && full_inverse) {
     // everything outside the diagonal squares starts at zero (the product U = P Linv^T reads whole tiles)
     for (int m = 0; m < s.nb; ++m)
@@ -403,7 +417,7 @@ int potrf_trtri(StepCtx& s, i64 r, bool adaptive, bool full_inverse,
   }
   for (i64 J0 = 0; J0 < r; J0 += NBO) {
     const i64 sz = (r - J0 < NBO) ? (r - J0) : NBO;
-    DION_TRY(potrf_inner(s, r, J0, sz, adaptive));
+    DION_TRY(potrf_inner(s, r, J0, sz, mode));
     if (after_block != nullptr) DION_TRY((*after_block)(J0, sz));   // block column J of the factor and its inverse are final
     const i64 rem = r - J0 - sz;
     if (rem > 0) {
@@ -437,14 +451,16 @@ int potrf_trtri(StepCtx& s, i64 r, bool adaptive, bool full_inverse,
 // rows x r panels, ld = r; pin_off / pout_off are offsets in the scratch slice.
 // adaptive: columns with negligible pivots are deflated, the round is skipped (Pout = Pin)
 // once the panel is orthonormal, and the round statistics are evaluated at the end.
-int cholqr_round(StepCtx& s, i64 pin_off, i64 pout_off, i64 rows, i64 r, bool adaptive) {
+int cholqr_round(StepCtx& s, i64 pin_off, i64 pout_off, i64 rows, i64 r, int mode) {
   dion_ctx* c = s.c;
-  const int* skip = adaptive ? (s.os + OS_DONE) : nullptr;
+  const bool adaptive = (mode == RM_ADAPTIVE);
+  const bool skips = rm_skips(mode);
+  const int* skip = skips ? (s.os + OS_DONE) : nullptr;
   GemmArgs g = gemm_args();
   g.M = r; g.N = r; g.K = rows;
   g.A = s.ws + pin_off; g.a_si = 1; g.a_sk = r;
   g.B = s.ws + pin_off; g.b_sk = r; g.b_sn = 1;
-  g.C = s.ws + s.L.Gram; g.ldc = r; g.epi = EPI_STORE; g.tri = TRI_LOWER; g.skip_flag = skip; g.precise = adaptive ? 1 : 0;
+  g.C = s.ws + s.L.Gram; g.ldc = r; g.epi = EPI_STORE; g.tri = TRI_LOWER; g.skip_flag = adaptive ? skip : nullptr; g.precise = rm_precise(mode) ? 1 : 0;
   for (int m = 0; m < s.nb; ++m) DION_TRY(launch_gemm(s, for_matrix(s, g, m, true, true, true), m));
   launch_pdl(k_round_begin, dim3((unsigned)(s.nb)), dim3(256), 0, s.st, s.ws + s.L.Gram, r, r, 0.f, s.ws + s.L.gdiag, s.ws + s.L.scal, s.os,
                                         adaptive ? 1 : 0, s.wstride);
@@ -454,7 +470,15 @@ int cholqr_round(StepCtx& s, i64 pin_off, i64 pout_off, i64 rows, i64 r, bool ad
   // alone, 512-column products need >= 128 row tiles to fill the GPU; beside the factorization
   // (second stream) they are background work at any height
   const bool trsm = (r > NBO) && (rows >= 8192 || c->side != nullptr);
-  if (adaptive) {   // a finished panel is passed through (before anything writes Pout)
+  if (mode == RM_CHECKED) {
+    // CholeskyQR2, second round: measure the first round's result; orthonormal to ORTH_TAU -> done
+    dim3 grid((unsigned)grid_for(c, r * r), (unsigned)s.nb);
+    launch_pdl(k_orth_check, grid, dim3(256), 0, s.st, (const float*)(s.ws + s.L.Gram), r, r, s.os, s.wstride);
+    DION_CHECK_LAUNCH(c);
+    launch_pdl(k_orth_decide, dim3((unsigned)s.nb), dim3(1), 0, s.st, s.os, ORTH_TAU, c->dev_ints + 2);
+    DION_CHECK_LAUNCH(c);
+  }
+  if (skips) {   // a finished panel is passed through (before anything writes Pout)
     dim3 grid((unsigned)grid_for(c, rows * r), (unsigned)s.nb);
     launch_pdl(k_copy_panel, grid, dim3(256), 0, s.st, s.ws + pin_off, r, s.ws + pout_off, r, rows, r, nullptr, s.os + OS_DONE, s.wstride);
     DION_CHECK_LAUNCH(c);
@@ -504,11 +528,11 @@ int cholqr_round(StepCtx& s, i64 pin_off, i64 pout_off, i64 rows, i64 r, bool ad
         s.st = main_st; s.no_split = false;
         return rc;
       };
-      DION_TRY(potrf_trtri(s, r, adaptive, false, &after_block));
+      DION_TRY(potrf_trtri(s, r, mode, false, &after_block));
       cudaEvent_t e = next_event();   // join: the round ends when the last solve has finished
       if (cudaEventRecord(e, c->side) != cudaSuccess || cudaStreamWaitEvent(main_st, e, 0) != cudaSuccess) return DION_ERR_CUDA;
     } else {
-      DION_TRY(potrf_trtri(s, r, adaptive, false));
+      DION_TRY(potrf_trtri(s, r, mode, false));
       for (i64 J0 = 0; J0 < r; J0 += NBO) DION_TRY(solve_block(J0, (r - J0 < NBO) ? (r - J0) : NBO));
     }
     if (adaptive) {
@@ -517,7 +541,7 @@ int cholqr_round(StepCtx& s, i64 pin_off, i64 pout_off, i64 rows, i64 r, bool ad
     }
     return DION_OK;
   }
-  DION_TRY(potrf_trtri(s, r, adaptive, true));
+  DION_TRY(potrf_trtri(s, r, mode, true));
   GemmArgs u = gemm_args();
   u.M = rows; u.N = r; u.K = r;
   u.A = s.ws + pin_off; u.a_si = r; u.a_sk = 1;
@@ -616,7 +640,7 @@ int rcqr(StepCtx& s, i64 rows, i64 r) {
   u.B = s.ws + s.L.Linv; u.b_sk = 1; u.b_sn = r; u.klimit = 1;
   u.C = s.ws + s.L.P1; u.ldc = r; u.epi = EPI_STORE; u.precise = 1;
   for (int m = 0; m < s.nb; ++m) DION_TRY(launch_gemm(s, for_matrix(s, u, m, true, true, true), m));
-  return cholqr_round(s, s.L.P1, s.L.P0, rows, r, false);
+  return cholqr_round(s, s.L.P1, s.L.P0, rows, r, RM_PLAIN);
 }
 
 // The orthonormalization a step on (m, n, r) will use.
@@ -633,15 +657,17 @@ int orthonormalize(StepCtx& s, i64 rows, i64 r, i64 short_dim, i64* U_off) {
   if (mode == DION_ORTH_RCQR && s.list == nullptr)   // no sketches on this path (Lazy-Dion): as AUTO
     mode = (4 * r <= short_dim) ? DION_ORTH_CHOLQR2 : DION_ORTH_SHIFTED3;
   if (mode == DION_ORTH_CHOLQR2) {
-    DION_TRY(cholqr_round(s, s.L.P0, s.L.P1, rows, r, false));
-    DION_TRY(cholqr_round(s, s.L.P1, s.L.P0, rows, r, false));
+    // the first round with the accurate products; the second one only if the first one's result is
+    // not yet orthonormal to ORTH_TAU (measured on its Gram matrix)
+    DION_TRY(cholqr_round(s, s.L.P0, s.L.P1, rows, r, RM_FIRST));
+    DION_TRY(cholqr_round(s, s.L.P1, s.L.P0, rows, r, RM_CHECKED));
     *U_off = s.L.P0;
   } else if (mode == DION_ORTH_SHIFTED3) {
     // Adaptive rounds: the device decides after each round whether the panel is done.
     static_assert(MAX_ROUNDS % 2 == 0, "the result must end in P0");
     for (int it = 0; it < MAX_ROUNDS; it += 2) {
-      DION_TRY(cholqr_round(s, s.L.P0, s.L.P1, rows, r, true));
-      DION_TRY(cholqr_round(s, s.L.P1, s.L.P0, rows, r, true));
+      DION_TRY(cholqr_round(s, s.L.P0, s.L.P1, rows, r, RM_ADAPTIVE));
+      DION_TRY(cholqr_round(s, s.L.P1, s.L.P0, rows, r, RM_ADAPTIVE));
     }
     launch_pdl(k_orth_finish, dim3((unsigned)(s.nb)), dim3(1), 0, s.st, s.os, s.c->dev_ints);
     s.c->launches++;

@@ -15,6 +15,7 @@ enum : int {
   OS_FLOORED = 3,   // pivots raised to the floor in the current round
   OS_MINREL = 4,    // float bits: min over columns of pivot / original diagonal, current round
   OS_ROUNDS = 5,    // rounds that did work
+  OS_MAXDEV = 6,    // float bits: max |G - I| over the lower triangle of a round's Gram matrix (CholeskyQR2 check)
   OS_SLOT_INTS = 8
 };
 
@@ -480,6 +481,46 @@ __global__ void k_round_end(int* __restrict__ os, float good_rel, float done_rel
     if (minrel >= done_rel) os[OS_DONE] = 1;
     else if (minrel >= good_rel) os[OS_GOOD] = 1;
   }
+}
+
+// CholeskyQR2, second round: max |G[i][j] - delta_ij| over the lower triangle of the Gram matrix of
+// the first round's result, into os[OS_MAXDEV] (zero at the start of a step).  grid = (blocks, matrices).
+__global__ void __launch_bounds__(256) k_orth_check(const float* __restrict__ G, i64 ld, i64 r, int* __restrict__ os,
+                                                    i64 wstride) {
+  pdl_enter();
+  G += (i64)blockIdx.y * wstride;
+  os += (i64)blockIdx.y * OS_SLOT_INTS;
+  __shared__ float red[256];
+  const float inf = __int_as_float(0x7f800000);
+  float mx = 0.f;
+  const i64 total = r * r;
+  for (i64 e = (i64)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (i64)gridDim.x * blockDim.x) {
+    const i64 i = e / r, j = e % r;
+    if (j <= i) {
+      float dev = fabsf(G[i * ld + j] - ((i == j) ? 1.f : 0.f));
+      if (!(dev == dev)) dev = inf;            // NaN
+      mx = fmaxf(mx, dev);
+    }
+  }
+  red[threadIdx.x] = mx;
+  __syncthreads();
+  for (int w = 128; w > 0; w >>= 1) {
+    if ((int)threadIdx.x < w) red[threadIdx.x] = fmaxf(red[threadIdx.x], red[threadIdx.x + w]);
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) atomicMax(&os[OS_MAXDEV], __float_as_int(red[0]));   // non-negative floats order like ints
+}
+
+// ... and the decision: orthonormal to tau -> the rest of the round is skipped.  Counts the rounds
+// of the step that did work (1 or 2).
+__global__ void k_orth_decide(int* __restrict__ os, float tau, int* __restrict__ rounds_total) {
+  pdl_enter();
+  os += (i64)blockIdx.x * OS_SLOT_INTS;
+  const float maxdev = __int_as_float(os[OS_MAXDEV]);
+  const bool done = (os[OS_FAIL] == 0) && (maxdev <= tau);
+  os[OS_DONE] = done ? 1 : 0;
+  os[OS_ROUNDS] = done ? 1 : 2;
+  atomicAdd(rounds_total, done ? 1 : 2);
 }
 
 // After the last adaptive round: a panel that never became well conditioned is
