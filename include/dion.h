@@ -68,7 +68,7 @@ typedef enum { DION_PREC_FP32 = 0, DION_PREC_BF16_OPERANDS = 1 } dion_precision;
  * DION_ORTH_CHOLQR2:     two rounds of Cholesky QR (cond(P) up to about 4e3); a
  *                        non-positive pivot cancels the step (DION_STATUS_BREAKDOWN).
  *                        The Gram matrix of the second round doubles as a measurement of
- *                        the first: if max |U1^T U1 - I| <= 1e-5 the rest of the second
+ *                        the first: if max |U1^T U1 - I| <= 3e-5 the rest of the second
  *                        round is skipped on the device (well-conditioned panels).
  * DION_ORTH_SHIFTED3:    adaptive Cholesky QR rounds for ill-conditioned panels such as
  *                        full rank: a column whose pivot falls below 1e-4 of its
