@@ -225,6 +225,32 @@ def test_repeated_runs_are_bit_identical(m, n, r, precision):
         assert opt.get_status() == (0, 0)
 
 
+def test_cholqr2_takes_its_second_round_only_when_the_first_is_not_enough():
+    m, n, r = 1024, 768, 128
+    pb = inputs.make_problem(m, n, r, seed=15, ks=16)
+    G = pb.grad(0)
+    # (i) the workload's own warm start: cond(P) of a few units -> one round passes the device's check
+    X, M, Q = device_state(pb)
+    with binding.Dion(mu=MU, eps=EPS, orth=binding.ORTH_CHOLQR2) as opt:
+        opt.step(X, M, G.cuda(), Q, ETA)
+        assert opt.get_status() == (0, 0) and opt.orth_rounds() == 1
+    ref = oracle_steps(pb, 1)[0]
+    assert rel(to_np64(Q), ref.Q) <= TOL_FP32 and rel(to_np64(M), ref.M) <= TOL_FP32 and rel(to_np64(X), ref.X) <= TOL_FP32
+    # (ii) a warm start whose columns are nearly parallel (every column = the first one + 3 % of its own:
+    # cond(P) in the hundreds, not curable by column scaling): the first round's result fails the check,
+    # the second round runs, and the outputs still meet the bar
+    Qbad = pb.Q[:, :1] + 0.03 * pb.Q
+    Qbad = Qbad / Qbad.norm(dim=0)
+    from oracle import dion_oracle as orc
+    want = orc.step(to_np64(pb.X), to_np64(pb.M), to_np64(G), to_np64(Qbad), MU, ETA, EPS)
+    X, M, Q = pb.X.cuda().clone(), pb.M.cuda().clone(), Qbad.cuda().clone()
+    with binding.Dion(mu=MU, eps=EPS, orth=binding.ORTH_CHOLQR2) as opt:
+        opt.step(X, M, G.cuda(), Q, ETA)
+        assert opt.get_status() == (0, 0) and opt.orth_rounds() == 2
+    assert rel(to_np64(M), want.M) <= TOL_FP32 and rel(to_np64(X), want.X) <= TOL_FP32
+    assert rel(to_np64(Q), want.Q) <= 10 * TOL_FP32     # Q inherits cond(P) times the rounding of P
+
+
 def test_checkpoint_resume_is_bit_identical():
     m, n, r, ks = inputs.config1()
     pb = inputs.make_problem(m, n, r, seed=0, ks=ks)
