@@ -93,12 +93,14 @@ def phase_flops(m, n, r, orth, rounds=None):
     if rounds is None:
         rounds = {1: 2, 2: 4}.get(orth_mode(m, n, r, orth), 0)
     if orth == 4:
-        # randomized Cholesky QR (the paper's cost table): sketch 2.5 m r^2, QR of the sketch 11/6 r^3,
-        # triangular solve m r^2, then one Cholesky-QR round
-        o = 2.5 * m * r * r + 11.0 / 6.0 * r ** 3 + m * r * r + (2.0 * m * r * r + r ** 3 / 3.0)
+        # randomized Cholesky QR: sketch product 2.5 m r^2, ~2 rounds on the stacked panel [S P; P] (Gram matrix
+        # from the 1.25 r sketch rows, factor, solve over 1.25 r + m rows), then one Cholesky-QR round on B
+        # plus the Gram matrix of its check
+        k = 1.25 * r
+        rnd = 2.0 * (k * r * r + r ** 3 / 3.0 + (k + m) * r * r)
+        o = 2.5 * m * r * r + rnd + 3.0 * m * r * r + r ** 3 / 3.0
         g = 2.0 * m * n * r
-        og = 3.5 * m * r * r + r ** 3 / 3.0 + (2.0 * m * r * r + 2.0 / 3.0 * r ** 3)
-        return {"P": g, "ORTH": o, "R": g, "EF": g, "COLNORM": 3.0 * n * r, "X": g, "ORTH_GEMM": og}
+        return {"P": g, "ORTH": o, "R": g, "EF": g, "COLNORM": 3.0 * n * r, "X": g, "ORTH_GEMM": o}
     if rounds == 1 and orth_mode(m, n, r, orth) == 1:
         # CholeskyQR2 whose second round was skipped on the device: one round plus the Gram matrix of the check
         o = 3.0 * m * r * r + r ** 3 / 3.0

@@ -79,11 +79,12 @@ typedef enum { DION_PREC_FP32 = 0, DION_PREC_BF16_OPERANDS = 1 } dion_precision;
  * DION_ORTH_HOUSEHOLDER: Householder QR (slow, most robust).
  * DION_ORTH_RCQR:        randomized Cholesky QR, the paper's Distributed-Orthonormalize
  *                        (Algorithm 4) on one device: with the caller's sketching matrix S
- *                        (dion_matrix.sketch), R1 = triangular factor of QR(S P) (Householder,
- *                        on the small sketch), B = P R1^-1, R2 = Cholesky(B^T B),
- *                        U = B R2^-1.  Handles ill-conditioned panels with one Gram matrix;
- *                        the unblocked Householder factorization of the sketch makes it slow
- *                        for large r.  dion_lazy_step treats it as DION_ORTH_AUTO.           */
+ *                        (dion_matrix.sketch), R1 = triangular factor of QR(S P), B = P R1^-1,
+ *                        R2 = Cholesky(B^T B), U = B R2^-1.  The QR of the small sketch is done
+ *                        by the deflating Cholesky QR rounds (R1 is never formed: each round's
+ *                        triangular factor is applied to the sketch and to P at once), so the
+ *                        Gram matrices of an ill-conditioned panel are taken from the sketch
+ *                        rows only.  dion_lazy_step treats it as DION_ORTH_AUTO.           */
 typedef enum {
   DION_ORTH_AUTO = 0,
   DION_ORTH_CHOLQR2 = 1,

@@ -33,11 +33,13 @@ constexpr float ORTH_TAU = 3e-5f;
 constexpr float DONE_REL = 0.9f;          // smallest relative pivot of a round whose input was already orthonormal
 constexpr i64 PART_CAP_FLOATS = (i64)16 << 20;  // split-K partial sums, at most 64 MiB
 
+constexpr i64 NBO_COLS = 512;  // = NBO, the outer block of the two-level Cholesky (defined below)
+
 inline i64 align64(i64 floats) { return (floats + 63) / 64 * 64; }  // 256-byte granules
 
 struct Layout {
   i64 P0, P1, R, Gram, Linv, Tbuf, Dinv, DinvP, part, cn_part, d, gdiag, scal, total;
-  i64 Sk, SkV;              // randomized Cholesky QR: the sketch S P and its Householder vectors (2r x r each)
+  i64 Sk, SkV, SkW;         // randomized Cholesky QR: the two stacked panels [S P; P] and a solve temporary
   i64 B16, Q16, U16, R16;   // bf16-operand mode: bf16(M + G) and the bf16 copies of Q, U, R (offsets in floats)
   i64 part_floats;
   int cn_chunks;
@@ -101,9 +103,13 @@ Layout make_layout(const dion_ctx* c, i64 m, i64 n, i64 r) {
   L.gdiag = o; o += align64(r);
   L.scal = o; o += 64;
   L.Sk = L.SkV = 0;
+  L.SkW = 0;
   if (c->cfg.orth == DION_ORTH_RCQR) {
-    L.Sk = o; o += align64(2 * r * r);
-    L.SkV = o; o += align64(2 * r * r);
+    // two (sketch rows + panel rows) x r buffers for the rounds on the stacked panel [S P; P], and the
+    // 512-column temporary of their blocked solves
+    L.Sk = o; o += align64((2 * r + big) * r);
+    L.SkV = o; o += align64((2 * r + big) * r);
+    L.SkW = o; o += align64((2 * r + big) * NBO_COLS);
   }
   L.B16 = L.Q16 = L.U16 = L.R16 = 0;
   if (c->cfg.precision == DION_PREC_BF16_OPERANDS) {
@@ -241,6 +247,7 @@ struct StepCtx {
   bool tensor;  // tensor-core engine allowed for this matrix
   bool in_orth; // inside the orthonormalization (for the profiling phases)
   const dion_matrix* const* list = nullptr;   // the matrices of the chain (sketch pointers of the RCQR mode)
+  i64 wt_off = -1;        // >= 0: scratch offset of the blocked solves' rows x 512 temporary (default: the R panel)
   bool no_split = false;  // launches on the side stream: the split-K scratch belongs to the main stream
   float* W(int b, i64 off) const { return ws + (i64)b * wstride + off; }
   int* OS(int b) const { return os + (i64)b * OS_SLOT_INTS; }
@@ -284,7 +291,7 @@ int configure_kernels() {
   return DION_OK;
 }
 
-constexpr i64 NBO = 512;  // outer block of the two-level Cholesky
+constexpr i64 NBO = NBO_COLS;  // outer block of the two-level Cholesky
 
 int grid_for(const dion_ctx* c, i64 total) {
   i64 blocks = (total + 255) / 256;
@@ -455,13 +462,15 @@ int potrf_trtri(StepCtx& s, i64 r, int mode, bool full_inverse,
 // rows x r panels, ld = r; pin_off / pout_off are offsets in the scratch slice.
 // adaptive: columns with negligible pivots are deflated, the round is skipped (Pout = Pin)
 // once the panel is orthonormal, and the round statistics are evaluated at the end.
-int cholqr_round(StepCtx& s, i64 pin_off, i64 pout_off, i64 rows, i64 r, int mode) {
+int cholqr_round(StepCtx& s, i64 pin_off, i64 pout_off, i64 rows, i64 r, int mode, i64 gram_rows = 0) {
+  // gram_rows > 0: the Gram matrix is formed from the first gram_rows rows only (a sketch stacked on
+  // top of the panel); the factor is applied to all rows
   dion_ctx* c = s.c;
   const bool adaptive = (mode == RM_ADAPTIVE);
   const bool skips = rm_skips(mode);
   const int* skip = skips ? (s.os + OS_DONE) : nullptr;
   GemmArgs g = gemm_args();
-  g.M = r; g.N = r; g.K = rows;
+  g.M = r; g.N = r; g.K = gram_rows > 0 ? gram_rows : rows;
   g.A = s.ws + pin_off; g.a_si = 1; g.a_sk = r;
   g.B = s.ws + pin_off; g.b_sk = r; g.b_sn = 1;
   g.C = s.ws + s.L.Gram; g.ldc = r; g.epi = EPI_STORE; g.tri = TRI_LOWER; g.skip_flag = adaptive ? skip : nullptr; g.precise = rm_precise(mode) ? 1 : 0;
@@ -495,7 +504,7 @@ int cholqr_round(StepCtx& s, i64 pin_off, i64 pout_off, i64 rows, i64 r, int mod
     // final once the factorization has passed J: the solves run on a second stream beside the rest
     // of the factorization, whose serial 64-column chain leaves most SMs idle.
     const float* Lm = s.ws + s.L.Gram;     // the factor, lower
-    float* Wt = s.ws + s.L.R;              // rows x 512 temporary (R is free during the orthonormalization)
+    float* Wt = s.ws + (s.wt_off >= 0 ? s.wt_off : s.L.R);   // rows x 512 temporary (R is free during the orthonormalization)
     auto solve_block = [&](i64 J0, i64 sz) -> int {
       const float* rhs = s.ws + pin_off + J0;
       i64 rhs_ld = r;
@@ -598,53 +607,55 @@ int householder(StepCtx& s, float* A, float* V, i64 rows, i64 r, int b) {
   return DION_OK;
 }
 
+// Adaptive rounds on the panel at off_a (ping-pong with off_b; the result ends at off_a): the device
+// decides after each round whether the panel is done.
+int adaptive_rounds(StepCtx& s, i64 off_a, i64 off_b, i64 rows, i64 r, i64 gram_rows) {
+  static_assert(MAX_ROUNDS % 2 == 0, "the result must end in the first buffer");
+  for (int it = 0; it < MAX_ROUNDS; it += 2) {
+    DION_TRY(cholqr_round(s, off_a, off_b, rows, r, RM_ADAPTIVE, gram_rows));
+    DION_TRY(cholqr_round(s, off_b, off_a, rows, r, RM_ADAPTIVE, gram_rows));
+  }
+  launch_pdl(k_orth_finish, dim3((unsigned)(s.nb)), dim3(1), 0, s.st, s.os, s.c->dev_ints);
+  s.c->launches++;
+  if (cudaGetLastError() != cudaSuccess) return DION_ERR_CUDA;
+  return DION_OK;
+}
+
 // Randomized Cholesky QR (Algorithm 4 on one device) of the rows x r panel in P0 of every
 // matrix of the chain; U ends in P0.
-//   Pt = S P (sketch_rows x r);  R1 = triangular factor of QR(Pt), diag > 0 (Householder);
-//   B = P R1^-1 (as P Linv^T with Linv = (R1^T)^-1, the triangular-inverse path of the
-//   Cholesky-QR rounds);  then one plain Cholesky-QR round on B: R2 = Cholesky(B^T B), U = B R2^-1.
+//   Pt = S P (k x r sketch).  R1 = triangular factor of QR(Pt): computed by deflating Cholesky-QR
+//   rounds on the sketch, never formed explicitly -- the rounds run on the stacked panel [Pt; P] with
+//   their Gram matrices taken from the sketch rows only, so every round's triangular factor is applied
+//   to the sketch and to P at once; when the sketch has become orthonormal, the lower rows hold
+//   B = P R1^-1.  Then Cholesky QR on B (R2 = Cholesky(B^T B), U = B R2^-1; a second pass only if the
+//   device's check asks for it).  All matrices of a chain have the same number of sketch rows.
 int rcqr(StepCtx& s, i64 rows, i64 r) {
   dion_ctx* c = s.c;
   if (s.list == nullptr) return DION_ERR_INVALID;
+  const i64 k = s.list[0]->sketch_rows;
   for (int b = 0; b < s.nb; ++b) {
     const dion_matrix* a = s.list[b];
-    const i64 k = a->sketch_rows;
-    float* Pt = s.W(b, s.L.Sk);
+    if (a->sketch_rows != k) return DION_ERR_INVALID;
+    float* stack = s.W(b, s.L.Sk);
     GemmArgs g = gemm_args();
     g.M = k; g.N = r; g.K = rows;
     g.A = (const float*)a->sketch; g.a_si = a->ld_sketch; g.a_sk = 1;
     g.B = s.W(b, s.L.P0); g.b_sk = r; g.b_sn = 1;
-    g.C = Pt; g.ldc = r; g.epi = EPI_STORE; g.precise = 1;
+    g.C = stack; g.ldc = r; g.epi = EPI_STORE; g.precise = 1;
     DION_TRY(launch_gemm(s, g, b));
-    DION_TRY(householder_factor(s, Pt, s.W(b, s.L.SkV), k, r, b));
-    launch_pdl(k_rt_to_lower, dim3((unsigned)(grid_for(c, r * r))), dim3(256), 0, s.st, Pt, r, s.W(b, s.L.d), s.W(b, s.L.Gram), r, r,
-                                                         s.OS(b) + OS_FAIL, c->dev_ints);
+    dim3 grid((unsigned)grid_for(c, rows * r), 1);
+    launch_pdl(k_copy_block, grid, dim3(256), 0, s.st, (const float*)s.W(b, s.L.P0), r, stack + k * r, r, rows, r, nullptr, 0);
     DION_CHECK_LAUNCH(c);
   }
-  // Linv = (R1^T)^-1: 64 x 64 diagonal inverses, then the doubling levels
-  {
-    dim3 grid((unsigned)((r + NB - 1) / NB), (unsigned)s.nb);
-    launch_pdl(k_trtri_diag, grid, dim3(256), 0, s.st, s.ws + s.L.Gram, r, r, s.ws + s.L.Dinv, s.wstride);
-    DION_CHECK_LAUNCH(c);
-  }
-  if (r > NBO)
-    for (int m = 0; m < s.nb; ++m)
-      if (cudaMemsetAsync(s.W(m, s.L.Linv), 0, sizeof(float) * (size_t)r * (size_t)r, s.st) != cudaSuccess) return DION_ERR_CUDA;
-  for (i64 J0 = 0; J0 < r; J0 += NBO) {
-    const i64 sz = (r - J0 < NBO) ? (r - J0) : NBO;
-    dim3 grid((unsigned)grid_for(c, sz * sz), (unsigned)s.nb);
-    launch_pdl(k_linv_init, grid, dim3(256), 0, s.st, s.ws + s.L.Linv, r, J0, sz, s.ws + s.L.Dinv, nullptr, s.wstride);
-    DION_CHECK_LAUNCH(c);
-    DION_TRY(trtri_levels(s, r, J0, sz, NB, nullptr, 0));
-  }
-  if (r > NBO) DION_TRY(trtri_levels(s, r, 0, r, NBO, nullptr, 1));
-  GemmArgs u = gemm_args();   // B = P Linv^T
-  u.M = rows; u.N = r; u.K = r;
-  u.A = s.ws + s.L.P0; u.a_si = r; u.a_sk = 1;
-  u.B = s.ws + s.L.Linv; u.b_sk = 1; u.b_sn = r; u.klimit = 1;
-  u.C = s.ws + s.L.P1; u.ldc = r; u.epi = EPI_STORE; u.precise = 1;
-  for (int m = 0; m < s.nb; ++m) DION_TRY(launch_gemm(s, for_matrix(s, u, m, true, true, true), m));
-  return cholqr_round(s, s.L.P1, s.L.P0, rows, r, RM_PLAIN);
+  s.wt_off = s.L.SkW;
+  const int rc = adaptive_rounds(s, s.L.Sk, s.L.SkV, k + rows, r, k);
+  s.wt_off = -1;
+  DION_TRY(rc);
+  // B = the panel rows of the stack; the step's state slot starts afresh for its Cholesky QR
+  launch_pdl(k_reset_rounds, dim3((unsigned)s.nb), dim3(1), 0, s.st, s.os);
+  DION_CHECK_LAUNCH(c);
+  DION_TRY(cholqr_round(s, s.L.Sk + k * r, s.L.P1, rows, r, RM_FIRST));
+  return cholqr_round(s, s.L.P1, s.L.P0, rows, r, RM_CHECKED);
 }
 
 // The orthonormalization a step on (m, n, r) will use.
@@ -667,15 +678,7 @@ int orthonormalize(StepCtx& s, i64 rows, i64 r, i64 short_dim, i64* U_off) {
     DION_TRY(cholqr_round(s, s.L.P1, s.L.P0, rows, r, RM_CHECKED));
     *U_off = s.L.P0;
   } else if (mode == DION_ORTH_SHIFTED3) {
-    // Adaptive rounds: the device decides after each round whether the panel is done.
-    static_assert(MAX_ROUNDS % 2 == 0, "the result must end in P0");
-    for (int it = 0; it < MAX_ROUNDS; it += 2) {
-      DION_TRY(cholqr_round(s, s.L.P0, s.L.P1, rows, r, RM_ADAPTIVE));
-      DION_TRY(cholqr_round(s, s.L.P1, s.L.P0, rows, r, RM_ADAPTIVE));
-    }
-    launch_pdl(k_orth_finish, dim3((unsigned)(s.nb)), dim3(1), 0, s.st, s.os, s.c->dev_ints);
-    s.c->launches++;
-    if (cudaGetLastError() != cudaSuccess) return DION_ERR_CUDA;
+    DION_TRY(adaptive_rounds(s, s.L.P0, s.L.P1, rows, r, 0));
     *U_off = s.L.P0;
   } else if (mode == DION_ORTH_RCQR) {
     DION_TRY(rcqr(s, rows, r));
@@ -1147,7 +1150,7 @@ int dion_step_grouped(dion_ctx* ctx, const dion_matrix* list, int count, float l
     chain.clear();
     for (int j = i; j < count; ++j) {
       if (done[j] || list[j].m != list[i].m || list[j].n != list[i].n || list[j].r != list[i].r ||
-          list[j].transposed != list[i].transposed) continue;
+          list[j].transposed != list[i].transposed || list[j].sketch_rows != list[i].sketch_rows) continue;
       done[j] = 1;
       chain.push_back(&list[j]);
       if (chain.size() == cap) { chains.push_back(chain); chain.clear(); }

@@ -523,6 +523,13 @@ __global__ void k_orth_decide(int* __restrict__ os, float tau, int* __restrict__
   atomicAdd(rounds_total, done ? 1 : 2);
 }
 
+// Clears the round state of a step slot (keeps the fail flag): a second orthonormalization in one step.
+__global__ void k_reset_rounds(int* __restrict__ os) {
+  pdl_enter();
+  os += (i64)blockIdx.x * OS_SLOT_INTS;
+  os[OS_DONE] = 0; os[OS_GOOD] = 0; os[OS_FLOORED] = 0; os[OS_MAXDEV] = 0; os[OS_ROUNDS] = 0;
+}
+
 // After the last adaptive round: a panel that never became well conditioned is
 // reported; if pivots were still being raised the step is cancelled (rank-deficient P).
 __global__ void k_orth_finish(int* __restrict__ os, int* __restrict__ status) {
@@ -639,60 +646,6 @@ __global__ void k_latch_flag(const int* __restrict__ src, int* __restrict__ dst)
 __global__ void k_finish_step(const int* __restrict__ step_flag, int* __restrict__ skipped) {
   pdl_enter();
   if (step_flag[(i64)blockIdx.x * OS_SLOT_INTS] != 0) atomicAdd(skipped, 1);
-}
-
-// Inverse of every 64 x 64 diagonal block of the lower-triangular r x r matrix A into Dinv
-// (block j -> Dinv + j * 64 * 64, zero padded).  grid = (blocks, matrices).
-__global__ void __launch_bounds__(256) k_trtri_diag(const float* __restrict__ A, i64 ld, i64 r,
-                                                    float* __restrict__ Dinv, i64 wstride) {
-  pdl_enter();
-  A += (i64)blockIdx.y * wstride; Dinv += (i64)blockIdx.y * wstride;
-  __shared__ float L[NB][NB + 1];
-  __shared__ float X[NB][NB + 1];
-  __shared__ float T[NB / 2][NB / 2 + 1];
-  __shared__ float rdiag[NB];
-  const int tid = threadIdx.x;
-  const i64 j0 = (i64)blockIdx.x * NB;
-  const int jb = (int)((r - j0 < NB) ? (r - j0) : NB);
-  for (int e = tid; e < NB * NB; e += 256) {
-    const int i = e / NB, c = e % NB;
-    float v = (i < jb && c <= i) ? A[(j0 + i) * ld + j0 + c] : 0.f;
-    if (i == c && i >= jb) v = 1.f;
-    L[i][c] = v;
-    X[i][c] = 0.f;
-  }
-  __syncthreads();
-  if (tid < NB) rdiag[tid] = 1.f / L[tid][tid];
-  __syncthreads();
-  invert_block(L, X, T, rdiag, tid);
-  float* D = Dinv + (i64)blockIdx.x * (NB * NB);
-  for (int e = tid; e < NB * NB; e += 256) D[e] = X[e / NB][e % NB];
-}
-
-// After the Householder factorization of a k x r sketch held in A (rows 0..r-1 carry the
-// triangular factor above the diagonal, diag[] its diagonal): writes L = R^T with the sign
-// convention diag(R) > 0 (row j of R is negated when diag[j] < 0) into the lower triangle of G,
-// zeros above.  A diagonal entry that is zero or not finite (rank-deficient sketch) sets
-// *fail and the BREAKDOWN status bit and is replaced by 1.
-__global__ void k_rt_to_lower(const float* __restrict__ A, i64 lda, const float* __restrict__ diag,
-                              float* __restrict__ G, i64 ldg, i64 r, int* __restrict__ fail, int* __restrict__ status) {
-  pdl_enter();
-  const i64 total = r * r;
-  for (i64 e = (i64)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (i64)gridDim.x * blockDim.x) {
-    const i64 i = e / r, j = e % r;     // L[i][j] = R[j][i]
-    float v = 0.f;
-    if (j < i) {
-      v = (diag[j] < 0.f) ? -A[j * lda + i] : A[j * lda + i];
-    } else if (j == i) {
-      v = fabsf(diag[i]);
-      if (!(v > 0.f) || !isfinite(v)) {
-        v = 1.f;
-        *fail = 1;
-        atomicOr(status, DION_STATUS_BREAKDOWN);
-      }
-    }
-    G[i * ldg + j] = v;
-  }
 }
 
 // ---------------------------------------------------------------------------
