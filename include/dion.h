@@ -60,7 +60,9 @@ typedef enum { DION_F32 = 0, DION_BF16 = 1 } dion_dtype;
 /* Arithmetic of the four large contractions (P, R, U R^T, U Q^T).
  * DION_PREC_FP32:           products carry fp32 accuracy (fp32 FMA, or a 3-term
  *                           TF32 split on the tensor cores), fp32 accumulation.
- * DION_PREC_BF16_OPERANDS:  operands rounded to bf16, fp32 accumulation.       */
+ * DION_PREC_BF16_OPERANDS:  operands rounded to bf16 (M + G is added in fp32, then
+ *                           rounded), fp32 accumulation.
+ * The products inside Orthonormalize keep fp32 accuracy in both modes.          */
 typedef enum { DION_PREC_FP32 = 0, DION_PREC_BF16_OPERANDS = 1 } dion_precision;
 
 /* Orthonormalize (Section 3.2 and the appendix on Cholesky QR).
