@@ -505,7 +505,10 @@ __global__ void __launch_bounds__(TMA ? NUM_THREADS_TMA : NUM_THREADS, 1) k_gemm
         if (!mbar_wait(accf_bar(ab), ph, dead, p.status, 256)) { alive = false; break; }
         tc_fence_after();
 #pragma unroll 1
-        for (int cb = half * SLABS; cb < (half + 1) * SLABS; ++cb) {
+        for (int sj = 0; sj < SLABS; ++sj) {
+          // slab sj of the warps of one row quadrant lie side by side, so that the quadrant reads and
+          // writes contiguous row segments of 32 * (EPI_WARPS / 4) columns at about the same time
+          const int cb = sj * (C::EPI_WARPS / 4) + half;
           float acc[32];
           tmem_ld32(tmem_base + (uint32_t)(ab * ACCS * BN + cb * 32) + ((uint32_t)(quad * 32) << 16), acc);
           if (SPLIT) {
