@@ -407,15 +407,19 @@ struct Cfg {
   static constexpr int B_BYTES = BN * 128;
   static constexpr int STAGE_BYTES = BT ? (2 * A_BYTES + B_BYTES + A_BYTES / 2 + B_BYTES / 2)
                                         : (BF16 ? 1 : 2) * (A_BYTES + B_BYTES);
-  // CE (coalesced epilogue): each epilogue warp transposes its 32 x 32 accumulator slabs through a
-  // private shared-memory tile (32 rows of 36 floats), so that one global access of the warp
-  // covers four 128-byte row segments instead of 32 rows; paid for with one stage.
-  static constexpr int EPI_TILE_FLOATS = 32 * 36;
   // D16: the producer warps have no conversion work and serve as epilogue warps too
   static constexpr int EPI_WARPS = D16 ? NUM_EPI_WARPS + NUM_PROD_WARPS : NUM_EPI_WARPS;
+  // CE (coalesced epilogue): an epilogue warp owns 32 rows x EPI_W columns of the tile and passes them
+  // through a private shared-memory tile in passes of EPI_RPP rows (EPI_RPP * EPI_W = 1024 elements),
+  // so that one global access of the warp covers whole row segments instead of 32 rows; paid for with
+  // a pipeline stage (bf16 arrays) or the addend staging (fp32 operands: the products that use this
+  // epilogue have no fused addend).
+  static constexpr int EPI_W = 32 * (BN / 32) / (EPI_WARPS / 4);
+  static constexpr int EPI_RPP = 1024 / EPI_W;
+  static constexpr int EPI_TILE_FLOATS = EPI_RPP * (EPI_W + 4);
   static constexpr int EPI_BYTES = CE ? EPI_WARPS * EPI_TILE_FLOATS * 4 : 0;
   static constexpr int STAGES = CE ? (232448 - 1536 - EPI_BYTES) / STAGE_BYTES : (192 * 1024) / STAGE_BYTES;
-  static constexpr int G16_BYTES = ((BF16 && !TMA) || D16) ? 0 : BM * 32 * 2;   // bf16 addend tile of the TMA variants (per stage)
+  static constexpr int G16_BYTES = ((BF16 && !TMA) || D16 || CE) ? 0 : BM * 32 * 2;   // bf16 addend tile of the TMA variants (per stage)
   static constexpr int SMEM_BYTES = STAGES * (STAGE_BYTES + G16_BYTES) + EPI_BYTES + 1024 + 512;
   static constexpr int A_CHUNKS = BM * 8 / NUM_PROD_THREADS;  // 16-byte chunks per producer thread
   static constexpr int B_CHUNKS = BN * 8 / NUM_PROD_THREADS;
@@ -439,7 +443,7 @@ template <int BN, bool A_MN, bool B_MN, bool BF16, bool SPLIT, bool TMA, bool D1
 __global__ void __launch_bounds__(TMA ? NUM_THREADS_TMA : NUM_THREADS, 1) k_gemm_umma(const __grid_constant__ Params p) {
   static_assert(!(BF16 && SPLIT), "split accumulators belong to the 3xTF32 mode");
   static_assert(!D16 || (BF16 && TMA), "bf16 operands in memory are loaded by TMA");
-  static_assert(!CE || D16, "the coalesced epilogue is built for the bf16-array variant");
+  static_assert(!CE || (TMA && !SPLIT && (D16 || !BF16)), "the coalesced epilogue serves the bf16-array and the plain fp32 TMA variants");
   using C = Cfg<BN, BF16, SPLIT, TMA, D16, CE>;
   constexpr int NBUF = C::NBUF, ACCS = C::ACCS;
   constexpr int BKE = C::BKE, EPC = C::EPC, STAGES = C::STAGES;
@@ -509,18 +513,19 @@ __global__ void __launch_bounds__(TMA ? NUM_THREADS_TMA : NUM_THREADS, 1) k_gemm
         if constexpr (CE) {
           // Coalesced epilogue.  A TMEM lane is a row, so a warp that wrote its accumulator rows straight
           // out would touch 32 rows per global access.  Instead the warp handles its 32 rows x W columns
-          // (W = 32 SLABS) in two passes of 16 rows: it reads the slabs from TMEM, the lanes of the pass's
-          // 16 rows put theirs into the warp's shared-memory tile, and the warp then accesses memory row
-          // by row (an instruction covers RPI rows of W contiguous columns).  The four warps of a row
-          // quadrant own neighbouring column ranges, so a quadrant pass reads and writes 16 full row
+          // (W = 32 SLABS) in passes of RPP rows: it reads its slabs from TMEM, the lanes of the pass's
+          // rows put theirs into the warp's shared-memory tile, and the warp then accesses memory row
+          // by row (an instruction covers RPI rows of W contiguous columns).  The warps of a row
+          // quadrant own neighbouring column ranges, so a quadrant pass reads and writes RPP full row
           // segments of the tile (BN columns: 1 KB at BN = 256) at about the same time; that locality
           // is worth 25-30 % of DRAM bandwidth against 32 x 32 slabs handled one after another.
-          constexpr int W = 32 * SLABS;
+          constexpr int W = C::EPI_W;
+          constexpr int RPP = C::EPI_RPP;     // rows per pass
           constexpr int LPR = W / 4;          // lanes per row
           constexpr int RPI = 32 / LPR;       // rows per instruction
-          constexpr int NI = 16 / RPI;        // instructions per pass
+          constexpr int NI = RPP / RPI;       // instructions per pass (8)
           constexpr int TS = W + 4;           // tile row stride (floats)
-          static_assert(!CE || 16 * TS <= C::EPI_TILE_FLOATS, "tile of one pass");
+          static_assert(W == 32 * SLABS && NI == 8, "pass geometry");
           float* tb = epi_tiles + warp * C::EPI_TILE_FLOATS;
           const bool to_part = p.splits > 1;
           const bool need_c = !first || (!to_part && g.epi != EPI_STORE && g.epi != EPI_C2_SUB);
@@ -530,20 +535,16 @@ __global__ void __launch_bounds__(TMA ? NUM_THREADS_TMA : NUM_THREADS, 1) k_gemm
           float f = 1.f;
           if (!to_part) f = (g.epi != EPI_STORE) ? -alpha : alpha;
 #pragma unroll 1
-          for (int hp = 0; hp < 2; ++hp) {
-            {
-              float acc[SLABS][32];
+          for (int ps = 0; ps < 32 / RPP; ++ps) {
 #pragma unroll
-              for (int sl = 0; sl < SLABS; ++sl)
-                tmem_ld32<false>(tmem_base + (uint32_t)(ab * ACCS * BN + half * W + sl * 32) + ((uint32_t)(quad * 32) << 16), acc[sl]);
-              tmem_ld_wait();
-              if ((lane >> 4) == hp) {
+            for (int sl = 0; sl < SLABS; ++sl) {
+              float acc[32];
+              tmem_ld32(tmem_base + (uint32_t)(ab * ACCS * BN + half * W + sl * 32) + ((uint32_t)(quad * 32) << 16), acc);
+              if (lane / RPP == ps) {
 #pragma unroll
-                for (int sl = 0; sl < SLABS; ++sl)
-#pragma unroll
-                  for (int q = 0; q < 8; ++q)
-                    *reinterpret_cast<float4*>(tb + (lane & 15) * TS + sl * 32 + 4 * q) =
-                        make_float4(acc[sl][4 * q], acc[sl][4 * q + 1], acc[sl][4 * q + 2], acc[sl][4 * q + 3]);
+                for (int q = 0; q < 8; ++q)
+                  *reinterpret_cast<float4*>(tb + (lane % RPP) * TS + sl * 32 + 4 * q) =
+                      make_float4(acc[4 * q], acc[4 * q + 1], acc[4 * q + 2], acc[4 * q + 3]);
               }
             }
             __syncwarp();
@@ -552,7 +553,7 @@ __global__ void __launch_bounds__(TMA ? NUM_THREADS_TMA : NUM_THREADS, 1) k_gemm
             bool ok[NI];
 #pragma unroll
             for (int q = 0; q < NI; ++q) {
-              const i64 row = (i64)it.mi * BM + quad * 32 + hp * 16 + RPI * q + lane / LPR;
+              const i64 row = (i64)it.mi * BM + quad * 32 + ps * RPP + RPI * q + lane / LPR;
               ok[q] = row < g.M && col < g.N;
               cptr[q] = to_part ? reinterpret_cast<float4*>(g.part + ((i64)it.ks * g.M + row) * g.N + col)
                                 : reinterpret_cast<float4*>(g.C + row * g.ldc + col);
@@ -1046,7 +1047,8 @@ inline int umma_configure() {
   if (e == cudaSuccess && !F) e = set_smem_attr<BN, A, B, false, true, true>();  \
   if (e == cudaSuccess && F) e = set_smem_attr<BN, A, B, true, false, true>();    \
   if (e == cudaSuccess && F) e = set_smem_attr<BN, A, B, true, false, true, true>();    \
-  if (e == cudaSuccess && F) e = set_smem_attr<BN, A, B, true, false, true, true, true>();
+  if (e == cudaSuccess && F) e = set_smem_attr<BN, A, B, true, false, true, true, true>();  \
+  if (e == cudaSuccess && !F) e = set_smem_attr<BN, A, B, false, false, true, false, true>();
   DION_SET(128, false, false, false) DION_SET(128, false, true, false) DION_SET(128, true, true, false) DION_SET(128, true, false, false)
   DION_SET(256, false, false, false) DION_SET(256, false, true, false) DION_SET(256, true, true, false) DION_SET(256, true, false, false)
   DION_SET(128, false, false, true) DION_SET(128, false, true, true) DION_SET(128, true, true, true) DION_SET(128, true, false, true)
@@ -1150,6 +1152,9 @@ inline int umma_try_launch(const GemmArgs& g_in, int precision, int sm_count, fl
   } else if (bf16) {
     if (BN == 256) launch_variant<256, true, false, false>(p, a_mn, b_mn, grid, st);
     else launch_variant<128, true, false, false>(p, a_mn, b_mn, grid, st);
+  } else if (tma && !g.precise && g.epi != EPI_STORE && g.a2_mode == ADD_NONE) {   // output-bound products
+    if (BN == 256) launch_variant<256, false, false, true, false, true>(p, a_mn, b_mn, grid, st);
+    else launch_variant<128, false, false, true, false, true>(p, a_mn, b_mn, grid, st);
   } else if (tma) {
     if (g.precise) {
       if (BN == 256) launch_variant<256, false, true, true>(p, a_mn, b_mn, grid, st);
