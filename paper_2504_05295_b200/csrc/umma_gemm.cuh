@@ -443,7 +443,7 @@ template <int BN, bool A_MN, bool B_MN, bool BF16, bool SPLIT, bool TMA, bool D1
 __global__ void __launch_bounds__(TMA ? NUM_THREADS_TMA : NUM_THREADS, 1) k_gemm_umma(const __grid_constant__ Params p) {
   static_assert(!(BF16 && SPLIT), "split accumulators belong to the 3xTF32 mode");
   static_assert(!D16 || (BF16 && TMA), "bf16 operands in memory are loaded by TMA");
-  static_assert(!CE || (TMA && !SPLIT && (D16 || !BF16)), "the coalesced epilogue serves the bf16-array and the plain fp32 TMA variants");
+  static_assert(!CE || (TMA && (D16 || !BF16)), "the coalesced epilogue serves the bf16-array and the fp32 TMA variants");
   using C = Cfg<BN, BF16, SPLIT, TMA, D16, CE>;
   constexpr int NBUF = C::NBUF, ACCS = C::ACCS;
   constexpr int BKE = C::BKE, EPC = C::EPC, STAGES = C::STAGES;
@@ -540,6 +540,12 @@ __global__ void __launch_bounds__(TMA ? NUM_THREADS_TMA : NUM_THREADS, 1) k_gemm
             for (int sl = 0; sl < SLABS; ++sl) {
               float acc[32];
               tmem_ld32(tmem_base + (uint32_t)(ab * ACCS * BN + half * W + sl * 32) + ((uint32_t)(quad * 32) << 16), acc);
+              if (SPLIT) {
+                float small[32];
+                tmem_ld32(tmem_base + (uint32_t)(ab * ACCS * BN + BN + half * W + sl * 32) + ((uint32_t)(quad * 32) << 16), small);
+#pragma unroll
+                for (int e = 0; e < 32; ++e) acc[e] += small[e];
+              }
               if (lane / RPP == ps) {
 #pragma unroll
                 for (int q = 0; q < 8; ++q)
@@ -1048,7 +1054,8 @@ inline int umma_configure() {
   if (e == cudaSuccess && F) e = set_smem_attr<BN, A, B, true, false, true>();    \
   if (e == cudaSuccess && F) e = set_smem_attr<BN, A, B, true, false, true, true>();    \
   if (e == cudaSuccess && F) e = set_smem_attr<BN, A, B, true, false, true, true, true>();  \
-  if (e == cudaSuccess && !F) e = set_smem_attr<BN, A, B, false, false, true, false, true>();
+  if (e == cudaSuccess && !F) e = set_smem_attr<BN, A, B, false, false, true, false, true>();  \
+  if (e == cudaSuccess && !F) e = set_smem_attr<BN, A, B, false, true, true, false, true>();
   DION_SET(128, false, false, false) DION_SET(128, false, true, false) DION_SET(128, true, true, false) DION_SET(128, true, false, false)
   DION_SET(256, false, false, false) DION_SET(256, false, true, false) DION_SET(256, true, true, false) DION_SET(256, true, false, false)
   DION_SET(128, false, false, true) DION_SET(128, false, true, true) DION_SET(128, true, true, true) DION_SET(128, true, false, true)
@@ -1152,9 +1159,14 @@ inline int umma_try_launch(const GemmArgs& g_in, int precision, int sm_count, fl
   } else if (bf16) {
     if (BN == 256) launch_variant<256, true, false, false>(p, a_mn, b_mn, grid, st);
     else launch_variant<128, true, false, false>(p, a_mn, b_mn, grid, st);
-  } else if (tma && !g.precise && g.epi != EPI_STORE && g.a2_mode == ADD_NONE) {   // output-bound products
-    if (BN == 256) launch_variant<256, false, false, true, false, true>(p, a_mn, b_mn, grid, st);
-    else launch_variant<128, false, false, true, false, true>(p, a_mn, b_mn, grid, st);
+  } else if (tma && g.a2_mode != ADD_BF16 && (!g.precise || BN == 256)) {   // coalesced epilogue in place of the bf16 addend staging
+    if (g.precise) {
+      if (BN == 256) launch_variant<256, false, true, true, false, true>(p, a_mn, b_mn, grid, st);
+      else launch_variant<128, false, true, true, false, true>(p, a_mn, b_mn, grid, st);
+    } else {
+      if (BN == 256) launch_variant<256, false, false, true, false, true>(p, a_mn, b_mn, grid, st);
+      else launch_variant<128, false, false, true, false, true>(p, a_mn, b_mn, grid, st);
+    }
   } else if (tma) {
     if (g.precise) {
       if (BN == 256) launch_variant<256, false, true, true>(p, a_mn, b_mn, grid, st);
