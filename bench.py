@@ -35,9 +35,9 @@ UNIT = "ms"
 MU, ETA, EPS = 0.95, 0.01, 1e-8
 FFMA_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12     # 148 SMs x 128 FMA lanes x 2 flop x max clock
 # DRAM bytes (read + write) of the four large k_gemm_umma launches of a 4096^2 / r = 1024 step in one ncu
-# capture (profiles/k_gemm_umma_tma_4096sq_r1024.md) over their algorithmic bytes: 646.5 MB / 738.3 MB.
+# capture (profiles/k_gemm_umma_tma_4096sq_r1024.md) over their algorithmic bytes: 653.4 MB / 738.3 MB.
 # Traffic grows in proportion to the matrix sizes, so the ratio scales the algorithmic bytes of any workload.
-NCU_TRAFFIC_RATIO = 0.876
+NCU_TRAFFIC_RATIO = 0.885
 
 
 def load_peaks():
@@ -546,9 +546,9 @@ def run_ours(args):
                  "phases": gemm_phases, "ms_per_step": dom_ms, "share_of_step": dom_ms * args.steps / max(total_phase_ms, 1e-9),
                  "launches_per_step": dom_launches,
                  "algorithmic_flops_per_step": dom_fl, "algorithmic_bytes_per_step": dom_by,
-                 "traffic_note": "algorithmic bytes x 0.876, the DRAM (read + write) / algorithmic ratio of this kernel's "
+                 "traffic_note": "algorithmic bytes x %.3f, the DRAM (read + write) / algorithmic ratio of this kernel's "
                                  "four large launches in the ncu capture at 4096^2 r=1024 (profiles/k_gemm_umma_tma_4096sq_r1024.md); "
-                                 "per step, all launches"})
+                                 "per step, all launches" % NCU_TRAFFIC_RATIO})
     if tensor_engine:
         roof["traffic"] = NCU_TRAFFIC_RATIO * dom_by
     # The four large products alone (never overlapped with other work; the products inside the

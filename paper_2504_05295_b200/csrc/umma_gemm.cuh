@@ -1147,7 +1147,7 @@ inline int umma_try_launch(const GemmArgs& g_in, int precision, int sm_count, fl
   // split accumulators); 2048 k for bf16 operands loaded through registers
   p.kc = 32;
   const int grid = p.num_items < sm_count ? p.num_items : sm_count;
-  if (d16 && g.epi != EPI_STORE) {   // output-bound products: coalesced epilogue
+  if (d16) {   // coalesced epilogue
     if (BN == 256) launch_variant<256, true, false, true, true, true>(p, a_mn, b_mn, grid, st);
     else launch_variant<128, true, false, true, true, true>(p, a_mn, b_mn, grid, st);
   } else if (d16) {
