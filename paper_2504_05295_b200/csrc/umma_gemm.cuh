@@ -16,9 +16,14 @@
 //   TMA, bf16 operands from fp32 arrays: same loads; the producer warps add, round and
 //     write bf16 operand tiles.
 //   bf16 arrays (D16): TMA writes the operand tiles themselves; the producer warps join
-//     the epilogue; optionally with the coalesced epilogue (CE).
+//     the epilogue.
 //   register path: the producer warps load global memory through registers (operands a
 //     tensor map cannot describe).
+// Coalesced epilogue (CE; the bf16-array variant and the fp32 TMA variant when there is no
+// bf16 addend to stage): the epilogue warps pass their accumulator rows through shared-
+// memory tiles and access global memory in whole row segments, 8 or 16 rows of the tile's
+// full width per row quadrant at a time.  The plain epilogue (a lane writes its own row)
+// remains for the other variants.
 //
 // Every wait on an mbarrier is bounded by a cycle budget: when it runs out the CTA
 // marks itself dead, raises DION_STATUS_TIMEOUT and drains, so a protocol bug
@@ -1052,7 +1057,6 @@ inline int umma_configure() {
   if (e == cudaSuccess && !F) e = set_smem_attr<BN, A, B, false, false, true>();  \
   if (e == cudaSuccess && !F) e = set_smem_attr<BN, A, B, false, true, true>();  \
   if (e == cudaSuccess && F) e = set_smem_attr<BN, A, B, true, false, true>();    \
-  if (e == cudaSuccess && F) e = set_smem_attr<BN, A, B, true, false, true, true>();    \
   if (e == cudaSuccess && F) e = set_smem_attr<BN, A, B, true, false, true, true, true>();  \
   if (e == cudaSuccess && !F) e = set_smem_attr<BN, A, B, false, false, true, false, true>();  \
   if (e == cudaSuccess && !F) e = set_smem_attr<BN, A, B, false, true, true, false, true>();
@@ -1147,12 +1151,9 @@ inline int umma_try_launch(const GemmArgs& g_in, int precision, int sm_count, fl
   // split accumulators); 2048 k for bf16 operands loaded through registers
   p.kc = 32;
   const int grid = p.num_items < sm_count ? p.num_items : sm_count;
-  if (d16) {   // coalesced epilogue
+  if (d16) {   // bf16 arrays: always with the coalesced epilogue
     if (BN == 256) launch_variant<256, true, false, true, true, true>(p, a_mn, b_mn, grid, st);
     else launch_variant<128, true, false, true, true, true>(p, a_mn, b_mn, grid, st);
-  } else if (d16) {
-    if (BN == 256) launch_variant<256, true, false, true, true>(p, a_mn, b_mn, grid, st);
-    else launch_variant<128, true, false, true, true>(p, a_mn, b_mn, grid, st);
   } else if (bf16 && tma) {
     if (BN == 256) launch_variant<256, true, false, true>(p, a_mn, b_mn, grid, st);
     else launch_variant<128, true, false, true>(p, a_mn, b_mn, grid, st);
