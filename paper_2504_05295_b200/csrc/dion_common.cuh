@@ -41,7 +41,7 @@ struct GemmArgs {
   int batch2; i64 bs2;           // outer batch (one per matrix of a grouped call): stride of A, B, C alike
   i64 skip_stride;               // ints between the skip flags of consecutive outer batch entries
   int splits; float* part;       // split-K: partial sums, [splits][M][N]
-  int tri;                       // TRI_LOWER: tiles strictly above the diagonal are skipped
+  int tri;                       // TRI_LOWER: only the elements on or below the diagonal are needed (tiles above it are skipped)
   int klimit;                    // 1: B(k,j) == 0 for k > j  (K loop ends at the tile's last column)
   const int* skip_flag;          // optional: if *skip_flag != 0 the kernel does nothing
   int precise;                   // tensor engine: keep the small split terms in their own accumulator

@@ -18,7 +18,7 @@ typedef struct {
   int epi;                                       /* 0 C=a*acc, 1 C-=a*acc, 2 C=C+C2-a*acc  */
   const void* C2; int64_t ldc2; int c2_mode;
   float alpha;
-  int tri;                                       /* 1: only tiles on or below the diagonal */
+  int tri;                                       /* 1: only elements on or below the diagonal are guaranteed */
   int klimit;                                    /* 1: B(k,j) = 0 for k > j                */
   int precise;                                   /* 1: split accumulators (tensor engine)  */
   int ab16;                                      /* 1: A and B are bf16 arrays (tensor engine) */

@@ -235,6 +235,8 @@ __device__ __forceinline__ uint32_t make_idesc(bool bf16, bool a_mn, bool b_mn, 
   return d;
 }
 
+constexpr i64 TRI_WIDE_MIN = 4096;   // smallest lower-triangular output computed in 128 x 256 tiles
+
 struct Item {
   int mi, ni, ks, kb0, kb1;
 };
@@ -244,7 +246,16 @@ __device__ __forceinline__ Item decode_item(const Params& p, int item) {
   Item it;
   const int tile = item / p.splits;
   it.ks = item - tile * p.splits;
-  if (p.g.tri == TRI_LOWER) {
+  if (p.g.tri == TRI_LOWER && BN == 2 * BM) {
+    // 128 x 256 tiles that reach the diagonal or lie below it: tile row mi has mi / 2 + 1 of them,
+    // (mi + 1)^2 / 4 (rounded down) lie in the rows above it
+    int mi = (int)(2.f * sqrtf((float)tile)) - 1;
+    if (mi < 0) mi = 0;
+    while ((mi + 2) * (mi + 2) / 4 <= tile) ++mi;
+    while ((mi + 1) * (mi + 1) / 4 > tile) --mi;
+    it.mi = mi;
+    it.ni = tile - (mi + 1) * (mi + 1) / 4;
+  } else if (p.g.tri == TRI_LOWER) {
     int mi = (int)((sqrtf(8.f * (float)tile + 1.f) - 1.f) * 0.5f);
     while ((mi + 1) * (mi + 2) / 2 <= tile) ++mi;
     while (mi * (mi + 1) / 2 > tile) --mi;
@@ -1103,7 +1114,10 @@ inline int umma_try_launch(const GemmArgs& g_in, int precision, int sm_count, fl
   }
   if (g.tri == TRI_LOWER && g.M != g.N) return 0;
 
-  const int BN = (g.tri == TRI_LOWER || g.N < 256) ? 128 : 256;
+  // lower-triangular output: 128 x 256 tiles (more flops per operand byte; the tiles on the diagonal
+  // compute up to 128 columns too many) once the matrix has enough tile rows for that to pay
+  const bool tri_wide = g.tri == TRI_LOWER && g.epi == EPI_STORE && g.N >= TRI_WIDE_MIN && !(debug & 32);
+  const int BN = ((g.tri == TRI_LOWER && !tri_wide) || g.N < 256) ? 128 : 256;
   Params p;
   p.g = g;
   // TMA variant: fp32 operands in memory (both precision modes), dimensions the tensor maps can describe
@@ -1129,7 +1143,9 @@ inline int umma_try_launch(const GemmArgs& g_in, int precision, int sm_count, fl
   p.nM = (int)((g.M + BM - 1) / BM);
   p.nN = (int)((g.N + BN - 1) / BN);
   p.nkb = (int)((g.K + bke - 1) / bke);
-  const i64 tiles = (g.tri == TRI_LOWER) ? (i64)p.nM * (p.nM + 1) / 2 : (i64)p.nM * p.nN;
+  const i64 tiles = (g.tri != TRI_LOWER) ? (i64)p.nM * p.nN
+                    : (BN == 256)          ? ((i64)p.nM + 1) * (p.nM + 1) / 4
+                                           : (i64)p.nM * (p.nM + 1) / 2;
   int splits = 1;
   if (g.epi == EPI_STORE && !g.klimit && part != nullptr && tiles < sm_count) {
     i64 want = sm_count / tiles;

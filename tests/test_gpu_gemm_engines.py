@@ -139,6 +139,9 @@ def test_gram_lower_triangle_and_split_k(lib, engine):
     # Gram matrix P^T P: both operands row-contiguous, only lower tiles, long K -> split-K
     assert run(lib, engine, 0, 512, 512, 8192, True, True, tri=1) < TOL[engine]
     assert run(lib, engine, 0, 256, 256, 4096, True, True, tri=1) < TOL[engine]
+    # large enough for the tensor engine's 128 x 256 lower tiles, with a ragged last tile row
+    assert run(lib, engine, 0, 4096, 4096, 512, True, True, tri=1) < TOL[engine]
+    assert run(lib, engine, 0, 4360, 4360, 264, True, True, tri=1, precise=1) < TOL[engine]
     # tall-skinny product with few tiles -> split-K
     assert run(lib, engine, 0, 2048, 128, 2048, False, True) < TOL[engine]
 
