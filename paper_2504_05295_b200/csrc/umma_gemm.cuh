@@ -1176,7 +1176,7 @@ inline int umma_try_launch(const GemmArgs& g_in, int precision, int sm_count, fl
   } else if (bf16) {
     if (BN == 256) launch_variant<256, true, false, false>(p, a_mn, b_mn, grid, st);
     else launch_variant<128, true, false, false>(p, a_mn, b_mn, grid, st);
-  } else if (tma && g.a2_mode != ADD_BF16 && (!g.precise || BN == 256)) {   // coalesced epilogue in place of the bf16 addend staging
+  } else if (tma && g.a2_mode != ADD_BF16 && (!g.precise || BN == 256 || g.epi != EPI_STORE)) {   // coalesced epilogue in place of the bf16 addend staging
     if (g.precise) {
       if (BN == 256) launch_variant<256, false, true, true, false, true>(p, a_mn, b_mn, grid, st);
       else launch_variant<128, false, true, true, false, true>(p, a_mn, b_mn, grid, st);
