@@ -387,25 +387,23 @@ int potrf_inner(StepCtx& s, i64 r, i64 o, i64 sz, int mode) {
                DinvP + (o / NB) * (NB * NB), gdiag + o, floor_rel, s.os, adaptive ? 1 : 0, status, s.wstride);
     DION_CHECK_LAUNCH(c);
   }
-  // one launch per block column: panel, trailing update and the next diagonal block
+  // one launch per block column: panel, trailing update and the next diagonal block; behind them, j CTAs
+  // that form block row j of the inverse of the square's factor (off the critical path)
   for (int j = 0; j + 1 < nblk; ++j) {
     const int nt = nblk - 1 - j;
-    dim3 grid((unsigned)(nt * (nt + 1) / 2), (unsigned)s.nb);
-    launch_pdl(k_chol_step, grid, dim3(256), CHOL_STEP_SMEM, s.st, Gm, r, o, sz, j, Dinv, DinvP, Tbuf, gdiag, floor_rel,
+    dim3 grid((unsigned)(nt * (nt + 1) / 2 + j), (unsigned)s.nb);
+    launch_pdl(k_chol_step, grid, dim3(256), CHOL_STEP_SMEM, s.st, Gm, r, o, sz, j, Dinv, DinvP, Tbuf, Linv, gdiag, floor_rel,
                s.os, adaptive ? 1 : 0, status, s.wstride);
     DION_CHECK_LAUNCH(c);
   }
-  if (nblk > 1) {
-    dim3 grid((unsigned)grid_for(c, sz * sz), (unsigned)s.nb);
-    launch_pdl(k_copy_lower_blocks, grid, dim3(256), 0, s.st, (const float*)Tbuf, Gm, r, o, sz, skip, s.wstride);
-    DION_CHECK_LAUNCH(c);
-  }
   {
-    dim3 grid((unsigned)grid_for(c, sz * sz), (unsigned)s.nb);
-    launch_pdl(k_linv_init, grid, dim3(256), 0, s.st, Linv, r, o, sz, (const float*)Dinv, skip, s.wstride);
+    // last block row of the inverse, the factor's blocks into the Gram buffer, diagonal inverses into Linv
+    dim3 grid((unsigned)(nblk - 1 + grid_for(c, sz * sz)), (unsigned)s.nb);
+    launch_pdl(k_inv_finish, grid, dim3(256), INV_FINISH_SMEM, s.st, (const float*)Tbuf, Gm, Linv, r, o, sz, (const float*)Dinv, skip,
+               s.wstride);
     DION_CHECK_LAUNCH(c);
   }
-  return trtri_levels(s, r, o, sz, NB, skip, 0);
+  return DION_OK;
 }
 
 // Two-level blocked Cholesky of each r x r Gram matrix (lower) and the full inverse of its

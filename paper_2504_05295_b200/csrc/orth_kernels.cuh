@@ -324,6 +324,51 @@ __device__ __forceinline__ void mm_nt_64(mm_t A, mm_t B, int ty, int tx, float (
 
 constexpr int CHOL_STEP_SMEM = 3 * NB * MMS * (int)sizeof(float);
 
+// Block (i, m), m < i, of the inverse X of the factor of the diagonal square [o, o+sz), from the block
+// rows above it:  X_im = -Dinv_i * sum_{k=m}^{i-1} L_ik X_km  with X_mm = Dinv_m  (64 x 64 blocks).
+// L_ik is read from Lsrc (the panels the steps have written), X_km from Linv (written by the CTAs of
+// earlier launches), the diagonal inverses from Dinv.  One CTA of 256 threads; smem holds two tiles.
+__device__ __forceinline__ void inv_tile(const float* __restrict__ Lsrc, float* __restrict__ Linv, i64 ld,
+                                         const float* __restrict__ Dinv, i64 o, i64 sz, int i, int m, float* smem) {
+  mm_t S0 = reinterpret_cast<mm_t>(smem);
+  mm_t S1 = reinterpret_cast<mm_t>(smem + NB * MMS);
+  const int tid = threadIdx.x, ty = tid >> 4, tx = tid & 15;
+  const i64 ri = o + (i64)i * NB, cm = o + (i64)m * NB;
+  const int rows_i = (int)((o + sz - ri < NB) ? (o + sz - ri) : NB);
+  float acc[4][4] = {};
+  for (int k = m; k < i; ++k) {
+    const i64 rk = o + (i64)k * NB;
+    const float* Dk = Dinv + (rk / NB) * (NB * NB);
+#pragma unroll 4
+    for (int l = 0; l < NB * NB / 256; ++l) {
+      const int e = tid + l * 256, rr = e / NB, cc = e % NB;
+      S0[rr][cc] = (rr < rows_i) ? Lsrc[(ri + rr) * ld + rk + cc] : 0.f;
+      S1[cc][rr] = (k == m) ? Dk[e] : Linv[(rk + rr) * ld + cm + cc];   // transposed: the product below is A * B^T
+    }
+    __syncthreads();
+    mm_nt_64(S0, S1, ty, tx, acc);
+    __syncthreads();
+  }
+  const float* Di = Dinv + (ri / NB) * (NB * NB);
+#pragma unroll
+  for (int a = 0; a < 4; ++a)
+#pragma unroll
+    for (int b = 0; b < 4; ++b) S1[tx + 16 * b][ty * 4 + a] = acc[a][b];
+#pragma unroll 4
+  for (int l = 0; l < NB * NB / 256; ++l) {
+    const int e = tid + l * 256;
+    S0[e / NB][e % NB] = Di[e];
+  }
+  __syncthreads();
+  float x[4][4] = {};
+  mm_nt_64(S0, S1, ty, tx, x);
+#pragma unroll
+  for (int a = 0; a < 4; ++a)
+#pragma unroll
+    for (int b = 0; b < 4; ++b)
+      if (ty * 4 + a < rows_i) Linv[(ri + ty * 4 + a) * ld + cm + tx + 16 * b] = -x[a][b];
+}
+
 // One step of the right-looking 64-column Cholesky inside the diagonal square [o, o+sz)
 // of the Gram matrix, in ONE launch: with the diagonal block of block column j already
 // factored (its inverse in DinvP), CTA (bi, bk), bk <= bi, forms the two 64-row pieces
@@ -335,13 +380,13 @@ constexpr int CHOL_STEP_SMEM = 3 * NB * MMS * (int)sizeof(float);
 // launch, so it cannot be overwritten here; the caller copies Lout back after the last step.
 __global__ void __launch_bounds__(256) k_chol_step(float* __restrict__ A, i64 ld, i64 o, i64 sz, int j,
                                                    float* __restrict__ Dinv, float* __restrict__ DinvP,
-                                                   float* __restrict__ Lout,
+                                                   float* __restrict__ Lout, float* __restrict__ Linv,
                                                    const float* __restrict__ gdiag, float floor_rel,
                                                    int* __restrict__ os, int adaptive,
                                                    int* __restrict__ status, i64 wstride) {
   {
     const i64 wo = (i64)blockIdx.y * wstride;
-    A += wo; Dinv += wo; DinvP += wo; Lout += wo; gdiag += wo;
+    A += wo; Dinv += wo; DinvP += wo; Lout += wo; Linv += wo; gdiag += wo;
     os += (i64)blockIdx.y * OS_SLOT_INTS;
   }
   // Launched with programmatic stream serialization: the next step's CTAs may be scheduled while
@@ -349,6 +394,16 @@ __global__ void __launch_bounds__(256) k_chol_step(float* __restrict__ A, i64 ld
   pdl_enter();
   if (adaptive && os[OS_DONE] != 0) return;
   extern __shared__ __align__(16) float chol_smem[];
+  {
+    // the CTAs behind the trailing blocks: block row j of the inverse of the square's factor (its
+    // inputs, the rows above and the diagonal inverse of block j, are final since the last launch)
+    const int nt = (int)((sz + NB - 1) / NB) - 1 - j;
+    const int ntri = nt * (nt + 1) / 2;
+    if ((int)blockIdx.x >= ntri) {
+      inv_tile(Lout, Linv, ld, Dinv, o, sz, j, (int)blockIdx.x - ntri, chol_smem);
+      return;
+    }
+  }
   mm_t S0 = reinterpret_cast<mm_t>(chol_smem);
   mm_t S1 = reinterpret_cast<mm_t>(chol_smem + NB * MMS);
   mm_t S2 = reinterpret_cast<mm_t>(chol_smem + 2 * NB * MMS);
@@ -448,17 +503,35 @@ __global__ void __launch_bounds__(256) k_chol_step(float* __restrict__ A, i64 ld
   }
 }
 
-// After the last k_chol_step of a square: the blocks of the factor strictly below the
-// block diagonal move from Lout into A.
-__global__ void k_copy_lower_blocks(const float* __restrict__ Lout, float* __restrict__ A, i64 ld, i64 o, i64 sz,
-                                    const int* __restrict__ skip_flag, i64 wstride) {
+// After the last k_chol_step of a square [o, o+sz): the first CTAs form the last block row of the
+// inverse of the factor (inv_tile); the others move the factor's blocks below the block diagonal from
+// Lout into A, put the diagonal inverses into Linv and clear Linv above the block diagonal.
+constexpr int INV_FINISH_SMEM = 2 * NB * MMS * (int)sizeof(float);
+__global__ void __launch_bounds__(256) k_inv_finish(const float* __restrict__ Lout, float* __restrict__ A,
+                                                    float* __restrict__ Linv, i64 ld, i64 o, i64 sz,
+                                                    const float* __restrict__ Dinv,
+                                                    const int* __restrict__ skip_flag, i64 wstride) {
   Lout += (i64)blockIdx.y * wstride; A += (i64)blockIdx.y * wstride;
+  Linv += (i64)blockIdx.y * wstride; Dinv += (i64)blockIdx.y * wstride;
   pdl_enter();
   if (skip_flag != nullptr && skip_flag[(i64)blockIdx.y * OS_SLOT_INTS] != 0) return;
+  extern __shared__ __align__(16) float fin_smem[];
+  const int nblk = (int)((sz + NB - 1) / NB);
+  if ((int)blockIdx.x < nblk - 1) {
+    inv_tile(Lout, Linv, ld, Dinv, o, sz, nblk - 1, (int)blockIdx.x, fin_smem);
+    return;
+  }
   const i64 total = sz * sz;
-  for (i64 e = (i64)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (i64)gridDim.x * blockDim.x) {
+  const i64 first = (i64)((int)blockIdx.x - (nblk - 1)) * blockDim.x + threadIdx.x;
+  const i64 step = (i64)((int)gridDim.x - (nblk - 1)) * blockDim.x;
+  for (i64 e = first; e < total; e += step) {
     const i64 i = e / sz, c = e % sz;
-    if (i / NB > c / NB) A[(o + i) * ld + o + c] = Lout[(o + i) * ld + o + c];
+    const i64 bi = i / NB, bc = c / NB;
+    if (bi > bc) {
+      A[(o + i) * ld + o + c] = Lout[(o + i) * ld + o + c];
+    } else {
+      Linv[(o + i) * ld + o + c] = (bi == bc) ? Dinv[((o + i) / NB) * (NB * NB) + (i % NB) * NB + (c % NB)] : 0.f;
+    }
   }
 }
 
@@ -541,22 +614,6 @@ __global__ void k_orth_finish(int* __restrict__ os, int* __restrict__ status) {
     atomicOr(status, DION_STATUS_BREAKDOWN);
   } else {
     atomicOr(status, DION_STATUS_ILLCOND);
-  }
-}
-
-// The sz x sz diagonal square of Linv that starts at row/column o (a multiple of 64):
-// zero, except its 64 x 64 diagonal blocks, which are copied from Dinv.
-__global__ void k_linv_init(float* __restrict__ Linv, i64 ld, i64 o, i64 sz, const float* __restrict__ Dinv,
-                            const int* __restrict__ skip_flag, i64 wstride) {
-  Linv += (i64)blockIdx.y * wstride; Dinv += (i64)blockIdx.y * wstride;   // batched over blockIdx.y
-  pdl_enter();
-  if (skip_flag != nullptr && skip_flag[(i64)blockIdx.y * OS_SLOT_INTS] != 0) return;
-  const i64 total = sz * sz;
-  for (i64 e = (i64)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (i64)gridDim.x * blockDim.x) {
-    const i64 i = o + e / sz, c = o + e % sz;
-    float v = 0.f;
-    if (i / NB == c / NB) v = Dinv[(i / NB) * (NB * NB) + (i % NB) * NB + (c % NB)];
-    Linv[i * ld + c] = v;
   }
 }
 
