@@ -328,15 +328,29 @@ constexpr int CHOL_STEP_SMEM = 3 * NB * MMS * (int)sizeof(float);
 // rows above it:  X_im = -Dinv_i * sum_{k=m}^{i-1} L_ik X_km  with X_mm = Dinv_m  (64 x 64 blocks).
 // L_ik is read from Lsrc (the panels the steps have written), X_km from Linv (written by the CTAs of
 // earlier launches), the diagonal inverses from Dinv.  One CTA of 256 threads; smem holds two tiles.
+// The sum may be cut in two: INV_PARTIAL adds the terms k < k_end and leaves the bare sum in X_im's
+// place; INV_RESUME starts from that sum and adds the terms k >= k_begin (so that the last block row,
+// which is on the serial chain, has one term left when its last input arrives).
+enum : int { INV_WHOLE = 0, INV_PARTIAL = 1, INV_RESUME = 2 };
 __device__ __forceinline__ void inv_tile(const float* __restrict__ Lsrc, float* __restrict__ Linv, i64 ld,
-                                         const float* __restrict__ Dinv, i64 o, i64 sz, int i, int m, float* smem) {
+                                         const float* __restrict__ Dinv, i64 o, i64 sz, int i, int m, float* smem,
+                                         int part = INV_WHOLE, int k_cut = 0) {
   mm_t S0 = reinterpret_cast<mm_t>(smem);
   mm_t S1 = reinterpret_cast<mm_t>(smem + NB * MMS);
   const int tid = threadIdx.x, ty = tid >> 4, tx = tid & 15;
   const i64 ri = o + (i64)i * NB, cm = o + (i64)m * NB;
   const int rows_i = (int)((o + sz - ri < NB) ? (o + sz - ri) : NB);
   float acc[4][4] = {};
-  for (int k = m; k < i; ++k) {
+  if (part == INV_RESUME) {
+#pragma unroll
+    for (int a = 0; a < 4; ++a)
+#pragma unroll
+      for (int b = 0; b < 4; ++b)
+        acc[a][b] = (ty * 4 + a < rows_i) ? Linv[(ri + ty * 4 + a) * ld + cm + tx + 16 * b] : 0.f;
+  }
+  const int k_first = (part == INV_RESUME) ? k_cut : m;
+  const int k_last = (part == INV_PARTIAL) ? k_cut : i;      // exclusive
+  for (int k = k_first; k < k_last; ++k) {
     const i64 rk = o + (i64)k * NB;
     const float* Dk = Dinv + (rk / NB) * (NB * NB);
 #pragma unroll 4
@@ -348,6 +362,14 @@ __device__ __forceinline__ void inv_tile(const float* __restrict__ Lsrc, float* 
     __syncthreads();
     mm_nt_64(S0, S1, ty, tx, acc);
     __syncthreads();
+  }
+  if (part == INV_PARTIAL) {
+#pragma unroll
+    for (int a = 0; a < 4; ++a)
+#pragma unroll
+      for (int b = 0; b < 4; ++b)
+        if (ty * 4 + a < rows_i) Linv[(ri + ty * 4 + a) * ld + cm + tx + 16 * b] = acc[a][b];
+    return;
   }
   const float* Di = Dinv + (ri / NB) * (NB * NB);
 #pragma unroll
@@ -400,7 +422,10 @@ __global__ void __launch_bounds__(256) k_chol_step(float* __restrict__ A, i64 ld
     const int nt = (int)((sz + NB - 1) / NB) - 1 - j;
     const int ntri = nt * (nt + 1) / 2;
     if ((int)blockIdx.x >= ntri) {
-      inv_tile(Lout, Linv, ld, Dinv, o, sz, j, (int)blockIdx.x - ntri, chol_smem);
+      const int x = (int)blockIdx.x - ntri;
+      if (x < j) inv_tile(Lout, Linv, ld, Dinv, o, sz, j, x, chol_smem);
+      else       // last step: the last block row's sums over the rows that are already final (k < j)
+        inv_tile(Lout, Linv, ld, Dinv, o, sz, j + 1, x - j, chol_smem, INV_PARTIAL, j);
       return;
     }
   }
@@ -518,7 +543,9 @@ __global__ void __launch_bounds__(256) k_inv_finish(const float* __restrict__ Lo
   extern __shared__ __align__(16) float fin_smem[];
   const int nblk = (int)((sz + NB - 1) / NB);
   if ((int)blockIdx.x < nblk - 1) {
-    inv_tile(Lout, Linv, ld, Dinv, o, sz, nblk - 1, (int)blockIdx.x, fin_smem);
+    const int m = (int)blockIdx.x;
+    if (m < nblk - 2) inv_tile(Lout, Linv, ld, Dinv, o, sz, nblk - 1, m, fin_smem, INV_RESUME, nblk - 2);
+    else inv_tile(Lout, Linv, ld, Dinv, o, sz, nblk - 1, m, fin_smem);
     return;
   }
   const i64 total = sz * sz;
