@@ -387,12 +387,12 @@ int potrf_inner(StepCtx& s, i64 r, i64 o, i64 sz, int mode) {
                DinvP + (o / NB) * (NB * NB), gdiag + o, floor_rel, s.os, adaptive ? 1 : 0, status, s.wstride);
     DION_CHECK_LAUNCH(c);
   }
-  // one launch per block column: panel, trailing update and the next diagonal block; behind them, j CTAs
-  // that form block row j of the inverse of the square's factor (off the critical path)
+  // one launch per block column: panel, trailing update and the next diagonal block; behind them the CTAs
+  // that add one term to every unfinished block row of the inverse of the square's factor (j blocks in each
+  // of the rows j .. nblk-1), off the critical path
   for (int j = 0; j + 1 < nblk; ++j) {
     const int nt = nblk - 1 - j;
-    // in the last step also the last block row's sums over the rows that are final by then (j more CTAs)
-    const int extra = (j + 2 == nblk) ? 2 * j : j;
+    const int extra = (nblk - j) * j;
     dim3 grid((unsigned)(nt * (nt + 1) / 2 + extra), (unsigned)s.nb);
     launch_pdl(k_chol_step, grid, dim3(256), CHOL_STEP_SMEM, s.st, Gm, r, o, sz, j, Dinv, DinvP, Tbuf, Linv, gdiag, floor_rel,
                s.os, adaptive ? 1 : 0, status, s.wstride);

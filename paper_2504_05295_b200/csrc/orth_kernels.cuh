@@ -324,46 +324,39 @@ __device__ __forceinline__ void mm_nt_64(mm_t A, mm_t B, int ty, int tx, float (
 
 constexpr int CHOL_STEP_SMEM = 3 * NB * MMS * (int)sizeof(float);
 
-// Block (i, m), m < i, of the inverse X of the factor of the diagonal square [o, o+sz), from the block
-// rows above it:  X_im = -Dinv_i * sum_{k=m}^{i-1} L_ik X_km  with X_mm = Dinv_m  (64 x 64 blocks).
-// L_ik is read from Lsrc (the panels the steps have written), X_km from Linv (written by the CTAs of
-// earlier launches), the diagonal inverses from Dinv.  One CTA of 256 threads; smem holds two tiles.
-// The sum may be cut in two: INV_PARTIAL adds the terms k < k_end and leaves the bare sum in X_im's
-// place; INV_RESUME starts from that sum and adds the terms k >= k_begin (so that the last block row,
-// which is on the serial chain, has one term left when its last input arrives).
-enum : int { INV_WHOLE = 0, INV_PARTIAL = 1, INV_RESUME = 2 };
-__device__ __forceinline__ void inv_tile(const float* __restrict__ Lsrc, float* __restrict__ Linv, i64 ld,
-                                         const float* __restrict__ Dinv, i64 o, i64 sz, int i, int m, float* smem,
-                                         int part = INV_WHOLE, int k_cut = 0) {
+// The inverse X of the factor of the diagonal square [o, o+sz), 64 x 64 blocks:
+//   X_im = -Dinv_i * S_im,   S_im = sum_{k=m}^{i-1} L_ik X_km,   X_mm = Dinv_m   (m < i).
+// The sums are accumulated right-looking, one term per launch: as soon as block column kk of the factor
+// and block row kk of X are final, every later row adds its term k = kk,
+//   S_im (+)= L_{i,kk} X_{kk,m}   (the first term, m = kk, takes X_kk,kk = Dinv_kk),
+// and the row that is complete with it (i = kk + 1, `finish`) is multiplied by -Dinv_i.  S_im lives in
+// X_im's place in Linv until then.  L is read from Lsrc (the panels the steps have written).  One CTA of
+// 256 threads per block and launch: one 64^3 product, two for the finishing row; smem holds two tiles.
+__device__ __forceinline__ void inv_term(const float* __restrict__ Lsrc, float* __restrict__ Linv, i64 ld,
+                                         const float* __restrict__ Dinv, i64 o, i64 sz, int i, int m, int kk,
+                                         bool finish, float* smem) {
   mm_t S0 = reinterpret_cast<mm_t>(smem);
   mm_t S1 = reinterpret_cast<mm_t>(smem + NB * MMS);
   const int tid = threadIdx.x, ty = tid >> 4, tx = tid & 15;
-  const i64 ri = o + (i64)i * NB, cm = o + (i64)m * NB;
+  const i64 ri = o + (i64)i * NB, cm = o + (i64)m * NB, rk = o + (i64)kk * NB;
   const int rows_i = (int)((o + sz - ri < NB) ? (o + sz - ri) : NB);
-  float acc[4][4] = {};
-  if (part == INV_RESUME) {
+  const bool first = (m == kk);
+  const float* Dk = Dinv + (rk / NB) * (NB * NB);
+  float acc[4][4];
 #pragma unroll
-    for (int a = 0; a < 4; ++a)
+  for (int a = 0; a < 4; ++a)
 #pragma unroll
-      for (int b = 0; b < 4; ++b)
-        acc[a][b] = (ty * 4 + a < rows_i) ? Linv[(ri + ty * 4 + a) * ld + cm + tx + 16 * b] : 0.f;
-  }
-  const int k_first = (part == INV_RESUME) ? k_cut : m;
-  const int k_last = (part == INV_PARTIAL) ? k_cut : i;      // exclusive
-  for (int k = k_first; k < k_last; ++k) {
-    const i64 rk = o + (i64)k * NB;
-    const float* Dk = Dinv + (rk / NB) * (NB * NB);
+    for (int b = 0; b < 4; ++b)
+      acc[a][b] = (!first && ty * 4 + a < rows_i) ? Linv[(ri + ty * 4 + a) * ld + cm + tx + 16 * b] : 0.f;
 #pragma unroll 4
-    for (int l = 0; l < NB * NB / 256; ++l) {
-      const int e = tid + l * 256, rr = e / NB, cc = e % NB;
-      S0[rr][cc] = (rr < rows_i) ? Lsrc[(ri + rr) * ld + rk + cc] : 0.f;
-      S1[cc][rr] = (k == m) ? Dk[e] : Linv[(rk + rr) * ld + cm + cc];   // transposed: the product below is A * B^T
-    }
-    __syncthreads();
-    mm_nt_64(S0, S1, ty, tx, acc);
-    __syncthreads();
+  for (int l = 0; l < NB * NB / 256; ++l) {
+    const int e = tid + l * 256, rr = e / NB, cc = e % NB;
+    S0[rr][cc] = (rr < rows_i) ? Lsrc[(ri + rr) * ld + rk + cc] : 0.f;
+    S1[cc][rr] = first ? Dk[e] : Linv[(rk + rr) * ld + cm + cc];   // transposed: the product below is A * B^T
   }
-  if (part == INV_PARTIAL) {
+  __syncthreads();
+  mm_nt_64(S0, S1, ty, tx, acc);
+  if (!finish) {
 #pragma unroll
     for (int a = 0; a < 4; ++a)
 #pragma unroll
@@ -371,6 +364,7 @@ __device__ __forceinline__ void inv_tile(const float* __restrict__ Lsrc, float* 
         if (ty * 4 + a < rows_i) Linv[(ri + ty * 4 + a) * ld + cm + tx + 16 * b] = acc[a][b];
     return;
   }
+  __syncthreads();
   const float* Di = Dinv + (ri / NB) * (NB * NB);
 #pragma unroll
   for (int a = 0; a < 4; ++a)
@@ -417,15 +411,16 @@ __global__ void __launch_bounds__(256) k_chol_step(float* __restrict__ A, i64 ld
   if (adaptive && os[OS_DONE] != 0) return;
   extern __shared__ __align__(16) float chol_smem[];
   {
-    // the CTAs behind the trailing blocks: block row j of the inverse of the square's factor (its
-    // inputs, the rows above and the diagonal inverse of block j, are final since the last launch)
-    const int nt = (int)((sz + NB - 1) / NB) - 1 - j;
+    // the CTAs behind the trailing blocks: block column j - 1 of the factor and block row j - 1 of the
+    // square's inverse are final since the last launch; every row i >= j of the inverse adds that term
+    // (j blocks per row), and row j is complete with it
+    const int nblk = (int)((sz + NB - 1) / NB);
+    const int nt = nblk - 1 - j;
     const int ntri = nt * (nt + 1) / 2;
     if ((int)blockIdx.x >= ntri) {
       const int x = (int)blockIdx.x - ntri;
-      if (x < j) inv_tile(Lout, Linv, ld, Dinv, o, sz, j, x, chol_smem);
-      else       // last step: the last block row's sums over the rows that are already final (k < j)
-        inv_tile(Lout, Linv, ld, Dinv, o, sz, j + 1, x - j, chol_smem, INV_PARTIAL, j);
+      const int i = j + x / j, m = x % j;
+      inv_term(Lout, Linv, ld, Dinv, o, sz, i, m, j - 1, i == j, chol_smem);
       return;
     }
   }
@@ -528,8 +523,8 @@ __global__ void __launch_bounds__(256) k_chol_step(float* __restrict__ A, i64 ld
   }
 }
 
-// After the last k_chol_step of a square [o, o+sz): the first CTAs form the last block row of the
-// inverse of the factor (inv_tile); the others move the factor's blocks below the block diagonal from
+// After the last k_chol_step of a square [o, o+sz): the first CTAs complete the last block row of the
+// inverse of the factor (inv_term); the others move the factor's blocks below the block diagonal from
 // Lout into A, put the diagonal inverses into Linv and clear Linv above the block diagonal.
 constexpr int INV_FINISH_SMEM = 2 * NB * MMS * (int)sizeof(float);
 __global__ void __launch_bounds__(256) k_inv_finish(const float* __restrict__ Lout, float* __restrict__ A,
@@ -542,10 +537,8 @@ __global__ void __launch_bounds__(256) k_inv_finish(const float* __restrict__ Lo
   if (skip_flag != nullptr && skip_flag[(i64)blockIdx.y * OS_SLOT_INTS] != 0) return;
   extern __shared__ __align__(16) float fin_smem[];
   const int nblk = (int)((sz + NB - 1) / NB);
-  if ((int)blockIdx.x < nblk - 1) {
-    const int m = (int)blockIdx.x;
-    if (m < nblk - 2) inv_tile(Lout, Linv, ld, Dinv, o, sz, nblk - 1, m, fin_smem, INV_RESUME, nblk - 2);
-    else inv_tile(Lout, Linv, ld, Dinv, o, sz, nblk - 1, m, fin_smem);
+  if ((int)blockIdx.x < nblk - 1) {   // the last row's last term (block column nblk - 2), and its finish
+    inv_term(Lout, Linv, ld, Dinv, o, sz, nblk - 1, (int)blockIdx.x, nblk - 2, true, fin_smem);
     return;
   }
   const i64 total = sz * sz;
