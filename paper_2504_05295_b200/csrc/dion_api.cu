@@ -440,15 +440,27 @@ int potrf_trtri(StepCtx& s, i64 r, int mode, bool full_inverse,
       g.B = Linv + J0 * r + J0; g.b_sk = 1; g.b_sn = r; g.klimit = 1;
       g.C = ptmp; g.ldc = r; g.epi = EPI_STORE; g.skip_flag = skip; g.precise = precise;
       for (int m = 0; m < s.nb; ++m) DION_TRY(launch_gemm(s, for_matrix(s, g, m, true, true, true), m));
+      // With the solves on the second stream, the copy of Lpanel into the Gram buffer goes there too: its
+      // only readers are the solves of later block columns (queued behind it on that stream); the trailing
+      // update reads the temporary, so the copy leaves the serial chain.
+      const bool side_copy = after_block != nullptr && c->side != nullptr;
       {
+        cudaStream_t cst = s.st;
+        if (side_copy) {
+          cudaEvent_t e = c->side_ev[c->side_cursor];
+          c->side_cursor = (c->side_cursor + 1) % 32;
+          if (cudaEventRecord(e, s.st) != cudaSuccess || cudaStreamWaitEvent(c->side, e, 0) != cudaSuccess) return DION_ERR_CUDA;
+          cst = c->side;
+        }
         dim3 grid((unsigned)grid_for(c, rem * sz), (unsigned)s.nb);
-        launch_pdl(k_copy_block, grid, dim3(256), 0, s.st, ptmp, r, panel, r, rem, sz, skip, s.wstride);
+        launch_pdl(k_copy_block, grid, dim3(256), 0, cst, ptmp, r, panel, r, rem, sz, skip, s.wstride);
         DION_CHECK_LAUNCH(c);
       }
+      const float* lp = side_copy ? ptmp : panel;
       GemmArgs t = gemm_args();  // A22 -= Lpanel * Lpanel^T (lower tiles)
       t.M = rem; t.N = rem; t.K = sz;
-      t.A = panel; t.a_si = r; t.a_sk = 1;
-      t.B = panel; t.b_sk = 1; t.b_sn = r;
+      t.A = lp; t.a_si = r; t.a_sk = 1;
+      t.B = lp; t.b_sk = 1; t.b_sn = r;
       t.C = Gm + (J0 + sz) * r + (J0 + sz); t.ldc = r; t.epi = EPI_SUB; t.tri = TRI_LOWER; t.skip_flag = skip;
       t.precise = precise;
       for (int m = 0; m < s.nb; ++m) DION_TRY(launch_gemm(s, for_matrix(s, t, m, true, true, true), m));
