@@ -183,7 +183,9 @@ def test_grouped_equals_single_calls():
         assert rel(to_np64(X2), ref[1].X) <= TOL_FP32 and rel(to_np64(Q2), ref[1].Q) <= TOL_FP32
 
 
-@pytest.mark.parametrize("shape,orth", [((2560, 1536, 640), binding.ORTH_AUTO), ((1280, 1280, 1280), binding.ORTH_AUTO)])
+@pytest.mark.parametrize("shape,orth", [((2560, 1536, 640), binding.ORTH_AUTO), ((1280, 1280, 1280), binding.ORTH_AUTO),
+                                        # ragged: a second square of 188 columns (blocks of 64, 64, 60)
+                                        ((1400, 1100, 700), binding.ORTH_AUTO), ((3000, 2900, 700), binding.ORTH_AUTO)])
 def test_grouped_chain_above_512_columns_equals_single_calls(shape, orth):
     # r > 512: two-level Cholesky, blocked solves on the second stream, three matrices sharing every small launch
     m, n, r = shape
