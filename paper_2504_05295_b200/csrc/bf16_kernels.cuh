@@ -62,6 +62,43 @@ __global__ void __launch_bounds__(256) k_form_b16(const float* __restrict__ M, i
   }
 }
 
+// B32 = M + G in fp32, rows x cols (cols a multiple of 4), B32 dense with leading dimension cols: the sum the
+// fused operand formation of the contraction kernel computes, formed once per step where two products and the
+// error feedback read it.  One thread per 4 consecutive elements of a row; VEC as above.
+template <bool VEC>
+__global__ void __launch_bounds__(256) k_form_b32(const float* __restrict__ M, i64 ldm, const void* __restrict__ G,
+                                                  i64 ldg, int g_mode, i64 rows, i64 cols, float* __restrict__ out) {
+  pdl_enter();
+  const i64 per_row = cols / 4;
+  const i64 total = rows * per_row;
+  for (i64 e = (i64)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (i64)gridDim.x * blockDim.x) {
+    const i64 i = e / per_row, c = (e - i * per_row) * 4;
+    float4 v;
+    const float* mp = M + i * ldm + c;
+    if (VEC) v = __ldg(reinterpret_cast<const float4*>(mp));
+    else v = make_float4(mp[0], mp[1], mp[2], mp[3]);
+    if (g_mode == ADD_F32) {
+      const float* gp = reinterpret_cast<const float*>(G) + i * ldg + c;
+      float4 g;
+      if (VEC) g = __ldg(reinterpret_cast<const float4*>(gp));
+      else g = make_float4(gp[0], gp[1], gp[2], gp[3]);
+      v.x += g.x; v.y += g.y; v.z += g.z; v.w += g.w;
+    } else if (g_mode == ADD_BF16) {
+      const __nv_bfloat16* gp = reinterpret_cast<const __nv_bfloat16*>(G) + i * ldg + c;
+      if (VEC) {
+        const uint2 w = __ldg(reinterpret_cast<const uint2*>(gp));
+        const __nv_bfloat162 lo = *reinterpret_cast<const __nv_bfloat162*>(&w.x);
+        const __nv_bfloat162 hi = *reinterpret_cast<const __nv_bfloat162*>(&w.y);
+        v.x += __low2float(lo); v.y += __high2float(lo); v.z += __low2float(hi); v.w += __high2float(hi);
+      } else {
+        v.x += __bfloat162float(gp[0]); v.y += __bfloat162float(gp[1]);
+        v.z += __bfloat162float(gp[2]); v.w += __bfloat162float(gp[3]);
+      }
+    }
+    *reinterpret_cast<float4*>(out + i * cols + c) = v;
+  }
+}
+
 // out = bf16(src), rows x cols (cols a multiple of 8, src rows 16-byte aligned), out dense.
 // skip_flag (optional): nothing is written when *skip_flag != 0.
 __global__ void __launch_bounds__(256) k_to_bf16(const float* __restrict__ src, i64 lds, i64 rows, i64 cols,

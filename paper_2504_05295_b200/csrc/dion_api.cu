@@ -41,6 +41,7 @@ struct Layout {
   i64 P0, P1, R, Gram, Linv, Tbuf, Dinv, DinvP, part, cn_part, d, gdiag, scal, total;
   i64 Sk, SkV, SkW;         // randomized Cholesky QR: the two stacked panels [S P; P] and a solve temporary
   i64 B16, Q16, U16, R16;   // bf16-operand mode: bf16(M + G) and the bf16 copies of Q, U, R (offsets in floats)
+  i64 B32;                  // fp32 mode: M + G formed once per step (0: the products form it on the fly)
   i64 part_floats;
   int cn_chunks;
   i64 cn_rows;
@@ -63,6 +64,7 @@ struct dion_ctx {
   struct ProfRec { int phase; cudaEvent_t e0, e1; int64_t launches; };
   std::vector<ProfRec> prof_recs;
   // second stream for work that can run beside the serial Cholesky chain, and its fork/join events
+  bool form_sum = true;   // fp32 mode may keep M + G in scratch (off for the fixed-scratch entry point)
   cudaStream_t side = nullptr;
   cudaEvent_t side_ev[32] = {};
   int side_cursor = 0;
@@ -78,6 +80,17 @@ void colnorm_plan(i64 rows, i64 r, int sm, int* chunks, i64* rows_per) {
   if (per < 32) per = 32;
   *rows_per = per;
   *chunks = (int)((rows + per - 1) / per);
+}
+
+// fp32 mode on the tensor engine, tensor-bound ranks: M + G is formed once per step in scratch (12 bytes per
+// element) and P, R and the error feedback read it.  Forming it inside the two products costs their converter
+// warps a second tile and a rewrite of the "hi" half (those products ran 25-30 % slower than the two that read
+// plain operands); at rank fractions below 1/8 the gain no longer pays for the extra pass (measured at 1/16), and
+// at low rank the products are HBM bound and the on-the-fly form moves fewer bytes.
+bool sum_in_scratch(const dion_ctx* c, i64 m, i64 n, i64 r) {
+  const i64 sd = (m < n) ? m : n;
+  return c->form_sum && c->cfg.precision == DION_PREC_FP32 && c->cfg.engine != DION_ENGINE_SIMT &&
+         m % 4 == 0 && n % 4 == 0 && m >= 128 && n >= 128 && r >= 64 && 8 * r >= sd;
 }
 
 Layout make_layout(const dion_ctx* c, i64 m, i64 n, i64 r) {
@@ -118,6 +131,8 @@ Layout make_layout(const dion_ctx* c, i64 m, i64 n, i64 r) {
     L.U16 = o; o += align64((big * r + 1) / 2);
     L.R16 = o; o += align64((big * r + 1) / 2);
   }
+  L.B32 = 0;
+  if (sum_in_scratch(c, m, n, r)) { L.B32 = o; o += align64(m * n); }
   L.total = o;
   return L;
 }
@@ -806,6 +821,9 @@ int step_batch(dion_ctx* c, const dion_matrix* const* list, int nb, float lr, cu
     return DION_OK;
   };
 
+  // fp32 mode: M + G kept in scratch for P, R and the error feedback (see sum_in_scratch)
+  const bool b32 = !d16 && s.tensor && s.L.B32 > 0;
+
   // P = (M + G) Q   (transposed form: (M + G)^T Q)
   {
   PhaseScope ps(c, st, DION_PHASE_P);
@@ -825,6 +843,16 @@ int step_batch(dion_ctx* c, const dion_matrix* const* list, int nb, float lr, cu
       p.ab16 = 1;
       p.A = (const float*)bf(b, s.L.B16); p.a_si = tr ? 1 : n; p.a_sk = tr ? n : 1;
       p.B = (const float*)bf(b, s.L.Q16); p.b_sk = r; p.b_sn = 1;
+    } else if (b32) {
+      const bool vec = !((uintptr_t)a->M & 15) && a->ldm % 4 == 0 &&
+                       (a->g_dtype == DION_BF16 ? (!((uintptr_t)a->G & 7) && a->ldg % 4 == 0)
+                                                : (!((uintptr_t)a->G & 15) && a->ldg % 4 == 0));
+      const int grid = grid_for(c, m * n / 4);
+      if (vec) launch_pdl(k_form_b32<true>, grid, dim3(256), 0, st, (const float*)a->M, a->ldm, a->G, a->ldg, g_mode(a), m, n, s.W(b, s.L.B32));
+      else launch_pdl(k_form_b32<false>, grid, dim3(256), 0, st, (const float*)a->M, a->ldm, a->G, a->ldg, g_mode(a), m, n, s.W(b, s.L.B32));
+      DION_CHECK_LAUNCH(c);
+      p.A = s.W(b, s.L.B32); p.a_si = tr ? 1 : n; p.a_sk = tr ? n : 1;
+      p.B = (const float*)a->Q; p.b_sk = a->ldq; p.b_sn = 1;
     } else {
       p.A = (const float*)a->M; p.a_si = tr ? 1 : a->ldm; p.a_sk = tr ? a->ldm : 1;
       p.A2 = a->G; p.a2_si = tr ? 1 : a->ldg; p.a2_sk = tr ? a->ldg : 1; p.a2_mode = g_mode(a);
@@ -859,6 +887,9 @@ int step_batch(dion_ctx* c, const dion_matrix* const* list, int nb, float lr, cu
       w.ab16 = 1;
       w.A = (const float*)bf(b, s.L.B16); w.a_si = tr ? n : 1; w.a_sk = tr ? 1 : n;
       w.B = (const float*)bf(b, s.L.U16); w.b_sk = r; w.b_sn = 1;
+    } else if (b32) {
+      w.A = s.W(b, s.L.B32); w.a_si = tr ? n : 1; w.a_sk = tr ? 1 : n;
+      w.B = s.W(b, U_off); w.b_sk = r; w.b_sn = 1;
     } else {
       w.A = (const float*)a->M; w.a_si = tr ? a->ldm : 1; w.a_sk = tr ? 1 : a->ldm;
       w.A2 = a->G; w.a2_si = tr ? a->ldg : 1; w.a2_sk = tr ? 1 : a->ldg; w.a2_mode = g_mode(a);
@@ -885,8 +916,9 @@ int step_batch(dion_ctx* c, const dion_matrix* const* list, int nb, float lr, cu
       e.A = s.W(b, tr ? s.L.R : U_off); e.a_si = r; e.a_sk = 1;
       e.B = s.W(b, tr ? U_off : s.L.R); e.b_sk = 1; e.b_sn = r;
     }
-    e.C = (float*)a->M; e.ldc = a->ldm; e.epi = EPI_ADD2_SUB;
-    e.C2 = a->G; e.ldc2 = a->ldg; e.c2_mode = g_mode(a);
+    e.C = (float*)a->M; e.ldc = a->ldm;
+    if (b32) { e.epi = EPI_C2_SUB; e.C2 = s.W(b, s.L.B32); e.ldc2 = n; e.c2_mode = ADD_F32; }
+    else { e.epi = EPI_ADD2_SUB; e.C2 = a->G; e.ldc2 = a->ldg; e.c2_mode = g_mode(a); }
     e.alpha = 1.f - c->cfg.mu;
     e.skip_flag = s.OS(b) + OS_FAIL;
     DION_TRY(launch_gemm(s, e, b));
@@ -1439,6 +1471,7 @@ extern "C" int dion_step_noalloc(const dion_matrix* a, float lr, float mu, float
   c.launches = 0;
   c.prof_on = false;
   c.prof_used = 0;
+  c.form_sum = false;
   const size_t need = (size_t)make_layout(&c, a->m, a->n, a->r).total * sizeof(float);
   if (need > c.ws_bytes) return DION_ERR_TOO_LARGE;
   // The array keeps what the previous call left: clear the status word and counters.
