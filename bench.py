@@ -35,9 +35,12 @@ UNIT = "ms"
 MU, ETA, EPS = 0.95, 0.01, 1e-8
 FFMA_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12     # 148 SMs x 128 FMA lanes x 2 flop x max clock
 # DRAM bytes (read + write) of the four large k_gemm_umma launches of a 4096^2 / r = 1024 step in one ncu
-# capture (profiles/k_gemm_umma_tma_4096sq_r1024.md) over their algorithmic bytes: 653.4 MB / 738.3 MB.
+# capture (profiles/k_gemm_umma_tma_4096sq_r1024.md) over their algorithmic bytes: 445.6 MB / 738.3 MB.  At this
+# rank fraction the library keeps M + G in scratch, so P, R and the error feedback read 4 bytes per element where
+# the algorithmic model counts M and G (the pass that forms the sum, 201 MB here, is another kernel); with the sum
+# formed inside the products (rank fractions below 1/8) the same ratio was 0.885.
 # Traffic grows in proportion to the matrix sizes, so the ratio scales the algorithmic bytes of any workload.
-NCU_TRAFFIC_RATIO = 0.885
+NCU_TRAFFIC_RATIO = 0.604
 
 
 def load_peaks():
