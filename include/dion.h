@@ -67,8 +67,15 @@ typedef enum { DION_PREC_FP32 = 0, DION_PREC_BF16_OPERANDS = 1 } dion_precision;
 
 /* Orthonormalize (Section 3.2 and the appendix on Cholesky QR).
  * DION_ORTH_AUTO:        CholeskyQR2 when 4 r <= min(m, n), else the adaptive rounds.
- * DION_ORTH_CHOLQR2:     two rounds of Cholesky QR (cond(P) up to about 4e3); a
- *                        non-positive pivot cancels the step (DION_STATUS_BREAKDOWN).
+ * DION_ORTH_CHOLQR2:     two rounds of Cholesky QR (cond(P) up to about 4e3).  A pivot that
+ *                        is not positive is the paper's "CQR failure ... fall back to QR"
+ *                        (appendix on Cholesky QR): the library keeps the panel and, in the
+ *                        same call and without a host round trip, one more launch
+ *                        orthonormalizes it column by column (classical Gram-Schmidt twice:
+ *                        the same thin-QR factor); that launch returns at once when no
+ *                        pivot failed.  Counted by dion_get_fallbacks.  Only a panel that
+ *                        is rank deficient to fp32 accuracy (a column shrinking below 2e-6
+ *                        of its norm) still cancels the step (DION_STATUS_BREAKDOWN).
  *                        The Gram matrix of the second round doubles as a measurement of
  *                        the first: if max |U1^T U1 - I| <= 3e-5 the rest of the second
  *                        round is skipped on the device (well-conditioned panels).
@@ -116,9 +123,11 @@ enum {
 
 /* Bits of the device status word (dion_get_status). */
 enum {
-  DION_STATUS_BREAKDOWN = 1,  /* a Cholesky pivot was <= 0 or not finite: the step
-                                 that saw it left X, M and Q unchanged            */
-  DION_STATUS_NONFINITE = 2,  /* a column norm of R was not finite                 */
+  DION_STATUS_BREAKDOWN = 1,  /* the panel was rank deficient (a Cholesky pivot <= 0 that the
+                                 fallback could not cure either): the step that saw it left
+                                 X, M and Q unchanged                              */
+  DION_STATUS_NONFINITE = 2,  /* NaN or Inf in M, G or Q (seen in the trace of the panel's Gram
+                                 matrix: the step is cancelled), or in a column norm of R */
   DION_STATUS_TIMEOUT = 4,    /* a bounded device-side wait ran out                */
   DION_STATUS_ILLCOND = 8     /* the adaptive rounds ran out before the panel was seen
                                  well conditioned; the result may be less accurate  */
@@ -252,6 +261,11 @@ int dion_profile_read(dion_ctx* ctx, float* ms, int64_t* launches);
  * device are not counted. */
 int dion_get_orth_rounds(dion_ctx* ctx, void* cuda_stream, int64_t* rounds);
 
+/* Synchronises `cuda_stream`, then reports and clears the number of matrices whose CholeskyQR2
+ * broke down and was redone by the device-side fallback since the last call (the paper reports
+ * under 1 % of calls in training). */
+int dion_get_fallbacks(dion_ctx* ctx, void* cuda_stream, int64_t* fallbacks);
+
 /* Number of kernel launches issued by this context so far (host counter). */
 int64_t dion_launch_count(const dion_ctx* ctx);
 
@@ -282,7 +296,10 @@ int64_t dion_launch_count(const dion_ctx* ctx);
  *     4 * (3 * max(m,n) * r + 3 * r * r) bytes plus 10 MiB of fixed buffers; for
  *     example 2048 x 2048 with r = 128 fits, 4096 x 4096 with r = 1024 does not.
  *   - The first call on a device looks up the array's device address and the
- *     device's attributes.  Make that first call outside any stream capture.
+ *     device's attributes and has every kernel of the launch chain loaded.  Make
+ *     that first call outside any stream capture.  The set-up is guarded by a
+ *     mutex, so first calls from several host threads are safe on the host side
+ *     (their kernels still share the one array, see the next rule).
  *   - All calls share the one array, which keeps whatever the previous call left
  *     in it; each call clears the words that must start at zero.  Two calls whose
  *     kernels overlap on the GPU (different streams, or several host threads) race

@@ -137,6 +137,45 @@ def step(X, M, G, Q, mu: float, eta: float, eps: float = 1e-8) -> StepResult:
     return StepResult(X, M, Q, d, P, U, R, rc)
 
 
+def step_rows(X, M, G, Q, rows, mu: float, eta: float, eps: float = 1e-8):
+    """The Dion step (Algorithm 1 + 2) with its two m x n outputs formed for the given
+    rows only, for matrices too large to run ``step`` on: B = M + G; P = B V; U = Householder
+    thin-QR factor of P (positive diagonal); W = B^T U; V_new = ColNorm(W); then, for each
+    requested row i, M_new[i] = B[i] - (1 - mu) U[i] W^T and X_new[i] = X[i] - eta sqrt(m/n)
+    U[i] V_new^T.  The factors are those of the whole matrix; only the rank-r outer products
+    are restricted to the rows.  The two large contractions are library matrix products in
+    float64.  Returns (X_rows, M_rows, V_new, d)."""
+    X = _f64(X); M = _f64(M); G = _f64(G); Q = _f64(Q)
+    m, n = X.shape
+    rows = np.asarray(rows, dtype=np.int64)
+    B = M + G
+    P = B @ Q
+    U, _ = householder_qr(P)
+    W = B.T @ U
+    Qn, d = colnorm(W, eps)
+    Ur = U[rows]
+    Mr = B[rows] - (1.0 - mu) * (Ur @ W.T)
+    Xr = X[rows] - eta * np.sqrt(m / n) * (Ur @ Qn.T)
+    return Xr, Mr, Qn, d
+
+
+def step_given_panel(X, M, G, Q, P, mu: float, eta: float, eps: float = 1e-8) -> StepResult:
+    """The Dion step (Algorithm 1 + 2) from PowerIter1's second line on, with the panel P handed in
+    by the caller instead of being formed as B V: U = Householder thin-QR factor of P, W = B^T U,
+    M_new = B - (1 - mu) U W^T, V_new = ColNorm(W), X_new = X - eta sqrt(m/n) U V_new^T.
+    With P = (M + G) Q it is ``step``.  Tests use it to measure how far the float64 rule itself moves
+    when P carries the rounding error of a float32 product (the rule's own conditioning)."""
+    X = _f64(X); M = _f64(M); G = _f64(G); Q = _f64(Q); P = _f64(P)
+    m, n = X.shape
+    B = M + G
+    U, _ = householder_qr(P)
+    W = B.T @ U
+    Qn, d = colnorm(W, eps)
+    Mn = B - (1.0 - mu) * (U @ W.T)
+    Xn = X - eta * np.sqrt(m / n) * (U @ Qn.T)
+    return StepResult(Xn, Mn, Qn, d, P, U, W, 0)
+
+
 def step_transposed(X, M, G, Q, mu: float, eta: float, eps: float = 1e-8) -> StepResult:
     """One Dion step in the transposed form (Section 4.3, "other variants": the power
     iteration runs on M^T).  By definition this is the standard step on the transposed

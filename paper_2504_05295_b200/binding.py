@@ -24,7 +24,7 @@ STATUS_BREAKDOWN, STATUS_NONFINITE, STATUS_TIMEOUT, STATUS_ILLCOND = 1, 2, 4, 8
 
 EXPORTS = ["dion_default_config", "dion_init", "dion_step", "dion_step_grouped", "dion_lazy_step",
            "dion_workspace_bytes", "dion_get_status", "dion_launch_count", "dion_destroy",
-           "dion_strerror", "dion_profile_enable", "dion_profile_read", "dion_get_orth_rounds",
+           "dion_strerror", "dion_profile_enable", "dion_profile_read", "dion_get_orth_rounds", "dion_get_fallbacks",
            "dion_step_noalloc", "dion_noalloc_scratch_limit", "dion_dp_project", "dion_dp_factor",
            "dion_dp_finish"]
 PHASES = ["P", "ORTH", "R", "EF", "COLNORM", "X", "ORTH_GEMM"]
@@ -87,6 +87,8 @@ def load_library() -> ctypes.CDLL:
     lib.dion_profile_read.restype = ci
     lib.dion_get_orth_rounds.argtypes = [vp, vp, ctypes.POINTER(i64)]
     lib.dion_get_orth_rounds.restype = ci
+    lib.dion_get_fallbacks.argtypes = [vp, vp, ctypes.POINTER(i64)]
+    lib.dion_get_fallbacks.restype = ci
     lib.dion_step_noalloc.argtypes = [ctypes.POINTER(DionMatrix), f32, f32, f32, vp]
     lib.dion_step_noalloc.restype = ci
     lib.dion_noalloc_scratch_limit.argtypes = []
@@ -267,6 +269,12 @@ class Dion:
         """Adaptive Cholesky QR rounds executed since the last call (synchronises)."""
         n = ctypes.c_int64(0)
         _check(self._lib.dion_get_orth_rounds(self._ctx, _stream_ptr(stream), ctypes.byref(n)))
+        return int(n.value)
+
+    def fallbacks(self, stream=None) -> int:
+        """Matrices redone by the device-side fallback of CholeskyQR2 since the last call (synchronises)."""
+        n = ctypes.c_int64(0)
+        _check(self._lib.dion_get_fallbacks(self._ctx, _stream_ptr(stream), ctypes.byref(n)))
         return int(n.value)
 
     def launch_count(self) -> int:

@@ -1,4 +1,5 @@
-// bf16-operand mode: the operands of the four large contractions as bf16 arrays in scratch.
+// Operand preparation in scratch: bf16(M + G) and bf16 copies (bf16-operand mode), M + G in fp32, and
+// TF32-rounded copies of the factors of the weight update (fp32 mode).
 #pragma once
 
 #include "dion_common.cuh"
@@ -114,6 +115,29 @@ __global__ void __launch_bounds__(256) k_to_bf16(const float* __restrict__ src, 
     uint4 o;
     o.x = pack_bf16x2(a.x, a.y); o.y = pack_bf16x2(a.z, a.w);
     o.z = pack_bf16x2(b.x, b.y); o.w = pack_bf16x2(b.z, b.w);
+    *reinterpret_cast<uint4*>(out + i * cols + c) = o;
+  }
+}
+
+// out = src with every value rounded to the nearest TF32 number (10 explicit mantissa bits, ties away
+// from zero), rows x cols (cols a multiple of 4, src rows 16-byte aligned), out dense.  The tensor core
+// truncates an fp32 operand to TF32 when it reads it; on pre-rounded values that truncation is exact, so a
+// single-pass TF32 product of such arrays carries an unbiased operand error of at most 2^-11 relative.
+// skip_flag (optional): nothing is written when *skip_flag != 0.
+__global__ void __launch_bounds__(256) k_round_tf32(const float* __restrict__ src, i64 lds, i64 rows, i64 cols,
+                                                    float* __restrict__ out, const int* __restrict__ skip_flag) {
+  pdl_enter();
+  if (skip_flag != nullptr && *skip_flag != 0) return;
+  const i64 per_row = cols / 4;
+  const i64 total = rows * per_row;
+  for (i64 e = (i64)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (i64)gridDim.x * blockDim.x) {
+    const i64 i = e / per_row, c = (e - i * per_row) * 4;
+    const float4 a = *reinterpret_cast<const float4*>(src + i * lds + c);
+    uint4 o;
+    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(o.x) : "f"(a.x));
+    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(o.y) : "f"(a.y));
+    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(o.z) : "f"(a.z));
+    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(o.w) : "f"(a.w));
     *reinterpret_cast<uint4*>(out + i * cols + c) = o;
   }
 }

@@ -3,7 +3,9 @@
 // directory; the host code only validates and launches.
 #include <math.h>
 #include <stdlib.h>
+#include <atomic>
 #include <functional>
+#include <mutex>
 #include <new>
 #include <string.h>
 #include <vector>
@@ -42,6 +44,8 @@ struct Layout {
   i64 Sk, SkV, SkW;         // randomized Cholesky QR: the two stacked panels [S P; P] and a solve temporary
   i64 B16, Q16, U16, R16;   // bf16-operand mode: bf16(M + G) and the bf16 copies of Q, U, R (offsets in floats)
   i64 B32;                  // fp32 mode: M + G formed once per step (0: the products form it on the fly)
+  i64 Psave;                // CholeskyQR2: the panel as the product wrote it, kept for the fallback (0: none)
+  i64 fb_part, fb_h, fb_n;  // fallback kernel: partial dot products (SMs x r), their sums (r), partial norms (SMs)
   i64 part_floats;
   int cn_chunks;
   i64 cn_rows;
@@ -93,6 +97,13 @@ bool sum_in_scratch(const dion_ctx* c, i64 m, i64 n, i64 r) {
          m % 4 == 0 && n % 4 == 0 && m >= 128 && n >= 128 && r >= 64 && 8 * r >= sd;
 }
 
+// A step whose orthonormalization may resolve to CholeskyQR2 keeps the panel for the device-side fallback.
+bool may_fallback(const dion_ctx* c, i64 m, i64 n, i64 r) {
+  const i64 sd = (m < n) ? m : n;
+  const int o = c->cfg.orth;
+  return o == DION_ORTH_CHOLQR2 || ((o == DION_ORTH_AUTO || o == DION_ORTH_RCQR) && 4 * r <= sd);
+}
+
 Layout make_layout(const dion_ctx* c, i64 m, i64 n, i64 r) {
   Layout L;
   const i64 big = (m > n) ? m : n;
@@ -133,6 +144,13 @@ Layout make_layout(const dion_ctx* c, i64 m, i64 n, i64 r) {
   }
   L.B32 = 0;
   if (sum_in_scratch(c, m, n, r)) { L.B32 = o; o += align64(m * n); }
+  L.Psave = L.fb_part = L.fb_h = L.fb_n = 0;
+  if (may_fallback(c, m, n, r)) {
+    L.Psave = o; o += align64(big * r);
+    L.fb_part = o; o += align64((i64)c->sm_count * r);
+    L.fb_h = o; o += align64(r);
+    L.fb_n = o; o += align64(c->sm_count);
+  }
   L.total = o;
   return L;
 }
@@ -264,6 +282,7 @@ struct StepCtx {
   const dion_matrix* const* list = nullptr;   // the matrices of the chain (sketch pointers of the RCQR mode)
   i64 wt_off = -1;        // >= 0: scratch offset of the blocked solves' rows x 512 temporary (default: the R panel)
   bool no_split = false;  // launches on the side stream: the split-K scratch belongs to the main stream
+  bool quiet_fail = false;  // a failed pivot only sets the step's fail flag: the fallback kernel follows
   float* W(int b, i64 off) const { return ws + (i64)b * wstride + off; }
   int* OS(int b) const { return os + (i64)b * OS_SLOT_INTS; }
 };
@@ -392,7 +411,7 @@ int potrf_inner(StepCtx& s, i64 r, i64 o, i64 sz, int mode) {
   float* Linv = s.ws + s.L.Linv;
   float* Tbuf = s.ws + s.L.Tbuf;
   const float* gdiag = s.ws + s.L.gdiag;
-  int* status = c->dev_ints;
+  int* status = s.quiet_fail ? nullptr : c->dev_ints;
   const int* skip = adaptive ? (s.os + OS_DONE) : nullptr;
   const float floor_rel = (mode == RM_ADAPTIVE) ? FLOOR_REL : 0.f;
   const int nblk = (int)((sz + NB - 1) / NB);
@@ -503,7 +522,7 @@ int cholqr_round(StepCtx& s, i64 pin_off, i64 pout_off, i64 rows, i64 r, int mod
   g.C = s.ws + s.L.Gram; g.ldc = r; g.epi = EPI_STORE; g.tri = TRI_LOWER; g.skip_flag = adaptive ? skip : nullptr; g.precise = rm_precise(mode) ? 1 : 0;
   for (int m = 0; m < s.nb; ++m) DION_TRY(launch_gemm(s, for_matrix(s, g, m, true, true, true), m));
   launch_pdl(k_round_begin, dim3((unsigned)(s.nb)), dim3(256), 0, s.st, s.ws + s.L.Gram, r, r, 0.f, s.ws + s.L.gdiag, s.ws + s.L.scal, s.os,
-                                        adaptive ? 1 : 0, s.wstride);
+                                        adaptive ? 1 : 0, s.wstride, c->dev_ints);
   DION_CHECK_LAUNCH(c);
   // Tall panels with r > 512: blocked triangular solve with the 512-column diagonal inverses
   // only (the levels of the triangular inverse above 512 are never formed).
@@ -692,17 +711,66 @@ int resolve_orth(const dion_ctx* c, i64 r, i64 short_dim) {
   return mode;
 }
 
-// Orthonormalize the rows x r panel in P0 of every matrix of the chain; *U_off is the
+// ... for a chain with (step) or without (Lazy-Dion, data-parallel calls) the sketches of the RCQR mode.
+int resolve_orth_for(const dion_ctx* c, i64 r, i64 short_dim, bool has_sketches) {
+  int mode = resolve_orth(c, r, short_dim);
+  if (mode == DION_ORTH_RCQR && !has_sketches) mode = (4 * r <= short_dim) ? DION_ORTH_CHOLQR2 : DION_ORTH_SHIFTED3;
+  return mode;
+}
+
+// Where the product that forms the panel writes it: CholeskyQR2 reads it from the save buffer (round one goes
+// Psave -> P1, round two P1 -> P0), so that the panel is still there if a pivot fails; every other mode works in P0.
+i64 panel_offset(const StepCtx& s, i64 r, i64 short_dim) {
+  const bool cq2 = resolve_orth_for(s.c, r, short_dim, s.list != nullptr) == DION_ORTH_CHOLQR2;
+  return (cq2 && s.L.Psave > 0) ? s.L.Psave : s.L.P0;
+}
+
+// The device-side fallback of CholeskyQR2 (k_cgs_fallback): one cooperative launch over the chain's matrices.
+int cgs_fallback(StepCtx& s, i64 pin_off, i64 pout_off, i64 rows, i64 r) {
+  dion_ctx* c = s.c;
+  i64 G = rows / 8;
+  if (G < 1) G = 1;
+  if (G > c->sm_count) G = c->sm_count;
+  const float* Pin = s.ws + pin_off;
+  float* U = s.ws + pout_off;
+  float* part = s.ws + s.L.fb_part;
+  float* hvec = s.ws + s.L.fb_h;
+  float* npart = s.ws + s.L.fb_n;
+  int* os = s.os;
+  int* status = c->dev_ints;
+  int* fallbacks = c->dev_ints + 3;
+  i64 ld = r, wstride = s.wstride;
+  int nb = s.nb;
+  long long limit = umma::SPIN_LIMIT_CYCLES;
+  void* args[] = {&Pin, &U, &ld, &rows, &r, &part, &hvec, &npart, &os, &status, &fallbacks, &wstride, &nb, &limit};
+  if (cudaLaunchCooperativeKernel((const void*)k_cgs_fallback, dim3((unsigned)G), dim3(256), args, 0, s.st) != cudaSuccess) {
+    cudaGetLastError();
+    return DION_ERR_CUDA;
+  }
+  c->launches++;
+  return DION_OK;
+}
+
+bool fallback_fits(const dion_ctx* c, i64 rows) {
+  return (rows + c->sm_count - 1) / c->sm_count <= CGS_MAX_ROWS_PER_CTA;
+}
+
+// Orthonormalize the rows x r panel at pin_off (= panel_offset) of every matrix of the chain; *U_off is the
 // scratch offset of the buffer that holds U afterwards.
-int orthonormalize(StepCtx& s, i64 rows, i64 r, i64 short_dim, i64* U_off) {
-  int mode = resolve_orth(s.c, r, short_dim);
-  if (mode == DION_ORTH_RCQR && s.list == nullptr)   // no sketches on this path (Lazy-Dion): as AUTO
-    mode = (4 * r <= short_dim) ? DION_ORTH_CHOLQR2 : DION_ORTH_SHIFTED3;
+int orthonormalize(StepCtx& s, i64 rows, i64 r, i64 short_dim, i64 pin_off, i64* U_off) {
+  const int mode = resolve_orth_for(s.c, r, short_dim, s.list != nullptr);
   if (mode == DION_ORTH_CHOLQR2) {
     // the first round with the accurate products; the second one only if the first one's result is
-    // not yet orthonormal to ORTH_TAU (measured on its Gram matrix)
-    DION_TRY(cholqr_round(s, s.L.P0, s.L.P1, rows, r, RM_FIRST));
-    DION_TRY(cholqr_round(s, s.L.P1, s.L.P0, rows, r, RM_CHECKED));
+    // not yet orthonormal to ORTH_TAU (measured on its Gram matrix).  A pivot that is not positive in
+    // either round (the paper's "CQR failure") raises the step's fail flag only; the fallback kernel then
+    // orthonormalizes the saved panel and clears the flag, or confirms the breakdown.
+    const bool fb = pin_off != s.L.P0 && fallback_fits(s.c, rows);
+    s.quiet_fail = fb;
+    int rc = cholqr_round(s, pin_off, s.L.P1, rows, r, RM_FIRST);
+    if (rc == DION_OK) rc = cholqr_round(s, s.L.P1, s.L.P0, rows, r, RM_CHECKED);
+    s.quiet_fail = false;
+    DION_TRY(rc);
+    if (fb) DION_TRY(cgs_fallback(s, pin_off, s.L.P0, rows, r));   // else: the failed pivot was reported as a breakdown
     *U_off = s.L.P0;
   } else if (mode == DION_ORTH_SHIFTED3) {
     DION_TRY(adaptive_rounds(s, s.L.P0, s.L.P1, rows, r, 0));
@@ -783,6 +851,41 @@ int begin_step(dion_ctx* c, const dion_matrix* a, int nb, cudaStream_t st, StepC
   return DION_OK;
 }
 
+// The weight update X <- X - alpha F1 F2^T in fp32 mode on the tensor engine (F1: m x r with leading dimension
+// ld1, F2: n x r with ld2; U Q^T, or Q U^T in the transposed form).  The update feeds nothing else, so its two
+// factors are rounded to TF32 once (to nearest: unbiased) into `r1`, `r2` (scratch, dense) and the product takes
+// one MMA per K step instead of three.  Returns false when the shape or the alignment does not qualify.
+bool x_single_pass(const StepCtx& s, const dion_matrix* a, const float* F1, i64 ld1, const float* F2, i64 ld2) {
+  const i64 m = a->m, n = a->n, r = a->r;
+  return s.tensor && s.c->cfg.precision == DION_PREC_FP32 && m >= 128 && n >= 64 && r >= 64 && m % 4 == 0 &&
+         n % 4 == 0 && r % 4 == 0 && !((uintptr_t)a->X & 15) && a->ldx % 4 == 0 && !((uintptr_t)F1 & 15) &&
+         ld1 % 4 == 0 && !((uintptr_t)F2 & 15) && ld2 % 4 == 0;
+}
+
+int x_update(StepCtx& s, int b, const dion_matrix* a, const float* F1, i64 ld1, const float* F2, i64 ld2, float* r1,
+             float* r2, float alpha, const int* skip) {
+  dion_ctx* c = s.c;
+  const i64 m = a->m, n = a->n, r = a->r;
+  GemmArgs x = gemm_args();
+  x.M = m; x.N = n; x.K = r;
+  if (x_single_pass(s, a, F1, ld1, F2, ld2)) {
+    launch_pdl(k_round_tf32, dim3((unsigned)grid_for(c, m * r / 4)), dim3(256), 0, s.st, F1, ld1, m, r, r1, skip);
+    DION_CHECK_LAUNCH(c);
+    launch_pdl(k_round_tf32, dim3((unsigned)grid_for(c, n * r / 4)), dim3(256), 0, s.st, F2, ld2, n, r, r2, skip);
+    DION_CHECK_LAUNCH(c);
+    x.tf32x1 = 1;
+    x.A = r1; x.a_si = r; x.a_sk = 1;
+    x.B = r2; x.b_sk = 1; x.b_sn = r;
+  } else {
+    x.A = F1; x.a_si = ld1; x.a_sk = 1;
+    x.B = F2; x.b_sk = 1; x.b_sn = ld2;
+  }
+  x.C = (float*)a->X; x.ldc = a->ldx; x.epi = EPI_SUB;
+  x.alpha = alpha;
+  x.skip_flag = skip;
+  return launch_gemm(s, x, b);
+}
+
 // The launch chain of one Dion step (Algorithm 1 + 2) on `nb` matrices of identical
 // (m, n, r), phase by phase.  Scratch must hold nb slices.
 int step_batch(dion_ctx* c, const dion_matrix* const* list, int nb, float lr, cudaStream_t st) {
@@ -825,6 +928,7 @@ int step_batch(dion_ctx* c, const dion_matrix* const* list, int nb, float lr, cu
   const bool b32 = !d16 && s.tensor && s.L.B32 > 0;
 
   // P = (M + G) Q   (transposed form: (M + G)^T Q)
+  const i64 pin_off = panel_offset(s, r, (m < n) ? m : n);
   {
   PhaseScope ps(c, st, DION_PHASE_P);
   for (int b = 0; b < nb; ++b) {
@@ -858,7 +962,7 @@ int step_batch(dion_ctx* c, const dion_matrix* const* list, int nb, float lr, cu
       p.A2 = a->G; p.a2_si = tr ? 1 : a->ldg; p.a2_sk = tr ? a->ldg : 1; p.a2_mode = g_mode(a);
       p.B = (const float*)a->Q; p.b_sk = a->ldq; p.b_sn = 1;
     }
-    p.C = s.W(b, s.L.P0); p.ldc = r; p.epi = EPI_STORE;
+    p.C = s.W(b, pin_off); p.ldc = r; p.epi = EPI_STORE;
     // an ill-conditioned panel amplifies the error of P: use the accurate product there
     p.precise = (!d16 && resolve_orth(c, r, (m < n) ? m : n) == DION_ORTH_SHIFTED3) ? 1 : 0;
     DION_TRY(launch_gemm(s, p, b));
@@ -870,7 +974,7 @@ int step_batch(dion_ctx* c, const dion_matrix* const* list, int nb, float lr, cu
   {
   PhaseScope ps(c, st, DION_PHASE_ORTH);
   s.in_orth = true;
-  const int rc_orth = orthonormalize(s, prow, r, (m < n) ? m : n, &U_off);
+  const int rc_orth = orthonormalize(s, prow, r, (m < n) ? m : n, pin_off, &U_off);
   s.in_orth = false;
   DION_TRY(rc_orth);
   }
@@ -937,26 +1041,29 @@ int step_batch(dion_ctx* c, const dion_matrix* const* list, int nb, float lr, cu
   // X <- X - lr sqrt(m/n) U Q^T   (transposed form: Q U^T)
   {
   PhaseScope ps(c, st, DION_PHASE_X);
+  const float x_alpha = lr * sqrtf((float)((double)m / (double)n));
   for (int b = 0; b < nb; ++b) {
     const dion_matrix* a = list[b];
-    GemmArgs x = gemm_args();
-    x.M = m; x.N = n; x.K = r;
     if (d16) {
+      GemmArgs x = gemm_args();
+      x.M = m; x.N = n; x.K = r;
       DION_TRY(to_bf16((const float*)a->Q, a->ldq, qrow, r, bf(b, s.L.Q16)));
       x.ab16 = 1;
       x.A = (const float*)bf(b, tr ? s.L.Q16 : s.L.U16); x.a_si = r; x.a_sk = 1;
       x.B = (const float*)bf(b, tr ? s.L.U16 : s.L.Q16); x.b_sk = 1; x.b_sn = r;
-    } else if (tr) {
-      x.A = (const float*)a->Q; x.a_si = a->ldq; x.a_sk = 1;
-      x.B = s.W(b, U_off); x.b_sk = 1; x.b_sn = r;
-    } else {
-      x.A = s.W(b, U_off); x.a_si = r; x.a_sk = 1;
-      x.B = (const float*)a->Q; x.b_sk = 1; x.b_sn = a->ldq;
+      x.C = (float*)a->X; x.ldc = a->ldx; x.epi = EPI_SUB;
+      x.alpha = x_alpha;
+      x.skip_flag = s.OS(b) + OS_FAIL;
+      DION_TRY(launch_gemm(s, x, b));
+      continue;
     }
-    x.C = (float*)a->X; x.ldc = a->ldx; x.epi = EPI_SUB;
-    x.alpha = lr * sqrtf((float)((double)m / (double)n));
-    x.skip_flag = s.OS(b) + OS_FAIL;
-    DION_TRY(launch_gemm(s, x, b));
+    // the rounded copies of the single-pass form go to the other panel buffer and to R's, both free by now
+    float* other = s.W(b, U_off == s.L.P0 ? s.L.P1 : s.L.P0);
+    float* rbuf = s.W(b, s.L.R);
+    const float* Uf = s.W(b, U_off);
+    const float* Qf = (const float*)a->Q;
+    if (tr) DION_TRY(x_update(s, b, a, Qf, a->ldq, Uf, r, rbuf, other, x_alpha, s.OS(b) + OS_FAIL));
+    else DION_TRY(x_update(s, b, a, Uf, r, Qf, a->ldq, other, rbuf, x_alpha, s.OS(b) + OS_FAIL));
   }
   launch_pdl(k_finish_step, dim3((unsigned)(nb)), dim3(1), 0, st, s.flag, c->dev_ints + 1);
   DION_CHECK_LAUNCH(c);
@@ -1033,11 +1140,12 @@ int lazy_one(dion_ctx* c, const dion_matrix* a, float lr, int refresh, cudaStrea
       z.B = R; z.b_sk = r; z.b_sn = 1;
       z.precise = precise;
     }
-    z.C = P0; z.ldc = r; z.epi = EPI_STORE;
+    const i64 pin_off = panel_offset(s, r, (m < n) ? m : n);
+    z.C = s.ws + pin_off; z.ldc = r; z.epi = EPI_STORE;
     DION_TRY(launch_gemm(s, z));
     i64 V_off = 0;
     s.in_orth = true;
-    const int rc_orth = orthonormalize(s, n, r, (m < n) ? m : n, &V_off);
+    const int rc_orth = orthonormalize(s, n, r, (m < n) ? m : n, pin_off, &V_off);
     s.in_orth = false;
     DION_TRY(rc_orth);
     const float* V = s.ws + V_off;
@@ -1266,11 +1374,12 @@ int dion_dp_factor(dion_ctx* ctx, const dion_matrix* a, float* PU, float* W, int
   DION_TRY(begin_step(ctx, a, 1, st, &s));
   const i64 m = a->m, n = a->n, r = a->r;
   dim3 grid((unsigned)grid_for(ctx, m * r), 1);
-  launch_pdl(k_copy_block, grid, dim3(256), 0, st, PU, r, s.ws + s.L.P0, r, m, r, nullptr, 0);
+  const i64 pin_off = panel_offset(s, r, (m < n) ? m : n);
+  launch_pdl(k_copy_block, grid, dim3(256), 0, st, PU, r, s.ws + pin_off, r, m, r, nullptr, 0);
   DION_CHECK_LAUNCH(ctx);
   i64 U_off = 0;
   s.in_orth = true;
-  const int rc = orthonormalize(s, m, r, (m < n) ? m : n, &U_off);
+  const int rc = orthonormalize(s, m, r, (m < n) ? m : n, pin_off, &U_off);
   s.in_orth = false;
   DION_TRY(rc);
   launch_pdl(k_copy_block, grid, dim3(256), 0, st, s.ws + U_off, r, PU, r, m, r, nullptr, 0);
@@ -1297,14 +1406,9 @@ int dion_dp_finish(dion_ctx* ctx, const dion_matrix* a, const float* U, const fl
   e.skip_flag = dp_flag;
   DION_TRY(launch_gemm(s, e, 0));
   DION_TRY(colnorm(s, 0, W, n, r, (float*)a->Q, a->ldq, a->colnorm_out, dp_flag));
-  GemmArgs x = gemm_args();      // X <- X - lr sqrt(m/n) U Q^T
-  x.M = m; x.N = n; x.K = r;
-  x.A = U; x.a_si = r; x.a_sk = 1;
-  x.B = (const float*)a->Q; x.b_sk = 1; x.b_sn = a->ldq;
-  x.C = (float*)a->X; x.ldc = a->ldx; x.epi = EPI_SUB;
-  x.alpha = lr * sqrtf((float)((double)m / (double)n));
-  x.skip_flag = dp_flag;
-  DION_TRY(launch_gemm(s, x, 0));
+  // X <- X - lr sqrt(m/n) U Q^T, as in dion_step (rounded copies in the two panel buffers of the scratch)
+  DION_TRY(x_update(s, 0, a, U, r, (const float*)a->Q, a->ldq, s.ws + s.L.P1, s.ws + s.L.R,
+                    lr * sqrtf((float)((double)m / (double)n)), dp_flag));
   launch_pdl(k_finish_step, dim3((unsigned)(1)), dim3(1), 0, st, dp_flag, ctx->dev_ints + 1);
   DION_CHECK_LAUNCH(ctx);
   return DION_OK;
@@ -1366,6 +1470,18 @@ int dion_get_orth_rounds(dion_ctx* ctx, void* cuda_stream, int64_t* rounds) {
   return DION_OK;
 }
 
+int dion_get_fallbacks(dion_ctx* ctx, void* cuda_stream, int64_t* fallbacks) {
+  if (ctx == nullptr || fallbacks == nullptr) return DION_ERR_INVALID;
+  if (cudaSetDevice(ctx->cfg.device) != cudaSuccess) return DION_ERR_CUDA;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  int host = 0;
+  if (cudaMemcpyAsync(&host, ctx->dev_ints + 3, sizeof(int), cudaMemcpyDeviceToHost, st) != cudaSuccess) return DION_ERR_CUDA;
+  if (cudaMemsetAsync(ctx->dev_ints + 3, 0, sizeof(int), st) != cudaSuccess) return DION_ERR_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return DION_ERR_CUDA;
+  *fallbacks = host;
+  return DION_OK;
+}
+
 int64_t dion_launch_count(const dion_ctx* ctx) { return ctx == nullptr ? 0 : ctx->launches; }
 
 void dion_destroy(dion_ctx* ctx) {
@@ -1413,18 +1529,46 @@ constexpr int NOALLOC_MAX_DEVICES = 64;
 static __device__ __align__(256) unsigned char g_noalloc_scratch[NOALLOC_SCRATCH_BYTES];
 
 struct NoallocDevice {
-  bool ready;
+  std::atomic<bool> ready;
   unsigned char* base;
   int sm_count;
 };
 NoallocDevice g_noalloc_dev[NOALLOC_MAX_DEVICES];
+std::mutex g_noalloc_mutex;
+
+template <typename K>
+bool touch_kernel(K kernel) {
+  cudaFuncAttributes fa;
+  if (cudaFuncGetAttributes(&fa, kernel) != cudaSuccess) { cudaGetLastError(); return false; }
+  return true;
+}
+
+// With lazy module loading a kernel's code is loaded at its first use, which may allocate device memory.
+// Asking for the attributes of every kernel the launch chain can reach loads them all at set-up (the
+// tensor-core variants are covered by configure_kernels, which sets an attribute on each).
+bool preload_kernels() {
+  bool ok = true;
+  ok = ok && touch_kernel(k_gemm_simt<128, 128, 8, 8, 8>) && touch_kernel(k_gemm_simt<64, 64, 16, 4, 4>);
+  ok = ok && touch_kernel(k_splitk_reduce) && touch_kernel(k_round_begin) && touch_kernel(k_potrf_diag);
+  ok = ok && touch_kernel(k_chol_step) && touch_kernel(k_inv_finish) && touch_kernel(k_round_end);
+  ok = ok && touch_kernel(k_orth_check) && touch_kernel(k_orth_decide) && touch_kernel(k_reset_rounds);
+  ok = ok && touch_kernel(k_orth_finish) && touch_kernel(k_cgs_fallback) && touch_kernel(k_copy_block);
+  ok = ok && touch_kernel(k_colsumsq_partial) && touch_kernel(k_colnorm_apply) && touch_kernel(k_copy_panel);
+  ok = ok && touch_kernel(k_latch_flag) && touch_kernel(k_finish_step) && touch_kernel(k_hh_reflector);
+  ok = ok && touch_kernel(k_hh_apply) && touch_kernel(k_set_identity) && touch_kernel(k_sign_fix);
+  ok = ok && touch_kernel(k_form_b16<true>) && touch_kernel(k_form_b16<false>) && touch_kernel(k_form_b32<true>);
+  ok = ok && touch_kernel(k_form_b32<false>) && touch_kernel(k_to_bf16) && touch_kernel(k_round_tf32);
+  return ok;
+}
 
 // First use on the current device: resolve the array's device address and read the
 // device attributes.  No allocation; must not run inside a stream capture.
 int noalloc_setup(int device, NoallocDevice** out) {
   if (device < 0 || device >= NOALLOC_MAX_DEVICES) return DION_ERR_INVALID;
   NoallocDevice* d = &g_noalloc_dev[device];
-  if (!d->ready) {
+  if (!d->ready.load(std::memory_order_acquire)) {
+    std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+    if (d->ready.load(std::memory_order_relaxed)) { *out = d; return DION_OK; }
     int major = 0, sms = 0;
     if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, device) != cudaSuccess ||
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device) != cudaSuccess) {
@@ -1437,10 +1581,10 @@ int noalloc_setup(int device, NoallocDevice** out) {
       cudaGetLastError();
       return DION_ERR_CUDA;
     }
-    if (configure_kernels() != DION_OK) return DION_ERR_CUDA;
+    if (configure_kernels() != DION_OK || !preload_kernels()) return DION_ERR_CUDA;
     d->base = (unsigned char*)ptr;
     d->sm_count = sms;
-    d->ready = true;
+    d->ready.store(true, std::memory_order_release);
   }
   *out = d;
   return DION_OK;
@@ -1499,11 +1643,10 @@ extern "C" int dion_debug_gemm(int engine, int precision, const dion_debug_gemm_
   g.B = a->B; g.b_sk = a->b_sk; g.b_sn = a->b_sn;
   g.C = a->C; g.ldc = a->ldc; g.epi = a->epi;
   g.C2 = a->C2; g.ldc2 = a->ldc2; g.c2_mode = a->c2_mode;
-  g.alpha = a->alpha; g.tri = a->tri; g.klimit = a->klimit; g.precise = a->precise; g.ab16 = a->ab16;
+  g.alpha = a->alpha; g.tri = a->tri; g.klimit = a->klimit; g.precise = a->precise; g.ab16 = a->ab16; g.tf32x1 = a->tf32x1;
   cudaStream_t st = (cudaStream_t)cuda_stream;
   if (engine == DION_ENGINE_TENSOR) {
-    const char* dbg = getenv("DION_DEBUG_GEMM");   // timing experiments of this hook only
-    const int rc = umma_try_launch(g, precision, sms, part, part_floats, status, st, dbg ? atoi(dbg) : 0);
+    const int rc = umma_try_launch(g, precision, sms, part, part_floats, status, st, a->variant);
     if (rc > 0) return DION_OK;
     return rc < 0 ? rc : DION_ERR_UNSUPPORTED;
   }

@@ -46,6 +46,8 @@ struct GemmArgs {
   const int* skip_flag;          // optional: if *skip_flag != 0 the kernel does nothing
   int precise;                   // tensor engine: keep the small split terms in their own accumulator
   int ab16;                      // tensor engine only: A and B point to bf16 arrays (strides in elements), no addend
+  int tf32x1;                    // tensor engine, fp32 mode: the operands' values fit TF32 already (k_round_tf32): one MMA
+                                 // per K step instead of the three-term split.  Ignored by the FMA engine.
 };
 
 // Programmatic dependent launch (the small kernels of the serial Cholesky chain): lets the next

@@ -22,6 +22,11 @@ typedef struct {
   int klimit;                                    /* 1: B(k,j) = 0 for k > j                */
   int precise;                                   /* 1: split accumulators (tensor engine)  */
   int ab16;                                      /* 1: A and B are bf16 arrays (tensor engine) */
+  int tf32x1;                                    /* 1: single-pass TF32 (tensor engine, fp32 mode; operands pre-rounded) */
+  int variant;                                   /* tensor engine: bit 0 operands through registers instead of TMA;
+                                                    bit 1 (with bit 0) one producer arrival is withheld and every wait
+                                                    has a 1 ms budget: the kernel must give up, set DION_STATUS_TIMEOUT
+                                                    in *status and return */
 } dion_debug_gemm_args;
 
 /* engine: 1 = fp32 FMA, 2 = tensor cores (returns DION_ERR_UNSUPPORTED if the

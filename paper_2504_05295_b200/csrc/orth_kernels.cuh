@@ -16,6 +16,7 @@ enum : int {
   OS_MINREL = 4,    // float bits: min over columns of pivot / original diagonal, current round
   OS_ROUNDS = 5,    // rounds that did work
   OS_MAXDEV = 6,    // float bits: max |G - I| over the lower triangle of a round's Gram matrix (CholeskyQR2 check)
+  OS_BARRIER = 7,   // arrival counter of the fallback kernel's grid-wide barriers (zero at the start of a step)
   OS_SLOT_INTS = 8
 };
 
@@ -23,9 +24,11 @@ enum : int {
 // shift = scale * trace(G) (fixed summation order) and resets the round statistics.
 // Batched: block b works on the matrix whose scratch starts b * wstride floats further and
 // whose state slot is b slots further.
+// A trace that is not finite means a NaN or Inf in M, G or Q (every entry of the Gram matrix sums over all
+// rows of the panel): the step is cancelled and DION_STATUS_NONFINITE raised.
 __global__ void k_round_begin(const float* __restrict__ G, i64 ld, i64 r, float scale,
                               float* __restrict__ gdiag, float* __restrict__ shift,
-                              int* __restrict__ os, int adaptive, i64 wstride) {
+                              int* __restrict__ os, int adaptive, i64 wstride, int* __restrict__ status) {
   pdl_enter();
   G += (i64)blockIdx.x * wstride; gdiag += (i64)blockIdx.x * wstride; shift += (i64)blockIdx.x * wstride;
   os += (i64)blockIdx.x * OS_SLOT_INTS;
@@ -47,6 +50,10 @@ __global__ void k_round_begin(const float* __restrict__ G, i64 ld, i64 r, float 
     *shift = red[0] * scale;
     os[OS_FLOORED] = 0;
     os[OS_MINREL] = 0x7f800000;  // +inf
+    if (!(fabsf(red[0]) < __int_as_float(0x7f800000))) {
+      os[OS_FAIL] = 1;
+      atomicOr(status, DION_STATUS_NONFINITE);
+    }
   }
 }
 
@@ -223,7 +230,7 @@ __device__ __forceinline__ void potrf_block(blk_t L, blk_t X, half_blk_t T, cons
       atomicMin(&os[OS_MINREL], __float_as_int(minrel));
     } else if (failed) {
       os[OS_FAIL] = 1;
-      atomicOr(status, DION_STATUS_BREAKDOWN);
+      if (status != nullptr) atomicOr(status, DION_STATUS_BREAKDOWN);   // nullptr: a fallback follows in the same step
     }
   }
 
@@ -634,6 +641,188 @@ __global__ void k_orth_finish(int* __restrict__ os, int* __restrict__ status) {
     atomicOr(status, DION_STATUS_BREAKDOWN);
   } else {
     atomicOr(status, DION_STATUS_ILLCOND);
+  }
+}
+
+// ---------------------------------------------------------------------------
+// Fallback of Cholesky QR, on the device: when a pivot of CholeskyQR2 was not positive (the panel is too
+// ill conditioned for the Gram matrix in fp32; the paper falls back to a QR factorization), the panel saved
+// before the first round is orthonormalized column by column with classical Gram-Schmidt applied twice
+// (the thin-QR factor with positive diagonal, like every other mode), in ONE cooperative launch that returns
+// at once when no matrix of the chain failed: no host round trip, no launches beyond this one.
+//
+// CTA c owns a block of rows of the panel and only ever touches its own rows of U; what crosses CTAs are the
+// partial dot products (part[c][k], summed in fixed CTA order into h[k]) and the partial squared norms,
+// separated by grid-wide barriers (5 per column).  Column j, pass p: h_k = sum_i U[i][k] U[i][j] for k < j
+// (pass 0 also k = j: the squared norm before orthogonalization), U[:, j] -= U[:, <j] h, then the norm and
+// the scaling.  A column whose norm falls below CGS_DEFLATE_REL of what it was is linearly dependent on its
+// predecessors to fp32 accuracy: the step is cancelled (OS_FAIL, DION_STATUS_BREAKDOWN) as before.
+// Every barrier wait is bounded; when one runs out the kernel gives up with DION_STATUS_TIMEOUT and the step
+// stays cancelled.
+// ---------------------------------------------------------------------------
+constexpr float CGS_DEFLATE_REL = 2e-6f;
+constexpr int CGS_PASSES = 2;
+constexpr int CGS_MAX_ROWS_PER_CTA = 1024;   // floats of shared memory for the CTA's piece of the current column
+
+__device__ __forceinline__ unsigned ld_acquire_u32(const unsigned* p) {
+  unsigned v;
+  asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+
+// Grid-wide barrier on a monotonic arrival counter: barrier number `epoch` (1, 2, ...) is passed when
+// epoch * gridDim.x arrivals have been counted.  Returns false when the wait ran out or an earlier one did.
+__device__ __forceinline__ bool cgs_grid_barrier(unsigned* counter, unsigned& epoch, long long limit, int* status,
+                                                 volatile int* s_dead) {
+  __syncthreads();
+  ++epoch;
+  if (threadIdx.x == 0 && !*s_dead) {
+    __threadfence();
+    atomicAdd(counter, 1u);
+    const unsigned target = epoch * gridDim.x;
+    const long long t0 = clock64();
+    while (ld_acquire_u32(counter) < target) {
+      if (clock64() - t0 > limit) {
+        *s_dead = 1;
+        atomicOr(status, DION_STATUS_TIMEOUT);
+        break;
+      }
+      __nanosleep(100);
+    }
+    __threadfence();
+  }
+  __syncthreads();
+  return *s_dead == 0;
+}
+
+__device__ __forceinline__ float cgs_block_sum(float v, float* red) {
+  const int tid = threadIdx.x;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  if ((tid & 31) == 0) red[tid >> 5] = v;
+  __syncthreads();
+  float t = 0.f;
+  if (tid < 8) t = red[tid];
+  if (tid < 32) {
+#pragma unroll
+    for (int o = 4; o > 0; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
+    if (tid == 0) red[8] = t;
+  }
+  __syncthreads();
+  const float out = red[8];
+  __syncthreads();
+  return out;
+}
+
+// Pin: the saved panel (rows x r, ld); U: where the orthonormal factor goes (ld).  part: gridDim.x * r floats,
+// hvec: r floats, npart: gridDim.x floats -- per matrix, wstride floats apart like every scratch offset.
+__global__ void __launch_bounds__(256) k_cgs_fallback(const float* __restrict__ Pin, float* __restrict__ U, i64 ld,
+                                                      i64 rows, i64 r, float* __restrict__ part, float* __restrict__ hvec,
+                                                      float* __restrict__ npart, int* __restrict__ os_base,
+                                                      int* __restrict__ status, int* __restrict__ fallbacks,
+                                                      i64 wstride, int nb, long long spin_limit) {
+  __shared__ float colj[CGS_MAX_ROWS_PER_CTA];
+  __shared__ float red[9];
+  __shared__ int s_dead;
+  __shared__ float s_val;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int G = (int)gridDim.x, c = (int)blockIdx.x;
+  const i64 rpc = (rows + G - 1) / G;
+  const i64 i0 = min(rows, (i64)c * rpc), i1 = min(rows, i0 + rpc);
+  const int nmy = (int)(i1 - i0);
+  for (int b = 0; b < nb; ++b) {
+    int* os = os_base + (i64)b * OS_SLOT_INTS;
+    if (os[OS_FAIL] == 0) continue;                 // written by an earlier launch: every CTA reads the same value
+    const float* Pb = Pin + (i64)b * wstride;
+    float* Ub = U + (i64)b * wstride;
+    float* partb = part + (i64)b * wstride;
+    float* hb = hvec + (i64)b * wstride;
+    float* nb_part = npart + (i64)b * wstride;
+    unsigned* counter = reinterpret_cast<unsigned*>(os + OS_BARRIER);
+    unsigned epoch = 0;
+    if (tid == 0) s_dead = 0;
+    __syncthreads();
+    bool ok = true, deficient = false;
+    for (i64 e = tid; e < (i64)nmy * r; e += 256) {
+      const i64 i = i0 + e / r, k = e % r;
+      Ub[i * ld + k] = Pb[i * ld + k];
+    }
+    __syncthreads();
+    for (i64 j = 0; j < r && ok && !deficient; ++j) {
+      for (int i = tid; i < nmy; i += 256) colj[i] = Ub[(i0 + i) * ld + j];
+      __syncthreads();
+      float before = 0.f;
+      for (int pass = 0; pass < CGS_PASSES && ok; ++pass) {
+        const i64 nk = j + (pass == 0 ? 1 : 0);     // pass 0: k = j is the squared norm before orthogonalization
+        for (i64 k = tid; k < nk; k += 256) {
+          float a0 = 0.f, a1 = 0.f;
+          int i = 0;
+          for (; i + 1 < nmy; i += 2) {
+            a0 = fmaf(Ub[(i0 + i) * ld + k], colj[i], a0);
+            a1 = fmaf(Ub[(i0 + i + 1) * ld + k], colj[i + 1], a1);
+          }
+          if (i < nmy) a0 = fmaf(Ub[(i0 + i) * ld + k], colj[i], a0);
+          partb[(i64)c * r + k] = a0 + a1;
+        }
+        ok = cgs_grid_barrier(counter, epoch, spin_limit, status, &s_dead);
+        if (!ok) break;
+        {   // fixed-order sums over the CTAs, the k range split over the grid
+          const i64 per = (nk + G - 1) / G;
+          const i64 k0 = (i64)c * per, k1 = min(nk, k0 + per);
+          for (i64 k = k0 + tid; k < k1; k += 256) {
+            float sum = 0.f;
+            for (int cc = 0; cc < G; ++cc) sum += partb[(i64)cc * r + k];
+            hb[k] = sum;
+          }
+        }
+        ok = cgs_grid_barrier(counter, epoch, spin_limit, status, &s_dead);
+        if (!ok) break;
+        if (pass == 0) before = hb[j];
+        if (j > 0) {
+          for (int i = warp; i < nmy; i += 8) {       // a warp per row: lanes stride over k
+            const float* urow = Ub + (i0 + i) * ld;
+            float acc = 0.f;
+            for (i64 k = lane; k < j; k += 32) acc = fmaf(urow[k], hb[k], acc);
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+            if (lane == 0) colj[i] -= acc;
+          }
+          __syncthreads();
+        }
+      }
+      if (!ok) break;
+      float sq = 0.f;
+      for (int i = tid; i < nmy; i += 256) sq = fmaf(colj[i], colj[i], sq);
+      sq = cgs_block_sum(sq, red);
+      if (tid == 0) nb_part[c] = sq;
+      ok = cgs_grid_barrier(counter, epoch, spin_limit, status, &s_dead);
+      if (!ok) break;
+      if (tid == 0) {
+        float tot = 0.f;
+        for (int cc = 0; cc < G; ++cc) tot += nb_part[cc];
+        s_val = tot;
+      }
+      __syncthreads();
+      const float after = s_val;
+      // every CTA sees the same two sums: the same decision everywhere
+      if (!(after > CGS_DEFLATE_REL * CGS_DEFLATE_REL * before) || !(before < __int_as_float(0x7f800000))) {
+        deficient = true;
+        break;
+      }
+      const float inv = rsqrtf(after);
+      for (int i = tid; i < nmy; i += 256) Ub[(i0 + i) * ld + j] = colj[i] * inv;
+      __syncthreads();
+    }
+    if (c == 0 && tid == 0) {
+      if (ok && !deficient) {
+        os[OS_FAIL] = 0;
+        atomicAdd(fallbacks, 1);
+      } else {
+        os[OS_FAIL] = 1;
+        if (deficient) atomicOr(status, DION_STATUS_BREAKDOWN);
+      }
+    }
+    __syncthreads();
   }
 }
 

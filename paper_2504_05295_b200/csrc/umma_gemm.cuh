@@ -56,7 +56,9 @@ struct Params {
   int num_items;      // tiles * splits
   int kc;             // K blocks per accumulation chunk (see k_gemm_umma)
   int* status;        // device status word (DION_STATUS_TIMEOUT)
-  int debug;          // internal timing experiments: 1 no global loads, 2 no loads/stores, 4 no MMAs
+  long long spin_limit;   // cycle budget of every mbarrier wait (SPIN_LIMIT_CYCLES unless a test shortens it)
+  int withhold_arrive;    // test hook of the register-path variant: the producer warps do not arrive for the first
+                          // K block, so that the consumer's bounded wait runs out (no copy is in flight then)
 };
 
 // ------------------------------------------------------------------ PTX wrappers
@@ -170,7 +172,7 @@ __device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t
 // `sleep_ns` > 0 backs off between polls so that a waiting warp does not take issue
 // slots from the producer warps.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* dead, int* status,
-                                          unsigned sleep_ns = 0) {
+                                          long long limit, unsigned sleep_ns = 0) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   unsigned polls = 0;
@@ -179,7 +181,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     if (sleep_ns) __nanosleep(sleep_ns);
     if ((++polls & 63u) == 0) {
       if (*dead) return false;
-      if (clock64() - t0 > SPIN_LIMIT_CYCLES) {
+      if (clock64() - t0 > limit) {
         *dead = 1;
         atomicOr(status, DION_STATUS_TIMEOUT);
         return false;
@@ -371,7 +373,7 @@ struct TileMap {
 
   // Writes the chunks to shared memory.  fp32 mode: TF32 "hi" part to s_hi and the TF32-
   // rounded remainder to s_lo; bf16 mode: rounded to bf16 into s_hi.
-  __device__ __forceinline__ void store(uint32_t s_hi, uint32_t s_lo, const float (&v)[NCHUNK][EPC], bool raw_hi = false) const {
+  __device__ __forceinline__ void store(uint32_t s_hi, uint32_t s_lo, const float (&v)[NCHUNK][EPC]) const {
 #pragma unroll
     for (int l = 0; l < NCHUNK; ++l) {
       const uint32_t off = soff[l] & 0xFFFFFu;
@@ -387,13 +389,8 @@ struct TileMap {
         uint32_t h[4], lo[4];
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
-          if (raw_hi) {   // experiment: the MMA reads the fp32 word itself; lo is the truncation remainder
-            h[q] = __float_as_uint(v[l][q]);
-            lo[q] = __float_as_uint(v[l][q] - __uint_as_float(h[q] & 0xFFFFE000u));
-          } else {
-            h[q] = cvt_tf32(v[l][q]);
-            lo[q] = __float_as_uint(v[l][q] - __uint_as_float(h[q]));
-          }
+          h[q] = cvt_tf32(v[l][q]);
+          lo[q] = __float_as_uint(v[l][q] - __uint_as_float(h[q]));
         }
         st_shared_v4(s_hi + off, h[0], h[1], h[2], h[3]);
         st_shared_v4(s_lo + off, lo[0], lo[1], lo[2], lo[3]);
@@ -409,7 +406,12 @@ struct TileMap {
 // brings the product to the accuracy of an fp32 FMA loop (measured 3.3e-7 against
 // 9.1e-7 relative error on Gaussian data).  Used for the products whose error the
 // conditioning of an ill-conditioned panel amplifies.
-template <int BN, bool BF16, bool SPLIT = false, bool TMA = false, bool D16 = false, bool CE = false>
+// ONE (fp32 mode, single pass): the operands are fp32 arrays whose values already fit TF32 (rounded to
+// nearest beforehand, k_round_tf32), so one kind::tf32 MMA per K step reads the raw tiles TMA has written:
+// no "lo" halves, no conversion pass, the producer warps join the epilogue as in the bf16-array variant.
+// Used for the rank-r update of X, whose result feeds nothing else: an unbiased 2^-12 relative operand
+// error there moves X by ~1e-6.
+template <int BN, bool BF16, bool SPLIT = false, bool TMA = false, bool D16 = false, bool CE = false, bool ONE = false>
 struct Cfg {
   // BT: bf16 operands formed in shared memory from TMA-loaded fp32 tiles (K block of 32, as in
   // the fp32 TMA variant).  A stage then holds the raw fp32 tiles of A, of its fp32 addend and
@@ -422,9 +424,9 @@ struct Cfg {
   static constexpr int A_BYTES = BM * 128;
   static constexpr int B_BYTES = BN * 128;
   static constexpr int STAGE_BYTES = BT ? (2 * A_BYTES + B_BYTES + A_BYTES / 2 + B_BYTES / 2)
-                                        : (BF16 ? 1 : 2) * (A_BYTES + B_BYTES);
+                                        : ((BF16 || ONE) ? 1 : 2) * (A_BYTES + B_BYTES);
   // D16: the producer warps have no conversion work and serve as epilogue warps too
-  static constexpr int EPI_WARPS = D16 ? NUM_EPI_WARPS + NUM_PROD_WARPS : NUM_EPI_WARPS;
+  static constexpr int EPI_WARPS = (D16 || ONE) ? NUM_EPI_WARPS + NUM_PROD_WARPS : NUM_EPI_WARPS;
   // CE (coalesced epilogue): an epilogue warp owns 32 rows x EPI_W columns of the tile and passes them
   // through a private shared-memory tile in passes of EPI_RPP rows (EPI_RPP * EPI_W = 1024 elements),
   // so that one global access of the warp covers whole row segments instead of 32 rows; paid for with
@@ -455,12 +457,14 @@ struct Cfg {
 // TMA with bf16 operands: the same loads; the producer warps add, round to bf16 and write
 // the operand tiles the MMA reads (k-contiguous: rows of 64 bytes, 64-byte swizzle;
 // row-contiguous: 128-byte rows of 64 row indices, 128-byte swizzle); one MMA per K step.
-template <int BN, bool A_MN, bool B_MN, bool BF16, bool SPLIT, bool TMA, bool D16 = false, bool CE = false>
+template <int BN, bool A_MN, bool B_MN, bool BF16, bool SPLIT, bool TMA, bool D16 = false, bool CE = false, bool ONE = false>
 __global__ void __launch_bounds__(TMA ? NUM_THREADS_TMA : NUM_THREADS, 1) k_gemm_umma(const __grid_constant__ Params p) {
   static_assert(!(BF16 && SPLIT), "split accumulators belong to the 3xTF32 mode");
   static_assert(!D16 || (BF16 && TMA), "bf16 operands in memory are loaded by TMA");
   static_assert(!CE || (TMA && (D16 || !BF16)), "the coalesced epilogue serves the bf16-array and the fp32 TMA variants");
-  using C = Cfg<BN, BF16, SPLIT, TMA, D16, CE>;
+  static_assert(!ONE || (TMA && CE && !BF16 && !SPLIT && !A_MN && !B_MN), "single pass: k-contiguous fp32 operands by TMA");
+  using C = Cfg<BN, BF16, SPLIT, TMA, D16, CE, ONE>;
+  constexpr bool NOCONV = D16 || ONE;    // the operand tiles are what TMA writes: nothing to convert
   constexpr int NBUF = C::NBUF, ACCS = C::ACCS;
   constexpr int BKE = C::BKE, EPC = C::EPC, STAGES = C::STAGES;
   if (p.g.skip_flag != nullptr && *p.g.skip_flag != 0) return;
@@ -524,7 +528,7 @@ __global__ void __launch_bounds__(TMA ? NUM_THREADS_TMA : NUM_THREADS, 1) k_gemm
         const bool first = (kb == it.kb0);
         const int ab = iter % NBUF;
         const uint32_t ph = (uint32_t)(iter / NBUF) & 1u;
-        if (!mbar_wait(accf_bar(ab), ph, dead, p.status, 256)) { alive = false; break; }
+        if (!mbar_wait(accf_bar(ab), ph, dead, p.status, p.spin_limit, 256)) { alive = false; break; }
         tc_fence_after();
         if constexpr (CE) {
           // Coalesced epilogue.  A TMEM lane is a row, so a warp that wrote its accumulator rows straight
@@ -666,7 +670,7 @@ __global__ void __launch_bounds__(TMA ? NUM_THREADS_TMA : NUM_THREADS, 1) k_gemm
   } else if (warp < NUM_EPI_WARPS + NUM_PROD_WARPS) {
     // ------------------------------------------------------------ producers
     const int ptid = threadIdx.x - NUM_EPI_WARPS * 32;
-    if (D16) {
+    if (NOCONV) {
       // nothing to convert: the TMA warp fills the operand tiles
     } else if (TMA) {
       // in-place conversion of the tiles the TMA warp loaded; the split is elementwise, so
@@ -712,7 +716,7 @@ __global__ void __launch_bounds__(TMA ? NUM_THREADS_TMA : NUM_THREADS, 1) k_gemm
       for (int item = blockIdx.x; item < p.num_items && alive; item += gridDim.x) {
         const Item it = decode_item<BN, BKE>(p, item);
         for (int kb = it.kb0; kb < it.kb1; ++kb) {
-          if (!mbar_wait(raw_bar(stage), phase, dead, p.status)) { alive = false; break; }
+          if (!mbar_wait(raw_bar(stage), phase, dead, p.status, p.spin_limit)) { alive = false; break; }
           const uint32_t sg16 = g16_base + stage * C::G16_BYTES;
           const uint32_t sa = smem_base + stage * C::STAGE_BYTES + (uint32_t)ptid * 16u;
           const uint32_t sa_lo = sa + C::A_BYTES;
@@ -787,34 +791,22 @@ __global__ void __launch_bounds__(TMA ? NUM_THREADS_TMA : NUM_THREADS, 1) k_gemm
         const i64 k0 = (i64)kb * BKE;
         float va[C::A_CHUNKS][EPC], wa[C::A_CHUNKS][EPC];
         float vb[C::B_CHUNKS][EPC];
-        if (p.debug & 3) {
-#pragma unroll
-          for (int l = 0; l < C::A_CHUNKS; ++l)
-#pragma unroll
-            for (int e = 0; e < EPC; ++e) { va[l][e] = 1.f; wa[l][e] = 0.f; }
-#pragma unroll
-          for (int l = 0; l < C::B_CHUNKS; ++l)
-#pragma unroll
-            for (int e = 0; e < EPC; ++e) vb[l][e] = 1.f;
-        } else {
         ma.load(a_row + k0 * g.a_sk, a2_row + k0 * g.a2_sk * a2_elem, g.a2_mode, g.M - row0a, k_end - k0, va, wa);
         mb.load(b_row + k0 * g.b_sk, nullptr, ADD_NONE, g.N - row0b, k_end - k0, vb, vb);
-        }
-        if (!mbar_wait(empty_bar(stage), phase ^ 1u, dead, p.status)) { alive = false; break; }
+        if (!mbar_wait(empty_bar(stage), phase ^ 1u, dead, p.status, p.spin_limit)) { alive = false; break; }
         ma.add(g.a2_mode, va, wa);
         const uint32_t sa = smem_base + stage * C::STAGE_BYTES;
         const uint32_t sa_lo = sa + C::A_BYTES;
         const uint32_t sb = sa + (BF16 ? 1 : 2) * C::A_BYTES;
         const uint32_t sb_lo = sb + C::B_BYTES;
-        if (!(p.debug & 2)) {
-          ma.store(sa, sa_lo, va, (p.debug & 8) != 0);
-          mb.store(sb, sb_lo, vb, (p.debug & 8) != 0);
-        }
+        ma.store(sa, sa_lo, va);
+        mb.store(sb, sb_lo, vb);
         // every thread makes its own writes visible to the tensor core's (async) proxy, then
         // one lane per warp arrives: 8 arrivals per stage instead of 256 serialised ones
         fence_proxy_async();
         __syncwarp();
-        if (lane == 0) mbar_arrive(full_bar(stage));
+        const bool withheld = p.withhold_arrive != 0 && item == (int)blockIdx.x && kb == it.kb0;
+        if (lane == 0 && !withheld) mbar_arrive(full_bar(stage));
         if (++stage == STAGES) { stage = 0; phase ^= 1u; }
       }
     }
@@ -832,12 +824,19 @@ __global__ void __launch_bounds__(TMA ? NUM_THREADS_TMA : NUM_THREADS, 1) k_gemm
         const Item it = decode_item<BN, BKE>(p, item);
         const int row0a = it.mi * BM, row0b = it.ni * BN;
         for (int kb = it.kb0; kb < it.kb1; ++kb) {
-          if (!mbar_wait(empty_bar(stage), phase ^ 1u, dead, p.status, 32)) { alive = false; break; }
+          if (!mbar_wait(empty_bar(stage), phase ^ 1u, dead, p.status, p.spin_limit, 32)) { alive = false; break; }
           const int k0 = kb * BKE;
           const uint32_t sa = smem_base + stage * C::STAGE_BYTES;
           const uint32_t sa_lo = sa + C::A_BYTES;
-          const uint32_t sb = sa + (D16 ? 1 : 2) * C::A_BYTES;
+          const uint32_t sb = sa + (NOCONV ? 1 : 2) * C::A_BYTES;
           const uint32_t bar = raw_bar(stage);
+          if (ONE) {   // raw fp32 tiles, [rows][32 k] boxes
+            mbar_expect_tx(bar, (uint32_t)(C::A_BYTES + C::B_BYTES));
+            tma_load_2d(sa, &p.tmA, k0, row0a, bar);
+            tma_load_2d(sb, &p.tmB, k0, row0b, bar);
+            if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+            continue;
+          }
           if (D16) {   // bf16 tiles: [rows][64 k] boxes, or [64 k][64 rows] boxes per 64-row chunk
             mbar_expect_tx(bar, (uint32_t)(C::A_BYTES + C::B_BYTES));
             if (!A_MN) tma_load_2d(sa, &p.tmA, k0, row0a, bar);
@@ -896,26 +895,29 @@ __global__ void __launch_bounds__(TMA ? NUM_THREADS_TMA : NUM_THREADS, 1) k_gemm
         const int kbc1 = min(it.kb1, kbc + p.kc);
         const int ab = iter % NBUF;
         const uint32_t aph = (uint32_t)(iter / NBUF) & 1u;
-        if (!mbar_wait(acce_bar(ab), aph ^ 1u, dead, p.status, 64)) { alive = false; break; }
+        if (!mbar_wait(acce_bar(ab), aph ^ 1u, dead, p.status, p.spin_limit, 64)) { alive = false; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(ab * ACCS * BN);
         const uint32_t d_small = d_tmem + (SPLIT ? BN : 0);
         uint32_t accumulate = 0;
         for (int kb = kbc; kb < kbc1; ++kb) {
-          if (!mbar_wait(D16 ? raw_bar(stage) : full_bar(stage), phase, dead, p.status)) { alive = false; break; }
+          if (!mbar_wait(NOCONV ? raw_bar(stage) : full_bar(stage), phase, dead, p.status, p.spin_limit)) { alive = false; break; }
           tc_fence_after();
           const uint32_t st0 = smem_base + stage * C::STAGE_BYTES;
           // bf16 operands formed from TMA tiles sit behind the raw tiles of the stage
           const uint32_t sa = C::BT ? st0 + 2 * C::A_BYTES + C::B_BYTES : st0;
           const uint32_t sa_lo = sa + C::A_BYTES;
-          const uint32_t sb = C::BT ? sa + C::A_BYTES / 2 : sa + (BF16 ? 1 : 2) * C::A_BYTES;
+          const uint32_t sb = C::BT ? sa + C::A_BYTES / 2 : sa + ((BF16 || ONE) ? 1 : 2) * C::A_BYTES;
           const uint32_t sb_lo = sb + C::B_BYTES;
 #pragma unroll
-          for (int ks = 0; ks < ((p.debug & 4) ? 0 : C::KSTEPS); ++ks) {
+          for (int ks = 0; ks < C::KSTEPS; ++ks) {
             const uint64_t a_hi = (C::BT && !A_MN) ? make_desc_k64(sa + ks * A_KSTEP) : make_desc<BF16>(sa + ks * A_KSTEP, A_MN, lbo);
             const uint64_t b_hi = (C::BT && !B_MN) ? make_desc_k64(sb + ks * B_KSTEP) : make_desc<BF16>(sb + ks * B_KSTEP, B_MN, lbo);
             if (BF16) {
               umma<true>(d_tmem, a_hi, b_hi, idesc, accumulate);
+              accumulate = 1;
+            } else if (ONE) {
+              umma<false>(d_tmem, a_hi, b_hi, idesc, accumulate);
               accumulate = 1;
             } else {
               const uint64_t a_lo = make_desc<BF16>(sa_lo + ks * A_KSTEP, A_MN, lbo);
@@ -943,7 +945,7 @@ __global__ void __launch_bounds__(TMA ? NUM_THREADS_TMA : NUM_THREADS, 1) k_gemm
       }
       // drain: every issued MMA must have finished before TMEM is released
       umma_commit(drain_bar);
-      mbar_wait(drain_bar, 0u, dead, p.status, 64);
+      mbar_wait(drain_bar, 0u, dead, p.status, p.spin_limit, 64);
     }
     __syncwarp();
   }
@@ -956,10 +958,17 @@ __global__ void __launch_bounds__(TMA ? NUM_THREADS_TMA : NUM_THREADS, 1) k_gemm
   }
 }
 
-template <int BN, bool A_MN, bool B_MN, bool BF16, bool SPLIT, bool TMA, bool D16 = false, bool CE = false>
+template <int BN, bool A_MN, bool B_MN, bool BF16, bool SPLIT, bool TMA, bool D16 = false, bool CE = false, bool ONE = false>
 inline cudaError_t set_smem_attr() {
-  return cudaFuncSetAttribute(k_gemm_umma<BN, A_MN, B_MN, BF16, SPLIT, TMA, D16, CE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              Cfg<BN, BF16, SPLIT, TMA, D16, CE>::SMEM_BYTES);
+  return cudaFuncSetAttribute(k_gemm_umma<BN, A_MN, B_MN, BF16, SPLIT, TMA, D16, CE, ONE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              Cfg<BN, BF16, SPLIT, TMA, D16, CE, ONE>::SMEM_BYTES);
+}
+
+// single-pass TF32 (k-contiguous operands only)
+template <int BN>
+inline void launch_one(const Params& p, int grid, cudaStream_t st) {
+  constexpr int smem = Cfg<BN, false, false, true, false, true, true>::SMEM_BYTES;
+  k_gemm_umma<BN, false, false, false, false, true, false, true, true><<<grid, NUM_THREADS_TMA, smem, st>>>(p);
 }
 
 template <int BN, bool BF16, bool SPLIT, bool TMA, bool D16 = false, bool CE = false>
@@ -1076,6 +1085,8 @@ inline int umma_configure() {
   DION_SET(128, false, false, true) DION_SET(128, false, true, true) DION_SET(128, true, true, true) DION_SET(128, true, false, true)
   DION_SET(256, false, false, true) DION_SET(256, false, true, true) DION_SET(256, true, true, true) DION_SET(256, true, false, true)
 #undef DION_SET
+  if (e == cudaSuccess) e = set_smem_attr<128, false, false, false, false, true, false, true, true>();
+  if (e == cudaSuccess) e = set_smem_attr<256, false, false, false, false, true, false, true, true>();
   if (e != cudaSuccess) { cudaGetLastError(); return DION_ERR_CUDA; }
   if (tracked) done_on[dev] = true;
   return DION_OK;
@@ -1084,8 +1095,13 @@ inline int umma_configure() {
 // Launches the product on the tensor cores if it qualifies.  Returns the number of
 // kernels launched (1, or 2 with a split-K reduction), 0 if this engine does not take
 // the product, or a negative DION_ERR_* code.
+// `variant` (test hook, 0 in the product): UMMA_VARIANT_* bits.
+enum : int {
+  UMMA_VARIANT_REGISTER_LOADS = 1,   // operands through registers instead of TMA
+  UMMA_VARIANT_WITHHOLD = 2          // with register loads: withhold one producer arrival, 1 ms wait budget
+};
 inline int umma_try_launch(const GemmArgs& g_in, int precision, int sm_count, float* part, i64 part_floats,
-                           int* status, cudaStream_t st, int debug = 0) {
+                           int* status, cudaStream_t st, int variant = 0) {
   using namespace umma;
   GemmArgs g = g_in;
   const bool d16 = g.ab16 != 0;      // bf16 operands in memory
@@ -1116,12 +1132,12 @@ inline int umma_try_launch(const GemmArgs& g_in, int precision, int sm_count, fl
 
   // lower-triangular output: 128 x 256 tiles (more flops per operand byte; the tiles on the diagonal
   // compute up to 128 columns too many) once the matrix has enough tile rows for that to pay
-  const bool tri_wide = g.tri == TRI_LOWER && g.epi == EPI_STORE && g.N >= TRI_WIDE_MIN && !(debug & 32);
+  const bool tri_wide = g.tri == TRI_LOWER && g.epi == EPI_STORE && g.N >= TRI_WIDE_MIN;
   const int BN = ((g.tri == TRI_LOWER && !tri_wide) || g.N < 256) ? 128 : 256;
   Params p;
   p.g = g;
   // TMA variant: fp32 operands in memory (both precision modes), dimensions the tensor maps can describe
-  bool tma = (d16 || !(debug & 16)) && g.M < (1ll << 31) && g.N < (1ll << 31) && g.K < (1ll << 31);
+  bool tma = (d16 || !(variant & UMMA_VARIANT_REGISTER_LOADS)) && g.M < (1ll << 31) && g.N < (1ll << 31) && g.K < (1ll << 31);
   if (d16) {
     const i64 lda = a_mn ? g.a_sk : g.a_si, ldb = b_mn ? g.b_sk : g.b_sn;
     if (!tma || !make_operand16_map(&p.tmA, g.A, g.M, g.K, lda, a_mn, BM) ||
@@ -1162,12 +1178,18 @@ inline int umma_try_launch(const GemmArgs& g_in, int precision, int sm_count, fl
   if (tiles * splits > 0x7fffffff) return 0;
   p.num_items = (int)(tiles * splits);
   p.status = status;
-  p.debug = debug;
+  const bool withhold = (variant & UMMA_VARIANT_WITHHOLD) && !tma;
+  p.spin_limit = withhold ? 2000000LL : SPIN_LIMIT_CYCLES;
+  p.withhold_arrive = withhold ? 1 : 0;
   // 32 K blocks per accumulation chain: 1024 k (8e-6 relative error in fp32 mode, 1.4e-6 with
   // split accumulators); 2048 k for bf16 operands loaded through registers
   p.kc = 32;
   const int grid = p.num_items < sm_count ? p.num_items : sm_count;
-  if (d16) {   // bf16 arrays: always with the coalesced epilogue
+  const bool one = g.tf32x1 && !bf16 && tma && !a_mn && !b_mn && g.a2_mode == ADD_NONE && !g.precise && splits == 1;
+  if (one) {
+    if (BN == 256) launch_one<256>(p, grid, st);
+    else launch_one<128>(p, grid, st);
+  } else if (d16) {   // bf16 arrays: always with the coalesced epilogue
     if (BN == 256) launch_variant<256, true, false, true, true, true>(p, a_mn, b_mn, grid, st);
     else launch_variant<128, true, false, true, true, true>(p, a_mn, b_mn, grid, st);
   } else if (bf16 && tma) {

@@ -16,14 +16,19 @@ import torch.distributed as dist
 
 
 def all_reduce_mean(buf: torch.Tensor, group=None) -> None:
-    """In-place mean over the ranks of `group` (a no-op without an initialised process group)."""
+    """In-place mean over the ranks of `group` (a no-op without an initialised process group).
+    On GPUs the division is part of the NCCL collective (ReduceOp.AVG); the gloo backend of the CPU
+    tests has no averaging reduction, so there the sum is divided afterwards."""
     if not dist.is_available() or not dist.is_initialized():
         return
     world = dist.get_world_size(group)
     if world == 1:
         return
-    dist.all_reduce(buf, op=dist.ReduceOp.SUM, group=group)
-    buf.div_(world)
+    if buf.is_cuda and dist.get_backend(group) == "nccl":
+        dist.all_reduce(buf, op=dist.ReduceOp.AVG, group=group)
+    else:
+        dist.all_reduce(buf, op=dist.ReduceOp.SUM, group=group)
+        buf.div_(world)
 
 
 def flat_views(shapes: Sequence[Sequence[int]], device, dtype=torch.float32, align: int = 4):
@@ -59,6 +64,16 @@ class DpStepper:
         self.flags = torch.zeros(max(len(self.descs), 1), dtype=torch.int32, device=device)
 
     def step(self, lr: float, stream: Optional[torch.cuda.Stream] = None) -> None:
+        """One step.  The library's kernels run on `stream`; the two collectives run on torch's current
+        stream, so `stream` is made current for the whole step: otherwise the all-reduces would not be
+        ordered against the kernels that write and read the factor buffers."""
+        if stream is not None and self.flatP.is_cuda:
+            with torch.cuda.stream(stream):
+                self._step(lr, stream)
+        else:
+            self._step(lr, stream)
+
+    def _step(self, lr: float, stream) -> None:
         opt = self.opt
         for k, d in enumerate(self.descs):
             opt.dp_project(d, self.P[k], self.flags[k:k + 1], stream)

@@ -38,3 +38,72 @@ def oracle_steps(pb: inputs.DionProblem, steps: int, grads=None, mu=MU, eta=ETA,
 
 def device_state(pb: inputs.DionProblem, dev="cuda"):
     return (pb.X.to(dev).clone(), pb.M.to(dev).clone(), pb.Q.to(dev).clone())
+
+
+# ---------------------------------------------------------------------------
+# Where the 1e-4 bar cannot bind: ill-conditioned panels.
+#
+# At rank fractions above 1/4 (full rank above all) the panel P = (M + G) Q of the seeded workloads
+# has a condition number of 1e4 .. 1e7, and the thin-QR factor -- hence Q_new and the update -- of the
+# float64 rule itself moves by more than 1e-4 when P merely carries the rounding error of ONE float32
+# matrix product.  No float32 evaluation can then be asked for 1e-4.  The tests measure that movement
+# on the very input: they run the oracle a second time with nothing changed except that each step's
+# panel is formed by a plain float32 product (``orc.step_given_panel``), and allow the CUDA path
+# FLOOR_FACTOR times the distance between the two oracle runs (it evaluates about ten
+# float32-accurate products and triangular solves on that panel: P, the Gram matrix, the factor and the
+# solve of two to three Cholesky-QR rounds, and W), never less than the 1e-4 bar.  On well-conditioned
+# panels the distance is ~1e-6 and the bar is the plain 1e-4.
+# ---------------------------------------------------------------------------
+FLOOR_FACTOR = 10.0
+
+
+def fp32_panel(M64, G64, Q64):
+    """(M + G) Q by a plain float32 matrix product of the float32-rounded operands, as float64."""
+    B32 = torch.from_numpy(np.asarray(M64 + G64, dtype=np.float32))
+    Q32 = torch.from_numpy(np.asarray(Q64, dtype=np.float32))
+    return (B32 @ Q32).double().numpy()
+
+
+def oracle_steps_fp32_panel(pb, steps: int, grads=None, mu=MU, eta=ETA, eps=EPS):
+    """The oracle trajectory with each step's panel formed by a float32 product (state in float64)."""
+    X, M, Q = to_np64(pb.X), to_np64(pb.M), to_np64(pb.Q)
+    out = []
+    for t in range(steps):
+        G = to_np64(grads[t] if grads is not None else pb.grad(t))
+        res = orc.step_given_panel(X, M, G, Q, fp32_panel(M, G, Q), mu, eta, eps)
+        X, M, Q = res.X, res.M, res.Q
+        out.append(res)
+    return out
+
+
+def conditioned_tol(exact, moved, base=TOL_FP32):
+    """Per-array tolerance: the bar, or FLOOR_FACTOR x how far the float64 rule moved (see above)."""
+    return {nm: max(base, FLOOR_FACTOR * rel(getattr(moved, nm), getattr(exact, nm))) for nm in ("X", "M", "Q", "d")}
+
+
+def check_conditioned(got, exact, moved, tag=""):
+    """got: (X, M, Q, d) float64 arrays of the CUDA path."""
+    tol = conditioned_tol(exact, moved)
+    errs = {nm: rel(g, getattr(exact, nm)) for nm, g in zip(("X", "M", "Q", "d"), got)}
+    print(f"{tag}: " + " ".join(f"{k} {errs[k]:.2e}/{tol[k]:.1e}" for k in errs))
+    assert all(errs[k] <= tol[k] for k in errs), f"{tag}: errors {errs} tolerances {tol}"
+    return errs, tol
+
+
+def one_step_movement(X64, M64, G64, Q64, transposed=False, mu=MU, eta=ETA, eps=EPS):
+    """How far one step of the float64 rule moves, from the given float64 state, when its panel is formed by
+    a float32 product: {array name: relative Frobenius distance}.  transposed: the transposed form (the
+    standard step on the transposed arrays, eta scaled by m / n)."""
+    if transposed:
+        m, n = X64.shape
+        Xt, Mt, Gt = (np.ascontiguousarray(a.T) for a in (X64, M64, G64))
+        exact = orc.step(Xt, Mt, Gt, Q64, mu, eta * m / n, eps)
+        moved = orc.step_given_panel(Xt, Mt, Gt, Q64, fp32_panel(Mt, Gt, Q64), mu, eta * m / n, eps)
+    else:
+        exact = orc.step(X64, M64, G64, Q64, mu, eta, eps)
+        moved = orc.step_given_panel(X64, M64, G64, Q64, fp32_panel(M64, G64, Q64), mu, eta, eps)
+    return {nm: rel(getattr(moved, nm), getattr(exact, nm)) for nm in ("X", "M", "Q", "d")}
+
+
+def movement_tol(movement, base=TOL_FP32):
+    return {nm: max(base, FLOOR_FACTOR * v) for nm, v in movement.items()}

@@ -25,6 +25,14 @@ def test_workloads_match_the_configurations():
     assert (53248, 16384, 4096, "bf16") in l405 and (16384, 53248, 1024, "bf16") in l405 and len(l405) == 14
     assert bench.parse_cases("4096:1024,1024x4096:256:bf16", inputs) == [(4096, 4096, 1024), (1024, 4096, 256, "bf16")]
     assert bench.case_gbytes((1, 1, 1, "bf16")) == 2 and bench.case_gbytes((1, 1, 1)) == 4
+    assert bench.parse_cases("", inputs, "config1") == [(256, 512, 64)]
+    assert bench.ALL_WORKLOADS[-1] == bench.HEADLINE == "llama8b" and len(bench.ALL_WORKLOADS) == 5
+    # the oracle's bounded samples: the three 2048^2 cases of the sweep, else the cheapest distinct case(s)
+    assert sorted(bench.oracle_sample_cases(sweep, "sweep")) == [(2048, 2048, 128), (2048, 2048, 512), (2048, 2048, 2048)]
+    assert bench.oracle_sample_cases(l8, "llama8b") == [(1024, 4096, 256), (4096, 4096, 1024)]
+    assert bench.oracle_sample_cases(large, "large") == [(16384, 16384, 256)]
+    assert bench.traffic_variant(4096, 4096, 1024, 0) == "fp32_sum_in_scratch"
+    assert bench.traffic_variant(4096, 4096, 256, 0) == "fp32_fused_add" and bench.traffic_variant(4096, 4096, 256, 1) == "bf16_arrays"
 
 
 def test_flop_and_byte_models():
@@ -88,3 +96,5 @@ def test_reference_arm_prints_one_json_line():
     assert line["impl"] == "reference" and line["unit"] == "ms" and line["higher_is_better"] is False
     assert line["cpu_baseline"]["kind"] == "oracle" and line["cpu_baseline"]["cores"] >= 1
     assert line["e2e"]["h2d_bytes_per_step"] == 0 and line["vs_baseline"] is None
+    # the value is a timing of the sample; the flop-scaled figure has its own field
+    assert line["value"] == line["workloads"]["custom"]["value"] and line["projected_ms"] >= line["value"] * 0.999

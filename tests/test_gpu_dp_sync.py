@@ -5,7 +5,7 @@ all-reduce between the calls is a mean taken by the test."""
 import pytest
 import torch
 
-from helpers import EPS, ETA, MU, TOL_FP32, rel, to_np64
+from helpers import EPS, ETA, FLOOR_FACTOR, MU, TOL_FP32, one_step_movement, rel, to_np64
 from oracle import dion_oracle as orc
 from paper_2504_05295_b200 import binding, build, inputs
 
@@ -46,11 +46,18 @@ def test_two_and_three_ranks_match_the_oracle(m, n, r, ranks):
     M64 = [to_np64(pb.M) for pb in pbs]
     Xs = [pb.X.cuda().clone() for pb in pbs]; Ms = [pb.M.cuda().clone() for pb in pbs]
     Qs = [pb.Q.cuda().clone() for pb in pbs]; ds = [torch.zeros(r, device="cuda") for _ in pbs]
-    tol = TOL_FP32 if r < min(m, n) else 2e-3
+    tol = TOL_FP32
+    moved = 0.0
     with binding.Dion(mu=MU, eps=EPS) as opt:
         for t in range(3):
             # rank i sees its own gradient: the seeded gradient of step 3 t + i
             Gs = [pbs[0].grad(3 * t + i) for i in range(ranks)]
+            if r == min(m, n):
+                # ill-conditioned panel: allow what the float64 rule itself moves by under a float32 panel, summed
+                # over the steps (the sync step equals the plain step on the rank-averaged M and G)
+                mv = one_step_movement(X64, sum(M64) / ranks, sum(to_np64(g) for g in Gs) / ranks, Q64)
+                moved += max(mv.values())
+                tol = max(TOL_FP32, FLOOR_FACTOR * moved)
             X64, M64, Q64, d64 = orc.dp_step(X64, M64, [to_np64(g) for g in Gs], Q64, MU, ETA, EPS)
             dp_step(opt, Xs, Ms, [g.cuda() for g in Gs], Qs, ds, ETA)
         assert opt.get_status() == (0, 0)
@@ -111,3 +118,32 @@ def test_stepper_with_one_rank_equals_dion_step_on_a_list():
     for k, (a, b) in enumerate(zip(ref, got)):
         for name, u, v in zip("XMQ", a, b):
             assert torch.equal(u, v), f"matrix {k}: {name}"
+
+
+def test_stepper_on_a_stream_that_is_not_current_orders_its_collectives(monkeypatch):
+    # the collectives run on torch's current stream: the stepper must make the caller's stream current,
+    # or the all-reduce of P would race the kernels that write and read it
+    from paper_2504_05295_b200 import dp
+    m, n, r = 1024, 768, 128
+    pb = inputs.make_problem(m, n, r, seed=34, ks=16)
+    G = pb.grad(0).cuda()
+    seen = []
+
+    def fake_all_reduce_mean(buf, group=None):
+        seen.append(torch.cuda.current_stream().cuda_stream)
+        buf.mul_(1.0)                       # touches the buffer on the current stream, as a collective would
+
+    monkeypatch.setattr(dp, "all_reduce_mean", fake_all_reduce_mean)
+    side = torch.cuda.Stream()
+    with binding.Dion(mu=MU, eps=EPS) as opt:
+        Xa, Ma, Qa = pb.X.cuda().clone(), pb.M.cuda().clone(), pb.Q.cuda().clone()
+        opt.step(Xa, Ma, G, Qa, ETA)
+        Xb, Mb, Qb = pb.X.cuda().clone(), pb.M.cuda().clone(), pb.Q.cuda().clone()
+        torch.cuda.synchronize()
+        stepper = dp.DpStepper(opt, [binding.matrix_desc(Xb, Mb, G, Qb)], "cuda")
+        for _ in range(1):
+            stepper.step(ETA, side)
+        side.synchronize()
+        assert opt.get_status(side) == (0, 0)
+    assert seen == [side.cuda_stream, side.cuda_stream]
+    assert torch.equal(Xa, Xb) and torch.equal(Ma, Mb) and torch.equal(Qa, Qb)

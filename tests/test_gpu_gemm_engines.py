@@ -25,7 +25,7 @@ class GemmArgs(ctypes.Structure):
                 ("C", ctypes.c_void_p), ("ldc", ctypes.c_int64), ("epi", ctypes.c_int),
                 ("C2", ctypes.c_void_p), ("ldc2", ctypes.c_int64), ("c2_mode", ctypes.c_int),
                 ("alpha", ctypes.c_float), ("tri", ctypes.c_int), ("klimit", ctypes.c_int), ("precise", ctypes.c_int),
-                ("ab16", ctypes.c_int)]
+                ("ab16", ctypes.c_int), ("tf32x1", ctypes.c_int), ("variant", ctypes.c_int)]
 
 
 @pytest.fixture(scope="module")
@@ -40,13 +40,15 @@ def lib():
 
 
 def run(lib, engine, precision, M, N, K, a_mn, b_mn, add=None, epi=0, tri=0, klimit=0, alpha=1.0, seed=0,
-        precise=0, ab16=False):
+        precise=0, ab16=False, variant=0, tf32x1=False, expect_status=0):
     g = torch.Generator(device="cuda"); g.manual_seed(seed)
     rn = lambda *s: torch.randn(*s, generator=g, device="cuda")
     # A(i,k): stored M x K (k contiguous) or K x M (row index contiguous)
     A_store = rn(K, M) if a_mn else rn(M, K)
     if ab16:                             # operands stored as bf16: the reference sees the rounded values
         A_store = A_store.to(torch.bfloat16)
+    if tf32x1:                           # values that fit TF32 (10 explicit mantissa bits): bf16 values do
+        A_store = A_store.to(torch.bfloat16).float()
     A_log = A_store.t() if a_mn else A_store
     A2_store = None
     if add is not None:
@@ -58,6 +60,8 @@ def run(lib, engine, precision, M, N, K, a_mn, b_mn, add=None, epi=0, tri=0, kli
     B_store = rn(K, N) if b_mn else rn(N, K)
     if ab16:
         B_store = B_store.to(torch.bfloat16)
+    if tf32x1:
+        B_store = B_store.to(torch.bfloat16).float()
     B_log = B_store if b_mn else B_store.t()
     if klimit:
         B_log = torch.triu(B_log)       # B(k,j) = 0 for k > j
@@ -85,13 +89,16 @@ def run(lib, engine, precision, M, N, K, a_mn, b_mn, add=None, epi=0, tri=0, kli
     a.C = C.data_ptr(); a.ldc = N; a.epi = epi
     a.C2 = C2.data_ptr(); a.ldc2 = N; a.c2_mode = 1 if C2.dtype == torch.float32 else 2
     a.alpha = alpha; a.tri = tri; a.klimit = klimit; a.precise = precise; a.ab16 = int(ab16)
+    a.tf32x1 = int(tf32x1); a.variant = variant
     part = torch.empty(8 << 20, device="cuda")
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
     rc = lib.dion_debug_gemm(engine, precision, ctypes.byref(a), part.data_ptr(), part.numel(), status.data_ptr(),
                              int(torch.cuda.current_stream().cuda_stream))
     torch.cuda.synchronize()
     assert rc == 0, f"dion_debug_gemm returned {rc}"
-    assert int(status.item()) == 0, f"device status {int(status.item())}"
+    assert int(status.item()) == expect_status, f"device status {int(status.item())}"
+    if expect_status:
+        return None
     got = C.double()
     if tri:
         # only the elements on or below the diagonal are guaranteed to be written
@@ -154,35 +161,31 @@ def test_triangular_operand_k_limit(lib, engine):
 
 
 @pytest.fixture(params=["tma", "registers"])
-def bf16_path(request, monkeypatch):
-    # bf16 operands are formed from TMA-loaded fp32 tiles by default; bit 16 of the hook's
-    # debug word selects the variant whose producer warps load through registers
-    if request.param == "registers":
-        monkeypatch.setenv("DION_DEBUG_GEMM", "16")
-    else:
-        monkeypatch.delenv("DION_DEBUG_GEMM", raising=False)
-    return request.param
+def bf16_path(request):
+    # bf16 operands are formed from TMA-loaded fp32 tiles by default; bit 0 of the hook's variant word
+    # selects the kernel whose producer warps load through registers
+    return 1 if request.param == "registers" else 0
 
 
 @pytest.mark.parametrize("a_mn,b_mn", LAYOUTS)
 def test_bf16_operand_mode(lib, bf16_path, a_mn, b_mn):
-    err = run(lib, 2, 1, 512, 512, 1024, a_mn, b_mn)
+    err = run(lib, 2, 1, 512, 512, 1024, a_mn, b_mn, variant=bf16_path)
     assert err < 6e-3, err
-    err = run(lib, 2, 1, 648, 392, 328, a_mn, b_mn, seed=5)
+    err = run(lib, 2, 1, 648, 392, 328, a_mn, b_mn, seed=5, variant=bf16_path)
     assert err < 6e-3, err
-    err = run(lib, 2, 1, 256, 1024, 2080, a_mn, b_mn, seed=6)      # two accumulation chunks on the TMA path
+    err = run(lib, 2, 1, 256, 1024, 2080, a_mn, b_mn, seed=6, variant=bf16_path)      # two accumulation chunks on the TMA path
     assert err < 6e-3, err
 
 
 @pytest.mark.parametrize("add", [torch.float32, torch.bfloat16])
 def test_bf16_operand_mode_fused_add_and_epilogues(lib, bf16_path, add):
-    assert run(lib, 2, 1, 1024, 256, 768, False, True, add=add) < 6e-3
-    assert run(lib, 2, 1, 768, 256, 1024, True, True, add=add) < 6e-3
+    assert run(lib, 2, 1, 1024, 256, 768, False, True, add=add, variant=bf16_path) < 6e-3
+    assert run(lib, 2, 1, 768, 256, 1024, True, True, add=add, variant=bf16_path) < 6e-3
     # the rank-r updates: the product (entries ~16 here) is scaled by alpha before it meets C (entries ~1)
-    assert run(lib, 2, 1, 1024, 768, 256, False, False, add=add, epi=2, alpha=0.05) < 3e-3
-    assert run(lib, 2, 1, 1024, 768, 256, False, False, epi=1, alpha=0.01) < 1e-3
-    assert run(lib, 2, 1, 512, 512, 4096, True, True, tri=1) < 6e-3
-    assert run(lib, 2, 1, 1024, 768, 768, False, False, klimit=1) < 6e-3
+    assert run(lib, 2, 1, 1024, 768, 256, False, False, add=add, epi=2, alpha=0.05, variant=bf16_path) < 3e-3
+    assert run(lib, 2, 1, 1024, 768, 256, False, False, epi=1, alpha=0.01, variant=bf16_path) < 1e-3
+    assert run(lib, 2, 1, 512, 512, 4096, True, True, tri=1, variant=bf16_path) < 6e-3
+    assert run(lib, 2, 1, 1024, 768, 768, False, False, klimit=1, variant=bf16_path) < 6e-3
 
 
 @pytest.mark.parametrize("a_mn,b_mn", LAYOUTS)
@@ -208,3 +211,28 @@ def test_split_accumulators_reach_fma_accuracy(lib, a_mn, b_mn):
     # a Gram matrix sums same-sign terms on its diagonal, where the truncating adder is biased
     assert run(lib, 2, 0, 512, 512, 8192, True, True, tri=1, precise=1) < 2e-6
     assert run(lib, 2, 0, 2048, 512, 512, False, False, klimit=1, precise=1) < 1.5e-6
+
+
+def test_register_path_fp32(lib):
+    # the fp32 (3xTF32) kernel whose producer warps load through registers: operands TMA cannot describe
+    for a_mn, b_mn in LAYOUTS:
+        assert run(lib, 2, 0, 640, 384, 200, a_mn, b_mn, variant=1, seed=3) < TOL[2]
+
+
+@pytest.mark.parametrize("M,N,K,epi", [(1024, 768, 256, 1), (640, 392, 96, 1), (2048, 256, 2080, 1), (256, 128, 64, 0),
+                                       (512, 512, 512, 2)])
+def test_single_pass_tf32_on_operands_that_fit_tf32(lib, M, N, K, epi):
+    # operands whose values fit TF32 are read exactly by one MMA per K step: the only error left is the
+    # tensor core's fp32 accumulation
+    err = run(lib, 2, 0, M, N, K, False, False, epi=epi, alpha=0.05, tf32x1=True, seed=K)
+    assert err < 8e-6, err
+
+
+def test_a_wait_that_runs_out_reports_timeout_and_the_next_product_is_correct(lib):
+    # bit 1 of the variant word: the producer warps of the register-path kernel withhold their first arrival
+    # and every barrier wait has a 1 ms budget.  The kernel must give up (no trap, no endless wait), set
+    # DION_STATUS_TIMEOUT (4) and return; the context stays usable.
+    assert run(lib, 2, 0, 128, 128, 64, False, False, variant=3, expect_status=4) is None
+    assert run(lib, 2, 0, 256, 384, 128, False, False, variant=3, expect_status=4) is None      # several CTAs
+    assert run(lib, 2, 0, 128, 128, 64, False, False, variant=1) < TOL[2]
+    assert run(lib, 2, 0, 512, 512, 1024, False, True) < TOL[2]

@@ -8,7 +8,8 @@ import numpy as np
 import pytest
 import torch
 
-from helpers import EPS, ETA, MU, TOL_BF16, TOL_FP32, device_state, oracle_steps, rel, to_np64
+from helpers import (EPS, ETA, MU, TOL_BF16, TOL_FP32, check_conditioned, device_state, movement_tol, one_step_movement,
+                     oracle_steps, oracle_steps_fp32_panel, rel, to_np64)
 from paper_2504_05295_b200 import binding, build, inputs
 
 pytestmark = pytest.mark.gpu
@@ -64,14 +65,18 @@ def test_config1_after_1_and_10_steps(engine, orth):
                                    (200, 333, 65), (129, 1000, 129), (640, 384, 160)])
 def test_ragged_shapes_all_tiles_and_tails(engine, m, n, r):
     pb = inputs.make_problem(m, n, r, seed=3, ks=min(8, m, n))
-    # at full rank the panel is ill conditioned; use the robust mode there
-    orth = binding.ORTH_HOUSEHOLDER if r == min(m, n) else binding.ORTH_AUTO
     ref = oracle_steps(pb, 3)
-    snaps, status, skipped = run_gpu(pb, 3, engine=engine, orth=orth)
+    snaps, status, skipped = run_gpu(pb, 3, engine=engine)        # AUTO at every rank fraction
     assert status == 0 and skipped == 0
-    tol = TOL_FP32 if r < min(m, n) else 2e-3   # tiny full-rank panels: cond(P) up to 1e4+
-    check(snaps[0], ref[0], tol, "step 1")
-    check(snaps[2], ref[2], tol, "step 3")
+    if r < min(m, n):
+        check(snaps[0], ref[0], TOL_FP32, "step 1")
+        check(snaps[2], ref[2], TOL_FP32, "step 3")
+    else:
+        # full-rank panels are ill conditioned: the bar is 1e-4 or what the float64 rule itself moves by
+        # under a float32 panel, whichever is larger (helpers.py)
+        moved = oracle_steps_fp32_panel(pb, 3)
+        check_conditioned(snaps[0], ref[0], moved[0], f"{m}x{n} r={r} step 1")
+        check_conditioned(snaps[2], ref[2], moved[2], f"{m}x{n} r={r} step 3")
 
 
 @pytest.mark.parametrize("engine", ENGINES)
@@ -202,7 +207,10 @@ def test_grouped_chain_above_512_columns_equals_single_calls(shape, orth):
     for k, ((X1, M1, Q1), (X2, M2, Q2)) in enumerate(zip(single, states)):
         assert torch.equal(X1, X2) and torch.equal(M1, M2) and torch.equal(Q1, Q2), k
     ref = oracle_steps(pbs[0], 1)[0]
-    tol = TOL_FP32 if r < min(m, n) else 2e-3
+    tol = TOL_FP32
+    if r == min(m, n):      # ill-conditioned panel: the conditioned bar of helpers.py
+        pb = pbs[0]
+        tol = movement_tol(one_step_movement(to_np64(pb.X), to_np64(pb.M), to_np64(pb.grad(0)), to_np64(pb.Q)))["X"]
     assert rel(to_np64(states[0][1]), ref.M) <= TOL_FP32 and rel(to_np64(states[0][0]), ref.X) <= tol
 
 
@@ -250,7 +258,12 @@ def test_cholqr2_takes_its_second_round_only_when_the_first_is_not_enough():
         opt.step(X, M, G.cuda(), Q, ETA)
         assert opt.get_status() == (0, 0) and opt.orth_rounds() == 2
     assert rel(to_np64(M), want.M) <= TOL_FP32 and rel(to_np64(X), want.X) <= TOL_FP32
-    assert rel(to_np64(Q), want.Q) <= 10 * TOL_FP32     # Q inherits cond(P) times the rounding of P
+    # cond(P) is in the hundreds here: Q is held to 1e-4 or to what the float64 rule moves by under a float32
+    # panel on this input, whichever is larger
+    tolq = movement_tol(one_step_movement(to_np64(pb.X), to_np64(pb.M), to_np64(G), to_np64(Qbad)))["Q"]
+    eq = rel(to_np64(Q), want.Q)
+    print(f"nearly parallel warm start: Q {eq:.2e} / {tolq:.1e}")
+    assert eq <= tolq
 
 
 def test_checkpoint_resume_is_bit_identical():
@@ -369,29 +382,36 @@ def test_4096_square_quarter_rank_against_oracle():
 
 
 def step_properties(m, n, r, g_dtype, tol=TOL_FP32, precision=binding.PREC_FP32, steps=2):
-    """Runs `steps` library steps on device-generated inputs and checks, in float64, what the
-    rule fixes for the last one: the factors can be read back from the outputs because
-    (X - X')/s = U Q'^T and R = Q' diag(d + eps)."""
+    """Runs `steps` library steps on device-generated inputs and checks, in float64, what the rule fixes for
+    the last one.  U is the one the library computes for that step (handed out by the data-parallel entry
+    points from the same state); R is read back from the outputs, R = Q' diag(d + eps)."""
     pb = inputs.make_problem(m, n, r, seed=16, ks=64, g_dtype=g_dtype, device="cuda", keep_signal=False)
     X, M, Q = pb.X, pb.M, pb.Q
     d = torch.zeros(r, device="cuda")
+    Pbuf = torch.empty(m, r, device="cuda")
+    Wbuf = torch.empty(n, r, device="cuda")
+    flag = torch.zeros(1, dtype=torch.int32, device="cuda")
     with binding.Dion(mu=MU, eps=EPS, precision=precision) as opt:
         for t in range(steps):
             G = pb.grad(t)
-            X0, M0 = X.clone(), M.clone()
+            if t == steps - 1:
+                X0, M0 = X.clone(), M.clone()
+                desc = binding.matrix_desc(X, M, G, Q)
+                opt.dp_project(desc, Pbuf, flag)
+                opt.dp_factor(desc, Pbuf, Wbuf, flag)          # Pbuf <- U
             opt.step(X, M, G, Q, ETA, colnorm_out=d)
         assert opt.get_status() == (0, 0)
+    del Wbuf
     s = ETA * (m / n) ** 0.5
     B = M0.double() + G.double()
     Qn = Q.double()
-    delta = (X0.double() - X.double()) / s                      # U Q'^T
-    U = torch.linalg.solve(Qn.t() @ Qn, (delta @ Qn).t()).t()   # U = delta Q' (Q'^T Q')^-1
-    del delta
+    U = Pbuf.double()
     R = Qn * (d.double() + EPS)
     eye = torch.eye(r, device="cuda", dtype=torch.float64)
-    # fp32 X carries eta-scaled updates: U is read back with ~1e-7 / (eta * |U_ij|) relative noise
-    tol_u = max(tol, 3e-4)
-    assert float((U.t() @ U - eye).abs().max()) <= tol_u
+    # in bf16-operand mode the data-parallel calls form their products from fp32 tiles while dion_step reads
+    # bf16 copies made once: the two U agree to the mode's bar only
+    tol_u = tol
+    assert float((U.t() @ U - eye).abs().max()) <= TOL_FP32
     assert float(torch.linalg.norm(B.t() @ U - R) / torch.linalg.norm(R)) <= tol_u
     assert float(torch.linalg.norm(B - (1 - MU) * (U @ R.t()) - M.double()) / torch.linalg.norm(M.double())) <= tol
     nq = torch.linalg.norm(Qn, dim=0)
@@ -399,6 +419,10 @@ def step_properties(m, n, r, g_dtype, tol=TOL_FP32, precision=binding.PREC_FP32,
     upd = float(torch.linalg.norm(X0.double() - X.double()))
     assert abs(upd - s * r ** 0.5) <= 1e-3 * s * r ** 0.5
     assert float(torch.linalg.norm(d.double() - torch.linalg.norm(B.t() @ U, dim=0)) / torch.linalg.norm(d.double())) <= tol_u
+    # the update is built from this U and the Q' the step wrote (single-pass TF32 on rounded factors in fp32
+    # mode, bf16 operands in bf16 mode; read back from fp32 X by subtraction)
+    delta = (X0.double() - X.double()) / s
+    assert float(torch.linalg.norm(delta - U @ Qn.t()) / torch.linalg.norm(delta)) <= max(10 * tol, 1e-3)
 
 
 @pytest.mark.parametrize("m,n,r", [(8192, 8192, 512), (8192, 8192, 2048), (2048, 2048, 2048), (4096, 4096, 4096)])
@@ -454,3 +478,87 @@ def test_grouped_llama_like_block_list_against_oracle():
         ref = oracle_steps(pb, 2)
         assert rel(to_np64(X), ref[1].X) <= TOL_FP32 and rel(to_np64(M), ref[1].M) <= TOL_FP32
         assert rel(to_np64(Q), ref[1].Q) <= TOL_FP32
+
+
+# ---------------------------------------------------------------------------
+# Failure handling on the device: Cholesky QR breakdown -> fallback; non-finite inputs
+# ---------------------------------------------------------------------------
+
+def _nearly_parallel(Q, delta):
+    Qb = Q[:, :1] + delta * Q
+    return (Qb / Qb.norm(dim=0)).contiguous()
+
+
+def test_cholesky_breakdown_falls_back_on_the_device():
+    # rank fraction 1/8 through AUTO (CholeskyQR2) with a warm start whose columns are nearly parallel: the
+    # Gram matrix of P is not positive definite in fp32, a pivot fails, and the same call redoes the panel with
+    # the Gram-Schmidt fallback: no breakdown reported, no step skipped, outputs on the conditioned bar
+    m, n, r = 1024, 1024, 128
+    pb = inputs.make_problem(m, n, r, seed=41, ks=16)
+    G = pb.grad(0)
+    Qbad = _nearly_parallel(pb.Q, 1e-4)
+    from oracle import dion_oracle as orc
+    want = orc.step(to_np64(pb.X), to_np64(pb.M), to_np64(G), to_np64(Qbad), MU, ETA, EPS)
+    cond = np.linalg.cond(want.P)
+    X, M, Q = pb.X.cuda().clone(), pb.M.cuda().clone(), Qbad.cuda().clone()
+    d = torch.zeros(r, device="cuda")
+    with binding.Dion(mu=MU, eps=EPS) as opt:
+        opt.step(X, M, G.cuda(), Q, ETA, colnorm_out=d)
+        assert opt.get_status() == (0, 0)
+        assert opt.fallbacks() == 1
+        # a healthy step afterwards takes no fallback
+        Xh, Mh, Qh = device_state(pb)
+        opt.step(Xh, Mh, G.cuda(), Qh, ETA)
+        assert opt.get_status() == (0, 0) and opt.fallbacks() == 0
+    tol = movement_tol(one_step_movement(to_np64(pb.X), to_np64(pb.M), to_np64(G), to_np64(Qbad)))
+    errs = {"X": rel(to_np64(X), want.X), "M": rel(to_np64(M), want.M), "Q": rel(to_np64(Q), want.Q),
+            "d": rel(to_np64(d), want.d)}
+    print(f"fallback, cond(P) {cond:.1e}: " + " ".join(f"{k} {errs[k]:.2e}/{tol[k]:.1e}" for k in errs))
+    assert all(errs[k] <= tol[k] for k in errs), (errs, tol)
+
+
+def test_fallback_inside_a_grouped_chain_touches_only_the_failed_matrix():
+    m, n, r = 768, 512, 64
+    pbs = [inputs.make_problem(m, n, r, seed=42, k=k, ks=16) for k in range(3)]
+    Q0 = [pb.Q for pb in pbs]
+    Q0[1] = _nearly_parallel(pbs[1].Q, 1e-4)
+    with binding.Dion(mu=MU, eps=EPS) as opt:
+        single = []
+        for pb, q in zip(pbs, Q0):
+            X, M, Q = pb.X.cuda().clone(), pb.M.cuda().clone(), q.cuda().clone()
+            opt.step(X, M, pb.grad(0).cuda(), Q, ETA)
+            single.append((X, M, Q))
+        assert opt.get_status() == (0, 0) and opt.fallbacks() == 1
+        grouped = [(pb.X.cuda().clone(), pb.M.cuda().clone(), q.cuda().clone()) for pb, q in zip(pbs, Q0)]
+        opt.step_grouped([(X, M, pb.grad(0).cuda(), Q) for pb, (X, M, Q) in zip(pbs, grouped)], ETA)
+        assert opt.get_status() == (0, 0) and opt.fallbacks() == 1
+    for k, (a, b) in enumerate(zip(single, grouped)):
+        for name, u, v in zip("XMQ", a, b):
+            assert torch.equal(u, v), f"matrix {k}: {name} differs between dion_step and dion_step_grouped"
+    ref = oracle_steps(pbs[0], 1)[0]
+    assert rel(to_np64(grouped[0][2]), ref.Q) <= TOL_FP32
+
+
+@pytest.mark.parametrize("m,n,r", [(512, 384, 64), (512, 512, 512)])
+def test_non_finite_gradient_is_flagged_and_cancels_the_step(m, n, r):
+    pb = inputs.make_problem(m, n, r, seed=43, ks=8)
+    X, M, Q = device_state(pb)
+    X0, M0, Q0 = X.clone(), M.clone(), Q.clone()
+    G = pb.grad(0).cuda()
+    G[17, 5] = float("nan")
+    with binding.Dion(mu=MU, eps=EPS) as opt:
+        opt.step(X, M, G, Q, ETA)
+        status, skipped = opt.get_status()
+        assert status & binding.STATUS_NONFINITE and skipped == 1
+        assert torch.equal(X, X0) and torch.equal(M, M0) and torch.equal(Q, Q0)
+        G[17, 5] = float("inf")
+        opt.step(X, M, G, Q, ETA)
+        status, skipped = opt.get_status()
+        assert status & binding.STATUS_NONFINITE and skipped == 1
+        assert torch.equal(X, X0) and torch.equal(M, M0) and torch.equal(Q, Q0)
+        # the context stays usable
+        opt.step(X, M, pb.grad(0).cuda(), Q, ETA)
+        assert opt.get_status() == (0, 0)
+    ref = oracle_steps(pb, 1)
+    if r < min(m, n):
+        assert rel(to_np64(X), ref[0].X) <= TOL_FP32 and rel(to_np64(Q), ref[0].Q) <= TOL_FP32

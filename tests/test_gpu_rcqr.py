@@ -5,7 +5,7 @@ plain oracle step as well)."""
 import pytest
 import torch
 
-from helpers import EPS, ETA, MU, TOL_FP32, oracle_steps, rel, to_np64
+from helpers import EPS, ETA, MU, TOL_FP32, movement_tol, one_step_movement, oracle_steps, rel, to_np64
 from oracle import dion_oracle as orc
 from paper_2504_05295_b200 import binding, build, inputs
 
@@ -55,7 +55,11 @@ def test_rcqr_full_rank_panel_and_transposed_form():
         opt.step(X, M, pb.grad(0).cuda(), Q, ETA, transposed=True, sketch=S.cuda())
         assert opt.get_status() == (0, 0)
     assert rel(to_np64(M), ref.M) <= TOL_FP32
-    assert rel(to_np64(X), ref.X) <= 2e-3        # limited by the conditioning of the panel, as in every mode
+    # limited by the conditioning of the panel, as in every mode: the conditioned bar of helpers.py
+    tol = movement_tol(one_step_movement(to_np64(pb.X), to_np64(pb.M), to_np64(pb.grad(0)), to_np64(Q0), transposed=True))
+    ex = rel(to_np64(X), ref.X)
+    print(f"rcqr transposed full rank: X {ex:.2e}/{tol['X']:.1e}")
+    assert ex <= tol["X"]
 
 
 def test_rcqr_larger_rank_and_grouped_call():

@@ -9,7 +9,7 @@ import numpy as np
 import pytest
 import torch
 
-from helpers import EPS, ETA, MU, TOL_BF16, TOL_FP32, rel, to_np64
+from helpers import EPS, ETA, MU, TOL_BF16, TOL_FP32, movement_tol, one_step_movement, rel, to_np64
 from oracle import dion_oracle as orc
 from paper_2504_05295_b200 import binding, build, inputs
 
@@ -72,8 +72,12 @@ def test_transposed_full_rank_on_the_short_side():
         assert opt.get_status() == (0, 0)
     assert rel(to_np64(M), MU * B) <= TOL_FP32
     assert rel(to_np64(M), ref[0].M) <= TOL_FP32
-    # the update itself is only as well determined as the panel's conditioning allows
-    assert rel(to_np64(X), ref[0].X) <= 2e-3
+    # the update itself is only as well determined as the panel's conditioning allows: 1e-4, or what the
+    # float64 rule moves by under a float32 panel on this input (helpers.py)
+    tol = movement_tol(one_step_movement(to_np64(pb.X), to_np64(pb.M), to_np64(pb.grad(0)), to_np64(Q0), transposed=True))
+    ex, eq = rel(to_np64(X), ref[0].X), rel(to_np64(Q), ref[0].Q)
+    print(f"transposed full rank: X {ex:.2e}/{tol['X']:.1e} Q {eq:.2e}/{tol['Q']:.1e}")
+    assert ex <= tol["X"] and eq <= tol["Q"]
 
 
 def test_grouped_list_mixes_both_forms():

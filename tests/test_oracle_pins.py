@@ -351,6 +351,70 @@ def test_sym_power_iter_and_lazy_step():
     assert rel(Mn @ Qn, MU * (M + G) @ Qn) < 1e-12
 
 
+def test_lazy_step_update_norm_with_orthonormal_right_factor():
+    # after a refresh V is orthonormal, so ||ColNorm(W) V^T||_F = ||ColNorm(W)||_F: the update has
+    # norm eta sqrt(m/n) sqrt(sum_j (d_j / (d_j + eps))^2), whatever W is (fixes the scale factor,
+    # the use of the normalised W and of V in the update of Algorithm 6)
+    rng = np.random.default_rng(21)
+    for m, n, r in ((30, 20, 5), (18, 44, 7)):
+        X, M, G, Q = draw(rng, m, n, r)
+        Xn, Mn, Qn, d = orc.lazy_step(X, M, G, Q, MU, ETA, EPS, refresh=True)
+        assert rel(Qn.T @ Qn, np.eye(r)) < 1e-12
+        want = ETA * np.sqrt(m / n) * np.sqrt(np.sum((d / (d + EPS)) ** 2))
+        assert abs(np.linalg.norm(Xn - X) - want) < 1e-9 * want
+        assert abs(want - ETA * np.sqrt(m / n) * np.sqrt(r)) < 1e-6 * want
+        # the update lies in span(V) on the right: (X - X_new) (I - V V^T) = 0
+        D = X - Xn
+        assert np.linalg.norm(D - D @ Qn @ Qn.T) < 1e-12 * np.linalg.norm(D)
+
+
+def test_lazy_dion_with_refresh_every_step_converges_to_truncated_svd():
+    # Lazy-Dion_k with k = 1 on a static buffer: V <- Orthonormalize(B^T B V) is orthogonal iteration,
+    # so V -> V_r column by column, W = B V -> U_r Sigma_r, ColNorm(W) V^T -> U_r V_r^T, d -> sigma and
+    # M_new -> B - beta B_r, against a brute-force SVD
+    rng = np.random.default_rng(22)
+    m, n, r, k = 24, 40, 6, 8
+    sig = 2.0 ** -np.arange(k)
+    B0 = orth(rng, m, k) @ np.diag(sig) @ orth(rng, n, k).T
+    Ub, sb, Vbt = np.linalg.svd(B0)
+    polar_r = Ub[:, :r] @ Vbt[:r]
+    B_r = (Ub[:, :r] * sb[:r]) @ Vbt[:r]
+    Q = rng.standard_normal((n, r)); Q /= np.linalg.norm(Q, axis=0)
+    errs = []
+    for t in range(40):
+        Xn, Mn, Q, d = orc.lazy_step(np.zeros((m, n)), np.zeros((m, n)), B0, Q, MU, ETA, EPS, refresh=True)
+        O = -Xn / (ETA * np.sqrt(m / n))
+        errs.append(np.linalg.norm(O - polar_r))
+    assert errs[0] > 0.1
+    assert errs[-1] < 10 * EPS / sig[r - 1]
+    assert np.abs(d - sb[:r]).max() < 1e-10
+    assert rel(Mn, B0 - (1 - MU) * B_r) < 1e-9
+
+
+def test_row_sampled_step_equals_the_full_step_on_those_rows():
+    rng = np.random.default_rng(23)
+    m, n, r = 37, 29, 9
+    X, M, G, Q = draw(rng, m, n, r)
+    res = orc.step(X, M, G, Q, MU, ETA, EPS)
+    rows = np.array([0, 5, 36, 17, 5])
+    Xr, Mr, Qn, d = orc.step_rows(X, M, G, Q, rows, MU, ETA, EPS)
+    assert rel(Xr, res.X[rows]) < 1e-13 and rel(Mr, res.M[rows]) < 1e-13
+    assert rel(Qn, res.Q) < 1e-13 and rel(d, res.d) < 1e-13
+
+
+def test_step_given_panel_is_the_step_when_the_panel_is_exact():
+    rng = np.random.default_rng(24)
+    m, n, r = 33, 21, 8
+    X, M, G, Q = draw(rng, m, n, r)
+    res = orc.step(X, M, G, Q, MU, ETA, EPS)
+    alt = orc.step_given_panel(X, M, G, Q, (M + G) @ Q, MU, ETA, EPS)
+    for a, b in ((alt.X, res.X), (alt.M, res.M), (alt.Q, res.Q), (alt.d, res.d), (alt.U, res.U)):
+        assert rel(a, b) < 1e-12
+    # a scaled panel has the same thin-QR factor: the outputs do not move
+    alt2 = orc.step_given_panel(X, M, G, Q, 3.0 * ((M + G) @ Q), MU, ETA, EPS)
+    assert rel(alt2.X, res.X) < 1e-12 and rel(alt2.Q, res.Q) < 1e-12
+
+
 # -- generated benchmark inputs are in contract ---------------------------------
 
 def test_config1_ten_steps_stay_in_contract():
