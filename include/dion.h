@@ -228,6 +228,34 @@ int dion_dp_factor(dion_ctx* ctx, const dion_matrix* a, float* PU, float* W, int
 int dion_dp_finish(dion_ctx* ctx, const dion_matrix* a, const float* U, const float* W, const int* dp_flag,
                    float lr, void* cuda_stream);
 
+/* 1D-sharded Dion (Section 4.1, Algorithm 3): L layers of identical shape, their X, M, G and V sharded by columns
+ * over L ranks (rank x holds the columns J_x of every layer and the rows J_x of every V).  The library supplies
+ * what a rank computes between the collectives; the caller makes the collectives (any implementation; the
+ * library makes no collective call) and the payloads must be in this GPU's memory before a call reads them.
+ * `a` describes ONE layer's local shard: m x n_shard arrays X, M, G and Q = V[J_x, :] (n_shard x r; here r may
+ * exceed n_shard).  n_total = |J|, the unsharded number of columns (it fixes sqrt(m/n) and the automatic
+ * choice of Orthonormalize).  All buffers are DEVICE pointers, dense with leading dimension r, 16-byte aligned.
+ *   dion_shard_project (lines 1-2): P (m x r) <- (M + G) V on the shard: this rank's addend of layer l's P;
+ *                      clears *flag.
+ *   -- caller: ReduceScatter over the ranks along L: rank l receives the sum of every rank's P for layer l --
+ *   dion_orthonormalize (line 4, on the rank that owns the layer): PU holds P on entry, U on return;
+ *                      sets *flag if the panel broke down.
+ *   -- caller: AllGather of U (and of the owners' flags) --
+ *   dion_shard_factor  (line 6): W (n_shard x r) <- (M + G)^T U on the shard; colsumsq[r] <- the squared column
+ *                      norms of these n_shard rows of W.
+ *   -- caller: AllReduce(sum) of colsumsq over the ranks (r numbers per layer) --
+ *   dion_shard_finish  (lines 7-10): M <- (M + G) - (1 - mu) U W^T, Q <- W / (sqrt(colsumsq) + eps),
+ *                      X <- X - lr sqrt(m / n_total) U Q^T, all on the shard; does nothing (and counts a
+ *                      skipped step) when *flag != 0.  colnorm_out, if given, receives sqrt(colsumsq).
+ * Every layer's outputs equal those of dion_step on the unsharded layer up to the order of the sums.
+ * Standard form only; DION_ORTH_RCQR is not available in dion_orthonormalize.  Asynchronous on `cuda_stream`. */
+int dion_shard_project(dion_ctx* ctx, const dion_matrix* a, int64_t n_total, float* P, int* flag, void* cuda_stream);
+int dion_orthonormalize(dion_ctx* ctx, int64_t m, int64_t r, int64_t n_total, float* PU, int* flag, void* cuda_stream);
+int dion_shard_factor(dion_ctx* ctx, const dion_matrix* a, int64_t n_total, const float* U, float* W, float* colsumsq,
+                      const int* flag, void* cuda_stream);
+int dion_shard_finish(dion_ctx* ctx, const dion_matrix* a, int64_t n_total, const float* U, const float* W,
+                      const float* colsumsq, const int* flag, float lr, void* cuda_stream);
+
 /* Synchronises `cuda_stream`, then reports and clears the latched device status
  * (DION_STATUS_* bits) and the number of steps skipped because of a breakdown
  * since the last call.  Either output pointer may be NULL. */

@@ -243,6 +243,56 @@ def dp_step(X, Ms, Gs, Q, mu: float, eta: float, eps: float = 1e-8):
     return Xn, Mn, Qn, d
 
 
+def shard_bounds(n: int, ranks: int):
+    """Contiguous column blocks J_0, ..., J_{ranks-1} of 0..n-1 (the first n % ranks blocks one longer)."""
+    base, extra = divmod(n, ranks)
+    out, lo = [], 0
+    for x in range(ranks):
+        hi = lo + base + (1 if x < extra else 0)
+        out.append((lo, hi))
+        lo = hi
+    return out
+
+
+def sharded_step(X, M, G, Q, mu: float, eta: float, eps: float = 1e-8):
+    """1D-sharded Dion (Algorithm 3) on L layers of identical shape over |X| = L ranks, emulated rank by rank.
+    X, M, G: lists of L arrays (m x n); Q: list of L arrays (n x r).  Rank x holds the columns J_x of every layer's
+    X, M, G and the rows J_x of every layer's V; what it computes below uses only those (and what the
+    collectives hand it).  The lines follow the algorithm:
+      1  B = M + G on the local shards
+      2  partial P_x[l] = B[l][:, J_x] V[l][J_x, :]                        (unreduced over the ranks)
+      3  ReduceScatter along L: rank l receives P[l] = sum_x P_x[l]
+      4  rank l: U[l] = Orthonormalize(P[l])  (Householder thin QR, positive diagonal)
+      5  AllGather: every rank holds U[l] for all l
+      6  W_x[l] = B[l][:, J_x]^T U[l]                                      (rows J_x of W[l])
+      7  M_new[l][:, J_x] = B[l][:, J_x] - (1 - mu) U[l] W_x[l]^T
+      8  ColNorm with an AllReduce(sum) of the squared column norms over the ranks
+      9  O = U V_new^T on the shard; X_new = X - eta sqrt(m/n) O with n the full number of columns.
+    Returns (X_new, M_new, V_new, d): lists of L full arrays reassembled from the shards."""
+    L = len(X)
+    X = [_f64(a) for a in X]; M = [_f64(a) for a in M]; G = [_f64(a) for a in G]; Q = [_f64(a) for a in Q]
+    m, n = X[0].shape
+    r = Q[0].shape[1]
+    J = shard_bounds(n, L)
+    B = [[M[l][:, lo:hi] + G[l][:, lo:hi] for l in range(L)] for (lo, hi) in J]          # B[x][l]: rank x, layer l
+    Ppart = [[B[x][l] @ Q[l][J[x][0]:J[x][1], :] for l in range(L)] for x in range(L)]
+    P = [sum(Ppart[x][l] for x in range(L)) for l in range(L)]                           # rank l owns P[l]
+    U = [householder_qr(P[l])[0] for l in range(L)]
+    W = [[B[x][l].T @ U[l] for l in range(L)] for x in range(L)]
+    sumsq = [sum((W[x][l] * W[x][l]).sum(axis=0) for x in range(L)) for l in range(L)]   # AllReduce of r scalars per layer
+    d = [np.sqrt(sq) for sq in sumsq]
+    Xn = [np.empty((m, n)) for _ in range(L)]
+    Mn = [np.empty((m, n)) for _ in range(L)]
+    Vn = [np.empty((n, r)) for _ in range(L)]
+    for x, (lo, hi) in enumerate(J):
+        for l in range(L):
+            Vx = W[x][l] / (d[l] + eps)
+            Mn[l][:, lo:hi] = B[x][l] - (1.0 - mu) * (U[l] @ W[x][l].T)
+            Xn[l][:, lo:hi] = X[l][:, lo:hi] - eta * np.sqrt(m / n) * (U[l] @ Vx.T)
+            Vn[l][lo:hi, :] = Vx
+    return Xn, Mn, Vn, d
+
+
 def sym_power_iter(M, Q):
     """SymPowerIter1 (Algorithm 6): Orthonormalize(M^T M V)."""
     M = _f64(M); Q = _f64(Q).copy()

@@ -26,7 +26,7 @@ EXPORTS = ["dion_default_config", "dion_init", "dion_step", "dion_step_grouped",
            "dion_workspace_bytes", "dion_get_status", "dion_launch_count", "dion_destroy",
            "dion_strerror", "dion_profile_enable", "dion_profile_read", "dion_get_orth_rounds", "dion_get_fallbacks",
            "dion_step_noalloc", "dion_noalloc_scratch_limit", "dion_dp_project", "dion_dp_factor",
-           "dion_dp_finish"]
+           "dion_dp_finish", "dion_shard_project", "dion_orthonormalize", "dion_shard_factor", "dion_shard_finish"]
 PHASES = ["P", "ORTH", "R", "EF", "COLNORM", "X", "ORTH_GEMM"]
 
 
@@ -99,6 +99,14 @@ def load_library() -> ctypes.CDLL:
     lib.dion_dp_factor.restype = ci
     lib.dion_dp_finish.argtypes = [vp, ctypes.POINTER(DionMatrix), vp, vp, vp, f32, vp]
     lib.dion_dp_finish.restype = ci
+    lib.dion_shard_project.argtypes = [vp, ctypes.POINTER(DionMatrix), i64, vp, vp, vp]
+    lib.dion_shard_project.restype = ci
+    lib.dion_orthonormalize.argtypes = [vp, i64, i64, i64, vp, vp, vp]
+    lib.dion_orthonormalize.restype = ci
+    lib.dion_shard_factor.argtypes = [vp, ctypes.POINTER(DionMatrix), i64, vp, vp, vp, vp, vp]
+    lib.dion_shard_factor.restype = ci
+    lib.dion_shard_finish.argtypes = [vp, ctypes.POINTER(DionMatrix), i64, vp, vp, vp, vp, f32, vp]
+    lib.dion_shard_finish.restype = ci
     lib.dion_destroy.argtypes = [vp]
     lib.dion_destroy.restype = None
     lib.dion_strerror.argtypes = [ci]
@@ -241,6 +249,25 @@ class Dion:
                   stream=None) -> None:
         _check(self._lib.dion_dp_finish(self._ctx, ctypes.byref(desc), U.data_ptr(), W.data_ptr(), flag.data_ptr(),
                                         float(lr), _stream_ptr(stream)))
+
+    # 1D-sharded Dion (Algorithm 3): the per-rank pieces; the caller makes the collectives between them
+    def shard_project(self, desc: DionMatrix, n_total: int, P: torch.Tensor, flag: torch.Tensor, stream=None) -> None:
+        _check(self._lib.dion_shard_project(self._ctx, ctypes.byref(desc), int(n_total), P.data_ptr(), flag.data_ptr(),
+                                            _stream_ptr(stream)))
+
+    def orthonormalize(self, m: int, r: int, n_total: int, PU: torch.Tensor, flag: torch.Tensor, stream=None) -> None:
+        _check(self._lib.dion_orthonormalize(self._ctx, int(m), int(r), int(n_total), PU.data_ptr(), flag.data_ptr(),
+                                             _stream_ptr(stream)))
+
+    def shard_factor(self, desc: DionMatrix, n_total: int, U: torch.Tensor, W: torch.Tensor, colsumsq: torch.Tensor,
+                     flag: torch.Tensor, stream=None) -> None:
+        _check(self._lib.dion_shard_factor(self._ctx, ctypes.byref(desc), int(n_total), U.data_ptr(), W.data_ptr(),
+                                           colsumsq.data_ptr(), flag.data_ptr(), _stream_ptr(stream)))
+
+    def shard_finish(self, desc: DionMatrix, n_total: int, U: torch.Tensor, W: torch.Tensor, colsumsq: torch.Tensor,
+                     flag: torch.Tensor, lr: float, stream=None) -> None:
+        _check(self._lib.dion_shard_finish(self._ctx, ctypes.byref(desc), int(n_total), U.data_ptr(), W.data_ptr(),
+                                           colsumsq.data_ptr(), flag.data_ptr(), float(lr), _stream_ptr(stream)))
 
     def lazy_step_desc(self, desc: DionMatrix, lr: float, refresh: bool, stream_ptr: int) -> None:
         _check(self._lib.dion_lazy_step(self._ctx, ctypes.byref(desc), float(lr), int(bool(refresh)), stream_ptr))

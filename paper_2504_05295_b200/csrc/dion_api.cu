@@ -807,12 +807,13 @@ bool overlap(const void* a, size_t na, const void* b, size_t nb) {
   return a0 < b0 + nb && b0 < a0 + na;
 }
 
-int validate(const dion_matrix* a) {
+// shard: `a` describes a column shard of a wider matrix (the sharded calls): r may exceed its n.
+int validate(const dion_matrix* a, bool shard = false) {
   if (a == nullptr) return DION_ERR_INVALID;
   if (a->X == nullptr || a->M == nullptr || a->G == nullptr || a->Q == nullptr) return DION_ERR_INVALID;
   if (a->g_dtype != DION_F32 && a->g_dtype != DION_BF16) return DION_ERR_INVALID;
   if (a->m < 1 || a->n < 1) return DION_ERR_SHAPE;
-  if (a->r < 1 || a->r > a->m || a->r > a->n) return DION_ERR_SHAPE;
+  if (a->r < 1 || a->r > a->m || (!shard && a->r > a->n)) return DION_ERR_SHAPE;
   if (a->ldx < a->n || a->ldm < a->n || a->ldg < a->n || a->ldq < a->r) return DION_ERR_SHAPE;
   if (a->transposed != 0 && a->transposed != 1) return DION_ERR_INVALID;
   const i64 qrows = a->transposed ? a->m : a->n;
@@ -1410,6 +1411,117 @@ int dion_dp_finish(dion_ctx* ctx, const dion_matrix* a, const float* U, const fl
   DION_TRY(x_update(s, 0, a, U, r, (const float*)a->Q, a->ldq, s.ws + s.L.P1, s.ws + s.L.R,
                     lr * sqrtf((float)((double)m / (double)n)), dp_flag));
   launch_pdl(k_finish_step, dim3((unsigned)(1)), dim3(1), 0, st, dp_flag, ctx->dev_ints + 1);
+  DION_CHECK_LAUNCH(ctx);
+  return DION_OK;
+}
+
+// ---- 1D-sharded Dion (Algorithm 3): the per-rank pieces between its collectives -------------------
+
+namespace {
+
+int shard_check(dion_ctx* ctx, const dion_matrix* a, int64_t n_total, const void* p0, const void* p1, const int* flag) {
+  if (ctx == nullptr || p0 == nullptr || p1 == nullptr || flag == nullptr) return DION_ERR_INVALID;
+  DION_TRY(validate(a, true));
+  if (a->transposed || n_total < a->n || a->r > n_total) return DION_ERR_INVALID;
+  if (((uintptr_t)p0 & 15) || ((uintptr_t)p1 & 15) || ((uintptr_t)flag & 3)) return DION_ERR_ALIGN;
+  if (cudaSetDevice(ctx->cfg.device) != cudaSuccess) return DION_ERR_CUDA;
+  return ensure_ws(ctx, (size_t)make_layout(ctx, a->m, a->n, a->r).total * sizeof(float));
+}
+
+}  // namespace
+
+int dion_shard_project(dion_ctx* ctx, const dion_matrix* a, int64_t n_total, float* P, int* flag, void* cuda_stream) {
+  DION_TRY(shard_check(ctx, a, n_total, P, P, flag));
+  StepCtx s;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  DION_TRY(begin_step(ctx, a, 1, st, &s));
+  if (cudaMemsetAsync(flag, 0, sizeof(int), st) != cudaSuccess) return DION_ERR_CUDA;
+  GemmArgs p = dp_b_product(a, false, (const float*)a->Q, P);
+  p.b_sk = a->ldq;
+  p.precise = (resolve_orth(ctx, a->r, (a->m < n_total) ? a->m : n_total) == DION_ORTH_SHIFTED3) ? 1 : 0;
+  return launch_gemm(s, p, 0);
+}
+
+int dion_orthonormalize(dion_ctx* ctx, int64_t m, int64_t r, int64_t n_total, float* PU, int* flag, void* cuda_stream) {
+  if (ctx == nullptr || PU == nullptr || flag == nullptr) return DION_ERR_INVALID;
+  if (m < 1 || n_total < 1 || r < 1 || r > m || r > n_total) return DION_ERR_SHAPE;
+  if (((uintptr_t)PU & 15) || ((uintptr_t)flag & 3)) return DION_ERR_ALIGN;
+  if (ctx->cfg.orth == DION_ORTH_RCQR) return DION_ERR_UNSUPPORTED;
+  if (cudaSetDevice(ctx->cfg.device) != cudaSuccess) return DION_ERR_CUDA;
+  dion_matrix shape;
+  memset(&shape, 0, sizeof(shape));
+  shape.m = m; shape.n = n_total; shape.r = r;
+  DION_TRY(ensure_ws(ctx, (size_t)make_layout(ctx, m, n_total, r).total * sizeof(float)));
+  StepCtx s;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  DION_TRY(begin_step(ctx, &shape, 1, st, &s));
+  const i64 sd = (m < n_total) ? m : n_total;
+  const i64 pin_off = panel_offset(s, r, sd);
+  dim3 grid((unsigned)grid_for(ctx, m * r), 1);
+  launch_pdl(k_copy_block, grid, dim3(256), 0, st, (const float*)PU, r, s.ws + pin_off, r, m, r, nullptr, 0);
+  DION_CHECK_LAUNCH(ctx);
+  i64 U_off = 0;
+  s.in_orth = true;
+  const int rc = orthonormalize(s, m, r, sd, pin_off, &U_off);
+  s.in_orth = false;
+  DION_TRY(rc);
+  launch_pdl(k_copy_block, grid, dim3(256), 0, st, (const float*)(s.ws + U_off), r, PU, r, m, r, nullptr, 0);
+  DION_CHECK_LAUNCH(ctx);
+  launch_pdl(k_latch_flag, dim3(1), dim3(1), 0, st, (const int*)s.flag, flag);
+  DION_CHECK_LAUNCH(ctx);
+  return DION_OK;
+}
+
+int dion_shard_factor(dion_ctx* ctx, const dion_matrix* a, int64_t n_total, const float* U, float* W, float* colsumsq,
+                      const int* flag, void* cuda_stream) {
+  DION_TRY(shard_check(ctx, a, n_total, U, W, flag));
+  if (colsumsq == nullptr) return DION_ERR_INVALID;
+  StepCtx s;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  DION_TRY(begin_step(ctx, a, 1, st, &s));
+  GemmArgs w = dp_b_product(a, true, U, W);
+  w.skip_flag = flag;
+  DION_TRY(launch_gemm(s, w, 0));
+  int chunks; i64 per;
+  colnorm_plan(a->n, a->r, ctx->sm_count, &chunks, &per);
+  float* part = s.W(0, s.L.cn_part);
+  dim3 grid((unsigned)((a->r + 127) / 128), (unsigned)chunks);
+  launch_pdl(k_colsumsq_partial, grid, dim3(128), 0, st, (const float*)W, a->r, a->n, a->r, per, part, flag);
+  DION_CHECK_LAUNCH(ctx);
+  launch_pdl(k_colsumsq_finish, dim3((unsigned)((a->r + 127) / 128)), dim3(128), 0, st, (const float*)part, chunks, a->r, colsumsq, flag);
+  DION_CHECK_LAUNCH(ctx);
+  return DION_OK;
+}
+
+int dion_shard_finish(dion_ctx* ctx, const dion_matrix* a, int64_t n_total, const float* U, const float* W,
+                      const float* colsumsq, const int* flag, float lr, void* cuda_stream) {
+  DION_TRY(shard_check(ctx, a, n_total, U, W, flag));
+  if (colsumsq == nullptr) return DION_ERR_INVALID;
+  StepCtx s;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  DION_TRY(begin_step(ctx, a, 1, st, &s));
+  const i64 m = a->m, n = a->n, r = a->r;
+  GemmArgs e = gemm_args();      // M <- (M + G) - (1 - mu) U W^T on the shard's columns
+  e.M = m; e.N = n; e.K = r;
+  e.A = U; e.a_si = r; e.a_sk = 1;
+  e.B = W; e.b_sk = 1; e.b_sn = r;
+  e.C = (float*)a->M; e.ldc = a->ldm; e.epi = EPI_ADD2_SUB;
+  e.C2 = a->G; e.ldc2 = a->ldg; e.c2_mode = (a->g_dtype == DION_BF16) ? ADD_BF16 : ADD_F32;
+  e.alpha = 1.f - ctx->cfg.mu;
+  e.skip_flag = flag;
+  DION_TRY(launch_gemm(s, e, 0));
+  {   // Q <- W / (sqrt(colsumsq) + eps): the squared column norms are the all-reduced ones (one "chunk")
+    int chunks; i64 per;
+    colnorm_plan(n, r, ctx->sm_count, &chunks, &per);
+    dim3 grid((unsigned)((r + 127) / 128), (unsigned)chunks);
+    launch_pdl(k_colnorm_apply, grid, dim3(128), 0, st, W, r, n, r, per, 1, colsumsq, ctx->cfg.eps, (float*)a->Q, a->ldq,
+               s.W(0, s.L.d), a->colnorm_out, ctx->dev_ints, flag);
+    DION_CHECK_LAUNCH(ctx);
+  }
+  // X <- X - lr sqrt(m / n_total) U Q^T on the shard's columns
+  DION_TRY(x_update(s, 0, a, U, r, (const float*)a->Q, a->ldq, s.ws + s.L.P1, s.ws + s.L.R,
+                    lr * sqrtf((float)((double)m / (double)n_total)), flag));
+  launch_pdl(k_finish_step, dim3(1), dim3(1), 0, st, flag, ctx->dev_ints + 1);
   DION_CHECK_LAUNCH(ctx);
   return DION_OK;
 }

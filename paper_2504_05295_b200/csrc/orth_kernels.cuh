@@ -858,6 +858,19 @@ __global__ void __launch_bounds__(128) k_colsumsq_partial(const float* __restric
   part[(i64)blockIdx.y * r + j] = s;
 }
 
+// out[j] = sum over the chunks (in order) of part[chunk][j]: the squared column norms of a shard's rows,
+// handed to the caller for the all-reduce over the shards (1D-sharded Dion).
+__global__ void __launch_bounds__(128) k_colsumsq_finish(const float* __restrict__ part, int chunks, i64 r,
+                                                         float* __restrict__ out, const int* __restrict__ skip_flag) {
+  pdl_enter();
+  if (skip_flag != nullptr && *skip_flag != 0) return;
+  const i64 j = (i64)blockIdx.x * 128 + threadIdx.x;
+  if (j >= r) return;
+  float s = 0.f;
+  for (int c = 0; c < chunks; ++c) s += part[(i64)c * r + j];
+  out[j] = s;
+}
+
 // ColNorm: d_j = sqrt(sum of the partials in chunk order); Q[i][j] = R[i][j] / (d_j + eps).
 // Same grid as k_colsumsq_partial.  The chunk-0 blocks also export d.
 __global__ void __launch_bounds__(128) k_colnorm_apply(const float* __restrict__ R, i64 ldr, i64 n, i64 r,

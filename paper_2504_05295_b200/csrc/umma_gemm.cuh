@@ -113,6 +113,59 @@ __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
+// ---- CTA pair (cta_group::2): two CTAs of a cluster share one 256-row MMA
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// arrive on the mbarrier at the same shared-memory offset in CTA `rank` of the cluster
+__device__ __forceinline__ void mbar_arrive_remote(uint32_t bar, uint32_t rank) {
+  asm volatile(
+      "{\n\t.reg .b32 ra;\n\t"
+      "mapa.shared::cluster.u32 ra, %0, %1;\n\t"
+      "mbarrier.arrive.release.cluster.shared::cluster.b64 _, [ra];\n\t}" ::"r"(bar), "r"(rank)
+      : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ void tmem_alloc2(uint32_t slot, uint32_t ncols) {
+  asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(slot), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish2() {
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc2(uint32_t taddr, uint32_t ncols) {
+  asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+// one 256 x N x 8 TF32 MMA of the CTA pair, issued by the leader CTA
+__device__ __forceinline__ void umma2_tf32(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::tf32 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+      "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// commit of the pair's MMAs: arrives on the mbarrier at this offset in every CTA of `mask`
+__device__ __forceinline__ void umma2_commit(uint32_t bar, uint16_t mask) {
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::"r"(bar),
+               "h"(mask)
+               : "memory");
+}
+
 __device__ __forceinline__ void tmem_alloc(uint32_t slot, uint32_t ncols) {
   asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(slot), "r"(ncols) : "memory");
 }
@@ -171,13 +224,15 @@ __device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t
 // Bounded wait: false when the CTA is (or becomes) dead.
 // `sleep_ns` > 0 backs off between polls so that a waiting warp does not take issue
 // slots from the producer warps.
+template <bool CLUSTER = false>
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* dead, int* status,
                                           long long limit, unsigned sleep_ns = 0) {
-  if (mbar_try_wait(bar, parity)) return true;
+  // CLUSTER: the barrier takes arrivals from the peer CTA (acquire at cluster scope)
+  if (CLUSTER ? mbar_try_wait_cluster(bar, parity) : mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   unsigned polls = 0;
   while (true) {
-    if (mbar_try_wait(bar, parity)) return true;
+    if (CLUSTER ? mbar_try_wait_cluster(bar, parity) : mbar_try_wait(bar, parity)) return true;
     if (sleep_ns) __nanosleep(sleep_ns);
     if ((++polls & 63u) == 0) {
       if (*dead) return false;
@@ -225,7 +280,7 @@ __device__ __forceinline__ uint64_t make_desc_k64(uint32_t saddr) {
 }
 
 // Instruction descriptor: fp32 accumulate, TF32 or BF16 operands, M = 128, N = BN.
-__device__ __forceinline__ uint32_t make_idesc(bool bf16, bool a_mn, bool b_mn, int bn) {
+__device__ __forceinline__ uint32_t make_idesc(bool bf16, bool a_mn, bool b_mn, int bn, int bm = BM) {
   uint32_t d = 0;
   d |= 1u << 4;                         // D format: F32
   d |= (bf16 ? 1u : 2u) << 7;           // A format
@@ -233,7 +288,7 @@ __device__ __forceinline__ uint32_t make_idesc(bool bf16, bool a_mn, bool b_mn, 
   d |= (a_mn ? 1u : 0u) << 15;
   d |= (b_mn ? 1u : 0u) << 16;
   d |= (uint32_t)(bn >> 3) << 17;
-  d |= (uint32_t)(BM >> 4) << 24;
+  d |= (uint32_t)(bm >> 4) << 24;
   return d;
 }
 
@@ -243,12 +298,13 @@ struct Item {
   int mi, ni, ks, kb0, kb1;
 };
 
-template <int BN, int BKE>
+// CG2: `mi` counts 256-row tiles of a CTA pair (256 x 256 lower tiles in the triangular case).
+template <int BN, int BKE, bool CG2 = false>
 __device__ __forceinline__ Item decode_item(const Params& p, int item) {
   Item it;
   const int tile = item / p.splits;
   it.ks = item - tile * p.splits;
-  if (p.g.tri == TRI_LOWER && BN == 2 * BM) {
+  if (p.g.tri == TRI_LOWER && BN == 2 * BM && !CG2) {
     // 128 x 256 tiles that reach the diagonal or lie below it: tile row mi has mi / 2 + 1 of them,
     // (mi + 1)^2 / 4 (rounded down) lie in the rows above it
     int mi = (int)(2.f * sqrtf((float)tile)) - 1;
@@ -411,7 +467,13 @@ struct TileMap {
 // no "lo" halves, no conversion pass, the producer warps join the epilogue as in the bf16-array variant.
 // Used for the rank-r update of X, whose result feeds nothing else: an unbiased 2^-12 relative operand
 // error there moves X by ~1e-6.
-template <int BN, bool BF16, bool SPLIT = false, bool TMA = false, bool D16 = false, bool CE = false, bool ONE = false>
+// CG2 (fp32 mode, TMA, BN = 256): two CTAs of a cluster form one 256 x 256 tile with cta_group::2 MMAs.
+// Each CTA loads and converts its own 128 rows of A and HALF of the B tile (128 of the 256 columns), so a
+// K block costs a CTA two thirds of the shared-memory traffic of the single-CTA form (which is bound by
+// it: three MMAs re-read both operand tiles) and a stage is 64 KB instead of 96 KB (3 stages instead of 2).
+// The leader CTA issues the MMAs for both; accumulators and epilogue stay per CTA (128 rows x 256 columns).
+template <int BN, bool BF16, bool SPLIT = false, bool TMA = false, bool D16 = false, bool CE = false, bool ONE = false,
+          bool CG2 = false>
 struct Cfg {
   // BT: bf16 operands formed in shared memory from TMA-loaded fp32 tiles (K block of 32, as in
   // the fp32 TMA variant).  A stage then holds the raw fp32 tiles of A, of its fp32 addend and
@@ -422,7 +484,8 @@ struct Cfg {
   static constexpr int BKE = (BF16 && (!TMA || D16)) ? 64 : 32;   // K elements per stage
   static constexpr int EPC = (BF16 && !TMA) ? 8 : 4;         // elements per 16-byte chunk of the register path
   static constexpr int A_BYTES = BM * 128;
-  static constexpr int B_BYTES = BN * 128;
+  static constexpr int BN_L = CG2 ? BN / 2 : BN;             // columns of the B tile this CTA holds
+  static constexpr int B_BYTES = BN_L * 128;
   static constexpr int STAGE_BYTES = BT ? (2 * A_BYTES + B_BYTES + A_BYTES / 2 + B_BYTES / 2)
                                         : ((BF16 || ONE) ? 1 : 2) * (A_BYTES + B_BYTES);
   // D16: the producer warps have no conversion work and serve as epilogue warps too
@@ -440,7 +503,7 @@ struct Cfg {
   static constexpr int G16_BYTES = ((BF16 && !TMA) || D16 || CE) ? 0 : BM * 32 * 2;   // bf16 addend tile of the TMA variants (per stage)
   static constexpr int SMEM_BYTES = STAGES * (STAGE_BYTES + G16_BYTES) + EPI_BYTES + 1024 + 512;
   static constexpr int A_CHUNKS = BM * 8 / NUM_PROD_THREADS;  // 16-byte chunks per producer thread
-  static constexpr int B_CHUNKS = BN * 8 / NUM_PROD_THREADS;
+  static constexpr int B_CHUNKS = BN_L * 8 / NUM_PROD_THREADS;
   static constexpr int ACCS = SPLIT ? 2 : 1;                 // accumulators per tile
   static constexpr int NBUF = (512 / (ACCS * BN)) >= 2 ? 2 : 1;  // tiles in flight in TMEM
   static constexpr int TMEM_COLS = NBUF * ACCS * BN;
@@ -457,14 +520,20 @@ struct Cfg {
 // TMA with bf16 operands: the same loads; the producer warps add, round to bf16 and write
 // the operand tiles the MMA reads (k-contiguous: rows of 64 bytes, 64-byte swizzle;
 // row-contiguous: 128-byte rows of 64 row indices, 128-byte swizzle); one MMA per K step.
-template <int BN, bool A_MN, bool B_MN, bool BF16, bool SPLIT, bool TMA, bool D16 = false, bool CE = false, bool ONE = false>
+template <int BN, bool A_MN, bool B_MN, bool BF16, bool SPLIT, bool TMA, bool D16 = false, bool CE = false, bool ONE = false,
+          bool CG2 = false>
 __global__ void __launch_bounds__(TMA ? NUM_THREADS_TMA : NUM_THREADS, 1) k_gemm_umma(const __grid_constant__ Params p) {
+  static_assert(!CG2 || (TMA && !BF16 && !D16 && !ONE && BN == 256), "CTA pairs: the fp32 TMA variants with 256-column tiles");
   static_assert(!(BF16 && SPLIT), "split accumulators belong to the 3xTF32 mode");
   static_assert(!D16 || (BF16 && TMA), "bf16 operands in memory are loaded by TMA");
   static_assert(!CE || (TMA && (D16 || !BF16)), "the coalesced epilogue serves the bf16-array and the fp32 TMA variants");
   static_assert(!ONE || (TMA && CE && !BF16 && !SPLIT && !A_MN && !B_MN), "single pass: k-contiguous fp32 operands by TMA");
-  using C = Cfg<BN, BF16, SPLIT, TMA, D16, CE, ONE>;
+  using C = Cfg<BN, BF16, SPLIT, TMA, D16, CE, ONE, CG2>;
   constexpr bool NOCONV = D16 || ONE;    // the operand tiles are what TMA writes: nothing to convert
+  constexpr int BN_L = C::BN_L;
+  const uint32_t cta_rank = CG2 ? cluster_ctarank() : 0u;   // 0: the leader of the pair
+  const int worker = CG2 ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;       // which tile stream this CTA (pair) walks
+  const int workers = CG2 ? (int)(gridDim.x >> 1) : (int)gridDim.x;
   constexpr int NBUF = C::NBUF, ACCS = C::ACCS;
   constexpr int BKE = C::BKE, EPC = C::EPC, STAGES = C::STAGES;
   if (p.g.skip_flag != nullptr && *p.g.skip_flag != 0) return;
@@ -490,19 +559,21 @@ __global__ void __launch_bounds__(TMA ? NUM_THREADS_TMA : NUM_THREADS, 1) k_gemm
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), NUM_PROD_WARPS); mbar_init(empty_bar(s), 1); }
-    for (int b = 0; b < 2; ++b) { mbar_init(accf_bar(b), 1); mbar_init(acce_bar(b), C::EPI_WARPS * 32); }
+    // CTA pair: the leader's "full" and "accumulator free" barriers take the arrivals of both CTAs
+    for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), NUM_PROD_WARPS * (CG2 ? 2 : 1)); mbar_init(empty_bar(s), 1); }
+    for (int b = 0; b < 2; ++b) { mbar_init(accf_bar(b), 1); mbar_init(acce_bar(b), C::EPI_WARPS * 32 * (CG2 ? 2 : 1)); }
     mbar_init(drain_bar, 1);
     if (TMA) for (int s = 0; s < STAGES; ++s) mbar_init(raw_bar(s), 1);
     *dead = 0;
     fence_barrier_init();
   }
   if (warp == NUM_EPI_WARPS + NUM_PROD_WARPS) {
-    tmem_alloc(smem_u32((const void*)tmem_slot), C::TMEM_COLS);
-    tmem_relinquish();
+    if (CG2) { tmem_alloc2(smem_u32((const void*)tmem_slot), C::TMEM_COLS); tmem_relinquish2(); }
+    else { tmem_alloc(smem_u32((const void*)tmem_slot), C::TMEM_COLS); tmem_relinquish(); }
   }
   tc_fence_before();
   __syncthreads();
+  if (CG2) cluster_sync_all();      // the peer's barriers are initialised before anything arrives on them
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
@@ -517,8 +588,9 @@ __global__ void __launch_bounds__(TMA ? NUM_THREADS_TMA : NUM_THREADS, 1) k_gemm
     // running result in global memory.
     int iter = 0;
     bool alive = true;
-    for (int item = blockIdx.x; item < p.num_items && alive; item += gridDim.x) {
-      const Item it = decode_item<BN, BKE>(p, item);
+    for (int item = worker; item < p.num_items && alive; item += workers) {
+      Item it = decode_item<BN, BKE, CG2>(p, item);
+      if (CG2) it.mi = 2 * it.mi + (int)cta_rank;     // this CTA's 128 rows of the pair's tile
       const int quad = warp & 3, half = warp >> 2;   // TMEM lane quadrant, column part
       constexpr int SLABS = (BN / 32) / (C::EPI_WARPS / 4);   // 32-column slabs per warp
       const i64 gi = (i64)it.mi * BM + quad * 32 + lane;
@@ -664,7 +736,8 @@ __global__ void __launch_bounds__(TMA ? NUM_THREADS_TMA : NUM_THREADS, 1) k_gemm
           }
         }
         tc_fence_before();
-        mbar_arrive(acce_bar(ab));
+        if (CG2 && cta_rank != 0) mbar_arrive_remote(acce_bar(ab), 0u);
+        else mbar_arrive(acce_bar(ab));
       }
     }
   } else if (warp < NUM_EPI_WARPS + NUM_PROD_WARPS) {
@@ -713,8 +786,8 @@ __global__ void __launch_bounds__(TMA ? NUM_THREADS_TMA : NUM_THREADS, 1) k_gemm
       int stage = 0;
       uint32_t phase = 0;
       bool alive = true;
-      for (int item = blockIdx.x; item < p.num_items && alive; item += gridDim.x) {
-        const Item it = decode_item<BN, BKE>(p, item);
+      for (int item = worker; item < p.num_items && alive; item += workers) {
+        const Item it = decode_item<BN, BKE, CG2>(p, item);
         for (int kb = it.kb0; kb < it.kb1; ++kb) {
           if (!mbar_wait(raw_bar(stage), phase, dead, p.status, p.spin_limit)) { alive = false; break; }
           const uint32_t sg16 = g16_base + stage * C::G16_BYTES;
@@ -766,7 +839,10 @@ __global__ void __launch_bounds__(TMA ? NUM_THREADS_TMA : NUM_THREADS, 1) k_gemm
           }
           fence_proxy_async();
           __syncwarp();
-          if (lane == 0) mbar_arrive(full_bar(stage));
+          if (lane == 0) {
+            if (CG2 && cta_rank != 0) mbar_arrive_remote(full_bar(stage), 0u);
+            else mbar_arrive(full_bar(stage));
+          }
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
       }
@@ -820,9 +896,11 @@ __global__ void __launch_bounds__(TMA ? NUM_THREADS_TMA : NUM_THREADS, 1) k_gemm
       int stage = 0;
       uint32_t phase = 0;
       bool alive = true;
-      for (int item = blockIdx.x; item < p.num_items && alive; item += gridDim.x) {
-        const Item it = decode_item<BN, BKE>(p, item);
-        const int row0a = it.mi * BM, row0b = it.ni * BN;
+      for (int item = worker; item < p.num_items && alive; item += workers) {
+        const Item it = decode_item<BN, BKE, CG2>(p, item);
+        // CTA pair: this CTA's 128 rows of A and its half of the B tile's columns
+        const int row0a = (CG2 ? 2 * it.mi + (int)cta_rank : it.mi) * BM;
+        const int row0b = it.ni * BN + (CG2 ? (int)cta_rank * BN_L : 0);
         for (int kb = it.kb0; kb < it.kb1; ++kb) {
           if (!mbar_wait(empty_bar(stage), phase ^ 1u, dead, p.status, p.spin_limit, 32)) { alive = false; break; }
           const int k0 = kb * BKE;
@@ -871,7 +949,7 @@ __global__ void __launch_bounds__(TMA ? NUM_THREADS_TMA : NUM_THREADS, 1) k_gemm
             tma_load_2d(sb, &p.tmB, k0, row0b, bar);
           } else {
 #pragma unroll
-            for (int c = 0; c < BN / 32; ++c) tma_load_2d(sb + c * (BKE * 128), &p.tmB, row0b + 32 * c, k0, bar);
+            for (int c = 0; c < BN_L / 32; ++c) tma_load_2d(sb + c * (BKE * 128), &p.tmB, row0b + 32 * c, k0, bar);
           }
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
@@ -879,9 +957,9 @@ __global__ void __launch_bounds__(TMA ? NUM_THREADS_TMA : NUM_THREADS, 1) k_gemm
     }
     __syncwarp();
   } else {
-    // ------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
-      const uint32_t idesc = make_idesc(BF16, A_MN, B_MN, BN);
+    // ------------------------------------------------------------ MMA issuer (CTA pair: the leader only)
+    if (lane == 0 && (!CG2 || cta_rank == 0)) {
+      const uint32_t idesc = make_idesc(BF16, A_MN, B_MN, BN, CG2 ? 2 * BM : BM);
       const uint32_t lbo = BKE * 128;
       constexpr uint32_t A_KSTEP = A_MN ? (BF16 ? 2048u : 1024u) : 32u;   // bytes per UMMA K step
       constexpr uint32_t B_KSTEP = B_MN ? (BF16 ? 2048u : 1024u) : 32u;
@@ -889,19 +967,19 @@ __global__ void __launch_bounds__(TMA ? NUM_THREADS_TMA : NUM_THREADS, 1) k_gemm
       uint32_t phase = 0;
       int iter = 0;
       bool alive = true;
-      for (int item = blockIdx.x; item < p.num_items && alive; item += gridDim.x) {
-        const Item it = decode_item<BN, BKE>(p, item);
+      for (int item = worker; item < p.num_items && alive; item += workers) {
+        const Item it = decode_item<BN, BKE, CG2>(p, item);
         for (int kbc = it.kb0; kbc < it.kb1 && alive; kbc += p.kc, ++iter) {   // one accumulation chunk
         const int kbc1 = min(it.kb1, kbc + p.kc);
         const int ab = iter % NBUF;
         const uint32_t aph = (uint32_t)(iter / NBUF) & 1u;
-        if (!mbar_wait(acce_bar(ab), aph ^ 1u, dead, p.status, p.spin_limit, 64)) { alive = false; break; }
+        if (!mbar_wait<CG2>(acce_bar(ab), aph ^ 1u, dead, p.status, p.spin_limit, 64)) { alive = false; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(ab * ACCS * BN);
         const uint32_t d_small = d_tmem + (SPLIT ? BN : 0);
         uint32_t accumulate = 0;
         for (int kb = kbc; kb < kbc1; ++kb) {
-          if (!mbar_wait(NOCONV ? raw_bar(stage) : full_bar(stage), phase, dead, p.status, p.spin_limit)) { alive = false; break; }
+          if (!mbar_wait<CG2>(NOCONV ? raw_bar(stage) : full_bar(stage), phase, dead, p.status, p.spin_limit)) { alive = false; break; }
           tc_fence_after();
           const uint32_t st0 = smem_base + stage * C::STAGE_BYTES;
           // bf16 operands formed from TMA tiles sit behind the raw tiles of the stage
@@ -922,7 +1000,18 @@ __global__ void __launch_bounds__(TMA ? NUM_THREADS_TMA : NUM_THREADS, 1) k_gemm
             } else {
               const uint64_t a_lo = make_desc<BF16>(sa_lo + ks * A_KSTEP, A_MN, lbo);
               const uint64_t b_lo = make_desc<BF16>(sb_lo + ks * B_KSTEP, B_MN, lbo);
-              if (SPLIT) {
+              if (CG2) {
+                if (SPLIT) {
+                  umma2_tf32(d_small, a_hi, b_lo, idesc, accumulate);
+                  umma2_tf32(d_small, a_lo, b_hi, idesc, 1u);
+                  umma2_tf32(d_small, a_lo, b_lo, idesc, 1u);
+                  umma2_tf32(d_tmem, a_hi, b_hi, idesc, accumulate);
+                } else {
+                  umma2_tf32(d_tmem, a_hi, b_lo, idesc, accumulate);
+                  umma2_tf32(d_tmem, a_lo, b_hi, idesc, 1u);
+                  umma2_tf32(d_tmem, a_hi, b_hi, idesc, 1u);
+                }
+              } else if (SPLIT) {
                 umma<false>(d_small, a_hi, b_lo, idesc, accumulate);
                 umma<false>(d_small, a_lo, b_hi, idesc, 1u);
                 // truncation remainders all carry the sign of their operand: lo * lo is not noise
@@ -936,15 +1025,18 @@ __global__ void __launch_bounds__(TMA ? NUM_THREADS_TMA : NUM_THREADS, 1) k_gemm
               accumulate = 1;
             }
           }
-          umma_commit(empty_bar(stage));        // the stage may be refilled once these MMAs are done
+          if (CG2) umma2_commit(empty_bar(stage), (uint16_t)3);   // both CTAs may refill the stage
+          else umma_commit(empty_bar(stage));   // the stage may be refilled once these MMAs are done
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
         if (!alive) break;
-        umma_commit(accf_bar(ab));              // this chunk's accumulator is complete
+        if (CG2) umma2_commit(accf_bar(ab), (uint16_t)3);   // each CTA's epilogue reads its own half
+        else umma_commit(accf_bar(ab));         // this chunk's accumulator is complete
         }
       }
       // drain: every issued MMA must have finished before TMEM is released
-      umma_commit(drain_bar);
+      if (CG2) umma2_commit(drain_bar, (uint16_t)1);
+      else umma_commit(drain_bar);
       mbar_wait(drain_bar, 0u, dead, p.status, p.spin_limit, 64);
     }
     __syncwarp();
@@ -952,16 +1044,70 @@ __global__ void __launch_bounds__(TMA ? NUM_THREADS_TMA : NUM_THREADS, 1) k_gemm
 
   tc_fence_before();
   __syncthreads();
+  // CTA pair: neither CTA may leave (or free its accumulators) while the other still arrives on its barriers
+  // or the leader's MMAs still read its shared memory
+  if (CG2) cluster_sync_all();
   if (warp == NUM_EPI_WARPS + NUM_PROD_WARPS) {
     tc_fence_after();
-    tmem_dealloc(tmem_base, C::TMEM_COLS);
+    if (CG2) tmem_dealloc2(tmem_base, C::TMEM_COLS);
+    else tmem_dealloc(tmem_base, C::TMEM_COLS);
   }
 }
 
-template <int BN, bool A_MN, bool B_MN, bool BF16, bool SPLIT, bool TMA, bool D16 = false, bool CE = false, bool ONE = false>
+template <int BN, bool A_MN, bool B_MN, bool BF16, bool SPLIT, bool TMA, bool D16 = false, bool CE = false, bool ONE = false,
+          bool CG2 = false>
 inline cudaError_t set_smem_attr() {
-  return cudaFuncSetAttribute(k_gemm_umma<BN, A_MN, B_MN, BF16, SPLIT, TMA, D16, CE, ONE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              Cfg<BN, BF16, SPLIT, TMA, D16, CE, ONE>::SMEM_BYTES);
+  return cudaFuncSetAttribute(k_gemm_umma<BN, A_MN, B_MN, BF16, SPLIT, TMA, D16, CE, ONE, CG2>,
+                              cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<BN, BF16, SPLIT, TMA, D16, CE, ONE, CG2>::SMEM_BYTES);
+}
+
+// CTA pairs: clusters of two CTAs, 256 x 256 tiles (fp32 mode, TMA, coalesced epilogue)
+template <bool A_MN, bool B_MN, bool SPLIT>
+inline cudaError_t launch_pair_one(const Params& p, int grid, cudaStream_t st) {
+  constexpr int smem = Cfg<256, false, SPLIT, true, false, true, false, true>::SMEM_BYTES;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)grid); cfg.blockDim = dim3(NUM_THREADS_TMA); cfg.dynamicSmemBytes = smem; cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr; cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, k_gemm_umma<256, A_MN, B_MN, false, SPLIT, true, false, true, false, true>, p);
+}
+template <bool SPLIT>
+inline cudaError_t launch_pair(const Params& p, bool a_mn, bool b_mn, int grid, cudaStream_t st) {
+  if (!a_mn && !b_mn) return launch_pair_one<false, false, SPLIT>(p, grid, st);
+  if (!a_mn && b_mn) return launch_pair_one<false, true, SPLIT>(p, grid, st);
+  if (a_mn && b_mn) return launch_pair_one<true, true, SPLIT>(p, grid, st);
+  return launch_pair_one<true, false, SPLIT>(p, grid, st);
+}
+template <bool A_MN, bool B_MN>
+inline cudaError_t set_pair_attr() {
+  cudaError_t e = set_smem_attr<256, A_MN, B_MN, false, false, true, false, true, false, true>();
+  if (e == cudaSuccess) e = set_smem_attr<256, A_MN, B_MN, false, true, true, false, true, false, true>();
+  return e;
+}
+// How many CTA pairs can be resident at once (per device, asked once).
+inline int pair_clusters(int sm_count) {
+  static int cached[64] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return sm_count / 2; }
+  if (dev >= 0 && dev < 64 && cached[dev] > 0) return cached[dev];
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)(sm_count / 2 * 2)); cfg.blockDim = dim3(NUM_THREADS_TMA);
+  cfg.dynamicSmemBytes = Cfg<256, false, false, true, false, true, false, true>::SMEM_BYTES;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr; cfg.numAttrs = 1;
+  int n = 0;
+  if (cudaOccupancyMaxActiveClusters(&n, k_gemm_umma<256, false, false, false, false, true, false, true, false, true>, &cfg) != cudaSuccess ||
+      n < 1) {
+    cudaGetLastError();
+    n = 0;
+  }
+  if (n > sm_count / 2) n = sm_count / 2;
+  if (dev >= 0 && dev < 64) cached[dev] = n > 0 ? n : -1;
+  return n;
 }
 
 // single-pass TF32 (k-contiguous operands only)
@@ -1087,6 +1233,10 @@ inline int umma_configure() {
 #undef DION_SET
   if (e == cudaSuccess) e = set_smem_attr<128, false, false, false, false, true, false, true, true>();
   if (e == cudaSuccess) e = set_smem_attr<256, false, false, false, false, true, false, true, true>();
+  if (e == cudaSuccess) e = set_pair_attr<false, false>();
+  if (e == cudaSuccess) e = set_pair_attr<false, true>();
+  if (e == cudaSuccess) e = set_pair_attr<true, true>();
+  if (e == cudaSuccess) e = set_pair_attr<true, false>();
   if (e != cudaSuccess) { cudaGetLastError(); return DION_ERR_CUDA; }
   if (tracked) done_on[dev] = true;
   return DION_OK;
@@ -1098,8 +1248,11 @@ inline int umma_configure() {
 // `variant` (test hook, 0 in the product): UMMA_VARIANT_* bits.
 enum : int {
   UMMA_VARIANT_REGISTER_LOADS = 1,   // operands through registers instead of TMA
-  UMMA_VARIANT_WITHHOLD = 2          // with register loads: withhold one producer arrival, 1 ms wait budget
+  UMMA_VARIANT_WITHHOLD = 2,         // with register loads: withhold one producer arrival, 1 ms wait budget
+  UMMA_VARIANT_NO_PAIRS = 4          // single-CTA tiles where the product would take CTA pairs
 };
+constexpr i64 PAIR_MIN_ROWS = 512;   // smallest output height given to CTA pairs
+constexpr i64 PAIR_MIN_TRI = 2048;   // smallest lower-triangular output given to CTA pairs
 inline int umma_try_launch(const GemmArgs& g_in, int precision, int sm_count, float* part, i64 part_floats,
                            int* status, cudaStream_t st, int variant = 0) {
   using namespace umma;
@@ -1133,7 +1286,12 @@ inline int umma_try_launch(const GemmArgs& g_in, int precision, int sm_count, fl
   // lower-triangular output: 128 x 256 tiles (more flops per operand byte; the tiles on the diagonal
   // compute up to 128 columns too many) once the matrix has enough tile rows for that to pay
   const bool tri_wide = g.tri == TRI_LOWER && g.epi == EPI_STORE && g.N >= TRI_WIDE_MIN;
-  const int BN = ((g.tri == TRI_LOWER && !tri_wide) || g.N < 256) ? 128 : 256;
+  // CTA pairs (cta_group::2, 256 x 256 tiles): the fp32 (3xTF32) products that the TMA variant with the
+  // coalesced epilogue takes, once the output is tall enough to give every pair work
+  const int nclusters = pair_clusters(sm_count);
+  bool cg2 = !bf16 && !g.tf32x1 && !(variant & (UMMA_VARIANT_REGISTER_LOADS | UMMA_VARIANT_NO_PAIRS)) && nclusters > 0 &&
+             g.a2_mode != ADD_BF16 && g.N >= 256 && g.M >= PAIR_MIN_ROWS && (g.tri != TRI_LOWER || g.N >= PAIR_MIN_TRI);
+  const int BN = ((g.tri == TRI_LOWER && !tri_wide && !cg2) || g.N < 256) ? 128 : 256;
   Params p;
   p.g = g;
   // TMA variant: fp32 operands in memory (both precision modes), dimensions the tensor maps can describe
@@ -1151,20 +1309,27 @@ inline int umma_try_launch(const GemmArgs& g_in, int precision, int sm_count, fl
   }
   if (tma && !d16) {
     const i64 lda = a_mn ? g.a_sk : g.a_si, ldb = b_mn ? g.b_sk : g.b_sn;
-    tma = make_operand_map(&p.tmA, g.A, g.M, g.K, lda, a_mn, BM) && make_operand_map(&p.tmB, g.B, g.N, g.K, ldb, b_mn, BN);
+    tma = make_operand_map(&p.tmA, g.A, g.M, g.K, lda, a_mn, BM) &&
+          make_operand_map(&p.tmB, g.B, g.N, g.K, ldb, b_mn, cg2 ? BN / 2 : BN);
     if (tma && g.a2_mode == ADD_F32)
       tma = make_operand_map(&p.tmA2, g.A2, g.M, g.K, a_mn ? g.a2_sk : g.a2_si, a_mn, BM);
   }
   const int bke = (bf16 && (!tma || d16)) ? 64 : 32;
-  p.nM = (int)((g.M + BM - 1) / BM);
+  if (cg2 && !tma) {   // no tensor maps: the register path knows no pairs; redo the tile choice without them
+    GemmArgs g2 = g_in;
+    return umma_try_launch(g2, precision, sm_count, part, part_floats, status, st, variant | UMMA_VARIANT_NO_PAIRS);
+  }
+  const int tile_m = cg2 ? 2 * BM : BM;
+  p.nM = (int)((g.M + tile_m - 1) / tile_m);
   p.nN = (int)((g.N + BN - 1) / BN);
   p.nkb = (int)((g.K + bke - 1) / bke);
   const i64 tiles = (g.tri != TRI_LOWER) ? (i64)p.nM * p.nN
-                    : (BN == 256)          ? ((i64)p.nM + 1) * (p.nM + 1) / 4
+                    : (BN == 256 && !cg2)  ? ((i64)p.nM + 1) * (p.nM + 1) / 4
                                            : (i64)p.nM * (p.nM + 1) / 2;
+  const int workers_max = cg2 ? nclusters : sm_count;   // CTAs, or CTA pairs, that can run at once
   int splits = 1;
-  if (g.epi == EPI_STORE && !g.klimit && part != nullptr && tiles < sm_count) {
-    i64 want = sm_count / tiles;
+  if (g.epi == EPI_STORE && !g.klimit && part != nullptr && tiles < workers_max) {
+    i64 want = workers_max / tiles;
     const i64 kmax = p.nkb / 4;                       // at least four K blocks per split
     if (want > kmax) want = kmax;
     if (want > 32) want = 32;
@@ -1184,9 +1349,13 @@ inline int umma_try_launch(const GemmArgs& g_in, int precision, int sm_count, fl
   // 32 K blocks per accumulation chain: 1024 k (8e-6 relative error in fp32 mode, 1.4e-6 with
   // split accumulators); 2048 k for bf16 operands loaded through registers
   p.kc = 32;
-  const int grid = p.num_items < sm_count ? p.num_items : sm_count;
+  const int grid = cg2 ? 2 * (p.num_items < nclusters ? p.num_items : nclusters)
+                       : (p.num_items < sm_count ? p.num_items : sm_count);
   const bool one = g.tf32x1 && !bf16 && tma && !a_mn && !b_mn && g.a2_mode == ADD_NONE && !g.precise && splits == 1;
-  if (one) {
+  if (cg2) {
+    const cudaError_t e = g.precise ? launch_pair<true>(p, a_mn, b_mn, grid, st) : launch_pair<false>(p, a_mn, b_mn, grid, st);
+    if (e != cudaSuccess) { cudaGetLastError(); return DION_ERR_CUDA; }
+  } else if (one) {
     if (BN == 256) launch_one<256>(p, grid, st);
     else launch_one<128>(p, grid, st);
   } else if (d16) {   // bf16 arrays: always with the coalesced epilogue

@@ -236,3 +236,29 @@ def test_a_wait_that_runs_out_reports_timeout_and_the_next_product_is_correct(li
     assert run(lib, 2, 0, 256, 384, 128, False, False, variant=3, expect_status=4) is None      # several CTAs
     assert run(lib, 2, 0, 128, 128, 64, False, False, variant=1) < TOL[2]
     assert run(lib, 2, 0, 512, 512, 1024, False, True) < TOL[2]
+
+
+# ---------------------------------------------------------------------------
+# CTA pairs (cta_group::2): fp32-mode products with at least 512 rows and 256 columns run on clusters of two
+# CTAs that share a 256 x 256 tile; bit 2 of the variant word keeps such a product on single-CTA tiles.
+# ---------------------------------------------------------------------------
+
+@pytest.mark.parametrize("a_mn,b_mn", LAYOUTS)
+@pytest.mark.parametrize("precise", [0, 1])
+def test_cta_pairs_all_layouts(lib, a_mn, b_mn, precise):
+    tol = 3e-6 if precise else TOL[2]          # the error grows with the number of 1024-k accumulation chunks
+    for (M, N, K) in [(1024, 512, 512), (2048, 768, 2080), (648, 392, 328), (1280, 256, 96)]:
+        err = run(lib, 2, 0, M, N, K, a_mn, b_mn, precise=precise, seed=M + K)
+        assert err < tol, (M, N, K, err)
+        ref = run(lib, 2, 0, M, N, K, a_mn, b_mn, precise=precise, seed=M + K, variant=4)
+        assert ref < tol, ("single-CTA tiles", M, N, K, ref)
+
+
+def test_cta_pairs_epilogues_triangle_and_k_limit(lib):
+    assert run(lib, 2, 0, 2048, 1536, 256, False, False, add=torch.float32, epi=2, alpha=0.05) < TOL[2]
+    assert run(lib, 2, 0, 2048, 1536, 256, False, False, epi=1, alpha=0.01) < TOL[2]
+    assert run(lib, 2, 0, 1100, 520, 300, False, True, add=torch.float32) < TOL[2]       # fused fp32 addend, ragged
+    assert run(lib, 2, 0, 2304, 2304, 512, True, True, tri=1, precise=1) < 2e-6           # lower 256 x 256 tiles
+    assert run(lib, 2, 0, 4360, 4360, 264, True, True, tri=1) < TOL[2]
+    assert run(lib, 2, 0, 2048, 512, 512, False, False, klimit=1) < TOL[2]
+    assert run(lib, 2, 0, 512, 512, 8192, True, True) < TOL[2]                             # few tiles: split-K over pairs

@@ -415,6 +415,22 @@ def test_step_given_panel_is_the_step_when_the_panel_is_exact():
     assert rel(alt2.X, res.X) < 1e-12 and rel(alt2.Q, res.Q) < 1e-12
 
 
+@pytest.mark.parametrize("ranks,m,n,r", [(2, 20, 30, 6), (3, 17, 31, 5), (4, 12, 16, 8), (1, 9, 7, 3)])
+def test_sharded_step_equals_the_centralised_step_layer_by_layer(ranks, m, n, r):
+    # Algorithm 3 is built to preserve the mathematics of Algorithm 2: whatever the number of column shards
+    # (ragged ones and shards narrower than r included), every layer must come out as the unsharded step
+    rng = np.random.default_rng(30 + ranks)
+    layers = [draw(rng, m, n, r) for _ in range(ranks)]
+    Xs, Ms, Gs, Qs = (list(t) for t in zip(*layers))
+    Xn, Mn, Vn, d = orc.sharded_step(Xs, Ms, Gs, Qs, MU, ETA, EPS)
+    for l in range(ranks):
+        res = orc.step(Xs[l], Ms[l], Gs[l], Qs[l], MU, ETA, EPS)
+        assert rel(Xn[l], res.X) < 1e-12 and rel(Mn[l], res.M) < 1e-12
+        assert rel(Vn[l], res.Q) < 1e-12 and rel(d[l], res.d) < 1e-12
+    bounds = orc.shard_bounds(n, ranks)
+    assert bounds[0][0] == 0 and bounds[-1][1] == n and all(a[1] == b[0] for a, b in zip(bounds, bounds[1:]))
+
+
 # -- generated benchmark inputs are in contract ---------------------------------
 
 def test_config1_ten_steps_stay_in_contract():
