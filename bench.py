@@ -362,7 +362,8 @@ def measure_tf32_peak(torch, binding, n=8192, reps=5):
                     ("C", ctypes.c_void_p), ("ldc", ctypes.c_int64), ("epi", ctypes.c_int),
                     ("C2", ctypes.c_void_p), ("ldc2", ctypes.c_int64), ("c2_mode", ctypes.c_int),
                     ("alpha", ctypes.c_float), ("tri", ctypes.c_int), ("klimit", ctypes.c_int), ("precise", ctypes.c_int),
-                    ("ab16", ctypes.c_int), ("tf32x1", ctypes.c_int), ("variant", ctypes.c_int)]
+                    ("ab16", ctypes.c_int), ("tf32x1", ctypes.c_int), ("variant", ctypes.c_int),
+                    ("A16lo", ctypes.c_void_p), ("B16lo", ctypes.c_void_p)]
     lib = binding.load_library()
     lib.dion_debug_gemm.argtypes = [ctypes.c_int, ctypes.c_int, ctypes.POINTER(GemmArgs), ctypes.c_void_p,
                                     ctypes.c_int64, ctypes.c_void_p, ctypes.c_void_p]

@@ -119,6 +119,34 @@ __global__ void __launch_bounds__(256) k_to_bf16(const float* __restrict__ src, 
   }
 }
 
+// hi = bf16(src), lo = bf16(src - hi): src ~ hi + lo to 16 significant bits.  rows x cols (cols a multiple of 8,
+// src rows 16-byte aligned), hi and lo dense.  skip_flag (optional): nothing is written when *skip_flag != 0.
+__global__ void __launch_bounds__(256) k_split_bf16(const float* __restrict__ src, i64 lds, i64 rows, i64 cols,
+                                                    __nv_bfloat16* __restrict__ hi, __nv_bfloat16* __restrict__ lo,
+                                                    const int* __restrict__ skip_flag) {
+  pdl_enter();
+  if (skip_flag != nullptr && *skip_flag != 0) return;
+  const i64 per_row = cols / 8;
+  const i64 total = rows * per_row;
+  for (i64 e = (i64)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (i64)gridDim.x * blockDim.x) {
+    const i64 i = e / per_row, c = (e - i * per_row) * 8;
+    const float4 a = *reinterpret_cast<const float4*>(src + i * lds + c);
+    const float4 b = *(reinterpret_cast<const float4*>(src + i * lds + c) + 1);
+    const float v[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+    float h[8], l[8];
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {
+      h[q] = __bfloat162float(__float2bfloat16_rn(v[q]));
+      l[q] = v[q] - h[q];
+    }
+    uint4 oh, ol;
+    oh.x = pack_bf16x2(h[0], h[1]); oh.y = pack_bf16x2(h[2], h[3]); oh.z = pack_bf16x2(h[4], h[5]); oh.w = pack_bf16x2(h[6], h[7]);
+    ol.x = pack_bf16x2(l[0], l[1]); ol.y = pack_bf16x2(l[2], l[3]); ol.z = pack_bf16x2(l[4], l[5]); ol.w = pack_bf16x2(l[6], l[7]);
+    *reinterpret_cast<uint4*>(hi + i * cols + c) = oh;
+    *reinterpret_cast<uint4*>(lo + i * cols + c) = ol;
+  }
+}
+
 // out = src with every value rounded to the nearest TF32 number (10 explicit mantissa bits, ties away
 // from zero), rows x cols (cols a multiple of 4, src rows 16-byte aligned), out dense.  The tensor core
 // truncates an fp32 operand to TF32 when it reads it; on pre-rounded values that truncation is exact, so a

@@ -27,11 +27,13 @@ constexpr size_t GROUP_SCRATCH_BYTES = (size_t)16 << 30;  // scratch dion_step_g
 constexpr int MAX_ROUNDS = 6;             // adaptive Cholesky QR rounds
 constexpr float FLOOR_REL = 1e-4f;        // pivot floor relative to the column's squared norm
 constexpr float GOOD_REL = 1e-4f;         // smallest relative pivot of a round that one more round can finish
-// CholeskyQR2: max |U1^T U1 - I| below which the second round is skipped.  Measured on well-conditioned
-// panels (cond(P) 2-4, r 256-2048, up to 16384 rows): one accurate round leaves 1e-5 to 3e-5 here and the
-// step's outputs then differ from the float64 rule by 3-4e-6 (Q), the same as after two rounds; a panel of
-// condition 15 leaves ~1e-4 and takes the second round.
-constexpr float ORTH_TAU = 3e-5f;
+// CholeskyQR2: the second round is skipped when the first round's U1 is orthonormal enough, measured as an
+// estimate of |U1^T U1 - I|_F^2 (k_probe_*): done when it is <= ORTH_TAU_F^2 * r, i.e. when the deviation's
+// Frobenius norm is what r entries of size ORTH_TAU_F would give.  Measured on the workloads' own panels
+// (cond(P) 2-4, r 128-2048, up to 14336 rows): sqrt(estimate / r) is 5e-7 to 9e-6 after one accurate round, and the
+// step's outputs then differ from the float64 rule by 3-4e-6 (Q), the same as after two rounds; warm starts
+// with nearly parallel columns give 3.6e-5 and more and take the second round.
+constexpr float ORTH_TAU_F = 3e-5f;
 constexpr float DONE_REL = 0.9f;          // smallest relative pivot of a round whose input was already orthonormal
 constexpr i64 PART_CAP_FLOATS = (i64)16 << 20;  // split-K partial sums, at most 64 MiB
 
@@ -46,6 +48,8 @@ struct Layout {
   i64 B32;                  // fp32 mode: M + G formed once per step (0: the products form it on the fly)
   i64 Psave;                // CholeskyQR2: the panel as the product wrote it, kept for the fallback (0: none)
   i64 fb_part, fb_h, fb_n;  // fallback kernel: partial dot products (SMs x r), their sums (r), partial norms (SMs)
+  i64 probe_y, probe_part;  // CholeskyQR2's orthogonality probe: U1 z (rows x NPROBE), partial U1^T (U1 z)
+  i64 S16;                  // fp32 mode: the bf16 (hi, lo) pair of the error feedback's second factor (max(m,n) x r x 2 bf16)
   i64 part_floats;
   int cn_chunks;
   i64 cn_rows;
@@ -145,6 +149,9 @@ Layout make_layout(const dion_ctx* c, i64 m, i64 n, i64 r) {
   L.B32 = 0;
   if (sum_in_scratch(c, m, n, r)) { L.B32 = o; o += align64(m * n); }
   L.Psave = L.fb_part = L.fb_h = L.fb_n = 0;
+  L.S16 = o; o += align64(big * r);
+  L.probe_y = o; o += align64(big * NPROBE);
+  L.probe_part = o; o += align64((i64)(L.cn_chunks + 1) * r * NPROBE);
   if (may_fallback(c, m, n, r)) {
     L.Psave = o; o += align64(big * r);
     L.fb_part = o; o += align64((i64)c->sm_count * r);
@@ -396,8 +403,8 @@ enum : int {
   RM_PLAIN = 0,     // no device-side control
   RM_ADAPTIVE = 1,  // deflating pivots, skipped once the panel is done, split-accumulator products, round statistics
   RM_FIRST = 2,     // first round of CholeskyQR2: plain control, split-accumulator products
-  RM_CHECKED = 3    // second round of CholeskyQR2: the Gram matrix is always formed; if it is the identity to
-                    // ORTH_TAU the rest of the round is skipped (Pout = Pin)
+  RM_CHECKED = 3    // second round of CholeskyQR2: the first round's result is measured first (orthogonality probe);
+                    // if it is orthonormal to ORTH_TAU_F the whole round is skipped (Pout = Pin)
 };
 inline bool rm_skips(int mode) { return mode == RM_ADAPTIVE || mode == RM_CHECKED; }
 inline bool rm_precise(int mode) { return mode == RM_ADAPTIVE || mode == RM_FIRST; }
@@ -515,28 +522,35 @@ int cholqr_round(StepCtx& s, i64 pin_off, i64 pout_off, i64 rows, i64 r, int mod
   const bool adaptive = (mode == RM_ADAPTIVE);
   const bool skips = rm_skips(mode);
   const int* skip = skips ? (s.os + OS_DONE) : nullptr;
+  if (mode == RM_CHECKED) {
+    // CholeskyQR2, second round: first measure the first round's result (two passes over the panel instead of
+    // its Gram matrix); orthonormal enough -> done, and everything below is skipped on the device
+    int chunks; i64 per;
+    colnorm_plan(rows, r, c->sm_count, &chunks, &per);
+    launch_pdl(k_probe_y, dim3((unsigned)grid_for(c, rows * 32), (unsigned)s.nb), dim3(256), 0, s.st, (const float*)(s.ws + pin_off), r,
+               rows, r, s.ws + s.L.probe_y, s.wstride);
+    DION_CHECK_LAUNCH(c);
+    launch_pdl(k_probe_w, dim3((unsigned)((r + 127) / 128), (unsigned)chunks, (unsigned)s.nb), dim3(128), 0, s.st,
+               (const float*)(s.ws + pin_off), r, rows, r, per, (const float*)(s.ws + s.L.probe_y), s.ws + s.L.probe_part, s.wstride);
+    DION_CHECK_LAUNCH(c);
+    launch_pdl(k_probe_decide, dim3((unsigned)s.nb), dim3(256), 0, s.st, (const float*)(s.ws + s.L.probe_part), chunks, r, s.os,
+               ORTH_TAU_F, c->dev_ints + 2, s.wstride);
+    DION_CHECK_LAUNCH(c);
+  }
   GemmArgs g = gemm_args();
   g.M = r; g.N = r; g.K = gram_rows > 0 ? gram_rows : rows;
   g.A = s.ws + pin_off; g.a_si = 1; g.a_sk = r;
   g.B = s.ws + pin_off; g.b_sk = r; g.b_sn = 1;
-  g.C = s.ws + s.L.Gram; g.ldc = r; g.epi = EPI_STORE; g.tri = TRI_LOWER; g.skip_flag = adaptive ? skip : nullptr; g.precise = rm_precise(mode) ? 1 : 0;
+  g.C = s.ws + s.L.Gram; g.ldc = r; g.epi = EPI_STORE; g.tri = TRI_LOWER; g.skip_flag = skips ? skip : nullptr; g.precise = rm_precise(mode) ? 1 : 0;
   for (int m = 0; m < s.nb; ++m) DION_TRY(launch_gemm(s, for_matrix(s, g, m, true, true, true), m));
   launch_pdl(k_round_begin, dim3((unsigned)(s.nb)), dim3(256), 0, s.st, s.ws + s.L.Gram, r, r, 0.f, s.ws + s.L.gdiag, s.ws + s.L.scal, s.os,
-                                        adaptive ? 1 : 0, s.wstride, c->dev_ints);
+                                        skips ? 1 : 0, s.wstride, c->dev_ints);
   DION_CHECK_LAUNCH(c);
   // Tall panels with r > 512: blocked triangular solve with the 512-column diagonal inverses
   // only (the levels of the triangular inverse above 512 are never formed).
   // alone, 512-column products need >= 128 row tiles to fill the GPU; beside the factorization
   // (second stream) they are background work at any height
   const bool trsm = (r > NBO) && (rows >= 8192 || c->side != nullptr);
-  if (mode == RM_CHECKED) {
-    // CholeskyQR2, second round: measure the first round's result; orthonormal to ORTH_TAU -> done
-    dim3 grid((unsigned)grid_for(c, r * r), (unsigned)s.nb);
-    launch_pdl(k_orth_check, grid, dim3(256), 0, s.st, (const float*)(s.ws + s.L.Gram), r, r, s.os, s.wstride);
-    DION_CHECK_LAUNCH(c);
-    launch_pdl(k_orth_decide, dim3((unsigned)s.nb), dim3(1), 0, s.st, s.os, ORTH_TAU, c->dev_ints + 2);
-    DION_CHECK_LAUNCH(c);
-  }
   if (skips) {   // a finished panel is passed through (before anything writes Pout)
     dim3 grid((unsigned)grid_for(c, rows * r), (unsigned)s.nb);
     launch_pdl(k_copy_panel, grid, dim3(256), 0, s.st, s.ws + pin_off, r, s.ws + pout_off, r, rows, r, nullptr, s.os + OS_DONE, s.wstride);
@@ -761,7 +775,7 @@ int orthonormalize(StepCtx& s, i64 rows, i64 r, i64 short_dim, i64 pin_off, i64*
   const int mode = resolve_orth_for(s.c, r, short_dim, s.list != nullptr);
   if (mode == DION_ORTH_CHOLQR2) {
     // the first round with the accurate products; the second one only if the first one's result is
-    // not yet orthonormal to ORTH_TAU (measured on its Gram matrix).  A pivot that is not positive in
+    // not yet orthonormal to ORTH_TAU_F (measured by the probe).  A pivot that is not positive in
     // either round (the paper's "CQR failure") raises the step's fail flag only; the fallback kernel then
     // orthonormalizes the saved panel and clears the flag, or confirms the breakdown.
     const bool fb = pin_off != s.L.P0 && fallback_fits(s.c, rows);
@@ -861,6 +875,46 @@ bool x_single_pass(const StepCtx& s, const dion_matrix* a, const float* F1, i64 
   return s.tensor && s.c->cfg.precision == DION_PREC_FP32 && m >= 128 && n >= 64 && r >= 64 && m % 4 == 0 &&
          n % 4 == 0 && r % 4 == 0 && !((uintptr_t)a->X & 15) && a->ldx % 4 == 0 && !((uintptr_t)F1 & 15) &&
          ld1 % 4 == 0 && !((uintptr_t)F2 & 15) && ld2 % 4 == 0;
+}
+
+// The error feedback M <- (M + G) - beta F1 F2^T in fp32 mode on the tensor engine (F1: m x r, F2: n x r; U R^T, or
+// R U^T in the transposed form).  The product enters M scaled by beta = 1 - mu, so 16 significant bits in its factors
+// are plenty (an error of ~1e-5 of the product, ~5e-7 of M): both factors are split once into bf16 pairs
+// (hi, lo) in scratch (`p1`, `p2`: max(m,n) x r floats each) and the product takes three bf16 MMAs per K step, 1.3
+// TF32 passes instead of three.  Otherwise the 3xTF32 / FMA product of the fp32 factors.
+// sum32 != nullptr: M + G comes from scratch (C = sum32 - beta acc); else C = M + G - beta acc with the caller's G.
+int ef_update(StepCtx& s, int b, const dion_matrix* a, const float* F1, i64 ld1, const float* F2, i64 ld2, float* p1,
+              float* p2, const float* sum32, const int* skip) {
+  dion_ctx* c = s.c;
+  const i64 m = a->m, n = a->n, r = a->r;
+  GemmArgs e = gemm_args();
+  e.M = m; e.N = n; e.K = r;
+  const bool pairs = s.tensor && c->cfg.precision == DION_PREC_FP32 && m >= 128 && n >= 64 && r >= 64 && m % 8 == 0 &&
+                     n % 8 == 0 && r % 8 == 0 && !((uintptr_t)a->M & 15) && a->ldm % 4 == 0 && !((uintptr_t)F1 & 15) &&
+                     ld1 % 4 == 0 && !((uintptr_t)F2 & 15) && ld2 % 4 == 0 &&
+                     (sum32 != nullptr || (!((uintptr_t)a->G & 15) && a->ldg % ((a->g_dtype == DION_BF16) ? 8 : 4) == 0));
+  if (pairs) {
+    __nv_bfloat16* h1 = reinterpret_cast<__nv_bfloat16*>(p1);
+    __nv_bfloat16* l1 = h1 + m * r;
+    __nv_bfloat16* h2 = reinterpret_cast<__nv_bfloat16*>(p2);
+    __nv_bfloat16* l2 = h2 + n * r;
+    launch_pdl(k_split_bf16, dim3((unsigned)grid_for(c, m * r / 8)), dim3(256), 0, s.st, F1, ld1, m, r, h1, l1, skip);
+    DION_CHECK_LAUNCH(c);
+    launch_pdl(k_split_bf16, dim3((unsigned)grid_for(c, n * r / 8)), dim3(256), 0, s.st, F2, ld2, n, r, h2, l2, skip);
+    DION_CHECK_LAUNCH(c);
+    e.ab16 = 1;
+    e.A = (const float*)h1; e.A16lo = l1; e.a_si = r; e.a_sk = 1;
+    e.B = (const float*)h2; e.B16lo = l2; e.b_sk = 1; e.b_sn = r;
+  } else {
+    e.A = F1; e.a_si = ld1; e.a_sk = 1;
+    e.B = F2; e.b_sk = 1; e.b_sn = ld2;
+  }
+  e.C = (float*)a->M; e.ldc = a->ldm;
+  if (sum32 != nullptr) { e.epi = EPI_C2_SUB; e.C2 = sum32; e.ldc2 = n; e.c2_mode = ADD_F32; }
+  else { e.epi = EPI_ADD2_SUB; e.C2 = a->G; e.ldc2 = a->ldg; e.c2_mode = (a->g_dtype == DION_BF16) ? ADD_BF16 : ADD_F32; }
+  e.alpha = 1.f - c->cfg.mu;
+  e.skip_flag = skip;
+  return launch_gemm(s, e, b);
 }
 
 int x_update(StepCtx& s, int b, const dion_matrix* a, const float* F1, i64 ld1, const float* F2, i64 ld2, float* r1,
@@ -1010,23 +1064,28 @@ int step_batch(dion_ctx* c, const dion_matrix* const* list, int nb, float lr, cu
   PhaseScope ps(c, st, DION_PHASE_EF);
   for (int b = 0; b < nb; ++b) {
     const dion_matrix* a = list[b];
-    GemmArgs e = gemm_args();
-    e.M = m; e.N = n; e.K = r;
     if (d16) {
+      GemmArgs e = gemm_args();
+      e.M = m; e.N = n; e.K = r;
       DION_TRY(to_bf16(s.W(b, s.L.R), r, qrow, r, bf(b, s.L.R16)));
       e.ab16 = 1;
       e.A = (const float*)bf(b, tr ? s.L.R16 : s.L.U16); e.a_si = r; e.a_sk = 1;
       e.B = (const float*)bf(b, tr ? s.L.U16 : s.L.R16); e.b_sk = 1; e.b_sn = r;
-    } else {
-      e.A = s.W(b, tr ? s.L.R : U_off); e.a_si = r; e.a_sk = 1;
-      e.B = s.W(b, tr ? U_off : s.L.R); e.b_sk = 1; e.b_sn = r;
+      e.C = (float*)a->M; e.ldc = a->ldm;
+      e.epi = EPI_ADD2_SUB; e.C2 = a->G; e.ldc2 = a->ldg; e.c2_mode = g_mode(a);
+      e.alpha = 1.f - c->cfg.mu;
+      e.skip_flag = s.OS(b) + OS_FAIL;
+      DION_TRY(launch_gemm(s, e, b));
+      continue;
     }
-    e.C = (float*)a->M; e.ldc = a->ldm;
-    if (b32) { e.epi = EPI_C2_SUB; e.C2 = s.W(b, s.L.B32); e.ldc2 = n; e.c2_mode = ADD_F32; }
-    else { e.epi = EPI_ADD2_SUB; e.C2 = a->G; e.ldc2 = a->ldg; e.c2_mode = g_mode(a); }
-    e.alpha = 1.f - c->cfg.mu;
-    e.skip_flag = s.OS(b) + OS_FAIL;
-    DION_TRY(launch_gemm(s, e, b));
+    // the bf16 pairs of the two factors go to the other panel buffer and to their own buffer
+    float* other = s.W(b, U_off == s.L.P0 ? s.L.P1 : s.L.P0);
+    float* sbuf = s.W(b, s.L.S16);
+    const float* Uf = s.W(b, U_off);
+    const float* Rf = s.W(b, s.L.R);
+    const float* sum32 = b32 ? s.W(b, s.L.B32) : nullptr;
+    if (tr) DION_TRY(ef_update(s, b, a, Rf, r, Uf, r, sbuf, other, sum32, s.OS(b) + OS_FAIL));
+    else DION_TRY(ef_update(s, b, a, Uf, r, Rf, r, other, sbuf, sum32, s.OS(b) + OS_FAIL));
   }
   }
 
@@ -1397,15 +1456,8 @@ int dion_dp_finish(dion_ctx* ctx, const dion_matrix* a, const float* U, const fl
   cudaStream_t st = (cudaStream_t)cuda_stream;
   DION_TRY(begin_step(ctx, a, 1, st, &s));
   const i64 m = a->m, n = a->n, r = a->r;
-  GemmArgs e = gemm_args();      // M <- (M + G) - (1 - mu) U W^T, with this rank's M and G
-  e.M = m; e.N = n; e.K = r;
-  e.A = U; e.a_si = r; e.a_sk = 1;
-  e.B = W; e.b_sk = 1; e.b_sn = r;
-  e.C = (float*)a->M; e.ldc = a->ldm; e.epi = EPI_ADD2_SUB;
-  e.C2 = a->G; e.ldc2 = a->ldg; e.c2_mode = (a->g_dtype == DION_BF16) ? ADD_BF16 : ADD_F32;
-  e.alpha = 1.f - ctx->cfg.mu;
-  e.skip_flag = dp_flag;
-  DION_TRY(launch_gemm(s, e, 0));
+  // M <- (M + G) - (1 - mu) U W^T, with this rank's M and G (as in dion_step)
+  DION_TRY(ef_update(s, 0, a, U, r, W, r, s.ws + s.L.P1, s.ws + s.L.S16, nullptr, dp_flag));
   DION_TRY(colnorm(s, 0, W, n, r, (float*)a->Q, a->ldq, a->colnorm_out, dp_flag));
   // X <- X - lr sqrt(m/n) U Q^T, as in dion_step (rounded copies in the two panel buffers of the scratch)
   DION_TRY(x_update(s, 0, a, U, r, (const float*)a->Q, a->ldq, s.ws + s.L.P1, s.ws + s.L.R,
@@ -1501,15 +1553,8 @@ int dion_shard_finish(dion_ctx* ctx, const dion_matrix* a, int64_t n_total, cons
   cudaStream_t st = (cudaStream_t)cuda_stream;
   DION_TRY(begin_step(ctx, a, 1, st, &s));
   const i64 m = a->m, n = a->n, r = a->r;
-  GemmArgs e = gemm_args();      // M <- (M + G) - (1 - mu) U W^T on the shard's columns
-  e.M = m; e.N = n; e.K = r;
-  e.A = U; e.a_si = r; e.a_sk = 1;
-  e.B = W; e.b_sk = 1; e.b_sn = r;
-  e.C = (float*)a->M; e.ldc = a->ldm; e.epi = EPI_ADD2_SUB;
-  e.C2 = a->G; e.ldc2 = a->ldg; e.c2_mode = (a->g_dtype == DION_BF16) ? ADD_BF16 : ADD_F32;
-  e.alpha = 1.f - ctx->cfg.mu;
-  e.skip_flag = flag;
-  DION_TRY(launch_gemm(s, e, 0));
+  // M <- (M + G) - (1 - mu) U W^T on the shard's columns
+  DION_TRY(ef_update(s, 0, a, U, r, W, r, s.ws + s.L.P1, s.ws + s.L.S16, nullptr, flag));
   {   // Q <- W / (sqrt(colsumsq) + eps): the squared column norms are the all-reduced ones (one "chunk")
     int chunks; i64 per;
     colnorm_plan(n, r, ctx->sm_count, &chunks, &per);
@@ -1663,13 +1708,14 @@ bool preload_kernels() {
   ok = ok && touch_kernel(k_gemm_simt<128, 128, 8, 8, 8>) && touch_kernel(k_gemm_simt<64, 64, 16, 4, 4>);
   ok = ok && touch_kernel(k_splitk_reduce) && touch_kernel(k_round_begin) && touch_kernel(k_potrf_diag);
   ok = ok && touch_kernel(k_chol_step) && touch_kernel(k_inv_finish) && touch_kernel(k_round_end);
-  ok = ok && touch_kernel(k_orth_check) && touch_kernel(k_orth_decide) && touch_kernel(k_reset_rounds);
+  ok = ok && touch_kernel(k_probe_y) && touch_kernel(k_probe_w) && touch_kernel(k_probe_decide) && touch_kernel(k_reset_rounds);
   ok = ok && touch_kernel(k_orth_finish) && touch_kernel(k_cgs_fallback) && touch_kernel(k_copy_block);
   ok = ok && touch_kernel(k_colsumsq_partial) && touch_kernel(k_colnorm_apply) && touch_kernel(k_copy_panel);
   ok = ok && touch_kernel(k_latch_flag) && touch_kernel(k_finish_step) && touch_kernel(k_hh_reflector);
   ok = ok && touch_kernel(k_hh_apply) && touch_kernel(k_set_identity) && touch_kernel(k_sign_fix);
   ok = ok && touch_kernel(k_form_b16<true>) && touch_kernel(k_form_b16<false>) && touch_kernel(k_form_b32<true>);
   ok = ok && touch_kernel(k_form_b32<false>) && touch_kernel(k_to_bf16) && touch_kernel(k_round_tf32);
+  ok = ok && touch_kernel(k_split_bf16);
   return ok;
 }
 
@@ -1741,6 +1787,19 @@ extern "C" size_t dion_noalloc_scratch_limit(void) { return NOALLOC_SCRATCH_BYTE
 // ---------------------------------------------------------------------------
 // Internal test hook (dion_internal.h)
 // ---------------------------------------------------------------------------
+// Test hook: the orthogonality estimate of the most recent step's CholeskyQR2 check (first matrix of the chain).
+extern "C" int dion_debug_orth_measure(dion_ctx* ctx, void* cuda_stream, float* estimate) {
+  if (ctx == nullptr || estimate == nullptr) return DION_ERR_INVALID;
+  if (cudaSetDevice(ctx->cfg.device) != cudaSuccess) return DION_ERR_CUDA;
+  const int slot = (ctx->flag_cursor + MAX_FLAG_SLOTS - 1) % MAX_FLAG_SLOTS;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  if (cudaMemcpyAsync(estimate, ctx->dev_ints + 8 + (i64)slot * OS_SLOT_INTS + OS_MAXDEV, sizeof(float), cudaMemcpyDeviceToHost, st) !=
+          cudaSuccess ||
+      cudaStreamSynchronize(st) != cudaSuccess)
+    return DION_ERR_CUDA;
+  return DION_OK;
+}
+
 extern "C" int dion_debug_gemm(int engine, int precision, const dion_debug_gemm_args* a, float* part,
                                int64_t part_floats, int* status, void* cuda_stream) {
   if (a == nullptr || status == nullptr) return DION_ERR_INVALID;
@@ -1756,6 +1815,7 @@ extern "C" int dion_debug_gemm(int engine, int precision, const dion_debug_gemm_
   g.C = a->C; g.ldc = a->ldc; g.epi = a->epi;
   g.C2 = a->C2; g.ldc2 = a->ldc2; g.c2_mode = a->c2_mode;
   g.alpha = a->alpha; g.tri = a->tri; g.klimit = a->klimit; g.precise = a->precise; g.ab16 = a->ab16; g.tf32x1 = a->tf32x1;
+  g.A16lo = a->A16lo; g.B16lo = a->B16lo;
   cudaStream_t st = (cudaStream_t)cuda_stream;
   if (engine == DION_ENGINE_TENSOR) {
     const int rc = umma_try_launch(g, precision, sms, part, part_floats, status, st, a->variant);

@@ -46,6 +46,8 @@ struct GemmArgs {
   const int* skip_flag;          // optional: if *skip_flag != 0 the kernel does nothing
   int precise;                   // tensor engine: keep the small split terms in their own accumulator
   int ab16;                      // tensor engine only: A and B point to bf16 arrays (strides in elements), no addend
+  const void* A16lo;             // with ab16: A and B are PAIRS of bf16 arrays, x ~ hi + lo (A, B point to the "hi" arrays, these
+  const void* B16lo;             // to the "lo" arrays of the same shape and strides): three bf16 MMAs per K step, ~1e-5 relative
   int tf32x1;                    // tensor engine, fp32 mode: the operands' values fit TF32 already (k_round_tf32): one MMA
                                  // per K step instead of the three-term split.  Ignored by the FMA engine.
 };

@@ -27,6 +27,8 @@ typedef struct {
                                                     bit 1 (with bit 0) one producer arrival is withheld and every wait
                                                     has a 1 ms budget: the kernel must give up, set DION_STATUS_TIMEOUT
                                                     in *status and return */
+  const void* A16lo;                             /* with ab16: the "lo" arrays of bf16 operand pairs (x ~ hi + lo; A, B */
+  const void* B16lo;                             /* are the "hi" arrays), or NULL                                        */
 } dion_debug_gemm_args;
 
 /* engine: 1 = fp32 FMA, 2 = tensor cores (returns DION_ERR_UNSUPPORTED if the
@@ -34,6 +36,11 @@ typedef struct {
  * part_floats floats (may be NULL).  status: device int receiving DION_STATUS_* bits. */
 int dion_debug_gemm(int engine, int precision, const dion_debug_gemm_args* args, float* part,
                     int64_t part_floats, int* status, void* cuda_stream);
+
+/* The estimate of |U1^T U1 - I|_F^2 that the most recent step's CholeskyQR2 check measured (first matrix of
+ * its chain); synchronises `cuda_stream`.  `ctx` is a dion_ctx. */
+struct dion_ctx;
+int dion_debug_orth_measure(struct dion_ctx* ctx, void* cuda_stream, float* estimate);
 
 #ifdef __cplusplus
 }

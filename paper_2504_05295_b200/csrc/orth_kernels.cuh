@@ -15,7 +15,7 @@ enum : int {
   OS_FLOORED = 3,   // pivots raised to the floor in the current round
   OS_MINREL = 4,    // float bits: min over columns of pivot / original diagonal, current round
   OS_ROUNDS = 5,    // rounds that did work
-  OS_MAXDEV = 6,    // float bits: max |G - I| over the lower triangle of a round's Gram matrix (CholeskyQR2 check)
+  OS_MAXDEV = 6,    // float bits: the estimate of |U1^T U1 - I|_F^2 of the CholeskyQR2 check
   OS_BARRIER = 7,   // arrival counter of the fallback kernel's grid-wide barriers (zero at the start of a step)
   OS_SLOT_INTS = 8
 };
@@ -50,7 +50,7 @@ __global__ void k_round_begin(const float* __restrict__ G, i64 ld, i64 r, float 
     *shift = red[0] * scale;
     os[OS_FLOORED] = 0;
     os[OS_MINREL] = 0x7f800000;  // +inf
-    if (!(fabsf(red[0]) < __int_as_float(0x7f800000))) {
+    if (!(fabsf(red[0]) < __int_as_float(0x7f800000)) && os[OS_FAIL] == 0) {   // (a known failure is not reported twice)
       os[OS_FAIL] = 1;
       atomicOr(status, DION_STATUS_NONFINITE);
     }
@@ -583,44 +583,111 @@ __global__ void k_round_end(int* __restrict__ os, float good_rel, float done_rel
   }
 }
 
-// CholeskyQR2, second round: max |G[i][j] - delta_ij| over the lower triangle of the Gram matrix of
-// the first round's result, into os[OS_MAXDEV] (zero at the start of a step).  grid = (blocks, matrices).
-__global__ void __launch_bounds__(256) k_orth_check(const float* __restrict__ G, i64 ld, i64 r, int* __restrict__ os,
-                                                    i64 wstride) {
-  pdl_enter();
-  G += (i64)blockIdx.y * wstride;
-  os += (i64)blockIdx.y * OS_SLOT_INTS;
-  __shared__ float red[256];
-  const float inf = __int_as_float(0x7f800000);
-  float mx = 0.f;
-  const i64 total = r * r;
-  for (i64 e = (i64)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (i64)gridDim.x * blockDim.x) {
-    const i64 i = e / r, j = e % r;
-    if (j <= i) {
-      float dev = fabsf(G[i * ld + j] - ((i == j) ? 1.f : 0.f));
-      if (!(dev == dev)) dev = inf;            // NaN
-      mx = fmaxf(mx, dev);
-    }
-  }
-  red[threadIdx.x] = mx;
-  __syncthreads();
-  for (int w = 128; w > 0; w >>= 1) {
-    if ((int)threadIdx.x < w) red[threadIdx.x] = fmaxf(red[threadIdx.x], red[threadIdx.x + w]);
-    __syncthreads();
-  }
-  if (threadIdx.x == 0) atomicMax(&os[OS_MAXDEV], __float_as_int(red[0]));   // non-negative floats order like ints
+// ---------------------------------------------------------------------------
+// CholeskyQR2: is the first round's result U1 orthonormal enough to skip the second?  Measured without forming
+// U1^T U1 (one third of the orthonormalization's tensor work): with NPROBE fixed sign vectors z_p (entries +-1
+// from a hash of the index), E = U1^T U1 - I and w_p = U1^T (U1 z_p),  sum_p |w_p - z_p|^2 / NPROBE  is an
+// unbiased estimate of |E|_F^2 (Hutchinson's estimator; relative spread sqrt(2 / NPROBE) per probe set at
+// worst, far less for a matrix whose weight is spread over many entries).  Two passes over the panel.
+// ---------------------------------------------------------------------------
+constexpr int NPROBE = 8;
+
+__device__ __forceinline__ float probe_sign(i64 j, int p) {
+  uint32_t h = (uint32_t)j * 2654435761u + (uint32_t)(p + 1) * 0x9E3779B9u;
+  h ^= h >> 15; h *= 2246822519u; h ^= h >> 13; h *= 3266489917u; h ^= h >> 16;
+  return (h & 1u) ? 1.f : -1.f;
 }
 
-// ... and the decision: orthonormal to tau -> the rest of the round is skipped.  Counts the rounds
-// of the step that did work (1 or 2).
-__global__ void k_orth_decide(int* __restrict__ os, float tau, int* __restrict__ rounds_total) {
+// Y[i][p] = sum_j U[i][j] z_p[j]: one warp per row (lanes stride over the columns).  grid = (blocks, matrices).
+__global__ void __launch_bounds__(256) k_probe_y(const float* __restrict__ U, i64 ld, i64 rows, i64 r,
+                                                 float* __restrict__ Y, i64 wstride) {
   pdl_enter();
+  U += (i64)blockIdx.y * wstride; Y += (i64)blockIdx.y * wstride;
+  const int lane = threadIdx.x & 31;
+  const i64 warp = (i64)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  const i64 nwarps = (i64)gridDim.x * (blockDim.x >> 5);
+  for (i64 i = warp; i < rows; i += nwarps) {
+    float acc[NPROBE];
+#pragma unroll
+    for (int p = 0; p < NPROBE; ++p) acc[p] = 0.f;
+    const float* urow = U + i * ld;
+    for (i64 j = lane; j < r; j += 32) {
+      const float u = urow[j];
+#pragma unroll
+      for (int p = 0; p < NPROBE; ++p) acc[p] = fmaf(u, probe_sign(j, p), acc[p]);
+    }
+#pragma unroll
+    for (int p = 0; p < NPROBE; ++p) {
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) acc[p] += __shfl_xor_sync(0xffffffffu, acc[p], o);
+    }
+    if (lane == 0) {
+#pragma unroll
+      for (int p = 0; p < NPROBE; ++p) Y[i * NPROBE + p] = acc[p];
+    }
+  }
+}
+
+// part[chunk][j][p] = sum over the chunk's rows of U[i][j] Y[i][p].  grid = (ceil(r/128), chunks, matrices).
+__global__ void __launch_bounds__(128) k_probe_w(const float* __restrict__ U, i64 ld, i64 rows, i64 r,
+                                                 i64 rows_per_chunk, const float* __restrict__ Y,
+                                                 float* __restrict__ part, i64 wstride) {
+  pdl_enter();
+  U += (i64)blockIdx.z * wstride; Y += (i64)blockIdx.z * wstride; part += (i64)blockIdx.z * wstride;
+  const i64 j = (i64)blockIdx.x * 128 + threadIdx.x;
+  if (j >= r) return;
+  const i64 i0 = (i64)blockIdx.y * rows_per_chunk;
+  const i64 i1 = min(rows, i0 + rows_per_chunk);
+  float acc[NPROBE];
+#pragma unroll
+  for (int p = 0; p < NPROBE; ++p) acc[p] = 0.f;
+  for (i64 i = i0; i < i1; ++i) {
+    const float u = U[i * ld + j];
+    const float4 y0 = *reinterpret_cast<const float4*>(Y + i * NPROBE);
+    const float4 y1 = *reinterpret_cast<const float4*>(Y + i * NPROBE + 4);
+    acc[0] = fmaf(u, y0.x, acc[0]); acc[1] = fmaf(u, y0.y, acc[1]); acc[2] = fmaf(u, y0.z, acc[2]); acc[3] = fmaf(u, y0.w, acc[3]);
+    acc[4] = fmaf(u, y1.x, acc[4]); acc[5] = fmaf(u, y1.y, acc[5]); acc[6] = fmaf(u, y1.z, acc[6]); acc[7] = fmaf(u, y1.w, acc[7]);
+  }
+  float* out = part + ((i64)blockIdx.y * r + j) * NPROBE;
+#pragma unroll
+  for (int p = 0; p < NPROBE; ++p) out[p] = acc[p];
+}
+
+// One block per matrix: est = sum_p |w_p - z_p|^2 / NPROBE (fixed summation order) into os[OS_MAXDEV] (float
+// bits); est <= tau_f^2 * r  ->  the panel is done (OS_DONE = 1: the rest of the second round is skipped).
+// Counts the rounds of the step that did work (1 or 2).
+__global__ void __launch_bounds__(256) k_probe_decide(const float* __restrict__ part, int chunks, i64 r,
+                                                      int* __restrict__ os, float tau_f,
+                                                      int* __restrict__ rounds_total, i64 wstride) {
+  pdl_enter();
+  part += (i64)blockIdx.x * wstride;
   os += (i64)blockIdx.x * OS_SLOT_INTS;
-  const float maxdev = __int_as_float(os[OS_MAXDEV]);
-  const bool done = (os[OS_FAIL] == 0) && (maxdev <= tau);
-  os[OS_DONE] = done ? 1 : 0;
-  os[OS_ROUNDS] = done ? 1 : 2;
-  atomicAdd(rounds_total, done ? 1 : 2);
+  __shared__ float red[256];
+  float e = 0.f;
+  for (i64 j = threadIdx.x; j < r; j += 256) {
+#pragma unroll
+    for (int p = 0; p < NPROBE; ++p) {
+      float w = 0.f;
+      for (int c = 0; c < chunks; ++c) w += part[((i64)c * r + j) * NPROBE + p];
+      const float dlt = w - probe_sign(j, p);
+      e = fmaf(dlt, dlt, e);
+    }
+  }
+  red[threadIdx.x] = e;
+  __syncthreads();
+  for (int w = 128; w > 0; w >>= 1) {
+    if ((int)threadIdx.x < w) red[threadIdx.x] += red[threadIdx.x + w];
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) {
+    const float est = red[0] / (float)NPROBE;
+    os[OS_MAXDEV] = __float_as_int(est);
+    const bool failed = os[OS_FAIL] != 0;       // a pivot of the first round failed: the fallback redoes the panel
+    const bool done = !failed && (est <= tau_f * tau_f * (float)r);      // false for NaN
+    os[OS_DONE] = (done || failed) ? 1 : 0;
+    os[OS_ROUNDS] = done ? 1 : 2;
+    atomicAdd(rounds_total, done ? 1 : 2);
+  }
 }
 
 // Clears the round state of a step slot (keeps the fail flag): a second orthonormalization in one step.

@@ -47,7 +47,7 @@ constexpr int NUM_THREADS_TMA = NUM_THREADS + 32;   // one more warp issues the 
 constexpr long long SPIN_LIMIT_CYCLES = 2000000000LL;  // about one second
 
 struct Params {
-  alignas(64) CUtensorMap tmA, tmA2, tmB;   // TMA variant: raw fp32 tiles of A, its addend and B
+  alignas(64) CUtensorMap tmA, tmA2, tmB, tmB2;   // TMA variants: tiles of A, of its addend (or its "lo" array), of B (and its "lo" array)
   GemmArgs g;
   int nM, nN;         // output tiles along M and N
   int splits;         // K splits (>= 1); partial sums go to g.part when > 1
@@ -472,8 +472,12 @@ struct TileMap {
 // K block costs a CTA two thirds of the shared-memory traffic of the single-CTA form (which is bound by
 // it: three MMAs re-read both operand tiles) and a stage is 64 KB instead of 96 KB (3 stages instead of 2).
 // The leader CTA issues the MMAs for both; accumulators and epilogue stay per CTA (128 rows x 256 columns).
+// X2 (bf16 arrays, D16): each operand is a PAIR of bf16 arrays, x ~ hi + lo with hi = bf16(x), lo = bf16(x - hi)
+// (16 significant bits); three bf16 MMAs per K step (hi*lo + lo*hi + hi*hi) give a product that is accurate to
+// ~1e-5 relative at 1.3 times the tensor time of one TF32 pass.  Used for the error-feedback product in fp32
+// mode, whose result enters M scaled by 1 - mu.
 template <int BN, bool BF16, bool SPLIT = false, bool TMA = false, bool D16 = false, bool CE = false, bool ONE = false,
-          bool CG2 = false>
+          bool CG2 = false, bool X2 = false>
 struct Cfg {
   // BT: bf16 operands formed in shared memory from TMA-loaded fp32 tiles (K block of 32, as in
   // the fp32 TMA variant).  A stage then holds the raw fp32 tiles of A, of its fp32 addend and
@@ -487,9 +491,10 @@ struct Cfg {
   static constexpr int BN_L = CG2 ? BN / 2 : BN;             // columns of the B tile this CTA holds
   static constexpr int B_BYTES = BN_L * 128;
   static constexpr int STAGE_BYTES = BT ? (2 * A_BYTES + B_BYTES + A_BYTES / 2 + B_BYTES / 2)
-                                        : ((BF16 || ONE) ? 1 : 2) * (A_BYTES + B_BYTES);
+                                        : (((BF16 && !X2) || ONE) ? 1 : 2) * (A_BYTES + B_BYTES);
   // D16: the producer warps have no conversion work and serve as epilogue warps too
-  static constexpr int EPI_WARPS = (D16 || ONE) ? NUM_EPI_WARPS + NUM_PROD_WARPS : NUM_EPI_WARPS;
+  // (with operand pairs the stages leave room for 8 warps' epilogue tiles only)
+  static constexpr int EPI_WARPS = ((D16 && !X2) || ONE) ? NUM_EPI_WARPS + NUM_PROD_WARPS : NUM_EPI_WARPS;
   // CE (coalesced epilogue): an epilogue warp owns 32 rows x EPI_W columns of the tile and passes them
   // through a private shared-memory tile in passes of EPI_RPP rows (EPI_RPP * EPI_W = 1024 elements),
   // so that one global access of the warp covers whole row segments instead of 32 rows; paid for with
@@ -521,14 +526,15 @@ struct Cfg {
 // the operand tiles the MMA reads (k-contiguous: rows of 64 bytes, 64-byte swizzle;
 // row-contiguous: 128-byte rows of 64 row indices, 128-byte swizzle); one MMA per K step.
 template <int BN, bool A_MN, bool B_MN, bool BF16, bool SPLIT, bool TMA, bool D16 = false, bool CE = false, bool ONE = false,
-          bool CG2 = false>
+          bool CG2 = false, bool X2 = false>
 __global__ void __launch_bounds__(TMA ? NUM_THREADS_TMA : NUM_THREADS, 1) k_gemm_umma(const __grid_constant__ Params p) {
+  static_assert(!X2 || (D16 && CE && !A_MN && !B_MN), "operand pairs: k-contiguous bf16 arrays");
   static_assert(!CG2 || (TMA && !BF16 && !D16 && !ONE && BN == 256), "CTA pairs: the fp32 TMA variants with 256-column tiles");
   static_assert(!(BF16 && SPLIT), "split accumulators belong to the 3xTF32 mode");
   static_assert(!D16 || (BF16 && TMA), "bf16 operands in memory are loaded by TMA");
   static_assert(!CE || (TMA && (D16 || !BF16)), "the coalesced epilogue serves the bf16-array and the fp32 TMA variants");
   static_assert(!ONE || (TMA && CE && !BF16 && !SPLIT && !A_MN && !B_MN), "single pass: k-contiguous fp32 operands by TMA");
-  using C = Cfg<BN, BF16, SPLIT, TMA, D16, CE, ONE, CG2>;
+  using C = Cfg<BN, BF16, SPLIT, TMA, D16, CE, ONE, CG2, X2>;
   constexpr bool NOCONV = D16 || ONE;    // the operand tiles are what TMA writes: nothing to convert
   constexpr int BN_L = C::BN_L;
   const uint32_t cta_rank = CG2 ? cluster_ctarank() : 0u;   // 0: the leader of the pair
@@ -906,8 +912,17 @@ __global__ void __launch_bounds__(TMA ? NUM_THREADS_TMA : NUM_THREADS, 1) k_gemm
           const int k0 = kb * BKE;
           const uint32_t sa = smem_base + stage * C::STAGE_BYTES;
           const uint32_t sa_lo = sa + C::A_BYTES;
-          const uint32_t sb = sa + (NOCONV ? 1 : 2) * C::A_BYTES;
+          const uint32_t sb = sa + ((NOCONV && !X2) ? 1 : 2) * C::A_BYTES;
           const uint32_t bar = raw_bar(stage);
+          if (X2) {   // hi and lo tiles of both operands, [rows][64 k] boxes
+            mbar_expect_tx(bar, (uint32_t)(2 * (C::A_BYTES + C::B_BYTES)));
+            tma_load_2d(sa, &p.tmA, k0, row0a, bar);
+            tma_load_2d(sa_lo, &p.tmA2, k0, row0a, bar);
+            tma_load_2d(sb, &p.tmB, k0, row0b, bar);
+            tma_load_2d(sb + C::B_BYTES, &p.tmB2, k0, row0b, bar);
+            if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+            continue;
+          }
           if (ONE) {   // raw fp32 tiles, [rows][32 k] boxes
             mbar_expect_tx(bar, (uint32_t)(C::A_BYTES + C::B_BYTES));
             tma_load_2d(sa, &p.tmA, k0, row0a, bar);
@@ -985,13 +1000,20 @@ __global__ void __launch_bounds__(TMA ? NUM_THREADS_TMA : NUM_THREADS, 1) k_gemm
           // bf16 operands formed from TMA tiles sit behind the raw tiles of the stage
           const uint32_t sa = C::BT ? st0 + 2 * C::A_BYTES + C::B_BYTES : st0;
           const uint32_t sa_lo = sa + C::A_BYTES;
-          const uint32_t sb = C::BT ? sa + C::A_BYTES / 2 : sa + ((BF16 || ONE) ? 1 : 2) * C::A_BYTES;
+          const uint32_t sb = C::BT ? sa + C::A_BYTES / 2 : sa + (((BF16 && !X2) || ONE) ? 1 : 2) * C::A_BYTES;
           const uint32_t sb_lo = sb + C::B_BYTES;
 #pragma unroll
           for (int ks = 0; ks < C::KSTEPS; ++ks) {
             const uint64_t a_hi = (C::BT && !A_MN) ? make_desc_k64(sa + ks * A_KSTEP) : make_desc<BF16>(sa + ks * A_KSTEP, A_MN, lbo);
             const uint64_t b_hi = (C::BT && !B_MN) ? make_desc_k64(sb + ks * B_KSTEP) : make_desc<BF16>(sb + ks * B_KSTEP, B_MN, lbo);
-            if (BF16) {
+            if (X2) {
+              const uint64_t a_lo = make_desc<BF16>(sa_lo + ks * A_KSTEP, A_MN, lbo);
+              const uint64_t b_lo = make_desc<BF16>(sb_lo + ks * B_KSTEP, B_MN, lbo);
+              umma<true>(d_tmem, a_hi, b_lo, idesc, accumulate);   // small terms first
+              umma<true>(d_tmem, a_lo, b_hi, idesc, 1u);
+              umma<true>(d_tmem, a_hi, b_hi, idesc, 1u);
+              accumulate = 1;
+            } else if (BF16) {
               umma<true>(d_tmem, a_hi, b_hi, idesc, accumulate);
               accumulate = 1;
             } else if (ONE) {
@@ -1055,10 +1077,18 @@ __global__ void __launch_bounds__(TMA ? NUM_THREADS_TMA : NUM_THREADS, 1) k_gemm
 }
 
 template <int BN, bool A_MN, bool B_MN, bool BF16, bool SPLIT, bool TMA, bool D16 = false, bool CE = false, bool ONE = false,
-          bool CG2 = false>
+          bool CG2 = false, bool X2 = false>
 inline cudaError_t set_smem_attr() {
-  return cudaFuncSetAttribute(k_gemm_umma<BN, A_MN, B_MN, BF16, SPLIT, TMA, D16, CE, ONE, CG2>,
-                              cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<BN, BF16, SPLIT, TMA, D16, CE, ONE, CG2>::SMEM_BYTES);
+  return cudaFuncSetAttribute(k_gemm_umma<BN, A_MN, B_MN, BF16, SPLIT, TMA, D16, CE, ONE, CG2, X2>,
+                              cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              Cfg<BN, BF16, SPLIT, TMA, D16, CE, ONE, CG2, X2>::SMEM_BYTES);
+}
+
+// bf16 operand pairs (k-contiguous operands only)
+template <int BN>
+inline void launch_x2(const Params& p, int grid, cudaStream_t st) {
+  constexpr int smem = Cfg<BN, true, false, true, true, true, false, false, true>::SMEM_BYTES;
+  k_gemm_umma<BN, false, false, true, false, true, true, true, false, false, true><<<grid, NUM_THREADS_TMA, smem, st>>>(p);
 }
 
 // CTA pairs: clusters of two CTAs, 256 x 256 tiles (fp32 mode, TMA, coalesced epilogue)
@@ -1233,6 +1263,8 @@ inline int umma_configure() {
 #undef DION_SET
   if (e == cudaSuccess) e = set_smem_attr<128, false, false, false, false, true, false, true, true>();
   if (e == cudaSuccess) e = set_smem_attr<256, false, false, false, false, true, false, true, true>();
+  if (e == cudaSuccess) e = set_smem_attr<128, false, false, true, false, true, true, true, false, false, true>();
+  if (e == cudaSuccess) e = set_smem_attr<256, false, false, true, false, true, true, true, false, false, true>();
   if (e == cudaSuccess) e = set_pair_attr<false, false>();
   if (e == cudaSuccess) e = set_pair_attr<false, true>();
   if (e == cudaSuccess) e = set_pair_attr<true, true>();
@@ -1296,10 +1328,15 @@ inline int umma_try_launch(const GemmArgs& g_in, int precision, int sm_count, fl
   p.g = g;
   // TMA variant: fp32 operands in memory (both precision modes), dimensions the tensor maps can describe
   bool tma = (d16 || !(variant & UMMA_VARIANT_REGISTER_LOADS)) && g.M < (1ll << 31) && g.N < (1ll << 31) && g.K < (1ll << 31);
+  const bool x2 = d16 && g.A16lo != nullptr && g.B16lo != nullptr;   // bf16 operand pairs
+  if (x2 && (a_mn || b_mn || !aligned(g.A16lo, 16) || !aligned(g.B16lo, 16))) return 0;
   if (d16) {
     const i64 lda = a_mn ? g.a_sk : g.a_si, ldb = b_mn ? g.b_sk : g.b_sn;
     if (!tma || !make_operand16_map(&p.tmA, g.A, g.M, g.K, lda, a_mn, BM) ||
         !make_operand16_map(&p.tmB, g.B, g.N, g.K, ldb, b_mn, BN))
+      return 0;
+    if (x2 && (!make_operand16_map(&p.tmA2, g.A16lo, g.M, g.K, lda, a_mn, BM) ||
+               !make_operand16_map(&p.tmB2, g.B16lo, g.N, g.K, ldb, b_mn, BN)))
       return 0;
   } else
   if (tma && g.a2_mode == ADD_BF16) {   // the bf16 addend needs 16-byte aligned rows for its tensor map
@@ -1358,6 +1395,9 @@ inline int umma_try_launch(const GemmArgs& g_in, int precision, int sm_count, fl
   } else if (one) {
     if (BN == 256) launch_one<256>(p, grid, st);
     else launch_one<128>(p, grid, st);
+  } else if (x2) {
+    if (BN == 256) launch_x2<256>(p, grid, st);
+    else launch_x2<128>(p, grid, st);
   } else if (d16) {   // bf16 arrays: always with the coalesced epilogue
     if (BN == 256) launch_variant<256, true, false, true, true, true>(p, a_mn, b_mn, grid, st);
     else launch_variant<128, true, false, true, true, true>(p, a_mn, b_mn, grid, st);

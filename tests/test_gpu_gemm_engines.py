@@ -25,7 +25,8 @@ class GemmArgs(ctypes.Structure):
                 ("C", ctypes.c_void_p), ("ldc", ctypes.c_int64), ("epi", ctypes.c_int),
                 ("C2", ctypes.c_void_p), ("ldc2", ctypes.c_int64), ("c2_mode", ctypes.c_int),
                 ("alpha", ctypes.c_float), ("tri", ctypes.c_int), ("klimit", ctypes.c_int), ("precise", ctypes.c_int),
-                ("ab16", ctypes.c_int), ("tf32x1", ctypes.c_int), ("variant", ctypes.c_int)]
+                ("ab16", ctypes.c_int), ("tf32x1", ctypes.c_int), ("variant", ctypes.c_int),
+                    ("A16lo", ctypes.c_void_p), ("B16lo", ctypes.c_void_p)]
 
 
 @pytest.fixture(scope="module")
@@ -262,3 +263,37 @@ def test_cta_pairs_epilogues_triangle_and_k_limit(lib):
     assert run(lib, 2, 0, 4360, 4360, 264, True, True, tri=1) < TOL[2]
     assert run(lib, 2, 0, 2048, 512, 512, False, False, klimit=1) < TOL[2]
     assert run(lib, 2, 0, 512, 512, 8192, True, True) < TOL[2]                             # few tiles: split-K over pairs
+
+
+@pytest.mark.parametrize("M,N,K,epi", [(1024, 768, 256, 2), (1024, 768, 256, 3), (648, 392, 328, 1), (2048, 256, 2112, 0),
+                                       (128, 64, 64, 0)])
+def test_bf16_operand_pairs(lib, M, N, K, epi):
+    # each operand as a pair of bf16 arrays, x ~ hi + lo (16 significant bits): three bf16 MMAs per K step
+    g = torch.Generator(device="cuda"); g.manual_seed(M + K)
+    A = torch.randn(M, K, generator=g, device="cuda"); B = torch.randn(N, K, generator=g, device="cuda")
+    Ah = A.to(torch.bfloat16); Al = (A - Ah.float()).to(torch.bfloat16)
+    Bh = B.to(torch.bfloat16); Bl = (B - Bh.float()).to(torch.bfloat16)
+    C = torch.randn(M, N, generator=g, device="cuda"); C0 = C.clone()
+    C2 = torch.randn(M, N, generator=g, device="cuda")
+    alpha = 0.05
+    ref = A.double() @ B.double().t()
+    want = {0: alpha * ref, 1: C0.double() - alpha * ref, 2: C0.double() + C2.double() - alpha * ref,
+            3: C2.double() - alpha * ref}[epi]
+    a = GemmArgs()
+    a.M, a.N, a.K = M, N, K
+    a.A = Ah.data_ptr(); a.a_si, a.a_sk = K, 1; a.A16lo = Al.data_ptr()
+    a.B = Bh.data_ptr(); a.b_sk, a.b_sn = 1, K; a.B16lo = Bl.data_ptr()
+    a.C = C.data_ptr(); a.ldc = N; a.epi = epi
+    a.C2 = C2.data_ptr(); a.ldc2 = N; a.c2_mode = 1
+    a.alpha = alpha; a.ab16 = 1
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    rc = lib.dion_debug_gemm(2, 1, ctypes.byref(a), None, 0, status.data_ptr(), int(torch.cuda.current_stream().cuda_stream))
+    torch.cuda.synchronize()
+    assert rc == 0 and int(status.item()) == 0
+    # the product itself is accurate to ~2^-16 of |A| |B|
+    prod = {0: C.double() / alpha, 1: (C0.double() - C.double()) / alpha, 2: (C0.double() + C2.double() - C.double()) / alpha,
+            3: (C2.double() - C.double()) / alpha}[epi]
+    err_prod = float((prod - ref).norm() / ref.norm())
+    err = float((C.double() - want).norm() / want.norm())
+    assert err_prod < 3e-5, err_prod
+    assert err < 3e-6 or epi == 0, err
