@@ -155,22 +155,37 @@ def phase_bytes(m, n, r, orth, gbytes=4, rounds=None):
             "ORTH_GEMM": rounds * 4.0 * (3 * m * r + 4 * r * r)}
 
 
+def pairs_apply(m, n, r):
+    """Shapes whose R and error-feedback products run on bf16 (hi, lo) pairs in fp32 mode (the library's own rule:
+    M + G kept in scratch, i.e. rank fraction >= 1/8, and dimensions that are multiples of 8)."""
+    return r >= 64 and 8 * r >= min(m, n) and m % 8 == 0 and n % 8 == 0 and r % 8 == 0 and m >= 128 and n >= 128
+
+
 def case_report(c, ms, rounds, args, peaks, binding):
     """Per-case line: time and the roofline that binds it.  t_hbm: the 7-pass model (read M and G twice,
-    read-modify-write M, read-modify-write X) at the measured copy bandwidth; t_tensor: the four products
-    (and the orthonormalization, always 3xTF32) at the tensor peak of their arithmetic, TF32 taken as half
-    the measured bf16 peak and a 3xTF32 product as three TF32 passes."""
+    read-modify-write M, read-modify-write X) at the measured copy bandwidth; t_tensor: every product at the
+    tensor peak of the arithmetic it runs in -- fp32 mode: P and the orthonormalization 3xTF32 (three TF32
+    passes, TF32 taken as half the measured bf16 peak), R and the error feedback three bf16 passes on (hi, lo)
+    pairs where the library uses them (else 3xTF32), the X update one TF32 pass; bf16-operand mode: one bf16 pass
+    for the four products."""
     m, n, r = c[:3]
-    out = {"m": m, "n": n, "r": r, "ms": ms, "orth_mode": ["auto", "cholqr2", "adaptive", "householder", "rcqr"][orth_mode(m, n, r, args.orth)], "orth_rounds": rounds}
+    out = {"m": m, "n": n, "r": r, "ms": ms,
+           "orth_mode": ["auto", "cholqr2", "adaptive", "householder", "rcqr"][orth_mode(m, n, r, args.orth)], "orth_rounds": rounds}
     if ms is None or args.engine == binding.ENGINE_SIMT or args.lazy:
         return out
     gb = case_gbytes(c)
     fl = phase_flops(m, n, r, args.orth, rounds=rounds)
     model_bytes = float(m) * n * (20 + 2 * gb) + 4.0 * (3 * n * r + 3 * m * r)
-    tf32x3 = peaks["bf16_sustained"] * 0.5 / 3.0
-    prod_peak = peaks["bf16_sustained"] if args.precision == binding.PREC_BF16_OPERANDS else tf32x3
+    bf16 = peaks["bf16_sustained"]
+    tf32 = 0.5 * bf16
     t_hbm = model_bytes / (peaks["hbm_gbs"] * 1e9) * 1e3
-    t_tensor = (sum(fl[p] for p in ("P", "R", "EF", "X")) / (prod_peak * 1e12) + fl["ORTH"] / (tf32x3 * 1e12)) * 1e3
+    if args.precision == binding.PREC_BF16_OPERANDS:
+        t_prod = sum(fl[p] for p in ("P", "R", "EF", "X")) / (bf16 * 1e12)
+    else:
+        pair_peak = bf16 / 3.0 if pairs_apply(m, n, r) else tf32 / 3.0
+        ef_peak = bf16 / 3.0 if (m % 8 == 0 and n % 8 == 0 and r % 8 == 0 and r >= 64) else tf32 / 3.0
+        t_prod = fl["P"] / (tf32 / 3.0 * 1e12) + fl["R"] / (pair_peak * 1e12) + fl["EF"] / (ef_peak * 1e12) + fl["X"] / (tf32 * 1e12)
+    t_tensor = (t_prod + fl["ORTH"] / (tf32 / 3.0 * 1e12)) * 1e3
     bound = "hbm" if t_hbm >= t_tensor else "tensor"
     out.update({"t_hbm_ms": t_hbm, "t_tensor_ms": t_tensor, "bound": bound,
                 "roofline_frac": max(t_hbm, t_tensor) / ms, "model_gbs": model_bytes / (ms * 1e-3) / 1e9})
@@ -692,8 +707,9 @@ def workload_record(wid, cases, grouped, args, peaks, binding, ms_step, e2e_ms, 
                                "ten consecutive dion_step calls per step" if reps_per_step > 1 else
                                "one dion_step call per matrix per step"),
                       "engine": ["auto", "simt", "tensor"][args.engine],
-                      "precision": ["fp32 (3xTF32 on tensor cores / FMA; the X update single-pass TF32 on rounded factors)",
-                                    "bf16 operands"][args.precision],
+                      "precision": ["fp32 (P and Orthonormalize 3xTF32; R and the error feedback on bf16 (hi, lo) pairs, 16 "
+                                    "significant bits, where M + G is kept in scratch; the X update single-pass TF32 on "
+                                    "rounded factors; FMA for ragged shapes)", "bf16 operands"][args.precision],
                       "orth": ["auto", "cholqr2", "shifted3", "householder", "rcqr"][args.orth],
                       "sync": ("compressed data-parallel sync: P and W all-reduced (mean) over the ranks"
                                if args.sync == "dp" else "none (independent replicas)"),

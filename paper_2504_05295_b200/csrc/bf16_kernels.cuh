@@ -66,9 +66,12 @@ __global__ void __launch_bounds__(256) k_form_b16(const float* __restrict__ M, i
 // B32 = M + G in fp32, rows x cols (cols a multiple of 4), B32 dense with leading dimension cols: the sum the
 // fused operand formation of the contraction kernel computes, formed once per step where two products and the
 // error feedback read it.  One thread per 4 consecutive elements of a row; VEC as above.
+// hi / lo (optional, both or neither; cols a multiple of 8 then): the same sum as a pair of bf16 arrays, hi = bf16(sum),
+// lo = bf16(sum - hi), dense like out: the operand of the products that run on bf16 pairs.
 template <bool VEC>
 __global__ void __launch_bounds__(256) k_form_b32(const float* __restrict__ M, i64 ldm, const void* __restrict__ G,
-                                                  i64 ldg, int g_mode, i64 rows, i64 cols, float* __restrict__ out) {
+                                                  i64 ldg, int g_mode, i64 rows, i64 cols, float* __restrict__ out,
+                                                  __nv_bfloat16* __restrict__ hi, __nv_bfloat16* __restrict__ lo) {
   pdl_enter();
   const i64 per_row = cols / 4;
   const i64 total = rows * per_row;
@@ -97,6 +100,15 @@ __global__ void __launch_bounds__(256) k_form_b32(const float* __restrict__ M, i
       }
     }
     *reinterpret_cast<float4*>(out + i * cols + c) = v;
+    if (hi != nullptr) {
+      const float h0 = __bfloat162float(__float2bfloat16_rn(v.x)), h1 = __bfloat162float(__float2bfloat16_rn(v.y));
+      const float h2 = __bfloat162float(__float2bfloat16_rn(v.z)), h3 = __bfloat162float(__float2bfloat16_rn(v.w));
+      uint2 oh, ol;
+      oh.x = pack_bf16x2(h0, h1); oh.y = pack_bf16x2(h2, h3);
+      ol.x = pack_bf16x2(v.x - h0, v.y - h1); ol.y = pack_bf16x2(v.z - h2, v.w - h3);
+      *reinterpret_cast<uint2*>(hi + i * cols + c) = oh;
+      *reinterpret_cast<uint2*>(lo + i * cols + c) = ol;
+    }
   }
 }
 

@@ -49,6 +49,7 @@ struct Layout {
   i64 Psave;                // CholeskyQR2: the panel as the product wrote it, kept for the fallback (0: none)
   i64 fb_part, fb_h, fb_n;  // fallback kernel: partial dot products (SMs x r), their sums (r), partial norms (SMs)
   i64 probe_y, probe_part;  // CholeskyQR2's orthogonality probe: U1 z (rows x NPROBE), partial U1^T (U1 z)
+  i64 Bp;                   // fp32 mode, M + G in scratch: the same sum as a bf16 (hi, lo) pair (m x n x 2 bf16) for R; 0: none
   i64 S16;                  // fp32 mode: the bf16 (hi, lo) pair of the error feedback's second factor (max(m,n) x r x 2 bf16)
   i64 part_floats;
   int cn_chunks;
@@ -146,8 +147,11 @@ Layout make_layout(const dion_ctx* c, i64 m, i64 n, i64 r) {
     L.U16 = o; o += align64((big * r + 1) / 2);
     L.R16 = o; o += align64((big * r + 1) / 2);
   }
-  L.B32 = 0;
-  if (sum_in_scratch(c, m, n, r)) { L.B32 = o; o += align64(m * n); }
+  L.B32 = L.Bp = 0;
+  if (sum_in_scratch(c, m, n, r)) {
+    L.B32 = o; o += align64(m * n);
+    if (m % 8 == 0 && n % 8 == 0 && r % 8 == 0) { L.Bp = o; o += align64(m * n); }
+  }
   L.Psave = L.fb_part = L.fb_h = L.fb_n = 0;
   L.S16 = o; o += align64(big * r);
   L.probe_y = o; o += align64(big * NPROBE);
@@ -515,7 +519,9 @@ int potrf_trtri(StepCtx& s, i64 r, int mode, bool full_inverse,
 // rows x r panels, ld = r; pin_off / pout_off are offsets in the scratch slice.
 // adaptive: columns with negligible pivots are deflated, the round is skipped (Pout = Pin)
 // once the panel is orthonormal, and the round statistics are evaluated at the end.
-int cholqr_round(StepCtx& s, i64 pin_off, i64 pout_off, i64 rows, i64 r, int mode, i64 gram_rows = 0) {
+int cholqr_round(StepCtx& s, i64 pin_off, i64 pout_off, i64 rows, i64 r, int mode, i64 gram_rows = 0,
+                 bool passthrough = true) {
+  // passthrough = false: a skipped round leaves Pout untouched (the caller keeps using Pin)
   // gram_rows > 0: the Gram matrix is formed from the first gram_rows rows only (a sketch stacked on
   // top of the panel); the factor is applied to all rows
   dion_ctx* c = s.c;
@@ -551,7 +557,7 @@ int cholqr_round(StepCtx& s, i64 pin_off, i64 pout_off, i64 rows, i64 r, int mod
   // alone, 512-column products need >= 128 row tiles to fill the GPU; beside the factorization
   // (second stream) they are background work at any height
   const bool trsm = (r > NBO) && (rows >= 8192 || c->side != nullptr);
-  if (skips) {   // a finished panel is passed through (before anything writes Pout)
+  if (skips && passthrough) {   // a finished panel is passed through (before anything writes Pout)
     dim3 grid((unsigned)grid_for(c, rows * r), (unsigned)s.nb);
     launch_pdl(k_copy_panel, grid, dim3(256), 0, s.st, s.ws + pin_off, r, s.ws + pout_off, r, rows, r, nullptr, s.os + OS_DONE, s.wstride);
     DION_CHECK_LAUNCH(c);
@@ -780,10 +786,18 @@ int orthonormalize(StepCtx& s, i64 rows, i64 r, i64 short_dim, i64 pin_off, i64*
     // orthonormalizes the saved panel and clears the flag, or confirms the breakdown.
     const bool fb = pin_off != s.L.P0 && fallback_fits(s.c, rows);
     s.quiet_fail = fb;
-    int rc = cholqr_round(s, pin_off, s.L.P1, rows, r, RM_FIRST);
-    if (rc == DION_OK) rc = cholqr_round(s, s.L.P1, s.L.P0, rows, r, RM_CHECKED);
+    // Round one writes P0, where U is expected; the second round, when it runs, goes P0 -> P1 and is copied
+    // back: the common case (one round) moves the panel once.
+    int rc = cholqr_round(s, pin_off, s.L.P0, rows, r, RM_FIRST);
+    if (rc == DION_OK) rc = cholqr_round(s, s.L.P0, s.L.P1, rows, r, RM_CHECKED, 0, false);
     s.quiet_fail = false;
     DION_TRY(rc);
+    {
+      dim3 grid((unsigned)grid_for(s.c, rows * r), (unsigned)s.nb);
+      launch_pdl(k_copy_panel, grid, dim3(256), 0, s.st, (const float*)(s.ws + s.L.P1), r, s.ws + s.L.P0, r, rows, r,
+                 (const int*)(s.os + OS_DONE), (const int*)nullptr, s.wstride);
+      DION_CHECK_LAUNCH(s.c);
+    }
     if (fb) DION_TRY(cgs_fallback(s, pin_off, s.L.P0, rows, r));   // else: the failed pivot was reported as a breakdown
     *U_off = s.L.P0;
   } else if (mode == DION_ORTH_SHIFTED3) {
@@ -866,6 +880,50 @@ int begin_step(dion_ctx* c, const dion_matrix* a, int nb, cudaStream_t st, StepC
   return DION_OK;
 }
 
+// R = (M + G)^T U on bf16 pairs (transposed form: (M + G) U): where M + G is kept in scratch (sum_in_scratch) the
+// product runs on the bf16 (hi, lo) pair of the sum and of U, three bf16 MMAs per K step (1.3 TF32 passes instead of
+// three); it is accurate to ~1e-5, which is what Q <- ColNorm(R) and the error feedback need of it.
+bool r_on_pairs(const StepCtx& s, i64 m, i64 n, i64 r) {
+  return s.tensor && s.c->cfg.precision == DION_PREC_FP32 && s.L.B32 > 0 && s.L.Bp > 0 && m >= 128 && n >= 128 && r >= 64;
+}
+
+// Forms M + G in scratch (fp32) and, when `pair`, as a bf16 pair beside it.
+int form_sum(StepCtx& s, int b, const dion_matrix* a, bool pair) {
+  dion_ctx* c = s.c;
+  const i64 m = a->m, n = a->n;
+  const bool vec = !((uintptr_t)a->M & 15) && a->ldm % 4 == 0 &&
+                   (a->g_dtype == DION_BF16 ? (!((uintptr_t)a->G & 7) && a->ldg % 4 == 0)
+                                            : (!((uintptr_t)a->G & 15) && a->ldg % 4 == 0));
+  const int g_mode = (a->g_dtype == DION_BF16) ? ADD_BF16 : ADD_F32;
+  const int grid = grid_for(c, m * n / 4);
+  __nv_bfloat16* bh = pair ? reinterpret_cast<__nv_bfloat16*>(s.W(b, s.L.Bp)) : nullptr;
+  __nv_bfloat16* bl = pair ? bh + m * n : nullptr;
+  if (vec) launch_pdl(k_form_b32<true>, grid, dim3(256), 0, s.st, (const float*)a->M, a->ldm, a->G, a->ldg, g_mode, m, n, s.W(b, s.L.B32), bh, bl);
+  else launch_pdl(k_form_b32<false>, grid, dim3(256), 0, s.st, (const float*)a->M, a->ldm, a->G, a->ldg, g_mode, m, n, s.W(b, s.L.B32), bh, bl);
+  DION_CHECK_LAUNCH(c);
+  return DION_OK;
+}
+
+// The product itself: U (prow x r, dense) is split into the panel buffer `upair`; the pair of M + G must be in place.
+int r_pairs(StepCtx& s, int b, const dion_matrix* a, bool tr, const float* U, float* upair, float* out, const int* skip) {
+  dion_ctx* c = s.c;
+  const i64 m = a->m, n = a->n, r = a->r;
+  const i64 prow = tr ? n : m, qrow = tr ? m : n;
+  __nv_bfloat16* uh = reinterpret_cast<__nv_bfloat16*>(upair);
+  __nv_bfloat16* ul = uh + prow * r;
+  launch_pdl(k_split_bf16, dim3((unsigned)grid_for(c, prow * r / 8)), dim3(256), 0, s.st, U, r, prow, r, uh, ul, skip);
+  DION_CHECK_LAUNCH(c);
+  __nv_bfloat16* bh = reinterpret_cast<__nv_bfloat16*>(s.W(b, s.L.Bp));
+  GemmArgs w = gemm_args();
+  w.M = qrow; w.N = r; w.K = prow;
+  w.ab16 = 1;
+  w.A = (const float*)bh; w.A16lo = bh + m * n; w.a_si = tr ? n : 1; w.a_sk = tr ? 1 : n;
+  w.B = (const float*)uh; w.B16lo = ul; w.b_sk = r; w.b_sn = 1;
+  w.C = out; w.ldc = r; w.epi = EPI_STORE;
+  w.skip_flag = skip;
+  return launch_gemm(s, w, b);
+}
+
 // The weight update X <- X - alpha F1 F2^T in fp32 mode on the tensor engine (F1: m x r with leading dimension
 // ld1, F2: n x r with ld2; U Q^T, or Q U^T in the transposed form).  The update feeds nothing else, so its two
 // factors are rounded to TF32 once (to nearest: unbiased) into `r1`, `r2` (scratch, dense) and the product takes
@@ -883,8 +941,9 @@ bool x_single_pass(const StepCtx& s, const dion_matrix* a, const float* F1, i64 
 // (hi, lo) in scratch (`p1`, `p2`: max(m,n) x r floats each) and the product takes three bf16 MMAs per K step, 1.3
 // TF32 passes instead of three.  Otherwise the 3xTF32 / FMA product of the fp32 factors.
 // sum32 != nullptr: M + G comes from scratch (C = sum32 - beta acc); else C = M + G - beta acc with the caller's G.
+// ready1 / ready2: that factor's pair already sits in p1 / p2 (the step splits U for R).
 int ef_update(StepCtx& s, int b, const dion_matrix* a, const float* F1, i64 ld1, const float* F2, i64 ld2, float* p1,
-              float* p2, const float* sum32, const int* skip) {
+              float* p2, const float* sum32, const int* skip, bool ready1 = false, bool ready2 = false) {
   dion_ctx* c = s.c;
   const i64 m = a->m, n = a->n, r = a->r;
   GemmArgs e = gemm_args();
@@ -898,10 +957,14 @@ int ef_update(StepCtx& s, int b, const dion_matrix* a, const float* F1, i64 ld1,
     __nv_bfloat16* l1 = h1 + m * r;
     __nv_bfloat16* h2 = reinterpret_cast<__nv_bfloat16*>(p2);
     __nv_bfloat16* l2 = h2 + n * r;
-    launch_pdl(k_split_bf16, dim3((unsigned)grid_for(c, m * r / 8)), dim3(256), 0, s.st, F1, ld1, m, r, h1, l1, skip);
-    DION_CHECK_LAUNCH(c);
-    launch_pdl(k_split_bf16, dim3((unsigned)grid_for(c, n * r / 8)), dim3(256), 0, s.st, F2, ld2, n, r, h2, l2, skip);
-    DION_CHECK_LAUNCH(c);
+    if (!ready1) {
+      launch_pdl(k_split_bf16, dim3((unsigned)grid_for(c, m * r / 8)), dim3(256), 0, s.st, F1, ld1, m, r, h1, l1, skip);
+      DION_CHECK_LAUNCH(c);
+    }
+    if (!ready2) {
+      launch_pdl(k_split_bf16, dim3((unsigned)grid_for(c, n * r / 8)), dim3(256), 0, s.st, F2, ld2, n, r, h2, l2, skip);
+      DION_CHECK_LAUNCH(c);
+    }
     e.ab16 = 1;
     e.A = (const float*)h1; e.A16lo = l1; e.a_si = r; e.a_sk = 1;
     e.B = (const float*)h2; e.B16lo = l2; e.b_sk = 1; e.b_sn = r;
@@ -981,6 +1044,9 @@ int step_batch(dion_ctx* c, const dion_matrix* const* list, int nb, float lr, cu
 
   // fp32 mode: M + G kept in scratch for P, R and the error feedback (see sum_in_scratch)
   const bool b32 = !d16 && s.tensor && s.L.B32 > 0;
+  // ... R then runs on bf16 pairs of M + G and of U (three bf16 MMAs per K step: 1.3 TF32 passes instead of 3; the
+  // product is accurate to ~1e-5, which is what Q <- ColNorm(R) and the error feedback need of it)
+  const bool bpair = b32 && r_on_pairs(s, m, n, r);
 
   // P = (M + G) Q   (transposed form: (M + G)^T Q)
   const i64 pin_off = panel_offset(s, r, (m < n) ? m : n);
@@ -1003,13 +1069,7 @@ int step_batch(dion_ctx* c, const dion_matrix* const* list, int nb, float lr, cu
       p.A = (const float*)bf(b, s.L.B16); p.a_si = tr ? 1 : n; p.a_sk = tr ? n : 1;
       p.B = (const float*)bf(b, s.L.Q16); p.b_sk = r; p.b_sn = 1;
     } else if (b32) {
-      const bool vec = !((uintptr_t)a->M & 15) && a->ldm % 4 == 0 &&
-                       (a->g_dtype == DION_BF16 ? (!((uintptr_t)a->G & 7) && a->ldg % 4 == 0)
-                                                : (!((uintptr_t)a->G & 15) && a->ldg % 4 == 0));
-      const int grid = grid_for(c, m * n / 4);
-      if (vec) launch_pdl(k_form_b32<true>, grid, dim3(256), 0, st, (const float*)a->M, a->ldm, a->G, a->ldg, g_mode(a), m, n, s.W(b, s.L.B32));
-      else launch_pdl(k_form_b32<false>, grid, dim3(256), 0, st, (const float*)a->M, a->ldm, a->G, a->ldg, g_mode(a), m, n, s.W(b, s.L.B32));
-      DION_CHECK_LAUNCH(c);
+      DION_TRY(form_sum(s, b, a, bpair));
       p.A = s.W(b, s.L.B32); p.a_si = tr ? 1 : n; p.a_sk = tr ? n : 1;
       p.B = (const float*)a->Q; p.b_sk = a->ldq; p.b_sn = 1;
     } else {
@@ -1046,6 +1106,10 @@ int step_batch(dion_ctx* c, const dion_matrix* const* list, int nb, float lr, cu
       w.ab16 = 1;
       w.A = (const float*)bf(b, s.L.B16); w.a_si = tr ? n : 1; w.a_sk = tr ? 1 : n;
       w.B = (const float*)bf(b, s.L.U16); w.b_sk = r; w.b_sn = 1;
+    } else if (bpair) {
+      // U as a bf16 pair in the other panel buffer (the error feedback reuses it)
+      DION_TRY(r_pairs(s, b, a, tr, s.W(b, U_off), s.W(b, U_off == s.L.P0 ? s.L.P1 : s.L.P0), s.W(b, s.L.R), s.OS(b) + OS_FAIL));
+      continue;
     } else if (b32) {
       w.A = s.W(b, s.L.B32); w.a_si = tr ? n : 1; w.a_sk = tr ? 1 : n;
       w.B = s.W(b, U_off); w.b_sk = r; w.b_sn = 1;
@@ -1084,8 +1148,8 @@ int step_batch(dion_ctx* c, const dion_matrix* const* list, int nb, float lr, cu
     const float* Uf = s.W(b, U_off);
     const float* Rf = s.W(b, s.L.R);
     const float* sum32 = b32 ? s.W(b, s.L.B32) : nullptr;
-    if (tr) DION_TRY(ef_update(s, b, a, Rf, r, Uf, r, sbuf, other, sum32, s.OS(b) + OS_FAIL));
-    else DION_TRY(ef_update(s, b, a, Uf, r, Rf, r, other, sbuf, sum32, s.OS(b) + OS_FAIL));
+    if (tr) DION_TRY(ef_update(s, b, a, Rf, r, Uf, r, sbuf, other, sum32, s.OS(b) + OS_FAIL, false, bpair));
+    else DION_TRY(ef_update(s, b, a, Uf, r, Rf, r, other, sbuf, sum32, s.OS(b) + OS_FAIL, bpair, false));
   }
   }
 
@@ -1446,6 +1510,10 @@ int dion_dp_factor(dion_ctx* ctx, const dion_matrix* a, float* PU, float* W, int
   DION_CHECK_LAUNCH(ctx);
   launch_pdl(k_latch_flag, dim3((unsigned)(1)), dim3(1), 0, st, s.flag, dp_flag);      // a breakdown cancels dion_dp_finish
   DION_CHECK_LAUNCH(ctx);
+  if (r_on_pairs(s, m, n, r)) {       // as dion_step: W on the bf16 pairs of M + G and U
+    DION_TRY(form_sum(s, 0, a, true));
+    return r_pairs(s, 0, a, false, PU, s.ws + s.L.P1, W, nullptr);
+  }
   return launch_gemm(s, dp_b_product(a, true, PU, W), 0);
 }
 
@@ -1531,9 +1599,14 @@ int dion_shard_factor(dion_ctx* ctx, const dion_matrix* a, int64_t n_total, cons
   StepCtx s;
   cudaStream_t st = (cudaStream_t)cuda_stream;
   DION_TRY(begin_step(ctx, a, 1, st, &s));
-  GemmArgs w = dp_b_product(a, true, U, W);
-  w.skip_flag = flag;
-  DION_TRY(launch_gemm(s, w, 0));
+  if (r_on_pairs(s, a->m, a->n, a->r)) {       // as dion_step: W on the bf16 pairs of M + G and U
+    DION_TRY(form_sum(s, 0, a, true));
+    DION_TRY(r_pairs(s, 0, a, false, U, s.ws + s.L.P1, W, flag));
+  } else {
+    GemmArgs w = dp_b_product(a, true, U, W);
+    w.skip_flag = flag;
+    DION_TRY(launch_gemm(s, w, 0));
+  }
   int chunks; i64 per;
   colnorm_plan(a->n, a->r, ctx->sm_count, &chunks, &per);
   float* part = s.W(0, s.L.cn_part);

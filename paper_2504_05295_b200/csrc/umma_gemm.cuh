@@ -528,7 +528,7 @@ struct Cfg {
 template <int BN, bool A_MN, bool B_MN, bool BF16, bool SPLIT, bool TMA, bool D16 = false, bool CE = false, bool ONE = false,
           bool CG2 = false, bool X2 = false>
 __global__ void __launch_bounds__(TMA ? NUM_THREADS_TMA : NUM_THREADS, 1) k_gemm_umma(const __grid_constant__ Params p) {
-  static_assert(!X2 || (D16 && CE && !A_MN && !B_MN), "operand pairs: k-contiguous bf16 arrays");
+  static_assert(!X2 || (D16 && CE), "operand pairs are bf16 arrays");
   static_assert(!CG2 || (TMA && !BF16 && !D16 && !ONE && BN == 256), "CTA pairs: the fp32 TMA variants with 256-column tiles");
   static_assert(!(BF16 && SPLIT), "split accumulators belong to the 3xTF32 mode");
   static_assert(!D16 || (BF16 && TMA), "bf16 operands in memory are loaded by TMA");
@@ -914,12 +914,29 @@ __global__ void __launch_bounds__(TMA ? NUM_THREADS_TMA : NUM_THREADS, 1) k_gemm
           const uint32_t sa_lo = sa + C::A_BYTES;
           const uint32_t sb = sa + ((NOCONV && !X2) ? 1 : 2) * C::A_BYTES;
           const uint32_t bar = raw_bar(stage);
-          if (X2) {   // hi and lo tiles of both operands, [rows][64 k] boxes
+          if (X2) {   // hi and lo tiles of both operands: [rows][64 k] boxes, or [64 k][64 rows] boxes per 64-row chunk
             mbar_expect_tx(bar, (uint32_t)(2 * (C::A_BYTES + C::B_BYTES)));
-            tma_load_2d(sa, &p.tmA, k0, row0a, bar);
-            tma_load_2d(sa_lo, &p.tmA2, k0, row0a, bar);
-            tma_load_2d(sb, &p.tmB, k0, row0b, bar);
-            tma_load_2d(sb + C::B_BYTES, &p.tmB2, k0, row0b, bar);
+            const uint32_t sb_lo2 = sb + C::B_BYTES;
+            if (!A_MN) {
+              tma_load_2d(sa, &p.tmA, k0, row0a, bar);
+              tma_load_2d(sa_lo, &p.tmA2, k0, row0a, bar);
+            } else {
+#pragma unroll
+              for (int c = 0; c < BM / 64; ++c) {
+                tma_load_2d(sa + c * (BKE * 128), &p.tmA, row0a + 64 * c, k0, bar);
+                tma_load_2d(sa_lo + c * (BKE * 128), &p.tmA2, row0a + 64 * c, k0, bar);
+              }
+            }
+            if (!B_MN) {
+              tma_load_2d(sb, &p.tmB, k0, row0b, bar);
+              tma_load_2d(sb_lo2, &p.tmB2, k0, row0b, bar);
+            } else {
+#pragma unroll
+              for (int c = 0; c < BN / 64; ++c) {
+                tma_load_2d(sb + c * (BKE * 128), &p.tmB, row0b + 64 * c, k0, bar);
+                tma_load_2d(sb_lo2 + c * (BKE * 128), &p.tmB2, row0b + 64 * c, k0, bar);
+              }
+            }
             if (++stage == STAGES) { stage = 0; phase ^= 1u; }
             continue;
           }
@@ -1084,11 +1101,22 @@ inline cudaError_t set_smem_attr() {
                               Cfg<BN, BF16, SPLIT, TMA, D16, CE, ONE, CG2, X2>::SMEM_BYTES);
 }
 
-// bf16 operand pairs (k-contiguous operands only)
-template <int BN>
-inline void launch_x2(const Params& p, int grid, cudaStream_t st) {
+// bf16 operand pairs
+template <int BN, bool A_MN, bool B_MN>
+inline void launch_x2_one(const Params& p, int grid, cudaStream_t st) {
   constexpr int smem = Cfg<BN, true, false, true, true, true, false, false, true>::SMEM_BYTES;
-  k_gemm_umma<BN, false, false, true, false, true, true, true, false, false, true><<<grid, NUM_THREADS_TMA, smem, st>>>(p);
+  k_gemm_umma<BN, A_MN, B_MN, true, false, true, true, true, false, false, true><<<grid, NUM_THREADS_TMA, smem, st>>>(p);
+}
+template <int BN>
+inline void launch_x2(const Params& p, bool a_mn, bool b_mn, int grid, cudaStream_t st) {
+  if (!a_mn && !b_mn) launch_x2_one<BN, false, false>(p, grid, st);
+  else if (!a_mn && b_mn) launch_x2_one<BN, false, true>(p, grid, st);
+  else if (a_mn && b_mn) launch_x2_one<BN, true, true>(p, grid, st);
+  else launch_x2_one<BN, true, false>(p, grid, st);
+}
+template <int BN, bool A_MN, bool B_MN>
+inline cudaError_t set_x2_attr() {
+  return set_smem_attr<BN, A_MN, B_MN, true, false, true, true, true, false, false, true>();
 }
 
 // CTA pairs: clusters of two CTAs, 256 x 256 tiles (fp32 mode, TMA, coalesced epilogue)
@@ -1263,8 +1291,14 @@ inline int umma_configure() {
 #undef DION_SET
   if (e == cudaSuccess) e = set_smem_attr<128, false, false, false, false, true, false, true, true>();
   if (e == cudaSuccess) e = set_smem_attr<256, false, false, false, false, true, false, true, true>();
-  if (e == cudaSuccess) e = set_smem_attr<128, false, false, true, false, true, true, true, false, false, true>();
-  if (e == cudaSuccess) e = set_smem_attr<256, false, false, true, false, true, true, true, false, false, true>();
+  if (e == cudaSuccess) e = set_x2_attr<128, false, false>();
+  if (e == cudaSuccess) e = set_x2_attr<128, false, true>();
+  if (e == cudaSuccess) e = set_x2_attr<128, true, true>();
+  if (e == cudaSuccess) e = set_x2_attr<128, true, false>();
+  if (e == cudaSuccess) e = set_x2_attr<256, false, false>();
+  if (e == cudaSuccess) e = set_x2_attr<256, false, true>();
+  if (e == cudaSuccess) e = set_x2_attr<256, true, true>();
+  if (e == cudaSuccess) e = set_x2_attr<256, true, false>();
   if (e == cudaSuccess) e = set_pair_attr<false, false>();
   if (e == cudaSuccess) e = set_pair_attr<false, true>();
   if (e == cudaSuccess) e = set_pair_attr<true, true>();
@@ -1329,7 +1363,7 @@ inline int umma_try_launch(const GemmArgs& g_in, int precision, int sm_count, fl
   // TMA variant: fp32 operands in memory (both precision modes), dimensions the tensor maps can describe
   bool tma = (d16 || !(variant & UMMA_VARIANT_REGISTER_LOADS)) && g.M < (1ll << 31) && g.N < (1ll << 31) && g.K < (1ll << 31);
   const bool x2 = d16 && g.A16lo != nullptr && g.B16lo != nullptr;   // bf16 operand pairs
-  if (x2 && (a_mn || b_mn || !aligned(g.A16lo, 16) || !aligned(g.B16lo, 16))) return 0;
+  if (x2 && (!aligned(g.A16lo, 16) || !aligned(g.B16lo, 16))) return 0;
   if (d16) {
     const i64 lda = a_mn ? g.a_sk : g.a_si, ldb = b_mn ? g.b_sk : g.b_sn;
     if (!tma || !make_operand16_map(&p.tmA, g.A, g.M, g.K, lda, a_mn, BM) ||
@@ -1396,8 +1430,8 @@ inline int umma_try_launch(const GemmArgs& g_in, int precision, int sm_count, fl
     if (BN == 256) launch_one<256>(p, grid, st);
     else launch_one<128>(p, grid, st);
   } else if (x2) {
-    if (BN == 256) launch_x2<256>(p, grid, st);
-    else launch_x2<128>(p, grid, st);
+    if (BN == 256) launch_x2<256>(p, a_mn, b_mn, grid, st);
+    else launch_x2<128>(p, a_mn, b_mn, grid, st);
   } else if (d16) {   // bf16 arrays: always with the coalesced epilogue
     if (BN == 256) launch_variant<256, true, false, true, true, true>(p, a_mn, b_mn, grid, st);
     else launch_variant<128, true, false, true, true, true>(p, a_mn, b_mn, grid, st);
