@@ -508,9 +508,15 @@ def run_workload(wid, cases, grouped, args, ctx):
     # The gradients arrive matrix by matrix on a copy stream; a matrix is stepped as soon as its
     # gradient has landed, so the copy of the next one overlaps the kernels of this one (within a
     # step only: a step's gradients cannot exist before the previous step's update).  A grouped
-    # workload waits for its last gradient and makes its one dion_step_grouped call.
+    # workload is stepped in up to E2E_GROUPS dion_step_grouped calls, one per group of consecutive
+    # matrices (whole layers), each as soon as its group's gradients have landed: with one call for the
+    # whole list the 14 GB of gradients of the 8B list would have to land before the first kernel.
     copy_stream = torch.cuda.Stream(device=dev)
     done_ev = [None] * len(state)       # matrix k's kernels of the previous step (they read G_k)
+    E2E_GROUPS = 4
+    ngroups = min(E2E_GROUPS, max(1, len(state) // 7)) if grouped else 1
+    bounds = [len(state) * i // ngroups for i in range(ngroups + 1)]
+    group_packed = [binding.Dion.pack([st["descs"][0] for st in state[bounds[i]:bounds[i + 1]]]) for i in range(ngroups)] if grouped else []
 
     def e2e_once(after=None):
         landed = []
@@ -523,12 +529,18 @@ def run_workload(wid, cases, grouped, args, ctx):
                 st["G"][0].copy_(hg, non_blocking=True)
                 ev = torch.cuda.Event(); ev.record(copy_stream)
                 landed.append(ev)
-        if grouped or dp_sync:
+        if grouped:
+            for gi in range(ngroups):
+                lo, hi = bounds[gi], bounds[gi + 1]
+                stream.wait_event(landed[hi - 1])
+                opt.step_grouped_packed(group_packed[gi], hi - lo, ETA, sptr)
+                ev = torch.cuda.Event(); ev.record(stream)
+                for k in range(lo, hi):
+                    host_d[k].copy_(state[k]["d"], non_blocking=True)
+                    done_ev[k] = ev
+        elif dp_sync:
             stream.wait_event(landed[-1])
-            if grouped:
-                opt.step_grouped_packed(packed[0], len(state), ETA, sptr)
-            else:
-                steppers[0].step(ETA, stream)
+            steppers[0].step(ETA, stream)
             ev = torch.cuda.Event(); ev.record(stream)
             for k, (st, hd) in enumerate(zip(state, host_d)):
                 hd.copy_(st["d"], non_blocking=True)
@@ -596,19 +608,20 @@ def run_workload(wid, cases, grouped, args, ctx):
         sample_gpu_ms = tot
 
     rec = None
+    e2e_calls = (ngroups if grouped else len(state)) * reps_per_step
     if rank == 0:
-        rec = workload_record(wid, cases, grouped, args, peaks, binding, ms_step, e2e_ms, e2e_steps, h2d, d2h,
+        rec = workload_record(wid, cases, grouped, args, peaks, binding, ms_step, e2e_ms, e2e_steps, e2e_calls, h2d, d2h,
                               launches, clocks, phase_ms, phase_launches, case_ms, case_rounds, need,
                               (status, status2, status3, skipped + skipped2), reps_per_step, world,
                               sum(1 for st in state if st["transposed"]))
         rec["sample_gpu_ms"] = sample_gpu_ms
     opt.close()
-    del state, packed, steppers, host_d
+    del state, packed, steppers, host_d, group_packed
     torch.cuda.empty_cache()
     return rec
 
 
-def workload_record(wid, cases, grouped, args, peaks, binding, ms_step, e2e_ms, e2e_steps, h2d, d2h, launches, clocks,
+def workload_record(wid, cases, grouped, args, peaks, binding, ms_step, e2e_ms, e2e_steps, e2e_calls, h2d, d2h, launches, clocks,
                     phase_ms, phase_launches, case_ms, case_rounds, need, stat, reps_per_step, world, n_transposed):
     # ---- roofline of the dominant phase ---------------------------------------------------
     # Algorithmic work: the four products, 8 m n r flops, plus the orthonormalization counted as CholeskyQR2
@@ -722,7 +735,8 @@ def workload_record(wid, cases, grouped, args, peaks, binding, ms_step, e2e_ms, 
            "cases": ([] if len(cases) > 32 else
                      [case_report(c, ms, nr, args, peaks, binding) for c, ms, nr in zip(cases, case_ms, case_rounds)]),
            "phases": phases, "roofline": roof,
-           "e2e": {"value": e2e_ms, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps},
+           "e2e": {"value": e2e_ms, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps,
+                   "calls_per_step": e2e_calls},
            "gpu_launches": launches, "launches_per_step": launches / args.steps, "clocks": clocks,
            "device_status": {"warmup": status, "timed": status2, "e2e": status3, "steps_skipped": skipped}}
     if reps_per_step > 1:

@@ -21,7 +21,7 @@
  * Notation used here (state names of the library): Q is the paper's V
  * (n x r right factor), R is the paper's W (n x r), mu = 1 - beta.
  *
- * Readings where the paper is silent (listed in the design notes as well):
+ * Readings where the paper is silent:
  *   - the QR factor is made unique by requiring diag(R_qr) >= 0;
  *   - ColNorm divides column j by (||column j||_2 + eps), eps passed in;
  *   - the update O uses V_new, the error feedback uses the un-normalised W;
