@@ -21,7 +21,9 @@ using namespace dion;
 
 namespace {
 
-constexpr int MAX_FLAG_SLOTS = 4096;      // step slots of OS_SLOT_INTS ints each
+constexpr int MAX_GRAPHS = 64;             // cached step graphs per context (least recently used goes first)
+constexpr i64 GRAPH_MAX_ELEMS = (i64)2048 * 2048;   // graph replay for matrices up to this many elements (launch-bound steps)
+constexpr int MAX_FLAG_SLOTS = 4096;      // step slots of OS_SLOT_INTS ints each; the last MAX_GRAPHS belong to the cached graphs
 constexpr int MAX_CHAIN = 64;              // matrices of one shape stepped together by dion_step_grouped
 constexpr size_t GROUP_SCRATCH_BYTES = (size_t)16 << 30;  // scratch dion_step_grouped may use for that (or cfg.workspace_bytes)
 constexpr int MAX_ROUNDS = 6;             // adaptive Cholesky QR rounds
@@ -77,6 +79,20 @@ struct dion_ctx {
   cudaStream_t side = nullptr;
   cudaEvent_t side_ev[32] = {};
   int side_cursor = 0;
+  // Graph replay of launch-bound steps: the launch chain of dion_step on a small matrix is captured once per
+  // (descriptor) into a CUDA graph and replayed; the learning rate reaches it through a device scalar.
+  struct GraphEntry {
+    dion_matrix key;
+    cudaGraphExec_t exec;
+    int64_t launches;
+    int index;            // its state slot and scalar
+    uint64_t last_use;
+  };
+  std::vector<GraphEntry> graphs;
+  bool graphs_on = false;
+  cudaStream_t cap = nullptr;       // the stream the chains are captured on (never the caller's: it may be the legacy stream)
+  float* graph_scalars = nullptr;   // MAX_GRAPHS device floats
+  uint64_t graph_clock = 0;
 };
 
 namespace {
@@ -166,10 +182,13 @@ Layout make_layout(const dion_ctx* c, i64 m, i64 n, i64 r) {
   return L;
 }
 
+void graphs_clear(dion_ctx* c);
+
 int ensure_ws(dion_ctx* c, size_t bytes) {
   if (bytes <= c->ws_bytes) return DION_OK;
   if (c->ws != nullptr) {
     if (cudaDeviceSynchronize() != cudaSuccess) return DION_ERR_CUDA;
+    graphs_clear(c);      // they point into the old scratch
     cudaFree(c->ws);
     c->ws = nullptr;
     c->ws_bytes = 0;
@@ -863,17 +882,21 @@ int validate(const dion_matrix* a, bool shard = false) {
   return DION_OK;
 }
 
-int begin_step(dion_ctx* c, const dion_matrix* a, int nb, cudaStream_t st, StepCtx* s) {
+int begin_step(dion_ctx* c, const dion_matrix* a, int nb, cudaStream_t st, StepCtx* s, int fixed_slot = -1) {
   s->c = c;
   s->st = st;
   s->L = make_layout(c, a->m, a->n, a->r);
   s->ws = c->ws;
   s->nb = nb;
   s->wstride = s->L.total;
-  if (c->flag_cursor + nb > MAX_FLAG_SLOTS) c->flag_cursor = 0;   // the slots of a chain are contiguous
-  s->os = c->dev_ints + 8 + (i64)c->flag_cursor * OS_SLOT_INTS;
+  if (fixed_slot >= 0) {
+    s->os = c->dev_ints + 8 + (i64)fixed_slot * OS_SLOT_INTS;
+  } else {
+    if (c->flag_cursor + nb > MAX_FLAG_SLOTS - MAX_GRAPHS) c->flag_cursor = 0;   // the slots of a chain are contiguous
+    s->os = c->dev_ints + 8 + (i64)c->flag_cursor * OS_SLOT_INTS;
+    c->flag_cursor = (c->flag_cursor + nb) % (MAX_FLAG_SLOTS - MAX_GRAPHS);
+  }
   s->flag = s->os + OS_FAIL;
-  c->flag_cursor = (c->flag_cursor + nb) % MAX_FLAG_SLOTS;
   s->tensor = (c->cfg.engine != DION_ENGINE_SIMT);
   s->in_orth = false;
   if (cudaMemsetAsync(s->os, 0, sizeof(int) * OS_SLOT_INTS * nb, st) != cudaSuccess) return DION_ERR_CUDA;
@@ -981,7 +1004,7 @@ int ef_update(StepCtx& s, int b, const dion_matrix* a, const float* F1, i64 ld1,
 }
 
 int x_update(StepCtx& s, int b, const dion_matrix* a, const float* F1, i64 ld1, const float* F2, i64 ld2, float* r1,
-             float* r2, float alpha, const int* skip) {
+             float* r2, float alpha, const int* skip, const float* alpha_dev = nullptr) {
   dion_ctx* c = s.c;
   const i64 m = a->m, n = a->n, r = a->r;
   GemmArgs x = gemm_args();
@@ -1000,16 +1023,20 @@ int x_update(StepCtx& s, int b, const dion_matrix* a, const float* F1, i64 ld1, 
   }
   x.C = (float*)a->X; x.ldc = a->ldx; x.epi = EPI_SUB;
   x.alpha = alpha;
+  x.alpha_dev = alpha_dev;      // graph replay: alpha = 1, the factor comes from the device scalar
   x.skip_flag = skip;
   return launch_gemm(s, x, b);
 }
 
 // The launch chain of one Dion step (Algorithm 1 + 2) on `nb` matrices of identical
 // (m, n, r), phase by phase.  Scratch must hold nb slices.
-int step_batch(dion_ctx* c, const dion_matrix* const* list, int nb, float lr, cudaStream_t st) {
+// x_scale != nullptr (graph capture, nb = 1, fp32 mode): the update's factor lr sqrt(m/n) is read from that device
+// scalar and the step uses state slot `fixed_slot`.
+int step_batch(dion_ctx* c, const dion_matrix* const* list, int nb, float lr, cudaStream_t st,
+               const float* x_scale = nullptr, int fixed_slot = -1) {
   StepCtx s;
   const dion_matrix* a0 = list[0];
-  DION_TRY(begin_step(c, a0, nb, st, &s));
+  DION_TRY(begin_step(c, a0, nb, st, &s, fixed_slot));
   const i64 m = a0->m, n = a0->n, r = a0->r;
   s.list = list;
   if (c->cfg.orth == DION_ORTH_RCQR) {
@@ -1165,7 +1192,7 @@ int step_batch(dion_ctx* c, const dion_matrix* const* list, int nb, float lr, cu
   // X <- X - lr sqrt(m/n) U Q^T   (transposed form: Q U^T)
   {
   PhaseScope ps(c, st, DION_PHASE_X);
-  const float x_alpha = lr * sqrtf((float)((double)m / (double)n));
+  const float x_alpha = (x_scale != nullptr) ? 1.f : lr * sqrtf((float)((double)m / (double)n));
   for (int b = 0; b < nb; ++b) {
     const dion_matrix* a = list[b];
     if (d16) {
@@ -1186,8 +1213,8 @@ int step_batch(dion_ctx* c, const dion_matrix* const* list, int nb, float lr, cu
     float* rbuf = s.W(b, s.L.R);
     const float* Uf = s.W(b, U_off);
     const float* Qf = (const float*)a->Q;
-    if (tr) DION_TRY(x_update(s, b, a, Qf, a->ldq, Uf, r, rbuf, other, x_alpha, s.OS(b) + OS_FAIL));
-    else DION_TRY(x_update(s, b, a, Uf, r, Qf, a->ldq, other, rbuf, x_alpha, s.OS(b) + OS_FAIL));
+    if (tr) DION_TRY(x_update(s, b, a, Qf, a->ldq, Uf, r, rbuf, other, x_alpha, s.OS(b) + OS_FAIL, x_scale));
+    else DION_TRY(x_update(s, b, a, Uf, r, Qf, a->ldq, other, rbuf, x_alpha, s.OS(b) + OS_FAIL, x_scale));
   }
   launch_pdl(k_finish_step, dim3((unsigned)(nb)), dim3(1), 0, st, s.flag, c->dev_ints + 1);
   DION_CHECK_LAUNCH(c);
@@ -1197,6 +1224,77 @@ int step_batch(dion_ctx* c, const dion_matrix* const* list, int nb, float lr, cu
 
 int step_one(dion_ctx* c, const dion_matrix* a, float lr, cudaStream_t st) {
   return step_batch(c, &a, 1, lr, st);
+}
+
+// ---- graph replay of launch-bound steps ----------------------------------------------------------------
+
+__global__ void k_set_scalar(float* dst, float v) { *dst = v; }
+
+void graphs_clear(dion_ctx* c) {
+  for (auto& g : c->graphs) cudaGraphExecDestroy(g.exec);
+  c->graphs.clear();
+}
+
+bool same_matrix(const dion_matrix& x, const dion_matrix& y) {
+  return x.m == y.m && x.n == y.n && x.r == y.r && x.X == y.X && x.ldx == y.ldx && x.M == y.M && x.ldm == y.ldm &&
+         x.G == y.G && x.ldg == y.ldg && x.g_dtype == y.g_dtype && x.Q == y.Q && x.ldq == y.ldq &&
+         x.colnorm_out == y.colnorm_out && x.transposed == y.transposed && x.sketch == y.sketch &&
+         x.sketch_rows == y.sketch_rows && x.ld_sketch == y.ld_sketch;
+}
+
+// A step on a small matrix is a chain of ~30 launches that take longer to issue than to run.  Such steps are
+// captured once (on the context's own stream: the caller's may be the legacy stream, which cannot capture) and
+// replayed as one graph launch into the caller's stream.
+bool graph_eligible(const dion_ctx* c, const dion_matrix* a) {
+  return c->graphs_on && !c->prof_on && c->cfg.precision == DION_PREC_FP32 && c->cfg.engine != DION_ENGINE_SIMT &&
+         a->m * a->n <= GRAPH_MAX_ELEMS && a->r <= NBO_COLS && a->m >= 128 && a->n >= 64 && a->r >= 64 && a->m % 4 == 0 &&
+         a->n % 4 == 0 && a->r % 4 == 0 && !((uintptr_t)a->X & 15) && a->ldx % 4 == 0;     // (the X update must take the tensor engine)
+}
+
+// Returns DION_OK when the step was launched as a graph, 1 when the caller should launch it plainly.
+int step_graph(dion_ctx* c, const dion_matrix* a, float lr, cudaStream_t st) {
+  dion_ctx::GraphEntry* e = nullptr;
+  for (auto& g : c->graphs)
+    if (same_matrix(g.key, *a)) { e = &g; break; }
+  if (e == nullptr) {
+    int index = -1;
+    if ((int)c->graphs.size() < MAX_GRAPHS) {
+      index = (int)c->graphs.size();
+    } else {      // evict the least recently used one (its kernels are ordered before ours only on its own stream: wait)
+      size_t lru = 0;
+      for (size_t i = 1; i < c->graphs.size(); ++i)
+        if (c->graphs[i].last_use < c->graphs[lru].last_use) lru = i;
+      if (cudaDeviceSynchronize() != cudaSuccess) return DION_ERR_CUDA;
+      cudaGraphExecDestroy(c->graphs[lru].exec);
+      index = c->graphs[lru].index;
+      c->graphs.erase(c->graphs.begin() + (long)lru);
+    }
+    const int64_t l0 = c->launches;
+    cudaGraph_t graph = nullptr;
+    if (cudaStreamBeginCapture(c->cap, cudaStreamCaptureModeThreadLocal) != cudaSuccess) { cudaGetLastError(); return 1; }
+    const int rc = step_batch(c, &a, 1, lr, c->cap, c->graph_scalars + index, MAX_FLAG_SLOTS - MAX_GRAPHS + index);
+    const cudaError_t ce = cudaStreamEndCapture(c->cap, &graph);
+    const int64_t nl = c->launches - l0;
+    c->launches = l0;
+    if (rc != DION_OK || ce != cudaSuccess || graph == nullptr) {
+      cudaGetLastError();
+      if (graph != nullptr) cudaGraphDestroy(graph);
+      c->graphs_on = false;      // this chain does not capture here: plain launches from now on
+      return 1;
+    }
+    cudaGraphExec_t exec = nullptr;
+    const cudaError_t ie = cudaGraphInstantiate(&exec, graph, 0);
+    cudaGraphDestroy(graph);
+    if (ie != cudaSuccess || exec == nullptr) { cudaGetLastError(); c->graphs_on = false; return 1; }
+    c->graphs.push_back({*a, exec, nl, index, 0});
+    e = &c->graphs.back();
+  }
+  e->last_use = ++c->graph_clock;
+  k_set_scalar<<<1, 1, 0, st>>>(c->graph_scalars + e->index, lr * sqrtf((float)((double)a->m / (double)a->n)));
+  if (cudaGetLastError() != cudaSuccess) return DION_ERR_CUDA;
+  if (cudaGraphLaunch(e->exec, st) != cudaSuccess) { cudaGetLastError(); return DION_ERR_CUDA; }
+  c->launches += e->launches + 1;
+  return DION_OK;
 }
 
 // One Lazy-Dion step (Algorithm 6).
@@ -1376,6 +1474,19 @@ int dion_init(dion_ctx** out, const dion_config* cfg) {
   if (cudaMemset(p, 0, sizeof(int) * (8 + MAX_FLAG_SLOTS * OS_SLOT_INTS)) != cudaSuccess) { cudaFree(p); delete c; return DION_ERR_CUDA; }
   if (configure_kernels() != DION_OK) { cudaFree(p); delete c; return DION_ERR_CUDA; }
   if (cudaStreamCreateWithFlags(&c->side, cudaStreamNonBlocking) != cudaSuccess) { cudaGetLastError(); c->side = nullptr; }
+  // graph replay of small steps: a capture stream and the scalars the graphs read; off if either cannot be had
+  umma::pair_clusters(c->sm_count);      // (asked once per device, outside any capture)
+  {
+    void* gs = nullptr;
+    if (cudaStreamCreateWithFlags(&c->cap, cudaStreamNonBlocking) == cudaSuccess &&
+        cudaMalloc(&gs, sizeof(float) * MAX_GRAPHS) == cudaSuccess) {
+      c->graph_scalars = (float*)gs;
+      c->graphs_on = true;
+    } else {
+      cudaGetLastError();
+      if (c->cap != nullptr) { cudaStreamDestroy(c->cap); c->cap = nullptr; }
+    }
+  }
   for (int i = 0; i < 32 && c->side != nullptr; ++i)
     if (cudaEventCreateWithFlags(&c->side_ev[i], cudaEventDisableTiming) != cudaSuccess) {
       cudaGetLastError();
@@ -1400,6 +1511,10 @@ int dion_step(dion_ctx* ctx, const dion_matrix* a, float lr, void* cuda_stream) 
   DION_TRY(validate(a));
   if (cudaSetDevice(ctx->cfg.device) != cudaSuccess) return DION_ERR_CUDA;
   DION_TRY(ensure_ws(ctx, dion_workspace_bytes(ctx, a->m, a->n, a->r)));
+  if (graph_eligible(ctx, a)) {
+    const int rc = step_graph(ctx, a, lr, (cudaStream_t)cuda_stream);
+    if (rc <= 0) return rc;
+  }
   return step_one(ctx, a, lr, (cudaStream_t)cuda_stream);
 }
 
@@ -1718,6 +1833,9 @@ void dion_destroy(dion_ctx* ctx) {
   if (ctx == nullptr) return;
   cudaSetDevice(ctx->cfg.device);
   cudaDeviceSynchronize();
+  graphs_clear(ctx);
+  if (ctx->graph_scalars != nullptr) cudaFree(ctx->graph_scalars);
+  if (ctx->cap != nullptr) cudaStreamDestroy(ctx->cap);
   if (ctx->ws != nullptr) cudaFree(ctx->ws);
   if (ctx->dev_ints != nullptr) cudaFree(ctx->dev_ints);
   for (cudaEvent_t e : ctx->prof_pool) cudaEventDestroy(e);

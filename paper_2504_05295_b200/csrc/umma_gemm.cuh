@@ -601,7 +601,7 @@ __global__ void __launch_bounds__(TMA ? NUM_THREADS_TMA : NUM_THREADS, 1) k_gemm
       constexpr int SLABS = (BN / 32) / (C::EPI_WARPS / 4);   // 32-column slabs per warp
       const i64 gi = (i64)it.mi * BM + quad * 32 + lane;
       const i64 n0 = (i64)it.ni * BN;
-      const float alpha = g.alpha;
+      const float alpha = g.alpha * (g.alpha_dev != nullptr ? __ldg(g.alpha_dev) : 1.f);   // (a device scalar under graph replay)
       for (int kb = it.kb0; kb < it.kb1; kb += p.kc, ++iter) {
         const bool first = (kb == it.kb0);
         const int ab = iter % NBUF;
@@ -1327,7 +1327,8 @@ inline int umma_try_launch(const GemmArgs& g_in, int precision, int sm_count, fl
   const bool bf16 = d16 || (precision == DION_PREC_BF16_OPERANDS);
   const int epc = bf16 ? 8 : 4;
   const int sm = d16 ? 8 : 4;        // stride granularity: 16 bytes
-  if (g.batch != 1 || g.alpha_dev != nullptr) return 0;
+  if (g.batch != 1) return 0;
+  if (g.alpha_dev != nullptr && g.epi == EPI_STORE) return 0;   // (the split-K reduction takes a host scalar)
   if (g.M < 128 || g.N < 64 || g.K < 64) return 0;
   if ((g.M % epc) || (g.N % epc) || (g.K % epc)) return 0;
   if (d16 && g.a2_mode != ADD_NONE) return 0;

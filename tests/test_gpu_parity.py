@@ -562,3 +562,49 @@ def test_non_finite_gradient_is_flagged_and_cancels_the_step(m, n, r):
     ref = oracle_steps(pb, 1)
     if r < min(m, n):
         assert rel(to_np64(X), ref[0].X) <= TOL_FP32 and rel(to_np64(Q), ref[0].Q) <= TOL_FP32
+
+
+# ---------------------------------------------------------------------------
+# Graph replay of launch-bound steps: small matrices are stepped by replaying a captured CUDA graph
+# ---------------------------------------------------------------------------
+
+def test_graph_replay_equals_the_plain_launch_chain_and_follows_the_learning_rate():
+    m, n, r = 512, 384, 64
+    pb = inputs.make_problem(m, n, r, seed=44, ks=16)
+    grads = [pb.grad(t).cuda() for t in range(4)]
+    lrs = [0.01, 0.02, 0.005, 0.01]
+    # plain chain: profiling on keeps the library from replaying graphs
+    Xa, Ma, Qa = device_state(pb)
+    with binding.Dion(mu=MU, eps=EPS) as opt:
+        opt.profile_enable(True)
+        G = grads[0].clone()
+        for t in range(4):
+            G.copy_(grads[t])
+            opt.step(Xa, Ma, G, Qa, lrs[t])
+        opt.profile_enable(False)
+        assert opt.get_status() == (0, 0)
+    # replayed: the same descriptor every step (one gradient buffer, refilled), a different learning rate each time
+    Xb, Mb, Qb = device_state(pb)
+    with binding.Dion(mu=MU, eps=EPS) as opt:
+        G = grads[0].clone()
+        n0 = opt.launch_count()
+        for t in range(4):
+            G.copy_(grads[t])
+            opt.step(Xb, Mb, G, Qb, lrs[t])
+        assert opt.get_status() == (0, 0) and opt.launch_count() > n0
+        # a second matrix and a non-default stream go through their own graph
+        side = torch.cuda.Stream()
+        Xc, Mc, Qc = device_state(pb)
+        torch.cuda.synchronize()
+        for t in range(4):
+            G.copy_(grads[t])
+            torch.cuda.synchronize()
+            opt.step(Xc, Mc, G, Qc, lrs[t], stream=side)
+            side.synchronize()
+        assert opt.get_status(side) == (0, 0)
+    for name, u, v, w in zip("XMQ", (Xa, Ma, Qa), (Xb, Mb, Qb), (Xc, Mc, Qc)):
+        assert torch.equal(u, v), f"{name}: graph replay differs from the plain launch chain"
+        assert torch.equal(u, w), f"{name}: graph replay on a side stream differs"
+    ref = oracle_steps(pb, 1)
+    # (the oracle comparison with eta = 0.01 after one step is covered elsewhere; here: finite and moved)
+    assert torch.isfinite(Xb).all() and not torch.equal(Xb, pb.X.cuda())
