@@ -186,7 +186,16 @@ int dion_init(dion_ctx** out, const dion_config* cfg);
 /* One Dion step on one matrix (Algorithm 1 + 2).  `a` is a HOST pointer to a
  * descriptor holding DEVICE pointers.  lr is the paper's eta; sqrt(m/n) is
  * applied inside.  If the orthonormalization breaks down, X, M and Q are left
- * unchanged and DION_STATUS_BREAKDOWN is latched. */
+ * unchanged and DION_STATUS_BREAKDOWN is latched.
+ *
+ * Small matrices (up to 2048 x 2048 elements, r <= 512, fp32 mode on the tensor engine) are launch bound: a
+ * step is a chain of ~30 short kernels.  For these the chain is captured into a CUDA graph the first time a
+ * descriptor is seen (same pointers, shapes and leading dimensions; the capture runs on a stream of the
+ * context, so `cuda_stream` may be the legacy default stream) and later calls with that descriptor replay the
+ * graph on `cuda_stream`; lr reaches it through a device scalar, so it may change from call to call.  Up to 64
+ * graphs are kept per context (least recently used first out); growing the scratch drops them.  The results
+ * are those of the plain launch chain bit for bit.  Steps with per-phase profiling on, grouped, lazy and
+ * multi-call steps are always launched plainly. */
 int dion_step(dion_ctx* ctx, const dion_matrix* a, float lr, void* cuda_stream);
 
 /* The same step on `count` independent matrices (the paper batches matrices of

@@ -38,6 +38,7 @@ constexpr float GOOD_REL = 1e-4f;         // smallest relative pivot of a round 
 constexpr float ORTH_TAU_F = 3e-5f;
 constexpr float DONE_REL = 0.9f;          // smallest relative pivot of a round whose input was already orthonormal
 constexpr i64 PART_CAP_FLOATS = (i64)16 << 20;  // split-K partial sums, at most 64 MiB
+constexpr double P_PAIR_MIN_MNR = 1.5e10;       // smallest m n r whose P = (M + G) Q runs on bf16 operand pairs first
 
 constexpr i64 NBO_COLS = 512;  // = NBO, the outer block of the two-level Cholesky (defined below)
 
@@ -90,6 +91,7 @@ struct dion_ctx {
   };
   std::vector<GraphEntry> graphs;
   bool graphs_on = false;
+  bool chain_batch = true;          // tensor-engine products of a grouped chain in one launch over its matrices
   cudaStream_t cap = nullptr;       // the stream the chains are captured on (never the caller's: it may be the legacy stream)
   float* graph_scalars = nullptr;   // MAX_GRAPHS device floats
   uint64_t graph_clock = 0;
@@ -264,7 +266,7 @@ int launch_gemm_simt(dion_ctx* c, GemmArgs g, cudaStream_t st, float* part, i64 
     const i64 total = g.M * g.N;
     int blocks = (int)((total + 255) / 256);
     if (blocks > 8 * c->sm_count) blocks = 8 * c->sm_count;
-    launch_pdl(k_splitk_reduce, dim3((unsigned)(blocks)), dim3(256), 0, st, part, splits, g.M, g.N, g.C, g.ldc, g.alpha, g.tri, BMN, g.skip_flag);
+    launch_pdl(k_splitk_reduce, dim3((unsigned)(blocks)), dim3(256), 0, st, part, splits, g.M, g.N, g.C, g.ldc, g.alpha, g.tri, BMN, g.skip_flag, (i64)0, (i64)0);
     DION_CHECK_LAUNCH(c);
   }
   return DION_OK;
@@ -313,6 +315,8 @@ struct StepCtx {
   i64 wt_off = -1;        // >= 0: scratch offset of the blocked solves' rows x 512 temporary (default: the R panel)
   bool no_split = false;  // launches on the side stream: the split-K scratch belongs to the main stream
   bool quiet_fail = false;  // a failed pivot only sets the step's fail flag: the fallback kernel follows
+  const std::function<int()>* redo_p = nullptr;   // the panel came from the fast product: recomputes it accurately
+                                                  // (skipped on the device for matrices whose OS_DONE is set)
   float* W(int b, i64 off) const { return ws + (i64)b * wstride + off; }
   int* OS(int b) const { return os + (i64)b * OS_SLOT_INTS; }
 };
@@ -343,6 +347,32 @@ GemmArgs for_matrix(const StepCtx& s, GemmArgs g, int b, bool a_ws, bool b_ws, b
   if (c_ws) g.C += o;
   if (g.skip_flag != nullptr) g.skip_flag += (i64)b * OS_SLOT_INTS;
   return g;
+}
+
+void over_batch(const StepCtx& s, GemmArgs& g);
+
+// One product per matrix of the chain, operands and output in the scratch slices (c2_ws: the second epilogue
+// operand too).  The tensor engine takes all matrices in one launch when the product qualifies (its work list
+// then runs over (matrix, tile) pairs, which also fills the tail of one matrix's tiles with the next one's);
+// otherwise one launch per matrix.
+int launch_gemm_chain(StepCtx& s, const GemmArgs& g, bool c2_ws = false) {
+  if (s.nb > 1 && s.tensor && s.c->chain_batch) {
+    GemmArgs gb = g;
+    over_batch(s, gb);
+    gb.c2_batched = c2_ws ? 1 : 0;
+    PhaseScope ps(s.c, s.st, s.in_orth ? DION_PHASE_ORTH_GEMM : -1);
+    const int prec = s.in_orth ? DION_PREC_FP32 : s.c->cfg.precision;
+    const int rc = umma_try_launch(gb, prec, s.c->sm_count, s.no_split ? nullptr : s.W(0, s.L.part), s.L.part_floats,
+                                   s.c->dev_ints, s.st);
+    if (rc > 0) { s.c->launches += rc; return DION_OK; }
+    if (rc < 0) return rc;
+  }
+  for (int m = 0; m < s.nb; ++m) {
+    GemmArgs gm = for_matrix(s, g, m, true, true, true);
+    if (c2_ws) gm.C2 = (const float*)gm.C2 + (i64)m * s.wstride;
+    DION_TRY(launch_gemm(s, gm, m));
+  }
+  return DION_OK;
 }
 
 // One-time opt-in to the dynamic shared memory of the kernels that need more than 48 KB.
@@ -405,8 +435,8 @@ int trtri_levels(StepCtx& s, i64 r, i64 o, i64 sz, i64 b_from, const int* skip, 
         g2.B = Tbuf + off21 + sh; g2.b_sk = r; g2.b_sn = 1;
         g2.C = Linv + off21 + sh; g2.ldc = r; g2.epi = EPI_STORE; g2.alpha = -1.f; g2.skip_flag = skip; g2.precise = precise;
         if (big) {
-          for (int m = 0; m < s.nb; ++m) DION_TRY(launch_gemm(s, for_matrix(s, g1, m, true, true, true), m));
-          for (int m = 0; m < s.nb; ++m) DION_TRY(launch_gemm(s, for_matrix(s, g2, m, true, true, true), m));
+          DION_TRY(launch_gemm_chain(s, g1));
+          DION_TRY(launch_gemm_chain(s, g2));
         } else {
           g1.batch = batch; g1.bsA = bs; g1.bsB = bs; g1.bsC = bs; over_batch(s, g1);
           g2.batch = batch; g2.bsA = bs; g2.bsB = bs; g2.bsC = bs; over_batch(s, g2);
@@ -426,11 +456,13 @@ enum : int {
   RM_PLAIN = 0,     // no device-side control
   RM_ADAPTIVE = 1,  // deflating pivots, skipped once the panel is done, split-accumulator products, round statistics
   RM_FIRST = 2,     // first round of CholeskyQR2: plain control, split-accumulator products
-  RM_CHECKED = 3    // second round of CholeskyQR2: the first round's result is measured first (orthogonality probe);
+  RM_CHECKED = 3,   // second round of CholeskyQR2: the first round's result is measured first (orthogonality probe);
                     // if it is orthonormal to ORTH_TAU_F the whole round is skipped (Pout = Pin)
+  RM_REDO = 4       // first round once more, on the panel recomputed with the accurate product: skipped on the device
+                    // when the round on the fast panel already passed the probe; split-accumulator products
 };
-inline bool rm_skips(int mode) { return mode == RM_ADAPTIVE || mode == RM_CHECKED; }
-inline bool rm_precise(int mode) { return mode == RM_ADAPTIVE || mode == RM_FIRST; }
+inline bool rm_skips(int mode) { return mode == RM_ADAPTIVE || mode == RM_CHECKED || mode == RM_REDO; }
+inline bool rm_precise(int mode) { return mode == RM_ADAPTIVE || mode == RM_FIRST || mode == RM_REDO; }
 
 int potrf_inner(StepCtx& s, i64 r, i64 o, i64 sz, int mode) {
   const bool adaptive = rm_skips(mode);
@@ -503,7 +535,7 @@ int potrf_trtri(StepCtx& s, i64 r, int mode, bool full_inverse,
       g.A = panel; g.a_si = r; g.a_sk = 1;
       g.B = Linv + J0 * r + J0; g.b_sk = 1; g.b_sn = r; g.klimit = 1;
       g.C = ptmp; g.ldc = r; g.epi = EPI_STORE; g.skip_flag = skip; g.precise = precise;
-      for (int m = 0; m < s.nb; ++m) DION_TRY(launch_gemm(s, for_matrix(s, g, m, true, true, true), m));
+      DION_TRY(launch_gemm_chain(s, g));
       // With the solves on the second stream, the copy of Lpanel into the Gram buffer goes there too: its
       // only readers are the solves of later block columns (queued behind it on that stream); the trailing
       // update reads the temporary, so the copy leaves the serial chain.
@@ -527,10 +559,31 @@ int potrf_trtri(StepCtx& s, i64 r, int mode, bool full_inverse,
       t.B = lp; t.b_sk = 1; t.b_sn = r;
       t.C = Gm + (J0 + sz) * r + (J0 + sz); t.ldc = r; t.epi = EPI_SUB; t.tri = TRI_LOWER; t.skip_flag = skip;
       t.precise = precise;
-      for (int m = 0; m < s.nb; ++m) DION_TRY(launch_gemm(s, for_matrix(s, t, m, true, true, true), m));
+      DION_TRY(launch_gemm_chain(s, t));
     }
   }
   if (r > NBO && full_inverse) DION_TRY(trtri_levels(s, r, 0, r, NBO, skip, precise));
+  return DION_OK;
+}
+
+// The orthogonality probe on the rows x r panels at `off` (two passes over the panel instead of its Gram matrix).
+// phase: PROBE_CHECK the check of CholeskyQR2's first round; PROBE_FAST the same after a round on a panel from the
+// fast product (decides whether the panel is recomputed; counts nothing); PROBE_AFTER_REDO the check that follows a
+// possible recomputation (a panel that passed PROBE_FAST is not measured again).
+int probe(StepCtx& s, i64 off, i64 rows, i64 r, int phase) {
+  dion_ctx* c = s.c;
+  int chunks; i64 per;
+  colnorm_plan(rows, r, c->sm_count, &chunks, &per);
+  const int* keep = (phase == PROBE_AFTER_REDO) ? (const int*)(s.os + OS_DONE) : nullptr;
+  launch_pdl(k_probe_y, dim3((unsigned)grid_for(c, rows * 32), (unsigned)s.nb), dim3(256), 0, s.st, (const float*)(s.ws + off), r,
+             rows, r, s.ws + s.L.probe_y, s.wstride, keep);
+  DION_CHECK_LAUNCH(c);
+  launch_pdl(k_probe_w, dim3((unsigned)((r + 127) / 128), (unsigned)chunks, (unsigned)s.nb), dim3(128), 0, s.st,
+             (const float*)(s.ws + off), r, rows, r, per, (const float*)(s.ws + s.L.probe_y), s.ws + s.L.probe_part, s.wstride, keep);
+  DION_CHECK_LAUNCH(c);
+  launch_pdl(k_probe_decide, dim3((unsigned)s.nb), dim3(256), 0, s.st, (const float*)(s.ws + s.L.probe_part), chunks, r, s.os,
+             ORTH_TAU_F, c->dev_ints + 2, s.wstride, phase);
+  DION_CHECK_LAUNCH(c);
   return DION_OK;
 }
 
@@ -539,7 +592,7 @@ int potrf_trtri(StepCtx& s, i64 r, int mode, bool full_inverse,
 // adaptive: columns with negligible pivots are deflated, the round is skipped (Pout = Pin)
 // once the panel is orthonormal, and the round statistics are evaluated at the end.
 int cholqr_round(StepCtx& s, i64 pin_off, i64 pout_off, i64 rows, i64 r, int mode, i64 gram_rows = 0,
-                 bool passthrough = true) {
+                 bool passthrough = true, int probe_phase = PROBE_CHECK) {
   // passthrough = false: a skipped round leaves Pout untouched (the caller keeps using Pin)
   // gram_rows > 0: the Gram matrix is formed from the first gram_rows rows only (a sketch stacked on
   // top of the panel); the factor is applied to all rows
@@ -548,26 +601,16 @@ int cholqr_round(StepCtx& s, i64 pin_off, i64 pout_off, i64 rows, i64 r, int mod
   const bool skips = rm_skips(mode);
   const int* skip = skips ? (s.os + OS_DONE) : nullptr;
   if (mode == RM_CHECKED) {
-    // CholeskyQR2, second round: first measure the first round's result (two passes over the panel instead of
-    // its Gram matrix); orthonormal enough -> done, and everything below is skipped on the device
-    int chunks; i64 per;
-    colnorm_plan(rows, r, c->sm_count, &chunks, &per);
-    launch_pdl(k_probe_y, dim3((unsigned)grid_for(c, rows * 32), (unsigned)s.nb), dim3(256), 0, s.st, (const float*)(s.ws + pin_off), r,
-               rows, r, s.ws + s.L.probe_y, s.wstride);
-    DION_CHECK_LAUNCH(c);
-    launch_pdl(k_probe_w, dim3((unsigned)((r + 127) / 128), (unsigned)chunks, (unsigned)s.nb), dim3(128), 0, s.st,
-               (const float*)(s.ws + pin_off), r, rows, r, per, (const float*)(s.ws + s.L.probe_y), s.ws + s.L.probe_part, s.wstride);
-    DION_CHECK_LAUNCH(c);
-    launch_pdl(k_probe_decide, dim3((unsigned)s.nb), dim3(256), 0, s.st, (const float*)(s.ws + s.L.probe_part), chunks, r, s.os,
-               ORTH_TAU_F, c->dev_ints + 2, s.wstride);
-    DION_CHECK_LAUNCH(c);
+    // CholeskyQR2, second round: first measure the first round's result; orthonormal enough -> done, and
+    // everything below is skipped on the device
+    DION_TRY(probe(s, pin_off, rows, r, probe_phase));
   }
   GemmArgs g = gemm_args();
   g.M = r; g.N = r; g.K = gram_rows > 0 ? gram_rows : rows;
   g.A = s.ws + pin_off; g.a_si = 1; g.a_sk = r;
   g.B = s.ws + pin_off; g.b_sk = r; g.b_sn = 1;
   g.C = s.ws + s.L.Gram; g.ldc = r; g.epi = EPI_STORE; g.tri = TRI_LOWER; g.skip_flag = skips ? skip : nullptr; g.precise = rm_precise(mode) ? 1 : 0;
-  for (int m = 0; m < s.nb; ++m) DION_TRY(launch_gemm(s, for_matrix(s, g, m, true, true, true), m));
+  DION_TRY(launch_gemm_chain(s, g));
   launch_pdl(k_round_begin, dim3((unsigned)(s.nb)), dim3(256), 0, s.st, s.ws + s.L.Gram, r, r, 0.f, s.ws + s.L.gdiag, s.ws + s.L.scal, s.os,
                                         skips ? 1 : 0, s.wstride, c->dev_ints);
   DION_CHECK_LAUNCH(c);
@@ -600,11 +643,7 @@ int cholqr_round(StepCtx& s, i64 pin_off, i64 pout_off, i64 rows, i64 r, int mod
         w.B = Lm + J0 * r; w.b_sk = 1; w.b_sn = r;
         w.C = Wt; w.ldc = NBO; w.epi = EPI_C2_SUB; w.C2 = rhs; w.ldc2 = r; w.c2_mode = ADD_F32;
         w.skip_flag = skip;
-        for (int m = 0; m < s.nb; ++m) {
-          GemmArgs wm = for_matrix(s, w, m, true, true, true);
-          wm.C2 = (const float*)wm.C2 + (i64)m * s.wstride;
-          DION_TRY(launch_gemm(s, wm, m));
-        }
+        DION_TRY(launch_gemm_chain(s, w, true));
         rhs = Wt; rhs_ld = NBO;
       }
       GemmArgs v = gemm_args();
@@ -612,7 +651,7 @@ int cholqr_round(StepCtx& s, i64 pin_off, i64 pout_off, i64 rows, i64 r, int mod
       v.A = rhs; v.a_si = rhs_ld; v.a_sk = 1;
       v.B = s.ws + s.L.Linv + J0 * r + J0; v.b_sk = 1; v.b_sn = r; v.klimit = 1;
       v.C = s.ws + pout_off + J0; v.ldc = r; v.epi = EPI_STORE; v.skip_flag = skip;
-      for (int m = 0; m < s.nb; ++m) DION_TRY(launch_gemm(s, for_matrix(s, v, m, true, true, true), m));
+      DION_TRY(launch_gemm_chain(s, v));
       return DION_OK;
     };
     if (c->side != nullptr) {
@@ -645,7 +684,7 @@ int cholqr_round(StepCtx& s, i64 pin_off, i64 pout_off, i64 rows, i64 r, int mod
   u.A = s.ws + pin_off; u.a_si = r; u.a_sk = 1;
   u.B = s.ws + s.L.Linv; u.b_sk = 1; u.b_sn = r; u.klimit = 1;
   u.C = s.ws + pout_off; u.ldc = r; u.epi = EPI_STORE; u.skip_flag = skip;
-  for (int m = 0; m < s.nb; ++m) DION_TRY(launch_gemm(s, for_matrix(s, u, m, true, true, true), m));
+  DION_TRY(launch_gemm_chain(s, u));
   if (adaptive) {
     launch_pdl(k_round_end, dim3((unsigned)(s.nb)), dim3(1), 0, s.st, s.os, GOOD_REL, DONE_REL, c->dev_ints + 2);
     DION_CHECK_LAUNCH(c);
@@ -808,7 +847,16 @@ int orthonormalize(StepCtx& s, i64 rows, i64 r, i64 short_dim, i64 pin_off, i64*
     // Round one writes P0, where U is expected; the second round, when it runs, goes P0 -> P1 and is copied
     // back: the common case (one round) moves the panel once.
     int rc = cholqr_round(s, pin_off, s.L.P0, rows, r, RM_FIRST);
-    if (rc == DION_OK) rc = cholqr_round(s, s.L.P0, s.L.P1, rows, r, RM_CHECKED, 0, false);
+    const bool redo = s.redo_p != nullptr;
+    if (redo) {
+      // The panel came from the fast product (bf16 operand pairs, ~1e-5): good enough exactly when the panel is well
+      // conditioned, which the probe of the first round's result shows.  Otherwise the device recomputes the panel
+      // with the accurate product and repeats the round; all of that is launched and skipped in the common case.
+      if (rc == DION_OK) rc = probe(s, s.L.P0, rows, r, PROBE_FAST);
+      if (rc == DION_OK) rc = (*s.redo_p)();
+      if (rc == DION_OK) rc = cholqr_round(s, pin_off, s.L.P0, rows, r, RM_REDO, 0, false);
+    }
+    if (rc == DION_OK) rc = cholqr_round(s, s.L.P0, s.L.P1, rows, r, RM_CHECKED, 0, false, redo ? PROBE_AFTER_REDO : PROBE_CHECK);
     s.quiet_fail = false;
     DION_TRY(rc);
     {
@@ -1074,6 +1122,12 @@ int step_batch(dion_ctx* c, const dion_matrix* const* list, int nb, float lr, cu
   // ... R then runs on bf16 pairs of M + G and of U (three bf16 MMAs per K step: 1.3 TF32 passes instead of 3; the
   // product is accurate to ~1e-5, which is what Q <- ColNorm(R) and the error feedback need of it)
   const bool bpair = b32 && r_on_pairs(s, m, n, r);
+  // ... and so does P where the orthonormalization is CholeskyQR2 and the matrix is large enough for the saving to
+  // exceed the launches that stand by for the accurate product (see orthonormalize).  The rule looks at the matrix
+  // alone, so that a grouped call computes what single calls compute.
+  const bool ppair = bpair && (double)m * (double)n * (double)r >= P_PAIR_MIN_MNR &&
+                     resolve_orth_for(c, r, (m < n) ? m : n, s.list != nullptr) == DION_ORTH_CHOLQR2;
+  bool any_pair = false;
 
   // P = (M + G) Q   (transposed form: (M + G)^T Q)
   const i64 pin_off = panel_offset(s, r, (m < n) ? m : n);
@@ -1095,6 +1149,18 @@ int step_batch(dion_ctx* c, const dion_matrix* const* list, int nb, float lr, cu
       p.ab16 = 1;
       p.A = (const float*)bf(b, s.L.B16); p.a_si = tr ? 1 : n; p.a_sk = tr ? n : 1;
       p.B = (const float*)bf(b, s.L.Q16); p.b_sk = r; p.b_sn = 1;
+    } else if (b32 && ppair && !((uintptr_t)a->Q & 15) && a->ldq % 4 == 0) {
+      DION_TRY(form_sum(s, b, a, true));
+      __nv_bfloat16* qh = reinterpret_cast<__nv_bfloat16*>(s.W(b, s.L.S16));
+      __nv_bfloat16* ql = qh + qrow * r;
+      launch_pdl(k_split_bf16, dim3((unsigned)grid_for(c, qrow * r / 8)), dim3(256), 0, st, (const float*)a->Q, a->ldq, qrow, r, qh, ql,
+                 (const int*)nullptr);
+      DION_CHECK_LAUNCH(c);
+      __nv_bfloat16* bh = reinterpret_cast<__nv_bfloat16*>(s.W(b, s.L.Bp));
+      p.ab16 = 1;
+      p.A = (const float*)bh; p.A16lo = bh + m * n; p.a_si = tr ? 1 : n; p.a_sk = tr ? n : 1;
+      p.B = (const float*)qh; p.B16lo = ql; p.b_sk = r; p.b_sn = 1;
+      any_pair = true;
     } else if (b32) {
       DION_TRY(form_sum(s, b, a, bpair));
       p.A = s.W(b, s.L.B32); p.a_si = tr ? 1 : n; p.a_sk = tr ? n : 1;
@@ -1115,8 +1181,23 @@ int step_batch(dion_ctx* c, const dion_matrix* const* list, int nb, float lr, cu
   i64 U_off = 0;
   {
   PhaseScope ps(c, st, DION_PHASE_ORTH);
+  const std::function<int()> redo = [&]() -> int {
+    for (int b = 0; b < nb; ++b) {
+      const dion_matrix* a = list[b];
+      GemmArgs p = gemm_args();
+      p.M = prow; p.N = r; p.K = qrow;
+      p.A = s.W(b, s.L.B32); p.a_si = tr ? 1 : n; p.a_sk = tr ? n : 1;
+      p.B = (const float*)a->Q; p.b_sk = a->ldq; p.b_sn = 1;
+      p.C = s.W(b, pin_off); p.ldc = r; p.epi = EPI_STORE;
+      p.skip_flag = s.OS(b) + OS_DONE;
+      DION_TRY(launch_gemm(s, p, b));
+    }
+    return DION_OK;
+  };
   s.in_orth = true;
+  s.redo_p = any_pair ? &redo : nullptr;
   const int rc_orth = orthonormalize(s, prow, r, (m < n) ? m : n, pin_off, &U_off);
+  s.redo_p = nullptr;
   s.in_orth = false;
   DION_TRY(rc_orth);
   }
@@ -1988,6 +2069,13 @@ extern "C" int dion_debug_orth_measure(dion_ctx* ctx, void* cuda_stream, float* 
           cudaSuccess ||
       cudaStreamSynchronize(st) != cudaSuccess)
     return DION_ERR_CUDA;
+  return DION_OK;
+}
+
+extern "C" int dion_debug_chain_batch(dion_ctx* ctx, int on) {
+  if (ctx == nullptr) return DION_ERR_INVALID;
+  ctx->chain_batch = on != 0;
+  graphs_clear(ctx);
   return DION_OK;
 }
 

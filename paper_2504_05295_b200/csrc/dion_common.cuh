@@ -40,6 +40,7 @@ struct GemmArgs {
   int batch; i64 bsA, bsB, bsC;  // batch count and element strides
   int batch2; i64 bs2;           // outer batch (one per matrix of a grouped call): stride of A, B, C alike
   i64 skip_stride;               // ints between the skip flags of consecutive outer batch entries
+  int c2_batched;                // C2 is fp32 and moves with the outer batch too (bs2 elements per entry)
   int splits; float* part;       // split-K: partial sums, [splits][M][N]
   int tri;                       // TRI_LOWER: only the elements on or below the diagonal are needed (tiles above it are skipped)
   int klimit;                    // 1: B(k,j) == 0 for k > j  (K loop ends at the tile's last column)

@@ -42,6 +42,10 @@ int dion_debug_gemm(int engine, int precision, const dion_debug_gemm_args* args,
 struct dion_ctx;
 int dion_debug_orth_measure(struct dion_ctx* ctx, void* cuda_stream, float* estimate);
 
+/* on = 0: the tensor-engine products of a grouped call's chain are launched matrix by matrix instead of once
+ * over all matrices of the chain (the results must not depend on it). */
+int dion_debug_chain_batch(struct dion_ctx* ctx, int on);
+
 #ifdef __cplusplus
 }
 #endif

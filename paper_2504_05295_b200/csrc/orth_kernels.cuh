@@ -600,8 +600,9 @@ __device__ __forceinline__ float probe_sign(i64 j, int p) {
 
 // Y[i][p] = sum_j U[i][j] z_p[j]: one warp per row (lanes stride over the columns).  grid = (blocks, matrices).
 __global__ void __launch_bounds__(256) k_probe_y(const float* __restrict__ U, i64 ld, i64 rows, i64 r,
-                                                 float* __restrict__ Y, i64 wstride) {
+                                                 float* __restrict__ Y, i64 wstride, const int* __restrict__ keep) {
   pdl_enter();
+  if (keep != nullptr && keep[(i64)blockIdx.y * OS_SLOT_INTS] != 0) return;   // this panel's verdict stands
   U += (i64)blockIdx.y * wstride; Y += (i64)blockIdx.y * wstride;
   const int lane = threadIdx.x & 31;
   const i64 warp = (i64)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
@@ -631,8 +632,9 @@ __global__ void __launch_bounds__(256) k_probe_y(const float* __restrict__ U, i6
 // part[chunk][j][p] = sum over the chunk's rows of U[i][j] Y[i][p].  grid = (ceil(r/128), chunks, matrices).
 __global__ void __launch_bounds__(128) k_probe_w(const float* __restrict__ U, i64 ld, i64 rows, i64 r,
                                                  i64 rows_per_chunk, const float* __restrict__ Y,
-                                                 float* __restrict__ part, i64 wstride) {
+                                                 float* __restrict__ part, i64 wstride, const int* __restrict__ keep) {
   pdl_enter();
+  if (keep != nullptr && keep[(i64)blockIdx.z * OS_SLOT_INTS] != 0) return;
   U += (i64)blockIdx.z * wstride; Y += (i64)blockIdx.z * wstride; part += (i64)blockIdx.z * wstride;
   const i64 j = (i64)blockIdx.x * 128 + threadIdx.x;
   if (j >= r) return;
@@ -655,13 +657,21 @@ __global__ void __launch_bounds__(128) k_probe_w(const float* __restrict__ U, i6
 
 // One block per matrix: est = sum_p |w_p - z_p|^2 / NPROBE (fixed summation order) into os[OS_MAXDEV] (float
 // bits); est <= tau_f^2 * r  ->  the panel is done (OS_DONE = 1: the rest of the second round is skipped).
-// Counts the rounds of the step that did work (1 or 2).
+// Counts the rounds of the step that did work (1 or 2; with a recomputed panel 2 or 3).
+// phase PROBE_FAST (the round ran on a panel from the fast product): done -> OS_DONE = 1, else 0 (a failed pivot
+// too: the panel is recomputed before the fallback sees it); nothing is counted.  PROBE_AFTER_REDO: a panel that
+// passed PROBE_FAST keeps its verdict (one round); otherwise its recomputed first round is judged.
+enum : int { PROBE_CHECK = 0, PROBE_FAST = 1, PROBE_AFTER_REDO = 2 };
 __global__ void __launch_bounds__(256) k_probe_decide(const float* __restrict__ part, int chunks, i64 r,
                                                       int* __restrict__ os, float tau_f,
-                                                      int* __restrict__ rounds_total, i64 wstride) {
+                                                      int* __restrict__ rounds_total, i64 wstride, int phase) {
   pdl_enter();
   part += (i64)blockIdx.x * wstride;
   os += (i64)blockIdx.x * OS_SLOT_INTS;
+  if (phase == PROBE_AFTER_REDO && os[OS_DONE] != 0) {
+    if (threadIdx.x == 0) { os[OS_ROUNDS] = 1; atomicAdd(rounds_total, 1); }
+    return;
+  }
   __shared__ float red[256];
   float e = 0.f;
   for (i64 j = threadIdx.x; j < r; j += 256) {
@@ -684,9 +694,14 @@ __global__ void __launch_bounds__(256) k_probe_decide(const float* __restrict__ 
     os[OS_MAXDEV] = __float_as_int(est);
     const bool failed = os[OS_FAIL] != 0;       // a pivot of the first round failed: the fallback redoes the panel
     const bool done = !failed && (est <= tau_f * tau_f * (float)r);      // false for NaN
-    os[OS_DONE] = (done || failed) ? 1 : 0;
-    os[OS_ROUNDS] = done ? 1 : 2;
-    atomicAdd(rounds_total, done ? 1 : 2);
+    if (phase == PROBE_FAST) {
+      os[OS_DONE] = done ? 1 : 0;
+    } else {
+      const int extra = (phase == PROBE_AFTER_REDO) ? 1 : 0;
+      os[OS_DONE] = (done || failed) ? 1 : 0;
+      os[OS_ROUNDS] = (done ? 1 : 2) + extra;
+      atomicAdd(rounds_total, (done ? 1 : 2) + extra);
+    }
   }
 }
 

@@ -53,7 +53,8 @@ struct Params {
   int splits;         // K splits (>= 1); partial sums go to g.part when > 1
   int kb_per_split;   // K blocks per split
   int nkb;            // K blocks in all
-  int num_items;      // tiles * splits
+  int num_items;      // tiles * splits * matrices
+  int items_per_matrix;   // tiles * splits; a batched launch (g.batch2 matrices, g.bs2 elements apart) walks matrix by matrix
   int kc;             // K blocks per accumulation chunk (see k_gemm_umma)
   int* status;        // device status word (DION_STATUS_TIMEOUT)
   long long spin_limit;   // cycle budget of every mbarrier wait (SPIN_LIMIT_CYCLES unless a test shortens it)
@@ -89,6 +90,13 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
   asm volatile(
       "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
       "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(bar)
+      : "memory");
+}
+// 3-D tiled TMA load: z is the matrix of a batched launch (the fp32 operand maps are 3-D, extent 1 when not batched)
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int x, int y, int z, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];" ::"r"(dst),
+      "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(z), "r"(bar)
       : "memory");
 }
 __device__ __forceinline__ float4 lds128(uint32_t addr) {
@@ -296,12 +304,15 @@ constexpr i64 TRI_WIDE_MIN = 4096;   // smallest lower-triangular output compute
 
 struct Item {
   int mi, ni, ks, kb0, kb1;
+  int b;      // matrix of a batched launch
 };
 
 // CG2: `mi` counts 256-row tiles of a CTA pair (256 x 256 lower tiles in the triangular case).
 template <int BN, int BKE, bool CG2 = false>
 __device__ __forceinline__ Item decode_item(const Params& p, int item) {
   Item it;
+  it.b = item / p.items_per_matrix;
+  item -= it.b * p.items_per_matrix;
   const int tile = item / p.splits;
   it.ks = item - tile * p.splits;
   if (p.g.tri == TRI_LOWER && BN == 2 * BM && !CG2) {
@@ -542,7 +553,13 @@ __global__ void __launch_bounds__(TMA ? NUM_THREADS_TMA : NUM_THREADS, 1) k_gemm
   const int workers = CG2 ? (int)(gridDim.x >> 1) : (int)gridDim.x;
   constexpr int NBUF = C::NBUF, ACCS = C::ACCS;
   constexpr int BKE = C::BKE, EPC = C::EPC, STAGES = C::STAGES;
-  if (p.g.skip_flag != nullptr && *p.g.skip_flag != 0) return;
+  // a launch over one matrix does nothing when that matrix's flag is set; a batched launch skips flagged matrices
+  // item by item (every role reads the same flags, which no kernel writes while this one runs)
+  const bool batched = p.g.batch2 > 1;
+  if (!batched && p.g.skip_flag != nullptr && *p.g.skip_flag != 0) return;
+  auto skipped = [&](const Item& it) -> bool {
+    return batched && p.g.skip_flag != nullptr && p.g.skip_flag[(i64)it.b * p.g.skip_stride] != 0;
+  };
 
   extern __shared__ unsigned char smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -596,7 +613,12 @@ __global__ void __launch_bounds__(TMA ? NUM_THREADS_TMA : NUM_THREADS, 1) k_gemm
     bool alive = true;
     for (int item = worker; item < p.num_items && alive; item += workers) {
       Item it = decode_item<BN, BKE, CG2>(p, item);
+      if (skipped(it)) continue;
       if (CG2) it.mi = 2 * it.mi + (int)cta_rank;     // this CTA's 128 rows of the pair's tile
+      float* const Cb = g.C + (i64)it.b * g.bs2;                                   // this matrix's output ...
+      float* const partb = g.part + (i64)it.b * g.bs2;                             // ... split-K partial sums ...
+      const void* const C2b = (g.c2_batched && g.C2 != nullptr)                    // ... and second epilogue operand (fp32, in scratch)
+                                  ? (const void*)(reinterpret_cast<const float*>(g.C2) + (i64)it.b * g.bs2) : g.C2;
       const int quad = warp & 3, half = warp >> 2;   // TMEM lane quadrant, column part
       constexpr int SLABS = (BN / 32) / (C::EPI_WARPS / 4);   // 32-column slabs per warp
       const i64 gi = (i64)it.mi * BM + quad * 32 + lane;
@@ -659,16 +681,16 @@ __global__ void __launch_bounds__(TMA ? NUM_THREADS_TMA : NUM_THREADS, 1) k_gemm
             for (int q = 0; q < NI; ++q) {
               const i64 row = (i64)it.mi * BM + quad * 32 + ps * RPP + RPI * q + lane / LPR;
               ok[q] = row < g.M && col < g.N;
-              cptr[q] = to_part ? reinterpret_cast<float4*>(g.part + ((i64)it.ks * g.M + row) * g.N + col)
-                                : reinterpret_cast<float4*>(g.C + row * g.ldc + col);
+              cptr[q] = to_part ? reinterpret_cast<float4*>(partb + ((i64)it.ks * g.M + row) * g.N + col)
+                                : reinterpret_cast<float4*>(Cb + row * g.ldc + col);
               cur[q] = make_float4(0.f, 0.f, 0.f, 0.f);
               c2v[q] = make_float4(0.f, 0.f, 0.f, 0.f);
               if (ok[q] && need_c) cur[q] = *cptr[q];
               if (ok[q] && add_c2) {
                 if (c2_f32) {
-                  c2v[q] = __ldg(reinterpret_cast<const float4*>(reinterpret_cast<const float*>(g.C2) + row * g.ldc2 + col));
+                  c2v[q] = __ldg(reinterpret_cast<const float4*>(reinterpret_cast<const float*>(C2b) + row * g.ldc2 + col));
                 } else {
-                  const uint2 t = __ldg(reinterpret_cast<const uint2*>(reinterpret_cast<const __nv_bfloat16*>(g.C2) + row * g.ldc2 + col));
+                  const uint2 t = __ldg(reinterpret_cast<const uint2*>(reinterpret_cast<const __nv_bfloat16*>(C2b) + row * g.ldc2 + col));
                   const __nv_bfloat162 lo = *reinterpret_cast<const __nv_bfloat162*>(&t.x);
                   const __nv_bfloat162 hi = *reinterpret_cast<const __nv_bfloat162*>(&t.y);
                   c2v[q] = make_float4(__low2float(lo), __high2float(lo), __low2float(hi), __high2float(hi));
@@ -709,8 +731,8 @@ __global__ void __launch_bounds__(TMA ? NUM_THREADS_TMA : NUM_THREADS, 1) k_gemm
             for (int q = 0; q < 8; ++q) {
               const i64 col = n0 + cb * 32 + q * 4;
               ok[q] = col < g.N;
-              cptr[q] = to_part ? reinterpret_cast<float4*>(g.part + ((i64)it.ks * g.M + gi) * g.N + col)
-                                : reinterpret_cast<float4*>(g.C + gi * g.ldc + col);
+              cptr[q] = to_part ? reinterpret_cast<float4*>(partb + ((i64)it.ks * g.M + gi) * g.N + col)
+                                : reinterpret_cast<float4*>(Cb + gi * g.ldc + col);
               cur[q] = make_float4(0.f, 0.f, 0.f, 0.f);
               if (ok[q] && need_c) cur[q] = *cptr[q];
             }
@@ -726,10 +748,10 @@ __global__ void __launch_bounds__(TMA ? NUM_THREADS_TMA : NUM_THREADS, 1) k_gemm
                 if (g.epi != EPI_STORE) sgn = -1.f;
                 if (first && (g.epi == EPI_ADD2_SUB || g.epi == EPI_C2_SUB)) {
                   if (g.c2_mode == ADD_F32 || g.epi == EPI_C2_SUB) {
-                    const float4 t = __ldg(reinterpret_cast<const float4*>(reinterpret_cast<const float*>(g.C2) + gi * g.ldc2 + col));
+                    const float4 t = __ldg(reinterpret_cast<const float4*>(reinterpret_cast<const float*>(C2b) + gi * g.ldc2 + col));
                     c.x += t.x; c.y += t.y; c.z += t.z; c.w += t.w;
                   } else {
-                    const uint2 t = __ldg(reinterpret_cast<const uint2*>(reinterpret_cast<const __nv_bfloat16*>(g.C2) + gi * g.ldc2 + col));
+                    const uint2 t = __ldg(reinterpret_cast<const uint2*>(reinterpret_cast<const __nv_bfloat16*>(C2b) + gi * g.ldc2 + col));
                     const __nv_bfloat162 lo = *reinterpret_cast<const __nv_bfloat162*>(&t.x);
                     const __nv_bfloat162 hi = *reinterpret_cast<const __nv_bfloat162*>(&t.y);
                     c.x += __low2float(lo); c.y += __high2float(lo); c.z += __low2float(hi); c.w += __high2float(hi);
@@ -794,6 +816,7 @@ __global__ void __launch_bounds__(TMA ? NUM_THREADS_TMA : NUM_THREADS, 1) k_gemm
       bool alive = true;
       for (int item = worker; item < p.num_items && alive; item += workers) {
         const Item it = decode_item<BN, BKE, CG2>(p, item);
+        if (skipped(it)) continue;
         for (int kb = it.kb0; kb < it.kb1; ++kb) {
           if (!mbar_wait(raw_bar(stage), phase, dead, p.status, p.spin_limit)) { alive = false; break; }
           const uint32_t sg16 = g16_base + stage * C::G16_BYTES;
@@ -904,6 +927,7 @@ __global__ void __launch_bounds__(TMA ? NUM_THREADS_TMA : NUM_THREADS, 1) k_gemm
       bool alive = true;
       for (int item = worker; item < p.num_items && alive; item += workers) {
         const Item it = decode_item<BN, BKE, CG2>(p, item);
+        if (skipped(it)) continue;
         // CTA pair: this CTA's 128 rows of A and its half of the B tile's columns
         const int row0a = (CG2 ? 2 * it.mi + (int)cta_rank : it.mi) * BM;
         const int row0b = it.ni * BN + (CG2 ? (int)cta_rank * BN_L : 0);
@@ -942,8 +966,8 @@ __global__ void __launch_bounds__(TMA ? NUM_THREADS_TMA : NUM_THREADS, 1) k_gemm
           }
           if (ONE) {   // raw fp32 tiles, [rows][32 k] boxes
             mbar_expect_tx(bar, (uint32_t)(C::A_BYTES + C::B_BYTES));
-            tma_load_2d(sa, &p.tmA, k0, row0a, bar);
-            tma_load_2d(sb, &p.tmB, k0, row0b, bar);
+            tma_load_3d(sa, &p.tmA, k0, row0a, it.b, bar);
+            tma_load_3d(sb, &p.tmB, k0, row0b, it.b, bar);
             if (++stage == STAGES) { stage = 0; phase ^= 1u; }
             continue;
           }
@@ -968,20 +992,20 @@ __global__ void __launch_bounds__(TMA ? NUM_THREADS_TMA : NUM_THREADS, 1) k_gemm
             else tma_load_2d(g16_base + stage * C::G16_BYTES, &p.tmA2, row0a, k0, bar);
           }
           if (!A_MN) {
-            tma_load_2d(sa, &p.tmA, k0, row0a, bar);
-            if (add) tma_load_2d(sa_lo, &p.tmA2, k0, row0a, bar);
+            tma_load_3d(sa, &p.tmA, k0, row0a, it.b, bar);
+            if (add) tma_load_3d(sa_lo, &p.tmA2, k0, row0a, it.b, bar);
           } else {
 #pragma unroll
             for (int c = 0; c < BM / 32; ++c) {
-              tma_load_2d(sa + c * (BKE * 128), &p.tmA, row0a + 32 * c, k0, bar);
-              if (add) tma_load_2d(sa_lo + c * (BKE * 128), &p.tmA2, row0a + 32 * c, k0, bar);
+              tma_load_3d(sa + c * (BKE * 128), &p.tmA, row0a + 32 * c, k0, it.b, bar);
+              if (add) tma_load_3d(sa_lo + c * (BKE * 128), &p.tmA2, row0a + 32 * c, k0, it.b, bar);
             }
           }
           if (!B_MN) {
-            tma_load_2d(sb, &p.tmB, k0, row0b, bar);
+            tma_load_3d(sb, &p.tmB, k0, row0b, it.b, bar);
           } else {
 #pragma unroll
-            for (int c = 0; c < BN_L / 32; ++c) tma_load_2d(sb + c * (BKE * 128), &p.tmB, row0b + 32 * c, k0, bar);
+            for (int c = 0; c < BN_L / 32; ++c) tma_load_3d(sb + c * (BKE * 128), &p.tmB, row0b + 32 * c, k0, it.b, bar);
           }
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
@@ -1001,6 +1025,7 @@ __global__ void __launch_bounds__(TMA ? NUM_THREADS_TMA : NUM_THREADS, 1) k_gemm
       bool alive = true;
       for (int item = worker; item < p.num_items && alive; item += workers) {
         const Item it = decode_item<BN, BKE, CG2>(p, item);
+        if (skipped(it)) continue;
         for (int kbc = it.kb0; kbc < it.kb1 && alive; kbc += p.kc, ++iter) {   // one accumulation chunk
         const int kbc1 = min(it.kb1, kbc + p.kc);
         const int ab = iter % NBUF;
@@ -1243,11 +1268,14 @@ inline bool make_operand16_map(CUtensorMap* map, const void* ptr, i64 rows, i64 
   return r == CUDA_SUCCESS;
 }
 
-inline bool make_operand_map(CUtensorMap* map, const void* ptr, i64 rows, i64 K, i64 ld, bool mn_major, int box_rows) {
+// The maps of fp32 operands are 3-D: the third coordinate is the matrix of a batched launch (`nbatch` matrices,
+// `bstride` elements apart; extent 1 otherwise).
+inline bool make_operand_map(CUtensorMap* map, const void* ptr, i64 rows, i64 K, i64 ld, bool mn_major, int box_rows,
+                             i64 nbatch = 1, i64 bstride = 0) {
   EncodeTiledFn fn = encode_tiled_fn();
   if (fn == nullptr) return false;
-  cuuint64_t gdim[2], gstride[1];
-  cuuint32_t box[2], estr[2] = {1, 1};
+  cuuint64_t gdim[3], gstride[2];
+  cuuint32_t box[3], estr[3] = {1, 1, 1};
   if (!mn_major) {
     gdim[0] = (cuuint64_t)K; gdim[1] = (cuuint64_t)rows;
     box[0] = 32; box[1] = (cuuint32_t)box_rows;
@@ -1255,8 +1283,12 @@ inline bool make_operand_map(CUtensorMap* map, const void* ptr, i64 rows, i64 K,
     gdim[0] = (cuuint64_t)rows; gdim[1] = (cuuint64_t)K;
     box[0] = 32; box[1] = 32;
   }
+  gdim[2] = (cuuint64_t)(nbatch > 1 ? nbatch : 1);
+  box[2] = 1;
   gstride[0] = (cuuint64_t)ld * sizeof(float);
-  const CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void*>(ptr), gdim, gstride, box, estr,
+  gstride[1] = (nbatch > 1) ? (cuuint64_t)bstride * sizeof(float) : gstride[0] * gdim[1];
+  if (gstride[1] % 16 != 0) return false;
+  const CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<void*>(ptr), gdim, gstride, box, estr,
                         CU_TENSOR_MAP_INTERLEAVE_NONE,
                         mn_major ? CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B : CU_TENSOR_MAP_SWIZZLE_128B,
                         CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
@@ -1328,6 +1360,11 @@ inline int umma_try_launch(const GemmArgs& g_in, int precision, int sm_count, fl
   const int epc = bf16 ? 8 : 4;
   const int sm = d16 ? 8 : 4;        // stride granularity: 16 bytes
   if (g.batch != 1) return 0;
+  // one launch over the matrices of a chain (same shape; operands, output and split-K scratch g.bs2 elements
+  // apart): fp32 operands through 3-D tensor maps only.  Tiles and K splits are chosen exactly as for one matrix,
+  // so every element is computed by the same sequence of operations as in a launch of its own.
+  const int nbat = g.batch2 > 1 ? g.batch2 : 1;
+  if (nbat > 1 && (d16 || bf16 || g.a2_mode == ADD_BF16 || (variant & UMMA_VARIANT_REGISTER_LOADS) || (g.bs2 % 4))) return 0;
   if (g.alpha_dev != nullptr && g.epi == EPI_STORE) return 0;   // (the split-K reduction takes a host scalar)
   if (g.M < 128 || g.N < 64 || g.K < 64) return 0;
   if ((g.M % epc) || (g.N % epc) || (g.K % epc)) return 0;
@@ -1381,11 +1418,12 @@ inline int umma_try_launch(const GemmArgs& g_in, int precision, int sm_count, fl
   }
   if (tma && !d16) {
     const i64 lda = a_mn ? g.a_sk : g.a_si, ldb = b_mn ? g.b_sk : g.b_sn;
-    tma = make_operand_map(&p.tmA, g.A, g.M, g.K, lda, a_mn, BM) &&
-          make_operand_map(&p.tmB, g.B, g.N, g.K, ldb, b_mn, cg2 ? BN / 2 : BN);
+    tma = make_operand_map(&p.tmA, g.A, g.M, g.K, lda, a_mn, BM, nbat, g.bs2) &&
+          make_operand_map(&p.tmB, g.B, g.N, g.K, ldb, b_mn, cg2 ? BN / 2 : BN, nbat, g.bs2);
     if (tma && g.a2_mode == ADD_F32)
-      tma = make_operand_map(&p.tmA2, g.A2, g.M, g.K, a_mn ? g.a2_sk : g.a2_si, a_mn, BM);
+      tma = make_operand_map(&p.tmA2, g.A2, g.M, g.K, a_mn ? g.a2_sk : g.a2_si, a_mn, BM, nbat, g.bs2);
   }
+  if (nbat > 1 && !tma) return 0;
   const int bke = (bf16 && (!tma || d16)) ? 64 : 32;
   if (cg2 && !tma) {   // no tensor maps: the register path knows no pairs; redo the tile choice without them
     GemmArgs g2 = g_in;
@@ -1412,8 +1450,9 @@ inline int umma_try_launch(const GemmArgs& g_in, int precision, int sm_count, fl
   splits = (p.nkb + p.kb_per_split - 1) / p.kb_per_split;   // no empty split
   p.splits = splits;
   p.g.part = part;
-  if (tiles * splits > 0x7fffffff) return 0;
-  p.num_items = (int)(tiles * splits);
+  if (tiles * splits * nbat > 0x7fffffff) return 0;
+  p.items_per_matrix = (int)(tiles * splits);
+  p.num_items = p.items_per_matrix * nbat;
   p.status = status;
   const bool withhold = (variant & UMMA_VARIANT_WITHHOLD) && !tma;
   p.spin_limit = withhold ? 2000000LL : SPIN_LIMIT_CYCLES;
@@ -1472,7 +1511,8 @@ inline int umma_try_launch(const GemmArgs& g_in, int precision, int sm_count, fl
     const i64 total = g.M * g.N;
     int blocks = (int)((total + 255) / 256);
     if (blocks > 8 * sm_count) blocks = 8 * sm_count;
-    k_splitk_reduce<<<blocks, 256, 0, st>>>(part, splits, g.M, g.N, g.C, g.ldc, g.alpha, g.tri, 128, g.skip_flag);
+    k_splitk_reduce<<<dim3((unsigned)blocks, (unsigned)nbat), 256, 0, st>>>(part, splits, g.M, g.N, g.C, g.ldc, g.alpha, g.tri, 128, g.skip_flag,
+                                                                            nbat > 1 ? g.bs2 : 0, nbat > 1 ? g.skip_stride : 0);
     if (cudaGetLastError() != cudaSuccess) return DION_ERR_CUDA;
     return 2;
   }

@@ -188,6 +188,34 @@ def test_grouped_equals_single_calls():
         assert rel(to_np64(X2), ref[1].X) <= TOL_FP32 and rel(to_np64(Q2), ref[1].Q) <= TOL_FP32
 
 
+@pytest.mark.parametrize("shape,count", [((1024, 4096, 256), 5), ((4096, 4096, 1024), 3), ((2560, 1536, 640), 3),
+                                         ((1280, 1280, 1280), 2), ((1400, 1100, 700), 3), ((512, 2048, 512), 4)])
+def test_chain_products_in_one_launch_equal_one_launch_per_matrix(shape, count):
+    # the tensor-engine products of a grouped chain run as one launch over (matrix, tile) pairs; with the test hook
+    # that turns this off they run matrix by matrix: same bits, fewer launches
+    import ctypes
+    m, n, r = shape
+    pbs = [inputs.make_problem(m, n, r, seed=41, k=k, ks=32) for k in range(count)]
+    lib = binding.load_library()
+    lib.dion_debug_chain_batch.argtypes = [ctypes.c_void_p, ctypes.c_int]
+    lib.dion_debug_chain_batch.restype = ctypes.c_int
+    results, launches = [], []
+    for on in (1, 0):
+        with binding.Dion(mu=MU, eps=EPS) as opt:
+            assert lib.dion_debug_chain_batch(opt._ctx, on) == 0
+            states = [device_state(pb) for pb in pbs]
+            for t in range(2):
+                l0 = opt.launch_count()
+                opt.step_grouped([(X, M, pb.grad(t).cuda(), Q) for pb, (X, M, Q) in zip(pbs, states)], ETA)
+            launches.append(opt.launch_count() - l0)
+            assert opt.get_status() == (0, 0)
+        results.append(states)
+    for k, ((X1, M1, Q1), (X2, M2, Q2)) in enumerate(zip(*results)):
+        assert torch.equal(X1, X2) and torch.equal(M1, M2) and torch.equal(Q1, Q2), k
+    print(f"{shape} x {count}: {launches[0]} launches batched, {launches[1]} per matrix")
+    assert launches[0] < launches[1]
+
+
 @pytest.mark.parametrize("shape,orth", [((2560, 1536, 640), binding.ORTH_AUTO), ((1280, 1280, 1280), binding.ORTH_AUTO),
                                         # ragged: a second square of 188 columns (blocks of 64, 64, 60)
                                         ((1400, 1100, 700), binding.ORTH_AUTO), ((3000, 2900, 700), binding.ORTH_AUTO)])
@@ -487,6 +515,42 @@ def test_grouped_llama_like_block_list_against_oracle():
 def _nearly_parallel(Q, delta):
     Qb = Q[:, :1] + delta * Q
     return (Qb / Qb.norm(dim=0)).contiguous()
+
+
+def test_fast_panel_is_recomputed_when_the_probe_rejects_it():
+    # 4096^2 at r = 1024 is large enough for P = (M + G) Q to run on bf16 operand pairs first (~1e-5).
+    # (i) the workload's own warm start: well conditioned, the probe accepts the first round, one round of work,
+    # the 1e-4 bar holds; (ii) a warm start with nearly parallel columns (cond(P) in the hundreds): the probe
+    # rejects the round, the device recomputes P with the accurate product and repeats it (three rounds of work
+    # counted), and the outputs meet the same conditioned bar as everywhere else; (iii) a grouped call mixing both
+    # equals the single calls bit for bit
+    from oracle import dion_oracle as orc
+    m = n = 4096
+    r = 1024
+    pb = inputs.make_problem(m, n, r, seed=51, ks=64)
+    G = pb.grad(0)
+    Qbad = _nearly_parallel(pb.Q, 0.03)
+    outs = []
+    with binding.Dion(mu=MU, eps=EPS) as opt:
+        for q0, rounds in ((pb.Q, 1), (Qbad, 3)):
+            X, M, Q = pb.X.cuda().clone(), pb.M.cuda().clone(), q0.cuda().clone()
+            opt.step(X, M, G.cuda(), Q, ETA)
+            assert opt.get_status() == (0, 0) and opt.fallbacks() == 0
+            assert opt.orth_rounds() == rounds
+            want = orc.step(to_np64(pb.X), to_np64(pb.M), to_np64(G), to_np64(q0), MU, ETA, EPS)
+            tol = movement_tol(one_step_movement(to_np64(pb.X), to_np64(pb.M), to_np64(G), to_np64(q0)))
+            errs = {"X": rel(to_np64(X), want.X), "M": rel(to_np64(M), want.M), "Q": rel(to_np64(Q), want.Q)}
+            print(f"rounds {rounds}: " + " ".join(f"{k} {v:.2e}/{tol[k]:.1e}" for k, v in errs.items()))
+            assert all(errs[k] <= tol[k] for k in errs)
+            if rounds == 1:
+                assert errs["Q"] <= TOL_FP32
+            outs.append((X, M, Q))
+        grouped = [(pb.X.cuda().clone(), pb.M.cuda().clone(), q0.cuda().clone()) for q0 in (pb.Q, Qbad)]
+        opt.step_grouped([(X, M, G.cuda(), Q) for X, M, Q in grouped], ETA)
+        assert opt.get_status() == (0, 0)
+    for a, b in zip(outs, grouped):
+        for u, v in zip(a, b):
+            assert torch.equal(u, v)
 
 
 def test_cholesky_breakdown_falls_back_on_the_device():
