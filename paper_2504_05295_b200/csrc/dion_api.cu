@@ -375,6 +375,57 @@ int launch_gemm_chain(StepCtx& s, const GemmArgs& g, bool c2_ws = false) {
   return DION_OK;
 }
 
+// The same product on every matrix of the chain, given as one GemmArgs per matrix (as the per-matrix launch would
+// take them).  When the tensor engine can run them as ONE launch -- identical shapes and strides, operands in the
+// scratch slices (so that one 3-D tensor map covers them), outputs anywhere (a pointer table) -- it does: the work
+// list then runs over (matrix, tile) pairs and the last wave of one matrix is filled with the next one's tiles.
+// Every element is computed by the same sequence of operations either way.
+int launch_gemm_group(StepCtx& s, const std::vector<GemmArgs>& v) {
+  const int nb = (int)v.size();
+  bool one = nb > 1 && nb <= GEMM_TAB_MAX && s.tensor && s.c->chain_batch;
+  const GemmArgs& a = v[0];
+  bool c_strided = true, c2_strided = true;
+  const i64 wb = s.wstride * 4;   // bytes between scratch slices
+  auto at_stride = [&](const void* p0, const void* pb, int b) {
+    return (p0 == nullptr && pb == nullptr) ||
+           (p0 != nullptr && pb != nullptr && (const char*)pb - (const char*)p0 == (ptrdiff_t)((i64)b * wb));
+  };
+  for (int b = 1; b < nb && one; ++b) {
+    const GemmArgs& g = v[b];
+    one = g.M == a.M && g.N == a.N && g.K == a.K && g.a_si == a.a_si && g.a_sk == a.a_sk && g.a2_si == a.a2_si &&
+          g.a2_sk == a.a2_sk && g.a2_mode == a.a2_mode && g.b_sk == a.b_sk && g.b_sn == a.b_sn && g.ldc == a.ldc &&
+          g.epi == a.epi && g.ldc2 == a.ldc2 && g.c2_mode == a.c2_mode && g.alpha == a.alpha && g.alpha_dev == a.alpha_dev &&
+          g.batch == 1 && a.batch == 1 && g.tri == a.tri && g.klimit == a.klimit && g.precise == a.precise &&
+          g.ab16 == a.ab16 && g.tf32x1 == a.tf32x1 && at_stride(a.A, g.A, b) && at_stride(a.B, g.B, b) &&
+          at_stride(a.A2, g.A2, b) && at_stride(a.A16lo, g.A16lo, b) && at_stride(a.B16lo, g.B16lo, b) &&
+          ((a.skip_flag == nullptr && g.skip_flag == nullptr) ||
+           (a.skip_flag != nullptr && g.skip_flag == a.skip_flag + (i64)b * OS_SLOT_INTS));
+    c_strided = c_strided && at_stride(a.C, g.C, b);
+    c2_strided = c2_strided && at_stride(a.C2, g.C2, b);
+  }
+  if (one && !c_strided && a.epi == EPI_STORE) one = false;   // (a plain store may split K: its reduction wants one stride)
+  if (one) {
+    GemmArgs gb = a;
+    over_batch(s, gb);
+    float* ctab[GEMM_TAB_MAX];
+    const void* c2tab[GEMM_TAB_MAX];
+    for (int b = 0; b < nb; ++b) { ctab[b] = v[b].C; c2tab[b] = v[b].C2; }
+    if (!c_strided) gb.c_tab = ctab;
+    if (a.C2 != nullptr) {
+      if (c2_strided && a.c2_mode == ADD_F32) gb.c2_batched = 1;
+      else gb.c2_tab = c2tab;
+    }
+    PhaseScope ps(s.c, s.st, s.in_orth ? DION_PHASE_ORTH_GEMM : -1);
+    const int prec = s.in_orth ? DION_PREC_FP32 : s.c->cfg.precision;
+    const int rc = umma_try_launch(gb, prec, s.c->sm_count, s.no_split ? nullptr : s.W(0, s.L.part), s.L.part_floats,
+                                   s.c->dev_ints, s.st);
+    if (rc > 0) { s.c->launches += rc; return DION_OK; }
+    if (rc < 0) return rc;
+  }
+  for (int b = 0; b < nb; ++b) DION_TRY(launch_gemm(s, v[b], b));
+  return DION_OK;
+}
+
 // One-time opt-in to the dynamic shared memory of the kernels that need more than 48 KB.
 int configure_kernels() {
   if (umma_configure() != DION_OK) return DION_ERR_CUDA;
@@ -976,7 +1027,8 @@ int form_sum(StepCtx& s, int b, const dion_matrix* a, bool pair) {
 }
 
 // The product itself: U (prow x r, dense) is split into the panel buffer `upair`; the pair of M + G must be in place.
-int r_pairs(StepCtx& s, int b, const dion_matrix* a, bool tr, const float* U, float* upair, float* out, const int* skip) {
+int r_pairs(StepCtx& s, int b, const dion_matrix* a, bool tr, const float* U, float* upair, float* out, const int* skip,
+            GemmArgs* defer = nullptr) {   // defer: the product is handed back instead of launched
   dion_ctx* c = s.c;
   const i64 m = a->m, n = a->n, r = a->r;
   const i64 prow = tr ? n : m, qrow = tr ? m : n;
@@ -992,6 +1044,7 @@ int r_pairs(StepCtx& s, int b, const dion_matrix* a, bool tr, const float* U, fl
   w.B = (const float*)uh; w.B16lo = ul; w.b_sk = r; w.b_sn = 1;
   w.C = out; w.ldc = r; w.epi = EPI_STORE;
   w.skip_flag = skip;
+  if (defer != nullptr) { *defer = w; return DION_OK; }
   return launch_gemm(s, w, b);
 }
 
@@ -1014,7 +1067,8 @@ bool x_single_pass(const StepCtx& s, const dion_matrix* a, const float* F1, i64 
 // sum32 != nullptr: M + G comes from scratch (C = sum32 - beta acc); else C = M + G - beta acc with the caller's G.
 // ready1 / ready2: that factor's pair already sits in p1 / p2 (the step splits U for R).
 int ef_update(StepCtx& s, int b, const dion_matrix* a, const float* F1, i64 ld1, const float* F2, i64 ld2, float* p1,
-              float* p2, const float* sum32, const int* skip, bool ready1 = false, bool ready2 = false) {
+              float* p2, const float* sum32, const int* skip, bool ready1 = false, bool ready2 = false,
+              GemmArgs* defer = nullptr) {
   dion_ctx* c = s.c;
   const i64 m = a->m, n = a->n, r = a->r;
   GemmArgs e = gemm_args();
@@ -1048,11 +1102,12 @@ int ef_update(StepCtx& s, int b, const dion_matrix* a, const float* F1, i64 ld1,
   else { e.epi = EPI_ADD2_SUB; e.C2 = a->G; e.ldc2 = a->ldg; e.c2_mode = (a->g_dtype == DION_BF16) ? ADD_BF16 : ADD_F32; }
   e.alpha = 1.f - c->cfg.mu;
   e.skip_flag = skip;
+  if (defer != nullptr) { *defer = e; return DION_OK; }
   return launch_gemm(s, e, b);
 }
 
 int x_update(StepCtx& s, int b, const dion_matrix* a, const float* F1, i64 ld1, const float* F2, i64 ld2, float* r1,
-             float* r2, float alpha, const int* skip, const float* alpha_dev = nullptr) {
+             float* r2, float alpha, const int* skip, const float* alpha_dev = nullptr, GemmArgs* defer = nullptr) {
   dion_ctx* c = s.c;
   const i64 m = a->m, n = a->n, r = a->r;
   GemmArgs x = gemm_args();
@@ -1073,6 +1128,7 @@ int x_update(StepCtx& s, int b, const dion_matrix* a, const float* F1, i64 ld1, 
   x.alpha = alpha;
   x.alpha_dev = alpha_dev;      // graph replay: alpha = 1, the factor comes from the device scalar
   x.skip_flag = skip;
+  if (defer != nullptr) { *defer = x; return DION_OK; }
   return launch_gemm(s, x, b);
 }
 
@@ -1129,6 +1185,9 @@ int step_batch(dion_ctx* c, const dion_matrix* const* list, int nb, float lr, cu
                      resolve_orth_for(c, r, (m < n) ? m : n, s.list != nullptr) == DION_ORTH_CHOLQR2;
   bool any_pair = false;
 
+  // the large products: one GemmArgs per matrix, then one launch over the chain where that is possible
+  std::vector<GemmArgs> group((size_t)nb);
+
   // P = (M + G) Q   (transposed form: (M + G)^T Q)
   const i64 pin_off = panel_offset(s, r, (m < n) ? m : n);
   {
@@ -1173,8 +1232,9 @@ int step_batch(dion_ctx* c, const dion_matrix* const* list, int nb, float lr, cu
     p.C = s.W(b, pin_off); p.ldc = r; p.epi = EPI_STORE;
     // an ill-conditioned panel amplifies the error of P: use the accurate product there
     p.precise = (!d16 && resolve_orth(c, r, (m < n) ? m : n) == DION_ORTH_SHIFTED3) ? 1 : 0;
-    DION_TRY(launch_gemm(s, p, b));
+    group[b] = p;
   }
+  DION_TRY(launch_gemm_group(s, group));
   }
 
   // U = Orthonormalize(P)
@@ -1216,7 +1276,8 @@ int step_batch(dion_ctx* c, const dion_matrix* const* list, int nb, float lr, cu
       w.B = (const float*)bf(b, s.L.U16); w.b_sk = r; w.b_sn = 1;
     } else if (bpair) {
       // U as a bf16 pair in the other panel buffer (the error feedback reuses it)
-      DION_TRY(r_pairs(s, b, a, tr, s.W(b, U_off), s.W(b, U_off == s.L.P0 ? s.L.P1 : s.L.P0), s.W(b, s.L.R), s.OS(b) + OS_FAIL));
+      DION_TRY(r_pairs(s, b, a, tr, s.W(b, U_off), s.W(b, U_off == s.L.P0 ? s.L.P1 : s.L.P0), s.W(b, s.L.R), s.OS(b) + OS_FAIL,
+                       &group[b]));
       continue;
     } else if (b32) {
       w.A = s.W(b, s.L.B32); w.a_si = tr ? n : 1; w.a_sk = tr ? 1 : n;
@@ -1227,8 +1288,9 @@ int step_batch(dion_ctx* c, const dion_matrix* const* list, int nb, float lr, cu
       w.B = s.W(b, U_off); w.b_sk = r; w.b_sn = 1;
     }
     w.C = s.W(b, s.L.R); w.ldc = r; w.epi = EPI_STORE;
-    DION_TRY(launch_gemm(s, w, b));
+    group[b] = w;
   }
+  DION_TRY(launch_gemm_group(s, group));
   }
 
   // M <- (M + G) - (1 - mu) U R^T   (transposed form: R U^T)
@@ -1247,7 +1309,7 @@ int step_batch(dion_ctx* c, const dion_matrix* const* list, int nb, float lr, cu
       e.epi = EPI_ADD2_SUB; e.C2 = a->G; e.ldc2 = a->ldg; e.c2_mode = g_mode(a);
       e.alpha = 1.f - c->cfg.mu;
       e.skip_flag = s.OS(b) + OS_FAIL;
-      DION_TRY(launch_gemm(s, e, b));
+      group[b] = e;
       continue;
     }
     // the bf16 pairs of the two factors go to the other panel buffer and to their own buffer
@@ -1256,9 +1318,10 @@ int step_batch(dion_ctx* c, const dion_matrix* const* list, int nb, float lr, cu
     const float* Uf = s.W(b, U_off);
     const float* Rf = s.W(b, s.L.R);
     const float* sum32 = b32 ? s.W(b, s.L.B32) : nullptr;
-    if (tr) DION_TRY(ef_update(s, b, a, Rf, r, Uf, r, sbuf, other, sum32, s.OS(b) + OS_FAIL, false, bpair));
-    else DION_TRY(ef_update(s, b, a, Uf, r, Rf, r, other, sbuf, sum32, s.OS(b) + OS_FAIL, bpair, false));
+    if (tr) DION_TRY(ef_update(s, b, a, Rf, r, Uf, r, sbuf, other, sum32, s.OS(b) + OS_FAIL, false, bpair, &group[b]));
+    else DION_TRY(ef_update(s, b, a, Uf, r, Rf, r, other, sbuf, sum32, s.OS(b) + OS_FAIL, bpair, false, &group[b]));
   }
+  DION_TRY(launch_gemm_group(s, group));
   }
 
   // Q <- ColNorm(R)
@@ -1286,7 +1349,7 @@ int step_batch(dion_ctx* c, const dion_matrix* const* list, int nb, float lr, cu
       x.C = (float*)a->X; x.ldc = a->ldx; x.epi = EPI_SUB;
       x.alpha = x_alpha;
       x.skip_flag = s.OS(b) + OS_FAIL;
-      DION_TRY(launch_gemm(s, x, b));
+      group[b] = x;
       continue;
     }
     // the rounded copies of the single-pass form go to the other panel buffer and to R's, both free by now
@@ -1294,9 +1357,10 @@ int step_batch(dion_ctx* c, const dion_matrix* const* list, int nb, float lr, cu
     float* rbuf = s.W(b, s.L.R);
     const float* Uf = s.W(b, U_off);
     const float* Qf = (const float*)a->Q;
-    if (tr) DION_TRY(x_update(s, b, a, Qf, a->ldq, Uf, r, rbuf, other, x_alpha, s.OS(b) + OS_FAIL, x_scale));
-    else DION_TRY(x_update(s, b, a, Uf, r, Qf, a->ldq, other, rbuf, x_alpha, s.OS(b) + OS_FAIL, x_scale));
+    if (tr) DION_TRY(x_update(s, b, a, Qf, a->ldq, Uf, r, rbuf, other, x_alpha, s.OS(b) + OS_FAIL, x_scale, &group[b]));
+    else DION_TRY(x_update(s, b, a, Uf, r, Qf, a->ldq, other, rbuf, x_alpha, s.OS(b) + OS_FAIL, x_scale, &group[b]));
   }
+  DION_TRY(launch_gemm_group(s, group));
   launch_pdl(k_finish_step, dim3((unsigned)(nb)), dim3(1), 0, st, s.flag, c->dev_ints + 1);
   DION_CHECK_LAUNCH(c);
   }

@@ -27,6 +27,8 @@ enum : int { TRI_FULL = 0, TRI_LOWER = 1 };
 // A(i,k) = A[i*a_si + k*a_sk] (+ A2(i,k) of dtype a2_mode with its own strides)
 // B(k,j) = B[k*b_sk + j*b_sn]
 // C(i,j) = C[i*ldc + j]
+constexpr int GEMM_TAB_MAX = 64;   // most matrices in one batched tensor-engine launch with per-matrix output pointers
+
 struct GemmArgs {
   i64 M, N, K;
   const float* A; i64 a_si, a_sk;
@@ -41,6 +43,8 @@ struct GemmArgs {
   int batch2; i64 bs2;           // outer batch (one per matrix of a grouped call): stride of A, B, C alike
   i64 skip_stride;               // ints between the skip flags of consecutive outer batch entries
   int c2_batched;                // C2 is fp32 and moves with the outer batch too (bs2 elements per entry)
+  float* const* c_tab;           // tensor engine, outer batch: HOST arrays of batch2 (<= GEMM_TAB_MAX) pointers, the C (and C2) of
+  const void* const* c2_tab;     // every entry (the caller's arrays, at no common stride); copied into the launch parameters
   int splits; float* part;       // split-K: partial sums, [splits][M][N]
   int tri;                       // TRI_LOWER: only the elements on or below the diagonal are needed (tiles above it are skipped)
   int klimit;                    // 1: B(k,j) == 0 for k > j  (K loop ends at the tile's last column)

@@ -60,6 +60,9 @@ struct Params {
   long long spin_limit;   // cycle budget of every mbarrier wait (SPIN_LIMIT_CYCLES unless a test shortens it)
   int withhold_arrive;    // test hook of the register-path variant: the producer warps do not arrive for the first
                           // K block, so that the consumer's bounded wait runs out (no copy is in flight then)
+  // batched launch whose outputs are the caller's arrays (g.c_tab / g.c2_tab given): per-matrix C and C2
+  float* ctab[GEMM_TAB_MAX];
+  const void* c2tab[GEMM_TAB_MAX];
 };
 
 // ------------------------------------------------------------------ PTX wrappers
@@ -615,9 +618,10 @@ __global__ void __launch_bounds__(TMA ? NUM_THREADS_TMA : NUM_THREADS, 1) k_gemm
       Item it = decode_item<BN, BKE, CG2>(p, item);
       if (skipped(it)) continue;
       if (CG2) it.mi = 2 * it.mi + (int)cta_rank;     // this CTA's 128 rows of the pair's tile
-      float* const Cb = g.C + (i64)it.b * g.bs2;                                   // this matrix's output ...
+      float* const Cb = (g.c_tab != nullptr) ? p.ctab[it.b] : g.C + (i64)it.b * g.bs2;   // this matrix's output ...
       float* const partb = g.part + (i64)it.b * g.bs2;                             // ... split-K partial sums ...
-      const void* const C2b = (g.c2_batched && g.C2 != nullptr)                    // ... and second epilogue operand (fp32, in scratch)
+      const void* const C2b = (g.c2_tab != nullptr) ? p.c2tab[it.b]                // ... and second epilogue operand
+                              : (g.c2_batched && g.C2 != nullptr)                  //     (fp32, in scratch)
                                   ? (const void*)(reinterpret_cast<const float*>(g.C2) + (i64)it.b * g.bs2) : g.C2;
       const int quad = warp & 3, half = warp >> 2;   // TMEM lane quadrant, column part
       constexpr int SLABS = (BN / 32) / (C::EPI_WARPS / 4);   // 32-column slabs per warp
@@ -942,23 +946,23 @@ __global__ void __launch_bounds__(TMA ? NUM_THREADS_TMA : NUM_THREADS, 1) k_gemm
             mbar_expect_tx(bar, (uint32_t)(2 * (C::A_BYTES + C::B_BYTES)));
             const uint32_t sb_lo2 = sb + C::B_BYTES;
             if (!A_MN) {
-              tma_load_2d(sa, &p.tmA, k0, row0a, bar);
-              tma_load_2d(sa_lo, &p.tmA2, k0, row0a, bar);
+              tma_load_3d(sa, &p.tmA, k0, row0a, it.b, bar);
+              tma_load_3d(sa_lo, &p.tmA2, k0, row0a, it.b, bar);
             } else {
 #pragma unroll
               for (int c = 0; c < BM / 64; ++c) {
-                tma_load_2d(sa + c * (BKE * 128), &p.tmA, row0a + 64 * c, k0, bar);
-                tma_load_2d(sa_lo + c * (BKE * 128), &p.tmA2, row0a + 64 * c, k0, bar);
+                tma_load_3d(sa + c * (BKE * 128), &p.tmA, row0a + 64 * c, k0, it.b, bar);
+                tma_load_3d(sa_lo + c * (BKE * 128), &p.tmA2, row0a + 64 * c, k0, it.b, bar);
               }
             }
             if (!B_MN) {
-              tma_load_2d(sb, &p.tmB, k0, row0b, bar);
-              tma_load_2d(sb_lo2, &p.tmB2, k0, row0b, bar);
+              tma_load_3d(sb, &p.tmB, k0, row0b, it.b, bar);
+              tma_load_3d(sb_lo2, &p.tmB2, k0, row0b, it.b, bar);
             } else {
 #pragma unroll
               for (int c = 0; c < BN / 64; ++c) {
-                tma_load_2d(sb + c * (BKE * 128), &p.tmB, row0b + 64 * c, k0, bar);
-                tma_load_2d(sb_lo2 + c * (BKE * 128), &p.tmB2, row0b + 64 * c, k0, bar);
+                tma_load_3d(sb + c * (BKE * 128), &p.tmB, row0b + 64 * c, k0, it.b, bar);
+                tma_load_3d(sb_lo2 + c * (BKE * 128), &p.tmB2, row0b + 64 * c, k0, it.b, bar);
               }
             }
             if (++stage == STAGES) { stage = 0; phase ^= 1u; }
@@ -973,15 +977,15 @@ __global__ void __launch_bounds__(TMA ? NUM_THREADS_TMA : NUM_THREADS, 1) k_gemm
           }
           if (D16) {   // bf16 tiles: [rows][64 k] boxes, or [64 k][64 rows] boxes per 64-row chunk
             mbar_expect_tx(bar, (uint32_t)(C::A_BYTES + C::B_BYTES));
-            if (!A_MN) tma_load_2d(sa, &p.tmA, k0, row0a, bar);
+            if (!A_MN) tma_load_3d(sa, &p.tmA, k0, row0a, it.b, bar);
             else {
 #pragma unroll
-              for (int c = 0; c < BM / 64; ++c) tma_load_2d(sa + c * (BKE * 128), &p.tmA, row0a + 64 * c, k0, bar);
+              for (int c = 0; c < BM / 64; ++c) tma_load_3d(sa + c * (BKE * 128), &p.tmA, row0a + 64 * c, k0, it.b, bar);
             }
-            if (!B_MN) tma_load_2d(sb, &p.tmB, k0, row0b, bar);
+            if (!B_MN) tma_load_3d(sb, &p.tmB, k0, row0b, it.b, bar);
             else {
 #pragma unroll
-              for (int c = 0; c < BN / 64; ++c) tma_load_2d(sb + c * (BKE * 128), &p.tmB, row0b + 64 * c, k0, bar);
+              for (int c = 0; c < BN / 64; ++c) tma_load_3d(sb + c * (BKE * 128), &p.tmB, row0b + 64 * c, k0, it.b, bar);
             }
             if (++stage == STAGES) { stage = 0; phase ^= 1u; }
             continue;
@@ -1254,15 +1258,21 @@ inline bool make_addend16_map(CUtensorMap* map, const void* ptr, i64 rows, i64 K
 
 // Tensor map of a bf16 operand: box = 64 k x box_rows rows (k contiguous) or 64 rows x 64 k
 // (row index contiguous), 128-byte swizzle: exactly the tile the bf16 MMA reads.
-inline bool make_operand16_map(CUtensorMap* map, const void* ptr, i64 rows, i64 K, i64 ld, bool mn_major, int box_rows) {
+// (3-D like the fp32 operand maps; `bstride_bytes` between the matrices of a batched launch)
+inline bool make_operand16_map(CUtensorMap* map, const void* ptr, i64 rows, i64 K, i64 ld, bool mn_major, int box_rows,
+                               i64 nbatch = 1, i64 bstride_bytes = 0) {
   EncodeTiledFn fn = encode_tiled_fn();
   if (fn == nullptr) return false;
-  cuuint64_t gdim[2], gstride[1];
-  cuuint32_t box[2], estr[2] = {1, 1};
+  cuuint64_t gdim[3], gstride[2];
+  cuuint32_t box[3], estr[3] = {1, 1, 1};
   if (!mn_major) { gdim[0] = (cuuint64_t)K; gdim[1] = (cuuint64_t)rows; box[0] = 64; box[1] = (cuuint32_t)box_rows; }
   else { gdim[0] = (cuuint64_t)rows; gdim[1] = (cuuint64_t)K; box[0] = 64; box[1] = 64; }
+  gdim[2] = (cuuint64_t)(nbatch > 1 ? nbatch : 1);
+  box[2] = 1;
   gstride[0] = (cuuint64_t)ld * 2;
-  const CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), gdim, gstride, box, estr,
+  gstride[1] = (nbatch > 1) ? (cuuint64_t)bstride_bytes : gstride[0] * gdim[1];
+  if (gstride[1] % 16 != 0) return false;
+  const CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), gdim, gstride, box, estr,
                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS;
@@ -1360,11 +1370,13 @@ inline int umma_try_launch(const GemmArgs& g_in, int precision, int sm_count, fl
   const int epc = bf16 ? 8 : 4;
   const int sm = d16 ? 8 : 4;        // stride granularity: 16 bytes
   if (g.batch != 1) return 0;
-  // one launch over the matrices of a chain (same shape; operands, output and split-K scratch g.bs2 elements
-  // apart): fp32 operands through 3-D tensor maps only.  Tiles and K splits are chosen exactly as for one matrix,
+  // one launch over the matrices of a chain (same shape; operands, output and split-K scratch g.bs2 4-byte words
+  // apart): operands through 3-D tensor maps only.  Tiles and K splits are chosen exactly as for one matrix,
   // so every element is computed by the same sequence of operations as in a launch of its own.
   const int nbat = g.batch2 > 1 ? g.batch2 : 1;
-  if (nbat > 1 && (d16 || bf16 || g.a2_mode == ADD_BF16 || (variant & UMMA_VARIANT_REGISTER_LOADS) || (g.bs2 % 4))) return 0;
+  if (nbat > 1 && (g.a2_mode == ADD_BF16 || (variant & UMMA_VARIANT_REGISTER_LOADS) || (g.bs2 % 4))) return 0;
+  if ((g.c_tab != nullptr || g.c2_tab != nullptr) && (nbat < 2 || nbat > GEMM_TAB_MAX)) return 0;
+  if (g.c_tab != nullptr && g.epi == EPI_STORE) return 0;   // (a plain store may split K: its reduction wants one stride)
   if (g.alpha_dev != nullptr && g.epi == EPI_STORE) return 0;   // (the split-K reduction takes a host scalar)
   if (g.M < 128 || g.N < 64 || g.K < 64) return 0;
   if ((g.M % epc) || (g.N % epc) || (g.K % epc)) return 0;
@@ -1378,12 +1390,19 @@ inline int umma_try_launch(const GemmArgs& g_in, int precision, int sm_count, fl
   else if (g.b_sn == 1 && g.b_sk % sm == 0) b_mn = true;
   else return 0;
   if (!aligned(g.A, 16) || !aligned(g.B, 16) || !aligned(g.C, 16) || (g.ldc % 4)) return 0;
+  if (g.c_tab != nullptr)
+    for (int b = 0; b < nbat; ++b)
+      if (!aligned(g.c_tab[b], 16)) return 0;
   if (g.a2_mode != ADD_NONE) {
     if (a_mn ? (g.a2_si != 1 || g.a2_sk % 4) : (g.a2_sk != 1 || g.a2_si % 4)) return 0;
     if (!aligned(g.A2, g.a2_mode == ADD_BF16 ? 8 : 16)) return 0;
   }
   if (g.epi == EPI_ADD2_SUB || g.epi == EPI_C2_SUB) {
-    if ((g.ldc2 % 4) || !aligned(g.C2, (g.epi == EPI_ADD2_SUB && g.c2_mode == ADD_BF16) ? 8 : 16)) return 0;
+    const size_t al2 = (g.epi == EPI_ADD2_SUB && g.c2_mode == ADD_BF16) ? 8 : 16;
+    if ((g.ldc2 % 4) || !aligned(g.C2, al2)) return 0;
+    if (g.c2_tab != nullptr)
+      for (int b = 0; b < nbat; ++b)
+        if (!aligned(g.c2_tab[b], al2)) return 0;
   }
   if (g.tri == TRI_LOWER && g.M != g.N) return 0;
 
@@ -1398,17 +1417,20 @@ inline int umma_try_launch(const GemmArgs& g_in, int precision, int sm_count, fl
   const int BN = ((g.tri == TRI_LOWER && !tri_wide && !cg2) || g.N < 256) ? 128 : 256;
   Params p;
   p.g = g;
+  if (g.c_tab != nullptr) for (int b = 0; b < nbat; ++b) p.ctab[b] = g.c_tab[b];
+  if (g.c2_tab != nullptr) for (int b = 0; b < nbat; ++b) p.c2tab[b] = g.c2_tab[b];
   // TMA variant: fp32 operands in memory (both precision modes), dimensions the tensor maps can describe
   bool tma = (d16 || !(variant & UMMA_VARIANT_REGISTER_LOADS)) && g.M < (1ll << 31) && g.N < (1ll << 31) && g.K < (1ll << 31);
   const bool x2 = d16 && g.A16lo != nullptr && g.B16lo != nullptr;   // bf16 operand pairs
   if (x2 && (!aligned(g.A16lo, 16) || !aligned(g.B16lo, 16))) return 0;
   if (d16) {
     const i64 lda = a_mn ? g.a_sk : g.a_si, ldb = b_mn ? g.b_sk : g.b_sn;
-    if (!tma || !make_operand16_map(&p.tmA, g.A, g.M, g.K, lda, a_mn, BM) ||
-        !make_operand16_map(&p.tmB, g.B, g.N, g.K, ldb, b_mn, BN))
+    const i64 bsb = g.bs2 * 4;   // the batch stride counts 4-byte words for every operand type
+    if (!tma || !make_operand16_map(&p.tmA, g.A, g.M, g.K, lda, a_mn, BM, nbat, bsb) ||
+        !make_operand16_map(&p.tmB, g.B, g.N, g.K, ldb, b_mn, BN, nbat, bsb))
       return 0;
-    if (x2 && (!make_operand16_map(&p.tmA2, g.A16lo, g.M, g.K, lda, a_mn, BM) ||
-               !make_operand16_map(&p.tmB2, g.B16lo, g.N, g.K, ldb, b_mn, BN)))
+    if (x2 && (!make_operand16_map(&p.tmA2, g.A16lo, g.M, g.K, lda, a_mn, BM, nbat, bsb) ||
+               !make_operand16_map(&p.tmB2, g.B16lo, g.N, g.K, ldb, b_mn, BN, nbat, bsb)))
       return 0;
   } else
   if (tma && g.a2_mode == ADD_BF16) {   // the bf16 addend needs 16-byte aligned rows for its tensor map
