@@ -222,6 +222,20 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float* v) {
 #pragma unroll
   for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
+// 16 columns of the lane's row
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float* v) {
+  uint32_t r[16];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr)
+      : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+  for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ uint32_t cvt_tf32(float x) {
   uint32_t r;
@@ -632,8 +646,6 @@ __global__ void __launch_bounds__(TMA ? NUM_THREADS_TMA : NUM_THREADS, 1) k_gemm
         const bool first = (kb == it.kb0);
         const int ab = iter % NBUF;
         const uint32_t ph = (uint32_t)(iter / NBUF) & 1u;
-        if (!mbar_wait(accf_bar(ab), ph, dead, p.status, p.spin_limit, 256)) { alive = false; break; }
-        tc_fence_after();
         if constexpr (CE) {
           // Coalesced epilogue.  A TMEM lane is a row, so a warp that wrote its accumulator rows straight
           // out would touch 32 rows per global access.  Instead the warp handles its 32 rows x W columns
@@ -649,6 +661,7 @@ __global__ void __launch_bounds__(TMA ? NUM_THREADS_TMA : NUM_THREADS, 1) k_gemm
           constexpr int RPI = 32 / LPR;       // rows per instruction
           constexpr int NI = RPP / RPI;       // instructions per pass (8)
           constexpr int TS = W + 4;           // tile row stride (floats)
+          constexpr int NP = 32 / RPP;        // passes
           static_assert(W == 32 * SLABS && NI == 8, "pass geometry");
           float* tb = epi_tiles + warp * C::EPI_TILE_FLOATS;
           const bool to_part = p.splits > 1;
@@ -658,60 +671,114 @@ __global__ void __launch_bounds__(TMA ? NUM_THREADS_TMA : NUM_THREADS, 1) k_gemm
           const i64 col = n0 + half * W + 4 * (lane % LPR);
           float f = 1.f;
           if (!to_part) f = (g.epi != EPI_STORE) ? -alpha : alpha;
-#pragma unroll 1
-          for (int ps = 0; ps < 32 / RPP; ++ps) {
+          // rows of pass ps that this lane touches: row0 + ps * RPP + RPI * q
+          const i64 row0 = (i64)it.mi * BM + quad * 32 + lane / LPR;
+          auto out_ptr = [&](i64 row) -> float4* {
+            return to_part ? reinterpret_cast<float4*>(partb + ((i64)it.ks * g.M + row) * g.N + col)
+                           : reinterpret_cast<float4*>(Cb + row * g.ldc + col);
+          };
+          auto c2_load = [&](i64 row) -> float4 {
+            if (c2_f32) return __ldg(reinterpret_cast<const float4*>(reinterpret_cast<const float*>(C2b) + row * g.ldc2 + col));
+            const uint2 t = __ldg(reinterpret_cast<const uint2*>(reinterpret_cast<const __nv_bfloat16*>(C2b) + row * g.ldc2 + col));
+            const __nv_bfloat162 lo = *reinterpret_cast<const __nv_bfloat162*>(&t.x);
+            const __nv_bfloat162 hi = *reinterpret_cast<const __nv_bfloat162*>(&t.y);
+            return make_float4(__low2float(lo), __high2float(lo), __low2float(hi), __high2float(hi));
+          };
+          // What the accumulator is added to (the running C, the second operand, or both) does not depend on the
+          // MMAs: the loads of a pass are issued before its rows are read from TMEM and staged (those of the first
+          // pass before the wait for the accumulator) and meet them only in `combine`, so that their latency is
+          // covered by that work.
+          auto fetch = [&](int ps, float4 (&buf)[NI]) {
 #pragma unroll
-            for (int sl = 0; sl < SLABS; ++sl) {
-              float acc[32];
-              tmem_ld32(tmem_base + (uint32_t)(ab * ACCS * BN + half * W + sl * 32) + ((uint32_t)(quad * 32) << 16), acc);
+            for (int q = 0; q < NI; ++q) {
+              const i64 row = row0 + ps * RPP + RPI * q;
+              float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+              if (row < g.M && col < g.N) {
+                if (need_c && add_c2) {
+                  const float4 c = *out_ptr(row);
+                  const float4 t = c2_load(row);
+                  v = make_float4(c.x + t.x, c.y + t.y, c.z + t.z, c.w + t.w);
+                } else if (need_c) {
+                  v = *out_ptr(row);
+                } else if (add_c2) {
+                  v = c2_load(row);
+                }
+              }
+              buf[q] = v;
+            }
+          };
+          auto stage_rows = [&](int ps) {     // rows ps * RPP .. of the warp's 32, from TMEM into the warp's tile
+            // 16 columns at a time where the loads in flight need the registers (8 epilogue warps: wide passes)
+            constexpr int LDW = (C::EPI_WARPS > 8) ? 32 : 16;
+#pragma unroll
+            for (int sl = 0; sl < W / LDW; ++sl) {
+              float acc[LDW];
+              const uint32_t ta = tmem_base + (uint32_t)(ab * ACCS * BN + half * W + sl * LDW) + ((uint32_t)(quad * 32) << 16);
+              if constexpr (LDW == 32) tmem_ld32(ta, acc);
+              else tmem_ld16(ta, acc);
               if (SPLIT) {
-                float small[32];
-                tmem_ld32(tmem_base + (uint32_t)(ab * ACCS * BN + BN + half * W + sl * 32) + ((uint32_t)(quad * 32) << 16), small);
+                float small[LDW];
+                if constexpr (LDW == 32) tmem_ld32(ta + (uint32_t)BN, small);
+                else tmem_ld16(ta + (uint32_t)BN, small);
 #pragma unroll
-                for (int e = 0; e < 32; ++e) acc[e] += small[e];
+                for (int e = 0; e < LDW; ++e) acc[e] += small[e];
               }
               if (lane / RPP == ps) {
 #pragma unroll
-                for (int q = 0; q < 8; ++q)
-                  *reinterpret_cast<float4*>(tb + (lane % RPP) * TS + sl * 32 + 4 * q) =
+                for (int q = 0; q < LDW / 4; ++q)
+                  *reinterpret_cast<float4*>(tb + (lane % RPP) * TS + sl * LDW + 4 * q) =
                       make_float4(acc[4 * q], acc[4 * q + 1], acc[4 * q + 2], acc[4 * q + 3]);
               }
             }
-            __syncwarp();
-            float4* cptr[NI];
-            float4 cur[NI], c2v[NI];
-            bool ok[NI];
+          };
+          auto combine = [&](int ps, const float4 (&buf)[NI]) {
 #pragma unroll
             for (int q = 0; q < NI; ++q) {
-              const i64 row = (i64)it.mi * BM + quad * 32 + ps * RPP + RPI * q + lane / LPR;
-              ok[q] = row < g.M && col < g.N;
-              cptr[q] = to_part ? reinterpret_cast<float4*>(partb + ((i64)it.ks * g.M + row) * g.N + col)
-                                : reinterpret_cast<float4*>(Cb + row * g.ldc + col);
-              cur[q] = make_float4(0.f, 0.f, 0.f, 0.f);
-              c2v[q] = make_float4(0.f, 0.f, 0.f, 0.f);
-              if (ok[q] && need_c) cur[q] = *cptr[q];
-              if (ok[q] && add_c2) {
-                if (c2_f32) {
-                  c2v[q] = __ldg(reinterpret_cast<const float4*>(reinterpret_cast<const float*>(C2b) + row * g.ldc2 + col));
-                } else {
-                  const uint2 t = __ldg(reinterpret_cast<const uint2*>(reinterpret_cast<const __nv_bfloat16*>(C2b) + row * g.ldc2 + col));
-                  const __nv_bfloat162 lo = *reinterpret_cast<const __nv_bfloat162*>(&t.x);
-                  const __nv_bfloat162 hi = *reinterpret_cast<const __nv_bfloat162*>(&t.y);
-                  c2v[q] = make_float4(__low2float(lo), __high2float(lo), __low2float(hi), __high2float(hi));
-                }
-              }
-            }
-#pragma unroll
-            for (int q = 0; q < NI; ++q) {
-              if (!ok[q]) continue;
+              const i64 row = row0 + ps * RPP + RPI * q;
+              if (!(row < g.M && col < g.N)) continue;
               const float4 a4 = *reinterpret_cast<const float4*>(tb + (RPI * q + lane / LPR) * TS + 4 * (lane % LPR));
-              float4 c = cur[q];
-              c.x += c2v[q].x; c.y += c2v[q].y; c.z += c2v[q].z; c.w += c2v[q].w;
-              *cptr[q] = make_float4(fmaf(f, a4.x, c.x), fmaf(f, a4.y, c.y), fmaf(f, a4.z, c.z), fmaf(f, a4.w, c.w));
+              const float4 c = buf[q];
+              *out_ptr(row) = make_float4(fmaf(f, a4.x, c.x), fmaf(f, a4.y, c.y), fmaf(f, a4.z, c.z), fmaf(f, a4.w, c.w));
             }
-            __syncwarp();      // the tile is rewritten by the next pass
+          };
+          auto release = [&]() {     // the accumulator has been read: the next tile's MMAs may overwrite it
+            tc_fence_before();
+            if (CG2 && cta_rank != 0) mbar_arrive_remote(acce_bar(ab), 0u);
+            else mbar_arrive(acce_bar(ab));
+          };
+          if constexpr (SPLIT) {
+            // two accumulators to read per slab: no registers to spare for loads in flight across the staging
+            if (!mbar_wait(accf_bar(ab), ph, dead, p.status, p.spin_limit, 256)) { alive = false; break; }
+            tc_fence_after();
+            float4 b0[NI];
+#pragma unroll 1
+            for (int ps = 0; ps < NP; ++ps) {
+              stage_rows(ps);
+              __syncwarp();
+              if (ps + 1 == NP) release();
+              fetch(ps, b0);
+              combine(ps, b0);
+              __syncwarp();      // the tile is rewritten by the next pass
+            }
+          } else {
+            float4 b0[NI];
+            fetch(0, b0);
+            if (!mbar_wait(accf_bar(ab), ph, dead, p.status, p.spin_limit, 256)) { alive = false; break; }
+            tc_fence_after();
+#pragma unroll 1
+            for (int ps = 0; ps < NP; ++ps) {
+              stage_rows(ps);
+              __syncwarp();
+              if (ps + 1 == NP) release();
+              combine(ps, b0);
+              __syncwarp();      // the tile is rewritten by the next pass
+              if (ps + 1 < NP) fetch(ps + 1, b0);
+            }
           }
-        } else
+          continue;
+        }
+        if (!mbar_wait(accf_bar(ab), ph, dead, p.status, p.spin_limit, 256)) { alive = false; break; }
+        tc_fence_after();
 #pragma unroll 1
         for (int sj = 0; sj < SLABS; ++sj) {
           // slab sj of the warps of one row quadrant lie side by side, so that the quadrant reads and
