@@ -523,6 +523,11 @@ struct Cfg {
   // D16: the producer warps have no conversion work and serve as epilogue warps too
   // (with operand pairs the stages leave room for 8 warps' epilogue tiles only)
   static constexpr int EPI_WARPS = ((D16 && !X2) || ONE) ? NUM_EPI_WARPS + NUM_PROD_WARPS : NUM_EPI_WARPS;
+  // Operand pairs: nothing to convert and no room for more epilogue tiles, so the kernel runs without the producer
+  // warps (10 warps in all); the registers they would hold go to the epilogue warps' loads in flight (DEEP).
+  static constexpr bool DEEP = X2;
+  static constexpr int MMA_WARP = X2 ? NUM_EPI_WARPS : NUM_EPI_WARPS + NUM_PROD_WARPS;   // the warp that issues the MMAs
+  static constexpr int THREADS = (MMA_WARP + (TMA ? 2 : 1)) * 32;                         // ... then the TMA warp
   // CE (coalesced epilogue): an epilogue warp owns 32 rows x EPI_W columns of the tile and passes them
   // through a private shared-memory tile in passes of EPI_RPP rows (EPI_RPP * EPI_W = 1024 elements),
   // so that one global access of the warp covers whole row segments instead of 32 rows; paid for with
@@ -555,7 +560,8 @@ struct Cfg {
 // row-contiguous: 128-byte rows of 64 row indices, 128-byte swizzle); one MMA per K step.
 template <int BN, bool A_MN, bool B_MN, bool BF16, bool SPLIT, bool TMA, bool D16 = false, bool CE = false, bool ONE = false,
           bool CG2 = false, bool X2 = false>
-__global__ void __launch_bounds__(TMA ? NUM_THREADS_TMA : NUM_THREADS, 1) k_gemm_umma(const __grid_constant__ Params p) {
+__global__ void __launch_bounds__((Cfg<BN, BF16, SPLIT, TMA, D16, CE, ONE, CG2, X2>::THREADS), 1)
+k_gemm_umma(const __grid_constant__ Params p) {
   static_assert(!X2 || (D16 && CE), "operand pairs are bf16 arrays");
   static_assert(!CG2 || (TMA && !BF16 && !D16 && !ONE && BN == 256), "CTA pairs: the fp32 TMA variants with 256-column tiles");
   static_assert(!(BF16 && SPLIT), "split accumulators belong to the 3xTF32 mode");
@@ -607,7 +613,7 @@ __global__ void __launch_bounds__(TMA ? NUM_THREADS_TMA : NUM_THREADS, 1) k_gemm
     *dead = 0;
     fence_barrier_init();
   }
-  if (warp == NUM_EPI_WARPS + NUM_PROD_WARPS) {
+  if (warp == C::MMA_WARP) {
     if (CG2) { tmem_alloc2(smem_u32((const void*)tmem_slot), C::TMEM_COLS); tmem_relinquish2(); }
     else { tmem_alloc(smem_u32((const void*)tmem_slot), C::TMEM_COLS); tmem_relinquish(); }
   }
@@ -760,6 +766,43 @@ __global__ void __launch_bounds__(TMA ? NUM_THREADS_TMA : NUM_THREADS, 1) k_gemm
               combine(ps, b0);
               __syncwarp();      // the tile is rewritten by the next pass
             }
+          } else if constexpr (C::DEEP) {
+            // registers to spare: C and the second operand wait in registers of their own (no arithmetic, hence
+            // no wait, at issue time)
+            auto fetch2 = [&](int ps, float4 (&bc)[NI], float4 (&bt)[NI]) {
+#pragma unroll
+              for (int q = 0; q < NI; ++q) {
+                const i64 row = row0 + ps * RPP + RPI * q;
+                const bool ok = row < g.M && col < g.N;
+                bc[q] = make_float4(0.f, 0.f, 0.f, 0.f);
+                bt[q] = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (ok && need_c) bc[q] = *out_ptr(row);
+                if (ok && add_c2) bt[q] = c2_load(row);
+              }
+            };
+            auto combine2 = [&](int ps, const float4 (&bc)[NI], const float4 (&bt)[NI]) {
+#pragma unroll
+              for (int q = 0; q < NI; ++q) {
+                const i64 row = row0 + ps * RPP + RPI * q;
+                if (!(row < g.M && col < g.N)) continue;
+                const float4 a4 = *reinterpret_cast<const float4*>(tb + (RPI * q + lane / LPR) * TS + 4 * (lane % LPR));
+                const float4 c = make_float4(bc[q].x + bt[q].x, bc[q].y + bt[q].y, bc[q].z + bt[q].z, bc[q].w + bt[q].w);
+                *out_ptr(row) = make_float4(fmaf(f, a4.x, c.x), fmaf(f, a4.y, c.y), fmaf(f, a4.z, c.z), fmaf(f, a4.w, c.w));
+              }
+            };
+            float4 c0[NI], t0[NI];
+            fetch2(0, c0, t0);
+            if (!mbar_wait(accf_bar(ab), ph, dead, p.status, p.spin_limit, 256)) { alive = false; break; }
+            tc_fence_after();
+#pragma unroll 1
+            for (int ps = 0; ps < NP; ++ps) {
+              stage_rows(ps);
+              __syncwarp();
+              if (ps + 1 == NP) release();
+              combine2(ps, c0, t0);
+              __syncwarp();      // the tile is rewritten by the next pass
+              if (ps + 1 < NP) fetch2(ps + 1, c0, t0);
+            }
           } else {
             float4 b0[NI];
             fetch(0, b0);
@@ -839,7 +882,7 @@ __global__ void __launch_bounds__(TMA ? NUM_THREADS_TMA : NUM_THREADS, 1) k_gemm
         else mbar_arrive(acce_bar(ab));
       }
     }
-  } else if (warp < NUM_EPI_WARPS + NUM_PROD_WARPS) {
+  } else if (warp < C::MMA_WARP) {
     // ------------------------------------------------------------ producers
     const int ptid = threadIdx.x - NUM_EPI_WARPS * 32;
     if (NOCONV) {
@@ -987,7 +1030,7 @@ __global__ void __launch_bounds__(TMA ? NUM_THREADS_TMA : NUM_THREADS, 1) k_gemm
       }
     }
     }
-  } else if (TMA && warp == NUM_EPI_WARPS + NUM_PROD_WARPS + 1) {
+  } else if (TMA && warp == C::MMA_WARP + 1) {
     // ------------------------------------------------------------ TMA issuer
     if (lane == 0) {
       const bool add = (g.a2_mode == ADD_F32);
@@ -1182,7 +1225,7 @@ __global__ void __launch_bounds__(TMA ? NUM_THREADS_TMA : NUM_THREADS, 1) k_gemm
   // CTA pair: neither CTA may leave (or free its accumulators) while the other still arrives on its barriers
   // or the leader's MMAs still read its shared memory
   if (CG2) cluster_sync_all();
-  if (warp == NUM_EPI_WARPS + NUM_PROD_WARPS) {
+  if (warp == C::MMA_WARP) {
     tc_fence_after();
     if (CG2) tmem_dealloc2(tmem_base, C::TMEM_COLS);
     else tmem_dealloc(tmem_base, C::TMEM_COLS);
@@ -1201,7 +1244,8 @@ inline cudaError_t set_smem_attr() {
 template <int BN, bool A_MN, bool B_MN>
 inline void launch_x2_one(const Params& p, int grid, cudaStream_t st) {
   constexpr int smem = Cfg<BN, true, false, true, true, true, false, false, true>::SMEM_BYTES;
-  k_gemm_umma<BN, A_MN, B_MN, true, false, true, true, true, false, false, true><<<grid, NUM_THREADS_TMA, smem, st>>>(p);
+  constexpr int threads = Cfg<BN, true, false, true, true, true, false, false, true>::THREADS;
+  k_gemm_umma<BN, A_MN, B_MN, true, false, true, true, true, false, false, true><<<grid, threads, smem, st>>>(p);
 }
 template <int BN>
 inline void launch_x2(const Params& p, bool a_mn, bool b_mn, int grid, cudaStream_t st) {
