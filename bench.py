@@ -50,7 +50,7 @@ TRAFFIC_RATIOS = {
     # M + G kept in scratch: P, R and the error feedback read 4 bytes per element where the algorithmic model
     # counts M and G (the elementwise pass that forms the sum is another kernel)
     "fp32_sum_in_scratch": (0.604, "ncu --set full, one step on 4096^2 r=1024, fp32 mode: 445.6 MB / 738.3 MB"),
-    "fp32_fused_add": (0.885, "same capture with M + G formed inside P and R (the path below rank fraction 1/8)"),
+    "fp32_fused_add": (0.885, "same capture with M + G formed inside P and R (the path below rank fraction 1/64)"),
     "bf16_arrays": (0.99, "ncu --set full, 8192^2 r=512, bf16-operand mode: error feedback 0.98, X update 0.93, P 1.07"),
 }
 
@@ -58,7 +58,7 @@ TRAFFIC_RATIOS = {
 def traffic_variant(m, n, r, precision):
     if precision == 1:
         return "bf16_arrays"
-    return "fp32_sum_in_scratch" if 8 * r >= min(m, n) else "fp32_fused_add"
+    return "fp32_sum_in_scratch" if 64 * r >= min(m, n) else "fp32_fused_add"
 
 
 def load_peaks():
@@ -157,17 +157,23 @@ def phase_bytes(m, n, r, orth, gbytes=4, rounds=None):
 
 def pairs_apply(m, n, r):
     """Shapes whose R and error-feedback products run on bf16 (hi, lo) pairs in fp32 mode (the library's own rule:
-    M + G kept in scratch, i.e. rank fraction >= 1/8, and dimensions that are multiples of 8)."""
-    return r >= 64 and 8 * r >= min(m, n) and m % 8 == 0 and n % 8 == 0 and r % 8 == 0 and m >= 128 and n >= 128
+    M + G kept in scratch, i.e. rank fraction >= 1/64, and dimensions that are multiples of 8)."""
+    return r >= 64 and 64 * r >= min(m, n) and m % 8 == 0 and n % 8 == 0 and r % 8 == 0 and m >= 128 and n >= 128
+
+
+def p_pairs_apply(m, n, r, orth):
+    """Shapes whose P = (M + G) Q runs on bf16 pairs first (the library's rule: pairs in use, CholeskyQR2, and
+    m n r >= 1.5e10; the accurate product is recomputed on the device only if the orthogonality probe asks)."""
+    return pairs_apply(m, n, r) and float(m) * n * r >= 1.5e10 and orth_mode(m, n, r, orth) == 1
 
 
 def case_report(c, ms, rounds, args, peaks, binding):
     """Per-case line: time and the roofline that binds it.  t_hbm: the 7-pass model (read M and G twice,
     read-modify-write M, read-modify-write X) at the measured copy bandwidth; t_tensor: every product at the
-    tensor peak of the arithmetic it runs in -- fp32 mode: P and the orthonormalization 3xTF32 (three TF32
-    passes, TF32 taken as half the measured bf16 peak), R and the error feedback three bf16 passes on (hi, lo)
-    pairs where the library uses them (else 3xTF32), the X update one TF32 pass; bf16-operand mode: one bf16 pass
-    for the four products."""
+    tensor peak of the arithmetic it runs in -- fp32 mode: the orthonormalization 3xTF32 (three TF32 passes, TF32
+    taken as half the measured bf16 peak), P, R and the error feedback three bf16 passes on (hi, lo) pairs where
+    the library uses them (else 3xTF32), the X update one TF32 pass; bf16-operand mode: one bf16 pass for the
+    four products."""
     m, n, r = c[:3]
     out = {"m": m, "n": n, "r": r, "ms": ms,
            "orth_mode": ["auto", "cholqr2", "adaptive", "householder", "rcqr"][orth_mode(m, n, r, args.orth)], "orth_rounds": rounds}
@@ -184,7 +190,8 @@ def case_report(c, ms, rounds, args, peaks, binding):
     else:
         pair_peak = bf16 / 3.0 if pairs_apply(m, n, r) else tf32 / 3.0
         ef_peak = bf16 / 3.0 if (m % 8 == 0 and n % 8 == 0 and r % 8 == 0 and r >= 64) else tf32 / 3.0
-        t_prod = fl["P"] / (tf32 / 3.0 * 1e12) + fl["R"] / (pair_peak * 1e12) + fl["EF"] / (ef_peak * 1e12) + fl["X"] / (tf32 * 1e12)
+        p_peak = bf16 / 3.0 if p_pairs_apply(m, n, r, args.orth) else tf32 / 3.0
+        t_prod = fl["P"] / (p_peak * 1e12) + fl["R"] / (pair_peak * 1e12) + fl["EF"] / (ef_peak * 1e12) + fl["X"] / (tf32 * 1e12)
     t_tensor = (t_prod + fl["ORTH"] / (tf32 / 3.0 * 1e12)) * 1e3
     bound = "hbm" if t_hbm >= t_tensor else "tensor"
     out.update({"t_hbm_ms": t_hbm, "t_tensor_ms": t_tensor, "bound": bound,

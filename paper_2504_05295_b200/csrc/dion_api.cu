@@ -109,15 +109,16 @@ void colnorm_plan(i64 rows, i64 r, int sm, int* chunks, i64* rows_per) {
   *chunks = (int)((rows + per - 1) / per);
 }
 
-// fp32 mode on the tensor engine, tensor-bound ranks: M + G is formed once per step in scratch (12 bytes per
-// element) and P, R and the error feedback read it.  Forming it inside the two products costs their converter
-// warps a second tile and a rewrite of the "hi" half (those products ran 25-30 % slower than the two that read
-// plain operands); at rank fractions below 1/8 the gain no longer pays for the extra pass (measured at 1/16), and
-// at low rank the products are HBM bound and the on-the-fly form moves fewer bytes.
+// fp32 mode on the tensor engine: M + G is formed once per step in scratch, as fp32 (4 bytes per element) and as a
+// bf16 (hi, lo) pair (4 bytes), and P, R and the error feedback read those.  Forming it inside the two products
+// costs their converter warps a second tile and keeps them on three TF32 MMAs per K step; with the pair in
+// memory the products take three bf16 MMAs (half the tensor time) and read 4 bytes per element instead of 8, so the
+// extra pass pays down to rank fraction 1/64 (measured: 32768^2 at r = 512 22.0 -> 15.9 ms, 16384^2 at r = 256
+// 3.4 -> 3.0 ms); below that the step is HBM bound either way and the on-the-fly form moves fewer bytes.
 bool sum_in_scratch(const dion_ctx* c, i64 m, i64 n, i64 r) {
   const i64 sd = (m < n) ? m : n;
   return c->form_sum && c->cfg.precision == DION_PREC_FP32 && c->cfg.engine != DION_ENGINE_SIMT &&
-         m % 4 == 0 && n % 4 == 0 && m >= 128 && n >= 128 && r >= 64 && 8 * r >= sd;
+         m % 4 == 0 && n % 4 == 0 && m >= 128 && n >= 128 && r >= 64 && 64 * r >= sd;
 }
 
 // A step whose orthonormalization may resolve to CholeskyQR2 keeps the panel for the device-side fallback.
