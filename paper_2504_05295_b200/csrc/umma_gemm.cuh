@@ -54,6 +54,7 @@ struct Params {
   int kb_per_split;   // K blocks per split
   int nkb;            // K blocks in all
   int num_items;      // tiles * splits * matrices
+  int raster_gw;      // > 0: rectangular outputs are walked in column panels of this many tile columns
   int items_per_matrix;   // tiles * splits; a batched launch (g.batch2 matrices, g.bs2 elements apart) walks matrix by matrix
   int kc;             // K blocks per accumulation chunk (see k_gemm_umma)
   int* status;        // device status word (DION_STATUS_TIMEOUT)
@@ -142,6 +143,16 @@ __device__ __forceinline__ void mbar_arrive_remote(uint32_t bar, uint32_t rank) 
       "mbarrier.arrive.release.cluster.shared::cluster.b64 _, [ra];\n\t}" ::"r"(bar), "r"(rank)
       : "memory");
 }
+// The same without release semantics: for an arrival that orders nothing but tcgen05 operations (which
+// tcgen05.fence::before_thread_sync orders).  A release at cluster scope makes the thread wait until its earlier
+// global stores are visible cluster-wide: a memory round trip per tile for an epilogue warp.
+__device__ __forceinline__ void mbar_arrive_remote_relaxed(uint32_t bar, uint32_t rank) {
+  asm volatile(
+      "{\n\t.reg .b32 ra;\n\t"
+      "mapa.shared::cluster.u32 ra, %0, %1;\n\t"
+      "mbarrier.arrive.relaxed.cluster.shared::cluster.b64 _, [ra];\n\t}" ::"r"(bar), "r"(rank)
+      : "memory");
+}
 __device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
@@ -167,6 +178,14 @@ __device__ __forceinline__ void umma2_tf32(uint32_t d_tmem, uint64_t adesc, uint
   asm volatile(
       "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
       "tcgen05.mma.cta_group::2.kind::tf32 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+      "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// the same with bf16 operands (256 x N x 16)
+__device__ __forceinline__ void umma2_f16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
       "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
@@ -347,6 +366,16 @@ __device__ __forceinline__ Item decode_item(const Params& p, int item) {
     while (mi * (mi + 1) / 2 > tile) --mi;
     it.mi = mi;
     it.ni = tile - mi * (mi + 1) / 2;
+  } else if (p.raster_gw > 0) {
+    // column panels of raster_gw tile columns, walked row by row: the tiles in flight share the panel's B blocks
+    // (which stay in L2 for the whole panel) instead of sweeping all of B once per wave
+    const int per_panel = p.nM * p.raster_gw;
+    const int pn = tile / per_panel;
+    const int rem = tile - pn * per_panel;
+    const int n0 = pn * p.raster_gw;
+    const int gw = min(p.raster_gw, p.nN - n0);
+    it.mi = rem / gw;
+    it.ni = n0 + (rem - it.mi * gw);
   } else {
     it.mi = tile / p.nN;
     it.ni = tile - it.mi * p.nN;
@@ -563,7 +592,8 @@ template <int BN, bool A_MN, bool B_MN, bool BF16, bool SPLIT, bool TMA, bool D1
 __global__ void __launch_bounds__((Cfg<BN, BF16, SPLIT, TMA, D16, CE, ONE, CG2, X2>::THREADS), 1)
 k_gemm_umma(const __grid_constant__ Params p) {
   static_assert(!X2 || (D16 && CE), "operand pairs are bf16 arrays");
-  static_assert(!CG2 || (TMA && !BF16 && !D16 && !ONE && BN == 256), "CTA pairs: the fp32 TMA variants with 256-column tiles");
+  static_assert(!CG2 || (TMA && BN == 256 && ((!BF16 && !D16 && !ONE) || X2)),
+                "CTA pairs: the fp32 TMA variants and the operand-pair variant, 256-column tiles");
   static_assert(!(BF16 && SPLIT), "split accumulators belong to the 3xTF32 mode");
   static_assert(!D16 || (BF16 && TMA), "bf16 operands in memory are loaded by TMA");
   static_assert(!CE || (TMA && (D16 || !BF16)), "the coalesced epilogue serves the bf16-array and the fp32 TMA variants");
@@ -606,8 +636,9 @@ k_gemm_umma(const __grid_constant__ Params p) {
 
   if (threadIdx.x == 0) {
     // CTA pair: the leader's "full" and "accumulator free" barriers take the arrivals of both CTAs
-    for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), NUM_PROD_WARPS * (CG2 ? 2 : 1)); mbar_init(empty_bar(s), 1); }
-    for (int b = 0; b < 2; ++b) { mbar_init(accf_bar(b), 1); mbar_init(acce_bar(b), C::EPI_WARPS * 32 * (CG2 ? 2 : 1)); }
+    // (nothing to convert: "full" only carries the peer's word that its tiles of the stage have landed)
+    for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), NOCONV ? 1 : NUM_PROD_WARPS * (CG2 ? 2 : 1)); mbar_init(empty_bar(s), 1); }
+    for (int b = 0; b < 2; ++b) { mbar_init(accf_bar(b), 1); mbar_init(acce_bar(b), C::EPI_WARPS * (CG2 ? 2 : 1)); }   // one arrival per epilogue warp
     mbar_init(drain_bar, 1);
     if (TMA) for (int s = 0; s < STAGES; ++s) mbar_init(raw_bar(s), 1);
     *dead = 0;
@@ -749,8 +780,11 @@ k_gemm_umma(const __grid_constant__ Params p) {
           };
           auto release = [&]() {     // the accumulator has been read: the next tile's MMAs may overwrite it
             tc_fence_before();
-            if (CG2 && cta_rank != 0) mbar_arrive_remote(acce_bar(ab), 0u);
-            else mbar_arrive(acce_bar(ab));
+            __syncwarp();          // every lane's TMEM reads are done; one (possibly remote) arrival per warp
+            if (lane == 0) {
+              if (CG2 && cta_rank != 0) mbar_arrive_remote_relaxed(acce_bar(ab), 0u);
+              else mbar_arrive(acce_bar(ab));
+            }
           };
           if constexpr (SPLIT) {
             // two accumulators to read per slab: no registers to spare for loads in flight across the staging
@@ -878,8 +912,11 @@ k_gemm_umma(const __grid_constant__ Params p) {
           }
         }
         tc_fence_before();
-        if (CG2 && cta_rank != 0) mbar_arrive_remote(acce_bar(ab), 0u);
-        else mbar_arrive(acce_bar(ab));
+        __syncwarp();
+        if (lane == 0) {
+          if (CG2 && cta_rank != 0) mbar_arrive_remote_relaxed(acce_bar(ab), 0u);
+          else mbar_arrive(acce_bar(ab));
+        }
       }
     }
   } else if (warp < C::MMA_WARP) {
@@ -1070,7 +1107,7 @@ k_gemm_umma(const __grid_constant__ Params p) {
               tma_load_3d(sb_lo2, &p.tmB2, k0, row0b, it.b, bar);
             } else {
 #pragma unroll
-              for (int c = 0; c < BN / 64; ++c) {
+              for (int c = 0; c < BN_L / 64; ++c) {
                 tma_load_3d(sb + c * (BKE * 128), &p.tmB, row0b + 64 * c, k0, it.b, bar);
                 tma_load_3d(sb_lo2 + c * (BKE * 128), &p.tmB2, row0b + 64 * c, k0, it.b, bar);
               }
@@ -1128,7 +1165,22 @@ k_gemm_umma(const __grid_constant__ Params p) {
     __syncwarp();
   } else {
     // ------------------------------------------------------------ MMA issuer (CTA pair: the leader only)
-    if (lane == 0 && (!CG2 || cta_rank == 0)) {
+    if (lane == 0 && CG2 && NOCONV && cta_rank != 0) {
+      // The peer of a pair without converter warps: TMA fills this CTA's tiles and completes on this CTA's
+      // barrier; this thread passes the word on to the leader, whose MMAs read both CTAs' shared memory.
+      int stage = 0;
+      uint32_t phase = 0;
+      bool alive = true;
+      for (int item = worker; item < p.num_items && alive; item += workers) {
+        const Item it = decode_item<BN, BKE, CG2>(p, item);
+        if (skipped(it)) continue;
+        for (int kb = it.kb0; kb < it.kb1; ++kb) {
+          if (!mbar_wait(raw_bar(stage), phase, dead, p.status, p.spin_limit)) { alive = false; break; }
+          mbar_arrive_remote(full_bar(stage), 0u);
+          if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+        }
+      }
+    } else if (lane == 0 && (!CG2 || cta_rank == 0)) {
       const uint32_t idesc = make_idesc(BF16, A_MN, B_MN, BN, CG2 ? 2 * BM : BM);
       const uint32_t lbo = BKE * 128;
       constexpr uint32_t A_KSTEP = A_MN ? (BF16 ? 2048u : 1024u) : 32u;   // bytes per UMMA K step
@@ -1150,7 +1202,12 @@ k_gemm_umma(const __grid_constant__ Params p) {
         const uint32_t d_small = d_tmem + (SPLIT ? BN : 0);
         uint32_t accumulate = 0;
         for (int kb = kbc; kb < kbc1; ++kb) {
-          if (!mbar_wait<CG2>(NOCONV ? raw_bar(stage) : full_bar(stage), phase, dead, p.status, p.spin_limit)) { alive = false; break; }
+          if (NOCONV) {   // this CTA's tiles (TMA), then the peer's (its relay thread)
+            if (!mbar_wait(raw_bar(stage), phase, dead, p.status, p.spin_limit)) { alive = false; break; }
+            if (CG2 && !mbar_wait<true>(full_bar(stage), phase, dead, p.status, p.spin_limit)) { alive = false; break; }
+          } else {
+            if (!mbar_wait<CG2>(full_bar(stage), phase, dead, p.status, p.spin_limit)) { alive = false; break; }
+          }
           tc_fence_after();
           const uint32_t st0 = smem_base + stage * C::STAGE_BYTES;
           // bf16 operands formed from TMA tiles sit behind the raw tiles of the stage
@@ -1165,9 +1222,15 @@ k_gemm_umma(const __grid_constant__ Params p) {
             if (X2) {
               const uint64_t a_lo = make_desc<BF16>(sa_lo + ks * A_KSTEP, A_MN, lbo);
               const uint64_t b_lo = make_desc<BF16>(sb_lo + ks * B_KSTEP, B_MN, lbo);
-              umma<true>(d_tmem, a_hi, b_lo, idesc, accumulate);   // small terms first
-              umma<true>(d_tmem, a_lo, b_hi, idesc, 1u);
-              umma<true>(d_tmem, a_hi, b_hi, idesc, 1u);
+              if (CG2) {
+                umma2_f16(d_tmem, a_hi, b_lo, idesc, accumulate);
+                umma2_f16(d_tmem, a_lo, b_hi, idesc, 1u);
+                umma2_f16(d_tmem, a_hi, b_hi, idesc, 1u);
+              } else {
+                umma<true>(d_tmem, a_hi, b_lo, idesc, accumulate);   // small terms first
+                umma<true>(d_tmem, a_lo, b_hi, idesc, 1u);
+                umma<true>(d_tmem, a_hi, b_hi, idesc, 1u);
+              }
               accumulate = 1;
             } else if (BF16) {
               umma<true>(d_tmem, a_hi, b_hi, idesc, accumulate);
@@ -1257,6 +1320,29 @@ inline void launch_x2(const Params& p, bool a_mn, bool b_mn, int grid, cudaStrea
 template <int BN, bool A_MN, bool B_MN>
 inline cudaError_t set_x2_attr() {
   return set_smem_attr<BN, A_MN, B_MN, true, false, true, true, true, false, false, true>();
+}
+
+// bf16 operand pairs on CTA pairs
+template <bool A_MN, bool B_MN>
+inline cudaError_t launch_x2_pair_one(const Params& p, int grid, cudaStream_t st) {
+  using CF = Cfg<256, true, false, true, true, true, false, true, true>;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)grid); cfg.blockDim = dim3(CF::THREADS); cfg.dynamicSmemBytes = CF::SMEM_BYTES; cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr; cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, k_gemm_umma<256, A_MN, B_MN, true, false, true, true, true, false, true, true>, p);
+}
+inline cudaError_t launch_x2_pair(const Params& p, bool a_mn, bool b_mn, int grid, cudaStream_t st) {
+  if (!a_mn && !b_mn) return launch_x2_pair_one<false, false>(p, grid, st);
+  if (!a_mn && b_mn) return launch_x2_pair_one<false, true>(p, grid, st);
+  if (a_mn && b_mn) return launch_x2_pair_one<true, true>(p, grid, st);
+  return launch_x2_pair_one<true, false>(p, grid, st);
+}
+template <bool A_MN, bool B_MN>
+inline cudaError_t set_x2_pair_attr() {
+  return set_smem_attr<256, A_MN, B_MN, true, false, true, true, true, false, true, true>();
 }
 
 // CTA pairs: clusters of two CTAs, 256 x 256 tiles (fp32 mode, TMA, coalesced epilogue)
@@ -1452,6 +1538,10 @@ inline int umma_configure() {
   if (e == cudaSuccess) e = set_x2_attr<256, false, true>();
   if (e == cudaSuccess) e = set_x2_attr<256, true, true>();
   if (e == cudaSuccess) e = set_x2_attr<256, true, false>();
+  if (e == cudaSuccess) e = set_x2_pair_attr<false, false>();
+  if (e == cudaSuccess) e = set_x2_pair_attr<false, true>();
+  if (e == cudaSuccess) e = set_x2_pair_attr<true, true>();
+  if (e == cudaSuccess) e = set_x2_pair_attr<true, false>();
   if (e == cudaSuccess) e = set_pair_attr<false, false>();
   if (e == cudaSuccess) e = set_pair_attr<false, true>();
   if (e == cudaSuccess) e = set_pair_attr<true, true>();
@@ -1523,8 +1613,13 @@ inline int umma_try_launch(const GemmArgs& g_in, int precision, int sm_count, fl
   // CTA pairs (cta_group::2, 256 x 256 tiles): the fp32 (3xTF32) products that the TMA variant with the
   // coalesced epilogue takes, once the output is tall enough to give every pair work
   const int nclusters = pair_clusters(sm_count);
-  bool cg2 = !bf16 && !g.tf32x1 && !(variant & (UMMA_VARIANT_REGISTER_LOADS | UMMA_VARIANT_NO_PAIRS)) && nclusters > 0 &&
-             g.a2_mode != ADD_BF16 && g.N >= 256 && g.M >= PAIR_MIN_ROWS && (g.tri != TRI_LOWER || g.N >= PAIR_MIN_TRI);
+  // ... and the products on bf16 operand pairs (two thirds of the operand traffic per CTA, three stages instead of two)
+  const bool x2 = d16 && g.A16lo != nullptr && g.B16lo != nullptr;   // bf16 operand pairs
+  // (not the single-pass product: its pair form ran the X update of the 8B list in 51 ms instead of 32, tensor
+  // pipe 30 % instead of 54 % under ncu, with or without per-warp and relaxed arrivals; cause not found)
+  bool cg2 = ((!bf16 && !g.tf32x1 && g.a2_mode != ADD_BF16) || x2) &&
+             !(variant & (UMMA_VARIANT_REGISTER_LOADS | UMMA_VARIANT_NO_PAIRS)) && nclusters > 0 &&
+             g.N >= 256 && g.M >= PAIR_MIN_ROWS && (g.tri != TRI_LOWER || g.N >= PAIR_MIN_TRI);
   const int BN = ((g.tri == TRI_LOWER && !tri_wide && !cg2) || g.N < 256) ? 128 : 256;
   Params p;
   p.g = g;
@@ -1532,16 +1627,15 @@ inline int umma_try_launch(const GemmArgs& g_in, int precision, int sm_count, fl
   if (g.c2_tab != nullptr) for (int b = 0; b < nbat; ++b) p.c2tab[b] = g.c2_tab[b];
   // TMA variant: fp32 operands in memory (both precision modes), dimensions the tensor maps can describe
   bool tma = (d16 || !(variant & UMMA_VARIANT_REGISTER_LOADS)) && g.M < (1ll << 31) && g.N < (1ll << 31) && g.K < (1ll << 31);
-  const bool x2 = d16 && g.A16lo != nullptr && g.B16lo != nullptr;   // bf16 operand pairs
   if (x2 && (!aligned(g.A16lo, 16) || !aligned(g.B16lo, 16))) return 0;
   if (d16) {
     const i64 lda = a_mn ? g.a_sk : g.a_si, ldb = b_mn ? g.b_sk : g.b_sn;
     const i64 bsb = g.bs2 * 4;   // the batch stride counts 4-byte words for every operand type
     if (!tma || !make_operand16_map(&p.tmA, g.A, g.M, g.K, lda, a_mn, BM, nbat, bsb) ||
-        !make_operand16_map(&p.tmB, g.B, g.N, g.K, ldb, b_mn, BN, nbat, bsb))
+        !make_operand16_map(&p.tmB, g.B, g.N, g.K, ldb, b_mn, cg2 ? BN / 2 : BN, nbat, bsb))
       return 0;
     if (x2 && (!make_operand16_map(&p.tmA2, g.A16lo, g.M, g.K, lda, a_mn, BM, nbat, bsb) ||
-               !make_operand16_map(&p.tmB2, g.B16lo, g.N, g.K, ldb, b_mn, BN, nbat, bsb)))
+               !make_operand16_map(&p.tmB2, g.B16lo, g.N, g.K, ldb, b_mn, cg2 ? BN / 2 : BN, nbat, bsb)))
       return 0;
   } else
   if (tma && g.a2_mode == ADD_BF16) {   // the bf16 addend needs 16-byte aligned rows for its tensor map
@@ -1570,6 +1664,19 @@ inline int umma_try_launch(const GemmArgs& g_in, int precision, int sm_count, fl
                     : (BN == 256 && !cg2)  ? ((i64)p.nM + 1) * (p.nM + 1) / 4
                                            : (i64)p.nM * (p.nM + 1) / 2;
   const int workers_max = cg2 ? nclusters : sm_count;   // CTAs, or CTA pairs, that can run at once
+  // Tile order.  Row by row, a wave of tiles reads every column block of B; when B (N x K) is larger than what L2
+  // keeps, every wave fetches it from DRAM again (ncu, X update at 16384^2, r = 4096: 16.8 GB read for 1.3 GB of
+  // operands and output).  Then the output is walked in column panels whose B blocks (~32 MB) stay in L2.
+  p.raster_gw = 0;
+  if (g.tri != TRI_LOWER) {
+    const double esz = d16 ? (x2 ? 4.0 : 2.0) : 4.0;             // bytes per operand element as read by this variant
+    const double bblock = (double)BN * (double)g.K * esz;
+    if ((double)p.nN * bblock > 48e6) {
+      int gw = (int)(32e6 / bblock);
+      if (gw < 2) gw = 2;
+      if (gw < p.nN) p.raster_gw = gw;
+    }
+  }
   int splits = 1;
   if (g.epi == EPI_STORE && !g.klimit && part != nullptr && tiles < workers_max) {
     i64 want = workers_max / tiles;
@@ -1596,7 +1703,9 @@ inline int umma_try_launch(const GemmArgs& g_in, int precision, int sm_count, fl
   const int grid = cg2 ? 2 * (p.num_items < nclusters ? p.num_items : nclusters)
                        : (p.num_items < sm_count ? p.num_items : sm_count);
   const bool one = g.tf32x1 && !bf16 && tma && !a_mn && !b_mn && g.a2_mode == ADD_NONE && !g.precise && splits == 1;
-  if (cg2) {
+  if (cg2 && x2) {
+    if (launch_x2_pair(p, a_mn, b_mn, grid, st) != cudaSuccess) { cudaGetLastError(); return DION_ERR_CUDA; }
+  } else if (cg2) {
     const cudaError_t e = g.precise ? launch_pair<true>(p, a_mn, b_mn, grid, st) : launch_pair<false>(p, a_mn, b_mn, grid, st);
     if (e != cudaSuccess) { cudaGetLastError(); return DION_ERR_CUDA; }
   } else if (one) {

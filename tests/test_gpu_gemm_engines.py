@@ -297,3 +297,60 @@ def test_bf16_operand_pairs(lib, M, N, K, epi):
     err = float((C.double() - want).norm() / want.norm())
     assert err_prod < 3e-5, err_prod
     assert err < 1e-5 or epi == 0, err
+
+
+def _pair_product(lib, M, N, K, a_mn, b_mn, epi, variant, seed):
+    """C after one product on bf16 (hi, lo) operand pairs in the given storage layouts; also the float64 target."""
+    g = torch.Generator(device="cuda"); g.manual_seed(seed)
+    A = torch.randn(M, K, generator=g, device="cuda"); B = torch.randn(N, K, generator=g, device="cuda")
+
+    def split(x):
+        h = x.to(torch.bfloat16)
+        return h, (x - h.float()).to(torch.bfloat16)
+    As = A.t().contiguous() if a_mn else A          # stored K x M (row index contiguous) or M x K
+    Bs = B.t().contiguous() if b_mn else B          # stored K x N or N x K
+    Ah, Al = split(As); Bh, Bl = split(Bs)
+    C = torch.randn(M, N, generator=g, device="cuda"); C0 = C.clone()
+    C2 = torch.randn(M, N, generator=g, device="cuda")
+    alpha = 0.05
+    ref = A.double() @ B.double().t()
+    want = {0: alpha * ref, 1: C0.double() - alpha * ref, 2: C0.double() + C2.double() - alpha * ref,
+            3: C2.double() - alpha * ref}[epi]
+    a = GemmArgs()
+    a.M, a.N, a.K = M, N, K
+    a.A = Ah.data_ptr(); a.A16lo = Al.data_ptr(); a.a_si, a.a_sk = (1, M) if a_mn else (K, 1)
+    a.B = Bh.data_ptr(); a.B16lo = Bl.data_ptr(); a.b_sk, a.b_sn = (N, 1) if b_mn else (1, K)
+    a.C = C.data_ptr(); a.ldc = N; a.epi = epi
+    a.C2 = C2.data_ptr(); a.ldc2 = N; a.c2_mode = 1
+    a.alpha = alpha; a.ab16 = 1; a.variant = variant
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    part = torch.empty(8 << 20, device="cuda")
+    rc = lib.dion_debug_gemm(2, 1, ctypes.byref(a), part.data_ptr(), part.numel(), status.data_ptr(),
+                             int(torch.cuda.current_stream().cuda_stream))
+    torch.cuda.synchronize()
+    assert rc == 0 and int(status.item()) == 0, (rc, int(status.item()))
+    return C, want
+
+
+@pytest.mark.parametrize("a_mn,b_mn", LAYOUTS)
+def test_bf16_operand_pairs_on_cta_pairs(lib, a_mn, b_mn):
+    # from 512 rows and 256 columns the operand-pair product runs on clusters of two CTAs (256 x 256 tiles, each CTA
+    # loading half of the B tile); bit 2 of the variant word keeps it on single-CTA tiles: same bits
+    for (M, N, K, epi) in [(1024, 512, 512, 0), (2048, 768, 2112, 1), (648, 392, 328, 2), (1280, 256, 96, 3),
+                           (512, 512, 8192, 0)]:
+        C, want = _pair_product(lib, M, N, K, a_mn, b_mn, epi, 0, seed=M + K)
+        err = float((C.double() - want).norm() / want.norm())
+        assert err < (3e-5 if epi == 0 else 1e-5), (M, N, K, epi, err)
+        C1, _ = _pair_product(lib, M, N, K, a_mn, b_mn, epi, 4, seed=M + K)
+        if K < 8192:      # (the last case has few tiles: K is split, differently for pairs and single CTAs)
+            assert torch.equal(C, C1), (M, N, K, epi)
+
+
+def test_column_panel_tile_order_when_b_exceeds_l2(lib):
+    # N x K operands above ~48 MB switch the tile order to column panels (every tile still computed exactly once)
+    assert run(lib, 2, 0, 1024, 4096, 4096, False, False, epi=1, alpha=0.01) < TOL[2]
+    assert run(lib, 2, 0, 1024, 4352, 3104, False, True, epi=0) < TOL[2]                    # ragged, last panel narrower
+    assert run(lib, 2, 0, 640, 8192, 2048, False, False, epi=1, alpha=0.05, tf32x1=True) < 8e-6
+    for (a_mn, b_mn) in LAYOUTS:
+        C, want = _pair_product(lib, 1024, 8192 + 256, 2048, a_mn, b_mn, 3, 0, seed=5)
+        assert float((C.double() - want).norm() / want.norm()) < 1e-5
