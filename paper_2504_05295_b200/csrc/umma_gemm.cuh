@@ -1669,12 +1669,18 @@ inline int umma_try_launch(const GemmArgs& g_in, int precision, int sm_count, fl
   // operands and output).  Then the output is walked in column panels whose B blocks (~32 MB) stay in L2.
   p.raster_gw = 0;
   if (g.tri != TRI_LOWER) {
+    // DRAM bytes of the operands under either order (A block = one tile row of A, B block = one tile column of B;
+    // L2 keeps ~60 MB of a re-read operand, a panel is held to 40 MB): row by row A is read once and B once per
+    // wave unless it fits; in panels of gw columns B is read once and A once per panel
     const double esz = d16 ? (x2 ? 4.0 : 2.0) : 4.0;             // bytes per operand element as read by this variant
-    const double bblock = (double)BN * (double)g.K * esz;
-    if ((double)p.nN * bblock > 48e6) {
-      int gw = (int)(32e6 / bblock);
-      if (gw < 2) gw = 2;
-      if (gw < p.nN) p.raster_gw = gw;
+    const double ablock = (double)tile_m * (double)g.K * esz, bblock = (double)BN * (double)g.K * esz;
+    const double nM = p.nM, nN = p.nN, W = workers_max;
+    const double waves = nM * nN / W;
+    const double by_rows = nM * ablock + ((nN * bblock > 60e6) ? waves * (nN < W ? nN : W) * bblock : nN * bblock);
+    double best = 0.8 * by_rows;      // panels only for a clear gain
+    for (int gw = 2; gw < p.nN && gw * bblock <= 40e6; ++gw) {
+      const double cost = nM * ablock * (double)((p.nN + gw - 1) / gw) + nN * bblock;
+      if (cost < best) { best = cost; p.raster_gw = gw; }
     }
   }
   int splits = 1;
