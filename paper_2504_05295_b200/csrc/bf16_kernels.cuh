@@ -69,10 +69,9 @@ __global__ void __launch_bounds__(256) k_form_b16(const float* __restrict__ M, i
 // hi / lo (optional, both or neither; cols a multiple of 8 then): the same sum as a pair of bf16 arrays, hi = bf16(sum),
 // lo = bf16(sum - hi), dense like out: the operand of the products that run on bf16 pairs.
 template <bool VEC>
-__global__ void __launch_bounds__(256) k_form_b32(const float* __restrict__ M, i64 ldm, const void* __restrict__ G,
-                                                  i64 ldg, int g_mode, i64 rows, i64 cols, float* __restrict__ out,
-                                                  __nv_bfloat16* __restrict__ hi, __nv_bfloat16* __restrict__ lo) {
-  pdl_enter();
+__device__ __forceinline__ void form_b32_body(const float* __restrict__ M, i64 ldm, const void* __restrict__ G,
+                                              i64 ldg, int g_mode, i64 rows, i64 cols, float* __restrict__ out,
+                                              __nv_bfloat16* __restrict__ hi, __nv_bfloat16* __restrict__ lo) {
   const i64 per_row = cols / 4;
   const i64 total = rows * per_row;
   for (i64 e = (i64)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (i64)gridDim.x * blockDim.x) {
@@ -111,6 +110,25 @@ __global__ void __launch_bounds__(256) k_form_b32(const float* __restrict__ M, i
     }
   }
 }
+template <bool VEC>
+__global__ void __launch_bounds__(256) k_form_b32(const float* __restrict__ M, i64 ldm, const void* __restrict__ G,
+                                                  i64 ldg, int g_mode, i64 rows, i64 cols, float* __restrict__ out,
+                                                  __nv_bfloat16* __restrict__ hi, __nv_bfloat16* __restrict__ lo) {
+  pdl_enter();
+  form_b32_body<VEC>(M, ldm, G, ldg, g_mode, rows, cols, out, hi, lo);
+}
+// The same for every matrix of a chain in one launch (blockIdx.y): the caller's M and G from pointer tables, the
+// outputs in the scratch slices, `ostride` floats apart.
+template <bool VEC>
+__global__ void __launch_bounds__(256) k_form_b32_chain(const ChainPtrs Ms, i64 ldm, const ChainPtrs Gs, i64 ldg, int g_mode,
+                                                        i64 rows, i64 cols, float* __restrict__ out,
+                                                        __nv_bfloat16* __restrict__ hi, __nv_bfloat16* __restrict__ lo,
+                                                        i64 ostride) {
+  pdl_enter();
+  const i64 b = blockIdx.y;
+  form_b32_body<VEC>(reinterpret_cast<const float*>(Ms.p[b]), ldm, Gs.p[b], ldg, g_mode, rows, cols, out + b * ostride,
+                     hi != nullptr ? hi + 2 * b * ostride : nullptr, lo != nullptr ? lo + 2 * b * ostride : nullptr);
+}
 
 // out = bf16(src), rows x cols (cols a multiple of 8, src rows 16-byte aligned), out dense.
 // skip_flag (optional): nothing is written when *skip_flag != 0.
@@ -133,11 +151,8 @@ __global__ void __launch_bounds__(256) k_to_bf16(const float* __restrict__ src, 
 
 // hi = bf16(src), lo = bf16(src - hi): src ~ hi + lo to 16 significant bits.  rows x cols (cols a multiple of 8,
 // src rows 16-byte aligned), hi and lo dense.  skip_flag (optional): nothing is written when *skip_flag != 0.
-__global__ void __launch_bounds__(256) k_split_bf16(const float* __restrict__ src, i64 lds, i64 rows, i64 cols,
-                                                    __nv_bfloat16* __restrict__ hi, __nv_bfloat16* __restrict__ lo,
-                                                    const int* __restrict__ skip_flag) {
-  pdl_enter();
-  if (skip_flag != nullptr && *skip_flag != 0) return;
+__device__ __forceinline__ void split_bf16_body(const float* __restrict__ src, i64 lds, i64 rows, i64 cols,
+                                                __nv_bfloat16* __restrict__ hi, __nv_bfloat16* __restrict__ lo) {
   const i64 per_row = cols / 8;
   const i64 total = rows * per_row;
   for (i64 e = (i64)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (i64)gridDim.x * blockDim.x) {
@@ -158,16 +173,31 @@ __global__ void __launch_bounds__(256) k_split_bf16(const float* __restrict__ sr
     *reinterpret_cast<uint4*>(lo + i * cols + c) = ol;
   }
 }
+__global__ void __launch_bounds__(256) k_split_bf16(const float* __restrict__ src, i64 lds, i64 rows, i64 cols,
+                                                    __nv_bfloat16* __restrict__ hi, __nv_bfloat16* __restrict__ lo,
+                                                    const int* __restrict__ skip_flag) {
+  pdl_enter();
+  if (skip_flag != nullptr && *skip_flag != 0) return;
+  split_bf16_body(src, lds, rows, cols, hi, lo);
+}
+// One launch over the matrices of a chain (blockIdx.y): sources from a pointer table, outputs `ostride` floats
+// apart in the scratch slices, skip flags `skip_stride` ints apart.
+__global__ void __launch_bounds__(256) k_split_bf16_chain(const ChainPtrs srcs, i64 lds, i64 rows, i64 cols,
+                                                          __nv_bfloat16* __restrict__ hi, __nv_bfloat16* __restrict__ lo,
+                                                          i64 ostride, const int* __restrict__ skip_flag, i64 skip_stride) {
+  pdl_enter();
+  const i64 b = blockIdx.y;
+  if (skip_flag != nullptr && skip_flag[b * skip_stride] != 0) return;
+  split_bf16_body(reinterpret_cast<const float*>(srcs.p[b]), lds, rows, cols, hi + 2 * b * ostride, lo + 2 * b * ostride);
+}
 
 // out = src with every value rounded to the nearest TF32 number (10 explicit mantissa bits, ties away
 // from zero), rows x cols (cols a multiple of 4, src rows 16-byte aligned), out dense.  The tensor core
 // truncates an fp32 operand to TF32 when it reads it; on pre-rounded values that truncation is exact, so a
 // single-pass TF32 product of such arrays carries an unbiased operand error of at most 2^-11 relative.
 // skip_flag (optional): nothing is written when *skip_flag != 0.
-__global__ void __launch_bounds__(256) k_round_tf32(const float* __restrict__ src, i64 lds, i64 rows, i64 cols,
-                                                    float* __restrict__ out, const int* __restrict__ skip_flag) {
-  pdl_enter();
-  if (skip_flag != nullptr && *skip_flag != 0) return;
+__device__ __forceinline__ void round_tf32_body(const float* __restrict__ src, i64 lds, i64 rows, i64 cols,
+                                                float* __restrict__ out) {
   const i64 per_row = cols / 4;
   const i64 total = rows * per_row;
   for (i64 e = (i64)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (i64)gridDim.x * blockDim.x) {
@@ -180,6 +210,20 @@ __global__ void __launch_bounds__(256) k_round_tf32(const float* __restrict__ sr
     asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(o.w) : "f"(a.w));
     *reinterpret_cast<uint4*>(out + i * cols + c) = o;
   }
+}
+__global__ void __launch_bounds__(256) k_round_tf32(const float* __restrict__ src, i64 lds, i64 rows, i64 cols,
+                                                    float* __restrict__ out, const int* __restrict__ skip_flag) {
+  pdl_enter();
+  if (skip_flag != nullptr && *skip_flag != 0) return;
+  round_tf32_body(src, lds, rows, cols, out);
+}
+__global__ void __launch_bounds__(256) k_round_tf32_chain(const ChainPtrs srcs, i64 lds, i64 rows, i64 cols,
+                                                          float* __restrict__ out, i64 ostride,
+                                                          const int* __restrict__ skip_flag, i64 skip_stride) {
+  pdl_enter();
+  const i64 b = blockIdx.y;
+  if (skip_flag != nullptr && skip_flag[b * skip_stride] != 0) return;
+  round_tf32_body(reinterpret_cast<const float*>(srcs.p[b]), lds, rows, cols, out + b * ostride);
 }
 
 }  // namespace dion

@@ -941,11 +941,87 @@ int colnorm(StepCtx& s, int b, const float* W, i64 rows, i64 r, float* out, i64 
   colnorm_plan(rows, r, c->sm_count, &chunks, &per);
   float* part = s.W(b, s.L.cn_part);
   dim3 grid((unsigned)((r + 127) / 128), (unsigned)chunks);
-  launch_pdl(k_colsumsq_partial, grid, dim3(128), 0, s.st, W, ldw, rows, r, per, part, nullptr);
+  launch_pdl(k_colsumsq_partial, grid, dim3(128), 0, s.st, W, ldw, rows, r, per, part, (const int*)nullptr, (i64)0);
   DION_CHECK_LAUNCH(c);
-  launch_pdl(k_colnorm_apply, grid, dim3(128), 0, s.st, W, ldw, rows, r, per, chunks, part, c->cfg.eps, out, ldo,
-                                         s.W(b, s.L.d), d_out, c->dev_ints, skip != nullptr ? skip : s.OS(b) + OS_FAIL);
+  launch_pdl(k_colnorm_apply, grid, dim3(128), 0, s.st, W, ldw, rows, r, per, chunks, (const float*)part, c->cfg.eps, out, ldo,
+             s.W(b, s.L.d), d_out, c->dev_ints, skip != nullptr ? skip : (const int*)(s.OS(b) + OS_FAIL), (i64)0, ChainPtrs(), ChainPtrs());
   DION_CHECK_LAUNCH(c);
+  return DION_OK;
+}
+
+// ---- elementwise kernels over a whole chain -------------------------------------------------------------------
+// Each helper makes ONE launch over the chain's matrices (blockIdx.y or .z) when their arrays share leading
+// dimensions and alignment, else one launch per matrix; outputs are in the scratch slices either way.
+
+// ColNorm of every matrix's R (scratch, rows x r dense) into its Q, d exported to colnorm_out.
+int colnorm_chain(StepCtx& s, const dion_matrix* const* list, i64 rows, i64 r) {
+  dion_ctx* c = s.c;
+  bool one = s.nb > 1 && s.nb <= GEMM_TAB_MAX && c->chain_batch;
+  for (int b = 1; b < s.nb && one; ++b) one = list[b]->ldq == list[0]->ldq;
+  if (!one) {
+    for (int b = 0; b < s.nb; ++b)
+      DION_TRY(colnorm(s, b, s.W(b, s.L.R), rows, r, (float*)list[b]->Q, list[b]->ldq, list[b]->colnorm_out));
+    return DION_OK;
+  }
+  int chunks; i64 per;
+  colnorm_plan(rows, r, c->sm_count, &chunks, &per);
+  ChainPtrs Qs, ds;
+  for (int b = 0; b < s.nb; ++b) { Qs.p[b] = list[b]->Q; ds.p[b] = list[b]->colnorm_out; }
+  dim3 grid((unsigned)((r + 127) / 128), (unsigned)chunks, (unsigned)s.nb);
+  launch_pdl(k_colsumsq_partial, grid, dim3(128), 0, s.st, (const float*)(s.ws + s.L.R), r, rows, r, per, s.ws + s.L.cn_part,
+             (const int*)nullptr, s.wstride);
+  DION_CHECK_LAUNCH(c);
+  launch_pdl(k_colnorm_apply, grid, dim3(128), 0, s.st, (const float*)(s.ws + s.L.R), r, rows, r, per, chunks,
+             (const float*)(s.ws + s.L.cn_part), c->cfg.eps, (float*)nullptr, list[0]->ldq, s.ws + s.L.d, (float*)nullptr, c->dev_ints,
+             (const int*)(s.os + OS_FAIL), s.wstride, Qs, ds);
+  DION_CHECK_LAUNCH(c);
+  return DION_OK;
+}
+
+// hi / lo bf16 pair of src[b] (rows x cols, leading dimension ld[b]) into the scratch slices at out_off.
+// skip0: the flag of matrix 0 (a state slot apart per matrix), or nullptr.
+int split_chain(StepCtx& s, const float* const* src, const i64* ld, i64 rows, i64 cols, i64 out_off, const int* skip0) {
+  dion_ctx* c = s.c;
+  bool one = s.nb > 1 && s.nb <= GEMM_TAB_MAX && c->chain_batch;
+  for (int b = 1; b < s.nb && one; ++b) one = ld[b] == ld[0];
+  const unsigned gx = (unsigned)grid_for(c, rows * cols / 8);
+  if (one) {
+    ChainPtrs t;
+    for (int b = 0; b < s.nb; ++b) t.p[b] = src[b];
+    __nv_bfloat16* hi = reinterpret_cast<__nv_bfloat16*>(s.ws + out_off);
+    launch_pdl(k_split_bf16_chain, dim3(gx, (unsigned)s.nb), dim3(256), 0, s.st, t, ld[0], rows, cols, hi, hi + rows * cols, s.wstride, skip0,
+               (i64)OS_SLOT_INTS);
+    DION_CHECK_LAUNCH(c);
+    return DION_OK;
+  }
+  for (int b = 0; b < s.nb; ++b) {
+    __nv_bfloat16* hi = reinterpret_cast<__nv_bfloat16*>(s.W(b, out_off));
+    launch_pdl(k_split_bf16, dim3(gx), dim3(256), 0, s.st, src[b], ld[b], rows, cols, hi, hi + rows * cols,
+               skip0 != nullptr ? skip0 + (i64)b * OS_SLOT_INTS : (const int*)nullptr);
+    DION_CHECK_LAUNCH(c);
+  }
+  return DION_OK;
+}
+
+// src[b] rounded to TF32 into the scratch slices at out_off.
+int round_chain(StepCtx& s, const float* const* src, const i64* ld, i64 rows, i64 cols, i64 out_off, const int* skip0) {
+  dion_ctx* c = s.c;
+  bool one = s.nb > 1 && s.nb <= GEMM_TAB_MAX && c->chain_batch;
+  for (int b = 1; b < s.nb && one; ++b) one = ld[b] == ld[0];
+  const unsigned gx = (unsigned)grid_for(c, rows * cols / 4);
+  if (one) {
+    ChainPtrs t;
+    for (int b = 0; b < s.nb; ++b) t.p[b] = src[b];
+    launch_pdl(k_round_tf32_chain, dim3(gx, (unsigned)s.nb), dim3(256), 0, s.st, t, ld[0], rows, cols, s.ws + out_off, s.wstride, skip0,
+               (i64)OS_SLOT_INTS);
+    DION_CHECK_LAUNCH(c);
+    return DION_OK;
+  }
+  for (int b = 0; b < s.nb; ++b) {
+    launch_pdl(k_round_tf32, dim3(gx), dim3(256), 0, s.st, src[b], ld[b], rows, cols, s.W(b, out_off),
+               skip0 != nullptr ? skip0 + (i64)b * OS_SLOT_INTS : (const int*)nullptr);
+    DION_CHECK_LAUNCH(c);
+  }
   return DION_OK;
 }
 
@@ -1027,16 +1103,47 @@ int form_sum(StepCtx& s, int b, const dion_matrix* a, bool pair) {
   return DION_OK;
 }
 
+// form_sum for every matrix of the chain: one launch when M and G share leading dimensions and alignment.
+int form_sum_chain(StepCtx& s, const dion_matrix* const* list, bool pair) {
+  dion_ctx* c = s.c;
+  const dion_matrix* a0 = list[0];
+  auto vec_ok = [](const dion_matrix* a) {
+    return !((uintptr_t)a->M & 15) && a->ldm % 4 == 0 &&
+           (a->g_dtype == DION_BF16 ? (!((uintptr_t)a->G & 7) && a->ldg % 4 == 0) : (!((uintptr_t)a->G & 15) && a->ldg % 4 == 0));
+  };
+  bool one = s.nb > 1 && s.nb <= GEMM_TAB_MAX && c->chain_batch;
+  const bool vec = vec_ok(a0);
+  for (int b = 1; b < s.nb && one; ++b)
+    one = list[b]->ldm == a0->ldm && list[b]->ldg == a0->ldg && list[b]->g_dtype == a0->g_dtype && vec_ok(list[b]) == vec;
+  if (!one) {
+    for (int b = 0; b < s.nb; ++b) DION_TRY(form_sum(s, b, list[b], pair));
+    return DION_OK;
+  }
+  const i64 m = a0->m, n = a0->n;
+  ChainPtrs Ms, Gs;
+  for (int b = 0; b < s.nb; ++b) { Ms.p[b] = list[b]->M; Gs.p[b] = list[b]->G; }
+  const int g_mode = (a0->g_dtype == DION_BF16) ? ADD_BF16 : ADD_F32;
+  __nv_bfloat16* bh = pair ? reinterpret_cast<__nv_bfloat16*>(s.ws + s.L.Bp) : nullptr;
+  __nv_bfloat16* bl = pair ? bh + m * n : nullptr;
+  const dim3 grid((unsigned)grid_for(c, m * n / 4), (unsigned)s.nb);
+  if (vec) launch_pdl(k_form_b32_chain<true>, grid, dim3(256), 0, s.st, Ms, a0->ldm, Gs, a0->ldg, g_mode, m, n, s.ws + s.L.B32, bh, bl, s.wstride);
+  else launch_pdl(k_form_b32_chain<false>, grid, dim3(256), 0, s.st, Ms, a0->ldm, Gs, a0->ldg, g_mode, m, n, s.ws + s.L.B32, bh, bl, s.wstride);
+  DION_CHECK_LAUNCH(c);
+  return DION_OK;
+}
+
 // The product itself: U (prow x r, dense) is split into the panel buffer `upair`; the pair of M + G must be in place.
 int r_pairs(StepCtx& s, int b, const dion_matrix* a, bool tr, const float* U, float* upair, float* out, const int* skip,
-            GemmArgs* defer = nullptr) {   // defer: the product is handed back instead of launched
+            GemmArgs* defer = nullptr, bool split_done = false) {   // defer: the product is handed back instead of launched
   dion_ctx* c = s.c;
   const i64 m = a->m, n = a->n, r = a->r;
   const i64 prow = tr ? n : m, qrow = tr ? m : n;
   __nv_bfloat16* uh = reinterpret_cast<__nv_bfloat16*>(upair);
   __nv_bfloat16* ul = uh + prow * r;
-  launch_pdl(k_split_bf16, dim3((unsigned)grid_for(c, prow * r / 8)), dim3(256), 0, s.st, U, r, prow, r, uh, ul, skip);
-  DION_CHECK_LAUNCH(c);
+  if (!split_done) {      // (the step splits U for the whole chain beforehand)
+    launch_pdl(k_split_bf16, dim3((unsigned)grid_for(c, prow * r / 8)), dim3(256), 0, s.st, U, r, prow, r, uh, ul, skip);
+    DION_CHECK_LAUNCH(c);
+  }
   __nv_bfloat16* bh = reinterpret_cast<__nv_bfloat16*>(s.W(b, s.L.Bp));
   GemmArgs w = gemm_args();
   w.M = qrow; w.N = r; w.K = prow;
@@ -1067,6 +1174,14 @@ bool x_single_pass(const StepCtx& s, const dion_matrix* a, const float* F1, i64 
 // TF32 passes instead of three.  Otherwise the 3xTF32 / FMA product of the fp32 factors.
 // sum32 != nullptr: M + G comes from scratch (C = sum32 - beta acc); else C = M + G - beta acc with the caller's G.
 // ready1 / ready2: that factor's pair already sits in p1 / p2 (the step splits U for R).
+bool ef_on_pairs(const StepCtx& s, const dion_matrix* a, const float* F1, i64 ld1, const float* F2, i64 ld2, const float* sum32) {
+  const i64 m = a->m, n = a->n, r = a->r;
+  return s.tensor && s.c->cfg.precision == DION_PREC_FP32 && m >= 128 && n >= 64 && r >= 64 && m % 8 == 0 &&
+         n % 8 == 0 && r % 8 == 0 && !((uintptr_t)a->M & 15) && a->ldm % 4 == 0 && !((uintptr_t)F1 & 15) &&
+         ld1 % 4 == 0 && !((uintptr_t)F2 & 15) && ld2 % 4 == 0 &&
+         (sum32 != nullptr || (!((uintptr_t)a->G & 15) && a->ldg % ((a->g_dtype == DION_BF16) ? 8 : 4) == 0));
+}
+
 int ef_update(StepCtx& s, int b, const dion_matrix* a, const float* F1, i64 ld1, const float* F2, i64 ld2, float* p1,
               float* p2, const float* sum32, const int* skip, bool ready1 = false, bool ready2 = false,
               GemmArgs* defer = nullptr) {
@@ -1074,10 +1189,7 @@ int ef_update(StepCtx& s, int b, const dion_matrix* a, const float* F1, i64 ld1,
   const i64 m = a->m, n = a->n, r = a->r;
   GemmArgs e = gemm_args();
   e.M = m; e.N = n; e.K = r;
-  const bool pairs = s.tensor && c->cfg.precision == DION_PREC_FP32 && m >= 128 && n >= 64 && r >= 64 && m % 8 == 0 &&
-                     n % 8 == 0 && r % 8 == 0 && !((uintptr_t)a->M & 15) && a->ldm % 4 == 0 && !((uintptr_t)F1 & 15) &&
-                     ld1 % 4 == 0 && !((uintptr_t)F2 & 15) && ld2 % 4 == 0 &&
-                     (sum32 != nullptr || (!((uintptr_t)a->G & 15) && a->ldg % ((a->g_dtype == DION_BF16) ? 8 : 4) == 0));
+  const bool pairs = ef_on_pairs(s, a, F1, ld1, F2, ld2, sum32);
   if (pairs) {
     __nv_bfloat16* h1 = reinterpret_cast<__nv_bfloat16*>(p1);
     __nv_bfloat16* l1 = h1 + m * r;
@@ -1108,16 +1220,19 @@ int ef_update(StepCtx& s, int b, const dion_matrix* a, const float* F1, i64 ld1,
 }
 
 int x_update(StepCtx& s, int b, const dion_matrix* a, const float* F1, i64 ld1, const float* F2, i64 ld2, float* r1,
-             float* r2, float alpha, const int* skip, const float* alpha_dev = nullptr, GemmArgs* defer = nullptr) {
+             float* r2, float alpha, const int* skip, const float* alpha_dev = nullptr, GemmArgs* defer = nullptr,
+             bool rounded = false) {   // rounded: r1 and r2 already hold the rounded factors
   dion_ctx* c = s.c;
   const i64 m = a->m, n = a->n, r = a->r;
   GemmArgs x = gemm_args();
   x.M = m; x.N = n; x.K = r;
   if (x_single_pass(s, a, F1, ld1, F2, ld2)) {
-    launch_pdl(k_round_tf32, dim3((unsigned)grid_for(c, m * r / 4)), dim3(256), 0, s.st, F1, ld1, m, r, r1, skip);
-    DION_CHECK_LAUNCH(c);
-    launch_pdl(k_round_tf32, dim3((unsigned)grid_for(c, n * r / 4)), dim3(256), 0, s.st, F2, ld2, n, r, r2, skip);
-    DION_CHECK_LAUNCH(c);
+    if (!rounded) {
+      launch_pdl(k_round_tf32, dim3((unsigned)grid_for(c, m * r / 4)), dim3(256), 0, s.st, F1, ld1, m, r, r1, skip);
+      DION_CHECK_LAUNCH(c);
+      launch_pdl(k_round_tf32, dim3((unsigned)grid_for(c, n * r / 4)), dim3(256), 0, s.st, F2, ld2, n, r, r2, skip);
+      DION_CHECK_LAUNCH(c);
+    }
     x.tf32x1 = 1;
     x.A = r1; x.a_si = r; x.a_sk = 1;
     x.B = r2; x.b_sk = 1; x.b_sn = r;
@@ -1193,6 +1308,19 @@ int step_batch(dion_ctx* c, const dion_matrix* const* list, int nb, float lr, cu
   const i64 pin_off = panel_offset(s, r, (m < n) ? m : n);
   {
   PhaseScope ps(c, st, DION_PHASE_P);
+  // elementwise preparation for the whole chain: M + G (and its pair), the pair of Q where P takes pairs
+  const float* srcs[MAX_CHAIN];
+  i64 lds[MAX_CHAIN];
+  if (b32) DION_TRY(form_sum_chain(s, list, bpair));
+  bool q_split = false;
+  if (b32 && ppair) {
+    bool all_ok = true;
+    for (int b = 0; b < nb; ++b) {
+      all_ok = all_ok && !((uintptr_t)list[b]->Q & 15) && list[b]->ldq % 4 == 0;
+      srcs[b] = (const float*)list[b]->Q; lds[b] = list[b]->ldq;
+    }
+    if (all_ok) { DION_TRY(split_chain(s, srcs, lds, qrow, r, s.L.S16, nullptr)); q_split = true; }
+  }
   for (int b = 0; b < nb; ++b) {
     const dion_matrix* a = list[b];
     GemmArgs p = gemm_args();
@@ -1210,19 +1338,19 @@ int step_batch(dion_ctx* c, const dion_matrix* const* list, int nb, float lr, cu
       p.A = (const float*)bf(b, s.L.B16); p.a_si = tr ? 1 : n; p.a_sk = tr ? n : 1;
       p.B = (const float*)bf(b, s.L.Q16); p.b_sk = r; p.b_sn = 1;
     } else if (b32 && ppair && !((uintptr_t)a->Q & 15) && a->ldq % 4 == 0) {
-      DION_TRY(form_sum(s, b, a, true));
       __nv_bfloat16* qh = reinterpret_cast<__nv_bfloat16*>(s.W(b, s.L.S16));
       __nv_bfloat16* ql = qh + qrow * r;
-      launch_pdl(k_split_bf16, dim3((unsigned)grid_for(c, qrow * r / 8)), dim3(256), 0, st, (const float*)a->Q, a->ldq, qrow, r, qh, ql,
-                 (const int*)nullptr);
-      DION_CHECK_LAUNCH(c);
+      if (!q_split) {
+        launch_pdl(k_split_bf16, dim3((unsigned)grid_for(c, qrow * r / 8)), dim3(256), 0, st, (const float*)a->Q, a->ldq, qrow, r, qh, ql,
+                   (const int*)nullptr);
+        DION_CHECK_LAUNCH(c);
+      }
       __nv_bfloat16* bh = reinterpret_cast<__nv_bfloat16*>(s.W(b, s.L.Bp));
       p.ab16 = 1;
       p.A = (const float*)bh; p.A16lo = bh + m * n; p.a_si = tr ? 1 : n; p.a_sk = tr ? n : 1;
       p.B = (const float*)qh; p.B16lo = ql; p.b_sk = r; p.b_sn = 1;
       any_pair = true;
     } else if (b32) {
-      DION_TRY(form_sum(s, b, a, bpair));
       p.A = s.W(b, s.L.B32); p.a_si = tr ? 1 : n; p.a_sk = tr ? n : 1;
       p.B = (const float*)a->Q; p.b_sk = a->ldq; p.b_sn = 1;
     } else {
@@ -1266,6 +1394,13 @@ int step_batch(dion_ctx* c, const dion_matrix* const* list, int nb, float lr, cu
   // R = (M + G)^T U   (transposed form: (M + G) U)
   {
   PhaseScope ps(c, st, DION_PHASE_R);
+  const i64 other_off = (U_off == s.L.P0) ? s.L.P1 : s.L.P0;
+  if (!d16 && bpair) {   // U as a bf16 pair in the other panel buffer, for the whole chain
+    const float* srcs[MAX_CHAIN];
+    i64 lds[MAX_CHAIN];
+    for (int b = 0; b < nb; ++b) { srcs[b] = s.W(b, U_off); lds[b] = r; }
+    DION_TRY(split_chain(s, srcs, lds, prow, r, other_off, s.os + OS_FAIL));
+  }
   for (int b = 0; b < nb; ++b) {
     const dion_matrix* a = list[b];
     GemmArgs w = gemm_args();
@@ -1277,8 +1412,7 @@ int step_batch(dion_ctx* c, const dion_matrix* const* list, int nb, float lr, cu
       w.B = (const float*)bf(b, s.L.U16); w.b_sk = r; w.b_sn = 1;
     } else if (bpair) {
       // U as a bf16 pair in the other panel buffer (the error feedback reuses it)
-      DION_TRY(r_pairs(s, b, a, tr, s.W(b, U_off), s.W(b, U_off == s.L.P0 ? s.L.P1 : s.L.P0), s.W(b, s.L.R), s.OS(b) + OS_FAIL,
-                       &group[b]));
+      DION_TRY(r_pairs(s, b, a, tr, s.W(b, U_off), s.W(b, other_off), s.W(b, s.L.R), s.OS(b) + OS_FAIL, &group[b], true));
       continue;
     } else if (b32) {
       w.A = s.W(b, s.L.B32); w.a_si = tr ? n : 1; w.a_sk = tr ? 1 : n;
@@ -1297,6 +1431,27 @@ int step_batch(dion_ctx* c, const dion_matrix* const* list, int nb, float lr, cu
   // M <- (M + G) - (1 - mu) U R^T   (transposed form: R U^T)
   {
   PhaseScope ps(c, st, DION_PHASE_EF);
+  const i64 other_off = (U_off == s.L.P0) ? s.L.P1 : s.L.P0;
+  bool ef_split = false;      // the factors' pairs are made for the whole chain when every matrix takes pairs
+  if (!d16) {
+    const float* srcs[MAX_CHAIN];
+    i64 lds[MAX_CHAIN];
+    bool all_pairs = true;
+    for (int b = 0; b < nb; ++b) {
+      const float* sum32 = b32 ? s.W(b, s.L.B32) : nullptr;
+      all_pairs = all_pairs && (tr ? ef_on_pairs(s, list[b], s.W(b, s.L.R), r, s.W(b, U_off), r, sum32)
+                                   : ef_on_pairs(s, list[b], s.W(b, U_off), r, s.W(b, s.L.R), r, sum32));
+    }
+    if (all_pairs) {
+      for (int b = 0; b < nb; ++b) { srcs[b] = s.W(b, s.L.R); lds[b] = r; }
+      DION_TRY(split_chain(s, srcs, lds, qrow, r, s.L.S16, s.os + OS_FAIL));
+      if (!bpair) {
+        for (int b = 0; b < nb; ++b) srcs[b] = s.W(b, U_off);
+        DION_TRY(split_chain(s, srcs, lds, prow, r, other_off, s.os + OS_FAIL));
+      }
+      ef_split = true;
+    }
+  }
   for (int b = 0; b < nb; ++b) {
     const dion_matrix* a = list[b];
     if (d16) {
@@ -1319,8 +1474,8 @@ int step_batch(dion_ctx* c, const dion_matrix* const* list, int nb, float lr, cu
     const float* Uf = s.W(b, U_off);
     const float* Rf = s.W(b, s.L.R);
     const float* sum32 = b32 ? s.W(b, s.L.B32) : nullptr;
-    if (tr) DION_TRY(ef_update(s, b, a, Rf, r, Uf, r, sbuf, other, sum32, s.OS(b) + OS_FAIL, false, bpair, &group[b]));
-    else DION_TRY(ef_update(s, b, a, Uf, r, Rf, r, other, sbuf, sum32, s.OS(b) + OS_FAIL, bpair, false, &group[b]));
+    if (tr) DION_TRY(ef_update(s, b, a, Rf, r, Uf, r, sbuf, other, sum32, s.OS(b) + OS_FAIL, ef_split, bpair || ef_split, &group[b]));
+    else DION_TRY(ef_update(s, b, a, Uf, r, Rf, r, other, sbuf, sum32, s.OS(b) + OS_FAIL, bpair || ef_split, ef_split, &group[b]));
   }
   DION_TRY(launch_gemm_group(s, group));
   }
@@ -1328,16 +1483,32 @@ int step_batch(dion_ctx* c, const dion_matrix* const* list, int nb, float lr, cu
   // Q <- ColNorm(R)
   {
   PhaseScope ps(c, st, DION_PHASE_COLNORM);
-  for (int b = 0; b < nb; ++b) {
-    const dion_matrix* a = list[b];
-    DION_TRY(colnorm(s, b, s.W(b, s.L.R), qrow, r, (float*)a->Q, a->ldq, a->colnorm_out));
-  }
+  DION_TRY(colnorm_chain(s, list, qrow, r));
   }
 
   // X <- X - lr sqrt(m/n) U Q^T   (transposed form: Q U^T)
   {
   PhaseScope ps(c, st, DION_PHASE_X);
   const float x_alpha = (x_scale != nullptr) ? 1.f : lr * sqrtf((float)((double)m / (double)n));
+  const i64 other_off = (U_off == s.L.P0) ? s.L.P1 : s.L.P0;
+  bool x_rounded = false;     // the rounded factors are made for the whole chain when every matrix takes the single pass
+  if (!d16) {
+    const float* srcs[MAX_CHAIN];
+    i64 lds[MAX_CHAIN];
+    bool all_one = true;
+    for (int b = 0; b < nb; ++b) {
+      const dion_matrix* a = list[b];
+      all_one = all_one && (tr ? x_single_pass(s, a, (const float*)a->Q, a->ldq, s.W(b, U_off), r)
+                               : x_single_pass(s, a, s.W(b, U_off), r, (const float*)a->Q, a->ldq));
+    }
+    if (all_one) {
+      for (int b = 0; b < nb; ++b) { srcs[b] = s.W(b, U_off); lds[b] = r; }
+      DION_TRY(round_chain(s, srcs, lds, prow, r, other_off, s.os + OS_FAIL));
+      for (int b = 0; b < nb; ++b) { srcs[b] = (const float*)list[b]->Q; lds[b] = list[b]->ldq; }
+      DION_TRY(round_chain(s, srcs, lds, qrow, r, s.L.R, s.os + OS_FAIL));
+      x_rounded = true;
+    }
+  }
   for (int b = 0; b < nb; ++b) {
     const dion_matrix* a = list[b];
     if (d16) {
@@ -1358,8 +1529,8 @@ int step_batch(dion_ctx* c, const dion_matrix* const* list, int nb, float lr, cu
     float* rbuf = s.W(b, s.L.R);
     const float* Uf = s.W(b, U_off);
     const float* Qf = (const float*)a->Q;
-    if (tr) DION_TRY(x_update(s, b, a, Qf, a->ldq, Uf, r, rbuf, other, x_alpha, s.OS(b) + OS_FAIL, x_scale, &group[b]));
-    else DION_TRY(x_update(s, b, a, Uf, r, Qf, a->ldq, other, rbuf, x_alpha, s.OS(b) + OS_FAIL, x_scale, &group[b]));
+    if (tr) DION_TRY(x_update(s, b, a, Qf, a->ldq, Uf, r, rbuf, other, x_alpha, s.OS(b) + OS_FAIL, x_scale, &group[b], x_rounded));
+    else DION_TRY(x_update(s, b, a, Uf, r, Qf, a->ldq, other, rbuf, x_alpha, s.OS(b) + OS_FAIL, x_scale, &group[b], x_rounded));
   }
   DION_TRY(launch_gemm_group(s, group));
   launch_pdl(k_finish_step, dim3((unsigned)(nb)), dim3(1), 0, st, s.flag, c->dev_ints + 1);
@@ -1872,7 +2043,7 @@ int dion_shard_factor(dion_ctx* ctx, const dion_matrix* a, int64_t n_total, cons
   colnorm_plan(a->n, a->r, ctx->sm_count, &chunks, &per);
   float* part = s.W(0, s.L.cn_part);
   dim3 grid((unsigned)((a->r + 127) / 128), (unsigned)chunks);
-  launch_pdl(k_colsumsq_partial, grid, dim3(128), 0, st, (const float*)W, a->r, a->n, a->r, per, part, flag);
+  launch_pdl(k_colsumsq_partial, grid, dim3(128), 0, st, (const float*)W, a->r, a->n, a->r, per, part, (const int*)flag, (i64)0);
   DION_CHECK_LAUNCH(ctx);
   launch_pdl(k_colsumsq_finish, dim3((unsigned)((a->r + 127) / 128)), dim3(128), 0, st, (const float*)part, chunks, a->r, colsumsq, flag);
   DION_CHECK_LAUNCH(ctx);
@@ -1894,7 +2065,7 @@ int dion_shard_finish(dion_ctx* ctx, const dion_matrix* a, int64_t n_total, cons
     colnorm_plan(n, r, ctx->sm_count, &chunks, &per);
     dim3 grid((unsigned)((r + 127) / 128), (unsigned)chunks);
     launch_pdl(k_colnorm_apply, grid, dim3(128), 0, st, W, r, n, r, per, 1, colsumsq, ctx->cfg.eps, (float*)a->Q, a->ldq,
-               s.W(0, s.L.d), a->colnorm_out, ctx->dev_ints, flag);
+               s.W(0, s.L.d), a->colnorm_out, ctx->dev_ints, (const int*)flag, (i64)0, ChainPtrs(), ChainPtrs());
     DION_CHECK_LAUNCH(ctx);
   }
   // X <- X - lr sqrt(m / n_total) U Q^T on the shard's columns

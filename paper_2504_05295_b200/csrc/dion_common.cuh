@@ -29,6 +29,9 @@ enum : int { TRI_FULL = 0, TRI_LOWER = 1 };
 // C(i,j) = C[i*ldc + j]
 constexpr int GEMM_TAB_MAX = 64;   // most matrices in one batched tensor-engine launch with per-matrix output pointers
 
+// Per-matrix pointers of a chain for the elementwise kernels that run once over all its matrices.
+struct ChainPtrs { const void* p[GEMM_TAB_MAX]; };
+
 struct GemmArgs {
   i64 M, N, K;
   const float* A; i64 a_si, a_sk;

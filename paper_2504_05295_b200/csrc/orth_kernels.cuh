@@ -925,9 +925,11 @@ __global__ void k_copy_block(const float* __restrict__ src, i64 lds, float* __re
 // grid = (ceil(r/128), chunks); 128 threads, one column each (coalesced rows).
 __global__ void __launch_bounds__(128) k_colsumsq_partial(const float* __restrict__ R, i64 ld, i64 n, i64 r,
                                                           i64 rows_per_chunk, float* __restrict__ part,
-                                                          const int* __restrict__ skip_flag) {
+                                                          const int* __restrict__ skip_flag, i64 wstride) {
+  // blockIdx.z: the matrix of a chain (R and part wstride floats apart, skip flags a state slot apart)
   pdl_enter();
-  if (skip_flag != nullptr && *skip_flag != 0) return;
+  if (skip_flag != nullptr && skip_flag[(i64)blockIdx.z * OS_SLOT_INTS] != 0) return;
+  R += (i64)blockIdx.z * wstride; part += (i64)blockIdx.z * wstride;
   const i64 j = (i64)blockIdx.x * 128 + threadIdx.x;
   if (j >= r) return;
   const i64 i0 = (i64)blockIdx.y * rows_per_chunk;
@@ -961,9 +963,17 @@ __global__ void __launch_bounds__(128) k_colnorm_apply(const float* __restrict__
                                                        float* __restrict__ Q, i64 ldq,
                                                        float* __restrict__ d_ws, float* __restrict__ d_out,
                                                        int* __restrict__ status,
-                                                       const int* __restrict__ skip_flag) {
+                                                       const int* __restrict__ skip_flag, i64 wstride,
+                                                       const ChainPtrs Qs, const ChainPtrs ds) {
+  // wstride != 0: one launch over a chain (blockIdx.z): R, part and d_ws in the scratch slices, Q and d_out from
+  // the pointer tables
   pdl_enter();
-  if (skip_flag != nullptr && *skip_flag != 0) return;
+  if (skip_flag != nullptr && skip_flag[(i64)blockIdx.z * OS_SLOT_INTS] != 0) return;
+  if (wstride != 0) {
+    R += (i64)blockIdx.z * wstride; part += (i64)blockIdx.z * wstride; d_ws += (i64)blockIdx.z * wstride;
+    Q = reinterpret_cast<float*>(const_cast<void*>(Qs.p[blockIdx.z]));
+    d_out = reinterpret_cast<float*>(const_cast<void*>(ds.p[blockIdx.z]));
+  }
   const i64 j = (i64)blockIdx.x * 128 + threadIdx.x;
   if (j >= r) return;
   float s = 0.f;
