@@ -151,8 +151,10 @@ __global__ void __launch_bounds__(256) k_to_bf16(const float* __restrict__ src, 
 
 // hi = bf16(src), lo = bf16(src - hi): src ~ hi + lo to 16 significant bits.  rows x cols (cols a multiple of 8,
 // src rows 16-byte aligned), hi and lo dense.  skip_flag (optional): nothing is written when *skip_flag != 0.
+// copy (optional): src also as a dense fp32 array
 __device__ __forceinline__ void split_bf16_body(const float* __restrict__ src, i64 lds, i64 rows, i64 cols,
-                                                __nv_bfloat16* __restrict__ hi, __nv_bfloat16* __restrict__ lo) {
+                                                __nv_bfloat16* __restrict__ hi, __nv_bfloat16* __restrict__ lo,
+                                                float* __restrict__ copy = nullptr) {
   const i64 per_row = cols / 8;
   const i64 total = rows * per_row;
   for (i64 e = (i64)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (i64)gridDim.x * blockDim.x) {
@@ -171,6 +173,10 @@ __device__ __forceinline__ void split_bf16_body(const float* __restrict__ src, i
     ol.x = pack_bf16x2(l[0], l[1]); ol.y = pack_bf16x2(l[2], l[3]); ol.z = pack_bf16x2(l[4], l[5]); ol.w = pack_bf16x2(l[6], l[7]);
     *reinterpret_cast<uint4*>(hi + i * cols + c) = oh;
     *reinterpret_cast<uint4*>(lo + i * cols + c) = ol;
+    if (copy != nullptr) {
+      *reinterpret_cast<float4*>(copy + i * cols + c) = a;
+      *(reinterpret_cast<float4*>(copy + i * cols + c) + 1) = b;
+    }
   }
 }
 __global__ void __launch_bounds__(256) k_split_bf16(const float* __restrict__ src, i64 lds, i64 rows, i64 cols,
@@ -184,11 +190,13 @@ __global__ void __launch_bounds__(256) k_split_bf16(const float* __restrict__ sr
 // apart in the scratch slices, skip flags `skip_stride` ints apart.
 __global__ void __launch_bounds__(256) k_split_bf16_chain(const ChainPtrs srcs, i64 lds, i64 rows, i64 cols,
                                                           __nv_bfloat16* __restrict__ hi, __nv_bfloat16* __restrict__ lo,
-                                                          i64 ostride, const int* __restrict__ skip_flag, i64 skip_stride) {
+                                                          i64 ostride, const int* __restrict__ skip_flag, i64 skip_stride,
+                                                          float* __restrict__ copy) {
   pdl_enter();
   const i64 b = blockIdx.y;
   if (skip_flag != nullptr && skip_flag[b * skip_stride] != 0) return;
-  split_bf16_body(reinterpret_cast<const float*>(srcs.p[b]), lds, rows, cols, hi + 2 * b * ostride, lo + 2 * b * ostride);
+  split_bf16_body(reinterpret_cast<const float*>(srcs.p[b]), lds, rows, cols, hi + 2 * b * ostride, lo + 2 * b * ostride,
+                  copy != nullptr ? copy + b * ostride : nullptr);
 }
 
 // out = src with every value rounded to the nearest TF32 number (10 explicit mantissa bits, ties away

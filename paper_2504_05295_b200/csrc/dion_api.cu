@@ -53,6 +53,7 @@ struct Layout {
   i64 fb_part, fb_h, fb_n;  // fallback kernel: partial dot products (SMs x r), their sums (r), partial norms (SMs)
   i64 probe_y, probe_part;  // CholeskyQR2's orthogonality probe: U1 z (rows x NPROBE), partial U1^T (U1 z)
   i64 Bp;                   // fp32 mode, M + G in scratch: the same sum as a bf16 (hi, lo) pair (m x n x 2 bf16) for R; 0: none
+  i64 Qc;                   // fp32 mode, large matrices: dense fp32 copy of Q for the chain-wide recomputation of P (0: none)
   i64 S16;                  // fp32 mode: the bf16 (hi, lo) pair of the error feedback's second factor (max(m,n) x r x 2 bf16)
   i64 part_floats;
   int cn_chunks;
@@ -172,6 +173,8 @@ Layout make_layout(const dion_ctx* c, i64 m, i64 n, i64 r) {
     if (m % 8 == 0 && n % 8 == 0 && r % 8 == 0) { L.Bp = o; o += align64(m * n); }
   }
   L.Psave = L.fb_part = L.fb_h = L.fb_n = 0;
+  L.Qc = 0;
+  if (L.Bp > 0 && (double)m * (double)n * (double)r >= P_PAIR_MIN_MNR) { L.Qc = o; o += align64(big * r); }
   L.S16 = o; o += align64(big * r);
   L.probe_y = o; o += align64(big * NPROBE);
   L.probe_part = o; o += align64((i64)(L.cn_chunks + 1) * r * NPROBE);
@@ -430,7 +433,8 @@ int launch_gemm_group(StepCtx& s, const std::vector<GemmArgs>& v) {
 // One-time opt-in to the dynamic shared memory of the kernels that need more than 48 KB.
 int configure_kernels() {
   if (umma_configure() != DION_OK) return DION_ERR_CUDA;
-  if (cudaFuncSetAttribute(k_chol_step, cudaFuncAttributeMaxDynamicSharedMemorySize, CHOL_STEP_SMEM) != cudaSuccess) {
+  if (cudaFuncSetAttribute(k_probe_y4, cudaFuncAttributeMaxDynamicSharedMemorySize, PY_SMEM) != cudaSuccess ||
+      cudaFuncSetAttribute(k_chol_step, cudaFuncAttributeMaxDynamicSharedMemorySize, CHOL_STEP_SMEM) != cudaSuccess) {
     cudaGetLastError();
     return DION_ERR_CUDA;
   }
@@ -627,13 +631,20 @@ int probe(StepCtx& s, i64 off, i64 rows, i64 r, int phase) {
   int chunks; i64 per;
   colnorm_plan(rows, r, c->sm_count, &chunks, &per);
   const int* keep = (phase == PROBE_AFTER_REDO) ? (const int*)(s.os + OS_DONE) : nullptr;
-  launch_pdl(k_probe_y, dim3((unsigned)grid_for(c, rows * 32), (unsigned)s.nb), dim3(256), 0, s.st, (const float*)(s.ws + off), r,
-             rows, r, s.ws + s.L.probe_y, s.wstride, keep);
+  if (r % 4 == 0 && r >= 128) {
+    i64 blocks = (rows + 31) / 32;          // a block of 8 warps takes 32 rows at a time
+    if (blocks > 2 * (i64)c->sm_count) blocks = 2 * (i64)c->sm_count;
+    launch_pdl(k_probe_y4, dim3((unsigned)blocks, (unsigned)s.nb), dim3(256), (size_t)PY_SMEM, s.st, (const float*)(s.ws + off), r, rows, r,
+               s.ws + s.L.probe_y, s.wstride, keep);
+  } else {
+    launch_pdl(k_probe_y, dim3((unsigned)grid_for(c, rows * 32), (unsigned)s.nb), dim3(256), 0, s.st, (const float*)(s.ws + off), r,
+               rows, r, s.ws + s.L.probe_y, s.wstride, keep);
+  }
   DION_CHECK_LAUNCH(c);
   launch_pdl(k_probe_w, dim3((unsigned)((r + 127) / 128), (unsigned)chunks, (unsigned)s.nb), dim3(128), 0, s.st,
              (const float*)(s.ws + off), r, rows, r, per, (const float*)(s.ws + s.L.probe_y), s.ws + s.L.probe_part, s.wstride, keep);
   DION_CHECK_LAUNCH(c);
-  launch_pdl(k_probe_decide, dim3((unsigned)s.nb), dim3(256), 0, s.st, (const float*)(s.ws + s.L.probe_part), chunks, r, s.os,
+  launch_pdl(k_probe_decide, dim3((unsigned)s.nb), dim3(r >= 1024 ? 1024 : 256), 0, s.st, (const float*)(s.ws + s.L.probe_part), chunks, r, s.os,
              ORTH_TAU_F, c->dev_ints + 2, s.wstride, phase);
   DION_CHECK_LAUNCH(c);
   return DION_OK;
@@ -980,7 +991,9 @@ int colnorm_chain(StepCtx& s, const dion_matrix* const* list, i64 rows, i64 r) {
 
 // hi / lo bf16 pair of src[b] (rows x cols, leading dimension ld[b]) into the scratch slices at out_off.
 // skip0: the flag of matrix 0 (a state slot apart per matrix), or nullptr.
-int split_chain(StepCtx& s, const float* const* src, const i64* ld, i64 rows, i64 cols, i64 out_off, const int* skip0) {
+// copy_off >= 0 (chain launch only): a dense fp32 copy of the sources in the scratch slices too; *copied says whether it was made.
+int split_chain(StepCtx& s, const float* const* src, const i64* ld, i64 rows, i64 cols, i64 out_off, const int* skip0,
+                i64 copy_off = -1, bool* copied = nullptr) {
   dion_ctx* c = s.c;
   bool one = s.nb > 1 && s.nb <= GEMM_TAB_MAX && c->chain_batch;
   for (int b = 1; b < s.nb && one; ++b) one = ld[b] == ld[0];
@@ -990,10 +1003,12 @@ int split_chain(StepCtx& s, const float* const* src, const i64* ld, i64 rows, i6
     for (int b = 0; b < s.nb; ++b) t.p[b] = src[b];
     __nv_bfloat16* hi = reinterpret_cast<__nv_bfloat16*>(s.ws + out_off);
     launch_pdl(k_split_bf16_chain, dim3(gx, (unsigned)s.nb), dim3(256), 0, s.st, t, ld[0], rows, cols, hi, hi + rows * cols, s.wstride, skip0,
-               (i64)OS_SLOT_INTS);
+               (i64)OS_SLOT_INTS, copy_off >= 0 ? s.ws + copy_off : (float*)nullptr);
     DION_CHECK_LAUNCH(c);
+    if (copied != nullptr) *copied = copy_off >= 0;
     return DION_OK;
   }
+  if (copied != nullptr) *copied = false;
   for (int b = 0; b < s.nb; ++b) {
     __nv_bfloat16* hi = reinterpret_cast<__nv_bfloat16*>(s.W(b, out_off));
     launch_pdl(k_split_bf16, dim3(gx), dim3(256), 0, s.st, src[b], ld[b], rows, cols, hi, hi + rows * cols,
@@ -1306,6 +1321,7 @@ int step_batch(dion_ctx* c, const dion_matrix* const* list, int nb, float lr, cu
 
   // P = (M + G) Q   (transposed form: (M + G)^T Q)
   const i64 pin_off = panel_offset(s, r, (m < n) ? m : n);
+  bool q_copied = false;      // a dense copy of every Q of the chain sits in scratch (for the recomputation of P)
   {
   PhaseScope ps(c, st, DION_PHASE_P);
   // elementwise preparation for the whole chain: M + G (and its pair), the pair of Q where P takes pairs
@@ -1319,7 +1335,7 @@ int step_batch(dion_ctx* c, const dion_matrix* const* list, int nb, float lr, cu
       all_ok = all_ok && !((uintptr_t)list[b]->Q & 15) && list[b]->ldq % 4 == 0;
       srcs[b] = (const float*)list[b]->Q; lds[b] = list[b]->ldq;
     }
-    if (all_ok) { DION_TRY(split_chain(s, srcs, lds, qrow, r, s.L.S16, nullptr)); q_split = true; }
+    if (all_ok) { DION_TRY(split_chain(s, srcs, lds, qrow, r, s.L.S16, nullptr, s.L.Qc > 0 ? s.L.Qc : -1, &q_copied)); q_split = true; }
   }
   for (int b = 0; b < nb; ++b) {
     const dion_matrix* a = list[b];
@@ -1371,17 +1387,19 @@ int step_batch(dion_ctx* c, const dion_matrix* const* list, int nb, float lr, cu
   {
   PhaseScope ps(c, st, DION_PHASE_ORTH);
   const std::function<int()> redo = [&]() -> int {
+    std::vector<GemmArgs> again((size_t)nb);
     for (int b = 0; b < nb; ++b) {
       const dion_matrix* a = list[b];
       GemmArgs p = gemm_args();
       p.M = prow; p.N = r; p.K = qrow;
       p.A = s.W(b, s.L.B32); p.a_si = tr ? 1 : n; p.a_sk = tr ? n : 1;
-      p.B = (const float*)a->Q; p.b_sk = a->ldq; p.b_sn = 1;
+      if (q_copied) { p.B = s.W(b, s.L.Qc); p.b_sk = r; p.b_sn = 1; }     // (the same values: one launch over the chain)
+      else { p.B = (const float*)a->Q; p.b_sk = a->ldq; p.b_sn = 1; }
       p.C = s.W(b, pin_off); p.ldc = r; p.epi = EPI_STORE;
       p.skip_flag = s.OS(b) + OS_DONE;
-      DION_TRY(launch_gemm(s, p, b));
+      again[b] = p;
     }
-    return DION_OK;
+    return launch_gemm_group(s, again);
   };
   s.in_orth = true;
   s.redo_p = any_pair ? &redo : nullptr;
@@ -2216,7 +2234,7 @@ bool preload_kernels() {
   ok = ok && touch_kernel(k_gemm_simt<128, 128, 8, 8, 8>) && touch_kernel(k_gemm_simt<64, 64, 16, 4, 4>);
   ok = ok && touch_kernel(k_splitk_reduce) && touch_kernel(k_round_begin) && touch_kernel(k_potrf_diag);
   ok = ok && touch_kernel(k_chol_step) && touch_kernel(k_inv_finish) && touch_kernel(k_round_end);
-  ok = ok && touch_kernel(k_probe_y) && touch_kernel(k_probe_w) && touch_kernel(k_probe_decide) && touch_kernel(k_reset_rounds);
+  ok = ok && touch_kernel(k_probe_y) && touch_kernel(k_probe_y4) && touch_kernel(k_probe_w) && touch_kernel(k_probe_decide) && touch_kernel(k_reset_rounds);
   ok = ok && touch_kernel(k_orth_finish) && touch_kernel(k_cgs_fallback) && touch_kernel(k_copy_block);
   ok = ok && touch_kernel(k_colsumsq_partial) && touch_kernel(k_colnorm_apply) && touch_kernel(k_copy_panel);
   ok = ok && touch_kernel(k_latch_flag) && touch_kernel(k_finish_step) && touch_kernel(k_hh_reflector);

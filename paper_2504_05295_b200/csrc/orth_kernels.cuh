@@ -629,6 +629,71 @@ __global__ void __launch_bounds__(256) k_probe_y(const float* __restrict__ U, i6
   }
 }
 
+// The same for r a multiple of 4 (16-byte aligned rows): the +-1 entries of the probe vectors are hashed once per
+// CTA and column block into a shared-memory table of floats instead of once per matrix element (the hash made the
+// plain kernel ALU bound at a seventh of HBM speed), and a warp takes four rows at a time so that one read of a
+// column's eight signs serves four elements.  Lane l owns columns 128 t + 4 l .. + 3 of a block of PY_COLS
+// columns; wider panels add their later column blocks into Y (the same warp owns a row throughout).
+constexpr int PY_COLS = 2048;
+constexpr int PY_SMEM = PY_COLS * NPROBE * 4;
+__global__ void __launch_bounds__(256) k_probe_y4(const float* __restrict__ U, i64 ld, i64 rows, i64 r,
+                                                  float* __restrict__ Y, i64 wstride, const int* __restrict__ keep) {
+  extern __shared__ float py_sign[];      // [column in block][probe]
+  pdl_enter();
+  if (keep != nullptr && keep[(i64)blockIdx.y * OS_SLOT_INTS] != 0) return;   // this panel's verdict stands
+  U += (i64)blockIdx.y * wstride; Y += (i64)blockIdx.y * wstride;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const i64 group0 = (i64)blockIdx.x * 8 + warp, groups = (i64)gridDim.x * 8;
+  for (i64 c0 = 0; c0 < r; c0 += PY_COLS) {
+    const int nc = (int)min((i64)PY_COLS, r - c0);
+    __syncthreads();
+    for (int e = threadIdx.x; e < nc * NPROBE; e += 256) py_sign[e] = probe_sign(c0 + e / NPROBE, e % NPROBE);
+    __syncthreads();
+    for (i64 g = group0; g * 4 < rows; g += groups) {
+      const i64 i0 = g * 4;
+      float acc[4][NPROBE];
+#pragma unroll
+      for (int q = 0; q < 4; ++q)
+#pragma unroll
+        for (int p = 0; p < NPROBE; ++p) acc[q][p] = 0.f;
+      for (int j = 4 * lane; j < nc; j += 128) {
+        float4 u[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q)
+          u[q] = (i0 + q < rows) ? *reinterpret_cast<const float4*>(U + (i0 + q) * ld + c0 + j) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+        for (int cc = 0; cc < 4; ++cc) {
+          const float4 s0 = *reinterpret_cast<const float4*>(py_sign + (j + cc) * NPROBE);
+          const float4 s1 = *reinterpret_cast<const float4*>(py_sign + (j + cc) * NPROBE + 4);
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            const float v = (cc == 0) ? u[q].x : (cc == 1) ? u[q].y : (cc == 2) ? u[q].z : u[q].w;
+            acc[q][0] = fmaf(v, s0.x, acc[q][0]); acc[q][1] = fmaf(v, s0.y, acc[q][1]);
+            acc[q][2] = fmaf(v, s0.z, acc[q][2]); acc[q][3] = fmaf(v, s0.w, acc[q][3]);
+            acc[q][4] = fmaf(v, s1.x, acc[q][4]); acc[q][5] = fmaf(v, s1.y, acc[q][5]);
+            acc[q][6] = fmaf(v, s1.z, acc[q][6]); acc[q][7] = fmaf(v, s1.w, acc[q][7]);
+          }
+        }
+      }
+#pragma unroll
+      for (int q = 0; q < 4; ++q)
+#pragma unroll
+        for (int p = 0; p < NPROBE; ++p) {
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) acc[q][p] += __shfl_xor_sync(0xffffffffu, acc[q][p], o);
+        }
+      if (lane < 4 && i0 + lane < rows) {
+        float* y = Y + (i0 + lane) * NPROBE;
+#pragma unroll
+        for (int p = 0; p < NPROBE; ++p) {
+          const float v = (lane == 0) ? acc[0][p] : (lane == 1) ? acc[1][p] : (lane == 2) ? acc[2][p] : acc[3][p];
+          y[p] = (c0 == 0) ? v : y[p] + v;
+        }
+      }
+    }
+  }
+}
+
 // part[chunk][j][p] = sum over the chunk's rows of U[i][j] Y[i][p].  grid = (ceil(r/128), chunks, matrices).
 __global__ void __launch_bounds__(128) k_probe_w(const float* __restrict__ U, i64 ld, i64 rows, i64 r,
                                                  i64 rows_per_chunk, const float* __restrict__ Y,
@@ -662,7 +727,7 @@ __global__ void __launch_bounds__(128) k_probe_w(const float* __restrict__ U, i6
 // too: the panel is recomputed before the fallback sees it); nothing is counted.  PROBE_AFTER_REDO: a panel that
 // passed PROBE_FAST keeps its verdict (one round); otherwise its recomputed first round is judged.
 enum : int { PROBE_CHECK = 0, PROBE_FAST = 1, PROBE_AFTER_REDO = 2 };
-__global__ void __launch_bounds__(256) k_probe_decide(const float* __restrict__ part, int chunks, i64 r,
+__global__ void __launch_bounds__(1024) k_probe_decide(const float* __restrict__ part, int chunks, i64 r,
                                                       int* __restrict__ os, float tau_f,
                                                       int* __restrict__ rounds_total, i64 wstride, int phase) {
   pdl_enter();
@@ -672,9 +737,9 @@ __global__ void __launch_bounds__(256) k_probe_decide(const float* __restrict__ 
     if (threadIdx.x == 0) { os[OS_ROUNDS] = 1; atomicAdd(rounds_total, 1); }
     return;
   }
-  __shared__ float red[256];
+  __shared__ float red[1024];
   float e = 0.f;
-  for (i64 j = threadIdx.x; j < r; j += 256) {
+  for (i64 j = threadIdx.x; j < r; j += blockDim.x) {
 #pragma unroll
     for (int p = 0; p < NPROBE; ++p) {
       float w = 0.f;
@@ -685,7 +750,7 @@ __global__ void __launch_bounds__(256) k_probe_decide(const float* __restrict__ 
   }
   red[threadIdx.x] = e;
   __syncthreads();
-  for (int w = 128; w > 0; w >>= 1) {
+  for (int w = (int)blockDim.x / 2; w > 0; w >>= 1) {     // (the block size is a power of two)
     if ((int)threadIdx.x < w) red[threadIdx.x] += red[threadIdx.x + w];
     __syncthreads();
   }
