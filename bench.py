@@ -172,8 +172,8 @@ def case_report(c, ms, rounds, args, peaks, binding):
     read-modify-write M, read-modify-write X) at the measured copy bandwidth; t_tensor: every product at the
     tensor peak of the arithmetic it runs in -- fp32 mode: the orthonormalization 3xTF32 (three TF32 passes, TF32
     taken as half the measured bf16 peak), P, R and the error feedback three bf16 passes on (hi, lo) pairs where
-    the library uses them (else 3xTF32), the X update one TF32 pass; bf16-operand mode: one bf16 pass for the
-    four products."""
+    the library uses them (else 3xTF32), the X update one pass on IEEE half factors at the 16-bit rate where every
+    dimension is a multiple of 8 (else one TF32 pass); bf16-operand mode: one bf16 pass for the four products."""
     m, n, r = c[:3]
     out = {"m": m, "n": n, "r": r, "ms": ms,
            "orth_mode": ["auto", "cholqr2", "adaptive", "householder", "rcqr"][orth_mode(m, n, r, args.orth)], "orth_rounds": rounds}
@@ -191,7 +191,8 @@ def case_report(c, ms, rounds, args, peaks, binding):
         pair_peak = bf16 / 3.0 if pairs_apply(m, n, r) else tf32 / 3.0
         ef_peak = bf16 / 3.0 if (m % 8 == 0 and n % 8 == 0 and r % 8 == 0 and r >= 64) else tf32 / 3.0
         p_peak = bf16 / 3.0 if p_pairs_apply(m, n, r, args.orth) else tf32 / 3.0
-        t_prod = fl["P"] / (p_peak * 1e12) + fl["R"] / (pair_peak * 1e12) + fl["EF"] / (ef_peak * 1e12) + fl["X"] / (tf32 * 1e12)
+        x_peak = bf16 if (m % 8 == 0 and n % 8 == 0 and r % 8 == 0 and r >= 64 and m >= 128 and n >= 64) else tf32
+        t_prod = fl["P"] / (p_peak * 1e12) + fl["R"] / (pair_peak * 1e12) + fl["EF"] / (ef_peak * 1e12) + fl["X"] / (x_peak * 1e12)
     t_tensor = (t_prod + fl["ORTH"] / (tf32 / 3.0 * 1e12)) * 1e3
     bound = "hbm" if t_hbm >= t_tensor else "tensor"
     out.update({"t_hbm_ms": t_hbm, "t_tensor_ms": t_tensor, "bound": bound,
@@ -738,9 +739,10 @@ def workload_record(wid, cases, grouped, args, peaks, binding, ms_step, e2e_ms, 
                                "ten consecutive dion_step calls per step" if reps_per_step > 1 else
                                "one dion_step call per matrix per step"),
                       "engine": ["auto", "simt", "tensor"][args.engine],
-                      "precision": ["fp32 (P and Orthonormalize 3xTF32; R and the error feedback on bf16 (hi, lo) pairs, 16 "
-                                    "significant bits, where M + G is kept in scratch; the X update single-pass TF32 on "
-                                    "rounded factors; FMA for ragged shapes)", "bf16 operands"][args.precision],
+                      "precision": ["fp32 (Orthonormalize 3xTF32; R, the error feedback and, on large matrices, P on bf16 "
+                                    "(hi, lo) pairs, 16 significant bits, where M + G is kept in scratch, P recomputed in "
+                                    "3xTF32 when the orthogonality probe asks; the X update one pass on factors rounded to "
+                                    "IEEE half (11 significant bits); FMA for ragged shapes)", "bf16 operands"][args.precision],
                       "orth": ["auto", "cholqr2", "shifted3", "householder", "rcqr"][args.orth],
                       "sync": ("compressed data-parallel sync: P and W all-reduced (mean) over the ranks"
                                if args.sync == "dp" else "none (independent replicas)"),

@@ -2,6 +2,8 @@
 // TF32-rounded copies of the factors of the weight update (fp32 mode).
 #pragma once
 
+#include <cuda_fp16.h>
+
 #include "dion_common.cuh"
 
 namespace dion {
@@ -232,6 +234,42 @@ __global__ void __launch_bounds__(256) k_round_tf32_chain(const ChainPtrs srcs, 
   const i64 b = blockIdx.y;
   if (skip_flag != nullptr && skip_flag[b * skip_stride] != 0) return;
   round_tf32_body(reinterpret_cast<const float*>(srcs.p[b]), lds, rows, cols, out + b * ostride);
+}
+
+// out = half(scale * src), round to nearest: the factors of the weight update as IEEE half arrays (11 significant
+// bits, like TF32, at the 16-bit MMA rate and half the operand bytes).  `scale` is a power of two chosen by the caller
+// so that entries of a matrix with unit-norm columns sit around 1: far from half's subnormals, and at most
+// sqrt(2 rows) < 65504.  rows x cols (cols a multiple of 8, src rows 16-byte aligned), out dense.
+__device__ __forceinline__ void round_f16_body(const float* __restrict__ src, i64 lds, i64 rows, i64 cols, float scale,
+                                               __half* __restrict__ out) {
+  const i64 per_row = cols / 8;
+  const i64 total = rows * per_row;
+  for (i64 e = (i64)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (i64)gridDim.x * blockDim.x) {
+    const i64 i = e / per_row, c = (e - i * per_row) * 8;
+    const float4 a = *reinterpret_cast<const float4*>(src + i * lds + c);
+    const float4 b = *(reinterpret_cast<const float4*>(src + i * lds + c) + 1);
+    __half2 h0 = __floats2half2_rn(scale * a.x, scale * a.y), h1 = __floats2half2_rn(scale * a.z, scale * a.w);
+    __half2 h2 = __floats2half2_rn(scale * b.x, scale * b.y), h3 = __floats2half2_rn(scale * b.z, scale * b.w);
+    uint4 o;
+    o.x = *reinterpret_cast<uint32_t*>(&h0); o.y = *reinterpret_cast<uint32_t*>(&h1);
+    o.z = *reinterpret_cast<uint32_t*>(&h2); o.w = *reinterpret_cast<uint32_t*>(&h3);
+    *reinterpret_cast<uint4*>(out + i * cols + c) = o;
+  }
+}
+__global__ void __launch_bounds__(256) k_round_f16(const float* __restrict__ src, i64 lds, i64 rows, i64 cols, float scale,
+                                                   __half* __restrict__ out, const int* __restrict__ skip_flag) {
+  pdl_enter();
+  if (skip_flag != nullptr && *skip_flag != 0) return;
+  round_f16_body(src, lds, rows, cols, scale, out);
+}
+// (one launch over a chain: blockIdx.y, outputs `ostride` floats apart)
+__global__ void __launch_bounds__(256) k_round_f16_chain(const ChainPtrs srcs, i64 lds, i64 rows, i64 cols, float scale,
+                                                         __half* __restrict__ out, i64 ostride,
+                                                         const int* __restrict__ skip_flag, i64 skip_stride) {
+  pdl_enter();
+  const i64 b = blockIdx.y;
+  if (skip_flag != nullptr && skip_flag[b * skip_stride] != 0) return;
+  round_f16_body(reinterpret_cast<const float*>(srcs.p[b]), lds, rows, cols, scale, out + 2 * b * ostride);
 }
 
 }  // namespace dion

@@ -400,7 +400,7 @@ int launch_gemm_group(StepCtx& s, const std::vector<GemmArgs>& v) {
           g.a2_sk == a.a2_sk && g.a2_mode == a.a2_mode && g.b_sk == a.b_sk && g.b_sn == a.b_sn && g.ldc == a.ldc &&
           g.epi == a.epi && g.ldc2 == a.ldc2 && g.c2_mode == a.c2_mode && g.alpha == a.alpha && g.alpha_dev == a.alpha_dev &&
           g.batch == 1 && a.batch == 1 && g.tri == a.tri && g.klimit == a.klimit && g.precise == a.precise &&
-          g.ab16 == a.ab16 && g.tf32x1 == a.tf32x1 && at_stride(a.A, g.A, b) && at_stride(a.B, g.B, b) &&
+          g.ab16 == a.ab16 && g.f16 == a.f16 && g.tf32x1 == a.tf32x1 && at_stride(a.A, g.A, b) && at_stride(a.B, g.B, b) &&
           at_stride(a.A2, g.A2, b) && at_stride(a.A16lo, g.A16lo, b) && at_stride(a.B16lo, g.B16lo, b) &&
           ((a.skip_flag == nullptr && g.skip_flag == nullptr) ||
            (a.skip_flag != nullptr && g.skip_flag == a.skip_flag + (i64)b * OS_SLOT_INTS));
@@ -1019,10 +1019,29 @@ int split_chain(StepCtx& s, const float* const* src, const i64* ld, i64 rows, i6
 }
 
 // src[b] rounded to TF32 into the scratch slices at out_off.
-int round_chain(StepCtx& s, const float* const* src, const i64* ld, i64 rows, i64 cols, i64 out_off, const int* skip0) {
+// half_scale > 0: IEEE half values of half_scale * src instead (see x_half).
+int round_chain(StepCtx& s, const float* const* src, const i64* ld, i64 rows, i64 cols, i64 out_off, const int* skip0,
+                float half_scale = 0.f) {
   dion_ctx* c = s.c;
   bool one = s.nb > 1 && s.nb <= GEMM_TAB_MAX && c->chain_batch;
   for (int b = 1; b < s.nb && one; ++b) one = ld[b] == ld[0];
+  if (half_scale > 0.f) {
+    const unsigned g8 = (unsigned)grid_for(c, rows * cols / 8);
+    if (one) {
+      ChainPtrs t;
+      for (int b = 0; b < s.nb; ++b) t.p[b] = src[b];
+      launch_pdl(k_round_f16_chain, dim3(g8, (unsigned)s.nb), dim3(256), 0, s.st, t, ld[0], rows, cols, half_scale,
+                 reinterpret_cast<__half*>(s.ws + out_off), s.wstride, skip0, (i64)OS_SLOT_INTS);
+      DION_CHECK_LAUNCH(c);
+      return DION_OK;
+    }
+    for (int b = 0; b < s.nb; ++b) {
+      launch_pdl(k_round_f16, dim3(g8), dim3(256), 0, s.st, src[b], ld[b], rows, cols, half_scale, reinterpret_cast<__half*>(s.W(b, out_off)),
+                 skip0 != nullptr ? skip0 + (i64)b * OS_SLOT_INTS : (const int*)nullptr);
+      DION_CHECK_LAUNCH(c);
+    }
+    return DION_OK;
+  }
   const unsigned gx = (unsigned)grid_for(c, rows * cols / 4);
   if (one) {
     ChainPtrs t;
@@ -1182,6 +1201,14 @@ bool x_single_pass(const StepCtx& s, const dion_matrix* a, const float* F1, i64 
          ld1 % 4 == 0 && !((uintptr_t)F2 & 15) && ld2 % 4 == 0;
 }
 
+// ... and with every dimension a multiple of 8 the rounded factors are IEEE half arrays instead: the same 11
+// significant bits as TF32, read by one kind::f16 MMA per K step of 16 -- twice the MMA rate and half the operand
+// bytes.  Both factors have unit-norm columns (U orthonormal, Q column-normalized), so their entries are at most 1;
+// each is scaled by the power of two nearest the square root of its row count (entries around 1: far from half's
+// subnormals, at most sqrt(2 rows) < 65504) and alpha takes the scales back exactly.
+bool x_half(const dion_matrix* a) { return a->m % 8 == 0 && a->n % 8 == 0 && a->r % 8 == 0; }
+float half_scale(i64 rows) { return exp2f(rintf(0.5f * log2f((float)rows))); }
+
 // The error feedback M <- (M + G) - beta F1 F2^T in fp32 mode on the tensor engine (F1: m x r, F2: n x r; U R^T, or
 // R U^T in the transposed form).  The product enters M scaled by beta = 1 - mu, so 16 significant bits in its factors
 // are plenty (an error of ~1e-5 of the product, ~5e-7 of M): both factors are split once into bf16 pairs
@@ -1241,7 +1268,19 @@ int x_update(StepCtx& s, int b, const dion_matrix* a, const float* F1, i64 ld1, 
   const i64 m = a->m, n = a->n, r = a->r;
   GemmArgs x = gemm_args();
   x.M = m; x.N = n; x.K = r;
-  if (x_single_pass(s, a, F1, ld1, F2, ld2)) {
+  if (x_single_pass(s, a, F1, ld1, F2, ld2) && x_half(a)) {
+    const float s1 = half_scale(m), s2 = half_scale(n);
+    if (!rounded) {
+      launch_pdl(k_round_f16, dim3((unsigned)grid_for(c, m * r / 8)), dim3(256), 0, s.st, F1, ld1, m, r, s1, reinterpret_cast<__half*>(r1), skip);
+      DION_CHECK_LAUNCH(c);
+      launch_pdl(k_round_f16, dim3((unsigned)grid_for(c, n * r / 8)), dim3(256), 0, s.st, F2, ld2, n, r, s2, reinterpret_cast<__half*>(r2), skip);
+      DION_CHECK_LAUNCH(c);
+    }
+    x.ab16 = 1; x.f16 = 1;
+    x.A = r1; x.a_si = r; x.a_sk = 1;
+    x.B = r2; x.b_sk = 1; x.b_sn = r;
+    alpha /= s1 * s2;       // (powers of two: exact)
+  } else if (x_single_pass(s, a, F1, ld1, F2, ld2)) {
     if (!rounded) {
       launch_pdl(k_round_tf32, dim3((unsigned)grid_for(c, m * r / 4)), dim3(256), 0, s.st, F1, ld1, m, r, r1, skip);
       DION_CHECK_LAUNCH(c);
@@ -1521,9 +1560,10 @@ int step_batch(dion_ctx* c, const dion_matrix* const* list, int nb, float lr, cu
     }
     if (all_one) {
       for (int b = 0; b < nb; ++b) { srcs[b] = s.W(b, U_off); lds[b] = r; }
-      DION_TRY(round_chain(s, srcs, lds, prow, r, other_off, s.os + OS_FAIL));
+      const bool half = x_half(a0);
+      DION_TRY(round_chain(s, srcs, lds, prow, r, other_off, s.os + OS_FAIL, half ? half_scale(prow) : 0.f));
       for (int b = 0; b < nb; ++b) { srcs[b] = (const float*)list[b]->Q; lds[b] = list[b]->ldq; }
-      DION_TRY(round_chain(s, srcs, lds, qrow, r, s.L.R, s.os + OS_FAIL));
+      DION_TRY(round_chain(s, srcs, lds, qrow, r, s.L.R, s.os + OS_FAIL, half ? half_scale(qrow) : 0.f));
       x_rounded = true;
     }
   }
@@ -2347,7 +2387,7 @@ extern "C" int dion_debug_gemm(int engine, int precision, const dion_debug_gemm_
   g.B = a->B; g.b_sk = a->b_sk; g.b_sn = a->b_sn;
   g.C = a->C; g.ldc = a->ldc; g.epi = a->epi;
   g.C2 = a->C2; g.ldc2 = a->ldc2; g.c2_mode = a->c2_mode;
-  g.alpha = a->alpha; g.tri = a->tri; g.klimit = a->klimit; g.precise = a->precise; g.ab16 = a->ab16; g.tf32x1 = a->tf32x1;
+  g.alpha = a->alpha; g.tri = a->tri; g.klimit = a->klimit; g.precise = a->precise; g.ab16 = a->ab16; g.tf32x1 = a->tf32x1; g.f16 = a->f16;
   g.A16lo = a->A16lo; g.B16lo = a->B16lo;
   cudaStream_t st = (cudaStream_t)cuda_stream;
   if (engine == DION_ENGINE_TENSOR) {

@@ -56,6 +56,7 @@ struct GemmArgs {
   int ab16;                      // tensor engine only: A and B point to bf16 arrays (strides in elements), no addend
   const void* A16lo;             // with ab16: A and B are PAIRS of bf16 arrays, x ~ hi + lo (A, B point to the "hi" arrays, these
   const void* B16lo;             // to the "lo" arrays of the same shape and strides): three bf16 MMAs per K step, ~1e-5 relative
+  int f16;                       // with ab16 (no pairs): the arrays hold IEEE half values instead of bf16 (11 significant bits)
   int tf32x1;                    // tensor engine, fp32 mode: the operands' values fit TF32 already (k_round_tf32): one MMA
                                  // per K step instead of the three-term split.  Ignored by the FMA engine.
 };

@@ -29,6 +29,7 @@ typedef struct {
                                                     in *status and return */
   const void* A16lo;                             /* with ab16: the "lo" arrays of bf16 operand pairs (x ~ hi + lo; A, B */
   const void* B16lo;                             /* are the "hi" arrays), or NULL                                        */
+  int f16;                                       /* with ab16 (no pairs): the arrays hold IEEE half values */
 } dion_debug_gemm_args;
 
 /* engine: 1 = fp32 FMA, 2 = tensor cores (returns DION_ERR_UNSUPPORTED if the

@@ -324,11 +324,13 @@ __device__ __forceinline__ uint64_t make_desc_k64(uint32_t saddr) {
 }
 
 // Instruction descriptor: fp32 accumulate, TF32 or BF16 operands, M = 128, N = BN.
-__device__ __forceinline__ uint32_t make_idesc(bool bf16, bool a_mn, bool b_mn, int bn, int bm = BM) {
+// f16 (with bf16): the 16-bit operands are IEEE half values (kind::f16 takes either format)
+__device__ __forceinline__ uint32_t make_idesc(bool bf16, bool a_mn, bool b_mn, int bn, int bm = BM, bool f16 = false) {
   uint32_t d = 0;
+  const uint32_t fmt = bf16 ? (f16 ? 0u : 1u) : 2u;   // 0 F16, 1 BF16 (kind::f16); 2 TF32 (kind::tf32)
   d |= 1u << 4;                         // D format: F32
-  d |= (bf16 ? 1u : 2u) << 7;           // A format
-  d |= (bf16 ? 1u : 2u) << 10;          // B format
+  d |= fmt << 7;                        // A format
+  d |= fmt << 10;                       // B format
   d |= (a_mn ? 1u : 0u) << 15;
   d |= (b_mn ? 1u : 0u) << 16;
   d |= (uint32_t)(bn >> 3) << 17;
@@ -1181,7 +1183,7 @@ k_gemm_umma(const __grid_constant__ Params p) {
         }
       }
     } else if (lane == 0 && (!CG2 || cta_rank == 0)) {
-      const uint32_t idesc = make_idesc(BF16, A_MN, B_MN, BN, CG2 ? 2 * BM : BM);
+      const uint32_t idesc = make_idesc(BF16, A_MN, B_MN, BN, CG2 ? 2 * BM : BM, BF16 && p.g.f16 != 0);
       const uint32_t lbo = BKE * 128;
       constexpr uint32_t A_KSTEP = A_MN ? (BF16 ? 2048u : 1024u) : 32u;   // bytes per UMMA K step
       constexpr uint32_t B_KSTEP = B_MN ? (BF16 ? 2048u : 1024u) : 32u;

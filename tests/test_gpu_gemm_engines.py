@@ -26,7 +26,7 @@ class GemmArgs(ctypes.Structure):
                 ("C2", ctypes.c_void_p), ("ldc2", ctypes.c_int64), ("c2_mode", ctypes.c_int),
                 ("alpha", ctypes.c_float), ("tri", ctypes.c_int), ("klimit", ctypes.c_int), ("precise", ctypes.c_int),
                 ("ab16", ctypes.c_int), ("tf32x1", ctypes.c_int), ("variant", ctypes.c_int),
-                    ("A16lo", ctypes.c_void_p), ("B16lo", ctypes.c_void_p)]
+                    ("A16lo", ctypes.c_void_p), ("B16lo", ctypes.c_void_p), ("f16", ctypes.c_int)]
 
 
 @pytest.fixture(scope="module")
@@ -354,3 +354,27 @@ def test_column_panel_tile_order_when_b_exceeds_l2(lib):
     for (a_mn, b_mn) in LAYOUTS:
         C, want = _pair_product(lib, 1024, 8192 + 256, 2048, a_mn, b_mn, 3, 0, seed=5)
         assert float((C.double() - want).norm() / want.norm()) < 1e-5
+
+
+@pytest.mark.parametrize("M,N,K,epi", [(1024, 768, 256, 1), (640, 392, 96, 1), (2048, 256, 1024, 0), (4096, 4096, 128, 1)])
+def test_ieee_half_arrays_as_operands(lib, M, N, K, epi):
+    # the weight update's factors as IEEE half arrays: values that fit half exactly are multiplied exactly, so the
+    # only error left is the tensor core's fp32 accumulation
+    g = torch.Generator(device="cuda"); g.manual_seed(M + K)
+    A = torch.randn(M, K, generator=g, device="cuda").half(); B = torch.randn(N, K, generator=g, device="cuda").half()
+    C = torch.randn(M, N, generator=g, device="cuda"); C0 = C.clone()
+    alpha = 0.05
+    ref = A.double() @ B.double().t()
+    want = alpha * ref if epi == 0 else C0.double() - alpha * ref
+    a = GemmArgs()
+    a.M, a.N, a.K = M, N, K
+    a.A = A.data_ptr(); a.a_si, a.a_sk = K, 1
+    a.B = B.data_ptr(); a.b_sk, a.b_sn = 1, K
+    a.C = C.data_ptr(); a.ldc = N; a.epi = epi
+    a.alpha = alpha; a.ab16 = 1; a.f16 = 1
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    rc = lib.dion_debug_gemm(2, 0, ctypes.byref(a), None, 0, status.data_ptr(), int(torch.cuda.current_stream().cuda_stream))
+    torch.cuda.synchronize()
+    assert rc == 0 and int(status.item()) == 0
+    err = float((C.double() - want).norm() / want.norm())
+    assert err < 8e-6, err
