@@ -272,4 +272,74 @@ __global__ void __launch_bounds__(256) k_round_f16_chain(const ChainPtrs srcs, i
   round_f16_body(reinterpret_cast<const float*>(srcs.p[b]), lds, rows, cols, scale, out + 2 * b * ostride);
 }
 
+// ---- a panel as a pair of IEEE half arrays, scaled: 22 significant bits at the 16-bit MMA rate ----------------
+// Half has 5 exponent bits, so the panel is scaled by a power of two that puts its largest entry in [2^13, 2^14):
+// entries down to 2^-17 of the largest keep all 22 bits of the pair, smaller ones an absolute error of 2^-39 of
+// the largest.  Two launches: per-block maxima of |x|, then the split (every block reduces the maxima again, in
+// a fixed order; block 0 also writes 1 / scale^2, the factor that takes a Gram matrix of the pair back).
+// blockIdx.y: the matrix of a chain (arrays `wstride` floats apart); skip flags a state slot apart.
+constexpr int AMAX_PARTS = 512;
+__global__ void __launch_bounds__(256) k_absmax_partial(const float* __restrict__ src, i64 ld, i64 rows, i64 cols,
+                                                        float* __restrict__ part, i64 wstride, const int* __restrict__ skip_flag,
+                                                        i64 skip_stride) {
+  pdl_enter();
+  if (skip_flag != nullptr && skip_flag[(i64)blockIdx.y * skip_stride] != 0) return;
+  src += (i64)blockIdx.y * wstride; part += (i64)blockIdx.y * wstride;
+  const i64 per_row = cols / 4, total = rows * per_row;
+  float m = 0.f;
+  for (i64 e = (i64)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (i64)gridDim.x * blockDim.x) {
+    const i64 i = e / per_row, c = (e - i * per_row) * 4;
+    const float4 a = *reinterpret_cast<const float4*>(src + i * ld + c);
+    m = fmaxf(fmaxf(m, fmaxf(fabsf(a.x), fabsf(a.y))), fmaxf(fabsf(a.z), fabsf(a.w)));
+  }
+  __shared__ float red[256];
+  red[threadIdx.x] = m;
+  __syncthreads();
+  for (int w = 128; w > 0; w >>= 1) {
+    if ((int)threadIdx.x < w) red[threadIdx.x] = fmaxf(red[threadIdx.x], red[threadIdx.x + w]);
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) part[blockIdx.x] = red[0];
+}
+__global__ void __launch_bounds__(256) k_split_f16_scaled(const float* __restrict__ src, i64 ld, i64 rows, i64 cols,
+                                                          const float* __restrict__ part, int nparts,
+                                                          __half* __restrict__ hi, __half* __restrict__ lo,
+                                                          float* __restrict__ inv_scale2, i64 wstride,
+                                                          const int* __restrict__ skip_flag, i64 skip_stride) {
+  pdl_enter();
+  if (skip_flag != nullptr && skip_flag[(i64)blockIdx.y * skip_stride] != 0) return;
+  src += (i64)blockIdx.y * wstride; part += (i64)blockIdx.y * wstride; inv_scale2 += (i64)blockIdx.y * wstride;
+  hi += 2 * (i64)blockIdx.y * wstride; lo += 2 * (i64)blockIdx.y * wstride;
+  __shared__ float red[256];
+  float m = 0.f;
+  for (int e = threadIdx.x; e < nparts; e += 256) m = fmaxf(m, part[e]);
+  red[threadIdx.x] = m;
+  __syncthreads();
+  for (int w = 128; w > 0; w >>= 1) {
+    if ((int)threadIdx.x < w) red[threadIdx.x] = fmaxf(red[threadIdx.x], red[threadIdx.x + w]);
+    __syncthreads();
+  }
+  const float amax = red[0];
+  int ex = 14;                                   // amax = f 2^ex with f in [0.5, 1): scale 2^(14 - ex)
+  if (amax > 0.f && amax < 3.0e38f) frexpf(amax, &ex);
+  if (ex < -100) ex = -100;
+  const float scale = ldexpf(1.f, 14 - ex);
+  if (blockIdx.x == 0 && threadIdx.x == 0) *inv_scale2 = ldexpf(1.f, 2 * (ex - 14));
+  const i64 per_row = cols / 8, total = rows * per_row;
+  for (i64 e = (i64)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (i64)gridDim.x * blockDim.x) {
+    const i64 i = e / per_row, c = (e - i * per_row) * 8;
+    const float4 a = *reinterpret_cast<const float4*>(src + i * ld + c);
+    const float4 b = *(reinterpret_cast<const float4*>(src + i * ld + c) + 1);
+    const float v[8] = {scale * a.x, scale * a.y, scale * a.z, scale * a.w, scale * b.x, scale * b.y, scale * b.z, scale * b.w};
+    __half h[8], l[8];
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {
+      h[q] = __float2half_rn(v[q]);
+      l[q] = __float2half_rn(v[q] - __half2float(h[q]));
+    }
+    *reinterpret_cast<uint4*>(hi + i * cols + c) = *reinterpret_cast<const uint4*>(h);
+    *reinterpret_cast<uint4*>(lo + i * cols + c) = *reinterpret_cast<const uint4*>(l);
+  }
+}
+
 }  // namespace dion

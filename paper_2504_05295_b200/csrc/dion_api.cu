@@ -38,6 +38,7 @@ constexpr float GOOD_REL = 1e-4f;         // smallest relative pivot of a round 
 constexpr float ORTH_TAU_F = 3e-5f;
 constexpr float DONE_REL = 0.9f;          // smallest relative pivot of a round whose input was already orthonormal
 constexpr i64 PART_CAP_FLOATS = (i64)16 << 20;  // split-K partial sums, at most 64 MiB
+constexpr double GRAM_PAIR_MIN_FLOPS = 2e9;     // smallest rows r^2 whose Gram matrix runs on scaled half pairs
 constexpr double P_PAIR_MIN_MNR = 1.5e10;       // smallest m n r whose P = (M + G) Q runs on bf16 operand pairs first
 
 constexpr i64 NBO_COLS = 512;  // = NBO, the outer block of the two-level Cholesky (defined below)
@@ -53,6 +54,7 @@ struct Layout {
   i64 fb_part, fb_h, fb_n;  // fallback kernel: partial dot products (SMs x r), their sums (r), partial norms (SMs)
   i64 probe_y, probe_part;  // CholeskyQR2's orthogonality probe: U1 z (rows x NPROBE), partial U1^T (U1 z)
   i64 Bp;                   // fp32 mode, M + G in scratch: the same sum as a bf16 (hi, lo) pair (m x n x 2 bf16) for R; 0: none
+  i64 gmax;                 // Gram matrices on half pairs: AMAX_PARTS partial maxima of |P|, then 1 / scale^2
   i64 Qc;                   // fp32 mode, large matrices: dense fp32 copy of Q for the chain-wide recomputation of P (0: none)
   i64 S16;                  // fp32 mode: the bf16 (hi, lo) pair of the error feedback's second factor (max(m,n) x r x 2 bf16)
   i64 part_floats;
@@ -173,6 +175,7 @@ Layout make_layout(const dion_ctx* c, i64 m, i64 n, i64 r) {
     if (m % 8 == 0 && n % 8 == 0 && r % 8 == 0) { L.Bp = o; o += align64(m * n); }
   }
   L.Psave = L.fb_part = L.fb_h = L.fb_n = 0;
+  L.gmax = o; o += align64(AMAX_PARTS + 64);
   L.Qc = 0;
   if (L.Bp > 0 && (double)m * (double)n * (double)r >= P_PAIR_MIN_MNR) { L.Qc = o; o += align64(big * r); }
   L.S16 = o; o += align64(big * r);
@@ -270,7 +273,7 @@ int launch_gemm_simt(dion_ctx* c, GemmArgs g, cudaStream_t st, float* part, i64 
     const i64 total = g.M * g.N;
     int blocks = (int)((total + 255) / 256);
     if (blocks > 8 * c->sm_count) blocks = 8 * c->sm_count;
-    launch_pdl(k_splitk_reduce, dim3((unsigned)(blocks)), dim3(256), 0, st, part, splits, g.M, g.N, g.C, g.ldc, g.alpha, g.tri, BMN, g.skip_flag, (i64)0, (i64)0);
+    launch_pdl(k_splitk_reduce, dim3((unsigned)(blocks)), dim3(256), 0, st, part, splits, g.M, g.N, g.C, g.ldc, g.alpha, g.tri, BMN, g.skip_flag, (i64)0, (i64)0, (const float*)nullptr, (i64)0);
     DION_CHECK_LAUNCH(c);
   }
   return DION_OK;
@@ -349,6 +352,9 @@ GemmArgs for_matrix(const StepCtx& s, GemmArgs g, int b, bool a_ws, bool b_ws, b
   if (a_ws) g.A += o;
   if (b_ws) g.B += o;
   if (c_ws) g.C += o;
+  if (a_ws && g.A16lo != nullptr) g.A16lo = (const char*)g.A16lo + 4 * o;
+  if (b_ws && g.B16lo != nullptr) g.B16lo = (const char*)g.B16lo + 4 * o;
+  if (g.alpha_dev != nullptr) g.alpha_dev += (i64)b * g.alpha_dev_stride;
   if (g.skip_flag != nullptr) g.skip_flag += (i64)b * OS_SLOT_INTS;
   return g;
 }
@@ -650,6 +656,12 @@ int probe(StepCtx& s, i64 off, i64 rows, i64 r, int phase) {
   return DION_OK;
 }
 
+// Tall panels whose Gram matrix runs on scaled half pairs (the rule looks at the shape alone).
+bool gram_on_pairs(const StepCtx& s, i64 rows, i64 r) {
+  return s.tensor && s.c->cfg.precision == DION_PREC_FP32 && rows % 8 == 0 && r % 8 == 0 && r >= 128 &&
+         (double)rows * (double)r * (double)r >= GRAM_PAIR_MIN_FLOPS;
+}
+
 // One Cholesky-QR round on every matrix of the chain: Pout = Pin * chol(Pin^T Pin)^-T.
 // rows x r panels, ld = r; pin_off / pout_off are offsets in the scratch slice.
 // adaptive: columns with negligible pivots are deflated, the round is skipped (Pout = Pin)
@@ -672,6 +684,27 @@ int cholqr_round(StepCtx& s, i64 pin_off, i64 pout_off, i64 rows, i64 r, int mod
   g.M = r; g.N = r; g.K = gram_rows > 0 ? gram_rows : rows;
   g.A = s.ws + pin_off; g.a_si = 1; g.a_sk = r;
   g.B = s.ws + pin_off; g.b_sk = r; g.b_sn = 1;
+  if (gram_rows == 0 && gram_on_pairs(s, rows, r)) {
+    // The Gram matrix of a tall panel on half pairs: the panel is scaled and split into Pout's buffer (free until
+    // the solve writes it) and the product takes three kind::f16 MMAs per K step instead of the three or four
+    // kind::tf32 ones; the same 22 significant bits.  1 / scale^2 reaches the epilogue through a device scalar.
+    const int* sk = skips ? skip : nullptr;
+    __half* hi = reinterpret_cast<__half*>(s.ws + pout_off);
+    __half* lo = hi + rows * r;
+    i64 parts = (rows * r / 4 + 2047) / 2048;
+    if (parts > AMAX_PARTS) parts = AMAX_PARTS;
+    launch_pdl(k_absmax_partial, dim3((unsigned)parts, (unsigned)s.nb), dim3(256), 0, s.st, (const float*)(s.ws + pin_off), r, rows, r,
+               s.ws + s.L.gmax, s.wstride, sk, (i64)OS_SLOT_INTS);
+    DION_CHECK_LAUNCH(c);
+    launch_pdl(k_split_f16_scaled, dim3((unsigned)grid_for(c, rows * r / 8), (unsigned)s.nb), dim3(256), 0, s.st,
+               (const float*)(s.ws + pin_off), r, rows, r, (const float*)(s.ws + s.L.gmax), (int)parts, hi, lo, s.ws + s.L.gmax + AMAX_PARTS,
+               s.wstride, sk, (i64)OS_SLOT_INTS);
+    DION_CHECK_LAUNCH(c);
+    g.ab16 = 1; g.f16 = 1;
+    g.A = reinterpret_cast<const float*>(hi); g.A16lo = lo;
+    g.B = reinterpret_cast<const float*>(hi); g.B16lo = lo;
+    g.alpha_dev = s.ws + s.L.gmax + AMAX_PARTS; g.alpha_dev_stride = s.wstride;
+  }
   g.C = s.ws + s.L.Gram; g.ldc = r; g.epi = EPI_STORE; g.tri = TRI_LOWER; g.skip_flag = skips ? skip : nullptr; g.precise = rm_precise(mode) ? 1 : 0;
   DION_TRY(launch_gemm_chain(s, g));
   launch_pdl(k_round_begin, dim3((unsigned)(s.nb)), dim3(256), 0, s.st, s.ws + s.L.Gram, r, r, 0.f, s.ws + s.L.gdiag, s.ws + s.L.scal, s.os,

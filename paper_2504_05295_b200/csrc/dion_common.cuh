@@ -41,7 +41,8 @@ struct GemmArgs {
   int epi;
   const void* C2; i64 ldc2; int c2_mode;
   float alpha;
-  const float* alpha_dev;      // optional: alpha is multiplied by *alpha_dev
+  const float* alpha_dev;      // optional: alpha is multiplied by *alpha_dev ...
+  i64 alpha_dev_stride;        // ... of entry b of the outer batch: alpha_dev[b * alpha_dev_stride]
   int batch; i64 bsA, bsB, bsC;  // batch count and element strides
   int batch2; i64 bs2;           // outer batch (one per matrix of a grouped call): stride of A, B, C alike
   i64 skip_stride;               // ints between the skip flags of consecutive outer batch entries

@@ -167,10 +167,12 @@ __global__ void __launch_bounds__(256) k_gemm_simt(const GemmArgs g) {
 // Sums split-K partials in a fixed order: C = alpha * sum_s part[s].
 __global__ void k_splitk_reduce(const float* __restrict__ part, int splits, i64 M, i64 N,
                                 float* __restrict__ C, i64 ldc, float alpha, int tri, int tile,
-                                const int* skip_flag, i64 bstride, i64 skip_stride) {
+                                const int* skip_flag, i64 bstride, i64 skip_stride,
+                                const float* __restrict__ alpha_dev = nullptr, i64 alpha_dev_stride = 0) {
   // blockIdx.y: the matrix of a batched product (partials and output bstride elements apart)
   pdl_enter();
   if (skip_flag != nullptr && skip_flag[(i64)blockIdx.y * skip_stride] != 0) return;
+  if (alpha_dev != nullptr) alpha *= alpha_dev[(i64)blockIdx.y * alpha_dev_stride];
   part += (i64)blockIdx.y * bstride;
   C += (i64)blockIdx.y * bstride;
   const i64 total = M * N;

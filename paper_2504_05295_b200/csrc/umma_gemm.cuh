@@ -596,7 +596,7 @@ k_gemm_umma(const __grid_constant__ Params p) {
   static_assert(!X2 || (D16 && CE), "operand pairs are bf16 arrays");
   static_assert(!CG2 || (TMA && BN == 256 && ((!BF16 && !D16 && !ONE) || X2)),
                 "CTA pairs: the fp32 TMA variants and the operand-pair variant, 256-column tiles");
-  static_assert(!(BF16 && SPLIT), "split accumulators belong to the 3xTF32 mode");
+  static_assert(!(BF16 && SPLIT) || X2, "split accumulators belong to the 3xTF32 mode and to operand pairs");
   static_assert(!D16 || (BF16 && TMA), "bf16 operands in memory are loaded by TMA");
   static_assert(!CE || (TMA && (D16 || !BF16)), "the coalesced epilogue serves the bf16-array and the fp32 TMA variants");
   static_assert(!ONE || (TMA && CE && !BF16 && !SPLIT && !A_MN && !B_MN), "single pass: k-contiguous fp32 operands by TMA");
@@ -680,7 +680,8 @@ k_gemm_umma(const __grid_constant__ Params p) {
       constexpr int SLABS = (BN / 32) / (C::EPI_WARPS / 4);   // 32-column slabs per warp
       const i64 gi = (i64)it.mi * BM + quad * 32 + lane;
       const i64 n0 = (i64)it.ni * BN;
-      const float alpha = g.alpha * (g.alpha_dev != nullptr ? __ldg(g.alpha_dev) : 1.f);   // (a device scalar under graph replay)
+      // (a device scalar: the learning rate under graph replay, or a matrix's own scale)
+      const float alpha = g.alpha * (g.alpha_dev != nullptr ? __ldg(g.alpha_dev + (i64)it.b * g.alpha_dev_stride) : 1.f);
       for (int kb = it.kb0; kb < it.kb1; kb += p.kc, ++iter) {
         const bool first = (kb == it.kb0);
         const int ab = iter % NBUF;
@@ -1224,14 +1225,15 @@ k_gemm_umma(const __grid_constant__ Params p) {
             if (X2) {
               const uint64_t a_lo = make_desc<BF16>(sa_lo + ks * A_KSTEP, A_MN, lbo);
               const uint64_t b_lo = make_desc<BF16>(sb_lo + ks * B_KSTEP, B_MN, lbo);
+              // (split accumulators: the small terms in their own accumulator, one truncating add per K step on the main sum)
               if (CG2) {
-                umma2_f16(d_tmem, a_hi, b_lo, idesc, accumulate);
-                umma2_f16(d_tmem, a_lo, b_hi, idesc, 1u);
-                umma2_f16(d_tmem, a_hi, b_hi, idesc, 1u);
+                umma2_f16(d_small, a_hi, b_lo, idesc, accumulate);
+                umma2_f16(d_small, a_lo, b_hi, idesc, 1u);
+                umma2_f16(d_tmem, a_hi, b_hi, idesc, SPLIT ? accumulate : 1u);
               } else {
-                umma<true>(d_tmem, a_hi, b_lo, idesc, accumulate);   // small terms first
-                umma<true>(d_tmem, a_lo, b_hi, idesc, 1u);
-                umma<true>(d_tmem, a_hi, b_hi, idesc, 1u);
+                umma<true>(d_small, a_hi, b_lo, idesc, accumulate);   // small terms first
+                umma<true>(d_small, a_lo, b_hi, idesc, 1u);
+                umma<true>(d_tmem, a_hi, b_hi, idesc, SPLIT ? accumulate : 1u);
               }
               accumulate = 1;
             } else if (BF16) {
@@ -1322,6 +1324,23 @@ inline void launch_x2(const Params& p, bool a_mn, bool b_mn, int grid, cudaStrea
 template <int BN, bool A_MN, bool B_MN>
 inline cudaError_t set_x2_attr() {
   return set_smem_attr<BN, A_MN, B_MN, true, false, true, true, true, false, false, true>();
+}
+
+// operand pairs with split accumulators (Gram matrices: both operands row-index contiguous)
+template <int BN>
+inline void launch_x2s(const Params& p, int grid, cudaStream_t st) {
+  using CF = Cfg<BN, true, true, true, true, true, false, false, true>;
+  k_gemm_umma<BN, true, true, true, true, true, true, true, false, false, true><<<grid, CF::THREADS, CF::SMEM_BYTES, st>>>(p);
+}
+inline cudaError_t launch_x2s_pair(const Params& p, int grid, cudaStream_t st) {
+  using CF = Cfg<256, true, true, true, true, true, false, true, true>;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)grid); cfg.blockDim = dim3(CF::THREADS); cfg.dynamicSmemBytes = CF::SMEM_BYTES; cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr; cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, k_gemm_umma<256, true, true, true, true, true, true, true, false, true, true>, p);
 }
 
 // bf16 operand pairs on CTA pairs
@@ -1540,6 +1559,9 @@ inline int umma_configure() {
   if (e == cudaSuccess) e = set_x2_attr<256, false, true>();
   if (e == cudaSuccess) e = set_x2_attr<256, true, true>();
   if (e == cudaSuccess) e = set_x2_attr<256, true, false>();
+  if (e == cudaSuccess) e = set_smem_attr<128, true, true, true, true, true, true, true, false, false, true>();
+  if (e == cudaSuccess) e = set_smem_attr<256, true, true, true, true, true, true, true, false, false, true>();
+  if (e == cudaSuccess) e = set_smem_attr<256, true, true, true, true, true, true, true, false, true, true>();
   if (e == cudaSuccess) e = set_x2_pair_attr<false, false>();
   if (e == cudaSuccess) e = set_x2_pair_attr<false, true>();
   if (e == cudaSuccess) e = set_x2_pair_attr<true, true>();
@@ -1580,7 +1602,6 @@ inline int umma_try_launch(const GemmArgs& g_in, int precision, int sm_count, fl
   if (nbat > 1 && (g.a2_mode == ADD_BF16 || (variant & UMMA_VARIANT_REGISTER_LOADS) || (g.bs2 % 4))) return 0;
   if ((g.c_tab != nullptr || g.c2_tab != nullptr) && (nbat < 2 || nbat > GEMM_TAB_MAX)) return 0;
   if (g.c_tab != nullptr && g.epi == EPI_STORE) return 0;   // (a plain store may split K: its reduction wants one stride)
-  if (g.alpha_dev != nullptr && g.epi == EPI_STORE) return 0;   // (the split-K reduction takes a host scalar)
   if (g.M < 128 || g.N < 64 || g.K < 64) return 0;
   if ((g.M % epc) || (g.N % epc) || (g.K % epc)) return 0;
   if (d16 && g.a2_mode != ADD_NONE) return 0;
@@ -1707,11 +1728,20 @@ inline int umma_try_launch(const GemmArgs& g_in, int precision, int sm_count, fl
   p.withhold_arrive = withhold ? 1 : 0;
   // 32 K blocks per accumulation chain: 1024 k (8e-6 relative error in fp32 mode, 1.4e-6 with
   // split accumulators); 2048 k for bf16 operands loaded through registers
-  p.kc = 32;
+  p.kc = (x2 && g.precise) ? 16 : 32;      // (K blocks of 64 there: the same 1024 k per chain as the fp32 products)
   const int grid = cg2 ? 2 * (p.num_items < nclusters ? p.num_items : nclusters)
                        : (p.num_items < sm_count ? p.num_items : sm_count);
   const bool one = g.tf32x1 && !bf16 && tma && !a_mn && !b_mn && g.a2_mode == ADD_NONE && !g.precise && splits == 1;
-  if (cg2 && x2) {
+  if (x2 && g.precise) {   // (only the layout of a Gram matrix is built with split accumulators)
+    if (!a_mn || !b_mn) return 0;
+    if (cg2) {
+      if (launch_x2s_pair(p, grid, st) != cudaSuccess) { cudaGetLastError(); return DION_ERR_CUDA; }
+    } else if (BN == 256) {
+      launch_x2s<256>(p, grid, st);
+    } else {
+      launch_x2s<128>(p, grid, st);
+    }
+  } else if (cg2 && x2) {
     if (launch_x2_pair(p, a_mn, b_mn, grid, st) != cudaSuccess) { cudaGetLastError(); return DION_ERR_CUDA; }
   } else if (cg2) {
     const cudaError_t e = g.precise ? launch_pair<true>(p, a_mn, b_mn, grid, st) : launch_pair<false>(p, a_mn, b_mn, grid, st);
@@ -1762,7 +1792,8 @@ inline int umma_try_launch(const GemmArgs& g_in, int precision, int sm_count, fl
     int blocks = (int)((total + 255) / 256);
     if (blocks > 8 * sm_count) blocks = 8 * sm_count;
     k_splitk_reduce<<<dim3((unsigned)blocks, (unsigned)nbat), 256, 0, st>>>(part, splits, g.M, g.N, g.C, g.ldc, g.alpha, g.tri, 128, g.skip_flag,
-                                                                            nbat > 1 ? g.bs2 : 0, nbat > 1 ? g.skip_stride : 0);
+                                                                            nbat > 1 ? g.bs2 : 0, nbat > 1 ? g.skip_stride : 0, g.alpha_dev,
+                                                                            g.alpha_dev_stride);
     if (cudaGetLastError() != cudaSuccess) return DION_ERR_CUDA;
     return 2;
   }
