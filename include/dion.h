@@ -57,12 +57,17 @@ typedef struct dion_ctx dion_ctx; /* opaque; owns scratch memory only */
 
 typedef enum { DION_F32 = 0, DION_BF16 = 1 } dion_dtype;
 
-/* Arithmetic of the four large contractions (P, R, U R^T, U Q^T).
- * DION_PREC_FP32:           products carry fp32 accuracy (fp32 FMA, or a 3-term
- *                           TF32 split on the tensor cores), fp32 accumulation.
- * DION_PREC_BF16_OPERANDS:  operands rounded to bf16 (M + G is added in fp32, then
- *                           rounded), fp32 accumulation.
- * The products inside Orthonormalize keep fp32 accuracy in both modes.          */
+/* Arithmetic of the four large contractions (P, R, U R^T, U Q^T); accumulation is fp32 everywhere.
+ * DION_PREC_FP32:           X, M and Q stay within 1e-4 (relative, Frobenius) of the rule evaluated in float64
+ *                           wherever the rule itself is that well determined.  On the FMA engine every product is
+ *                           fp32.  On the tensor cores each product runs at the cheapest arithmetic that keeps
+ *                           the bound: P with 22 significant bits (3-term TF32 split), or, on large matrices, with
+ *                           16 bits first (pairs of bf16 arrays) and again with 22 when the orthonormalization's
+ *                           probe finds the panel ill conditioned; R and U R^T with 16 bits (bf16 pairs, ~1e-5 of
+ *                           the product; U R^T enters M scaled by 1 - mu); U Q^T with 11 bits on factors rounded
+ *                           to nearest (3e-4 of the update, 3e-6 of X).
+ * DION_PREC_BF16_OPERANDS:  operands rounded to bf16 (M + G is added in fp32, then rounded); 3e-2 on X, M, Q.
+ * The products inside Orthonormalize carry 22 significant bits in both modes.          */
 typedef enum { DION_PREC_FP32 = 0, DION_PREC_BF16_OPERANDS = 1 } dion_precision;
 
 /* Orthonormalize (Section 3.2 and the appendix on Cholesky QR).
