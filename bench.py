@@ -49,16 +49,25 @@ FFMA_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12     # 148 SMs x 128 FMA lanes 
 TRAFFIC_RATIOS = {
     # M + G kept in scratch: P, R and the error feedback read 4 bytes per element where the algorithmic model
     # counts M and G (the elementwise pass that forms the sum is another kernel)
-    "fp32_sum_in_scratch": (0.604, "ncu --set full, one step on 4096^2 r=1024, fp32 mode: 445.6 MB / 738.3 MB"),
+    "fp32_sum_in_scratch": (0.574, "ncu --set full, one step on 4096^2 r=1024, fp32 G, fp32 mode: P 90.9 + R 91.6 + error "
+                                   "feedback 144.8 + X 95.8 = 423.6 MB / 738.3 MB"),
+    "fp32_sum_in_scratch_bf16_g": (0.817, "the same on 14336x4096 r=1024 with bf16 G (the dominant shape of the Llama lists; the "
+                                          "model counts 2 bytes for G there): 368 + 317 + 549 + 451 = 1685 MB / 2063.6 MB"),
+    "fp32_sum_in_scratch_low_rank": (0.718, "the same on 16384^2 r=256 (rank fraction 1/64), fp32 G: 1.30 + 1.30 + 2.32 + 2.12 = "
+                                            "7.03 GB / 9.80 GB"),
     "fp32_fused_add": (0.885, "same capture with M + G formed inside P and R (the path below rank fraction 1/64)"),
     "bf16_arrays": (0.99, "ncu --set full, 8192^2 r=512, bf16-operand mode: error feedback 0.98, X update 0.93, P 1.07"),
 }
 
 
-def traffic_variant(m, n, r, precision):
+def traffic_variant(m, n, r, precision, gbytes=4):
     if precision == 1:
         return "bf16_arrays"
-    return "fp32_sum_in_scratch" if 64 * r >= min(m, n) else "fp32_fused_add"
+    if 64 * r < min(m, n):
+        return "fp32_fused_add"
+    if gbytes == 2:
+        return "fp32_sum_in_scratch_bf16_g"
+    return "fp32_sum_in_scratch" if 8 * r >= min(m, n) else "fp32_sum_in_scratch_low_rank"
 
 
 def load_peaks():
@@ -668,7 +677,7 @@ def workload_record(wid, cases, grouped, args, peaks, binding, ms_step, e2e_ms, 
                 f["COLNORM"] = 3.0 * m * r
             by["R"] = 0.0
             by["ORTH"] = refresh * (2.0 * by["P"] + by["ORTH"]); by["ORTH_GEMM"] = refresh * by["ORTH_GEMM"]
-        ratio = TRAFFIC_RATIOS[traffic_variant(m, n, r, args.precision)][0]
+        ratio = TRAFFIC_RATIOS[traffic_variant(m, n, r, args.precision, case_gbytes(c))][0]
         for p in binding.PHASES:
             tot_fl[p] += fl[p] * reps_per_step; tot_by[p] += by[p] * reps_per_step; exe_fl[p] += fx[p] * reps_per_step
         traffic += ratio * sum(by[p] for p in ("P", "R", "EF", "X")) * reps_per_step

@@ -658,8 +658,8 @@ int probe(StepCtx& s, i64 off, i64 rows, i64 r, int phase) {
 
 // Tall panels whose Gram matrix runs on scaled half pairs (the rule looks at the shape alone).
 bool gram_on_pairs(const StepCtx& s, i64 rows, i64 r) {
-  return s.tensor && s.c->cfg.precision == DION_PREC_FP32 && rows % 8 == 0 && r % 8 == 0 && r >= 128 &&
-         (double)rows * (double)r * (double)r >= GRAM_PAIR_MIN_FLOPS;
+  return s.tensor && rows % 8 == 0 && r % 8 == 0 && r >= 128 &&
+         (double)rows * (double)r * (double)r >= GRAM_PAIR_MIN_FLOPS;      // (in either precision mode)
 }
 
 // One Cholesky-QR round on every matrix of the chain: Pout = Pin * chol(Pin^T Pin)^-T.

@@ -32,7 +32,8 @@ def test_workloads_match_the_configurations():
     assert bench.oracle_sample_cases(l8, "llama8b") == [(1024, 4096, 256), (4096, 4096, 1024)]
     assert bench.oracle_sample_cases(large, "large") == [(16384, 16384, 256)]
     assert bench.traffic_variant(4096, 4096, 1024, 0) == "fp32_sum_in_scratch"
-    assert bench.traffic_variant(4096, 4096, 256, 0) == "fp32_sum_in_scratch" and bench.traffic_variant(16384, 16384, 128, 0) == "fp32_fused_add"
+    assert bench.traffic_variant(4096, 4096, 256, 0) == "fp32_sum_in_scratch_low_rank" and bench.traffic_variant(16384, 16384, 128, 0) == "fp32_fused_add"
+    assert bench.traffic_variant(14336, 4096, 1024, 0, 2) == "fp32_sum_in_scratch_bf16_g"
     assert bench.traffic_variant(4096, 4096, 256, 1) == "bf16_arrays"
 
 
