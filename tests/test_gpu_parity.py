@@ -517,6 +517,31 @@ def _nearly_parallel(Q, delta):
     return (Qb / Qb.norm(dim=0)).contiguous()
 
 
+@pytest.mark.parametrize("scale_exp", [-40, 20])
+def test_gradient_scale_does_not_matter_to_the_16_bit_paths(scale_exp):
+    # The Gram matrix of a tall panel runs on a pair of IEEE HALF arrays (5 exponent bits) after scaling the panel
+    # by a power of two found on the device, and the X update on half factors whose entries are at most 1: neither
+    # may depend on the scale of the gradient.  4096 x 4096 at r = 1024 takes both paths (and P on bf16 pairs);
+    # gradients scaled by 2^-40 and 2^20 must give the oracle's X, M, Q on the same scaled inputs.
+    from oracle import dion_oracle as orc
+    m = n = 4096
+    r = 1024
+    pb = inputs.make_problem(m, n, r, seed=61, ks=64)
+    sc = 2.0 ** scale_exp
+    G = pb.grad(0) * sc
+    M0 = (0.5 * pb.grad(1)) * sc                      # a non-zero momentum of the same scale
+    want = orc.step(to_np64(pb.X), to_np64(M0), to_np64(G), to_np64(pb.Q), MU, ETA, EPS)
+    X, M, Q = pb.X.cuda().clone(), M0.cuda().clone(), pb.Q.cuda().clone()
+    d = torch.zeros(r, device="cuda")
+    with binding.Dion(mu=MU, eps=EPS) as opt:
+        opt.step(X, M, G.cuda(), Q, ETA, colnorm_out=d)
+        assert opt.get_status() == (0, 0) and opt.orth_rounds() == 1 and opt.fallbacks() == 0
+    errs = {"X": rel(to_np64(X), want.X), "M": rel(to_np64(M), want.M), "Q": rel(to_np64(Q), want.Q),
+            "d": rel(to_np64(d), want.d)}
+    print(f"gradient scale 2^{scale_exp}: " + " ".join(f"{k} {v:.2e}" for k, v in errs.items()))
+    assert all(v <= TOL_FP32 for v in errs.values()), errs
+
+
 def test_fast_panel_is_recomputed_when_the_probe_rejects_it():
     # 4096^2 at r = 1024 is large enough for P = (M + G) Q to run on bf16 operand pairs first (~1e-5).
     # (i) the workload's own warm start: well conditioned, the probe accepts the first round, one round of work,
