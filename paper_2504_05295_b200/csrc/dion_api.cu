@@ -650,7 +650,7 @@ int probe(StepCtx& s, i64 off, i64 rows, i64 r, int phase) {
   launch_pdl(k_probe_w, dim3((unsigned)((r + 127) / 128), (unsigned)chunks, (unsigned)s.nb), dim3(128), 0, s.st,
              (const float*)(s.ws + off), r, rows, r, per, (const float*)(s.ws + s.L.probe_y), s.ws + s.L.probe_part, s.wstride, keep);
   DION_CHECK_LAUNCH(c);
-  launch_pdl(k_probe_decide, dim3((unsigned)s.nb), dim3(r >= 1024 ? 1024 : 256), 0, s.st, (const float*)(s.ws + s.L.probe_part), chunks, r, s.os,
+  launch_pdl(k_probe_decide, dim3((unsigned)s.nb), dim3(r >= 128 ? 1024 : 256), 0, s.st, (const float*)(s.ws + s.L.probe_part), chunks, r, s.os,
              ORTH_TAU_F, c->dev_ints + 2, s.wstride, phase);
   DION_CHECK_LAUNCH(c);
   return DION_OK;

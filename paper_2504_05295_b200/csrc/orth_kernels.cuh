@@ -739,14 +739,12 @@ __global__ void __launch_bounds__(1024) k_probe_decide(const float* __restrict__
   }
   __shared__ float red[1024];
   float e = 0.f;
-  for (i64 j = threadIdx.x; j < r; j += blockDim.x) {
-#pragma unroll
-    for (int p = 0; p < NPROBE; ++p) {
-      float w = 0.f;
-      for (int c = 0; c < chunks; ++c) w += part[((i64)c * r + j) * NPROBE + p];
-      const float dlt = w - probe_sign(j, p);
-      e = fmaf(dlt, dlt, e);
-    }
+  // one (column, probe) entry per thread at a time: consecutive threads read consecutive words of a chunk's partials
+  for (i64 x = threadIdx.x; x < r * NPROBE; x += blockDim.x) {
+    float w = 0.f;
+    for (int c = 0; c < chunks; ++c) w += part[(i64)c * r * NPROBE + x];
+    const float dlt = w - probe_sign(x / NPROBE, (int)(x % NPROBE));
+    e = fmaf(dlt, dlt, e);
   }
   red[threadIdx.x] = e;
   __syncthreads();
