@@ -602,7 +602,7 @@ __device__ __forceinline__ float probe_sign(i64 j, int p) {
 __global__ void __launch_bounds__(256) k_probe_y(const float* __restrict__ U, i64 ld, i64 rows, i64 r,
                                                  float* __restrict__ Y, i64 wstride, const int* __restrict__ keep) {
   pdl_enter();
-  if (keep != nullptr && keep[(i64)blockIdx.y * OS_SLOT_INTS] != 0) return;   // this panel's verdict stands
+  if (keep != nullptr && keep[(i64)blockIdx.y * OS_SLOT_INTS] != 0) return;   // this panel's decision stands
   U += (i64)blockIdx.y * wstride; Y += (i64)blockIdx.y * wstride;
   const int lane = threadIdx.x & 31;
   const i64 warp = (i64)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
@@ -640,7 +640,7 @@ __global__ void __launch_bounds__(256) k_probe_y4(const float* __restrict__ U, i
                                                   float* __restrict__ Y, i64 wstride, const int* __restrict__ keep) {
   extern __shared__ float py_sign[];      // [column in block][probe]
   pdl_enter();
-  if (keep != nullptr && keep[(i64)blockIdx.y * OS_SLOT_INTS] != 0) return;   // this panel's verdict stands
+  if (keep != nullptr && keep[(i64)blockIdx.y * OS_SLOT_INTS] != 0) return;   // this panel's decision stands
   U += (i64)blockIdx.y * wstride; Y += (i64)blockIdx.y * wstride;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const i64 group0 = (i64)blockIdx.x * 8 + warp, groups = (i64)gridDim.x * 8;
@@ -725,7 +725,7 @@ __global__ void __launch_bounds__(128) k_probe_w(const float* __restrict__ U, i6
 // Counts the rounds of the step that did work (1 or 2; with a recomputed panel 2 or 3).
 // phase PROBE_FAST (the round ran on a panel from the fast product): done -> OS_DONE = 1, else 0 (a failed pivot
 // too: the panel is recomputed before the fallback sees it); nothing is counted.  PROBE_AFTER_REDO: a panel that
-// passed PROBE_FAST keeps its verdict (one round); otherwise its recomputed first round is judged.
+// passed PROBE_FAST keeps its decision (one round); otherwise its recomputed first round is judged.
 enum : int { PROBE_CHECK = 0, PROBE_FAST = 1, PROBE_AFTER_REDO = 2 };
 __global__ void __launch_bounds__(1024) k_probe_decide(const float* __restrict__ part, int chunks, i64 r,
                                                       int* __restrict__ os, float tau_f,

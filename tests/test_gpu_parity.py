@@ -263,6 +263,35 @@ def test_repeated_runs_are_bit_identical(m, n, r, precision):
         assert opt.get_status() == (0, 0)
 
 
+@pytest.mark.parametrize("shape", [(2048, 1536, 256), (1024, 768, 100), (4096, 4096, 1024)])
+def test_orthogonality_probe_estimates_the_frobenius_deviation(shape):
+    # the device's estimate of |U1^T U1 - I|_F^2 (8 fixed sign vectors, two passes over the panel) against the same
+    # quantity computed in float64 from the U the step used (one round passed, so U = U1).  r a multiple of 4 from
+    # 128 up takes the kernel with the sign table in shared memory, smaller or odd r the plain one.
+    import ctypes
+    m, n, r = shape
+    pb = inputs.make_problem(m, n, r, seed=71, ks=32, device="cuda")
+    lib = binding.load_library()
+    lib.dion_debug_orth_measure.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.POINTER(ctypes.c_float)]
+    lib.dion_debug_orth_measure.restype = ctypes.c_int
+    P = torch.empty(m, r, device="cuda")
+    W = torch.empty(n, r, device="cuda")
+    flag = torch.zeros(1, dtype=torch.int32, device="cuda")
+    with binding.Dion(mu=MU, eps=EPS, orth=binding.ORTH_CHOLQR2) as opt:
+        desc = binding.matrix_desc(pb.X, pb.M, pb.grad(0), pb.Q)
+        opt.dp_project(desc, P, flag)
+        opt.dp_factor(desc, P, W, flag)
+        assert opt.get_status() == (0, 0) and opt.orth_rounds() == 1
+        est = ctypes.c_float(0.0)
+        assert lib.dion_debug_orth_measure(opt._ctx, ctypes.c_void_p(int(torch.cuda.current_stream().cuda_stream)),
+                                           ctypes.byref(est)) == 0
+    U = P.double()
+    true = float(((U.t() @ U - torch.eye(r, device="cuda", dtype=torch.float64)) ** 2).sum())
+    print(f"{shape}: estimate {est.value:.3e}, |U^T U - I|_F^2 {true:.3e}")
+    assert 0.4 * true <= est.value <= 2.5 * true
+    assert est.value <= (3e-5) ** 2 * r          # what let the device skip the second round
+
+
 def test_cholqr2_takes_its_second_round_only_when_the_first_is_not_enough():
     m, n, r = 1024, 768, 128
     pb = inputs.make_problem(m, n, r, seed=15, ks=16)
