@@ -38,6 +38,7 @@ constexpr float GOOD_REL = 1e-4f;         // smallest relative pivot of a round 
 constexpr float ORTH_TAU_F = 3e-5f;
 constexpr float DONE_REL = 0.9f;          // smallest relative pivot of a round whose input was already orthonormal
 constexpr i64 PART_CAP_FLOATS = (i64)16 << 20;  // split-K partial sums, at most 64 MiB
+constexpr double P_HALF_MIN_MNR = 4e9;          // smallest m n r whose full-rank P runs on scaled half pairs
 constexpr double GRAM_PAIR_MIN_FLOPS = 2e9;     // smallest rows r^2 whose Gram matrix runs on scaled half pairs
 constexpr double P_PAIR_MIN_MNR = 1.5e10;       // smallest m n r whose P = (M + G) Q runs on bf16 operand pairs first
 
@@ -54,6 +55,8 @@ struct Layout {
   i64 fb_part, fb_h, fb_n;  // fallback kernel: partial dot products (SMs x r), their sums (r), partial norms (SMs)
   i64 probe_y, probe_part;  // CholeskyQR2's orthogonality probe: U1 z (rows x NPROBE), partial U1^T (U1 z)
   i64 Bp;                   // fp32 mode, M + G in scratch: the same sum as a bf16 (hi, lo) pair (m x n x 2 bf16) for R; 0: none
+  i64 Bh;                   // full rank: M + G as a scaled pair of half arrays for P (m x n x 2 halves), 0: none
+  i64 pmax;                 // ... its partial maxima and the product's scale factor (like gmax)
   i64 gmax;                 // Gram matrices on half pairs: AMAX_PARTS partial maxima of |P|, then 1 / scale^2
   i64 Qc;                   // fp32 mode, large matrices: dense fp32 copy of Q for the chain-wide recomputation of P (0: none)
   i64 S16;                  // fp32 mode: the bf16 (hi, lo) pair of the error feedback's second factor (max(m,n) x r x 2 bf16)
@@ -124,6 +127,16 @@ bool sum_in_scratch(const dion_ctx* c, i64 m, i64 n, i64 r) {
          m % 4 == 0 && n % 4 == 0 && m >= 128 && n >= 128 && r >= 64 && 64 * r >= sd;
 }
 
+// Above rank fraction 1/4 (the adaptive rounds: ill-conditioned panels) P = (M + G) Q needs its 22 significant
+// bits.  On large matrices it takes them from scaled pairs of IEEE half arrays (three kind::f16 MMAs per K step,
+// split accumulators) instead of the 3xTF32 split with four kind::tf32 ones: M + G is scaled by a power of two
+// found on the device, Q (unit-norm columns) by 2^13.
+int resolve_orth(const dion_ctx* c, i64 r, i64 short_dim);
+bool p_on_half_pairs(const dion_ctx* c, i64 m, i64 n, i64 r) {
+  return c->cfg.precision == DION_PREC_FP32 && c->cfg.engine != DION_ENGINE_SIMT && m % 8 == 0 && n % 8 == 0 && r % 8 == 0 &&
+         (double)m * (double)n * (double)r >= P_HALF_MIN_MNR && resolve_orth(c, r, (m < n) ? m : n) == DION_ORTH_SHIFTED3;
+}
+
 // A step whose orthonormalization may resolve to CholeskyQR2 keeps the panel for the device-side fallback.
 bool may_fallback(const dion_ctx* c, i64 m, i64 n, i64 r) {
   const i64 sd = (m < n) ? m : n;
@@ -176,6 +189,11 @@ Layout make_layout(const dion_ctx* c, i64 m, i64 n, i64 r) {
   }
   L.Psave = L.fb_part = L.fb_h = L.fb_n = 0;
   L.gmax = o; o += align64(AMAX_PARTS + 64);
+  L.Bh = L.pmax = 0;
+  if (L.Bp > 0 && p_on_half_pairs(c, m, n, r)) {
+    L.Bh = o; o += align64(m * n);
+    L.pmax = o; o += align64(AMAX_PARTS + 64);
+  }
   L.Qc = 0;
   if (L.Bp > 0 && (double)m * (double)n * (double)r >= P_PAIR_MIN_MNR) { L.Qc = o; o += align64(big * r); }
   L.S16 = o; o += align64(big * r);
@@ -404,7 +422,8 @@ int launch_gemm_group(StepCtx& s, const std::vector<GemmArgs>& v) {
     const GemmArgs& g = v[b];
     one = g.M == a.M && g.N == a.N && g.K == a.K && g.a_si == a.a_si && g.a_sk == a.a_sk && g.a2_si == a.a2_si &&
           g.a2_sk == a.a2_sk && g.a2_mode == a.a2_mode && g.b_sk == a.b_sk && g.b_sn == a.b_sn && g.ldc == a.ldc &&
-          g.epi == a.epi && g.ldc2 == a.ldc2 && g.c2_mode == a.c2_mode && g.alpha == a.alpha && g.alpha_dev == a.alpha_dev &&
+          g.epi == a.epi && g.ldc2 == a.ldc2 && g.c2_mode == a.c2_mode && g.alpha == a.alpha &&
+          (g.alpha_dev == a.alpha_dev || at_stride(a.alpha_dev, g.alpha_dev, b)) &&
           g.batch == 1 && a.batch == 1 && g.tri == a.tri && g.klimit == a.klimit && g.precise == a.precise &&
           g.ab16 == a.ab16 && g.f16 == a.f16 && g.tf32x1 == a.tf32x1 && at_stride(a.A, g.A, b) && at_stride(a.B, g.B, b) &&
           at_stride(a.A2, g.A2, b) && at_stride(a.A16lo, g.A16lo, b) && at_stride(a.B16lo, g.B16lo, b) &&
@@ -417,6 +436,7 @@ int launch_gemm_group(StepCtx& s, const std::vector<GemmArgs>& v) {
   if (one) {
     GemmArgs gb = a;
     over_batch(s, gb);
+    if (nb > 1 && v[1].alpha_dev != a.alpha_dev) gb.alpha_dev_stride = s.wstride;     // a scale per matrix, in its scratch slice
     float* ctab[GEMM_TAB_MAX];
     const void* c2tab[GEMM_TAB_MAX];
     for (int b = 0; b < nb; ++b) { ctab[b] = v[b].C; c2tab[b] = v[b].C2; }
@@ -698,7 +718,7 @@ int cholqr_round(StepCtx& s, i64 pin_off, i64 pout_off, i64 rows, i64 r, int mod
     DION_CHECK_LAUNCH(c);
     launch_pdl(k_split_f16_scaled, dim3((unsigned)grid_for(c, rows * r / 8), (unsigned)s.nb), dim3(256), 0, s.st,
                (const float*)(s.ws + pin_off), r, rows, r, (const float*)(s.ws + s.L.gmax), (int)parts, hi, lo, s.ws + s.L.gmax + AMAX_PARTS,
-               s.wstride, sk, (i64)OS_SLOT_INTS);
+               s.wstride, sk, (i64)OS_SLOT_INTS, -1.f);
     DION_CHECK_LAUNCH(c);
     g.ab16 = 1; g.f16 = 1;
     g.A = reinterpret_cast<const float*>(hi); g.A16lo = lo;
@@ -1400,6 +1420,34 @@ int step_batch(dion_ctx* c, const dion_matrix* const* list, int nb, float lr, cu
   const float* srcs[MAX_CHAIN];
   i64 lds[MAX_CHAIN];
   if (b32) DION_TRY(form_sum_chain(s, list, bpair));
+  const bool phalf = b32 && s.L.Bh > 0;
+  bool p_half_ready = false;
+  if (phalf) {      // the scaled half pairs of M + G and of Q, for the whole chain
+    bool all_ok = true;
+    for (int b = 0; b < nb; ++b) {
+      all_ok = all_ok && !((uintptr_t)list[b]->Q & 15) && list[b]->ldq % 4 == 0 && list[b]->ldq == list[0]->ldq;
+      srcs[b] = (const float*)list[b]->Q;
+    }
+    if (all_ok && nb <= GEMM_TAB_MAX) {
+      i64 parts = (m * n / 4 + 2047) / 2048;
+      if (parts > AMAX_PARTS) parts = AMAX_PARTS;
+      __half* bh = reinterpret_cast<__half*>(s.ws + s.L.Bh);
+      launch_pdl(k_absmax_partial, dim3((unsigned)parts, (unsigned)nb), dim3(256), 0, st, (const float*)(s.ws + s.L.B32), n, m, n,
+                 s.ws + s.L.pmax, s.wstride, (const int*)nullptr, (i64)0);
+      DION_CHECK_LAUNCH(c);
+      launch_pdl(k_split_f16_scaled, dim3((unsigned)grid_for(c, m * n / 8), (unsigned)nb), dim3(256), 0, st,
+                 (const float*)(s.ws + s.L.B32), n, m, n, (const float*)(s.ws + s.L.pmax), (int)parts, bh, bh + m * n,
+                 s.ws + s.L.pmax + AMAX_PARTS, s.wstride, (const int*)nullptr, (i64)0, ldexpf(1.f, -13));
+      DION_CHECK_LAUNCH(c);
+      ChainPtrs t;
+      for (int b = 0; b < nb; ++b) t.p[b] = srcs[b];
+      __half* qh = reinterpret_cast<__half*>(s.ws + s.L.S16);
+      launch_pdl(k_split_f16_fixed, dim3((unsigned)grid_for(c, qrow * r / 8), (unsigned)nb), dim3(256), 0, st, t, list[0]->ldq, qrow, r,
+                 ldexpf(1.f, 13), qh, qh + qrow * r, s.wstride);
+      DION_CHECK_LAUNCH(c);
+      p_half_ready = true;
+    }
+  }
   bool q_split = false;
   if (b32 && ppair) {
     bool all_ok = true;
@@ -1438,6 +1486,13 @@ int step_batch(dion_ctx* c, const dion_matrix* const* list, int nb, float lr, cu
       p.A = (const float*)bh; p.A16lo = bh + m * n; p.a_si = tr ? 1 : n; p.a_sk = tr ? n : 1;
       p.B = (const float*)qh; p.B16lo = ql; p.b_sk = r; p.b_sn = 1;
       any_pair = true;
+    } else if (p_half_ready) {
+      __half* bh = reinterpret_cast<__half*>(s.W(b, s.L.Bh));
+      __half* qh = reinterpret_cast<__half*>(s.W(b, s.L.S16));
+      p.ab16 = 1; p.f16 = 1;
+      p.A = (const float*)bh; p.A16lo = bh + m * n; p.a_si = tr ? 1 : n; p.a_sk = tr ? n : 1;
+      p.B = (const float*)qh; p.B16lo = qh + qrow * r; p.b_sk = r; p.b_sn = 1;
+      p.alpha_dev = s.W(b, s.L.pmax) + AMAX_PARTS;
     } else if (b32) {
       p.A = s.W(b, s.L.B32); p.a_si = tr ? 1 : n; p.a_sk = tr ? n : 1;
       p.B = (const float*)a->Q; p.b_sk = a->ldq; p.b_sn = 1;

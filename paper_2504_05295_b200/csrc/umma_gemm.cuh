@@ -1326,12 +1326,13 @@ inline cudaError_t set_x2_attr() {
   return set_smem_attr<BN, A_MN, B_MN, true, false, true, true, true, false, false, true>();
 }
 
-// operand pairs with split accumulators (Gram matrices: both operands row-index contiguous)
-template <int BN>
+// operand pairs with split accumulators: B row-index contiguous (Gram matrices: A too; P = (M + G) Q: A k-contiguous)
+template <int BN, bool A_MN>
 inline void launch_x2s(const Params& p, int grid, cudaStream_t st) {
   using CF = Cfg<BN, true, true, true, true, true, false, false, true>;
-  k_gemm_umma<BN, true, true, true, true, true, true, true, false, false, true><<<grid, CF::THREADS, CF::SMEM_BYTES, st>>>(p);
+  k_gemm_umma<BN, A_MN, true, true, true, true, true, true, false, false, true><<<grid, CF::THREADS, CF::SMEM_BYTES, st>>>(p);
 }
+template <bool A_MN>
 inline cudaError_t launch_x2s_pair(const Params& p, int grid, cudaStream_t st) {
   using CF = Cfg<256, true, true, true, true, true, false, true, true>;
   cudaLaunchConfig_t cfg = {};
@@ -1340,7 +1341,7 @@ inline cudaError_t launch_x2s_pair(const Params& p, int grid, cudaStream_t st) {
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr; cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, k_gemm_umma<256, true, true, true, true, true, true, true, false, true, true>, p);
+  return cudaLaunchKernelEx(&cfg, k_gemm_umma<256, A_MN, true, true, true, true, true, true, false, true, true>, p);
 }
 
 // bf16 operand pairs on CTA pairs
@@ -1562,6 +1563,9 @@ inline int umma_configure() {
   if (e == cudaSuccess) e = set_smem_attr<128, true, true, true, true, true, true, true, false, false, true>();
   if (e == cudaSuccess) e = set_smem_attr<256, true, true, true, true, true, true, true, false, false, true>();
   if (e == cudaSuccess) e = set_smem_attr<256, true, true, true, true, true, true, true, false, true, true>();
+  if (e == cudaSuccess) e = set_smem_attr<128, false, true, true, true, true, true, true, false, false, true>();
+  if (e == cudaSuccess) e = set_smem_attr<256, false, true, true, true, true, true, true, false, false, true>();
+  if (e == cudaSuccess) e = set_smem_attr<256, false, true, true, true, true, true, true, false, true, true>();
   if (e == cudaSuccess) e = set_x2_pair_attr<false, false>();
   if (e == cudaSuccess) e = set_x2_pair_attr<false, true>();
   if (e == cudaSuccess) e = set_x2_pair_attr<true, true>();
@@ -1732,14 +1736,15 @@ inline int umma_try_launch(const GemmArgs& g_in, int precision, int sm_count, fl
   const int grid = cg2 ? 2 * (p.num_items < nclusters ? p.num_items : nclusters)
                        : (p.num_items < sm_count ? p.num_items : sm_count);
   const bool one = g.tf32x1 && !bf16 && tma && !a_mn && !b_mn && g.a2_mode == ADD_NONE && !g.precise && splits == 1;
-  if (x2 && g.precise) {   // (only the layout of a Gram matrix is built with split accumulators)
-    if (!a_mn || !b_mn) return 0;
+  if (x2 && g.precise) {   // (built with split accumulators for B row-index contiguous: Gram matrices and P)
+    if (!b_mn) return 0;
     if (cg2) {
-      if (launch_x2s_pair(p, grid, st) != cudaSuccess) { cudaGetLastError(); return DION_ERR_CUDA; }
+      const cudaError_t e = a_mn ? launch_x2s_pair<true>(p, grid, st) : launch_x2s_pair<false>(p, grid, st);
+      if (e != cudaSuccess) { cudaGetLastError(); return DION_ERR_CUDA; }
     } else if (BN == 256) {
-      launch_x2s<256>(p, grid, st);
+      if (a_mn) launch_x2s<256, true>(p, grid, st); else launch_x2s<256, false>(p, grid, st);
     } else {
-      launch_x2s<128>(p, grid, st);
+      if (a_mn) launch_x2s<128, true>(p, grid, st); else launch_x2s<128, false>(p, grid, st);
     }
   } else if (cg2 && x2) {
     if (launch_x2_pair(p, a_mn, b_mn, grid, st) != cudaSuccess) { cudaGetLastError(); return DION_ERR_CUDA; }
