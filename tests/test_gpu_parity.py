@@ -101,6 +101,44 @@ def test_strided_leading_dimensions(engine):
     assert torch.all(Xb[:, n:] == 7.0) and torch.all(Mb[:, n:] == 7.0) and torch.all(Qb[:, r:] == 7.0)
 
 
+@pytest.mark.parametrize("shape", [(512, 768, 128), (2048, 2048, 512)])
+def test_grouped_chain_with_mixed_leading_dimensions_equals_single_calls(shape):
+    # three matrices of one shape in a chain, one of them with padded leading dimensions (and one with only its Q
+    # padded): the chain-wide launches need common leading dimensions, so these chains fall back to one launch per
+    # matrix where they must -- same bits as single calls, padding untouched
+    m, n, r = shape
+    pbs = [inputs.make_problem(m, n, r, seed=81, k=k, ks=16) for k in range(3)]
+
+    def padded(t, pad):
+        buf = torch.full((t.shape[0], t.shape[1] + pad), 7.0, device="cuda", dtype=t.dtype)
+        v = buf[:, :t.shape[1]]
+        v.copy_(t)
+        return buf, v
+
+    def make_state():
+        out = []
+        for k, pb in enumerate(pbs):
+            px, pm, pq, pg = [(0, 0, 0, 0), (8, 4, 12, 16), (0, 0, 8, 0)][k]
+            Xb, X = padded(pb.X, px); Mb, M = padded(pb.M, pm); Qb, Q = padded(pb.Q, pq); Gb, G = padded(pb.grad(0), pg)
+            out.append((X, M, G, Q, (Xb, Mb, Qb)))
+        return out
+
+    with binding.Dion(mu=MU, eps=EPS) as opt:
+        single = make_state()
+        for X, M, G, Q, _ in single:
+            opt.step(X, M, G, Q, ETA)
+        grouped = make_state()
+        opt.step_grouped([(X, M, G, Q) for X, M, G, Q, _ in grouped], ETA)
+        assert opt.get_status() == (0, 0)
+    for k, (a, b) in enumerate(zip(single, grouped)):
+        for name, u, v in zip("XMQ", (a[0], a[1], a[3]), (b[0], b[1], b[3])):
+            assert torch.equal(u, v), f"matrix {k}: {name} differs between dion_step and dion_step_grouped"
+        Xb, Mb, Qb = b[4]
+        assert torch.all(Xb[:, n:] == 7.0) and torch.all(Mb[:, n:] == 7.0) and torch.all(Qb[:, r:] == 7.0)
+    ref = oracle_steps(pbs[1], 1)[0]
+    assert rel(to_np64(grouped[1][0]), ref.X) <= TOL_FP32 and rel(to_np64(grouped[1][3]), ref.Q) <= TOL_FP32
+
+
 @pytest.mark.parametrize("engine", ENGINES)
 def test_bf16_gradient_storage(engine):
     m, n, r = 512, 384, 96
