@@ -137,3 +137,20 @@ def test_transposed_form_in_bf16_operand_mode(m, n, r):
     for name, got, want in (("X", X, ref[4].X), ("M", M, ref[4].M), ("Q", Q, ref[4].Q)):
         e = rel(to_np64(got), want)
         assert e <= TOL_BF16, f"{name} off by {e:.2e}"
+
+
+def test_transposed_form_at_a_llama_shape_with_bf16_gradients():
+    # 14336 x 4096 at r = 1024 in the transposed form (the panel on the 4096 side): large enough for P on bf16 pairs
+    # with the probe-gated recomputation, the Gram matrix on half pairs and the chain of 512-column blocks
+    m, n, r = 14336, 4096, 1024
+    pb = inputs.make_problem(m, n, r, seed=29, ks=64, g_dtype=torch.bfloat16)
+    Q0 = row_side_factor(m, r, 7)
+    want = orc.step_transposed(to_np64(pb.X), to_np64(pb.M), to_np64(pb.grad(0)), to_np64(Q0), MU, ETA, EPS)
+    X, M, Q = pb.X.cuda().clone(), pb.M.cuda().clone(), Q0.cuda().clone()
+    d = torch.zeros(r, device="cuda")
+    with binding.Dion(mu=MU, eps=EPS) as opt:
+        opt.step(X, M, pb.grad(0).cuda(), Q, ETA, colnorm_out=d, transposed=True)
+        assert opt.get_status() == (0, 0) and opt.orth_rounds() == 1
+    errs = {"X": rel(to_np64(X), want.X), "M": rel(to_np64(M), want.M), "Q": rel(to_np64(Q), want.Q), "d": rel(to_np64(d), want.d)}
+    print("transposed 14336 x 4096 r=1024: " + " ".join(f"{k} {v:.2e}" for k, v in errs.items()))
+    assert all(v <= TOL_FP32 for v in errs.values()), errs
