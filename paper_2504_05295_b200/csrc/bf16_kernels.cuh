@@ -302,16 +302,18 @@ __global__ void __launch_bounds__(256) k_absmax_partial(const float* __restrict_
   if (threadIdx.x == 0) part[blockIdx.x] = red[0];
 }
 // other_inv < 0: the scalar written is 1 / scale^2 (both operands of the product are this array); else
-// other_inv / scale (the other operand carries a fixed scale of its own).
+// other_inv / scale (the other operand carries a fixed scale of its own), times *other_dev when that is given (the
+// other operand's own 1 / scale, written by its split; blockIdx.y entries wstride apart like everything else).
 __global__ void __launch_bounds__(256) k_split_f16_scaled(const float* __restrict__ src, i64 ld, i64 rows, i64 cols,
                                                           const float* __restrict__ part, int nparts,
                                                           __half* __restrict__ hi, __half* __restrict__ lo,
                                                           float* __restrict__ inv_scale2, i64 wstride,
                                                           const int* __restrict__ skip_flag, i64 skip_stride,
-                                                          float other_inv) {
+                                                          float other_inv, const float* __restrict__ other_dev = nullptr) {
   pdl_enter();
   if (skip_flag != nullptr && skip_flag[(i64)blockIdx.y * skip_stride] != 0) return;
   src += (i64)blockIdx.y * wstride; part += (i64)blockIdx.y * wstride; inv_scale2 += (i64)blockIdx.y * wstride;
+  if (other_dev != nullptr) other_dev += (i64)blockIdx.y * wstride;
   hi += 2 * (i64)blockIdx.y * wstride; lo += 2 * (i64)blockIdx.y * wstride;
   __shared__ float red[256];
   float m = 0.f;
@@ -328,7 +330,8 @@ __global__ void __launch_bounds__(256) k_split_f16_scaled(const float* __restric
   if (ex < -100) ex = -100;
   const float scale = ldexpf(1.f, 14 - ex);
   if (blockIdx.x == 0 && threadIdx.x == 0)
-    *inv_scale2 = (other_inv < 0.f) ? ldexpf(1.f, 2 * (ex - 14)) : other_inv * ldexpf(1.f, ex - 14);
+    *inv_scale2 = (other_inv < 0.f) ? ldexpf(1.f, 2 * (ex - 14))
+                                    : other_inv * ldexpf(1.f, ex - 14) * (other_dev != nullptr ? *other_dev : 1.f);
   const i64 per_row = cols / 8, total = rows * per_row;
   for (i64 e = (i64)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (i64)gridDim.x * blockDim.x) {
     const i64 i = e / per_row, c = (e - i * per_row) * 8;
@@ -349,10 +352,15 @@ __global__ void __launch_bounds__(256) k_split_f16_scaled(const float* __restric
 // hi = half(scale x), lo = half(scale x - hi) with a scale given by the caller (a power of two; for arrays whose
 // entries are bounded, like the unit-norm columns of Q).  Sources from a pointer table (blockIdx.y), outputs
 // `ostride` floats apart.
+// ldo: leading dimension of the outputs (0: dense).
 __global__ void __launch_bounds__(256) k_split_f16_fixed(const ChainPtrs srcs, i64 lds, i64 rows, i64 cols, float scale,
-                                                         __half* __restrict__ hi, __half* __restrict__ lo, i64 ostride) {
+                                                         __half* __restrict__ hi, __half* __restrict__ lo, i64 ostride,
+                                                         i64 ldo = 0, const int* __restrict__ skip_flag = nullptr,
+                                                         i64 skip_stride = 0) {
   pdl_enter();
   const i64 bm = blockIdx.y;
+  if (skip_flag != nullptr && skip_flag[bm * skip_stride] != 0) return;
+  if (ldo == 0) ldo = cols;
   const float* __restrict__ src = reinterpret_cast<const float*>(srcs.p[bm]);
   hi += 2 * bm * ostride; lo += 2 * bm * ostride;
   const i64 per_row = cols / 8, total = rows * per_row;
@@ -367,8 +375,8 @@ __global__ void __launch_bounds__(256) k_split_f16_fixed(const ChainPtrs srcs, i
       h[q] = __float2half_rn(v[q]);
       l[q] = __float2half_rn(v[q] - __half2float(h[q]));
     }
-    *reinterpret_cast<uint4*>(hi + i * cols + c) = *reinterpret_cast<const uint4*>(h);
-    *reinterpret_cast<uint4*>(lo + i * cols + c) = *reinterpret_cast<const uint4*>(l);
+    *reinterpret_cast<uint4*>(hi + i * ldo + c) = *reinterpret_cast<const uint4*>(h);
+    *reinterpret_cast<uint4*>(lo + i * ldo + c) = *reinterpret_cast<const uint4*>(l);
   }
 }
 

@@ -39,6 +39,7 @@ constexpr float ORTH_TAU_F = 3e-5f;
 constexpr float DONE_REL = 0.9f;          // smallest relative pivot of a round whose input was already orthonormal
 constexpr i64 PART_CAP_FLOATS = (i64)16 << 20;  // split-K partial sums, at most 64 MiB
 constexpr double P_HALF_MIN_MNR = 4e9;          // smallest m n r whose full-rank P runs on scaled half pairs
+constexpr double SOLVE_PAIR_MIN_PANEL = 3e7;    // smallest rows x r whose blocked solves run on scaled half pairs
 constexpr double GRAM_PAIR_MIN_FLOPS = 2e9;     // smallest rows r^2 whose Gram matrix runs on scaled half pairs
 constexpr double P_PAIR_MIN_MNR = 1.5e10;       // smallest m n r whose P = (M + G) Q runs on bf16 operand pairs first
 
@@ -57,6 +58,8 @@ struct Layout {
   i64 Bp;                   // fp32 mode, M + G in scratch: the same sum as a bf16 (hi, lo) pair (m x n x 2 bf16) for R; 0: none
   i64 Bh;                   // full rank: M + G as a scaled pair of half arrays for P (m x n x 2 halves), 0: none
   i64 pmax;                 // ... its partial maxima and the product's scale factor (like gmax)
+  i64 SolveP, LfP, smax;    // blocked solves on half pairs (r > 512): pair of a rows x 512 right-hand side; pairs of a row block of
+                            // the factor (512 x r) and of a diagonal inverse (512 x 512); partial maxima and scales
   i64 gmax;                 // Gram matrices on half pairs: AMAX_PARTS partial maxima of |P|, then 1 / scale^2
   i64 Qc;                   // fp32 mode, large matrices: dense fp32 copy of Q for the chain-wide recomputation of P (0: none)
   i64 S16;                  // fp32 mode: the bf16 (hi, lo) pair of the error feedback's second factor (max(m,n) x r x 2 bf16)
@@ -189,6 +192,12 @@ Layout make_layout(const dion_ctx* c, i64 m, i64 n, i64 r) {
   }
   L.Psave = L.fb_part = L.fb_h = L.fb_n = 0;
   L.gmax = o; o += align64(AMAX_PARTS + 64);
+  L.SolveP = L.LfP = L.smax = 0;
+  if (r > NBO_COLS && (double)big * (double)r >= SOLVE_PAIR_MIN_PANEL) {
+    L.SolveP = o; o += align64(big * NBO_COLS);
+    L.LfP = o; o += align64(NBO_COLS * r + NBO_COLS * NBO_COLS);
+    L.smax = o; o += align64(3 * (AMAX_PARTS + 64));
+  }
   L.Bh = L.pmax = 0;
   if (L.Bp > 0 && p_on_half_pairs(c, m, n, r)) {
     L.Bh = o; o += align64(m * n);
@@ -676,6 +685,15 @@ int probe(StepCtx& s, i64 off, i64 rows, i64 r, int phase) {
   return DION_OK;
 }
 
+// Tall panels whose blocked triangular solves run on scaled half pairs.
+// (where the solves are what the round waits for: CholeskyQR2 on large panels.  In the adaptive rounds they run
+// beside the serial chain, and on the panels of the 8B list the extra passes for scales and pairs cost what the
+// cheaper products save: measured, 42.1 -> 44.1 ms there, 48.1 -> 42.8 ms on the large squares.)
+bool solve_on_pairs(const StepCtx& s, i64 rows, i64 r, int mode) {
+  return s.tensor && s.nb <= GEMM_TAB_MAX && mode != RM_ADAPTIVE && rows % 8 == 0 && r % 8 == 0 &&
+         (double)rows * (double)r >= SOLVE_PAIR_MIN_PANEL;
+}
+
 // Tall panels whose Gram matrix runs on scaled half pairs (the rule looks at the shape alone).
 bool gram_on_pairs(const StepCtx& s, i64 rows, i64 r) {
   return s.tensor && rows % 8 == 0 && r % 8 == 0 && r >= 128 &&
@@ -718,7 +736,7 @@ int cholqr_round(StepCtx& s, i64 pin_off, i64 pout_off, i64 rows, i64 r, int mod
     DION_CHECK_LAUNCH(c);
     launch_pdl(k_split_f16_scaled, dim3((unsigned)grid_for(c, rows * r / 8), (unsigned)s.nb), dim3(256), 0, s.st,
                (const float*)(s.ws + pin_off), r, rows, r, (const float*)(s.ws + s.L.gmax), (int)parts, hi, lo, s.ws + s.L.gmax + AMAX_PARTS,
-               s.wstride, sk, (i64)OS_SLOT_INTS, -1.f);
+               s.wstride, sk, (i64)OS_SLOT_INTS, -1.f, (const float*)nullptr);
     DION_CHECK_LAUNCH(c);
     g.ab16 = 1; g.f16 = 1;
     g.A = reinterpret_cast<const float*>(hi); g.A16lo = lo;
@@ -749,7 +767,73 @@ int cholqr_round(StepCtx& s, i64 pin_off, i64 pout_off, i64 rows, i64 r, int mod
     // of the factorization, whose serial 64-column chain leaves most SMs idle.
     const float* Lm = s.ws + s.L.Gram;     // the factor, lower
     float* Wt = s.ws + (s.wt_off >= 0 ? s.wt_off : s.L.R);   // rows x 512 temporary (R is free during the orthonormalization)
+    // On tall panels the two products of a block column run on scaled half pairs (22 significant bits in three
+    // kind::f16 MMAs; 1024-k chains) like the Gram matrix: the right-hand side, the factor's row block and the
+    // diagonal inverse are scaled by powers of two found on the device, the finished columns of Pout (entries of
+    // an orthonormal basis; at most 1 / sqrt(pivot floor) = 100 in a deflating round) by 2^6.
+    const bool spairs = s.wt_off < 0 && s.L.SolveP > 0 && solve_on_pairs(s, rows, r, mode);
+    auto absmax_split = [&](const float* src, i64 ld, i64 nrows, i64 ncols, i64 out_off, i64 slot, float other_inv,
+                            const float* other_dev) -> int {
+      // pair of the nrows x ncols block at `src` (slice-relative pointer of matrix 0) into scratch at out_off; the
+      // scale factor goes to smax slot `slot`
+      i64 parts = (nrows * ncols / 4 + 2047) / 2048;
+      if (parts < 1) parts = 1;
+      if (parts > AMAX_PARTS) parts = AMAX_PARTS;
+      float* pm = s.ws + s.L.smax + slot * (AMAX_PARTS + 64);
+      launch_pdl(k_absmax_partial, dim3((unsigned)parts, (unsigned)s.nb), dim3(256), 0, s.st, src, ld, nrows, ncols, pm, s.wstride, skip,
+                 (i64)OS_SLOT_INTS);
+      DION_CHECK_LAUNCH(c);
+      __half* hi = reinterpret_cast<__half*>(s.ws + out_off);
+      launch_pdl(k_split_f16_scaled, dim3((unsigned)grid_for(c, nrows * ncols / 8), (unsigned)s.nb), dim3(256), 0, s.st, src, ld, nrows, ncols,
+                 (const float*)pm, (int)parts, hi, hi + nrows * ncols, pm + AMAX_PARTS, s.wstride, skip, (i64)OS_SLOT_INTS, other_inv, other_dev);
+      DION_CHECK_LAUNCH(c);
+      return DION_OK;
+    };
+    auto solve_block_pairs = [&](i64 J0, i64 sz) -> int {
+      const float* rhs = s.ws + pin_off + J0;
+      i64 rhs_ld = r;
+      __half* pop = reinterpret_cast<__half*>(s.ws + s.L.S16);          // pair of Pout: rows x r, dense
+      const float* sc = s.ws + s.L.smax;
+      if (J0 > 0) {
+        // W = rhs - Pout[:, :J0] L[J0:J0+sz, :J0]^T
+        DION_TRY(absmax_split(Lm + J0 * r, r, sz, J0, s.L.LfP, 0, ldexpf(1.f, -6), nullptr));
+        __half* lh = reinterpret_cast<__half*>(s.ws + s.L.LfP);
+        GemmArgs w = gemm_args();
+        w.M = rows; w.N = sz; w.K = J0;
+        w.ab16 = 1; w.f16 = 1;
+        w.A = (const float*)pop; w.A16lo = pop + rows * r; w.a_si = r; w.a_sk = 1;
+        w.B = (const float*)lh; w.B16lo = lh + sz * J0; w.b_sk = 1; w.b_sn = J0;
+        w.C = Wt; w.ldc = NBO; w.epi = EPI_C2_SUB; w.C2 = rhs; w.ldc2 = r; w.c2_mode = ADD_F32;
+        w.alpha_dev = sc + AMAX_PARTS; w.alpha_dev_stride = s.wstride;
+        w.skip_flag = skip;
+        DION_TRY(launch_gemm_chain(s, w, true));
+        rhs = Wt; rhs_ld = NBO;
+      }
+      // V = rhs Linv_JJ^T
+      DION_TRY(absmax_split(rhs, rhs_ld, rows, sz, s.L.SolveP, 1, 1.f, nullptr));
+      const i64 li_off = s.L.LfP + NBO * r;
+      DION_TRY(absmax_split(s.ws + s.L.Linv + J0 * r + J0, r, sz, sz, li_off, 2, 1.f, sc + (AMAX_PARTS + 64) + AMAX_PARTS));
+      __half* rh = reinterpret_cast<__half*>(s.ws + s.L.SolveP);
+      __half* ih = reinterpret_cast<__half*>(s.ws + li_off);
+      GemmArgs v = gemm_args();
+      v.M = rows; v.N = sz; v.K = sz;
+      v.ab16 = 1; v.f16 = 1;
+      v.A = (const float*)rh; v.A16lo = rh + rows * sz; v.a_si = sz; v.a_sk = 1;
+      v.B = (const float*)ih; v.B16lo = ih + sz * sz; v.b_sk = 1; v.b_sn = sz; v.klimit = 1;
+      v.C = s.ws + pout_off + J0; v.ldc = r; v.epi = EPI_STORE; v.skip_flag = skip;
+      v.alpha_dev = sc + 2 * (AMAX_PARTS + 64) + AMAX_PARTS; v.alpha_dev_stride = s.wstride;
+      DION_TRY(launch_gemm_chain(s, v));
+      if (J0 + sz < r) {      // the new block column of Pout joins the pair (later block columns read it)
+        ChainPtrs t;
+        for (int b = 0; b < s.nb; ++b) t.p[b] = s.W(b, pout_off + J0);
+        launch_pdl(k_split_f16_fixed, dim3((unsigned)grid_for(c, rows * sz / 8), (unsigned)s.nb), dim3(256), 0, s.st, t, r, rows, sz,
+                   ldexpf(1.f, 6), pop + J0, pop + rows * r + J0, s.wstride, r, skip, (i64)OS_SLOT_INTS);
+        DION_CHECK_LAUNCH(c);
+      }
+      return DION_OK;
+    };
     auto solve_block = [&](i64 J0, i64 sz) -> int {
+      if (spairs && sz >= 64 && sz % 8 == 0) return solve_block_pairs(J0, sz);
       const float* rhs = s.ws + pin_off + J0;
       i64 rhs_ld = r;
       if (J0 > 0) {
@@ -1437,13 +1521,13 @@ int step_batch(dion_ctx* c, const dion_matrix* const* list, int nb, float lr, cu
       DION_CHECK_LAUNCH(c);
       launch_pdl(k_split_f16_scaled, dim3((unsigned)grid_for(c, m * n / 8), (unsigned)nb), dim3(256), 0, st,
                  (const float*)(s.ws + s.L.B32), n, m, n, (const float*)(s.ws + s.L.pmax), (int)parts, bh, bh + m * n,
-                 s.ws + s.L.pmax + AMAX_PARTS, s.wstride, (const int*)nullptr, (i64)0, ldexpf(1.f, -13));
+                 s.ws + s.L.pmax + AMAX_PARTS, s.wstride, (const int*)nullptr, (i64)0, ldexpf(1.f, -13), (const float*)nullptr);
       DION_CHECK_LAUNCH(c);
       ChainPtrs t;
       for (int b = 0; b < nb; ++b) t.p[b] = srcs[b];
       __half* qh = reinterpret_cast<__half*>(s.ws + s.L.S16);
       launch_pdl(k_split_f16_fixed, dim3((unsigned)grid_for(c, qrow * r / 8), (unsigned)nb), dim3(256), 0, st, t, list[0]->ldq, qrow, r,
-                 ldexpf(1.f, 13), qh, qh + qrow * r, s.wstride);
+                 ldexpf(1.f, 13), qh, qh + qrow * r, s.wstride, (i64)0, (const int*)nullptr, (i64)0);
       DION_CHECK_LAUNCH(c);
       p_half_ready = true;
     }

@@ -1732,7 +1732,7 @@ inline int umma_try_launch(const GemmArgs& g_in, int precision, int sm_count, fl
   p.withhold_arrive = withhold ? 1 : 0;
   // 32 K blocks per accumulation chain: 1024 k (8e-6 relative error in fp32 mode, 1.4e-6 with
   // split accumulators); 2048 k for bf16 operands loaded through registers
-  p.kc = (x2 && g.precise) ? 16 : 32;      // (K blocks of 64 there: the same 1024 k per chain as the fp32 products)
+  p.kc = (x2 && (g.precise || g.f16)) ? 16 : 32;   // (K blocks of 64 there: the same 1024 k per chain as the fp32 products)
   const int grid = cg2 ? 2 * (p.num_items < nclusters ? p.num_items : nclusters)
                        : (p.num_items < sm_count ? p.num_items : sm_count);
   const bool one = g.tf32x1 && !bf16 && tma && !a_mn && !b_mn && g.a2_mode == ADD_NONE && !g.precise && splits == 1;
