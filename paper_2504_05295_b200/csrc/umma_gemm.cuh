@@ -638,11 +638,12 @@ k_gemm_umma(const __grid_constant__ Params p) {
 
   if (threadIdx.x == 0) {
     // CTA pair: the leader's "full" and "accumulator free" barriers take the arrivals of both CTAs
-    // (nothing to convert: "full" only carries the peer's word that its tiles of the stage have landed)
+    // (nothing to convert: "full" is unused then)
     for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), NOCONV ? 1 : NUM_PROD_WARPS * (CG2 ? 2 : 1)); mbar_init(empty_bar(s), 1); }
     for (int b = 0; b < 2; ++b) { mbar_init(accf_bar(b), 1); mbar_init(acce_bar(b), C::EPI_WARPS * (CG2 ? 2 : 1)); }   // one arrival per epilogue warp
     mbar_init(drain_bar, 1);
-    if (TMA) for (int s = 0; s < STAGES; ++s) mbar_init(raw_bar(s), 1);
+    // (pair without converters: the leader's "landed" barrier also takes the peer's word that ITS tiles have landed)
+    if (TMA) for (int s = 0; s < STAGES; ++s) mbar_init(raw_bar(s), (CG2 && NOCONV && cta_rank == 0) ? 2 : 1);
     *dead = 0;
     fence_barrier_init();
   }
@@ -1170,7 +1171,10 @@ k_gemm_umma(const __grid_constant__ Params p) {
     // ------------------------------------------------------------ MMA issuer (CTA pair: the leader only)
     if (lane == 0 && CG2 && NOCONV && cta_rank != 0) {
       // The peer of a pair without converter warps: TMA fills this CTA's tiles and completes on this CTA's
-      // barrier; this thread passes the word on to the leader, whose MMAs read both CTAs' shared memory.
+      // barrier; this thread passes the word on to the leader's barrier of the same stage (which expects two
+      // arrivals: this one and its own TMA thread's), whose MMAs read both CTAs' shared memory.  The peer's next
+      // arrival for a stage cannot come before the leader has consumed the stage: its refill waits for the
+      // leader's commit.
       int stage = 0;
       uint32_t phase = 0;
       bool alive = true;
@@ -1179,7 +1183,7 @@ k_gemm_umma(const __grid_constant__ Params p) {
         if (skipped(it)) continue;
         for (int kb = it.kb0; kb < it.kb1; ++kb) {
           if (!mbar_wait(raw_bar(stage), phase, dead, p.status, p.spin_limit)) { alive = false; break; }
-          mbar_arrive_remote(full_bar(stage), 0u);
+          mbar_arrive_remote(raw_bar(stage), 0u);
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
       }
@@ -1205,9 +1209,8 @@ k_gemm_umma(const __grid_constant__ Params p) {
         const uint32_t d_small = d_tmem + (SPLIT ? BN : 0);
         uint32_t accumulate = 0;
         for (int kb = kbc; kb < kbc1; ++kb) {
-          if (NOCONV) {   // this CTA's tiles (TMA), then the peer's (its relay thread)
-            if (!mbar_wait(raw_bar(stage), phase, dead, p.status, p.spin_limit)) { alive = false; break; }
-            if (CG2 && !mbar_wait<true>(full_bar(stage), phase, dead, p.status, p.spin_limit)) { alive = false; break; }
+          if (NOCONV) {   // this CTA's tiles (TMA) and, in a pair, the peer's (its relay thread arrives on the same barrier)
+            if (!mbar_wait<CG2>(raw_bar(stage), phase, dead, p.status, p.spin_limit)) { alive = false; break; }
           } else {
             if (!mbar_wait<CG2>(full_bar(stage), phase, dead, p.status, p.spin_limit)) { alive = false; break; }
           }
