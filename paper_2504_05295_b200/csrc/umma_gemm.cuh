@@ -103,6 +103,19 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map
       "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(z), "r"(bar)
       : "memory");
 }
+// The same for a CTA pair: the tile goes to THIS CTA's shared memory, the completion (complete_tx) to the mbarrier
+// at cluster address `bar_cluster`, which may belong to either CTA of the pair (here: the leader's).  No multicast.
+__device__ __forceinline__ void tma_load_3d_pair(uint32_t dst, const CUtensorMap* map, int x, int y, int z, uint32_t bar_cluster) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];" ::"r"(dst),
+      "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(z), "r"(bar_cluster)
+      : "memory");
+}
+__device__ __forceinline__ uint32_t cluster_addr(uint32_t addr, uint32_t rank) {   // `addr` as seen in CTA `rank`
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+  return r;
+}
 __device__ __forceinline__ float4 lds128(uint32_t addr) {
   float4 v;
   asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr) : "memory");
@@ -602,6 +615,7 @@ k_gemm_umma(const __grid_constant__ Params p) {
   static_assert(!ONE || (TMA && CE && !BF16 && !SPLIT && !A_MN && !B_MN), "single pass: k-contiguous fp32 operands by TMA");
   using C = Cfg<BN, BF16, SPLIT, TMA, D16, CE, ONE, CG2, X2>;
   constexpr bool NOCONV = D16 || ONE;    // the operand tiles are what TMA writes: nothing to convert
+  constexpr bool PAIRLOAD = CG2 && NOCONV;   // both CTAs' loads complete on the leader's barrier
   constexpr int BN_L = C::BN_L;
   const uint32_t cta_rank = CG2 ? cluster_ctarank() : 0u;   // 0: the leader of the pair
   const int worker = CG2 ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;       // which tile stream this CTA (pair) walks
@@ -643,7 +657,7 @@ k_gemm_umma(const __grid_constant__ Params p) {
     for (int b = 0; b < 2; ++b) { mbar_init(accf_bar(b), 1); mbar_init(acce_bar(b), C::EPI_WARPS * (CG2 ? 2 : 1)); }   // one arrival per epilogue warp
     mbar_init(drain_bar, 1);
     // (pair without converters: the leader's "landed" barrier also takes the peer's word that ITS tiles have landed)
-    if (TMA) for (int s = 0; s < STAGES; ++s) mbar_init(raw_bar(s), (CG2 && NOCONV && cta_rank == 0) ? 2 : 1);
+    if (TMA) for (int s = 0; s < STAGES; ++s) mbar_init(raw_bar(s), 1);
     *dead = 0;
     fence_barrier_init();
   }
@@ -1093,50 +1107,63 @@ k_gemm_umma(const __grid_constant__ Params p) {
           const uint32_t sa_lo = sa + C::A_BYTES;
           const uint32_t sb = sa + ((NOCONV && !X2) ? 1 : 2) * C::A_BYTES;
           const uint32_t bar = raw_bar(stage);
+          // A pair without converter warps: both CTAs' tiles complete on the LEADER's barrier of the stage, which
+          // its TMA thread arms for the bytes of both, and which its MMA thread waits on.  (A completion may reach
+          // the barrier before it is armed: the phase still cannot end before the arming arrival.)  The peer's
+          // loads for the stage's next use wait for the leader's commit, hence for the end of this phase.
+          const uint32_t bar_pair = PAIRLOAD ? cluster_addr(bar, 0u) : bar;
+          auto ld3 = [&](uint32_t dst, const CUtensorMap* map, int x, int y, int z) {
+            if constexpr (PAIRLOAD) tma_load_3d_pair(dst, map, x, y, z, bar_pair);
+            else tma_load_3d(dst, map, x, y, z, bar);
+          };
+          auto expect = [&](uint32_t nbytes) {
+            if constexpr (PAIRLOAD) { if (cta_rank == 0) mbar_expect_tx(bar, 2u * nbytes); }
+            else mbar_expect_tx(bar, nbytes);
+          };
           if (X2) {   // hi and lo tiles of both operands: [rows][64 k] boxes, or [64 k][64 rows] boxes per 64-row chunk
-            mbar_expect_tx(bar, (uint32_t)(2 * (C::A_BYTES + C::B_BYTES)));
+            expect((uint32_t)(2 * (C::A_BYTES + C::B_BYTES)));
             const uint32_t sb_lo2 = sb + C::B_BYTES;
             if (!A_MN) {
-              tma_load_3d(sa, &p.tmA, k0, row0a, it.b, bar);
-              tma_load_3d(sa_lo, &p.tmA2, k0, row0a, it.b, bar);
+              ld3(sa, &p.tmA, k0, row0a, it.b);
+              ld3(sa_lo, &p.tmA2, k0, row0a, it.b);
             } else {
 #pragma unroll
               for (int c = 0; c < BM / 64; ++c) {
-                tma_load_3d(sa + c * (BKE * 128), &p.tmA, row0a + 64 * c, k0, it.b, bar);
-                tma_load_3d(sa_lo + c * (BKE * 128), &p.tmA2, row0a + 64 * c, k0, it.b, bar);
+                ld3(sa + c * (BKE * 128), &p.tmA, row0a + 64 * c, k0, it.b);
+                ld3(sa_lo + c * (BKE * 128), &p.tmA2, row0a + 64 * c, k0, it.b);
               }
             }
             if (!B_MN) {
-              tma_load_3d(sb, &p.tmB, k0, row0b, it.b, bar);
-              tma_load_3d(sb_lo2, &p.tmB2, k0, row0b, it.b, bar);
+              ld3(sb, &p.tmB, k0, row0b, it.b);
+              ld3(sb_lo2, &p.tmB2, k0, row0b, it.b);
             } else {
 #pragma unroll
               for (int c = 0; c < BN_L / 64; ++c) {
-                tma_load_3d(sb + c * (BKE * 128), &p.tmB, row0b + 64 * c, k0, it.b, bar);
-                tma_load_3d(sb_lo2 + c * (BKE * 128), &p.tmB2, row0b + 64 * c, k0, it.b, bar);
+                ld3(sb + c * (BKE * 128), &p.tmB, row0b + 64 * c, k0, it.b);
+                ld3(sb_lo2 + c * (BKE * 128), &p.tmB2, row0b + 64 * c, k0, it.b);
               }
             }
             if (++stage == STAGES) { stage = 0; phase ^= 1u; }
             continue;
           }
           if (ONE) {   // raw fp32 tiles, [rows][32 k] boxes
-            mbar_expect_tx(bar, (uint32_t)(C::A_BYTES + C::B_BYTES));
-            tma_load_3d(sa, &p.tmA, k0, row0a, it.b, bar);
-            tma_load_3d(sb, &p.tmB, k0, row0b, it.b, bar);
+            expect((uint32_t)(C::A_BYTES + C::B_BYTES));
+            ld3(sa, &p.tmA, k0, row0a, it.b);
+            ld3(sb, &p.tmB, k0, row0b, it.b);
             if (++stage == STAGES) { stage = 0; phase ^= 1u; }
             continue;
           }
           if (D16) {   // bf16 tiles: [rows][64 k] boxes, or [64 k][64 rows] boxes per 64-row chunk
-            mbar_expect_tx(bar, (uint32_t)(C::A_BYTES + C::B_BYTES));
-            if (!A_MN) tma_load_3d(sa, &p.tmA, k0, row0a, it.b, bar);
+            expect((uint32_t)(C::A_BYTES + C::B_BYTES));
+            if (!A_MN) ld3(sa, &p.tmA, k0, row0a, it.b);
             else {
 #pragma unroll
-              for (int c = 0; c < BM / 64; ++c) tma_load_3d(sa + c * (BKE * 128), &p.tmA, row0a + 64 * c, k0, it.b, bar);
+              for (int c = 0; c < BM / 64; ++c) ld3(sa + c * (BKE * 128), &p.tmA, row0a + 64 * c, k0, it.b);
             }
-            if (!B_MN) tma_load_3d(sb, &p.tmB, k0, row0b, it.b, bar);
+            if (!B_MN) ld3(sb, &p.tmB, k0, row0b, it.b);
             else {
 #pragma unroll
-              for (int c = 0; c < BN / 64; ++c) tma_load_3d(sb + c * (BKE * 128), &p.tmB, row0b + 64 * c, k0, it.b, bar);
+              for (int c = 0; c < BN / 64; ++c) ld3(sb + c * (BKE * 128), &p.tmB, row0b + 64 * c, k0, it.b);
             }
             if (++stage == STAGES) { stage = 0; phase ^= 1u; }
             continue;
@@ -1169,25 +1196,7 @@ k_gemm_umma(const __grid_constant__ Params p) {
     __syncwarp();
   } else {
     // ------------------------------------------------------------ MMA issuer (CTA pair: the leader only)
-    if (lane == 0 && CG2 && NOCONV && cta_rank != 0) {
-      // The peer of a pair without converter warps: TMA fills this CTA's tiles and completes on this CTA's
-      // barrier; this thread passes the word on to the leader's barrier of the same stage (which expects two
-      // arrivals: this one and its own TMA thread's), whose MMAs read both CTAs' shared memory.  The peer's next
-      // arrival for a stage cannot come before the leader has consumed the stage: its refill waits for the
-      // leader's commit.
-      int stage = 0;
-      uint32_t phase = 0;
-      bool alive = true;
-      for (int item = worker; item < p.num_items && alive; item += workers) {
-        const Item it = decode_item<BN, BKE, CG2>(p, item);
-        if (skipped(it)) continue;
-        for (int kb = it.kb0; kb < it.kb1; ++kb) {
-          if (!mbar_wait(raw_bar(stage), phase, dead, p.status, p.spin_limit)) { alive = false; break; }
-          mbar_arrive_remote(raw_bar(stage), 0u);
-          if (++stage == STAGES) { stage = 0; phase ^= 1u; }
-        }
-      }
-    } else if (lane == 0 && (!CG2 || cta_rank == 0)) {
+    if (lane == 0 && (!CG2 || cta_rank == 0)) {
       const uint32_t idesc = make_idesc(BF16, A_MN, B_MN, BN, CG2 ? 2 * BM : BM, BF16 && p.g.f16 != 0);
       const uint32_t lbo = BKE * 128;
       constexpr uint32_t A_KSTEP = A_MN ? (BF16 ? 2048u : 1024u) : 32u;   // bytes per UMMA K step
@@ -1209,7 +1218,7 @@ k_gemm_umma(const __grid_constant__ Params p) {
         const uint32_t d_small = d_tmem + (SPLIT ? BN : 0);
         uint32_t accumulate = 0;
         for (int kb = kbc; kb < kbc1; ++kb) {
-          if (NOCONV) {   // this CTA's tiles (TMA) and, in a pair, the peer's (its relay thread arrives on the same barrier)
+          if (NOCONV) {   // this CTA's tiles (TMA) and, in a pair, the peer's (they complete on this barrier too)
             if (!mbar_wait<CG2>(raw_bar(stage), phase, dead, p.status, p.spin_limit)) { alive = false; break; }
           } else {
             if (!mbar_wait<CG2>(full_bar(stage), phase, dead, p.status, p.spin_limit)) { alive = false; break; }
