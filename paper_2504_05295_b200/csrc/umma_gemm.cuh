@@ -607,8 +607,8 @@ template <int BN, bool A_MN, bool B_MN, bool BF16, bool SPLIT, bool TMA, bool D1
 __global__ void __launch_bounds__((Cfg<BN, BF16, SPLIT, TMA, D16, CE, ONE, CG2, X2>::THREADS), 1)
 k_gemm_umma(const __grid_constant__ Params p) {
   static_assert(!X2 || (D16 && CE), "operand pairs are bf16 arrays");
-  static_assert(!CG2 || (TMA && BN == 256 && ((!BF16 && !D16 && !ONE) || X2)),
-                "CTA pairs: the fp32 TMA variants and the operand-pair variant, 256-column tiles");
+  static_assert(!CG2 || (TMA && BN == 256 && ((!BF16 && !D16 && !ONE) || (D16 && CE))),
+                "CTA pairs: the fp32 TMA variants and the 16-bit array variants (single arrays or pairs), 256-column tiles");
   static_assert(!(BF16 && SPLIT) || X2, "split accumulators belong to the 3xTF32 mode and to operand pairs");
   static_assert(!D16 || (BF16 && TMA), "bf16 operands in memory are loaded by TMA");
   static_assert(!CE || (TMA && (D16 || !BF16)), "the coalesced epilogue serves the bf16-array and the fp32 TMA variants");
@@ -1163,7 +1163,7 @@ k_gemm_umma(const __grid_constant__ Params p) {
             if (!B_MN) ld3(sb, &p.tmB, k0, row0b, it.b);
             else {
 #pragma unroll
-              for (int c = 0; c < BN / 64; ++c) ld3(sb + c * (BKE * 128), &p.tmB, row0b + 64 * c, k0, it.b);
+              for (int c = 0; c < BN_L / 64; ++c) ld3(sb + c * (BKE * 128), &p.tmB, row0b + 64 * c, k0, it.b);
             }
             if (++stage == STAGES) { stage = 0; phase ^= 1u; }
             continue;
@@ -1249,7 +1249,8 @@ k_gemm_umma(const __grid_constant__ Params p) {
               }
               accumulate = 1;
             } else if (BF16) {
-              umma<true>(d_tmem, a_hi, b_hi, idesc, accumulate);
+              if (CG2) umma2_f16(d_tmem, a_hi, b_hi, idesc, accumulate);
+              else umma<true>(d_tmem, a_hi, b_hi, idesc, accumulate);
               accumulate = 1;
             } else if (ONE) {
               umma<false>(d_tmem, a_hi, b_hi, idesc, accumulate);
@@ -1377,6 +1378,29 @@ inline cudaError_t launch_x2_pair(const Params& p, bool a_mn, bool b_mn, int gri
 template <bool A_MN, bool B_MN>
 inline cudaError_t set_x2_pair_attr() {
   return set_smem_attr<256, A_MN, B_MN, true, false, true, true, true, false, true, true>();
+}
+
+// 16-bit arrays (one array per operand) on CTA pairs
+template <bool A_MN, bool B_MN>
+inline cudaError_t launch_d16_pair_one(const Params& p, int grid, cudaStream_t st) {
+  using CF = Cfg<256, true, false, true, true, true, false, true, false>;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)grid); cfg.blockDim = dim3(CF::THREADS); cfg.dynamicSmemBytes = CF::SMEM_BYTES; cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr; cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, k_gemm_umma<256, A_MN, B_MN, true, false, true, true, true, false, true, false>, p);
+}
+inline cudaError_t launch_d16_pair(const Params& p, bool a_mn, bool b_mn, int grid, cudaStream_t st) {
+  if (!a_mn && !b_mn) return launch_d16_pair_one<false, false>(p, grid, st);
+  if (!a_mn && b_mn) return launch_d16_pair_one<false, true>(p, grid, st);
+  if (a_mn && b_mn) return launch_d16_pair_one<true, true>(p, grid, st);
+  return launch_d16_pair_one<true, false>(p, grid, st);
+}
+template <bool A_MN, bool B_MN>
+inline cudaError_t set_d16_pair_attr() {
+  return set_smem_attr<256, A_MN, B_MN, true, false, true, true, true, false, true, false>();
 }
 
 // CTA pairs: clusters of two CTAs, 256 x 256 tiles (fp32 mode, TMA, coalesced epilogue)
@@ -1582,6 +1606,10 @@ inline int umma_configure() {
   if (e == cudaSuccess) e = set_x2_pair_attr<false, true>();
   if (e == cudaSuccess) e = set_x2_pair_attr<true, true>();
   if (e == cudaSuccess) e = set_x2_pair_attr<true, false>();
+  if (e == cudaSuccess) e = set_d16_pair_attr<false, false>();
+  if (e == cudaSuccess) e = set_d16_pair_attr<false, true>();
+  if (e == cudaSuccess) e = set_d16_pair_attr<true, true>();
+  if (e == cudaSuccess) e = set_d16_pair_attr<true, false>();
   if (e == cudaSuccess) e = set_pair_attr<false, false>();
   if (e == cudaSuccess) e = set_pair_attr<false, true>();
   if (e == cudaSuccess) e = set_pair_attr<true, true>();
@@ -1654,9 +1682,9 @@ inline int umma_try_launch(const GemmArgs& g_in, int precision, int sm_count, fl
   const int nclusters = pair_clusters(sm_count);
   // ... and the products on bf16 operand pairs (two thirds of the operand traffic per CTA, three stages instead of two)
   const bool x2 = d16 && g.A16lo != nullptr && g.B16lo != nullptr;   // bf16 operand pairs
-  // (not the single-pass product: its pair form ran the X update of the 8B list in 51 ms instead of 32, tensor
-  // pipe 30 % instead of 54 % under ncu, with or without per-warp and relaxed arrivals; cause not found)
-  bool cg2 = ((!bf16 && !g.tf32x1 && g.a2_mode != ADD_BF16) || x2) &&
+  // ... and those on single 16-bit arrays (the operand tiles a CTA reads from L2 are what bounds them on single CTAs).
+  // (Not the single-pass TF32 product, which only ragged shapes still take.)
+  bool cg2 = ((!bf16 && !g.tf32x1 && g.a2_mode != ADD_BF16) || d16) &&
              !(variant & (UMMA_VARIANT_REGISTER_LOADS | UMMA_VARIANT_NO_PAIRS)) && nclusters > 0 &&
              g.N >= 256 && g.M >= PAIR_MIN_ROWS && (g.tri != TRI_LOWER || g.N >= PAIR_MIN_TRI);
   const int BN = ((g.tri == TRI_LOWER && !tri_wide && !cg2) || g.N < 256) ? 128 : 256;
@@ -1760,6 +1788,8 @@ inline int umma_try_launch(const GemmArgs& g_in, int precision, int sm_count, fl
     }
   } else if (cg2 && x2) {
     if (launch_x2_pair(p, a_mn, b_mn, grid, st) != cudaSuccess) { cudaGetLastError(); return DION_ERR_CUDA; }
+  } else if (cg2 && d16) {
+    if (launch_d16_pair(p, a_mn, b_mn, grid, st) != cudaSuccess) { cudaGetLastError(); return DION_ERR_CUDA; }
   } else if (cg2) {
     const cudaError_t e = g.precise ? launch_pair<true>(p, a_mn, b_mn, grid, st) : launch_pair<false>(p, a_mn, b_mn, grid, st);
     if (e != cudaSuccess) { cudaGetLastError(); return DION_ERR_CUDA; }

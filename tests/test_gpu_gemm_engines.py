@@ -41,7 +41,7 @@ def lib():
 
 
 def run(lib, engine, precision, M, N, K, a_mn, b_mn, add=None, epi=0, tri=0, klimit=0, alpha=1.0, seed=0,
-        precise=0, ab16=False, variant=0, tf32x1=False, expect_status=0):
+        precise=0, ab16=False, variant=0, tf32x1=False, expect_status=0, out=None):
     g = torch.Generator(device="cuda"); g.manual_seed(seed)
     rn = lambda *s: torch.randn(*s, generator=g, device="cuda")
     # A(i,k): stored M x K (k contiguous) or K x M (row index contiguous)
@@ -100,6 +100,8 @@ def run(lib, engine, precision, M, N, K, a_mn, b_mn, add=None, epi=0, tri=0, kli
     assert int(status.item()) == expect_status, f"device status {int(status.item())}"
     if expect_status:
         return None
+    if out is not None:
+        out.append(C)
     got = C.double()
     if tri:
         # only the elements on or below the diagonal are guaranteed to be written
@@ -195,6 +197,20 @@ def test_bf16_arrays_as_operands(lib, a_mn, b_mn):
     for (M, N, K) in [(512, 512, 1024), (648, 392, 328), (256, 1024, 4160), (128, 64, 64)]:
         err = run(lib, 2, 1, M, N, K, a_mn, b_mn, ab16=True, seed=M + K)
         assert err < 1e-5, (M, N, K, err)
+
+
+@pytest.mark.parametrize("a_mn,b_mn", LAYOUTS)
+def test_bf16_arrays_on_cta_pairs(lib, a_mn, b_mn):
+    # from 512 rows and 256 columns the products on single 16-bit arrays run on clusters of two CTAs too (both CTAs'
+    # tiles complete on the leader's barrier); bit 2 of the variant word keeps them on single CTAs: same bits
+    for (M, N, K, epi) in [(1024, 512, 512, 0), (2048, 768, 2112, 1), (648, 392, 328, 2), (1280, 256, 64, 1),
+                           (4096, 1024, 1024, 1)]:
+        got = []
+        err = run(lib, 2, 1, M, N, K, a_mn, b_mn, ab16=True, epi=epi, alpha=0.05, seed=M + K, out=got)
+        assert err < 1e-5, (M, N, K, epi, err)
+        err1 = run(lib, 2, 1, M, N, K, a_mn, b_mn, ab16=True, epi=epi, alpha=0.05, seed=M + K, variant=4, out=got)
+        assert err1 < 1e-5, (M, N, K, epi, err1)
+        assert torch.equal(got[0], got[1]), (M, N, K, epi)
 
 
 def test_bf16_arrays_epilogues_and_lower_triangle(lib):
