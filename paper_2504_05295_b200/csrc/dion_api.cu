@@ -469,7 +469,8 @@ int launch_gemm_group(StepCtx& s, const std::vector<GemmArgs>& v) {
 int configure_kernels() {
   if (umma_configure() != DION_OK) return DION_ERR_CUDA;
   if (cudaFuncSetAttribute(k_probe_y4, cudaFuncAttributeMaxDynamicSharedMemorySize, PY_SMEM) != cudaSuccess ||
-      cudaFuncSetAttribute(k_chol_step, cudaFuncAttributeMaxDynamicSharedMemorySize, CHOL_STEP_SMEM) != cudaSuccess) {
+      cudaFuncSetAttribute(k_chol_step, cudaFuncAttributeMaxDynamicSharedMemorySize, CHOL_STEP_SMEM) != cudaSuccess ||
+      cudaFuncSetAttribute(k_tiny_cholqr2, cudaFuncAttributeMaxDynamicSharedMemorySize, tiny_cholqr2_smem(TINY_MAX_ROWS)) != cudaSuccess) {
     cudaGetLastError();
     return DION_ERR_CUDA;
   }
@@ -1043,6 +1044,16 @@ int orthonormalize(StepCtx& s, i64 rows, i64 r, i64 short_dim, i64 pin_off, i64*
     // either round (the paper's "CQR failure") raises the step's fail flag only; the fallback kernel then
     // orthonormalizes the saved panel and clears the flag, or confirms the breakdown.
     const bool fb = pin_off != s.L.P0 && fallback_fits(s.c, rows);
+    if (r <= NB && rows <= TINY_MAX_ROWS && s.redo_p == nullptr) {
+      // a panel that fits one CTA's shared memory: both rounds and the test between them in one launch
+      launch_pdl(k_tiny_cholqr2, dim3((unsigned)s.nb), dim3(TINY_THREADS), (size_t)tiny_cholqr2_smem(rows), s.st, (const float*)(s.ws + pin_off),
+                 s.ws + s.L.P0, (int)rows, (int)r, s.os, ORTH_TAU_F, s.c->dev_ints + 2, fb ? (int*)nullptr : s.c->dev_ints, s.c->dev_ints,
+                 s.wstride);
+      DION_CHECK_LAUNCH(s.c);
+      if (fb) DION_TRY(cgs_fallback(s, pin_off, s.L.P0, rows, r));
+      *U_off = s.L.P0;
+      return DION_OK;
+    }
     s.quiet_fail = fb;
     // Round one writes P0, where U is expected; the second round, when it runs, goes P0 -> P1 and is copied
     // back: the common case (one round) moves the panel once.
@@ -2445,7 +2456,7 @@ bool preload_kernels() {
   bool ok = true;
   ok = ok && touch_kernel(k_gemm_simt<128, 128, 8, 8, 8>) && touch_kernel(k_gemm_simt<64, 64, 16, 4, 4>);
   ok = ok && touch_kernel(k_splitk_reduce) && touch_kernel(k_round_begin) && touch_kernel(k_potrf_diag);
-  ok = ok && touch_kernel(k_chol_step) && touch_kernel(k_inv_finish) && touch_kernel(k_round_end);
+  ok = ok && touch_kernel(k_chol_step) && touch_kernel(k_inv_finish) && touch_kernel(k_round_end) && touch_kernel(k_tiny_cholqr2);
   ok = ok && touch_kernel(k_probe_y) && touch_kernel(k_probe_y4) && touch_kernel(k_probe_w) && touch_kernel(k_probe_decide) && touch_kernel(k_reset_rounds);
   ok = ok && touch_kernel(k_orth_finish) && touch_kernel(k_cgs_fallback) && touch_kernel(k_copy_block);
   ok = ok && touch_kernel(k_colsumsq_partial) && touch_kernel(k_colnorm_apply) && touch_kernel(k_copy_panel);

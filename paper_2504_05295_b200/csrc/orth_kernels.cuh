@@ -62,7 +62,14 @@ typedef float (*half_blk_t)[NB / 2 + 1];
 
 // One doubling level of the triangular inverse inside a 64 x 64 block: for every pair of
 // adjacent B x B diagonal blocks, X21 = -X22 (L21 X11).  256 threads, two block-wide barriers.
-template <int B>
+// SUB: the 256 calling threads are the first eight warps of a larger CTA; they meet at a named barrier of their own.
+template <bool SUB>
+__device__ __forceinline__ void block_sync() {
+  if constexpr (SUB) asm volatile("bar.sync 1, 256;" ::: "memory");
+  else __syncthreads();
+}
+
+template <int B, bool SUB = false>
 __device__ __forceinline__ void trtri_level(blk_t L, blk_t X, half_blk_t T, int tid) {
   constexpr int NPAIRS = NB / (2 * B);
   for (int e = tid; e < NPAIRS * B * B; e += 256) {
@@ -76,7 +83,7 @@ __device__ __forceinline__ void trtri_level(blk_t L, blk_t X, half_blk_t T, int 
     }
     T[pr * B + rr][cc] = (s0 + s1) + (s2 + s3);
   }
-  __syncthreads();
+  block_sync<SUB>();
   for (int e = tid; e < NPAIRS * B * B; e += 256) {
     const int pr = e / (B * B), rr = (e / B) % B, cc = e % B, base = pr * 2 * B;
     float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;   // X22 is lower triangular: k <= rr; zeros above are stored
@@ -88,12 +95,13 @@ __device__ __forceinline__ void trtri_level(blk_t L, blk_t X, half_blk_t T, int 
     }
     X[base + B + rr][base + cc] = -((s0 + s1) + (s2 + s3));
   }
-  __syncthreads();
+  block_sync<SUB>();
 }
 
 // Inverse X of the lower-triangular 64 x 64 block L (shared memory; rdiag[i] = 1 / L[i][i];
 // X zero on entry): 16 x 16 diagonal inverses by forward substitution, then doubling.
 // Called by all 256 threads after a block-wide barrier; ends with one.
+template <bool SUB = false>
 __device__ __forceinline__ void invert_block(blk_t L, blk_t X, half_blk_t T, const float* rdiag, int tid) {
   constexpr int W = 16;
   if (tid < NB) {
@@ -110,10 +118,10 @@ __device__ __forceinline__ void invert_block(blk_t L, blk_t X, half_blk_t T, con
 #pragma unroll
     for (int i = 0; i < W; ++i) X[b0 + i][b0 + q] = x[i];
   }
-  __syncthreads();
+  block_sync<SUB>();
   // ... then [[X11, 0], [-X22 L21 X11, X22]] for block sizes 16 and 32
-  trtri_level<16>(L, X, T, tid);
-  trtri_level<32>(L, X, T, tid);
+  trtri_level<16, SUB>(L, X, T, tid);
+  trtri_level<32, SUB>(L, X, T, tid);
 }
 
 // Cholesky factor and its inverse of the 64 x 64 block held in L (shared memory; lower
@@ -125,6 +133,7 @@ __device__ __forceinline__ void invert_block(blk_t L, blk_t X, half_blk_t T, con
 // one warp (rows in registers, shuffles, no barrier), the rows below it by one thread per
 // row, the trailing update by all threads -- three block-wide barriers per sub-panel
 // instead of three per column.  The inverse is built from 16 x 16 inverses by doubling.
+template <bool SUB = false>
 __device__ __forceinline__ void potrf_block(blk_t L, blk_t X, half_blk_t T, const float* gd, float* rdiag,
                                             int* deflated, int jb, float floor_rel, int* __restrict__ os,
                                             int* __restrict__ status) {
@@ -195,7 +204,7 @@ __device__ __forceinline__ void potrf_block(blk_t L, blk_t X, half_blk_t T, cons
           L[i][c] -= sacc;
         }
     }
-    __syncthreads();
+    block_sync<SUB>();
     const int below = NB - c0 - WF;   // rows under the diagonal piece
     if (tid < below) {
       const int i = c0 + WF + tid;
@@ -210,7 +219,7 @@ __device__ __forceinline__ void potrf_block(blk_t L, blk_t X, half_blk_t T, cons
 #pragma unroll
       for (int j = 0; j < WF; ++j) L[i][c0 + j] = x[j];
     }
-    __syncthreads();
+    block_sync<SUB>();
     // trailing update, first part: the WF columns that the next diagonal piece and the panel below
     // it need (thread -> (row, column)); the rest is deferred to run beside the next diagonal piece
     for (int e = tid; e < below * WF; e += 256) {
@@ -222,7 +231,7 @@ __device__ __forceinline__ void potrf_block(blk_t L, blk_t X, half_blk_t T, cons
         L[i][c] -= sacc;
       }
     }
-    __syncthreads();
+    block_sync<SUB>();
   }
   if (tid == 0) {
     if (floor_rel > 0.f) {
@@ -234,7 +243,7 @@ __device__ __forceinline__ void potrf_block(blk_t L, blk_t X, half_blk_t T, cons
     }
   }
 
-  invert_block(L, X, T, rdiag, tid);
+  invert_block<SUB>(L, X, T, rdiag, tid);
 }
 
 // Cholesky of one jb x jb (jb <= 64) diagonal block, in place (lower factor, the
@@ -298,6 +307,232 @@ __global__ void __launch_bounds__(256) k_potrf_diag(float* __restrict__ A, i64 l
     if (i < jb && c < jb) A[(i64)i * ld + c] = (c <= i) ? L[i][c] : 0.f;
     Dinv[e] = X[i][c];
     DinvP[e] = deflated[i] ? 0.f : X[i][c];
+  }
+}
+
+// CholeskyQR2 of a small panel (rows x r, r <= 64, rows <= TINY_MAX_ROWS, leading dimension r) in ONE launch, one
+// CTA of 1024 threads per matrix, the panel resident in shared memory: Gram matrix, Cholesky factor and its inverse
+// (potrf_block, on the first eight warps), U1 = P L^-T, then the second round's Gram matrix G2 = U1^T U1, which
+// also says exactly how far U1 is from orthonormal: |G2 - I|_F^2 <= tau_f^2 r -> done after one round (the same
+// test the probe of the large panels estimates), else the second round runs on G2.  Replaces some seventeen
+// launches of a step on such a panel.  Every sum has a fixed order: same bits on every run.
+// State as the launch chain leaves it: OS_MAXDEV (the deviation), OS_DONE = 1, OS_ROUNDS and *rounds_total (1 or
+// 2); a pivot that is not positive raises OS_FAIL (and DION_STATUS_BREAKDOWN unless `status_fail` is nullptr: a
+// fallback follows), the panel is then left to the fallback; a Gram trace that is not finite raises OS_FAIL and
+// DION_STATUS_NONFINITE.  Pin may equal Pout.
+constexpr int TINY_MAX_ROWS = 512;
+constexpr int TINY_THREADS = 1024;
+constexpr int TINY_LD = NB + 1;
+constexpr int TINY_BLK = NB * (NB + 1);     // floats of a 64 x 65 block
+inline int tiny_cholqr2_smem(i64 rows) {    // panel, L, X, three partial Gram matrices, T, gd, rdiag, red, deflated
+  return (int)sizeof(float) * ((int)rows * TINY_LD + 5 * TINY_BLK + (NB / 2) * (NB / 2 + 1) + 2 * NB + TINY_THREADS) + (int)sizeof(int) * NB;
+}
+
+// acc[a][b] = sum over this thread's quarter of the rows (i = q, q + 4, ...) of Ps[i][4 ty + a] * Ps[i][tx + 16 b]
+__device__ __forceinline__ void tiny_gram_part(const float* __restrict__ Ps, int rows, int q, int ty, int tx, float (&acc)[4][4]) {
+#pragma unroll
+  for (int a = 0; a < 4; ++a)
+#pragma unroll
+    for (int b = 0; b < 4; ++b) acc[a][b] = 0.f;
+#pragma unroll 4
+  for (int i = q; i < rows; i += 4) {
+    const float* row = Ps + i * TINY_LD;
+    float av[4], bv[4];
+#pragma unroll
+    for (int a = 0; a < 4; ++a) av[a] = row[4 * ty + a];
+#pragma unroll
+    for (int b = 0; b < 4; ++b) bv[b] = row[tx + 16 * b];
+#pragma unroll
+    for (int a = 0; a < 4; ++a)
+#pragma unroll
+      for (int b = 0; b < 4; ++b) acc[a][b] = fmaf(av[a], bv[b], acc[a][b]);
+  }
+}
+
+__global__ void __launch_bounds__(TINY_THREADS) k_tiny_cholqr2(const float* __restrict__ Pin, float* __restrict__ Pout, int rows, int r,
+                                                               int* __restrict__ os, float tau_f, int* __restrict__ rounds_total,
+                                                               int* __restrict__ status_fail, int* __restrict__ status_always,
+                                                               i64 wstride) {
+  Pin += (i64)blockIdx.x * wstride; Pout += (i64)blockIdx.x * wstride;
+  os += (i64)blockIdx.x * OS_SLOT_INTS;
+  pdl_enter();
+  extern __shared__ __align__(16) float tiny_smem[];
+  float* Ps = tiny_smem;                                              // rows x 65
+  float* blocks = Ps + rows * TINY_LD;
+  blk_t L = reinterpret_cast<blk_t>(blocks);
+  blk_t X = reinterpret_cast<blk_t>(blocks + TINY_BLK);
+  float* Gp = blocks + 2 * TINY_BLK;                                  // partial Gram matrices of row quarters 1 .. 3
+  half_blk_t T = reinterpret_cast<half_blk_t>(blocks + 5 * TINY_BLK);
+  float* gd = blocks + 5 * TINY_BLK + (NB / 2) * (NB / 2 + 1);
+  float* rdiag = gd + NB;
+  float* red = rdiag + NB;                                            // TINY_THREADS
+  int* deflated = reinterpret_cast<int*>(red + TINY_THREADS);
+  const int tid = threadIdx.x;
+  const int q = tid >> 8, t8 = tid & 255, ty = t8 >> 4, tx = t8 & 15;   // q: warp-uniform quarter of the CTA
+
+  if (r % 4 == 0 && (reinterpret_cast<uintptr_t>(Pin) & 15u) == 0) {
+    // four 16-byte loads in flight per thread
+    const int nv = rows * r / 4;
+    const float4* src = reinterpret_cast<const float4*>(Pin);
+    for (int base = 0; base < nv; base += TINY_THREADS * 4) {
+      float4 v[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int idx = base + u * TINY_THREADS + tid;
+        v[u] = (idx < nv) ? __ldg(src + idx) : make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int idx = base + u * TINY_THREADS + tid;
+        if (idx < nv) {
+          float* d = Ps + (4 * idx / r) * TINY_LD + (4 * idx % r);
+          d[0] = v[u].x; d[1] = v[u].y; d[2] = v[u].z; d[3] = v[u].w;
+        }
+      }
+    }
+    if (r < NB)
+      for (int e = tid; e < rows * (NB - r); e += TINY_THREADS) Ps[(e / (NB - r)) * TINY_LD + r + e % (NB - r)] = 0.f;
+  } else {
+#pragma unroll 4
+    for (int e = tid; e < rows * NB; e += TINY_THREADS) {
+      const int i = e / NB, c = e % NB;
+      Ps[i * TINY_LD + c] = (c < r) ? Pin[(i64)i * r + c] : 0.f;      // columns r .. 63: zero
+    }
+  }
+  __syncthreads();
+
+  float acc[4][4];
+  // The Gram matrix of the panel in shared memory into the registers of quarter 0: every quarter sums its rows,
+  // quarters 1 .. 3 pass theirs through shared memory, quarter 0 adds them in order.
+  auto gram = [&]() {
+    tiny_gram_part(Ps, rows, q, ty, tx, acc);
+    if (q > 0) {
+      float* g = Gp + (q - 1) * TINY_BLK;
+#pragma unroll
+      for (int a = 0; a < 4; ++a)
+#pragma unroll
+        for (int b = 0; b < 4; ++b) g[(4 * ty + a) * (NB + 1) + tx + 16 * b] = acc[a][b];
+    }
+    __syncthreads();
+    if (q == 0) {
+#pragma unroll
+      for (int p = 0; p < 3; ++p)
+#pragma unroll
+        for (int a = 0; a < 4; ++a)
+#pragma unroll
+          for (int b = 0; b < 4; ++b) acc[a][b] += Gp[p * TINY_BLK + (4 * ty + a) * (NB + 1) + tx + 16 * b];
+    }
+  };
+  // (quarter 0) the Gram matrix from the registers into L: lower triangle, zero above, identity beyond column r;
+  // X, gd, deflated reset
+  auto stage_factor_input = [&]() {
+    if (q == 0) {
+#pragma unroll
+      for (int a = 0; a < 4; ++a)
+#pragma unroll
+        for (int b = 0; b < 4; ++b) {
+          const int i = 4 * ty + a, c = tx + 16 * b;
+          float v = (i < r && c <= i) ? acc[a][b] : 0.f;
+          if (i == c && i >= r) v = 1.f;
+          L[i][c] = v;
+          X[i][c] = 0.f;
+        }
+      if (tid < NB) { deflated[tid] = 0; gd[tid] = 0.f; }
+    }
+  };
+  // U = P X^T in place, X lower triangular (its zeros above the diagonal are stored).  Four threads per row, one
+  // from each quarter; a thread takes the column groups g = q, q + 4, ... of four columns each, four independent
+  // sums per loaded entry.  All sums of a batch of 256 rows are formed before any entry is overwritten.
+  auto apply_inverse = [&]() {
+    const int ngroups = (r + 3) / 4;
+    for (int i0 = 0; i0 < rows; i0 += 256) {
+      const int i = i0 + t8;
+      float* row = Ps + (i < rows ? i : 0) * TINY_LD;
+      float y[4][4];
+#pragma unroll
+      for (int s4 = 0; s4 < 4; ++s4) {
+        const int g = q + 4 * s4;
+        y[s4][0] = y[s4][1] = y[s4][2] = y[s4][3] = 0.f;
+        if (g < ngroups && i < rows) {
+          const int j0 = 4 * g;
+          float y0 = 0.f, y1 = 0.f, y2 = 0.f, y3 = 0.f;
+#pragma unroll 4
+          for (int k = 0; k < j0 + 4; ++k) {
+            const float x = row[k];
+            y0 = fmaf(x, X[j0][k], y0);
+            y1 = fmaf(x, X[j0 + 1][k], y1);
+            y2 = fmaf(x, X[j0 + 2][k], y2);
+            y3 = fmaf(x, X[j0 + 3][k], y3);
+          }
+          y[s4][0] = y0; y[s4][1] = y1; y[s4][2] = y2; y[s4][3] = y3;
+        }
+      }
+      __syncthreads();
+#pragma unroll
+      for (int s4 = 0; s4 < 4; ++s4) {
+        const int g = q + 4 * s4;
+        if (g < ngroups && i < rows) {
+          row[4 * g] = y[s4][0]; row[4 * g + 1] = y[s4][1]; row[4 * g + 2] = y[s4][2]; row[4 * g + 3] = y[s4][3];
+        }
+      }
+    }
+    __syncthreads();
+  };
+
+  gram();
+  stage_factor_input();
+  __syncthreads();
+  if (tid == 0) {
+    float tr = 0.f;
+    for (int i = 0; i < r; ++i) tr += L[i][i];
+    if (!(fabsf(tr) < __int_as_float(0x7f800000)) && os[OS_FAIL] == 0) {
+      os[OS_FAIL] = 1;
+      atomicOr(status_always, DION_STATUS_NONFINITE);
+    }
+  }
+  if (q == 0) potrf_block<true>(L, X, T, gd, rdiag, deflated, r, 0.f, os, status_fail);   // (ends with its own barrier)
+  __syncthreads();
+  const bool failed1 = reinterpret_cast<volatile int*>(os)[OS_FAIL] != 0;   // (written by this CTA's thread 0 before that barrier, or before this launch)
+  apply_inverse();
+
+  // the second round's Gram matrix, and with it the first round's distance from orthonormal
+  gram();
+  float e = 0.f;
+  if (q == 0) {
+#pragma unroll
+    for (int a = 0; a < 4; ++a)
+#pragma unroll
+      for (int b = 0; b < 4; ++b) {
+        const int i = 4 * ty + a, c = tx + 16 * b;
+        if (i < r && c < r) { const float d = acc[a][b] - ((i == c) ? 1.f : 0.f); e = fmaf(d, d, e); }
+      }
+  }
+  red[tid] = e;
+  __syncthreads();
+  for (int w = 128; w > 0; w >>= 1) {     // (quarter 0 holds the only terms)
+    if (tid < w) red[tid] += red[tid + w];
+    __syncthreads();
+  }
+  const float est = red[0];
+  const bool done = !failed1 && (est <= tau_f * tau_f * (float)r);      // false for NaN
+  if (!done && !failed1) {
+    __syncthreads();                 // everyone has read red[0]
+    stage_factor_input();
+    __syncthreads();
+    if (q == 0) potrf_block<true>(L, X, T, gd, rdiag, deflated, r, 0.f, os, status_fail);
+    __syncthreads();
+    apply_inverse();
+  }
+  if (tid == 0) {
+    os[OS_MAXDEV] = __float_as_int(est);
+    os[OS_DONE] = 1;
+    os[OS_ROUNDS] = done ? 1 : 2;
+    atomicAdd(rounds_total, done ? 1 : 2);
+  }
+#pragma unroll 4
+  for (int e2 = tid; e2 < rows * r; e2 += TINY_THREADS) {
+    const int i = e2 / r, c = e2 % r;
+    Pout[(i64)i * r + c] = Ps[i * TINY_LD + c];
   }
 }
 
