@@ -311,8 +311,8 @@ __global__ void __launch_bounds__(256) k_potrf_diag(float* __restrict__ A, i64 l
 }
 
 // CholeskyQR2 of a small panel (rows x r, r <= 64, rows <= TINY_MAX_ROWS, leading dimension r) in ONE launch, one
-// CTA of 1024 threads per matrix, the panel resident in shared memory: Gram matrix, Cholesky factor and its inverse
-// (potrf_block, on the first eight warps), U1 = P L^-T, then the second round's Gram matrix G2 = U1^T U1, which
+// CTA of 1024 threads per matrix, the panel resident in shared memory: Gram matrix (3xTF32 on the warp-level tensor
+// path), Cholesky factor and its inverse (potrf_block, on the first eight warps), U1 = P L^-T (3xTF32), then the second round's Gram matrix G2 = U1^T U1, which
 // also says exactly how far U1 is from orthonormal: |G2 - I|_F^2 <= tau_f^2 r -> done after one round (the same
 // test the probe of the large panels estimates), else the second round runs on G2.  Replaces some seventeen
 // launches of a step on such a panel.  Every sum has a fixed order: same bits on every run.
@@ -322,31 +322,40 @@ __global__ void __launch_bounds__(256) k_potrf_diag(float* __restrict__ A, i64 l
 // DION_STATUS_NONFINITE.  Pin may equal Pout.
 constexpr int TINY_MAX_ROWS = 512;
 constexpr int TINY_THREADS = 1024;
-constexpr int TINY_LD = NB + 1;
+// Row strides (floats) that keep the fragment loads of the two products off each other's banks: a lane reads
+// (row ft, column fg) of the panel for the Gram matrix (stride = 8 mod 32: no conflict) and (row fg, column ft)
+// of it (two-way) and of the inverse (copied to stride = 4 mod 32: none) for U.
+constexpr int TINY_LD = NB + 8;
+constexpr int TINY_XLD = NB + 4;
 constexpr int TINY_BLK = NB * (NB + 1);     // floats of a 64 x 65 block
-inline int tiny_cholqr2_smem(i64 rows) {    // panel, L, X, three partial Gram matrices, T, gd, rdiag, red, deflated
-  return (int)sizeof(float) * ((int)rows * TINY_LD + 5 * TINY_BLK + (NB / 2) * (NB / 2 + 1) + 2 * NB + TINY_THREADS) + (int)sizeof(int) * NB;
+inline int tiny_rows_pad(i64 rows) { return (int)((rows + 15) / 16 * 16); }
+inline int tiny_cholqr2_smem(i64 rows) {    // panel (rows padded to 16), L, X, the copy of X, T, gd, rdiag, red, deflated
+  return (int)sizeof(float) * (tiny_rows_pad(rows) * TINY_LD + 2 * TINY_BLK + NB * TINY_XLD + (NB / 2) * (NB / 2 + 1) + 2 * NB + TINY_THREADS) +
+         (int)sizeof(int) * NB;
 }
 
-// acc[a][b] = sum over this thread's quarter of the rows (i = q, q + 4, ...) of Ps[i][4 ty + a] * Ps[i][tx + 16 b]
-__device__ __forceinline__ void tiny_gram_part(const float* __restrict__ Ps, int rows, int q, int ty, int tx, float (&acc)[4][4]) {
+// The two small products of the kernel run on the warp-level tensor-core path (m16n8k8, TF32 operands, fp32
+// accumulation) as 3xTF32: x = hi + lo with hi = x truncated to TF32; lo x hi + hi x lo first, hi x hi last.
+__device__ __forceinline__ void mma_tf32_16x8x8(float (&c)[4], const uint32_t (&a)[4], const uint32_t (&b)[2]) {
+  asm volatile("mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+               : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b[0]), "r"(b[1]));
+}
+__device__ __forceinline__ void split_tf32(float x, uint32_t& hi, uint32_t& lo) {
+  hi = __float_as_uint(x) & 0xffffe000u;
+  lo = __float_as_uint(x - __uint_as_float(hi));
+}
+template <int NA, int NB_>
+__device__ __forceinline__ void mma_3xtf32(float (&c)[4], const float (&a)[NA], const float (&b)[NB_]) {
+  static_assert(NA == 4 && NB_ == 2, "m16n8k8 fragments");
+  uint32_t ah[4], al[4], bh[2], bl[2];
 #pragma unroll
-  for (int a = 0; a < 4; ++a)
+  for (int x = 0; x < 4; ++x) split_tf32(a[x], ah[x], al[x]);
 #pragma unroll
-    for (int b = 0; b < 4; ++b) acc[a][b] = 0.f;
-#pragma unroll 4
-  for (int i = q; i < rows; i += 4) {
-    const float* row = Ps + i * TINY_LD;
-    float av[4], bv[4];
-#pragma unroll
-    for (int a = 0; a < 4; ++a) av[a] = row[4 * ty + a];
-#pragma unroll
-    for (int b = 0; b < 4; ++b) bv[b] = row[tx + 16 * b];
-#pragma unroll
-    for (int a = 0; a < 4; ++a)
-#pragma unroll
-      for (int b = 0; b < 4; ++b) acc[a][b] = fmaf(av[a], bv[b], acc[a][b]);
-  }
+  for (int x = 0; x < 2; ++x) split_tf32(b[x], bh[x], bl[x]);
+  mma_tf32_16x8x8(c, al, bh);
+  mma_tf32_16x8x8(c, ah, bl);
+  mma_tf32_16x8x8(c, ah, bh);
 }
 
 __global__ void __launch_bounds__(TINY_THREADS) k_tiny_cholqr2(const float* __restrict__ Pin, float* __restrict__ Pout, int rows, int r,
@@ -357,18 +366,19 @@ __global__ void __launch_bounds__(TINY_THREADS) k_tiny_cholqr2(const float* __re
   os += (i64)blockIdx.x * OS_SLOT_INTS;
   pdl_enter();
   extern __shared__ __align__(16) float tiny_smem[];
-  float* Ps = tiny_smem;                                              // rows x 65
-  float* blocks = Ps + rows * TINY_LD;
+  const int rows_pad = (rows + 15) / 16 * 16;
+  float* Ps = tiny_smem;                                              // rows_pad x TINY_LD; rows beyond `rows` and columns beyond r are zero
+  float* blocks = Ps + rows_pad * TINY_LD;
   blk_t L = reinterpret_cast<blk_t>(blocks);
   blk_t X = reinterpret_cast<blk_t>(blocks + TINY_BLK);
-  float* Gp = blocks + 2 * TINY_BLK;                                  // partial Gram matrices of row quarters 1 .. 3
-  half_blk_t T = reinterpret_cast<half_blk_t>(blocks + 5 * TINY_BLK);
-  float* gd = blocks + 5 * TINY_BLK + (NB / 2) * (NB / 2 + 1);
+  float* XS = blocks + 2 * TINY_BLK;                                  // the inverse, row stride TINY_XLD
+  half_blk_t T = reinterpret_cast<half_blk_t>(XS + NB * TINY_XLD);
+  float* gd = XS + NB * TINY_XLD + (NB / 2) * (NB / 2 + 1);
   float* rdiag = gd + NB;
   float* red = rdiag + NB;                                            // TINY_THREADS
   int* deflated = reinterpret_cast<int*>(red + TINY_THREADS);
-  const int tid = threadIdx.x;
-  const int q = tid >> 8, t8 = tid & 255, ty = t8 >> 4, tx = t8 & 15;   // q: warp-uniform quarter of the CTA
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int fg = lane >> 2, ft = lane & 3;                            // fragment coordinates of the lane
 
   if (r % 4 == 0 && (reinterpret_cast<uintptr_t>(Pin) & 15u) == 0) {
     // four 16-byte loads in flight per thread
@@ -396,83 +406,74 @@ __global__ void __launch_bounds__(TINY_THREADS) k_tiny_cholqr2(const float* __re
 #pragma unroll 4
     for (int e = tid; e < rows * NB; e += TINY_THREADS) {
       const int i = e / NB, c = e % NB;
-      Ps[i * TINY_LD + c] = (c < r) ? Pin[(i64)i * r + c] : 0.f;      // columns r .. 63: zero
+      Ps[i * TINY_LD + c] = (c < r) ? Pin[(i64)i * r + c] : 0.f;
     }
   }
+  for (int e = rows * NB + tid; e < rows_pad * NB; e += TINY_THREADS) Ps[(e / NB) * TINY_LD + e % NB] = 0.f;
   __syncthreads();
 
-  float acc[4][4];
-  // The Gram matrix of the panel in shared memory into the registers of quarter 0: every quarter sums its rows,
-  // quarters 1 .. 3 pass theirs through shared memory, quarter 0 adds them in order.
+  // G = P^T P (64 x 64, K = rows_pad): warp w owns the 16 x 8 tile (w / 8, w % 8); lane (fg, ft) then holds
+  // G[m0 + fg][n0 + 2 ft], [..][n0 + 2 ft + 1], G[m0 + fg + 8][n0 + 2 ft], [..][n0 + 2 ft + 1].
+  const int m0 = (warp >> 3) * 16, n0 = (warp & 7) * 8;
+  float acc[4];
   auto gram = [&]() {
-    tiny_gram_part(Ps, rows, q, ty, tx, acc);
-    if (q > 0) {
-      float* g = Gp + (q - 1) * TINY_BLK;
-#pragma unroll
-      for (int a = 0; a < 4; ++a)
-#pragma unroll
-        for (int b = 0; b < 4; ++b) g[(4 * ty + a) * (NB + 1) + tx + 16 * b] = acc[a][b];
-    }
-    __syncthreads();
-    if (q == 0) {
-#pragma unroll
-      for (int p = 0; p < 3; ++p)
-#pragma unroll
-        for (int a = 0; a < 4; ++a)
-#pragma unroll
-          for (int b = 0; b < 4; ++b) acc[a][b] += Gp[p * TINY_BLK + (4 * ty + a) * (NB + 1) + tx + 16 * b];
+    acc[0] = acc[1] = acc[2] = acc[3] = 0.f;
+#pragma unroll 4
+    for (int k0 = 0; k0 < rows_pad; k0 += 8) {
+      const float* r0 = Ps + (k0 + ft) * TINY_LD;
+      const float* r1 = Ps + (k0 + ft + 4) * TINY_LD;
+      const float a[4] = {r0[m0 + fg], r0[m0 + fg + 8], r1[m0 + fg], r1[m0 + fg + 8]};    // A(m, k) = P[k][m]
+      const float b[2] = {r0[n0 + fg], r1[n0 + fg]};                                      // B(k, n) = P[k][n]
+      mma_3xtf32(acc, a, b);
     }
   };
-  // (quarter 0) the Gram matrix from the registers into L: lower triangle, zero above, identity beyond column r;
-  // X, gd, deflated reset
+  // the Gram matrix from the registers into L: lower triangle, zero above, identity beyond column r; X, gd,
+  // deflated reset
   auto stage_factor_input = [&]() {
-    if (q == 0) {
 #pragma unroll
-      for (int a = 0; a < 4; ++a)
-#pragma unroll
-        for (int b = 0; b < 4; ++b) {
-          const int i = 4 * ty + a, c = tx + 16 * b;
-          float v = (i < r && c <= i) ? acc[a][b] : 0.f;
-          if (i == c && i >= r) v = 1.f;
-          L[i][c] = v;
-          X[i][c] = 0.f;
-        }
-      if (tid < NB) { deflated[tid] = 0; gd[tid] = 0.f; }
+    for (int x = 0; x < 4; ++x) {
+      const int i = m0 + fg + ((x & 2) ? 8 : 0), c = n0 + 2 * ft + (x & 1);
+      float v = (i < r && c <= i) ? acc[x] : 0.f;
+      if (i == c && i >= r) v = 1.f;
+      L[i][c] = v;
+      X[i][c] = 0.f;
     }
+    if (tid < NB) { deflated[tid] = 0; gd[tid] = 0.f; }
   };
-  // U = P X^T in place, X lower triangular (its zeros above the diagonal are stored).  Four threads per row, one
-  // from each quarter; a thread takes the column groups g = q, q + 4, ... of four columns each, four independent
-  // sums per loaded entry.  All sums of a batch of 256 rows are formed before any entry is overwritten.
+  // U = P X^T in place (X lower triangular, its zeros above the diagonal stored): work item = 16 rows x 32
+  // columns, K = 64; the items of a sweep are all computed before any entry of the panel is overwritten.
   auto apply_inverse = [&]() {
-    const int ngroups = (r + 3) / 4;
-    for (int i0 = 0; i0 < rows; i0 += 256) {
-      const int i = i0 + t8;
-      float* row = Ps + (i < rows ? i : 0) * TINY_LD;
+    for (int e = tid; e < NB * NB; e += TINY_THREADS) XS[(e / NB) * TINY_XLD + e % NB] = X[e / NB][e % NB];
+    __syncthreads();
+    const int items = (rows_pad / 16) * 2;
+    for (int it0 = 0; it0 < items; it0 += TINY_THREADS / 32) {
+      const int it = it0 + warp;
+      const int i0 = (it >> 1) * 16, c0 = (it & 1) * 32;
       float y[4][4];
 #pragma unroll
-      for (int s4 = 0; s4 < 4; ++s4) {
-        const int g = q + 4 * s4;
-        y[s4][0] = y[s4][1] = y[s4][2] = y[s4][3] = 0.f;
-        if (g < ngroups && i < rows) {
-          const int j0 = 4 * g;
-          float y0 = 0.f, y1 = 0.f, y2 = 0.f, y3 = 0.f;
-#pragma unroll 4
-          for (int k = 0; k < j0 + 4; ++k) {
-            const float x = row[k];
-            y0 = fmaf(x, X[j0][k], y0);
-            y1 = fmaf(x, X[j0 + 1][k], y1);
-            y2 = fmaf(x, X[j0 + 2][k], y2);
-            y3 = fmaf(x, X[j0 + 3][k], y3);
+      for (int nt = 0; nt < 4; ++nt) y[nt][0] = y[nt][1] = y[nt][2] = y[nt][3] = 0.f;
+      if (it < items) {
+#pragma unroll 2
+        for (int k0 = 0; k0 < NB; k0 += 8) {
+          const float* r0 = Ps + (i0 + fg) * TINY_LD + k0;
+          const float* r1 = Ps + (i0 + fg + 8) * TINY_LD + k0;
+          const float a[4] = {r0[ft], r1[ft], r0[ft + 4], r1[ft + 4]};                    // A(m, k) = P[i0 + m][k]
+#pragma unroll
+          for (int nt = 0; nt < 4; ++nt) {
+            const float* xr = XS + (c0 + 8 * nt + fg) * TINY_XLD + k0;
+            const float b[2] = {xr[ft], xr[ft + 4]};                                      // B(k, n) = X[n][k]
+            mma_3xtf32(y[nt], a, b);
           }
-          y[s4][0] = y0; y[s4][1] = y1; y[s4][2] = y2; y[s4][3] = y3;
         }
       }
       __syncthreads();
+      if (it < items) {
 #pragma unroll
-      for (int s4 = 0; s4 < 4; ++s4) {
-        const int g = q + 4 * s4;
-        if (g < ngroups && i < rows) {
-          row[4 * g] = y[s4][0]; row[4 * g + 1] = y[s4][1]; row[4 * g + 2] = y[s4][2]; row[4 * g + 3] = y[s4][3];
+        for (int nt = 0; nt < 4; ++nt) {
+          const int c = c0 + 8 * nt + 2 * ft;
+          float* w0 = Ps + (i0 + fg) * TINY_LD + c;
+          float* w1 = Ps + (i0 + fg + 8) * TINY_LD + c;
+          w0[0] = y[nt][0]; w0[1] = y[nt][1]; w1[0] = y[nt][2]; w1[1] = y[nt][3];
         }
       }
     }
@@ -490,7 +491,7 @@ __global__ void __launch_bounds__(TINY_THREADS) k_tiny_cholqr2(const float* __re
       atomicOr(status_always, DION_STATUS_NONFINITE);
     }
   }
-  if (q == 0) potrf_block<true>(L, X, T, gd, rdiag, deflated, r, 0.f, os, status_fail);   // (ends with its own barrier)
+  if (tid < 256) potrf_block<true>(L, X, T, gd, rdiag, deflated, r, 0.f, os, status_fail);   // (ends with its own barrier)
   __syncthreads();
   const bool failed1 = reinterpret_cast<volatile int*>(os)[OS_FAIL] != 0;   // (written by this CTA's thread 0 before that barrier, or before this launch)
   apply_inverse();
@@ -498,18 +499,14 @@ __global__ void __launch_bounds__(TINY_THREADS) k_tiny_cholqr2(const float* __re
   // the second round's Gram matrix, and with it the first round's distance from orthonormal
   gram();
   float e = 0.f;
-  if (q == 0) {
 #pragma unroll
-    for (int a = 0; a < 4; ++a)
-#pragma unroll
-      for (int b = 0; b < 4; ++b) {
-        const int i = 4 * ty + a, c = tx + 16 * b;
-        if (i < r && c < r) { const float d = acc[a][b] - ((i == c) ? 1.f : 0.f); e = fmaf(d, d, e); }
-      }
+  for (int x = 0; x < 4; ++x) {
+    const int i = m0 + fg + ((x & 2) ? 8 : 0), c = n0 + 2 * ft + (x & 1);
+    if (i < r && c < r) { const float d = acc[x] - ((i == c) ? 1.f : 0.f); e = fmaf(d, d, e); }
   }
   red[tid] = e;
   __syncthreads();
-  for (int w = 128; w > 0; w >>= 1) {     // (quarter 0 holds the only terms)
+  for (int w = TINY_THREADS / 2; w > 0; w >>= 1) {
     if (tid < w) red[tid] += red[tid + w];
     __syncthreads();
   }
@@ -519,7 +516,7 @@ __global__ void __launch_bounds__(TINY_THREADS) k_tiny_cholqr2(const float* __re
     __syncthreads();                 // everyone has read red[0]
     stage_factor_input();
     __syncthreads();
-    if (q == 0) potrf_block<true>(L, X, T, gd, rdiag, deflated, r, 0.f, os, status_fail);
+    if (tid < 256) potrf_block<true>(L, X, T, gd, rdiag, deflated, r, 0.f, os, status_fail);
     __syncthreads();
     apply_inverse();
   }
