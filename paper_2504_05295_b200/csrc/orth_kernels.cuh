@@ -437,6 +437,7 @@ __global__ void __launch_bounds__(TINY_THREADS) k_tiny_cholqr2(const float* __re
       if (i == c && i >= r) v = 1.f;
       L[i][c] = v;
       X[i][c] = 0.f;
+      if (i == c) red[i] = (i < r) ? acc[x] : 0.f;      // the diagonal, for the trace
     }
     if (tid < NB) { deflated[tid] = 0; gd[tid] = 0.f; }
   };
@@ -483,10 +484,11 @@ __global__ void __launch_bounds__(TINY_THREADS) k_tiny_cholqr2(const float* __re
   gram();
   stage_factor_input();
   __syncthreads();
-  if (tid == 0) {
-    float tr = 0.f;
-    for (int i = 0; i < r; ++i) tr += L[i][i];
-    if (!(fabsf(tr) < __int_as_float(0x7f800000)) && os[OS_FAIL] == 0) {
+  if (warp == 8) {      // (a warp that has no part in the factorization: the trace from the staged diagonal, fixed order)
+    float tr = red[lane] + red[lane + 32];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) tr += __shfl_xor_sync(0xffffffffu, tr, o);
+    if (lane == 0 && !(fabsf(tr) < __int_as_float(0x7f800000)) && os[OS_FAIL] == 0) {
       os[OS_FAIL] = 1;
       atomicOr(status_always, DION_STATUS_NONFINITE);
     }
