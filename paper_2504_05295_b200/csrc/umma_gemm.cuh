@@ -539,11 +539,13 @@ struct TileMap {
 // no "lo" halves, no conversion pass, the producer warps join the epilogue as in the bf16-array variant.
 // Used for the rank-r update of X, whose result feeds nothing else: an unbiased 2^-12 relative operand
 // error there moves X by ~1e-6.
-// CG2 (fp32 mode, TMA, BN = 256): two CTAs of a cluster form one 256 x 256 tile with cta_group::2 MMAs.
+// CG2 (TMA, BN = 256): two CTAs of a cluster form one 256 x 256 tile with cta_group::2 MMAs.
 // Each CTA loads and converts its own 128 rows of A and HALF of the B tile (128 of the 256 columns), so a
 // K block costs a CTA two thirds of the shared-memory traffic of the single-CTA form (which is bound by
 // it: three MMAs re-read both operand tiles) and a stage is 64 KB instead of 96 KB (3 stages instead of 2).
 // The leader CTA issues the MMAs for both; accumulators and epilogue stay per CTA (128 rows x 256 columns).
+// The variants on 16-bit arrays (D16: nothing to convert) form pairs too: both CTAs' TMA loads then complete on the
+// leader's barrier (cta_group::2 load form), which the leader's MMA thread waits on.
 // X2 (bf16 arrays, D16): each operand is a PAIR of bf16 arrays, x ~ hi + lo with hi = bf16(x), lo = bf16(x - hi)
 // (16 significant bits); three bf16 MMAs per K step (hi*lo + lo*hi + hi*hi) give a product that is accurate to
 // ~1e-5 relative at 1.3 times the tensor time of one TF32 pass.  Used for the error-feedback product in fp32
@@ -656,7 +658,7 @@ k_gemm_umma(const __grid_constant__ Params p) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), NOCONV ? 1 : NUM_PROD_WARPS * (CG2 ? 2 : 1)); mbar_init(empty_bar(s), 1); }
     for (int b = 0; b < 2; ++b) { mbar_init(accf_bar(b), 1); mbar_init(acce_bar(b), C::EPI_WARPS * (CG2 ? 2 : 1)); }   // one arrival per epilogue warp
     mbar_init(drain_bar, 1);
-    // (pair without converters: the leader's "landed" barrier also takes the peer's word that ITS tiles have landed)
+    // (pair without converters: the leader's "landed" barrier counts the bytes of both CTAs' tiles, see the TMA issuer)
     if (TMA) for (int s = 0; s < STAGES; ++s) mbar_init(raw_bar(s), 1);
     *dead = 0;
     fence_barrier_init();
