@@ -942,6 +942,7 @@ __global__ void __launch_bounds__(128) k_probe_w(const float* __restrict__ U, i6
   float acc[NPROBE];
 #pragma unroll
   for (int p = 0; p < NPROBE; ++p) acc[p] = 0.f;
+#pragma unroll 8      // (eight rows' loads in flight per thread; the sums keep their order)
   for (i64 i = i0; i < i1; ++i) {
     const float u = U[i * ld + j];
     const float4 y0 = *reinterpret_cast<const float4*>(Y + i * NPROBE);
@@ -976,6 +977,7 @@ __global__ void __launch_bounds__(1024) k_probe_decide(const float* __restrict__
   // one (column, probe) entry per thread at a time: consecutive threads read consecutive words of a chunk's partials
   for (i64 x = threadIdx.x; x < r * NPROBE; x += blockDim.x) {
     float w = 0.f;
+#pragma unroll 8      // (eight chunks' loads in flight; the sum keeps its order)
     for (int c = 0; c < chunks; ++c) w += part[(i64)c * r * NPROBE + x];
     const float dlt = w - probe_sign(x / NPROBE, (int)(x % NPROBE));
     e = fmaf(dlt, dlt, e);
