@@ -83,8 +83,9 @@ typedef enum { DION_PREC_FP32 = 0, DION_PREC_BF16_OPERANDS = 1 } dion_precision;
  *                        of its norm) still cancels the step (DION_STATUS_BREAKDOWN).
  *                        Before the second round the first round's result U1 is measured on the
  *                        device (a randomized estimate of |U1^T U1 - I|_F from two passes over the
- *                        panel); if it is orthonormal to 3e-5 per column the second round is
- *                        skipped (well-conditioned panels).
+ *                        panel; the exact value for a panel of at most 512 rows and 64 columns, whose
+ *                        whole orthonormalization is one launch); if it is orthonormal to 3e-5 per
+ *                        column the second round is skipped (well-conditioned panels).
  * DION_ORTH_SHIFTED3:    adaptive Cholesky QR rounds for ill-conditioned panels such as
  *                        full rank: a column whose pivot falls below 1e-4 of its
  *                        squared norm is deflated, so a round cannot break down and
