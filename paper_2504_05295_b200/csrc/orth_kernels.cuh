@@ -872,7 +872,7 @@ constexpr int PY_COLS = 2048;
 constexpr int PY_SMEM = PY_COLS * NPROBE * 4;
 __global__ void __launch_bounds__(256) k_probe_y4(const float* __restrict__ U, i64 ld, i64 rows, i64 r,
                                                   float* __restrict__ Y, i64 wstride, const int* __restrict__ keep) {
-  extern __shared__ float py_sign[];      // [column in block][probe]
+  extern __shared__ __align__(16) float py_sign[];      // the signs of the block's columns (layout below)
   pdl_enter();
   if (keep != nullptr && keep[(i64)blockIdx.y * OS_SLOT_INTS] != 0) return;   // this panel's decision stands
   U += (i64)blockIdx.y * wstride; Y += (i64)blockIdx.y * wstride;
@@ -881,7 +881,13 @@ __global__ void __launch_bounds__(256) k_probe_y4(const float* __restrict__ U, i
   for (i64 c0 = 0; c0 < r; c0 += PY_COLS) {
     const int nc = (int)min((i64)PY_COLS, r - c0);
     __syncthreads();
-    for (int e = threadIdx.x; e < nc * NPROBE; e += 256) py_sign[e] = probe_sign(c0 + e / NPROBE, e % NPROBE);
+    // table layout: the four signs (probes 4 h .. 4 h + 3) of column 128 t + 4 l + cc sit in the 16-byte unit
+    // ((4 t + cc) 2 + h) 32 + l, so that the 32 lanes of a warp read 32 consecutive units (column-major by 8 floats
+    // put a quarter warp's reads on the same banks: eight-way conflicts on every read)
+    for (int e = threadIdx.x; e < nc * NPROBE; e += 256) {
+      const int col = e / NPROBE, pr = e % NPROBE;
+      py_sign[((((col >> 7) * 4 + (col & 3)) * 2 + (pr >> 2)) * 32 + ((col & 127) >> 2)) * 4 + (pr & 3)] = probe_sign(c0 + col, pr);
+    }
     __syncthreads();
     for (i64 g = group0; g * 4 < rows; g += groups) {
       const i64 i0 = g * 4;
@@ -897,8 +903,9 @@ __global__ void __launch_bounds__(256) k_probe_y4(const float* __restrict__ U, i
           u[q] = (i0 + q < rows) ? *reinterpret_cast<const float4*>(U + (i0 + q) * ld + c0 + j) : make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
         for (int cc = 0; cc < 4; ++cc) {
-          const float4 s0 = *reinterpret_cast<const float4*>(py_sign + (j + cc) * NPROBE);
-          const float4 s1 = *reinterpret_cast<const float4*>(py_sign + (j + cc) * NPROBE + 4);
+          const float4* su = reinterpret_cast<const float4*>(py_sign) + (((j >> 7) * 4 + cc) * 2) * 32 + lane;
+          const float4 s0 = su[0];
+          const float4 s1 = su[32];
 #pragma unroll
           for (int q = 0; q < 4; ++q) {
             const float v = (cc == 0) ? u[q].x : (cc == 1) ? u[q].y : (cc == 2) ? u[q].z : u[q].w;
