@@ -677,8 +677,12 @@ int probe(StepCtx& s, i64 off, i64 rows, i64 r, int phase) {
                rows, r, s.ws + s.L.probe_y, s.wstride, keep);
   }
   DION_CHECK_LAUNCH(c);
-  launch_pdl(k_probe_w, dim3((unsigned)((r + 127) / 128), (unsigned)chunks, (unsigned)s.nb), dim3(128), 0, s.st,
-             (const float*)(s.ws + off), r, rows, r, per, (const float*)(s.ws + s.L.probe_y), s.ws + s.L.probe_part, s.wstride, keep);
+  if (r % 4 == 0)
+    launch_pdl(k_probe_w4, dim3((unsigned)((r / 4 + 127) / 128), (unsigned)chunks, (unsigned)s.nb), dim3(128), 0, s.st,
+               (const float*)(s.ws + off), r, rows, r, per, (const float*)(s.ws + s.L.probe_y), s.ws + s.L.probe_part, s.wstride, keep);
+  else
+    launch_pdl(k_probe_w, dim3((unsigned)((r + 127) / 128), (unsigned)chunks, (unsigned)s.nb), dim3(128), 0, s.st,
+               (const float*)(s.ws + off), r, rows, r, per, (const float*)(s.ws + s.L.probe_y), s.ws + s.L.probe_part, s.wstride, keep);
   DION_CHECK_LAUNCH(c);
   launch_pdl(k_probe_decide, dim3((unsigned)s.nb), dim3(r >= 128 ? 1024 : 256), 0, s.st, (const float*)(s.ws + s.L.probe_part), chunks, r, s.os,
              ORTH_TAU_F, c->dev_ints + 2, s.wstride, phase);

@@ -962,6 +962,46 @@ __global__ void __launch_bounds__(128) k_probe_w(const float* __restrict__ U, i6
   for (int p = 0; p < NPROBE; ++p) out[p] = acc[p];
 }
 
+// The same for r a multiple of 4: a thread takes four neighbouring columns (one 16-byte load per row, four rows'
+// loads in flight); every column's sum runs over the chunk's rows in the same order as above.
+// grid = (ceil(r/512), chunks, matrices).
+__global__ void __launch_bounds__(128) k_probe_w4(const float* __restrict__ U, i64 ld, i64 rows, i64 r,
+                                                  i64 rows_per_chunk, const float* __restrict__ Y,
+                                                  float* __restrict__ part, i64 wstride, const int* __restrict__ keep) {
+  pdl_enter();
+  if (keep != nullptr && keep[(i64)blockIdx.z * OS_SLOT_INTS] != 0) return;
+  U += (i64)blockIdx.z * wstride; Y += (i64)blockIdx.z * wstride; part += (i64)blockIdx.z * wstride;
+  const i64 j = ((i64)blockIdx.x * 128 + threadIdx.x) * 4;
+  if (j >= r) return;
+  const i64 i0 = (i64)blockIdx.y * rows_per_chunk;
+  const i64 i1 = min(rows, i0 + rows_per_chunk);
+  float acc[4][NPROBE];
+#pragma unroll
+  for (int c = 0; c < 4; ++c)
+#pragma unroll
+    for (int p = 0; p < NPROBE; ++p) acc[c][p] = 0.f;
+#pragma unroll 4
+  for (i64 i = i0; i < i1; ++i) {
+    const float4 u4 = *reinterpret_cast<const float4*>(U + i * ld + j);
+    const float4 y0 = *reinterpret_cast<const float4*>(Y + i * NPROBE);
+    const float4 y1 = *reinterpret_cast<const float4*>(Y + i * NPROBE + 4);
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+      const float u = (c == 0) ? u4.x : (c == 1) ? u4.y : (c == 2) ? u4.z : u4.w;
+      acc[c][0] = fmaf(u, y0.x, acc[c][0]); acc[c][1] = fmaf(u, y0.y, acc[c][1]);
+      acc[c][2] = fmaf(u, y0.z, acc[c][2]); acc[c][3] = fmaf(u, y0.w, acc[c][3]);
+      acc[c][4] = fmaf(u, y1.x, acc[c][4]); acc[c][5] = fmaf(u, y1.y, acc[c][5]);
+      acc[c][6] = fmaf(u, y1.z, acc[c][6]); acc[c][7] = fmaf(u, y1.w, acc[c][7]);
+    }
+  }
+  float4* out = reinterpret_cast<float4*>(part + ((i64)blockIdx.y * r + j) * NPROBE);
+#pragma unroll
+  for (int c = 0; c < 4; ++c) {
+    out[2 * c] = make_float4(acc[c][0], acc[c][1], acc[c][2], acc[c][3]);
+    out[2 * c + 1] = make_float4(acc[c][4], acc[c][5], acc[c][6], acc[c][7]);
+  }
+}
+
 // One block per matrix: est = sum_p |w_p - z_p|^2 / NPROBE (fixed summation order) into os[OS_MAXDEV] (float
 // bits); est <= tau_f^2 * r  ->  the panel is done (OS_DONE = 1: the rest of the second round is skipped).
 // Counts the rounds of the step that did work (1 or 2; with a recomputed panel 2 or 3).
