@@ -509,6 +509,21 @@ def run_workload(wid, cases, grouped, args, ctx):
     clocks = sampler.stop()
     ms_total = e_start.elapsed_time(e_end)
     launches = opt.launch_count() - launches0
+    if clocks.get("samples", 0) == 0 and not dp_sync:
+        # a timed region shorter than nvidia-smi's first sample (config 1: ~20 ms): the same steps once more,
+        # untimed, for about a second under a fresh sampler, so that the record still says what clocks this load sees
+        sampler = ClockSampler(local)
+        sampler.start()
+        t_end = time.time() + 1.0
+        t_extra = 0
+        while time.time() < t_end:
+            one_step(args.warmup + args.steps + t_extra)
+            t_extra += 1
+            if t_extra % 8 == 0:
+                torch.cuda.synchronize()
+        torch.cuda.synchronize()
+        clocks = sampler.stop()
+        clocks["note"] = "timed region shorter than one sampling interval: sampled over the same steps repeated untimed right after it"
     status2, skipped2 = opt.get_status()
     ms_step = max_over_ranks(ms_total / args.steps, dev)
     case_ms = [sum(a.elapsed_time(b) for a, b in ev) / len(ev) if ev else None for ev in case_events]
