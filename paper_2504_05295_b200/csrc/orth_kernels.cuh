@@ -1022,6 +1022,7 @@ __global__ void __launch_bounds__(1024) k_probe_decide(const float* __restrict__
   __shared__ float red[1024];
   float e = 0.f;
   // one (column, probe) entry per thread at a time: consecutive threads read consecutive words of a chunk's partials
+#pragma unroll 4       // (four entries' chunk sums advance together: their loads are independent)
   for (i64 x = threadIdx.x; x < r * NPROBE; x += blockDim.x) {
     float w = 0.f;
 #pragma unroll 8      // (eight chunks' loads in flight; the sum keeps its order)
